@@ -1,0 +1,158 @@
+/*
+ * glide.h -- C ABI of the B200 (sm_100a) GLIDE hybrid-attention library.
+ *
+ * The operation (paper Sec. III-B "GLIDE Attention", Eq. 7 with its two component
+ * equations; Sec. II "Linearized Attention"; appendix Eq. 1-6): every layer l keeps a
+ * ring buffer of its newest w_l keys/values and runs exact softmax attention over it;
+ * a token that slides out of the window is folded into a recurrent linear-attention
+ * state  S += phi(k) v^T,  z += phi(k)  (phi = softmax over the head features, fp32);
+ * the output merges both parts under ONE normaliser:
+ *
+ *   O_t = (sum_W exp(scale q.k_j) v_j + phi(q)^T S) / (sum_W exp(scale q.k_j) + phi(q)^T z)
+ *
+ * with W = the newest w_l tokens including the current one and S,z holding every
+ * older token.  w_l >= context gives causal softmax attention, w_l = 0 pure linear
+ * attention.  Prefill over T tokens leaves the same state and outputs as T decode steps.
+ *
+ * Conventions for every call
+ *   - All pointers named dev_* or documented "device" are device pointers on the
+ *     CUDA device that was current at glide_create; "host" pointers are ordinary
+ *     host memory.  Device buffers must be contiguous and 16-byte aligned.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).  Calls
+ *     are asynchronous and stream-ordered; the library never synchronises the host on
+ *     the hot path and never allocates device memory: the caller owns the workspace
+ *     and every q/k/v/out buffer.  The library owns only the small host-side context.
+ *   - Every call returns a glide_status code (0 = success).  Arguments are validated
+ *     before anything is launched; a failing call changes no state.  Device code never
+ *     traps: internal range checks record a code in a status word (glide_device_status).
+ *   - Not thread-safe per context; different contexts are independent.
+ */
+#ifndef GLIDE_H_
+#define GLIDE_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct glide_ctx glide_ctx; /* opaque, host side */
+
+typedef enum {
+  GLIDE_OK = 0,
+  GLIDE_ERR_INVALID_ARG = 1,         /* NULL / misaligned pointer, negative size, bad layer range */
+  GLIDE_ERR_UNSUPPORTED = 2,         /* head_dim not in {64,128}, unequal GQA groups, group size not in {1,2,4,8} */
+  GLIDE_ERR_WORKSPACE_TOO_SMALL = 3,
+  GLIDE_ERR_CAPACITY = 4,            /* tokens absorbed + T would exceed max_tokens */
+  GLIDE_ERR_STATE = 5,               /* decode with layers at different positions */
+  GLIDE_ERR_CUDA = 6                 /* a CUDA runtime call or launch failed */
+} glide_status;
+
+typedef enum { GLIDE_F32 = 0, GLIDE_BF16 = 1 } glide_dtype;
+
+/* Feature map of the linear part.  GLIDE_PHI_SOFTMAX is the paper's default
+ * (Sec. III-B): phi(x) = softmax over the head_dim entries of x, no parameters,
+ * feature dimension = head_dim. */
+typedef enum { GLIDE_PHI_SOFTMAX = 0 } glide_phi;
+
+/* How the window part and the linear part are merged (Sec. III-B "(+)"; appendix
+ * "Retention-based SWA").  GLIDE_MERGE_SHARED is the shared normaliser above. */
+typedef enum { GLIDE_MERGE_SHARED = 0 } glide_merge;
+
+typedef struct {
+  int32_t n_layers;        /* L >= 1 */
+  int32_t batch;           /* B >= 1 independent sequences of equal length */
+  int32_t n_q_heads;       /* H */
+  int32_t n_kv_heads;      /* H_kv, H % H_kv == 0 */
+  int32_t head_dim;        /* d in {64, 128} */
+  int32_t io_dtype;        /* glide_dtype of q, k, v, out and of the ring; S and z are always fp32 */
+  int32_t phi;             /* glide_phi */
+  int32_t merge;           /* glide_merge */
+  const int64_t *windows;  /* host [n_layers]: w_l >= 0 (the layer-wise allocation w - delta_l, Sec. III-B).
+                              w_l >= max_tokens never evicts: that layer is full softmax attention. Copied. */
+  const int32_t *q_to_kv;  /* host [n_q_heads] KV head of each query head, or NULL for contiguous groups
+                              h / (H/H_kv) (the Llama/Mistral GQA convention). Groups must be equal-sized. Copied. */
+  int64_t max_tokens;      /* per-sequence capacity, prompt + generated tokens */
+  float softmax_scale;     /* scale of the window logits; 0 selects 1/sqrt(head_dim) (appendix Eq. 1) */
+  int32_t prefill_chunk;   /* tokens per chunk of the chunked linear scan; 0 selects 256; multiple of 16, <= 1024 */
+  int32_t decode_chunk;    /* window slots per split-K work item of the decode kernel; 0 selects automatically */
+  int32_t decode_state_splits; /* row blocks the S update/readout of one KV head is split into; 0 selects automatically */
+} glide_config;
+
+typedef struct {
+  int64_t window;     /* w_l as configured */
+  int64_t capacity;   /* ring slots allocated: min(w_l, max_tokens) */
+  int64_t n;          /* tokens absorbed so far (device counter) */
+  int64_t count;      /* valid ring entries: min(n, w_l) */
+  int64_t head_slot;  /* slot the next token will be written to: n mod capacity (0 if capacity == 0) */
+  int64_t n_evicted;  /* tokens folded into S,z so far: max(0, n - w_l) */
+} glide_layer_info_t;
+
+/* Bytes of device workspace glide_create needs for this configuration (rings, S, z,
+ * split-K scratch, work lists, chunk-scan scratch).  Host only, no CUDA calls. */
+int glide_workspace_bytes(const glide_config *cfg, size_t *bytes_out);
+
+/* Build a context over caller-owned device memory `dev_workspace` (>= glide_workspace_bytes,
+ * 256-byte aligned).  Sets the GQA head mapping and the per-layer windows, uploads the static
+ * work lists and zeroes rings' bookkeeping, S and z on `stream`.  The workspace must stay
+ * alive and untouched by the caller until glide_destroy. */
+int glide_create(const glide_config *cfg, void *dev_workspace, size_t workspace_bytes, void *stream,
+                 glide_ctx **ctx_out);
+
+/* Prefill stage (Sec. II "KV Cache"; appendix "KV Cache"): append T prompt tokens to layers
+ * [layer_begin, layer_begin + layer_count).  May be called repeatedly (chunked prefill); layers
+ * may be prefilled in separate calls.
+ *   dev_q   [layer_count][B][T][H][d]      (ignored when dev_out is NULL)
+ *   dev_k,v [layer_count][B][T][H_kv][d]
+ *   dev_out [layer_count][B][T][H][d] or NULL to build the state only.
+ * Output i of the call attends to the newest w_l tokens up to and including itself (from the ring
+ * and from this call) and, through S,z, to everything older.  Afterwards ring, S, z and counters
+ * are exactly as T decode steps would leave them. */
+int glide_prefill(glide_ctx *ctx, int32_t layer_begin, int32_t layer_count, int64_t T, const void *dev_q,
+                  const void *dev_k, const void *dev_v, void *dev_out, void *stream);
+
+/* Decode stage: one token for every layer and sequence, one fused launch.
+ *   dev_q, dev_out [L][B][H][d];  dev_k, dev_v [L][B][H_kv][d].
+ * Per layer: the token leaving the window (if any) is folded into S,z in place, the window is
+ * streamed once for all query heads of a KV head, the linear readout uses the updated state, and
+ * the merged output is written; then k,v are stored at slot n mod capacity and n advances.
+ * All layers must be at the same position (GLIDE_ERR_STATE otherwise). */
+int glide_decode_step(glide_ctx *ctx, const void *dev_q, const void *dev_k, const void *dev_v, void *dev_out,
+                      void *stream);
+
+/* Free the host context.  Does not touch the workspace. */
+int glide_destroy(glide_ctx *ctx);
+
+/* ---- test / benchmark support -------------------------------------------------------------- */
+
+/* Bookkeeping of one layer, read back from the device counters (synchronises `stream`). */
+int glide_layer_info(glide_ctx *ctx, int32_t layer, void *stream, glide_layer_info_t *out);
+
+/* Copy one layer's state to caller DEVICE buffers (any may be NULL):
+ *   dev_ringK, dev_ringV [B][H_kv][capacity][d] in the I/O dtype (slot order);
+ *   dev_S [B][H_kv][d][d] fp32 with S[r][c] = sum phi(k)_r v_c;  dev_z [B][H_kv][d] fp32. */
+int glide_export_state(glide_ctx *ctx, int32_t layer, void *dev_ringK, void *dev_ringV, float *dev_S,
+                       float *dev_z, void *stream);
+
+/* Overwrite one layer's state from caller DEVICE buffers (same layouts; NULL leaves that part
+ * as it is) and set its position to n (0 <= n <= max_tokens). */
+int glide_import_state(glide_ctx *ctx, int32_t layer, int64_t n, const void *dev_ringK, const void *dev_ringV,
+                       const float *dev_S, const float *dev_z, void *stream);
+
+/* Back to the empty state: counters, S and z zeroed (rings need no clearing). */
+int glide_reset(glide_ctx *ctx, void *stream);
+
+/* Status word written by device-side range checks (0 = none tripped).  Synchronises `stream`. */
+int glide_device_status(glide_ctx *ctx, void *stream, int32_t *status_out);
+
+/* Kernels one glide_decode_step launches and work items it processes (for launch accounting). */
+int glide_decode_launch_info(glide_ctx *ctx, int32_t *n_launches, int32_t *n_work_items, int32_t *grid_size);
+
+/* Static, NUL-terminated description of a status code. */
+const char *glide_strerror(int code);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* GLIDE_H_ */

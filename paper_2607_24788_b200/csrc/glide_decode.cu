@@ -1,0 +1,417 @@
+// Fused GLIDE decode step: ONE persistent launch over all layers.
+//
+// CTAs pull work items from a static, longest-first list through an atomic counter:
+//   window item  -- a run of ring slots of one (layer, sequence, KV head) unit: streams K/V rows
+//                   once for all G query heads of the KV head, online softmax, writes a split-K
+//                   partial (m, l, acc) to scratch;
+//   state item   -- a block of rows of the unit's recurrent state: folds the token that leaves the
+//                   window (S += phi(k) v^T, z += phi(k), in place, fp32) and reads the updated
+//                   rows out against phi(q) of the G heads, writes a linear partial (a, b).
+// Each finished item takes a ticket on its unit; the CTA that takes the last ticket merges the
+// partials in fixed order with the current token's own term under the shared normaliser, writes
+// the output, stores k,v in the ring slot and clears the ticket.  Nothing ever spins.
+// The last CTA to leave the kernel resets the work counter and advances the position counters,
+// so the step needs no host-side state and no second launch.
+#include "glide_device.cuh"
+
+namespace glide {
+
+namespace {
+
+template <int D, int G>
+constexpr int scratch_floats() {
+  // window items: [warps][G][D+2]; state items: [row groups][G][D]
+  constexpr int NW = kDecodeThreads / 32;
+  constexpr int RPI = kDecodeThreads / (D / 4);
+  return (NW * G * (D + 2) > RPI * G * D) ? NW * G * (D + 2) : RPI * G * D;
+}
+
+template <typename T, int D, int G>
+struct DecodeSmem {
+  float scratch[scratch_floats<D, G>()];
+  float phiq[G][D];
+  float phik[D];
+  float ve[D];
+  float scur[G];
+  float M[G];
+  float inv[G];
+  int item;
+  int last;
+};
+
+// ---- window item ---------------------------------------------------------------------------
+template <typename T, int D, int G>
+__device__ __forceinline__ void window_item(const DecodeParams &p, const WorkItem &it, const LayerDev &ld,
+                                            int64_t t, int b, int g, float *rec, DecodeSmem<T, D, G> &sm) {
+  constexpr int E = D / 32;
+  constexpr int NW = kDecodeThreads / 32;
+  constexpr int U = 4;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const size_t unit_rows = (size_t(b) * p.Hkv + g) * size_t(ld.cap);
+  const T *Kb = reinterpret_cast<const T *>(p.ws + ld.ringK) + unit_rows * D;
+  const T *Vb = reinterpret_cast<const T *>(p.ws + ld.ringV) + unit_rows * D;
+
+  float qr[G][E];
+#pragma unroll
+  for (int h = 0; h < G; ++h) {
+    const int head = p.heads_of[g * G + h];
+    const T *qp = reinterpret_cast<const T *>(p.q) + ((size_t(it.layer) * p.B + b) * p.H + head) * D + lane * E;
+    load_elems<T, E>(qp, qr[h]);
+#pragma unroll
+    for (int i = 0; i < E; ++i) qr[h][i] *= p.scale_log2;
+  }
+  float acc[G][E], m[G], l[G];
+#pragma unroll
+  for (int h = 0; h < G; ++h) {
+    m[h] = -CUDART_INF_F;
+    l[h] = 0.f;
+#pragma unroll
+    for (int i = 0; i < E; ++i) acc[h][i] = 0.f;
+  }
+  // Valid rows: the window's tokens other than the current one.  While the ring is not full they
+  // are slots [0, t); afterwards every slot but t mod cap, which holds the token leaving the window.
+  const int64_t lim = t < ld.cap ? t : ld.cap;
+  const int64_t cur = t % ld.cap;
+  const int end = it.begin + it.count;
+  for (int s0 = it.begin + warp; s0 < end; s0 += NW * U) {
+    float kx[U][E], vx[U][E];
+    bool ok[U];
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+      const int s = s0 + u * NW;
+      ok[u] = s < end && s < lim && s != cur;
+      if (ok[u]) {
+        load_elems<T, E>(Kb + size_t(s) * D + lane * E, kx[u]);
+        load_elems<T, E>(Vb + size_t(s) * D + lane * E, vx[u]);
+      }
+    }
+#pragma unroll
+    for (int u = 0; u < U; ++u)
+      if (ok[u]) online_row<E, G>(qr, kx[u], vx[u], m, l, acc);
+  }
+  // combine the warps
+  float *red = sm.scratch;  // [NW][G][D+2]
+#pragma unroll
+  for (int h = 0; h < G; ++h) {
+    float *r = red + (size_t(warp) * G + h) * (D + 2);
+#pragma unroll
+    for (int i = 0; i < E; ++i) r[lane * E + i] = acc[h][i];
+    if (lane == 0) {
+      r[D] = m[h];
+      r[D + 1] = l[h];
+    }
+  }
+  __syncthreads();
+  for (int idx = tid; idx < G * D; idx += kDecodeThreads) {
+    const int h = idx / D, c = idx - h * D;
+    float M = -CUDART_INF_F;
+#pragma unroll
+    for (int w = 0; w < NW; ++w) M = fmaxf(M, red[(size_t(w) * G + h) * (D + 2) + D]);
+    float val = 0.f, lsum = 0.f;
+#pragma unroll
+    for (int w = 0; w < NW; ++w) {
+      const float *r = red + (size_t(w) * G + h) * (D + 2);
+      const float f = r[D] == -CUDART_INF_F ? 0.f : exp2f(r[D] - M);
+      val = fmaf(r[c], f, val);
+      lsum = fmaf(r[D + 1], f, lsum);
+    }
+    rec[idx] = val;
+    if (c == 0) {
+      rec[G * D + h] = M;
+      rec[G * D + G + h] = lsum;
+    }
+  }
+}
+
+// ---- state item ----------------------------------------------------------------------------
+template <typename T, int D, int G>
+__device__ __forceinline__ void state_item(const DecodeParams &p, const WorkItem &it, const LayerDev &ld, int64_t t,
+                                           int b, int g, float *rec, DecodeSmem<T, D, G> &sm) {
+  constexpr int E = D / 32;
+  constexpr int NW = kDecodeThreads / 32;
+  constexpr int TPR = D / 4;                   // threads per state row (float4 each)
+  constexpr int RPI = kDecodeThreads / TPR;    // rows per iteration
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  if (!(ld.w == 0 || t >= ld.w)) return;       // nothing leaves the window yet: S,z are still zero
+  const int ub = b * p.Hkv + g;
+  const T *ke, *ve;
+  if (ld.w == 0) {  // no ring: the current token goes straight to the state
+    ke = reinterpret_cast<const T *>(p.k) + size_t(it.unit) * D;
+    ve = reinterpret_cast<const T *>(p.v) + size_t(it.unit) * D;
+  } else {          // slot t mod cap holds token t - w
+    const size_t row = (size_t(ub) * size_t(ld.cap) + size_t(t % ld.cap)) * D;
+    ke = reinterpret_cast<const T *>(p.ws + ld.ringK) + row;
+    ve = reinterpret_cast<const T *>(p.ws + ld.ringV) + row;
+  }
+  if (warp == 0) {
+    float x[E], y[E];
+    load_elems<T, E>(ke + lane * E, x);
+    load_elems<T, E>(ve + lane * E, y);
+    warp_phi<E>(x);
+#pragma unroll
+    for (int i = 0; i < E; ++i) {
+      sm.phik[lane * E + i] = x[i];
+      sm.ve[lane * E + i] = y[i];
+    }
+  }
+  for (int h = warp; h < G; h += NW) {
+    const int head = p.heads_of[g * G + h];
+    float x[E];
+    load_elems<T, E>(reinterpret_cast<const T *>(p.q) + ((size_t(it.layer) * p.B + b) * p.H + head) * D + lane * E, x);
+    warp_phi<E>(x);
+#pragma unroll
+    for (int i = 0; i < E; ++i) sm.phiq[h][lane * E + i] = x[i];
+  }
+  __syncthreads();
+
+  const int c4 = tid % TPR, rsub = tid / TPR;
+  const int r_end = it.begin + it.count;
+  float *Sb = reinterpret_cast<float *>(p.ws + ld.S) + size_t(ub) * D * D;
+  const float4 v4 = *reinterpret_cast<const float4 *>(&sm.ve[c4 * 4]);
+  float4 a[G];
+#pragma unroll
+  for (int h = 0; h < G; ++h) a[h] = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll 4
+  for (int r = it.begin + rsub; r < r_end; r += RPI) {
+    float4 *sp = reinterpret_cast<float4 *>(Sb + size_t(r) * D + c4 * 4);
+    float4 s = *sp;
+    const float pk = sm.phik[r];
+    s.x = fmaf(pk, v4.x, s.x);
+    s.y = fmaf(pk, v4.y, s.y);
+    s.z = fmaf(pk, v4.z, s.z);
+    s.w = fmaf(pk, v4.w, s.w);
+    *sp = s;
+#pragma unroll
+    for (int h = 0; h < G; ++h) {
+      const float f = sm.phiq[h][r];
+      a[h].x = fmaf(f, s.x, a[h].x);
+      a[h].y = fmaf(f, s.y, a[h].y);
+      a[h].z = fmaf(f, s.z, a[h].z);
+      a[h].w = fmaf(f, s.w, a[h].w);
+    }
+  }
+  // z rows of this block and the b_h readout: warp 0
+  if (warp == 0) {
+    float *zb = reinterpret_cast<float *>(p.ws + ld.z) + size_t(ub) * D;
+    float bp[G];
+#pragma unroll
+    for (int h = 0; h < G; ++h) bp[h] = 0.f;
+    for (int r = it.begin + lane; r < r_end; r += 32) {
+      const float zn = zb[r] + sm.phik[r];
+      zb[r] = zn;
+#pragma unroll
+      for (int h = 0; h < G; ++h) bp[h] = fmaf(sm.phiq[h][r], zn, bp[h]);
+    }
+#pragma unroll
+    for (int h = 0; h < G; ++h) {
+      const float bs = warp_sum(bp[h]);
+      if (lane == 0) {
+        rec[G * D + h] = bs;
+        rec[G * D + G + h] = 0.f;
+      }
+    }
+  }
+  float *red = sm.scratch;  // [RPI][G][D]
+#pragma unroll
+  for (int h = 0; h < G; ++h) *reinterpret_cast<float4 *>(red + (size_t(rsub) * G + h) * D + c4 * 4) = a[h];
+  __syncthreads();
+  for (int idx = tid; idx < G * D; idx += kDecodeThreads) {
+    float val = 0.f;
+#pragma unroll
+    for (int rs = 0; rs < RPI; ++rs) val += red[size_t(rs) * G * D + idx];
+    rec[idx] = val;
+  }
+}
+
+// ---- merge (last ticket of a unit) -----------------------------------------------------------
+template <typename T, int D, int G>
+__device__ __forceinline__ void merge_unit(const DecodeParams &p, const WorkItem &it, const LayerDev &ld, int64_t t,
+                                           int b, int g, DecodeSmem<T, D, G> &sm) {
+  constexpr int E = D / 32;
+  constexpr int NW = kDecodeThreads / 32;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int ub = b * p.Hkv + g;
+  const int per_unit = ld.n_win_items + ld.n_state_items;
+  const float *rec0 = p.partials + ld.part_base + size_t(ub) * per_unit * p.rec_floats;
+  const bool has_win = ld.cap > 0;
+  const bool has_state = ld.n_state_items > 0 && (ld.w == 0 || t >= ld.w);
+  const T *kt = reinterpret_cast<const T *>(p.k) + size_t(it.unit) * D;
+  const T *vt = reinterpret_cast<const T *>(p.v) + size_t(it.unit) * D;
+
+  if (has_win) {  // the current token's own logit, per head
+    float kx[E];
+    load_elems<T, E>(kt + lane * E, kx);
+    for (int h = warp; h < G; h += NW) {
+      const int head = p.heads_of[g * G + h];
+      float qx[E];
+      load_elems<T, E>(reinterpret_cast<const T *>(p.q) + ((size_t(it.layer) * p.B + b) * p.H + head) * D + lane * E, qx);
+      float part = 0.f;
+#pragma unroll
+      for (int i = 0; i < E; ++i) part = fmaf(qx[i] * p.scale_log2, kx[i], part);
+      part = warp_sum(part);
+      if (lane == 0) sm.scur[h] = part;
+    }
+  }
+  __syncthreads();
+  if (tid < G) {
+    const int h = tid;
+    float M = 0.f;  // m* = max(window max, 0): the linear terms carry the factor exp(-m*) <= 1
+    for (int i = 0; i < ld.n_win_items; ++i) M = fmaxf(M, __ldcg(rec0 + size_t(i) * p.rec_floats + G * D + h));
+    if (has_win) M = fmaxf(M, sm.scur[h]);
+    float den = 0.f;
+    for (int i = 0; i < ld.n_win_items; ++i) {
+      const float *r = rec0 + size_t(i) * p.rec_floats;
+      const float mi = __ldcg(r + G * D + h);
+      den = fmaf(__ldcg(r + G * D + G + h), exp2f(mi - M), den);
+    }
+    if (has_win) den += exp2f(sm.scur[h] - M);
+    if (has_state) {
+      float bsum = 0.f;
+      for (int i = 0; i < ld.n_state_items; ++i)
+        bsum += __ldcg(rec0 + size_t(ld.n_win_items + i) * p.rec_floats + G * D + h);
+      den = fmaf(exp2f(-M), bsum, den);
+    }
+    sm.M[h] = M;
+    sm.inv[h] = 1.0f / den;
+  }
+  __syncthreads();
+  T *outp = reinterpret_cast<T *>(p.out);
+  for (int idx = tid; idx < G * D; idx += kDecodeThreads) {
+    const int h = idx / D, c = idx - h * D;
+    const float M = sm.M[h];
+    float num = 0.f;
+    for (int i = 0; i < ld.n_win_items; ++i) {
+      const float *r = rec0 + size_t(i) * p.rec_floats;
+      num = fmaf(__ldcg(r + idx), exp2f(__ldcg(r + G * D + h) - M), num);
+    }
+    if (has_win) num = fmaf(exp2f(sm.scur[h] - M), to_f32(vt[c]), num);
+    if (has_state) {
+      float asum = 0.f;
+      for (int i = 0; i < ld.n_state_items; ++i) asum += __ldcg(rec0 + size_t(ld.n_win_items + i) * p.rec_floats + idx);
+      num = fmaf(exp2f(-M), asum, num);
+    }
+    const int head = p.heads_of[g * G + h];
+    from_f32(outp + ((size_t(it.layer) * p.B + b) * p.H + head) * D + c, num * sm.inv[h]);
+  }
+  if (has_win) {  // every reader of slot t mod cap has finished: store the new row
+    const size_t row = (size_t(ub) * size_t(ld.cap) + size_t(t % ld.cap)) * D;
+    T *Kd = reinterpret_cast<T *>(p.ws + ld.ringK) + row;
+    T *Vd = reinterpret_cast<T *>(p.ws + ld.ringV) + row;
+    for (int c = tid; c < D; c += kDecodeThreads) {
+      Kd[c] = kt[c];
+      Vd[c] = vt[c];
+    }
+  }
+}
+
+template <typename T, int D, int G>
+__global__ void __launch_bounds__(kDecodeThreads) glide_decode_kernel(const DecodeParams p) {
+  __shared__ DecodeSmem<T, D, G> sm;
+  const int tid = threadIdx.x;
+  const int units_per_layer = p.B * p.Hkv;
+  for (;;) {
+    __syncthreads();
+    if (tid == 0) sm.item = atomicAdd(&p.ctl->work_counter, 1);
+    __syncthreads();
+    const int idx = sm.item;
+    if (idx >= p.n_items) break;
+    const WorkItem it = p.items[idx];
+    if (it.layer < 0 || it.layer >= p.L || it.unit < 0) {  // corrupted list: record and skip
+      if (tid == 0) atomicExch(&p.ctl->status, kDevBadItem);
+      continue;
+    }
+    const LayerDev ld = p.layers[it.layer];
+    const int64_t t = p.n_dev[it.layer];
+    const int ub = it.unit - it.layer * units_per_layer;
+    const int b = ub / p.Hkv, g = ub - b * p.Hkv;
+    const int per_unit = ld.n_win_items + ld.n_state_items;
+    float *rec = p.partials + ld.part_base + (size_t(ub) * per_unit + it.part) * p.rec_floats;
+    if (it.kind == kItemWindow)
+      window_item<T, D, G>(p, it, ld, t, b, g, rec, sm);
+    else
+      state_item<T, D, G>(p, it, ld, t, b, g, rec, sm);
+    __threadfence();
+    __syncthreads();
+    if (tid == 0) sm.last = atomicAdd(&p.tickets[it.unit], 1) == per_unit - 1;
+    __syncthreads();
+    if (sm.last) {
+      __threadfence();
+      merge_unit<T, D, G>(p, it, ld, t, b, g, sm);
+      if (tid == 0) p.tickets[it.unit] = 0;
+    }
+  }
+  if (tid == 0) {
+    __threadfence();
+    if (atomicAdd(&p.ctl->done_counter, 1) == int(gridDim.x) - 1) {
+      // every CTA has drained the list: re-arm it and advance the positions
+      p.ctl->work_counter = 0;
+      p.ctl->done_counter = 0;
+      for (int l = 0; l < p.L; ++l) p.n_dev[l] += 1;
+      __threadfence();
+    }
+  }
+}
+
+__global__ void glide_advance_kernel(int64_t *n_dev, int layer_begin, int layer_count, int64_t T) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < layer_count) n_dev[layer_begin + i] += T;
+}
+
+DecodeParams make_params(const glide_ctx *ctx, const void *q, const void *k, const void *v, void *out) {
+  DecodeParams p{};
+  p.ws = ctx->ws;
+  p.layers = reinterpret_cast<const LayerDev *>(ctx->ws + ctx->off_layers);
+  p.items = reinterpret_cast<const WorkItem *>(ctx->ws + ctx->off_items);
+  p.heads_of = reinterpret_cast<const int32_t *>(ctx->ws + ctx->off_heads);
+  p.ctl = reinterpret_cast<Control *>(ctx->ws + ctx->off_ctl);
+  p.tickets = reinterpret_cast<int32_t *>(ctx->ws + ctx->off_tickets);
+  p.partials = reinterpret_cast<float *>(ctx->ws + ctx->off_partials);
+  p.n_dev = reinterpret_cast<int64_t *>(ctx->ws + ctx->off_ndev);
+  p.q = q;
+  p.k = k;
+  p.v = v;
+  p.out = out;
+  p.n_items = ctx->n_items;
+  p.L = ctx->cfg.n_layers;
+  p.B = ctx->cfg.batch;
+  p.H = ctx->cfg.n_q_heads;
+  p.Hkv = ctx->cfg.n_kv_heads;
+  p.rec_floats = ctx->rec_floats;
+  p.scale_log2 = ctx->scale * kLog2e;
+  return p;
+}
+
+}  // namespace
+
+int decode_occupancy(const glide_ctx *ctx, int *blocks_per_sm) {
+  return dispatch_config(ctx->cfg.io_dtype, ctx->cfg.head_dim, ctx->G, [&](auto tt, auto dd, auto gg) -> int {
+    using T = typename decltype(tt)::type;
+    constexpr int D = decltype(dd)::value, G = decltype(gg)::value;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(blocks_per_sm, glide_decode_kernel<T, D, G>, kDecodeThreads,
+                                                      0) != cudaSuccess) {
+      cudaGetLastError();
+      return GLIDE_ERR_CUDA;
+    }
+    return GLIDE_OK;
+  });
+}
+
+int launch_decode(glide_ctx *ctx, const void *q, const void *k, const void *v, void *out, cudaStream_t stream) {
+  const DecodeParams p = make_params(ctx, q, k, v, out);
+  return dispatch_config(ctx->cfg.io_dtype, ctx->cfg.head_dim, ctx->G, [&](auto tt, auto dd, auto gg) -> int {
+    using T = typename decltype(tt)::type;
+    constexpr int D = decltype(dd)::value, G = decltype(gg)::value;
+    glide_decode_kernel<T, D, G><<<ctx->decode_grid, kDecodeThreads, 0, stream>>>(p);
+    if (cudaGetLastError() != cudaSuccess) return GLIDE_ERR_CUDA;
+    return GLIDE_OK;
+  });
+}
+
+int launch_advance(glide_ctx *ctx, int layer_begin, int layer_count, int64_t T, cudaStream_t stream) {
+  int64_t *n_dev = reinterpret_cast<int64_t *>(ctx->ws + ctx->off_ndev);
+  glide_advance_kernel<<<(layer_count + 63) / 64, 64, 0, stream>>>(n_dev, layer_begin, layer_count, T);
+  if (cudaGetLastError() != cudaSuccess) return GLIDE_ERR_CUDA;
+  return GLIDE_OK;
+}
+
+}  // namespace glide

@@ -1,0 +1,388 @@
+// Host runtime of the GLIDE library: configuration checks, workspace layout, static decode
+// work list, state export/import and bookkeeping.  No device memory is allocated here.
+#include <algorithm>
+#include <cmath>
+#include <cstring>
+#include <new>
+
+#include "glide_internal.h"
+
+using namespace glide;
+
+namespace {
+
+size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+cudaStream_t as_stream(void *s) { return reinterpret_cast<cudaStream_t>(s); }
+
+bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+int validate_config(const glide_config *c) {
+  if (!c || !c->windows) return GLIDE_ERR_INVALID_ARG;
+  if (c->n_layers < 1 || c->batch < 1 || c->n_q_heads < 1 || c->n_kv_heads < 1 || c->max_tokens < 1)
+    return GLIDE_ERR_INVALID_ARG;
+  if (c->io_dtype != GLIDE_F32 && c->io_dtype != GLIDE_BF16) return GLIDE_ERR_INVALID_ARG;
+  if (c->softmax_scale < 0.f || !std::isfinite(c->softmax_scale)) return GLIDE_ERR_INVALID_ARG;
+  if (c->prefill_chunk < 0 || c->decode_chunk < 0 || c->decode_state_splits < 0) return GLIDE_ERR_INVALID_ARG;
+  if (c->prefill_chunk % 16 != 0 || c->prefill_chunk > 1024) return GLIDE_ERR_INVALID_ARG;
+  for (int l = 0; l < c->n_layers; ++l)
+    if (c->windows[l] < 0) return GLIDE_ERR_INVALID_ARG;
+  if (c->phi != GLIDE_PHI_SOFTMAX || c->merge != GLIDE_MERGE_SHARED) return GLIDE_ERR_UNSUPPORTED;
+  if (c->head_dim != 64 && c->head_dim != 128) return GLIDE_ERR_UNSUPPORTED;
+  if (c->n_q_heads % c->n_kv_heads != 0) return GLIDE_ERR_UNSUPPORTED;
+  int G = c->n_q_heads / c->n_kv_heads;
+  if (G != 1 && G != 2 && G != 4 && G != 8) return GLIDE_ERR_UNSUPPORTED;
+  if (c->n_q_heads > 64) return GLIDE_ERR_UNSUPPORTED;
+  if (c->max_tokens > (int64_t(1) << 30)) return GLIDE_ERR_UNSUPPORTED;
+  if (c->q_to_kv) {
+    std::vector<int> cnt(c->n_kv_heads, 0);
+    for (int h = 0; h < c->n_q_heads; ++h) {
+      int g = c->q_to_kv[h];
+      if (g < 0 || g >= c->n_kv_heads) return GLIDE_ERR_INVALID_ARG;
+      cnt[g]++;
+    }
+    for (int g = 0; g < c->n_kv_heads; ++g)
+      if (cnt[g] != G) return GLIDE_ERR_UNSUPPORTED;
+  }
+  return GLIDE_OK;
+}
+
+}  // namespace
+
+int glide::plan_context(const glide_config *cfg, glide_ctx *ctx, std::vector<WorkItem> *items) {
+  int rc = validate_config(cfg);
+  if (rc) return rc;
+  ctx->cfg = *cfg;
+  const int L = cfg->n_layers, B = cfg->batch, H = cfg->n_q_heads, Hkv = cfg->n_kv_heads, d = cfg->head_dim;
+  ctx->G = H / Hkv;
+  ctx->elem = cfg->io_dtype == GLIDE_F32 ? 4 : 2;
+  ctx->scale = cfg->softmax_scale > 0.f ? cfg->softmax_scale : 1.0f / std::sqrt(float(d));
+  ctx->prefill_chunk = cfg->prefill_chunk ? cfg->prefill_chunk : 256;
+  ctx->windows.assign(cfg->windows, cfg->windows + L);
+  ctx->q_to_kv.resize(H);
+  for (int h = 0; h < H; ++h) ctx->q_to_kv[h] = cfg->q_to_kv ? cfg->q_to_kv[h] : h / ctx->G;
+  ctx->heads_of.assign(size_t(Hkv) * ctx->G, 0);
+  {
+    std::vector<int> fill(Hkv, 0);
+    for (int h = 0; h < H; ++h) {
+      int g = ctx->q_to_kv[h];
+      ctx->heads_of[size_t(g) * ctx->G + fill[g]++] = h;
+    }
+  }
+  ctx->cfg.windows = nullptr;
+  ctx->cfg.q_to_kv = nullptr;
+  ctx->n_host.assign(L, 0);
+  ctx->rec_floats = int(align_up(size_t(ctx->G) * (d + 2), 4));
+
+  const int chunk = cfg->decode_chunk ? cfg->decode_chunk : 128;
+  const int splits = cfg->decode_state_splits ? std::min<int>(cfg->decode_state_splits, d) : (d == 128 ? 4 : 2);
+  const int64_t units_per_layer = int64_t(B) * Hkv;
+
+  ctx->layers.assign(L, LayerDev{});
+  size_t part_floats = 0;
+  int64_t n_items = 0;
+  for (int l = 0; l < L; ++l) {
+    LayerDev &ld = ctx->layers[l];
+    ld.w = ctx->windows[l];
+    ld.cap = std::min<int64_t>(ld.w, cfg->max_tokens);
+    ld.evicts = ld.w < cfg->max_tokens ? 1 : 0;
+    ld.n_win_items = int((ld.cap + chunk - 1) / chunk);
+    ld.n_state_items = ld.evicts ? splits : 0;
+    ld.part_base = part_floats;
+    int per_unit = ld.n_win_items + ld.n_state_items;
+    part_floats += size_t(units_per_layer) * per_unit * ctx->rec_floats;
+    n_items += units_per_layer * per_unit;
+  }
+  if (n_items > (int64_t(1) << 30)) return GLIDE_ERR_UNSUPPORTED;
+  ctx->n_items = int(n_items);
+
+  // ---- workspace layout ----
+  size_t off = 0;
+  ctx->off_ctl = off;
+  off = align_up(off + sizeof(Control), 256);
+  ctx->off_ndev = off;
+  off = align_up(off + sizeof(int64_t) * L, 256);
+  ctx->off_layers = off;
+  off = align_up(off + sizeof(LayerDev) * L, 256);
+  ctx->off_heads = off;
+  off = align_up(off + sizeof(int32_t) * H, 256);
+  ctx->off_items = off;
+  off = align_up(off + sizeof(WorkItem) * size_t(n_items), 256);
+  ctx->off_tickets = off;
+  off = align_up(off + sizeof(int32_t) * size_t(L) * units_per_layer, 256);
+  ctx->off_partials = off;
+  off = align_up(off + sizeof(float) * part_floats, 256);
+  ctx->off_phik = off;
+  off = align_up(off + sizeof(float) * size_t(L) * units_per_layer * ctx->prefill_chunk * d, 256);
+  ctx->off_state = off;
+  for (int l = 0; l < L; ++l) {
+    ctx->layers[l].S = off;
+    off += sizeof(float) * size_t(units_per_layer) * d * d;
+  }
+  for (int l = 0; l < L; ++l) {
+    ctx->layers[l].z = off;
+    off += sizeof(float) * size_t(units_per_layer) * d;
+  }
+  ctx->state_bytes = off - ctx->off_state;
+  off = align_up(off, 256);
+  ctx->off_ring = off;
+  for (int l = 0; l < L; ++l) {
+    size_t bytes = align_up(size_t(units_per_layer) * size_t(ctx->layers[l].cap) * d * ctx->elem, 256);
+    ctx->layers[l].ringK = off;
+    off += bytes;
+    ctx->layers[l].ringV = off;
+    off += bytes;
+  }
+  ctx->total = align_up(off, 256);
+
+  if (items) {
+    items->clear();
+    items->reserve(size_t(n_items));
+    for (int l = 0; l < L; ++l) {
+      const LayerDev &ld = ctx->layers[l];
+      for (int64_t u = 0; u < units_per_layer; ++u) {
+        int unit = int(int64_t(l) * units_per_layer + u);
+        int part = 0;
+        for (int i = 0; i < ld.n_win_items; ++i) {
+          WorkItem it{};
+          it.unit = unit;
+          it.layer = l;
+          it.kind = kItemWindow;
+          it.part = part++;
+          it.begin = i * chunk;
+          it.count = int(std::min<int64_t>(chunk, ld.cap - int64_t(i) * chunk));
+          items->push_back(it);
+        }
+        for (int i = 0; i < ld.n_state_items; ++i) {
+          WorkItem it{};
+          it.unit = unit;
+          it.layer = l;
+          it.kind = kItemState;
+          it.part = part++;
+          int r0 = int(int64_t(d) * i / ld.n_state_items), r1 = int(int64_t(d) * (i + 1) / ld.n_state_items);
+          it.begin = r0;
+          it.count = r1 - r0;
+          items->push_back(it);
+        }
+      }
+    }
+    // longest first: bytes an item moves
+    const size_t elem = ctx->elem;
+    auto cost = [&](const WorkItem &it) -> size_t {
+      return it.kind == kItemWindow ? size_t(it.count) * d * elem * 2 : size_t(it.count) * d * 4 * 2;
+    };
+    std::stable_sort(items->begin(), items->end(),
+                     [&](const WorkItem &a, const WorkItem &b) { return cost(a) > cost(b); });
+  }
+  return GLIDE_OK;
+}
+
+extern "C" {
+
+int glide_workspace_bytes(const glide_config *cfg, size_t *bytes_out) {
+  if (!bytes_out) return GLIDE_ERR_INVALID_ARG;
+  glide_ctx tmp;
+  int rc = plan_context(cfg, &tmp, nullptr);
+  if (rc) return rc;
+  *bytes_out = tmp.total;
+  return GLIDE_OK;
+}
+
+int glide_create(const glide_config *cfg, void *dev_workspace, size_t workspace_bytes, void *stream,
+                 glide_ctx **ctx_out) {
+  if (!ctx_out) return GLIDE_ERR_INVALID_ARG;
+  *ctx_out = nullptr;
+  glide_ctx *ctx = new (std::nothrow) glide_ctx;
+  if (!ctx) return GLIDE_ERR_INVALID_ARG;
+  std::vector<WorkItem> items;
+  int rc = plan_context(cfg, ctx, &items);
+  if (rc) {
+    delete ctx;
+    return rc;
+  }
+  if (!dev_workspace || (reinterpret_cast<uintptr_t>(dev_workspace) & 255u)) {
+    delete ctx;
+    return GLIDE_ERR_INVALID_ARG;
+  }
+  if (workspace_bytes < ctx->total) {
+    delete ctx;
+    return GLIDE_ERR_WORKSPACE_TOO_SMALL;
+  }
+  ctx->ws = static_cast<unsigned char *>(dev_workspace);
+  ctx->ws_bytes = workspace_bytes;
+  cudaStream_t st = as_stream(stream);
+  bool ok = cudaGetDevice(&ctx->device) == cudaSuccess &&
+            cudaDeviceGetAttribute(&ctx->sm_count, cudaDevAttrMultiProcessorCount, ctx->device) == cudaSuccess;
+  int per_sm = 0;
+  ok = ok && decode_occupancy(ctx, &per_sm) == GLIDE_OK && per_sm > 0;
+  if (ok) {
+    ctx->decode_grid = std::max(1, std::min(ctx->n_items, ctx->sm_count * per_sm));
+    // control words, counters, tickets, S and z start at zero
+    ok = cudaMemsetAsync(ctx->ws, 0, ctx->off_layers, st) == cudaSuccess &&
+         cudaMemsetAsync(ctx->ws + ctx->off_tickets, 0, ctx->off_partials - ctx->off_tickets, st) == cudaSuccess &&
+         cudaMemsetAsync(ctx->ws + ctx->off_state, 0, ctx->state_bytes, st) == cudaSuccess;
+    ok = ok && cudaMemcpyAsync(ctx->ws + ctx->off_layers, ctx->layers.data(), sizeof(LayerDev) * ctx->layers.size(),
+                               cudaMemcpyHostToDevice, st) == cudaSuccess;
+    ok = ok && cudaMemcpyAsync(ctx->ws + ctx->off_heads, ctx->heads_of.data(), sizeof(int32_t) * ctx->heads_of.size(),
+                               cudaMemcpyHostToDevice, st) == cudaSuccess;
+    ok = ok && cudaMemcpyAsync(ctx->ws + ctx->off_items, items.data(), sizeof(WorkItem) * items.size(),
+                               cudaMemcpyHostToDevice, st) == cudaSuccess;
+    // the host vectors above are pageable and go out of scope: finish the copies now
+    ok = ok && cudaStreamSynchronize(st) == cudaSuccess;
+  }
+  if (!ok) {
+    cudaGetLastError();
+    delete ctx;
+    return GLIDE_ERR_CUDA;
+  }
+  *ctx_out = ctx;
+  return GLIDE_OK;
+}
+
+int glide_destroy(glide_ctx *ctx) {
+  if (!ctx) return GLIDE_ERR_INVALID_ARG;
+  delete ctx;
+  return GLIDE_OK;
+}
+
+int glide_decode_step(glide_ctx *ctx, const void *q, const void *k, const void *v, void *out, void *stream) {
+  if (!ctx || !q || !k || !v || !out) return GLIDE_ERR_INVALID_ARG;
+  if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out)) return GLIDE_ERR_INVALID_ARG;
+  const int L = ctx->cfg.n_layers;
+  for (int l = 1; l < L; ++l)
+    if (ctx->n_host[l] != ctx->n_host[0]) return GLIDE_ERR_STATE;
+  if (ctx->n_host[0] + 1 > ctx->cfg.max_tokens) return GLIDE_ERR_CAPACITY;
+  int rc = launch_decode(ctx, q, k, v, out, as_stream(stream));
+  if (rc) return rc;
+  for (int l = 0; l < L; ++l) ctx->n_host[l] += 1;
+  return GLIDE_OK;
+}
+
+int glide_prefill(glide_ctx *ctx, int32_t layer_begin, int32_t layer_count, int64_t T, const void *q, const void *k,
+                  const void *v, void *out, void *stream) {
+  if (!ctx || !k || !v || T < 0) return GLIDE_ERR_INVALID_ARG;
+  if (out && !q) return GLIDE_ERR_INVALID_ARG;
+  if (layer_begin < 0 || layer_count < 1 || layer_begin + layer_count > ctx->cfg.n_layers)
+    return GLIDE_ERR_INVALID_ARG;
+  if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out)) return GLIDE_ERR_INVALID_ARG;
+  for (int l = layer_begin + 1; l < layer_begin + layer_count; ++l)
+    if (ctx->n_host[l] != ctx->n_host[layer_begin]) return GLIDE_ERR_STATE;
+  if (ctx->n_host[layer_begin] + T > ctx->cfg.max_tokens) return GLIDE_ERR_CAPACITY;
+  if (T == 0) return GLIDE_OK;
+  int rc = launch_prefill(ctx, layer_begin, layer_count, T, q, k, v, out, as_stream(stream));
+  if (rc) return rc;
+  for (int l = layer_begin; l < layer_begin + layer_count; ++l) ctx->n_host[l] += T;
+  return GLIDE_OK;
+}
+
+int glide_layer_info(glide_ctx *ctx, int32_t layer, void *stream, glide_layer_info_t *out) {
+  if (!ctx || !out || layer < 0 || layer >= ctx->cfg.n_layers) return GLIDE_ERR_INVALID_ARG;
+  int64_t n = 0;
+  cudaStream_t st = as_stream(stream);
+  if (cudaMemcpyAsync(&n, ctx->ws + ctx->off_ndev + sizeof(int64_t) * layer, sizeof(int64_t), cudaMemcpyDeviceToHost,
+                      st) != cudaSuccess ||
+      cudaStreamSynchronize(st) != cudaSuccess) {
+    cudaGetLastError();
+    return GLIDE_ERR_CUDA;
+  }
+  const LayerDev &ld = ctx->layers[layer];
+  out->window = ld.w;
+  out->capacity = ld.cap;
+  out->n = n;
+  out->count = std::min<int64_t>(n, ld.w);
+  out->head_slot = ld.cap > 0 ? n % ld.cap : 0;
+  out->n_evicted = std::max<int64_t>(0, n - ld.w);
+  return GLIDE_OK;
+}
+
+int glide_export_state(glide_ctx *ctx, int32_t layer, void *ringK, void *ringV, float *S, float *z, void *stream) {
+  if (!ctx || layer < 0 || layer >= ctx->cfg.n_layers) return GLIDE_ERR_INVALID_ARG;
+  const LayerDev &ld = ctx->layers[layer];
+  const size_t units = size_t(ctx->cfg.batch) * ctx->cfg.n_kv_heads, d = ctx->cfg.head_dim;
+  const size_t ring_bytes = units * size_t(ld.cap) * d * ctx->elem;
+  cudaStream_t st = as_stream(stream);
+  bool ok = true;
+  if (ringK && ring_bytes) ok = ok && cudaMemcpyAsync(ringK, ctx->ws + ld.ringK, ring_bytes, cudaMemcpyDeviceToDevice, st) == cudaSuccess;
+  if (ringV && ring_bytes) ok = ok && cudaMemcpyAsync(ringV, ctx->ws + ld.ringV, ring_bytes, cudaMemcpyDeviceToDevice, st) == cudaSuccess;
+  if (S) ok = ok && cudaMemcpyAsync(S, ctx->ws + ld.S, units * d * d * 4, cudaMemcpyDeviceToDevice, st) == cudaSuccess;
+  if (z) ok = ok && cudaMemcpyAsync(z, ctx->ws + ld.z, units * d * 4, cudaMemcpyDeviceToDevice, st) == cudaSuccess;
+  if (!ok) {
+    cudaGetLastError();
+    return GLIDE_ERR_CUDA;
+  }
+  return GLIDE_OK;
+}
+
+int glide_import_state(glide_ctx *ctx, int32_t layer, int64_t n, const void *ringK, const void *ringV, const float *S,
+                       const float *z, void *stream) {
+  if (!ctx || layer < 0 || layer >= ctx->cfg.n_layers || n < 0 || n > ctx->cfg.max_tokens)
+    return GLIDE_ERR_INVALID_ARG;
+  const LayerDev &ld = ctx->layers[layer];
+  const size_t units = size_t(ctx->cfg.batch) * ctx->cfg.n_kv_heads, d = ctx->cfg.head_dim;
+  const size_t ring_bytes = units * size_t(ld.cap) * d * ctx->elem;
+  cudaStream_t st = as_stream(stream);
+  bool ok = true;
+  if (ringK && ring_bytes) ok = ok && cudaMemcpyAsync(ctx->ws + ld.ringK, ringK, ring_bytes, cudaMemcpyDeviceToDevice, st) == cudaSuccess;
+  if (ringV && ring_bytes) ok = ok && cudaMemcpyAsync(ctx->ws + ld.ringV, ringV, ring_bytes, cudaMemcpyDeviceToDevice, st) == cudaSuccess;
+  if (S) ok = ok && cudaMemcpyAsync(ctx->ws + ld.S, S, units * d * d * 4, cudaMemcpyDeviceToDevice, st) == cudaSuccess;
+  if (z) ok = ok && cudaMemcpyAsync(ctx->ws + ld.z, z, units * d * 4, cudaMemcpyDeviceToDevice, st) == cudaSuccess;
+  // the counter is a pageable 8-byte source: the runtime stages it before returning
+  ok = ok && cudaMemcpyAsync(ctx->ws + ctx->off_ndev + sizeof(int64_t) * layer, &n, sizeof(int64_t),
+                             cudaMemcpyHostToDevice, st) == cudaSuccess;
+  if (!ok) {
+    cudaGetLastError();
+    return GLIDE_ERR_CUDA;
+  }
+  ctx->n_host[layer] = n;
+  return GLIDE_OK;
+}
+
+int glide_reset(glide_ctx *ctx, void *stream) {
+  if (!ctx) return GLIDE_ERR_INVALID_ARG;
+  cudaStream_t st = as_stream(stream);
+  bool ok = cudaMemsetAsync(ctx->ws, 0, ctx->off_layers, st) == cudaSuccess &&
+            cudaMemsetAsync(ctx->ws + ctx->off_tickets, 0, ctx->off_partials - ctx->off_tickets, st) == cudaSuccess &&
+            cudaMemsetAsync(ctx->ws + ctx->off_state, 0, ctx->state_bytes, st) == cudaSuccess;
+  if (!ok) {
+    cudaGetLastError();
+    return GLIDE_ERR_CUDA;
+  }
+  std::fill(ctx->n_host.begin(), ctx->n_host.end(), 0);
+  return GLIDE_OK;
+}
+
+int glide_device_status(glide_ctx *ctx, void *stream, int32_t *status_out) {
+  if (!ctx || !status_out) return GLIDE_ERR_INVALID_ARG;
+  cudaStream_t st = as_stream(stream);
+  Control c{};
+  if (cudaMemcpyAsync(&c, ctx->ws + ctx->off_ctl, sizeof(Control), cudaMemcpyDeviceToHost, st) != cudaSuccess ||
+      cudaStreamSynchronize(st) != cudaSuccess) {
+    cudaGetLastError();
+    return GLIDE_ERR_CUDA;
+  }
+  *status_out = c.status;
+  return GLIDE_OK;
+}
+
+int glide_decode_launch_info(glide_ctx *ctx, int32_t *n_launches, int32_t *n_work_items, int32_t *grid_size) {
+  if (!ctx) return GLIDE_ERR_INVALID_ARG;
+  if (n_launches) *n_launches = 1;
+  if (n_work_items) *n_work_items = ctx->n_items;
+  if (grid_size) *grid_size = ctx->decode_grid;
+  return GLIDE_OK;
+}
+
+const char *glide_strerror(int code) {
+  switch (code) {
+    case GLIDE_OK: return "ok";
+    case GLIDE_ERR_INVALID_ARG: return "invalid argument";
+    case GLIDE_ERR_UNSUPPORTED: return "unsupported configuration";
+    case GLIDE_ERR_WORKSPACE_TOO_SMALL: return "workspace too small";
+    case GLIDE_ERR_CAPACITY: return "sequence capacity (max_tokens) exceeded";
+    case GLIDE_ERR_STATE: return "layers are at different positions";
+    case GLIDE_ERR_CUDA: return "CUDA runtime error";
+    default: return "unknown status";
+  }
+}
+
+}  // extern "C"

@@ -1,0 +1,127 @@
+// Internal structures shared by the host runtime and the kernels of the GLIDE library.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include <vector>
+
+#include "glide.h"
+
+namespace glide {
+
+constexpr int kDecodeThreads = 128;   // 4 warps per CTA
+constexpr int kMaxGroup = 8;          // query heads per KV head
+
+// Per-layer constants, resident in the workspace (device) and mirrored on the host.
+struct LayerDev {
+  int64_t w;            // configured window
+  int64_t cap;          // ring slots: min(w, max_tokens)
+  size_t ringK;         // byte offset in the workspace: [B][Hkv][cap][d] (I/O dtype)
+  size_t ringV;
+  size_t S;             // byte offset: [B][Hkv][d][d] fp32
+  size_t z;             // byte offset: [B][Hkv][d] fp32
+  size_t part_base;     // float index into the split-K scratch of this layer's first unit
+  int32_t n_win_items;  // window work items per unit
+  int32_t n_state_items;// state work items per unit (0 if the layer never evicts)
+  int32_t evicts;       // 1 if w < max_tokens
+  int32_t pad_;
+};
+
+// One work item of the decode kernel.
+struct WorkItem {
+  int32_t unit;    // (layer * B + b) * Hkv + g
+  int32_t layer;
+  int32_t kind;    // 0 window slots [begin, begin + count), 1 state rows [begin, begin + count)
+  int32_t part;    // index of this item's partial record within the unit
+  int32_t begin;
+  int32_t count;
+  int32_t pad0_, pad1_;
+};
+
+enum : int { kItemWindow = 0, kItemState = 1 };
+
+// Device status codes (glide_device_status).
+enum : int { kDevOk = 0, kDevBadSlot = 1, kDevBadItem = 2 };
+
+// Control words at the start of the workspace.
+struct Control {
+  int32_t work_counter;
+  int32_t done_counter;
+  int32_t status;
+  int32_t pad_;
+};
+
+struct DecodeParams {
+  unsigned char *ws;
+  const LayerDev *layers;
+  const WorkItem *items;
+  const int32_t *heads_of;   // [Hkv][G] query heads of each KV head
+  Control *ctl;
+  int32_t *tickets;          // [units]
+  float *partials;
+  int64_t *n_dev;            // [L]
+  const void *q, *k, *v;
+  void *out;
+  int32_t n_items;
+  int32_t L, B, H, Hkv;
+  int32_t rec_floats;        // floats per partial record: G * (d + 2) rounded up to 4
+  float scale_log2;          // softmax_scale * log2(e)
+};
+
+struct PrefillParams {
+  unsigned char *ws;
+  const LayerDev *layers;
+  const int32_t *heads_of;
+  Control *ctl;
+  float *phik;               // chunk scratch: [layer_count][B][Hkv][C][d] fp32, phi of the delayed keys
+  const void *q, *k, *v;     // the call's inputs
+  void *out;
+  int64_t n0;                // tokens absorbed before this call (all layers of the call)
+  int64_t T;                 // tokens of this call
+  int64_t c0;                // first token (call-relative) of the current chunk
+  int32_t C;                 // tokens in the current chunk
+  int32_t Cmax;              // scratch stride (prefill_chunk)
+  int32_t layer_begin, layer_count;
+  int32_t L, B, H, Hkv;
+  float scale_log2;
+};
+
+}  // namespace glide
+
+struct glide_ctx {
+  glide_config cfg;                 // pointers inside are not used after create
+  std::vector<int64_t> windows;
+  std::vector<int32_t> q_to_kv;
+  std::vector<int32_t> heads_of;    // [Hkv][G]
+  std::vector<glide::LayerDev> layers;
+  std::vector<int64_t> n_host;      // mirror of the device counters
+  int G = 0;
+  int device = 0;
+  int sm_count = 0;
+  int decode_grid = 0;
+  int n_items = 0;
+  int rec_floats = 0;
+  int prefill_chunk = 0;
+  float scale = 0.f;
+  size_t elem = 0;
+  unsigned char *ws = nullptr;
+  size_t ws_bytes = 0;
+  // workspace regions (byte offsets)
+  size_t off_ctl = 0, off_ndev = 0, off_layers = 0, off_heads = 0, off_items = 0, off_tickets = 0,
+         off_partials = 0, off_phik = 0, off_state = 0, off_ring = 0, total = 0;
+  size_t state_bytes = 0;           // S and z of all layers (contiguous)
+};
+
+namespace glide {
+
+// Layout planning shared by glide_workspace_bytes and glide_create (host only).
+int plan_context(const glide_config *cfg, glide_ctx *ctx, std::vector<WorkItem> *items);
+
+int launch_decode(glide_ctx *ctx, const void *q, const void *k, const void *v, void *out, cudaStream_t stream);
+int decode_occupancy(const glide_ctx *ctx, int *blocks_per_sm);
+int launch_prefill(glide_ctx *ctx, int layer_begin, int layer_count, int64_t T, const void *q, const void *k,
+                   const void *v, void *out, cudaStream_t stream);
+int launch_advance(glide_ctx *ctx, int layer_begin, int layer_count, int64_t T, cudaStream_t stream);
+
+}  // namespace glide

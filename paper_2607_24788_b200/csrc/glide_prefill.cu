@@ -1,0 +1,332 @@
+// GLIDE prefill: append T prompt tokens, chunk by chunk (C tokens per chunk).
+//
+// For a layer with window w the linear part of query i sums over tokens j <= i - w, i.e. it is
+// ordinary causal (inclusive) linear attention on the stream delayed by w tokens:
+// k'_i = k_{i-w}, v'_i = v_{i-w}.  Per chunk, in stream order:
+//   1. phi kernel    phi(k') of the chunk's delayed tokens -> scratch (fp32)
+//   2. attn kernel   per query: sliding-window online softmax over ring-or-call rows, the readout
+//                    phi(q) S / phi(q) z of the state at chunk start, the intra-chunk delayed terms
+//                    (phi(q).phi(k'_j)) v'_j, merged under the shared normaliser -> out
+//   3. state kernel  S += phi(K'_c)^T V'_c, z += sum phi(K'_c)   (fp32 carry)
+//   4. ring kernel   the chunk's newest min(C, cap) tokens -> slot (position mod cap)
+// The delayed rows and the window rows older than the call come from the ring, which step 4 of
+// the same chunk overwrites only after steps 1-3 have read it.
+#include <algorithm>
+
+#include "glide_device.cuh"
+
+namespace glide {
+
+namespace {
+
+constexpr int kPrefillThreads = 128;
+
+template <typename T>
+struct RowSource {
+  const T *ringK, *ringV;   // unit base: [cap][D]
+  const T *callK, *callV;   // (layer, sequence) base: [T][Hkv][D], already offset to KV head g
+  int64_t n0, cap;
+  int64_t call_stride;      // Hkv * D
+  __device__ __forceinline__ const T *k(int64_t j, int D) const {
+    return j >= n0 ? callK + (j - n0) * call_stride : ringK + (j % cap) * D;
+  }
+  __device__ __forceinline__ const T *v(int64_t j, int D) const {
+    return j >= n0 ? callV + (j - n0) * call_stride : ringV + (j % cap) * D;
+  }
+};
+
+template <typename T, int D>
+__device__ __forceinline__ RowSource<T> make_source(const PrefillParams &p, const LayerDev &ld, int lrel, int b, int g) {
+  RowSource<T> s;
+  const size_t unit_rows = (size_t(b) * p.Hkv + g) * size_t(ld.cap);
+  s.ringK = reinterpret_cast<const T *>(p.ws + ld.ringK) + unit_rows * D;
+  s.ringV = reinterpret_cast<const T *>(p.ws + ld.ringV) + unit_rows * D;
+  const size_t seq = (size_t(lrel) * p.B + b) * size_t(p.T) * p.Hkv * D + size_t(g) * D;
+  s.callK = reinterpret_cast<const T *>(p.k) + seq;
+  s.callV = reinterpret_cast<const T *>(p.v) + seq;
+  s.n0 = p.n0;
+  s.cap = ld.cap > 0 ? ld.cap : 1;
+  s.call_stride = int64_t(p.Hkv) * D;
+  return s;
+}
+
+// 1. phi of the delayed keys of this chunk: one warp per (unit, chunk token)
+template <typename T, int D>
+__global__ void __launch_bounds__(kPrefillThreads) prefill_phi_kernel(const PrefillParams p) {
+  constexpr int E = D / 32;
+  const int lane = threadIdx.x & 31;
+  const int64_t wid = (int64_t(blockIdx.x) * kPrefillThreads + threadIdx.x) >> 5;
+  const int64_t units = int64_t(p.layer_count) * p.B * p.Hkv;
+  if (wid >= units * p.C) return;
+  const int i = int(wid % p.C);
+  const int64_t u = wid / p.C;
+  const int g = int(u % p.Hkv);
+  const int b = int((u / p.Hkv) % p.B);
+  const int lrel = int(u / (int64_t(p.Hkv) * p.B));
+  const LayerDev ld = p.layers[p.layer_begin + lrel];
+  if (!ld.evicts) return;
+  const int64_t j = p.n0 + p.c0 + i - ld.w;  // delayed token
+  if (j < 0) return;
+  const RowSource<T> src = make_source<T, D>(p, ld, lrel, b, g);
+  float x[E];
+  load_elems<T, E>(src.k(j, D) + lane * E, x);
+  warp_phi<E>(x);
+  float *dst = p.phik + (size_t(u) * p.Cmax + i) * D + lane * E;
+#pragma unroll
+  for (int e = 0; e < E; ++e) dst[e] = x[e];
+}
+
+// 2. outputs: one warp per (unit, query token), G heads at once
+template <typename T, int D, int G>
+__global__ void __launch_bounds__(kPrefillThreads) prefill_attn_kernel(const PrefillParams p) {
+  constexpr int E = D / 32;
+  constexpr int NW = kPrefillThreads / 32;
+  __shared__ float sm_phiq[NW][G][D];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int64_t wid = int64_t(blockIdx.x) * NW + warp;
+  const int64_t units = int64_t(p.layer_count) * p.B * p.Hkv;
+  if (wid >= units * p.C) return;
+  const int i = int(wid % p.C);
+  const int64_t u = wid / p.C;
+  const int g = int(u % p.Hkv);
+  const int b = int((u / p.Hkv) % p.B);
+  const int lrel = int(u / (int64_t(p.Hkv) * p.B));
+  const LayerDev ld = p.layers[p.layer_begin + lrel];
+  const RowSource<T> src = make_source<T, D>(p, ld, lrel, b, g);
+  const int64_t tq = p.n0 + p.c0 + i;  // absolute position of the query
+  const int ub = b * p.Hkv + g;
+
+  float qr[G][E];
+  const T *qbase = reinterpret_cast<const T *>(p.q) + ((size_t(lrel) * p.B + b) * size_t(p.T) + size_t(p.c0 + i)) * p.H * D;
+#pragma unroll
+  for (int h = 0; h < G; ++h) {
+    const int head = p.heads_of[g * G + h];
+    load_elems<T, E>(qbase + size_t(head) * D + lane * E, qr[h]);
+    float x[E];
+#pragma unroll
+    for (int e = 0; e < E; ++e) x[e] = qr[h][e];
+    warp_phi<E>(x);
+#pragma unroll
+    for (int e = 0; e < E; ++e) {
+      sm_phiq[warp][h][lane * E + e] = x[e];
+      qr[h][e] *= p.scale_log2;
+    }
+  }
+  __syncwarp();
+
+  // window part: tokens max(0, tq - w + 1) .. tq
+  float acc[G][E], m[G], l[G];
+#pragma unroll
+  for (int h = 0; h < G; ++h) {
+    m[h] = -CUDART_INF_F;
+    l[h] = 0.f;
+#pragma unroll
+    for (int e = 0; e < E; ++e) acc[h][e] = 0.f;
+  }
+  int64_t w_lo = tq - ld.w + 1;
+  if (w_lo < 0) w_lo = 0;
+  for (int64_t j = w_lo; j <= tq; j += 2) {
+    float kx[2][E], vx[2][E];
+    const bool two = j + 1 <= tq;
+    load_elems<T, E>(src.k(j, D) + lane * E, kx[0]);
+    load_elems<T, E>(src.v(j, D) + lane * E, vx[0]);
+    if (two) {
+      load_elems<T, E>(src.k(j + 1, D) + lane * E, kx[1]);
+      load_elems<T, E>(src.v(j + 1, D) + lane * E, vx[1]);
+    }
+    online_row<E, G>(qr, kx[0], vx[0], m, l, acc);
+    if (two) online_row<E, G>(qr, kx[1], vx[1], m, l, acc);
+  }
+
+  // linear part on the delayed stream
+  float lin[G][E], bl[G];
+#pragma unroll
+  for (int h = 0; h < G; ++h) {
+    bl[h] = 0.f;
+#pragma unroll
+    for (int e = 0; e < E; ++e) lin[h][e] = 0.f;
+  }
+  if (ld.evicts && tq >= ld.w) {
+    const int64_t folded_at_chunk_start = p.n0 + p.c0 - ld.w;  // tokens < this are in S,z
+    if (folded_at_chunk_start > 0) {
+      const float *Sb = reinterpret_cast<const float *>(p.ws + ld.S) + size_t(ub) * D * D;
+      const float *zb = reinterpret_cast<const float *>(p.ws + ld.z) + size_t(ub) * D;
+      for (int r = 0; r < D; ++r) {
+        float s[E];
+        load_elems<float, E>(Sb + size_t(r) * D + lane * E, s);
+#pragma unroll
+        for (int h = 0; h < G; ++h) {
+          const float f = sm_phiq[warp][h][r];
+#pragma unroll
+          for (int e = 0; e < E; ++e) lin[h][e] = fmaf(f, s[e], lin[h][e]);
+        }
+      }
+      float zz[E];
+      load_elems<float, E>(zb + lane * E, zz);
+#pragma unroll
+      for (int h = 0; h < G; ++h) {
+        float part = 0.f;
+#pragma unroll
+        for (int e = 0; e < E; ++e) part = fmaf(sm_phiq[warp][h][lane * E + e], zz[e], part);
+        bl[h] = warp_sum(part);
+      }
+    }
+    // delayed tokens of this chunk, up to and including the query's own delayed token
+    const float *pk = p.phik + size_t(u) * p.Cmax * D;
+    int i_lo = 0;
+    if (folded_at_chunk_start < 0) i_lo = int(-folded_at_chunk_start);  // delayed index < 0 does not exist
+    for (int ii = i_lo; ii <= i; ++ii) {
+      const int64_t j = p.n0 + p.c0 + ii - ld.w;
+      float fk[E], vx[E];
+      load_elems<float, E>(pk + size_t(ii) * D + lane * E, fk);
+      load_elems<T, E>(src.v(j, D) + lane * E, vx);
+#pragma unroll
+      for (int h = 0; h < G; ++h) {
+        float part = 0.f;
+#pragma unroll
+        for (int e = 0; e < E; ++e) part = fmaf(sm_phiq[warp][h][lane * E + e], fk[e], part);
+        const float c = warp_sum(part);
+        bl[h] += c;
+#pragma unroll
+        for (int e = 0; e < E; ++e) lin[h][e] = fmaf(c, vx[e], lin[h][e]);
+      }
+    }
+  }
+
+  // shared normaliser
+  T *obase = reinterpret_cast<T *>(p.out) + ((size_t(lrel) * p.B + b) * size_t(p.T) + size_t(p.c0 + i)) * p.H * D;
+#pragma unroll
+  for (int h = 0; h < G; ++h) {
+    const float M = fmaxf(m[h], 0.f);
+    const float fw = m[h] == -CUDART_INF_F ? 0.f : exp2f(m[h] - M);
+    const float fl = exp2f(-M);
+    const float inv = 1.0f / fmaf(l[h], fw, fl * bl[h]);
+    const int head = p.heads_of[g * G + h];
+#pragma unroll
+    for (int e = 0; e < E; ++e)
+      from_f32(obase + size_t(head) * D + lane * E + e, (acc[h][e] * fw + fl * lin[h][e]) * inv);
+  }
+}
+
+// 3. S += phi(K'_c)^T V'_c ; z += sum phi(K'_c): one CTA per (unit, block of RB state rows)
+template <typename T, int D>
+__global__ void __launch_bounds__(kPrefillThreads) prefill_state_kernel(const PrefillParams p) {
+  constexpr int RB = 16;                          // state rows per CTA
+  constexpr int NRS = kPrefillThreads / D > 0 ? kPrefillThreads / D : 1;  // row sub-groups (1 for D=128, 2 for D=64)
+  constexpr int RPT = RB / NRS;                   // rows per thread
+  const int blocks_per_unit = D / RB;
+  const int64_t u = blockIdx.x / blocks_per_unit;
+  const int rb = blockIdx.x % blocks_per_unit;
+  const int g = int(u % p.Hkv);
+  const int b = int((u / p.Hkv) % p.B);
+  const int lrel = int(u / (int64_t(p.Hkv) * p.B));
+  const LayerDev ld = p.layers[p.layer_begin + lrel];
+  if (!ld.evicts) return;
+  const int64_t first = p.n0 + p.c0 - ld.w;       // delayed token of chunk index 0
+  int i_lo = first < 0 ? int(first < -int64_t(p.C) ? p.C : -first) : 0;
+  if (i_lo >= p.C) return;
+  const RowSource<T> src = make_source<T, D>(p, ld, lrel, b, g);
+  const int ub = b * p.Hkv + g;
+  const int c = threadIdx.x % D, rs = threadIdx.x / D;
+  const int r0 = rb * RB + rs * RPT;
+  const float *pk = p.phik + size_t(u) * p.Cmax * D;
+  if (rs < NRS) {
+    float acc[RPT];
+#pragma unroll
+    for (int r = 0; r < RPT; ++r) acc[r] = 0.f;
+    for (int i = i_lo; i < p.C; ++i) {
+      const float vv = to_f32(src.v(first + i, D)[c]);
+      const float *f = pk + size_t(i) * D + r0;
+#pragma unroll
+      for (int r = 0; r < RPT; ++r) acc[r] = fmaf(f[r], vv, acc[r]);
+    }
+    float *Sb = reinterpret_cast<float *>(p.ws + ld.S) + size_t(ub) * D * D;
+#pragma unroll
+    for (int r = 0; r < RPT; ++r) Sb[size_t(r0 + r) * D + c] += acc[r];
+  }
+  if (rb == 0 && threadIdx.x < D) {
+    float zs = 0.f;
+    for (int i = i_lo; i < p.C; ++i) zs += pk[size_t(i) * D + threadIdx.x];
+    float *zb = reinterpret_cast<float *>(p.ws + ld.z) + size_t(ub) * D;
+    zb[threadIdx.x] += zs;
+  }
+}
+
+// 4. ring fill: the chunk's newest min(C, cap) tokens
+template <typename T, int D>
+__global__ void __launch_bounds__(kPrefillThreads) prefill_ring_kernel(const PrefillParams p) {
+  constexpr int E = D / 32;
+  const int lane = threadIdx.x & 31;
+  const int64_t wid = (int64_t(blockIdx.x) * kPrefillThreads + threadIdx.x) >> 5;
+  const int64_t units = int64_t(p.layer_count) * p.B * p.Hkv;
+  if (wid >= units * p.C) return;
+  const int i = int(wid % p.C);
+  const int64_t u = wid / p.C;
+  const int g = int(u % p.Hkv);
+  const int b = int((u / p.Hkv) % p.B);
+  const int lrel = int(u / (int64_t(p.Hkv) * p.B));
+  const LayerDev ld = p.layers[p.layer_begin + lrel];
+  if (ld.cap == 0 || int64_t(i) < int64_t(p.C) - ld.cap) return;  // older tokens of the chunk are overwritten anyway
+  const int64_t j = p.n0 + p.c0 + i;
+  const size_t src = (((size_t(lrel) * p.B + b) * size_t(p.T) + size_t(p.c0 + i)) * p.Hkv + g) * D + lane * E;
+  const size_t dst = ((size_t(b) * p.Hkv + g) * size_t(ld.cap) + size_t(j % ld.cap)) * D + lane * E;
+  const T *ks = reinterpret_cast<const T *>(p.k) + src;
+  const T *vs = reinterpret_cast<const T *>(p.v) + src;
+  T *kd = reinterpret_cast<T *>(p.ws + ld.ringK) + dst;
+  T *vd = reinterpret_cast<T *>(p.ws + ld.ringV) + dst;
+#pragma unroll
+  for (int e = 0; e < E; ++e) {
+    kd[e] = ks[e];
+    vd[e] = vs[e];
+  }
+}
+
+}  // namespace
+
+int launch_prefill(glide_ctx *ctx, int layer_begin, int layer_count, int64_t T, const void *q, const void *k,
+                   const void *v, void *out, cudaStream_t stream) {
+  PrefillParams p{};
+  p.ws = ctx->ws;
+  p.layers = reinterpret_cast<const LayerDev *>(ctx->ws + ctx->off_layers);
+  p.heads_of = reinterpret_cast<const int32_t *>(ctx->ws + ctx->off_heads);
+  p.ctl = reinterpret_cast<Control *>(ctx->ws + ctx->off_ctl);
+  p.phik = reinterpret_cast<float *>(ctx->ws + ctx->off_phik);
+  p.q = q;
+  p.k = k;
+  p.v = v;
+  p.out = out;
+  p.n0 = ctx->n_host[layer_begin];
+  p.T = T;
+  p.Cmax = ctx->prefill_chunk;
+  p.layer_begin = layer_begin;
+  p.layer_count = layer_count;
+  p.L = ctx->cfg.n_layers;
+  p.B = ctx->cfg.batch;
+  p.H = ctx->cfg.n_q_heads;
+  p.Hkv = ctx->cfg.n_kv_heads;
+  p.scale_log2 = ctx->scale * kLog2e;
+  const int64_t units = int64_t(layer_count) * p.B * p.Hkv;
+  bool any_evicts = false;
+  for (int l = layer_begin; l < layer_begin + layer_count; ++l) any_evicts = any_evicts || ctx->layers[l].evicts;
+
+  int rc = dispatch_config(ctx->cfg.io_dtype, ctx->cfg.head_dim, ctx->G, [&](auto tt, auto dd, auto gg) -> int {
+    using TT = typename decltype(tt)::type;
+    constexpr int D = decltype(dd)::value, G = decltype(gg)::value;
+    for (int64_t c0 = 0; c0 < T; c0 += p.Cmax) {
+      p.c0 = c0;
+      p.C = int(std::min<int64_t>(p.Cmax, T - c0));
+      const int64_t warps = units * p.C;
+      const unsigned warp_blocks = unsigned((warps * 32 + kPrefillThreads - 1) / kPrefillThreads);
+      if (any_evicts) prefill_phi_kernel<TT, D><<<warp_blocks, kPrefillThreads, 0, stream>>>(p);
+      if (out) prefill_attn_kernel<TT, D, G><<<warp_blocks, kPrefillThreads, 0, stream>>>(p);
+      if (any_evicts) prefill_state_kernel<TT, D><<<unsigned(units * (D / 16)), kPrefillThreads, 0, stream>>>(p);
+      prefill_ring_kernel<TT, D><<<warp_blocks, kPrefillThreads, 0, stream>>>(p);
+      if (cudaGetLastError() != cudaSuccess) return GLIDE_ERR_CUDA;
+    }
+    return GLIDE_OK;
+  });
+  if (rc) return rc;
+  return launch_advance(ctx, layer_begin, layer_count, T, stream);
+}
+
+}  // namespace glide

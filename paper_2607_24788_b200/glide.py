@@ -1,0 +1,221 @@
+"""Thin ctypes binding of the GLIDE C ABI (include/glide.h): argument marshalling only.
+
+Every step of the path runs in the CUDA kernels of libglide.so.  torch is used for
+device memory and streams.  There is no fallback: if the library has not been built
+(python -m paper_2607_24788_b200.build) loading raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional, Sequence
+
+import torch
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_PKG, "libglide.so")
+
+GLIDE_F32, GLIDE_BF16 = 0, 1
+GLIDE_PHI_SOFTMAX = 0
+GLIDE_MERGE_SHARED = 0
+
+GLIDE_OK = 0
+GLIDE_ERR_INVALID_ARG = 1
+GLIDE_ERR_UNSUPPORTED = 2
+GLIDE_ERR_WORKSPACE_TOO_SMALL = 3
+GLIDE_ERR_CAPACITY = 4
+GLIDE_ERR_STATE = 5
+GLIDE_ERR_CUDA = 6
+
+
+class GlideError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        super().__init__(f"{where}: {strerror(code)} (status {code})")
+
+
+class glide_config(ctypes.Structure):
+    _fields_ = [
+        ("n_layers", ctypes.c_int32), ("batch", ctypes.c_int32), ("n_q_heads", ctypes.c_int32),
+        ("n_kv_heads", ctypes.c_int32), ("head_dim", ctypes.c_int32), ("io_dtype", ctypes.c_int32),
+        ("phi", ctypes.c_int32), ("merge", ctypes.c_int32),
+        ("windows", ctypes.POINTER(ctypes.c_int64)), ("q_to_kv", ctypes.POINTER(ctypes.c_int32)),
+        ("max_tokens", ctypes.c_int64), ("softmax_scale", ctypes.c_float), ("prefill_chunk", ctypes.c_int32),
+        ("decode_chunk", ctypes.c_int32), ("decode_state_splits", ctypes.c_int32),
+    ]
+
+
+class glide_layer_info_t(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_int64) for n in ("window", "capacity", "n", "count", "head_slot", "n_evicted")]
+
+
+_lib = None
+
+
+def load_library() -> ctypes.CDLL:
+    """dlopen libglide.so and declare the prototypes. Raises if the library is missing."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise RuntimeError(f"{LIB_PATH} not built: run `python -m paper_2607_24788_b200.build` "
+                           "(there is no CPU or PyTorch fallback for the GLIDE kernels)")
+    lib = ctypes.CDLL(LIB_PATH)
+    vp, i32, i64 = ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64
+    cfgp = ctypes.POINTER(glide_config)
+    lib.glide_workspace_bytes.argtypes = [cfgp, ctypes.POINTER(ctypes.c_size_t)]
+    lib.glide_create.argtypes = [cfgp, vp, ctypes.c_size_t, vp, ctypes.POINTER(vp)]
+    lib.glide_prefill.argtypes = [vp, i32, i32, i64, vp, vp, vp, vp, vp]
+    lib.glide_decode_step.argtypes = [vp, vp, vp, vp, vp, vp]
+    lib.glide_destroy.argtypes = [vp]
+    lib.glide_layer_info.argtypes = [vp, i32, vp, ctypes.POINTER(glide_layer_info_t)]
+    lib.glide_export_state.argtypes = [vp, i32, vp, vp, vp, vp, vp]
+    lib.glide_import_state.argtypes = [vp, i32, i64, vp, vp, vp, vp, vp]
+    lib.glide_reset.argtypes = [vp, vp]
+    lib.glide_device_status.argtypes = [vp, vp, ctypes.POINTER(i32)]
+    lib.glide_decode_launch_info.argtypes = [vp, ctypes.POINTER(i32), ctypes.POINTER(i32), ctypes.POINTER(i32)]
+    lib.glide_strerror.argtypes = [ctypes.c_int]
+    lib.glide_strerror.restype = ctypes.c_char_p
+    for name in ("glide_workspace_bytes", "glide_create", "glide_prefill", "glide_decode_step", "glide_destroy",
+                 "glide_layer_info", "glide_export_state", "glide_import_state", "glide_reset",
+                 "glide_device_status", "glide_decode_launch_info"):
+        getattr(lib, name).restype = ctypes.c_int
+    _lib = lib
+    return lib
+
+
+def strerror(code: int) -> str:
+    return load_library().glide_strerror(int(code)).decode()
+
+
+def _check(code: int, where: str):
+    if code != GLIDE_OK:
+        raise GlideError(code, where)
+
+
+def _ptr(t: Optional[torch.Tensor]) -> Optional[int]:
+    if t is None:
+        return None
+    assert t.is_cuda and t.is_contiguous(), "device buffers must be contiguous CUDA tensors"
+    return t.data_ptr()
+
+
+def _stream(stream: Optional[torch.cuda.Stream]) -> Optional[int]:
+    s = stream if stream is not None else torch.cuda.current_stream()
+    return s.cuda_stream or None
+
+
+def make_config(windows: Sequence[int], batch: int, n_q_heads: int, n_kv_heads: int, head_dim: int, max_tokens: int,
+                dtype: torch.dtype = torch.bfloat16, q_to_kv: Optional[Sequence[int]] = None,
+                softmax_scale: float = 0.0, prefill_chunk: int = 0, decode_chunk: int = 0,
+                decode_state_splits: int = 0):
+    """Returns (glide_config, keepalive) -- keepalive holds the host arrays the struct points to."""
+    win = (ctypes.c_int64 * len(windows))(*[int(w) for w in windows])
+    qmap = (ctypes.c_int32 * len(q_to_kv))(*[int(x) for x in q_to_kv]) if q_to_kv is not None else None
+    cfg = glide_config()
+    cfg.n_layers, cfg.batch, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim = len(windows), batch, n_q_heads, n_kv_heads, head_dim
+    cfg.io_dtype = {torch.float32: GLIDE_F32, torch.bfloat16: GLIDE_BF16}[dtype]
+    cfg.phi, cfg.merge = GLIDE_PHI_SOFTMAX, GLIDE_MERGE_SHARED
+    cfg.windows = ctypes.cast(win, ctypes.POINTER(ctypes.c_int64))
+    cfg.q_to_kv = ctypes.cast(qmap, ctypes.POINTER(ctypes.c_int32)) if qmap is not None else None
+    cfg.max_tokens = int(max_tokens)
+    cfg.softmax_scale = float(softmax_scale)
+    cfg.prefill_chunk, cfg.decode_chunk, cfg.decode_state_splits = int(prefill_chunk), int(decode_chunk), int(decode_state_splits)
+    return cfg, (win, qmap)
+
+
+def glide_workspace_bytes(cfg: glide_config) -> int:
+    out = ctypes.c_size_t(0)
+    _check(load_library().glide_workspace_bytes(ctypes.byref(cfg), ctypes.byref(out)), "glide_workspace_bytes")
+    return int(out.value)
+
+
+class Glide:
+    """Owns a torch workspace and a glide_ctx; methods carry the C ABI's names."""
+
+    def __init__(self, windows: Sequence[int], batch: int, n_q_heads: int, n_kv_heads: int, head_dim: int,
+                 max_tokens: int, dtype: torch.dtype = torch.bfloat16, device="cuda", **kw):
+        self.lib = load_library()
+        self.device = torch.device(device)
+        self.dtype = dtype
+        self.L, self.B, self.H, self.Hkv, self.d = len(windows), batch, n_q_heads, n_kv_heads, head_dim
+        self.windows = [int(w) for w in windows]
+        self.max_tokens = int(max_tokens)
+        self.cfg, self._keep = make_config(windows, batch, n_q_heads, n_kv_heads, head_dim, max_tokens, dtype, **kw)
+        self.workspace_bytes = glide_workspace_bytes(self.cfg)
+        with torch.cuda.device(self.device):
+            self.workspace = torch.empty(self.workspace_bytes + 256, dtype=torch.uint8, device=self.device)
+            base = self.workspace.data_ptr()
+            self._ws_ptr = (base + 255) // 256 * 256
+            handle = ctypes.c_void_p()
+            _check(self.lib.glide_create(ctypes.byref(self.cfg), self._ws_ptr, self.workspace_bytes, _stream(None),
+                                         ctypes.byref(handle)), "glide_create")
+        self._h = handle
+
+    # -- the four calls of the hot path ---------------------------------------------------------
+    def glide_prefill(self, q: Optional[torch.Tensor], k: torch.Tensor, v: torch.Tensor,
+                      out: Optional[torch.Tensor] = None, layer_begin: int = 0, layer_count: Optional[int] = None,
+                      stream=None) -> None:
+        lc = self.L - layer_begin if layer_count is None else layer_count
+        T = k.shape[2]
+        assert k.shape == (lc, self.B, T, self.Hkv, self.d) and v.shape == k.shape and k.dtype == self.dtype
+        if out is not None:
+            assert q is not None and q.shape == (lc, self.B, T, self.H, self.d) and out.shape == q.shape
+        _check(self.lib.glide_prefill(self._h, layer_begin, lc, T, _ptr(q), _ptr(k), _ptr(v), _ptr(out),
+                                      _stream(stream)), "glide_prefill")
+
+    def glide_decode_step(self, q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, out: torch.Tensor,
+                          stream=None) -> None:
+        assert q.shape == (self.L, self.B, self.H, self.d) and out.shape == q.shape
+        assert k.shape == (self.L, self.B, self.Hkv, self.d) and v.shape == k.shape
+        assert q.dtype == k.dtype == v.dtype == out.dtype == self.dtype
+        _check(self.lib.glide_decode_step(self._h, _ptr(q), _ptr(k), _ptr(v), _ptr(out), _stream(stream)),
+               "glide_decode_step")
+
+    def glide_destroy(self) -> None:
+        if getattr(self, "_h", None):
+            self.lib.glide_destroy(self._h)
+            self._h = None
+
+    def __del__(self):
+        try:
+            self.glide_destroy()
+        except Exception:
+            pass
+
+    # -- support ----------------------------------------------------------------------------------
+    def glide_layer_info(self, layer: int) -> dict:
+        info = glide_layer_info_t()
+        _check(self.lib.glide_layer_info(self._h, layer, _stream(None), ctypes.byref(info)), "glide_layer_info")
+        return {n: int(getattr(info, n)) for n, _ in glide_layer_info_t._fields_}
+
+    def capacity(self, layer: int) -> int:
+        return min(self.windows[layer], self.max_tokens)
+
+    def glide_export_state(self, layer: int):
+        cap = self.capacity(layer)
+        rk = torch.empty((self.B, self.Hkv, cap, self.d), dtype=self.dtype, device=self.device)
+        rv = torch.empty_like(rk)
+        S = torch.empty((self.B, self.Hkv, self.d, self.d), dtype=torch.float32, device=self.device)
+        z = torch.empty((self.B, self.Hkv, self.d), dtype=torch.float32, device=self.device)
+        _check(self.lib.glide_export_state(self._h, layer, _ptr(rk) if cap else None, _ptr(rv) if cap else None,
+                                           _ptr(S), _ptr(z), _stream(None)), "glide_export_state")
+        return rk, rv, S, z
+
+    def glide_import_state(self, layer: int, n: int, ringK=None, ringV=None, S=None, z=None) -> None:
+        _check(self.lib.glide_import_state(self._h, layer, int(n), _ptr(ringK), _ptr(ringV), _ptr(S), _ptr(z),
+                                           _stream(None)), "glide_import_state")
+
+    def glide_reset(self) -> None:
+        _check(self.lib.glide_reset(self._h, _stream(None)), "glide_reset")
+
+    def glide_device_status(self) -> int:
+        out = ctypes.c_int32(0)
+        _check(self.lib.glide_device_status(self._h, _stream(None), ctypes.byref(out)), "glide_device_status")
+        return int(out.value)
+
+    def glide_decode_launch_info(self) -> dict:
+        a, b, c = ctypes.c_int32(0), ctypes.c_int32(0), ctypes.c_int32(0)
+        _check(self.lib.glide_decode_launch_info(self._h, ctypes.byref(a), ctypes.byref(b), ctypes.byref(c)),
+               "glide_decode_launch_info")
+        return dict(launches=a.value, work_items=b.value, grid=c.value)

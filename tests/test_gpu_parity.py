@@ -1,0 +1,97 @@
+"""GPU parity: the CUDA path through the C ABI vs the CPU oracle, element by element, same seeded inputs."""
+import pytest
+import torch
+
+from paper_2607_24788_b200 import configs as C
+from tests.parity_util import run_case
+
+pytestmark = pytest.mark.gpu
+
+F32, BF16 = torch.float32, torch.bfloat16
+
+
+def test_config0_tiny_fp32():
+    c = C.C0
+    run_case(c.windows, c.batch, c.n_q_heads, c.n_kv_heads, c.head_dim, F32, [c.context], c.decode_steps, amp=1.0)
+
+
+@pytest.mark.parametrize("w", [0, 1, 2, 3, 15, 16, 17, 63, 64, 65])
+def test_window_edge_sizes_decode_only(w):
+    # every token goes through decode: T crosses w, ring wraps several times
+    run_case([w], 1, 4, 4, 64, F32, [], 150, amp=1.0, seed=w)
+
+
+@pytest.mark.parametrize("w", [0, 1, 3, 16, 17, 64, 65, 300])
+@pytest.mark.parametrize("calls", [(97,), (16, 16, 65), (1, 50, 3, 43)])
+def test_prefill_then_decode_fp32(w, calls):
+    run_case([w], 2, 4, 2, 64, F32, list(calls), 12, amp=1.0, seed=w + len(calls), prefill_chunk=32)
+
+
+@pytest.mark.parametrize("G,Hkv", [(1, 2), (2, 2), (4, 2), (8, 1)])
+@pytest.mark.parametrize("d", [64, 128])
+@pytest.mark.parametrize("dtype", [F32, BF16])
+def test_group_sizes_and_head_dims(G, Hkv, d, dtype):
+    amp = 1.0 if dtype == F32 else 0.5
+    run_case([0, 5, 40, 1000], 2, G * Hkv, Hkv, d, dtype, [70], 20, amp=amp, prefill_chunk=32, decode_chunk=16)
+
+
+def test_large_logits_exercise_rescaling():
+    # q,k x3: window logits with std ~ 9/sqrt(64)*8 -> running-max rescaling and m* = max(m, 0) matter
+    run_case([7, 48], 1, 4, 2, 64, F32, [60], 40, amp=3.0, prefill_chunk=16, decode_chunk=8)
+
+
+def test_non_contiguous_head_map():
+    run_case([6, 20], 1, 4, 2, 64, F32, [30], 10, q_to_kv=[1, 0, 0, 1], prefill_chunk=16)
+
+
+def test_multi_layer_split_k_bf16():
+    # several split-K items per unit, ragged last item, several state row blocks
+    run_case([300, 129, 64, 0], 2, 8, 2, 128, BF16, [400], 40, amp=128 ** -0.5 * 4, decode_chunk=64,
+             decode_state_splits=4)
+
+
+def test_never_evicting_layer_is_full_softmax():
+    run_case([1 << 20, 50], 1, 4, 4, 64, F32, [100], 30, max_tokens=130)
+
+
+def test_layer_ranges_prefilled_separately():
+    import numpy as np
+    from oracle import glide_oracle as orc
+    from paper_2607_24788_b200 import glide, synth
+    from tests.parity_util import check_outputs, check_state, f32_scale, to_np
+    windows, B, H, Hkv, d, T = [5, 40, 12], 1, 4, 2, 64, 50
+    wl = synth.Workload(3, 3, B, H, Hkv, d, F32, 1.0)
+    g = glide.Glide(windows, B, H, Hkv, d, 64, dtype=F32, softmax_scale=f32_scale(d), prefill_chunk=16)
+    stack = orc.Stack(windows, B, H, Hkv, d, f32_scale(d))
+    for lb, lc in ((1, 2), (0, 1)):
+        q, k, v = wl.qkv(range(lb, lb + lc), range(B), range(T), device="cuda")
+        out = torch.empty_like(q)
+        g.glide_prefill(q, k, v, out, layer_begin=lb, layer_count=lc)
+        ref = stack.prefill(to_np(q), to_np(k), to_np(v), layer_begin=lb)
+        check_outputs(out, ref, F32, f"layers {lb}..{lb+lc}")
+    check_state(g, stack)
+    q, k, v = wl.decode_qkv(T, device="cuda")
+    out = torch.empty_like(q)
+    g.glide_decode_step(q, k, v, out)
+    check_outputs(out, stack.decode(to_np(q), to_np(k), to_np(v)), F32, "decode")
+
+
+def test_errors_and_capacity():
+    from paper_2607_24788_b200 import glide
+    g = glide.Glide([4, 4], 1, 2, 2, 64, 8, dtype=F32)
+    q = torch.zeros((2, 1, 2, 64), device="cuda")
+    kv = torch.zeros((2, 1, 2, 64), device="cuda")
+    k1 = torch.zeros((1, 1, 3, 2, 64), device="cuda")
+    g.glide_prefill(None, k1, k1, None, layer_begin=0, layer_count=1)
+    with pytest.raises(glide.GlideError) as e:       # layers at different positions
+        g.glide_decode_step(q, kv, kv, torch.empty_like(q))
+    assert e.value.code == glide.GLIDE_ERR_STATE
+    g.glide_prefill(None, k1, k1, None, layer_begin=1, layer_count=1)
+    for _ in range(5):
+        g.glide_decode_step(q, kv, kv, torch.empty_like(q))
+    with pytest.raises(glide.GlideError) as e:       # 8 tokens absorbed: full
+        g.glide_decode_step(q, kv, kv, torch.empty_like(q))
+    assert e.value.code == glide.GLIDE_ERR_CAPACITY
+    assert g.glide_layer_info(0)["n"] == 8
+    g.glide_reset()
+    assert g.glide_layer_info(1) == dict(window=4, capacity=4, n=0, count=0, head_slot=0, n_evicted=0)
