@@ -1,0 +1,380 @@
+#!/usr/bin/env python
+"""Benchmark of the GLIDE hybrid-attention decode step on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl glide|reference]
+
+A step is one glide_decode_step: one token for every layer and sequence of the workload, the
+fused launch covering ring append/eviction, phi, state fold, window attention, linear readout
+and the shared-normaliser merge.  The state the steps start from is built (untimed) by
+glide_prefill over the synthetic prompt.  Default workload: Llama-3-8B-shaped stack, batch 1,
+32K context (configs.C1).  Prints ONE JSON line.
+
+Timing: CUDA events on the launching stream around exactly K steps, repeated a few times while
+NVML samples the clocks; the median repetition is reported.  Consecutive steps rotate over
+several independent copies of the sequence state (total footprint well above the 126 MB L2), so
+no step finds its window or state in L2 from the step before.
+
+N > 1 (torchrun): the path does not shard -- every rank runs an independent replica of the
+workload on its own GPU, no collective on the data path; value = tokens of all ranks / max time.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import math
+import os
+import statistics
+import sys
+import threading
+import time
+
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2607_24788_b200 import configs, synth  # noqa: E402
+
+L2_BYTES = 126e6
+# dram__bytes_read.sum + dram__bytes_write.sum per decode launch from the committed ncu capture
+# (profiles/), keyed by workload name; None until a capture exists for that workload.
+NCU_TRAFFIC_BYTES = {}
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons through NVML (read-only) while the timed region runs."""
+
+    def __init__(self, index: int):
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop = threading.Event()
+        self._thread = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM))
+        except Exception:
+            self.nv = None
+
+    def _run(self):
+        nv = self.nv
+        names = {
+            "hw_slowdown": getattr(nv, "nvmlClocksEventReasonHwSlowdown", 0x8),
+            "hw_thermal_slowdown": getattr(nv, "nvmlClocksEventReasonHwThermalSlowdown", 0x40),
+            "sw_thermal_slowdown": getattr(nv, "nvmlClocksEventReasonSwThermalSlowdown", 0x20),
+            "sw_power_cap": getattr(nv, "nvmlClocksEventReasonSwPowerCap", 0x4),
+        }
+        while not self._stop.is_set():
+            try:
+                self.samples.append(int(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM)))
+                try:
+                    mask = int(nv.nvmlDeviceGetCurrentClocksEventReasons(self.h))
+                except Exception:
+                    mask = int(nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h))
+                for name, bit in names.items():
+                    if mask & bit:
+                        self.reasons.add(name)
+            except Exception:
+                pass
+            time.sleep(0.01)
+
+    def __enter__(self):
+        if self.nv is not None:
+            self._thread = threading.Thread(target=self._run, daemon=True)
+            self._thread.start()
+        return self
+
+    def __exit__(self, *exc):
+        self._stop.set()
+        if self._thread is not None:
+            self._thread.join()
+
+    def summary(self):
+        return {"sm_mhz": statistics.median(self.samples) if self.samples else None, "sm_max_mhz": self.max_mhz,
+                "reasons": sorted(self.reasons), "samples": len(self.samples)}
+
+
+def torch_dtype(shape):
+    return torch.float32 if shape.dtype == "f32" else torch.bfloat16
+
+
+def value_scale(shape):
+    return synth.default_value_scale(shape.head_dim, shape.unit_variance)
+
+
+# ---------------------------------------------------------------------------------------------
+# CPU oracle leg (cpu_baseline and --impl reference)
+# ---------------------------------------------------------------------------------------------
+def oracle_decode_rate(shape, steps: int, warmup: int):
+    """Times the oracle's decode step on the host cores on a bounded sample of the workload: one layer of
+    every distinct window size, sequence 0, state built by the oracle's own prefill of the full prompt.
+    Per-layer-class times are scaled by the number of layers and sequences of each class."""
+    from oracle import glide_oracle as orc
+    import numpy as np
+    dt = torch_dtype(shape)
+    wl = synth.Workload(shape.seed, shape.n_layers, shape.batch, shape.n_q_heads, shape.n_kv_heads, shape.head_dim, dt,
+                        value_scale(shape))
+    scale = float(np.float32(1.0) / np.sqrt(np.float32(shape.head_dim)))
+    classes = {}
+    for l, w in enumerate(shape.windows):
+        classes.setdefault(w, []).append(l)
+    per_class_s = {}
+    threads = orc.max_threads()
+    used = 1
+    for w, layers in classes.items():
+        l = layers[0]
+        stack = orc.Stack([w], 1, shape.n_q_heads, shape.n_kv_heads, shape.head_dim, scale)
+        # only the tokens that can still matter are absorbed one piece at a time
+        piece = 2048
+        for pos in range(0, shape.context, piece):
+            k, v = wl.kv([l], [0], range(pos, min(pos + piece, shape.context)))
+            stack.prefill(None, k.double().numpy(), v.double().numpy(), outputs=False)
+        times = []
+        for s in range(warmup + steps):
+            q, k, v = wl.qkv([l], [0], [shape.context + s])
+            q, k, v = (x[:, :, 0].double().numpy() for x in (q, k, v))
+            t0 = time.perf_counter()
+            stack.decode(q, k, v, threads=threads)
+            t1 = time.perf_counter()
+            used = max(used, stack.threads_used)
+            if s >= warmup:
+                times.append(t1 - t0)
+        per_class_s[w] = statistics.median(times)
+    step_s = sum(per_class_s[w] * len(layers) for w, layers in classes.items()) * shape.batch
+    sample = (f"layers {sorted(v[0] for v in classes.values())} (one per distinct window), sequence 0, "
+              f"{steps} decode steps each after the oracle's own {shape.context}-token prefill; "
+              f"per-class median step time x layers of the class x batch")
+    return shape.batch / step_s, step_s, used, sample
+
+
+def run_reference(args, shape):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    steps = min(args.steps, 16)
+    tok_s, step_s, cores, sample = oracle_decode_rate(shape, steps, min(args.warmup, 2))
+    line = {
+        "impl": "reference", "metric": "hybrid-attn decode tokens/s", "value": tok_s, "unit": "tokens/s",
+        "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup, "ms_per_step": step_s * 1e3,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": shape.name, "batch": shape.batch, "context": shape.context,
+                   "sum_windows": sum(shape.windows), "timed_oracle_steps_per_layer_class": steps},
+        "cpu_baseline": {"value": tok_s, "unit": "tokens/s", "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": tok_s, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+# ---------------------------------------------------------------------------------------------
+# GPU leg
+# ---------------------------------------------------------------------------------------------
+def build_states(shape, n_replicas: int, extra_tokens: int, device):
+    from paper_2607_24788_b200 import glide
+    dt = torch_dtype(shape)
+    wl = synth.Workload(shape.seed, shape.n_layers, shape.batch, shape.n_q_heads, shape.n_kv_heads, shape.head_dim, dt,
+                        value_scale(shape))
+    max_tokens = shape.context + extra_tokens
+    ctxs = [glide.Glide(shape.windows, shape.batch, shape.n_q_heads, shape.n_kv_heads, shape.head_dim, max_tokens,
+                        dtype=dt, device=device, prefill_chunk=shape.prefill_chunk) for _ in range(n_replicas)]
+    g0 = ctxs[0]
+    # prompt -> state (no outputs needed for a decode benchmark); layers in groups to bound the k/v buffers
+    budget_elems = 256 << 20
+    per_token_layer = shape.batch * shape.n_kv_heads * shape.head_dim
+    piece = 4096
+    lgroup = max(1, min(shape.n_layers, budget_elems // (piece * per_token_layer)))
+    for lb in range(0, shape.n_layers, lgroup):
+        lc = min(lgroup, shape.n_layers - lb)
+        for pos in range(0, shape.context, piece):
+            k, v = wl.kv(range(lb, lb + lc), range(shape.batch), range(pos, min(pos + piece, shape.context)), device)
+            g0.glide_prefill(None, k, v, None, layer_begin=lb, layer_count=lc)
+            del k, v
+    torch.cuda.synchronize()
+    for g in ctxs[1:]:
+        for l in range(shape.n_layers):
+            rk, rv, S, z = g0.glide_export_state(l)
+            cap = g0.capacity(l)
+            g.glide_import_state(l, shape.context, rk if cap else None, rv if cap else None, S, z)
+        torch.cuda.synchronize()
+    return ctxs, wl
+
+
+def run_glide(args, shape):
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device: the GLIDE path has no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    device = torch.device("cuda", local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=device)
+
+    K, W = args.steps, args.warmup
+    step_bytes = configs.decode_step_bytes(shape, shape.context)
+    n_rep = max(1, min(16, math.ceil(8 * L2_BYTES / step_bytes)))
+    reps = args.reps
+    extra = math.ceil((max(W, 3) + reps * K + 3 + 3 * K) / n_rep) + 3 * K + 16
+    ctxs, wl = build_states(shape, n_rep, extra, device)
+    L, B, H, Hkv, d = shape.n_layers, shape.batch, shape.n_q_heads, shape.n_kv_heads, shape.head_dim
+    dt = torch_dtype(shape)
+
+    # inputs of the timed steps, resident in HBM: one buffer per step holding q | k | v
+    n_in = min(K, 64)
+    nq, nk = L * B * H * d, L * B * Hkv * d
+    dev_in = torch.empty((n_in, nq + 2 * nk), dtype=dt, device=device)
+    for i in range(n_in):
+        q, k, v = wl.decode_qkv(shape.context + i, device)
+        dev_in[i, :nq] = q.reshape(-1)
+        dev_in[i, nq:nq + nk] = k.reshape(-1)
+        dev_in[i, nq + nk:] = v.reshape(-1)
+    outs = [torch.empty((L, B, H, d), dtype=dt, device=device) for _ in range(2)]
+
+    def views(buf):
+        return (buf[:nq].view(L, B, H, d), buf[nq:nq + nk].view(L, B, Hkv, d), buf[nq + nk:].view(L, B, Hkv, d))
+
+    step_no = [0]
+
+    def one_step(buf):
+        i = step_no[0]
+        step_no[0] += 1
+        q, k, v = views(buf)
+        ctxs[i % n_rep].glide_decode_step(q, k, v, outs[i & 1])
+
+    def barrier():
+        torch.cuda.synchronize()
+        if dist is not None:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    for i in range(max(W, 3)):
+        one_step(dev_in[i % n_in])
+    barrier()
+
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    times_ms = []
+    with ClockSampler(local_rank) as clocks:
+        for _ in range(reps):
+            barrier()
+            ev0.record()
+            for i in range(K):
+                one_step(dev_in[i % n_in])
+            ev1.record()
+            barrier()
+            times_ms.append(ev0.elapsed_time(ev1))
+    t_ms = statistics.median(times_ms)
+
+    # same context every step: window and state of the previous step may still sit in L2
+    hot_ms = []
+    for _ in range(3):
+        barrier()
+        ev0.record()
+        for i in range(K):
+            q, k, v = views(dev_in[i % n_in])
+            ctxs[0].glide_decode_step(q, k, v, outs[i & 1])
+        ev1.record()
+        barrier()
+        hot_ms.append(ev0.elapsed_time(ev1))
+    hot_ms = statistics.median(hot_ms)
+
+    # end to end through the public call with HOST buffers: pinned q|k|v -> device, step, out -> pinned host
+    host_in = torch.empty((n_in, nq + 2 * nk), dtype=dt).pin_memory()
+    host_in.copy_(dev_in.cpu())
+    host_out = torch.empty((L, B, H, d), dtype=dt).pin_memory()
+    stage = torch.empty((nq + 2 * nk,), dtype=dt, device=device)
+    e2e_steps = K
+
+    def e2e_step(i):
+        stage.copy_(host_in[i % n_in], non_blocking=True)
+        one_step(stage)
+        host_out.copy_(outs[(step_no[0] - 1) & 1], non_blocking=True)
+        torch.cuda.current_stream().synchronize()   # the next token depends on this result
+
+    for i in range(3):
+        e2e_step(i)
+    e2e_ms = []
+    for _ in range(3):
+        barrier()
+        ev0.record()
+        for i in range(e2e_steps):
+            e2e_step(i)
+        ev1.record()
+        barrier()
+        e2e_ms.append(ev0.elapsed_time(ev1))
+    e2e_t = statistics.median(e2e_ms)
+
+    if dist is not None:
+        t = torch.tensor([t_ms, hot_ms, e2e_t], dtype=torch.float64, device=device)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        t_ms, hot_ms, e2e_t = (float(x) for x in t.cpu())
+
+    if rank == 0:
+        peak, peak_kind = load_peaks()
+        launch_s = t_ms * 1e-3 / K
+        achieved = step_bytes / launch_s / 1e9
+        info = ctxs[0].glide_decode_launch_info()
+        elem = shape.elem_bytes
+        line = {
+            "metric": "hybrid-attn decode tokens/s", "value": world * B * K / (t_ms * 1e-3), "unit": "tokens/s",
+            "n_gpus": world, "steps": K, "warmup": max(W, 3), "ms_per_step": t_ms / K, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f32" if shape.dtype == "f32" else "bf16+f32state",
+            "data": "synthetic",
+            "config": {"workload": shape.name, "batch": B, "context": shape.context, "n_layers": L,
+                       "sum_windows": sum(shape.windows), "q_heads": H, "kv_heads": Hkv, "head_dim": d,
+                       "l2": f"steps rotate over {n_rep} independent state copies ({n_rep * step_bytes / 1e6:.0f} MB per "
+                             f"rotation > 126 MB L2); median of {reps} repetitions of K steps",
+                       "multi_gpu": "replicas only"},
+            "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                         "traffic": NCU_TRAFFIC_BYTES.get(shape.name), "peak_kind": f"of {peak_kind}",
+                         "kernel": "glide_decode_kernel", "algorithmic_bytes_per_launch": step_bytes,
+                         "frac_of_nominal_8TBps": achieved / 8000.0},
+            "per_step_attention_latency_us": launch_s * 1e6,
+            "hot_l2": {"tokens_per_s": world * B * K / (hot_ms * 1e-3), "us_per_step": hot_ms * 1e3 / K,
+                       "note": "same sequence state every step (L2 may hold part of it)"},
+            "e2e": {"value": world * B * e2e_steps / (e2e_t * 1e-3), "unit": "tokens/s",
+                    "h2d_bytes_per_step": (nq + 2 * nk) * elem, "d2h_bytes_per_step": nq * elem,
+                    "us_per_step": e2e_t * 1e3 / e2e_steps},
+            "gpu_launches": K * info["launches"],
+            "decode_launch": info,
+            "clocks": clocks.summary(),
+        }
+        if world == 1 and not args.no_cpu_baseline:
+            tok_s, step_s, cores, sample = oracle_decode_rate(shape, 4, 1)
+            line["cpu_baseline"] = {"value": tok_s, "unit": "tokens/s", "cores": cores, "kind": "oracle",
+                                    "sample": sample, "ms_per_step": step_s * 1e3}
+        print(json.dumps(line))
+    if dist is not None:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=256)
+    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--reps", type=int, default=15, help="repetitions of the K-step timed region (median reported)")
+    ap.add_argument("--workload", default=configs.C1.name, choices=sorted(configs.ALL))
+    ap.add_argument("--impl", default="glide", choices=["glide", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    shape = configs.ALL[args.workload]
+    if args.impl == "reference":
+        run_reference(args, shape)
+    else:
+        run_glide(args, shape)
+
+
+if __name__ == "__main__":
+    main()
