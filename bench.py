@@ -39,6 +39,7 @@ L2_BYTES = 126e6
 # dram__bytes_read.sum + dram__bytes_write.sum per decode launch from the committed ncu capture
 # (profiles/), keyed by workload name; None until a capture exists for that workload.
 NCU_TRAFFIC_BYTES = {}
+KERNEL_KNOBS = {}   # tuning overrides from the command line (decode_chunk, decode_state_splits, decode_impl)
 
 
 def load_peaks():
@@ -185,7 +186,8 @@ def build_states(shape, n_replicas: int, extra_tokens: int, device):
                         value_scale(shape))
     max_tokens = shape.context + extra_tokens
     ctxs = [glide.Glide(shape.windows, shape.batch, shape.n_q_heads, shape.n_kv_heads, shape.head_dim, max_tokens,
-                        dtype=dt, device=device, prefill_chunk=shape.prefill_chunk) for _ in range(n_replicas)]
+                        dtype=dt, device=device, prefill_chunk=shape.prefill_chunk, **KERNEL_KNOBS)
+             for _ in range(n_replicas)]
     g0 = ctxs[0]
     # prompt -> state (no outputs needed for a decode benchmark); layers in groups to bound the k/v buffers
     budget_elems = 256 << 20
@@ -368,8 +370,13 @@ def main():
     ap.add_argument("--workload", default=configs.C1.name, choices=sorted(configs.ALL))
     ap.add_argument("--impl", default="glide", choices=["glide", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--decode-chunk", type=int, default=0, help="window slots per split-K work item (0: library default)")
+    ap.add_argument("--state-splits", type=int, default=0, help="row blocks per state update (0: library default)")
+    ap.add_argument("--decode-impl", type=int, default=0, help="0 auto, 1 tensor-core/TMA kernel, 2 CUDA-core kernel")
     args = ap.parse_args()
     shape = configs.ALL[args.workload]
+    KERNEL_KNOBS.update(decode_chunk=args.decode_chunk, decode_state_splits=args.state_splits,
+                        decode_impl=args.decode_impl)
     if args.impl == "reference":
         run_reference(args, shape)
     else:

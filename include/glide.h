@@ -60,6 +60,9 @@ typedef enum { GLIDE_PHI_SOFTMAX = 0 } glide_phi;
  * "Retention-based SWA").  GLIDE_MERGE_SHARED is the shared normaliser above. */
 typedef enum { GLIDE_MERGE_SHARED = 0 } glide_merge;
 
+/* Decode kernel selection.  AUTO: tensor-core/TMA kernel for bf16 I/O, CUDA-core fp32 kernel for fp32 I/O. */
+typedef enum { GLIDE_DECODE_AUTO = 0, GLIDE_DECODE_MMA = 1, GLIDE_DECODE_FMA = 2 } glide_decode_impl;
+
 typedef struct {
   int32_t n_layers;        /* L >= 1 */
   int32_t batch;           /* B >= 1 independent sequences of equal length */
@@ -78,6 +81,7 @@ typedef struct {
   int32_t prefill_chunk;   /* tokens per chunk of the chunked linear scan; 0 selects 256; multiple of 16, <= 1024 */
   int32_t decode_chunk;    /* window slots per split-K work item of the decode kernel; 0 selects automatically */
   int32_t decode_state_splits; /* row blocks the S update/readout of one KV head is split into; 0 selects automatically */
+  int32_t decode_impl;     /* glide_decode_impl */
 } glide_config;
 
 typedef struct {

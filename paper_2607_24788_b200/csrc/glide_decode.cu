@@ -357,7 +357,9 @@ __global__ void glide_advance_kernel(int64_t *n_dev, int layer_begin, int layer_
   if (i < layer_count) n_dev[layer_begin + i] += T;
 }
 
-DecodeParams make_params(const glide_ctx *ctx, const void *q, const void *k, const void *v, void *out) {
+}  // namespace
+
+DecodeParams make_decode_params(const glide_ctx *ctx, const void *q, const void *k, const void *v, void *out) {
   DecodeParams p{};
   p.ws = ctx->ws;
   p.layers = reinterpret_cast<const LayerDev *>(ctx->ws + ctx->off_layers);
@@ -381,8 +383,6 @@ DecodeParams make_params(const glide_ctx *ctx, const void *q, const void *k, con
   return p;
 }
 
-}  // namespace
-
 int decode_occupancy(const glide_ctx *ctx, int *blocks_per_sm) {
   return dispatch_config(ctx->cfg.io_dtype, ctx->cfg.head_dim, ctx->G, [&](auto tt, auto dd, auto gg) -> int {
     using T = typename decltype(tt)::type;
@@ -397,7 +397,8 @@ int decode_occupancy(const glide_ctx *ctx, int *blocks_per_sm) {
 }
 
 int launch_decode(glide_ctx *ctx, const void *q, const void *k, const void *v, void *out, cudaStream_t stream) {
-  const DecodeParams p = make_params(ctx, q, k, v, out);
+  const DecodeParams p = make_decode_params(ctx, q, k, v, out);
+  if (ctx->use_mma) return launch_decode_mma(ctx, p, stream);
   return dispatch_config(ctx->cfg.io_dtype, ctx->cfg.head_dim, ctx->G, [&](auto tt, auto dd, auto gg) -> int {
     using T = typename decltype(tt)::type;
     constexpr int D = decltype(dd)::value, G = decltype(gg)::value;

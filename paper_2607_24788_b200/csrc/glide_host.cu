@@ -25,6 +25,8 @@ int validate_config(const glide_config *c) {
   if (c->softmax_scale < 0.f || !std::isfinite(c->softmax_scale)) return GLIDE_ERR_INVALID_ARG;
   if (c->prefill_chunk < 0 || c->decode_chunk < 0 || c->decode_state_splits < 0) return GLIDE_ERR_INVALID_ARG;
   if (c->prefill_chunk % 16 != 0 || c->prefill_chunk > 1024) return GLIDE_ERR_INVALID_ARG;
+  if (c->decode_impl < GLIDE_DECODE_AUTO || c->decode_impl > GLIDE_DECODE_FMA) return GLIDE_ERR_INVALID_ARG;
+  if (c->decode_impl == GLIDE_DECODE_MMA && c->io_dtype != GLIDE_BF16) return GLIDE_ERR_UNSUPPORTED;
   for (int l = 0; l < c->n_layers; ++l)
     if (c->windows[l] < 0) return GLIDE_ERR_INVALID_ARG;
   if (c->phi != GLIDE_PHI_SOFTMAX || c->merge != GLIDE_MERGE_SHARED) return GLIDE_ERR_UNSUPPORTED;
@@ -74,7 +76,9 @@ int glide::plan_context(const glide_config *cfg, glide_ctx *ctx, std::vector<Wor
   ctx->n_host.assign(L, 0);
   ctx->rec_floats = int(align_up(size_t(ctx->G) * (d + 2), 4));
 
-  const int chunk = cfg->decode_chunk ? cfg->decode_chunk : 128;
+  // window slots per split-K item: fixed by the caller, or 128 (512 for very long windows, to bound the
+  // number of partials one merge has to read)
+  auto chunk_of = [&](int64_t cap) -> int { return cfg->decode_chunk ? cfg->decode_chunk : (cap > 8192 ? 512 : 128); };
   const int splits = cfg->decode_state_splits ? std::min<int>(cfg->decode_state_splits, d) : (d == 128 ? 4 : 2);
   const int64_t units_per_layer = int64_t(B) * Hkv;
 
@@ -86,6 +90,7 @@ int glide::plan_context(const glide_config *cfg, glide_ctx *ctx, std::vector<Wor
     ld.w = ctx->windows[l];
     ld.cap = std::min<int64_t>(ld.w, cfg->max_tokens);
     ld.evicts = ld.w < cfg->max_tokens ? 1 : 0;
+    const int chunk = chunk_of(ld.cap);
     ld.n_win_items = int((ld.cap + chunk - 1) / chunk);
     ld.n_state_items = ld.evicts ? splits : 0;
     ld.part_base = part_floats;
@@ -112,6 +117,8 @@ int glide::plan_context(const glide_config *cfg, glide_ctx *ctx, std::vector<Wor
   off = align_up(off + sizeof(int32_t) * size_t(L) * units_per_layer, 256);
   ctx->off_partials = off;
   off = align_up(off + sizeof(float) * part_floats, 256);
+  ctx->off_tmaps = off;
+  off = align_up(off + size_t(128) * 2 * L, 256);
   ctx->off_phik = off;
   off = align_up(off + sizeof(float) * size_t(L) * units_per_layer * ctx->prefill_chunk * d, 256);
   ctx->off_state = off;
@@ -140,6 +147,7 @@ int glide::plan_context(const glide_config *cfg, glide_ctx *ctx, std::vector<Wor
     items->reserve(size_t(n_items));
     for (int l = 0; l < L; ++l) {
       const LayerDev &ld = ctx->layers[l];
+      const int chunk = chunk_of(ld.cap);
       for (int64_t u = 0; u < units_per_layer; ++u) {
         int unit = int(int64_t(l) * units_per_layer + u);
         int part = 0;
@@ -214,11 +222,19 @@ int glide_create(const glide_config *cfg, void *dev_workspace, size_t workspace_
   bool ok = cudaGetDevice(&ctx->device) == cudaSuccess &&
             cudaDeviceGetAttribute(&ctx->sm_count, cudaDevAttrMultiProcessorCount, ctx->device) == cudaSuccess;
   int per_sm = 0;
-  ok = ok && decode_occupancy(ctx, &per_sm) == GLIDE_OK && per_sm > 0;
+  ctx->use_mma = cfg->io_dtype == GLIDE_BF16 && cfg->decode_impl != GLIDE_DECODE_FMA;
+  if (ctx->use_mma) {
+    ok = ok && mma_decode_setup(ctx) == GLIDE_OK;
+  } else {
+    ok = ok && decode_occupancy(ctx, &per_sm) == GLIDE_OK && per_sm > 0;
+    if (ok) ctx->decode_grid = std::max(1, std::min(ctx->n_items, ctx->sm_count * per_sm));
+  }
   if (ok) {
-    ctx->decode_grid = std::max(1, std::min(ctx->n_items, ctx->sm_count * per_sm));
+    if (ctx->use_mma)
+      ok = cudaMemcpyAsync(ctx->ws + ctx->off_tmaps, ctx->tmaps_host.data(), ctx->tmaps_host.size(),
+                           cudaMemcpyHostToDevice, st) == cudaSuccess;
     // control words, counters, tickets, S and z start at zero
-    ok = cudaMemsetAsync(ctx->ws, 0, ctx->off_layers, st) == cudaSuccess &&
+    ok = ok && cudaMemsetAsync(ctx->ws, 0, ctx->off_layers, st) == cudaSuccess &&
          cudaMemsetAsync(ctx->ws + ctx->off_tickets, 0, ctx->off_partials - ctx->off_tickets, st) == cudaSuccess &&
          cudaMemsetAsync(ctx->ws + ctx->off_state, 0, ctx->state_bytes, st) == cudaSuccess;
     ok = ok && cudaMemcpyAsync(ctx->ws + ctx->off_layers, ctx->layers.data(), sizeof(LayerDev) * ctx->layers.size(),

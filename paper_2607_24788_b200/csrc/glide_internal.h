@@ -42,7 +42,7 @@ struct WorkItem {
 enum : int { kItemWindow = 0, kItemState = 1 };
 
 // Device status codes (glide_device_status).
-enum : int { kDevOk = 0, kDevBadSlot = 1, kDevBadItem = 2 };
+enum : int { kDevOk = 0, kDevBadSlot = 1, kDevBadItem = 2, kDevWaitTimeout = 3 };
 
 // Control words at the start of the workspace.
 struct Control {
@@ -96,6 +96,8 @@ struct glide_ctx {
   std::vector<int32_t> heads_of;    // [Hkv][G]
   std::vector<glide::LayerDev> layers;
   std::vector<int64_t> n_host;      // mirror of the device counters
+  std::vector<unsigned char> tmaps_host;  // TMA descriptors of the rings (bf16 tensor-core decode kernel)
+  bool use_mma = false;             // bf16: tensor-core decode kernel; fp32: CUDA-core kernel
   int G = 0;
   int device = 0;
   int sm_count = 0;
@@ -109,7 +111,7 @@ struct glide_ctx {
   size_t ws_bytes = 0;
   // workspace regions (byte offsets)
   size_t off_ctl = 0, off_ndev = 0, off_layers = 0, off_heads = 0, off_items = 0, off_tickets = 0,
-         off_partials = 0, off_phik = 0, off_state = 0, off_ring = 0, total = 0;
+         off_partials = 0, off_tmaps = 0, off_phik = 0, off_state = 0, off_ring = 0, total = 0;
   size_t state_bytes = 0;           // S and z of all layers (contiguous)
 };
 
@@ -118,6 +120,9 @@ namespace glide {
 // Layout planning shared by glide_workspace_bytes and glide_create (host only).
 int plan_context(const glide_config *cfg, glide_ctx *ctx, std::vector<WorkItem> *items);
 
+DecodeParams make_decode_params(const glide_ctx *ctx, const void *q, const void *k, const void *v, void *out);
+int mma_decode_setup(glide_ctx *ctx);   // builds the ring tensor maps (host copy) and sizes the grid
+int launch_decode_mma(glide_ctx *ctx, const DecodeParams &p, cudaStream_t stream);
 int launch_decode(glide_ctx *ctx, const void *q, const void *k, const void *v, void *out, cudaStream_t stream);
 int decode_occupancy(const glide_ctx *ctx, int *blocks_per_sm);
 int launch_prefill(glide_ctx *ctx, int layer_begin, int layer_count, int64_t T, const void *q, const void *k,

@@ -44,10 +44,22 @@ def test_non_contiguous_head_map():
     run_case([6, 20], 1, 4, 2, 64, F32, [30], 10, q_to_kv=[1, 0, 0, 1], prefill_chunk=16)
 
 
-def test_multi_layer_split_k_bf16():
+@pytest.mark.parametrize("impl", [1, 2])   # tensor-core/TMA kernel, CUDA-core kernel
+def test_multi_layer_split_k_bf16(impl):
     # several split-K items per unit, ragged last item, several state row blocks
     run_case([300, 129, 64, 0], 2, 8, 2, 128, BF16, [400], 40, amp=128 ** -0.5 * 4, decode_chunk=64,
-             decode_state_splits=4)
+             decode_state_splits=4, decode_impl=impl)
+
+
+@pytest.mark.parametrize("w", [1, 2, 15, 16, 17, 31, 33, 100])
+@pytest.mark.parametrize("d,G", [(128, 4), (64, 2), (64, 8), (128, 1)])
+def test_bf16_tensor_core_decode_window_edges(w, d, G):
+    # every token through decode: partially filled ring, wrap-around, the slot being evicted inside a tile
+    run_case([w], 2, 2 * G, 2, d, BF16, [], 2 * w + 40, amp=d ** -0.5 * 4, seed=w, decode_chunk=16 if w < 64 else 48)
+
+
+def test_bf16_large_logits():
+    run_case([40, 200], 1, 8, 2, 128, BF16, [250], 30, amp=128 ** -0.5 * 12)
 
 
 def test_never_evicting_layer_is_full_softmax():
