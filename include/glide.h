@@ -60,8 +60,10 @@ typedef enum { GLIDE_PHI_SOFTMAX = 0 } glide_phi;
  * "Retention-based SWA").  GLIDE_MERGE_SHARED is the shared normaliser above. */
 typedef enum { GLIDE_MERGE_SHARED = 0 } glide_merge;
 
-/* Decode kernel selection.  AUTO: tensor-core/TMA kernel for bf16 I/O, CUDA-core fp32 kernel for fp32 I/O. */
-typedef enum { GLIDE_DECODE_AUTO = 0, GLIDE_DECODE_MMA = 1, GLIDE_DECODE_FMA = 2 } glide_decode_impl;
+/* Decode kernel selection.  AUTO: for bf16 I/O the statically scheduled streaming tensor-core/TMA kernel
+ * (head_dim 128) or the per-item tensor-core/TMA kernel; for fp32 I/O the CUDA-core kernel.  The others
+ * force one kernel (GLIDE_ERR_UNSUPPORTED if it does not apply). */
+typedef enum { GLIDE_DECODE_AUTO = 0, GLIDE_DECODE_MMA = 1, GLIDE_DECODE_FMA = 2, GLIDE_DECODE_STREAM = 3 } glide_decode_impl;
 
 typedef struct {
   int32_t n_layers;        /* L >= 1 */

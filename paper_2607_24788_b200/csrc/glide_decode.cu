@@ -398,7 +398,8 @@ int decode_occupancy(const glide_ctx *ctx, int *blocks_per_sm) {
 
 int launch_decode(glide_ctx *ctx, const void *q, const void *k, const void *v, void *out, cudaStream_t stream) {
   const DecodeParams p = make_decode_params(ctx, q, k, v, out);
-  if (ctx->use_mma) return launch_decode_mma(ctx, p, stream);
+  if (ctx->decode_kind == 2) return launch_decode_stream(ctx, p, stream);
+  if (ctx->decode_kind == 1) return launch_decode_mma(ctx, p, stream);
   return dispatch_config(ctx->cfg.io_dtype, ctx->cfg.head_dim, ctx->G, [&](auto tt, auto dd, auto gg) -> int {
     using T = typename decltype(tt)::type;
     constexpr int D = decltype(dd)::value, G = decltype(gg)::value;

@@ -24,6 +24,22 @@ namespace glide {
 namespace {
 
 constexpr int kTileKeys = 16;
+
+// Optional per-warp event trace (debug builds only: -DGLIDE_TRACE).
+#ifdef GLIDE_TRACE
+__device__ unsigned long long *g_trace = nullptr;   // [warps][64] of (code << 56 | globaltimer ns)
+#define GLIDE_TRACE_EVENT(code)                                                                    \
+  do {                                                                                             \
+    if (g_trace && lane == 0 && trace_n < 64) {                                                    \
+      unsigned long long now;                                                                      \
+      asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(now));                                      \
+      g_trace[(size_t(blockIdx.x) * (blockDim.x >> 5) + (threadIdx.x >> 5)) * 64 + trace_n++] =    \
+          (static_cast<unsigned long long>(code) << 56) | (now & 0x00ffffffffffffffull);           \
+    }                                                                                              \
+  } while (0)
+#else
+#define GLIDE_TRACE_EVENT(code) do { } while (0)
+#endif
 constexpr uint32_t kWaitLimit = 1u << 24;   // polls of one mbarrier before giving up
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return uint32_t(__cvta_generic_to_shared(p)); }
@@ -398,14 +414,16 @@ __device__ __forceinline__ void state_item_warp(const DecodeParams &p, const Wor
 // ---- merge (the warp with the unit's last ticket) -------------------------------------------
 template <int D, int G>
 __device__ __forceinline__ void merge_unit_warp(const DecodeParams &p, const WorkItem &it, const LayerDev &ld, int64_t t,
-                                                int b, int g, int lane) {
+                                                int b, int g, float *scratch, int scratch_floats, int lane) {
   using bf16 = __nv_bfloat16;
   constexpr int E = D / 32;
   const int ub = b * p.Hkv + g;
-  const int per_unit = ld.n_win_items + ld.n_state_items;
+  const int n_win = ld.n_win_items, n_st = ld.n_state_items;
+  const int per_unit = n_win + n_st;
   const float *rec0 = p.partials + ld.part_base + size_t(ub) * per_unit * p.rec_floats;
   const bool has_win = ld.cap > 0;
-  const bool has_state = ld.n_state_items > 0 && (ld.w == 0 || t >= ld.w);
+  const bool has_state = n_st > 0 && (ld.w == 0 || t >= ld.w);
+  const bool cached = n_win * G <= scratch_floats;   // per-partial rescale factors kept in the warp's scratch
   const bf16 *kt = reinterpret_cast<const bf16 *>(p.k) + size_t(it.unit) * D;
   const bf16 *vt = reinterpret_cast<const bf16 *>(p.v) + size_t(it.unit) * D;
 
@@ -424,22 +442,30 @@ __device__ __forceinline__ void merge_unit_warp(const DecodeParams &p, const Wor
       for (int i = 0; i < E; ++i) part = fmaf(qx[i], kx[i], part);
       scur[h] = warp_sum(part) * p.scale_log2;
     }
-    // m* = max(window max, current logit, 0)
+  }
+  // m* = max(window max, current logit, 0); the partial maxima are read once, lane-strided
+#pragma unroll
+  for (int h = 0; h < G; ++h) {
     float mx = fmaxf(scur[h], 0.f);
-    for (int i = lane; i < ld.n_win_items; i += 32) mx = fmaxf(mx, __ldcg(rec0 + size_t(i) * p.rec_floats + G * D + h));
+    for (int i = lane; i < n_win; i += 32) mx = fmaxf(mx, __ldcg(rec0 + size_t(i) * p.rec_floats + G * D + h));
     M[h] = warp_max(mx);
+  }
+#pragma unroll
+  for (int h = 0; h < G; ++h) {
     float den = 0.f;
-    for (int i = lane; i < ld.n_win_items; i += 32) {
+    for (int i = lane; i < n_win; i += 32) {
       const float *r = rec0 + size_t(i) * p.rec_floats;
-      den = fmaf(__ldcg(r + G * D + G + h), exp2f(__ldcg(r + G * D + h) - M[h]), den);
+      const float f = exp2f(__ldcg(r + G * D + h) - M[h]);
+      if (cached) scratch[i * G + h] = f;
+      den = fmaf(__ldcg(r + G * D + G + h), f, den);
     }
     float bs = 0.f;
     if (has_state)
-      for (int i = lane; i < ld.n_state_items; i += 32)
-        bs += __ldcg(rec0 + size_t(ld.n_win_items + i) * p.rec_floats + G * D + h);
+      for (int i = lane; i < n_st; i += 32) bs += __ldcg(rec0 + size_t(n_win + i) * p.rec_floats + G * D + h);
     den = warp_sum(den) + (has_win ? exp2f(scur[h] - M[h]) : 0.f) + exp2f(-M[h]) * warp_sum(bs);
     inv[h] = 1.0f / den;
   }
+  __syncwarp();
   bf16 *outp = reinterpret_cast<bf16 *>(p.out);
 #pragma unroll
   for (int j = 0; j * 128 < G * D; ++j) {
@@ -455,14 +481,33 @@ __device__ __forceinline__ void merge_unit_warp(const DecodeParams &p, const Wor
         scurh = scur[hh];
       }
     float4 num = make_float4(0.f, 0.f, 0.f, 0.f);
-    for (int i = 0; i < ld.n_win_items; ++i) {
-      const float *r = rec0 + size_t(i) * p.rec_floats;
-      const float f = exp2f(__ldcg(r + G * D + h) - Mh);
-      const float4 a = __ldcg(reinterpret_cast<const float4 *>(r + idx));
-      num.x = fmaf(a.x, f, num.x);
-      num.y = fmaf(a.y, f, num.y);
-      num.z = fmaf(a.z, f, num.z);
-      num.w = fmaf(a.w, f, num.w);
+    if (cached) {
+      constexpr int MU = 8;   // independent loads in flight
+      for (int i0 = 0; i0 < n_win; i0 += MU) {
+        float4 a[MU];
+#pragma unroll
+        for (int u = 0; u < MU; ++u)
+          if (i0 + u < n_win) a[u] = __ldcg(reinterpret_cast<const float4 *>(rec0 + size_t(i0 + u) * p.rec_floats + idx));
+#pragma unroll
+        for (int u = 0; u < MU; ++u)
+          if (i0 + u < n_win) {
+            const float f = scratch[(i0 + u) * G + h];
+            num.x = fmaf(a[u].x, f, num.x);
+            num.y = fmaf(a[u].y, f, num.y);
+            num.z = fmaf(a[u].z, f, num.z);
+            num.w = fmaf(a[u].w, f, num.w);
+          }
+      }
+    } else {
+      for (int i = 0; i < n_win; ++i) {
+        const float *r = rec0 + size_t(i) * p.rec_floats;
+        const float f = exp2f(__ldcg(r + G * D + h) - Mh);
+        const float4 a = __ldcg(reinterpret_cast<const float4 *>(r + idx));
+        num.x = fmaf(a.x, f, num.x);
+        num.y = fmaf(a.y, f, num.y);
+        num.z = fmaf(a.z, f, num.z);
+        num.w = fmaf(a.w, f, num.w);
+      }
     }
     if (has_win) {
       const float f = exp2f(scurh - Mh);
@@ -475,8 +520,8 @@ __device__ __forceinline__ void merge_unit_warp(const DecodeParams &p, const Wor
     }
     if (has_state) {
       float4 asum = make_float4(0.f, 0.f, 0.f, 0.f);
-      for (int i = 0; i < ld.n_state_items; ++i) {
-        const float4 a = __ldcg(reinterpret_cast<const float4 *>(rec0 + size_t(ld.n_win_items + i) * p.rec_floats + idx));
+      for (int i = 0; i < n_st; ++i) {
+        const float4 a = __ldcg(reinterpret_cast<const float4 *>(rec0 + size_t(n_win + i) * p.rec_floats + idx));
         asum.x += a.x;
         asum.y += a.y;
         asum.z += a.z;
@@ -508,6 +553,7 @@ __device__ __forceinline__ void merge_unit_warp(const DecodeParams &p, const Wor
       *reinterpret_cast<uint32_t *>(Vd + lane * 2) = *reinterpret_cast<const uint32_t *>(vt + lane * 2);
     }
   }
+  __syncwarp();
 }
 
 template <int D, int G, int WARPS, int STAGES>
@@ -532,10 +578,15 @@ __global__ void __launch_bounds__(WARPS * 32, 1) glide_decode_mma_kernel(const D
   __syncwarp();
   const int units_per_layer = p.B * p.Hkv;
 
+#ifdef GLIDE_TRACE
+  int trace_n = 0;
+#endif
+  GLIDE_TRACE_EVENT(1);
   for (;;) {
     int idx = 0;
     if (lane == 0) idx = atomicAdd(&p.ctl->work_counter, 1);
     idx = __shfl_sync(0xffffffffu, idx, 0);
+    GLIDE_TRACE_EVENT(2);
     if (idx >= p.n_items) break;
     const WorkItem it = p.items[idx];
     if (it.layer < 0 || it.layer >= p.L || it.unit < 0) {
@@ -548,6 +599,7 @@ __global__ void __launch_bounds__(WARPS * 32, 1) glide_decode_mma_kernel(const D
     const int b = ub / p.Hkv, g = ub - b * p.Hkv;
     const int per_unit = ld.n_win_items + ld.n_state_items;
     float *rec = p.partials + ld.part_base + (size_t(ub) * per_unit + it.part) * p.rec_floats;
+    GLIDE_TRACE_EVENT(it.kind == kItemWindow ? 3 : 4);
     if (it.kind == kItemWindow) {
       window_item_mma<D, G, STAGES>(p, tmaps + 2 * it.layer, tmaps + 2 * it.layer + 1, it, ld, t, b, g, rec, pipe, lane);
       if (pipe.failed) {  // a TMA never completed: record it and stop taking work
@@ -557,17 +609,22 @@ __global__ void __launch_bounds__(WARPS * 32, 1) glide_decode_mma_kernel(const D
     } else {
       state_item_warp<D, G>(p, it, ld, t, b, g, rec, reinterpret_cast<float *>(my_stages), lane);
     }
+    GLIDE_TRACE_EVENT(5);
     __threadfence();
     __syncwarp();
+    GLIDE_TRACE_EVENT(6);
     int last = 0;
     if (lane == 0) last = atomicAdd(&p.tickets[it.unit], 1) == per_unit - 1;
     last = __shfl_sync(0xffffffffu, last, 0);
+    GLIDE_TRACE_EVENT(7);
     if (last) {
       __threadfence();
-      merge_unit_warp<D, G>(p, it, ld, t, b, g, lane);
+      merge_unit_warp<D, G>(p, it, ld, t, b, g, reinterpret_cast<float *>(my_stages), int(STAGES * STAGE_BYTES / 4), lane);
       if (lane == 0) p.tickets[it.unit] = 0;
+      GLIDE_TRACE_EVENT(8);
     }
   }
+  GLIDE_TRACE_EVENT(9);
   __syncthreads();
   if (threadIdx.x == 0) {
     __threadfence();
@@ -606,7 +663,7 @@ int dispatch_mma(int D, int G, F &&f) {
 
 }  // namespace
 
-int mma_decode_setup(glide_ctx *ctx) {
+int build_ring_tensor_maps(glide_ctx *ctx) {
   // tensor maps: per layer the K ring and the V ring as [rows = B*Hkv*cap][D] bf16, 64 x 16 boxes, 128-byte swizzle
   typedef CUresult (*EncodeFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
                                const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
@@ -638,7 +695,11 @@ int mma_decode_setup(glide_ctx *ctx) {
       if (r != CUDA_SUCCESS) return GLIDE_ERR_CUDA;
     }
   }
-  return dispatch_mma(D, ctx->G, [&](auto dd, auto gg) -> int {
+  return GLIDE_OK;
+}
+
+int mma_decode_setup(glide_ctx *ctx) {
+  return dispatch_mma(ctx->cfg.head_dim, ctx->G, [&](auto dd, auto gg) -> int {
     constexpr int DD = decltype(dd)::value, GG = decltype(gg)::value;
     auto kern = glide_decode_mma_kernel<DD, GG, kMmaWarps, kMmaStages>;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, int(mma_smem_bytes<DD>())) != cudaSuccess) {
@@ -655,6 +716,12 @@ int mma_decode_setup(glide_ctx *ctx) {
     return GLIDE_OK;
   });
 }
+
+#ifdef GLIDE_TRACE
+extern "C" int glide_debug_set_trace(void *dev_buf) {
+  return cudaMemcpyToSymbol(g_trace, &dev_buf, sizeof(void *)) == cudaSuccess ? 0 : 6;
+}
+#endif
 
 int launch_decode_mma(glide_ctx *ctx, const DecodeParams &p, cudaStream_t stream) {
   const CUtensorMap *tmaps = reinterpret_cast<const CUtensorMap *>(ctx->ws + ctx->off_tmaps);

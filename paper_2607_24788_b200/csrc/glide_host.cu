@@ -25,8 +25,9 @@ int validate_config(const glide_config *c) {
   if (c->softmax_scale < 0.f || !std::isfinite(c->softmax_scale)) return GLIDE_ERR_INVALID_ARG;
   if (c->prefill_chunk < 0 || c->decode_chunk < 0 || c->decode_state_splits < 0) return GLIDE_ERR_INVALID_ARG;
   if (c->prefill_chunk % 16 != 0 || c->prefill_chunk > 1024) return GLIDE_ERR_INVALID_ARG;
-  if (c->decode_impl < GLIDE_DECODE_AUTO || c->decode_impl > GLIDE_DECODE_FMA) return GLIDE_ERR_INVALID_ARG;
-  if (c->decode_impl == GLIDE_DECODE_MMA && c->io_dtype != GLIDE_BF16) return GLIDE_ERR_UNSUPPORTED;
+  if (c->decode_impl < GLIDE_DECODE_AUTO || c->decode_impl > GLIDE_DECODE_STREAM) return GLIDE_ERR_INVALID_ARG;
+  if ((c->decode_impl == GLIDE_DECODE_MMA || c->decode_impl == GLIDE_DECODE_STREAM) && c->io_dtype != GLIDE_BF16)
+    return GLIDE_ERR_UNSUPPORTED;
   for (int l = 0; l < c->n_layers; ++l)
     if (c->windows[l] < 0) return GLIDE_ERR_INVALID_ARG;
   if (c->phi != GLIDE_PHI_SOFTMAX || c->merge != GLIDE_MERGE_SHARED) return GLIDE_ERR_UNSUPPORTED;
@@ -116,7 +117,14 @@ int glide::plan_context(const glide_config *cfg, glide_ctx *ctx, std::vector<Wor
   ctx->off_tickets = off;
   off = align_up(off + sizeof(int32_t) * size_t(L) * units_per_layer, 256);
   ctx->off_partials = off;
+  ctx->stream_seg_capacity = size_t(L) * units_per_layer + kMaxStreamCtas;
+  ctx->stream_rec_capacity = ctx->stream_seg_capacity;
+  part_floats = std::max(part_floats, ctx->stream_rec_capacity * size_t(ctx->rec_floats));
   off = align_up(off + sizeof(float) * part_floats, 256);
+  ctx->off_stream_segs = off;
+  off = align_up(off + sizeof(StreamSegment) * ctx->stream_seg_capacity, 256);
+  ctx->off_stream_cta = off;
+  off = align_up(off + sizeof(int32_t) * (kMaxStreamCtas + 1), 256);
   ctx->off_tmaps = off;
   off = align_up(off + size_t(128) * 2 * L, 256);
   ctx->off_phik = off;
@@ -174,13 +182,19 @@ int glide::plan_context(const glide_config *cfg, glide_ctx *ctx, std::vector<Wor
         }
       }
     }
-    // longest first: bytes an item moves
+    // Units with the most bytes first, a unit's items adjacent: the merge of a long-window unit (many
+    // partials) then runs in the middle of the launch, and the tail is made of the cheapest units.
     const size_t elem = ctx->elem;
-    auto cost = [&](const WorkItem &it) -> size_t {
-      return it.kind == kItemWindow ? size_t(it.count) * d * elem * 2 : size_t(it.count) * d * 4 * 2;
+    auto layer_cost = [&](int l) -> size_t {
+      const LayerDev &ld = ctx->layers[l];
+      return size_t(ld.cap) * d * elem * 2 + (ld.evicts ? size_t(d) * d * 4 * 2 : 0);
     };
-    std::stable_sort(items->begin(), items->end(),
-                     [&](const WorkItem &a, const WorkItem &b) { return cost(a) > cost(b); });
+    std::stable_sort(items->begin(), items->end(), [&](const WorkItem &a, const WorkItem &b) {
+      const size_t ca = layer_cost(a.layer), cb = layer_cost(b.layer);
+      if (ca != cb) return ca > cb;
+      if (a.unit != b.unit) return a.unit < b.unit;
+      return a.kind > b.kind;   // state rows first, then the window runs
+    });
   }
   return GLIDE_OK;
 }
@@ -222,17 +236,38 @@ int glide_create(const glide_config *cfg, void *dev_workspace, size_t workspace_
   bool ok = cudaGetDevice(&ctx->device) == cudaSuccess &&
             cudaDeviceGetAttribute(&ctx->sm_count, cudaDevAttrMultiProcessorCount, ctx->device) == cudaSuccess;
   int per_sm = 0;
-  ctx->use_mma = cfg->io_dtype == GLIDE_BF16 && cfg->decode_impl != GLIDE_DECODE_FMA;
-  if (ctx->use_mma) {
-    ok = ok && mma_decode_setup(ctx) == GLIDE_OK;
-  } else {
-    ok = ok && decode_occupancy(ctx, &per_sm) == GLIDE_OK && per_sm > 0;
+  // kernel choice: fp32 -> CUDA cores; bf16 -> streaming tensor-core kernel when it applies, else per-item one
+  ctx->decode_kind = 0;
+  if (ok && cfg->io_dtype == GLIDE_BF16 && cfg->decode_impl != GLIDE_DECODE_FMA) {
+    ok = build_ring_tensor_maps(ctx) == GLIDE_OK;
+    const bool want_stream = cfg->decode_impl == GLIDE_DECODE_AUTO || cfg->decode_impl == GLIDE_DECODE_STREAM;
+    if (ok && want_stream && stream_decode_supported(ctx) && ctx->sm_count <= kMaxStreamCtas) {
+      int rc2 = stream_decode_setup(ctx);
+      if (rc2 == GLIDE_OK) ctx->decode_kind = 2;
+      else if (rc2 != GLIDE_ERR_UNSUPPORTED) ok = false;
+    }
+    if (ok && ctx->decode_kind == 0) {
+      if (cfg->decode_impl == GLIDE_DECODE_STREAM) {   // asked for explicitly but not applicable
+        delete ctx;
+        return GLIDE_ERR_UNSUPPORTED;
+      }
+      ok = mma_decode_setup(ctx) == GLIDE_OK;
+      ctx->decode_kind = 1;
+    }
+  } else if (ok) {
+    ok = decode_occupancy(ctx, &per_sm) == GLIDE_OK && per_sm > 0;
     if (ok) ctx->decode_grid = std::max(1, std::min(ctx->n_items, ctx->sm_count * per_sm));
   }
   if (ok) {
-    if (ctx->use_mma)
+    if (ctx->decode_kind >= 1)
       ok = cudaMemcpyAsync(ctx->ws + ctx->off_tmaps, ctx->tmaps_host.data(), ctx->tmaps_host.size(),
                            cudaMemcpyHostToDevice, st) == cudaSuccess;
+    if (ok && ctx->decode_kind == 2) {
+      ok = cudaMemcpyAsync(ctx->ws + ctx->off_stream_segs, ctx->stream_segs.data(),
+                           sizeof(StreamSegment) * ctx->stream_segs.size(), cudaMemcpyHostToDevice, st) == cudaSuccess &&
+           cudaMemcpyAsync(ctx->ws + ctx->off_stream_cta, ctx->stream_cta_begin.data(),
+                           sizeof(int32_t) * ctx->stream_cta_begin.size(), cudaMemcpyHostToDevice, st) == cudaSuccess;
+    }
     // control words, counters, tickets, S and z start at zero
     ok = ok && cudaMemsetAsync(ctx->ws, 0, ctx->off_layers, st) == cudaSuccess &&
          cudaMemsetAsync(ctx->ws + ctx->off_tickets, 0, ctx->off_partials - ctx->off_tickets, st) == cudaSuccess &&
@@ -383,7 +418,7 @@ int glide_device_status(glide_ctx *ctx, void *stream, int32_t *status_out) {
 int glide_decode_launch_info(glide_ctx *ctx, int32_t *n_launches, int32_t *n_work_items, int32_t *grid_size) {
   if (!ctx) return GLIDE_ERR_INVALID_ARG;
   if (n_launches) *n_launches = 1;
-  if (n_work_items) *n_work_items = ctx->n_items;
+  if (n_work_items) *n_work_items = ctx->decode_kind == 2 ? int32_t(ctx->stream_segs.size()) : ctx->n_items;
   if (grid_size) *grid_size = ctx->decode_grid;
   return GLIDE_OK;
 }

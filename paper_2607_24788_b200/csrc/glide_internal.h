@@ -69,6 +69,32 @@ struct DecodeParams {
   float scale_log2;          // softmax_scale * log2(e)
 };
 
+// One segment of the streaming decode kernel's schedule: the part of one unit that falls into one CTA's
+// range of the tile stream (state tiles first, then window tiles).  64 bytes.
+struct StreamSegment {
+  int32_t unit, layer;
+  int32_t tile0;             // CTA-relative index of the segment's first tile
+  int32_t n_state, state0;   // state tiles [state0, state0 + n_state): 16 rows of S each
+  int32_t n_win, win0;       // window tiles [win0, win0 + n_win): 16 ring slots each
+  int32_t part;              // this CTA's record among the unit's records, -1 if the whole unit is in this CTA
+  int32_t n_parts;           // records of the unit (ticket target)
+  int32_t rec0;              // index of the unit's first record in the split-K scratch
+  int32_t row_base;          // row of the unit's slot 0 in the layer's [rows][d] ring tensor
+  int32_t cap;               // ring slots
+  int32_t w;                 // window (clamped to INT32_MAX)
+  int32_t evicts;
+  int32_t S_off256, z_off256;  // workspace byte offsets / 256 of the unit's S and z
+};
+static_assert(sizeof(StreamSegment) == 64, "StreamSegment is copied as 16-byte chunks");
+
+struct StreamParams {
+  const StreamSegment *segs;
+  const int32_t *cta_seg_begin;    // [grid + 1]
+  const struct CUtensorMap_st *tmaps;   // [2 L]: K ring, V ring per layer
+  int32_t max_segs;
+  int32_t heads_contiguous;
+};
+
 struct PrefillParams {
   unsigned char *ws;
   const LayerDev *layers;
@@ -97,7 +123,14 @@ struct glide_ctx {
   std::vector<glide::LayerDev> layers;
   std::vector<int64_t> n_host;      // mirror of the device counters
   std::vector<unsigned char> tmaps_host;  // TMA descriptors of the rings (bf16 tensor-core decode kernel)
-  bool use_mma = false;             // bf16: tensor-core decode kernel; fp32: CUDA-core kernel
+  int decode_kind = 0;              // 0 CUDA-core kernel, 1 per-item tensor-core kernel, 2 streaming tensor-core kernel
+  std::vector<glide::StreamSegment> stream_segs;
+  std::vector<int32_t> stream_cta_begin;
+  int stream_max_segs = 0;
+  bool stream_heads_contiguous = true;
+  size_t stream_smem = 0;
+  size_t stream_seg_capacity = 0, stream_rec_capacity = 0;
+  size_t off_stream_segs = 0, off_stream_cta = 0;
   int G = 0;
   int device = 0;
   int sm_count = 0;
@@ -121,7 +154,12 @@ namespace glide {
 int plan_context(const glide_config *cfg, glide_ctx *ctx, std::vector<WorkItem> *items);
 
 DecodeParams make_decode_params(const glide_ctx *ctx, const void *q, const void *k, const void *v, void *out);
-int mma_decode_setup(glide_ctx *ctx);   // builds the ring tensor maps (host copy) and sizes the grid
+int build_ring_tensor_maps(glide_ctx *ctx);   // TMA descriptors of every layer's K and V ring (host copy)
+int mma_decode_setup(glide_ctx *ctx);         // sizes the grid of the per-item tensor-core kernel
+int stream_decode_supported(const glide_ctx *ctx);
+int stream_decode_setup(glide_ctx *ctx);      // builds the static schedule (host copy) and sizes the launch
+int launch_decode_stream(glide_ctx *ctx, const DecodeParams &p, cudaStream_t stream);
+constexpr int kMaxStreamCtas = 1024;          // upper bound on SMs used to size the schedule's workspace
 int launch_decode_mma(glide_ctx *ctx, const DecodeParams &p, cudaStream_t stream);
 int launch_decode(glide_ctx *ctx, const void *q, const void *k, const void *v, void *out, cudaStream_t stream);
 int decode_occupancy(const glide_ctx *ctx, int *blocks_per_sm);

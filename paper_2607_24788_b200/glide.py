@@ -18,7 +18,7 @@ LIB_PATH = os.path.join(_PKG, "libglide.so")
 GLIDE_F32, GLIDE_BF16 = 0, 1
 GLIDE_PHI_SOFTMAX = 0
 GLIDE_MERGE_SHARED = 0
-GLIDE_DECODE_AUTO, GLIDE_DECODE_MMA, GLIDE_DECODE_FMA = 0, 1, 2
+GLIDE_DECODE_AUTO, GLIDE_DECODE_MMA, GLIDE_DECODE_FMA, GLIDE_DECODE_STREAM = 0, 1, 2, 3
 
 GLIDE_OK = 0
 GLIDE_ERR_INVALID_ARG = 1

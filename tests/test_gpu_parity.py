@@ -44,7 +44,7 @@ def test_non_contiguous_head_map():
     run_case([6, 20], 1, 4, 2, 64, F32, [30], 10, q_to_kv=[1, 0, 0, 1], prefill_chunk=16)
 
 
-@pytest.mark.parametrize("impl", [1, 2])   # tensor-core/TMA kernel, CUDA-core kernel
+@pytest.mark.parametrize("impl", [1, 2, 3])   # per-item tensor-core kernel, CUDA-core kernel, streaming tensor-core kernel
 def test_multi_layer_split_k_bf16(impl):
     # several split-K items per unit, ragged last item, several state row blocks
     run_case([300, 129, 64, 0], 2, 8, 2, 128, BF16, [400], 40, amp=128 ** -0.5 * 4, decode_chunk=64,
@@ -56,6 +56,17 @@ def test_multi_layer_split_k_bf16(impl):
 def test_bf16_tensor_core_decode_window_edges(w, d, G):
     # every token through decode: partially filled ring, wrap-around, the slot being evicted inside a tile
     run_case([w], 2, 2 * G, 2, d, BF16, [], 2 * w + 40, amp=d ** -0.5 * 4, seed=w, decode_chunk=16 if w < 64 else 48)
+
+
+@pytest.mark.parametrize("w", [0, 16, 32, 100])
+def test_bf16_stream_many_small_units(w):
+    # 256 units over 148 CTAs: units that live inside one CTA and units cut by a CTA boundary
+    run_case([w] * 8, 8, 8, 4, 128, BF16, [w + 24], 6, amp=128 ** -0.5 * 4, seed=w, decode_impl=3, state_checks=True)
+
+
+def test_bf16_stream_mixed_windows_and_batch():
+    run_case([700, 300, 64, 16, 0, 0, 48, 1 << 20], 3, 8, 2, 128, BF16, [720], 24, amp=128 ** -0.5 * 4, decode_impl=3,
+             max_tokens=760)
 
 
 def test_bf16_large_logits():
