@@ -601,7 +601,7 @@ __global__ void __launch_bounds__(WARPS * 32, 1) glide_decode_mma_kernel(const D
     float *rec = p.partials + ld.part_base + (size_t(ub) * per_unit + it.part) * p.rec_floats;
     GLIDE_TRACE_EVENT(it.kind == kItemWindow ? 3 : 4);
     if (it.kind == kItemWindow) {
-      window_item_mma<D, G, STAGES>(p, tmaps + 2 * it.layer, tmaps + 2 * it.layer + 1, it, ld, t, b, g, rec, pipe, lane);
+      window_item_mma<D, G, STAGES>(p, tmaps + 3 * it.layer, tmaps + 3 * it.layer + 1, it, ld, t, b, g, rec, pipe, lane);
       if (pipe.failed) {  // a TMA never completed: record it and stop taking work
         if (lane == 0) atomicExch(&p.ctl->status, kDevWaitTimeout);
         break;
@@ -677,7 +677,8 @@ int build_ring_tensor_maps(glide_ctx *ctx) {
   }
   EncodeFn encode = reinterpret_cast<EncodeFn>(fn);
   const int L = ctx->cfg.n_layers, D = ctx->cfg.head_dim;
-  ctx->tmaps_host.assign(size_t(L) * 2 * sizeof(CUtensorMap), 0);
+  ctx->tmaps_host.assign(size_t(L) * 3 * sizeof(CUtensorMap), 0);
+  ctx->tmaps_kv4d = D == 128;
   CUtensorMap *maps = reinterpret_cast<CUtensorMap *>(ctx->tmaps_host.data());
   for (int l = 0; l < L; ++l) {
     const LayerDev &ld = ctx->layers[l];
@@ -689,10 +690,22 @@ int build_ring_tensor_maps(glide_ctx *ctx) {
     const cuuint32_t estr[2] = {1, 1};
     for (int kv = 0; kv < 2; ++kv) {
       void *gptr = ctx->ws + (kv == 0 ? ld.ringK : ld.ringV);
-      CUresult r = encode(&maps[2 * l + kv], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, gptr, dims, strides, box, estr,
+      CUresult r = encode(&maps[3 * l + kv], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, gptr, dims, strides, box, estr,
                           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
       if (r != CUDA_SUCCESS) return GLIDE_ERR_CUDA;
+    }
+    if (D == 128 && ctx->tmaps_kv4d) {
+      // K and V rings of the layer as one 4-D tensor [kv][half][row][64]: a single TMA then fills a whole
+      // window stage in the layout the 2-D boxes produce (K halves, then V halves)
+      const cuuint64_t dims4[4] = {64, rows, 2, 2};
+      const cuuint64_t strides4[3] = {cuuint64_t(D) * 2, 128, cuuint64_t(ld.ringV - ld.ringK)};
+      const cuuint32_t box4[4] = {64, kTileKeys, 2, 2};
+      const cuuint32_t estr4[4] = {1, 1, 1, 1};
+      CUresult r = encode(&maps[3 * l + 2], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, ctx->ws + ld.ringK, dims4, strides4, box4,
+                          estr4, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                          CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+      if (r != CUDA_SUCCESS) ctx->tmaps_kv4d = false;   // the driver refused the strides: keep the 2-D boxes
     }
   }
   return GLIDE_OK;

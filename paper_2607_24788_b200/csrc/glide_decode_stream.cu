@@ -38,6 +38,22 @@ constexpr uint32_t kTileKV = 2 * kBoxBytes;                // K (or V) part of a
 constexpr uint32_t kWaitLimit = 1u << 24;
 constexpr int kHdrSlots = 3;
 
+// Optional per-warp event trace (debug builds only: -DGLIDE_TRACE).
+#ifdef GLIDE_TRACE
+__device__ unsigned long long *g_stream_trace = nullptr;   // [warps][64] of (code << 56 | globaltimer ns)
+#define GLIDE_TRACE_EVENT(code)                                                                        \
+  do {                                                                                                 \
+    if (g_stream_trace && lane == 0 && trace_n < 64) {                                                 \
+      unsigned long long now;                                                                          \
+      asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(now));                                          \
+      g_stream_trace[(size_t(blockIdx.x) * kWarps + (threadIdx.x >> 5)) * 64 + trace_n++] =            \
+          (static_cast<unsigned long long>(code) << 56) | (now & 0x00ffffffffffffffull);               \
+    }                                                                                                  \
+  } while (0)
+#else
+#define GLIDE_TRACE_EVENT(code) do { } while (0)
+#endif
+
 // ---- PTX wrappers --------------------------------------------------------------------------
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return uint32_t(__cvta_generic_to_shared(p)); }
 __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
@@ -87,14 +103,14 @@ __device__ __forceinline__ void ldmatrix_x4_trans(uint32_t (&r)[4], uint32_t add
                : "r"(addr));
 }
 __device__ __forceinline__ void mma_bf16(float (&d)[4], const uint32_t (&a)[4], const uint32_t (&b)[2]) {
-  asm volatile(
+  asm(
       "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
       : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
       : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b[0]), "r"(b[1]));
 }
 __device__ __forceinline__ uint32_t movmatrix_trans(uint32_t x) {
   uint32_t y;
-  asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;" : "=r"(y) : "r"(x));
+  asm("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;" : "=r"(y) : "r"(x));
   return y;
 }
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi, float &lo_r, float &hi_r) {
@@ -128,41 +144,70 @@ __device__ __forceinline__ float4 lds_f32x4(uint32_t addr) {
   asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(addr));
   return v;
 }
-__device__ __forceinline__ float exp2_or_zero(float m, float M) { return m == -CUDART_INF_F ? 0.f : exp2f(m - M); }
-
 // ---- schedule walking ------------------------------------------------------------------------
-struct Cursor {
-  int i;    // CTA-relative index of this warp's next candidate tile
-  int seg;  // segment that holds it
-};
-struct TileRef {
-  int seg;
-  int index;     // state tile index (rows 16*index ..) or window tile index (slots 16*index ..) within the unit
-  bool is_state;
-};
+__device__ __forceinline__ float ex2_approx(float x) {   // 2^x, 2 ulp, 2^-inf = 0
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+__device__ __forceinline__ float exp2_or_zero(float m, float M) { return m == -CUDART_INF_F ? 0.f : ex2_approx(m - M); }
+
+__device__ __forceinline__ void tma_load_4d(uint32_t dst, const void *tmap, int c0, int c1, int c2, int c3, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5}], [%6];" ::"r"(dst),
+      "l"(tmap), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(bar)
+      : "memory");
+}
 
 __device__ __forceinline__ bool seg_evicting(const StreamSegment &s, int64_t t) {
   return s.evicts && (s.w == 0 || t >= int64_t(s.w));
 }
 
-// Next tile of this warp that has work at position t; both the issuing lane and the consuming warp walk
-// the same sequence.
+// A warp's position in the CTA's tile range with the fields of its current segment cached in registers.
+struct Cursor {
+  int i;         // CTA-relative index of this warp's next candidate tile
+  int seg;       // segment that holds it
+  int tile0, tile_end, n_state, state0, win0;
+  int n_valid_win;   // window tiles of the segment that hold window tokens at this position
+  int evicting;
+};
+struct TileRef {
+  int seg;
+  int index;     // state tile (rows 16*index ..) or window tile (slots 16*index ..) within the unit
+  bool is_state;
+};
+
+__device__ __forceinline__ void cursor_load(Cursor &c, const StreamSegment *segs, int64_t t) {
+  const StreamSegment &s = segs[c.seg];
+  c.tile0 = s.tile0;
+  c.n_state = s.n_state;
+  c.state0 = s.state0;
+  c.win0 = s.win0;
+  c.tile_end = s.tile0 + s.n_state + s.n_win;
+  const int64_t lim = t < int64_t(s.cap) ? t : int64_t(s.cap);
+  int nv = int((lim + kTileRows - 1) / kTileRows) - s.win0;
+  c.n_valid_win = nv < 0 ? 0 : (nv > s.n_win ? s.n_win : nv);
+  c.evicting = seg_evicting(s, t) ? 1 : 0;
+}
+
+// Next tile of this warp that has work; the issuing lane and the consuming warp walk the same sequence.
 __device__ __forceinline__ bool next_tile(Cursor &c, const StreamSegment *segs, int nseg, int ntiles, int64_t t,
                                           TileRef &ref) {
   while (c.i < ntiles) {
-    while (c.seg + 1 < nseg && c.i >= segs[c.seg].tile0 + segs[c.seg].n_state + segs[c.seg].n_win) ++c.seg;
-    const StreamSegment &s = segs[c.seg];
-    const int local = c.i - s.tile0;
+    if (c.i >= c.tile_end) {
+      do { ++c.seg; } while (c.seg + 1 < nseg && c.i >= segs[c.seg].tile0 + segs[c.seg].n_state + segs[c.seg].n_win);
+      cursor_load(c, segs, t);
+    }
+    const int local = c.i - c.tile0;
     bool valid;
-    if (local < s.n_state) {
+    if (local < c.n_state) {
       ref.is_state = true;
-      ref.index = s.state0 + local;
-      valid = seg_evicting(s, t);
+      ref.index = c.state0 + local;
+      valid = c.evicting != 0;
     } else {
       ref.is_state = false;
-      ref.index = s.win0 + local - s.n_state;
-      const int64_t lim = t < int64_t(s.cap) ? t : int64_t(s.cap);
-      valid = int64_t(ref.index) * kTileRows < lim;
+      ref.index = c.win0 + local - c.n_state;
+      valid = local - c.n_state < c.n_valid_win;
     }
     ref.seg = c.seg;
     c.i += kWarps;
@@ -176,6 +221,38 @@ struct Layout {
   static constexpr int kRecFloats = (G * kD + 2 * G + 3) / 4 * 4;
   static constexpr uint32_t kHdrBytes = G * 256 + 4 * 256;   // q rows | k_e | v_e | k_t | v_t
 };
+
+// phi = softmax over the 128 entries of N rows at once (lane holds 4 entries of each row); the N
+// reductions are interleaved so that their shuffle latencies overlap.
+template <int N>
+__device__ __forceinline__ void warp_phi_multi(float (&x)[N][4]) {
+  float mx[N], sm[N];
+#pragma unroll
+  for (int n = 0; n < N; ++n) mx[n] = fmaxf(fmaxf(x[n][0], x[n][1]), fmaxf(x[n][2], x[n][3]));
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1)
+#pragma unroll
+    for (int n = 0; n < N; ++n) mx[n] = fmaxf(mx[n], __shfl_xor_sync(0xffffffffu, mx[n], o));
+#pragma unroll
+  for (int n = 0; n < N; ++n) {
+    sm[n] = 0.f;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      x[n][i] = exp2f((x[n][i] - mx[n]) * kLog2e);
+      sm[n] += x[n][i];
+    }
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1)
+#pragma unroll
+    for (int n = 0; n < N; ++n) sm[n] += __shfl_xor_sync(0xffffffffu, sm[n], o);
+#pragma unroll
+  for (int n = 0; n < N; ++n) {
+    const float inv = 1.0f / sm[n];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) x[n][i] *= inv;
+  }
+}
 
 // ---- the kernel -----------------------------------------------------------------------------
 template <int G, int STAGES>
@@ -195,9 +272,13 @@ glide_decode_stream_kernel(const DecodeParams p, const StreamParams sp) {
   StreamSegment *sm_segs = reinterpret_cast<StreamSegment *>(sm_z + kWarps * STAGES * 16);      // [max_segs]
   uint64_t *sm_bars = reinterpret_cast<uint64_t *>(sm_segs + sp.max_segs);                        // [kWarps*STAGES + 3]
   float *sm_scur = reinterpret_cast<float *>(sm_bars + kWarps * STAGES + kHdrSlots);             // [8]
-  int *sm_flag = reinterpret_cast<int *>(sm_scur + 8);                                           // [4]
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+#ifdef GLIDE_TRACE
+  int trace_n = 0;
+#endif
+  GLIDE_TRACE_EVENT(1);
+  const int64_t t = p.n_dev[0];   // every layer is at the same position (checked by the host)
   const int col2 = (lane & 3) * 2, hrow = lane >> 2;
   const int seg_begin = sp.cta_seg_begin[blockIdx.x];
   const int nseg = sp.cta_seg_begin[blockIdx.x + 1] - seg_begin;
@@ -207,8 +288,10 @@ glide_decode_stream_kernel(const DecodeParams p, const StreamParams sp) {
     for (int i = tid; i < nseg * int(sizeof(StreamSegment) / 16); i += kThreads) dst[i] = src[i];
   }
   const uint32_t my_stages = smem_u32(sm_stages + size_t(warp) * STAGES * kStageBytes);
+  unsigned char *my_stages_ptr = sm_stages + size_t(warp) * STAGES * kStageBytes;
   const uint32_t my_bars = smem_u32(sm_bars + warp * STAGES);
   const uint32_t my_z = smem_u32(sm_z + warp * STAGES * 16);
+  const float *my_z_ptr = sm_z + warp * STAGES * 16;
   const uint32_t hdr_bars = smem_u32(sm_bars + kWarps * STAGES);
   if (lane == 0)
     for (int s = 0; s < STAGES; ++s) mbar_init(my_bars + s * 8, 1);
@@ -218,7 +301,6 @@ glide_decode_stream_kernel(const DecodeParams p, const StreamParams sp) {
   fence_async_smem();
   __syncthreads();
 
-  const int64_t t = p.n_dev[0];   // every layer is at the same position (checked by the host)
   const int ntiles = nseg > 0 ? sm_segs[nseg - 1].tile0 + sm_segs[nseg - 1].n_state + sm_segs[nseg - 1].n_win : 0;
   const int units_per_layer = p.B * p.Hkv;
   bool failed = false;
@@ -231,7 +313,6 @@ glide_decode_stream_kernel(const DecodeParams p, const StreamParams sp) {
     const bool ev = seg_evicting(sg, t);
     const int ub = sg.unit - sg.layer * units_per_layer;
     const int b = ub / p.Hkv, g = ub - b * p.Hkv;
-    fence_async_smem();
     mbar_expect_tx(bar, G * 256 + 512 + (ev ? 512 : 0));
     const bf16 *qb = reinterpret_cast<const bf16 *>(p.q) + (size_t(sg.layer) * p.B + b) * p.H * kD;
     if (sp.heads_contiguous) {
@@ -261,51 +342,79 @@ glide_decode_stream_kernel(const DecodeParams p, const StreamParams sp) {
   }
 
   // ---- tile issue (lane 0 of each warp) ---------------------------------------------------------
-  Cursor icur{warp, 0};
-  int n_issued = 0;
+  Cursor icur;
+  icur.i = warp;
+  icur.seg = 0;
+  icur.tile_end = 0;
+  if (nseg > 0) cursor_load(icur, sm_segs, t);
+  int issue_stage = 0;
   auto issue_next = [&]() {
     if (lane == 0) {
       TileRef r;
       if (next_tile(icur, sm_segs, nseg, ntiles, t, r)) {
         const StreamSegment &sg = sm_segs[r.seg];
-        const int stage = n_issued % STAGES;
-        const uint32_t bar = my_bars + stage * 8;
-        const uint32_t dst = my_stages + stage * kStageBytes;
-        fence_async_smem();   // earlier generic-proxy accesses to this stage precede the async-proxy fill
+        const uint32_t bar = my_bars + issue_stage * 8;
+        const uint32_t dst = my_stages + issue_stage * kStageBytes;
         if (r.is_state) {
           mbar_expect_tx(bar, kStageBytes + 64);
           const float *Sg = reinterpret_cast<const float *>(p.ws + size_t(sg.S_off256) * 256) + size_t(r.index) * kTileRows * kD;
           const float *zg = reinterpret_cast<const float *>(p.ws + size_t(sg.z_off256) * 256) + r.index * kTileRows;
           bulk_load(dst, Sg, kStageBytes, bar);
-          bulk_load(my_z + stage * 64, zg, 64, bar);
+          bulk_load(my_z + issue_stage * 64, zg, 64, bar);
         } else {
           mbar_expect_tx(bar, kStageBytes);
-          const CUtensorMap *tk = reinterpret_cast<const CUtensorMap *>(sp.tmaps) + 2 * sg.layer;
+          const CUtensorMap *tk = reinterpret_cast<const CUtensorMap *>(sp.tmaps) + 3 * sg.layer;
           const int y = sg.row_base + r.index * kTileRows;
-          tma_load_2d(dst, tk, 0, y, bar);
-          tma_load_2d(dst + kBoxBytes, tk, 64, y, bar);
-          tma_load_2d(dst + kTileKV, tk + 1, 0, y, bar);
-          tma_load_2d(dst + kTileKV + kBoxBytes, tk + 1, 64, y, bar);
+          if (sp.kv4d) {
+            tma_load_4d(dst, tk + 2, 0, y, 0, 0, bar);   // K halves then V halves: [kv][half][row][64]
+          } else {
+            tma_load_2d(dst, tk, 0, y, bar);
+            tma_load_2d(dst + kBoxBytes, tk, 64, y, bar);
+            tma_load_2d(dst + kTileKV, tk + 1, 0, y, bar);
+            tma_load_2d(dst + kTileKV + kBoxBytes, tk + 1, 64, y, bar);
+          }
         }
-        ++n_issued;
+        issue_stage = issue_stage + 1 == STAGES ? 0 : issue_stage + 1;
       }
     }
   };
   for (int s = 0; s < STAGES; ++s) issue_next();
+  GLIDE_TRACE_EVENT(2);
 
   // ---- per-unit register state ------------------------------------------------------------------
   uint32_t qb[KS][2];
   float o[KS][4];
   float m0 = -CUDART_INF_F, m1 = -CUDART_INF_F, l0 = 0.f, l1 = 0.f;
-  float phik[4], ve[4], phiq[G][4];
+  float phi[G + 1][4];     // phi(q_h) for the G heads, then phi(k_e); lane holds entries 4*lane .. 4*lane+3
+  float ve[4];
   float4 a[G];
   float bp[G];
-  bool had_state = false;
+  bool had_state = false, phi_ready = false;
   int acc_seg = -1;        // segment the accumulators belong to
+  int win_end = 0, win_cur = 0;   // window tokens live in slots [0, win_end) except slot win_cur
   uint32_t phases = 0;     // parity expected by the next wait on each stage
-  int n_consumed = 0;
+  int stage = 0;
 
-  auto reset_acc = [&]() {
+  auto wait_header = [&](int s) {
+    if (!mbar_wait(hdr_bars + (s % kHdrSlots) * 8, uint32_t(s / kHdrSlots) & 1u)) failed = true;
+  };
+
+  // q fragments of segment s into registers; accumulators cleared
+  auto load_unit = [&](int s) {
+    const StreamSegment &sg = sm_segs[s];
+    wait_header(s);
+    const uint32_t *hq = reinterpret_cast<const uint32_t *>(sm_hdr + size_t(s % kHdrSlots) * L::kHdrBytes);
+    const bool valid = hrow < G;
+#pragma unroll
+    for (int ks = 0; ks < KS; ++ks) {
+      qb[ks][0] = valid ? hq[hrow * 64 + ks * 8 + (lane & 3)] : 0u;
+      qb[ks][1] = valid ? hq[hrow * 64 + ks * 8 + 4 + (lane & 3)] : 0u;
+    }
+    if (sg.cap > 0) {
+      const int64_t lim = t < int64_t(sg.cap) ? t : int64_t(sg.cap);
+      win_end = int(lim);
+      win_cur = int(t % int64_t(sg.cap));
+    }
 #pragma unroll
     for (int mt = 0; mt < KS; ++mt) o[mt][0] = o[mt][1] = o[mt][2] = o[mt][3] = 0.f;
     m0 = m1 = -CUDART_INF_F;
@@ -316,80 +425,62 @@ glide_decode_stream_kernel(const DecodeParams p, const StreamParams sp) {
       bp[h] = 0.f;
     }
     had_state = false;
-  };
-
-  auto wait_header = [&](int s) {
-    if (!mbar_wait(hdr_bars + (s % kHdrSlots) * 8, uint32_t(s / kHdrSlots) & 1u)) failed = true;
-  };
-
-  // q fragments and feature maps of segment s into registers
-  auto load_unit = [&](int s) {
-    const StreamSegment &sg = sm_segs[s];
-    wait_header(s);
-    const uint32_t hdr = smem_u32(sm_hdr + size_t(s % kHdrSlots) * L::kHdrBytes);
-    const bool valid = hrow < G;
-#pragma unroll
-    for (int ks = 0; ks < KS; ++ks) {
-      qb[ks][0] = valid ? lds_u32(hdr + hrow * 256 + (ks * 8 + (lane & 3)) * 4) : 0u;
-      qb[ks][1] = valid ? lds_u32(hdr + hrow * 256 + (ks * 8 + 4 + (lane & 3)) * 4) : 0u;
-    }
-    if (sg.n_state > 0 && seg_evicting(sg, t)) {
-      const bf16 *hk = reinterpret_cast<const bf16 *>(sm_hdr + size_t(s % kHdrSlots) * L::kHdrBytes + G * 256);
-      load_elems<bf16, 4>(hk + lane * 4, phik);
-      load_elems<bf16, 4>(hk + kD + lane * 4, ve);
-      warp_phi<4>(phik);
-#pragma unroll
-      for (int h = 0; h < G; ++h) {
-        load_elems<bf16, 4>(reinterpret_cast<const bf16 *>(sm_hdr + size_t(s % kHdrSlots) * L::kHdrBytes) + h * kD + lane * 4,
-                            phiq[h]);
-        warp_phi<4>(phiq[h]);
-      }
-    }
-    reset_acc();
+    phi_ready = false;
     acc_seg = s;
   };
 
+  // feature maps of the unit's queries and of the evicted key (first state tile of a segment only)
+  auto load_phi = [&](int s) {
+    const bf16 *h0 = reinterpret_cast<const bf16 *>(sm_hdr + size_t(s % kHdrSlots) * L::kHdrBytes);
+#pragma unroll
+    for (int h = 0; h < G; ++h) load_elems<bf16, 4>(h0 + h * kD + lane * 4, phi[h]);
+    load_elems<bf16, 4>(h0 + G * kD + lane * 4, phi[G]);
+    load_elems<bf16, 4>(h0 + (G + 1) * kD + lane * 4, ve);
+    warp_phi_multi<G + 1>(phi);
+    phi_ready = true;
+  };
+
   // ---- window tile ------------------------------------------------------------------------------
-  auto consume_window = [&](const StreamSegment &sg, int wtile, uint32_t stage_addr) {
+  auto consume_window = [&](int wtile, uint32_t stage_addr) {
     const uint32_t Kst = stage_addr, Vst = stage_addr + kTileKV;
-    const int64_t lim64 = t < int64_t(sg.cap) ? t : int64_t(sg.cap);
-    const int end = int(lim64);
-    const int cur = int(t % int64_t(sg.cap));
     const int slot0 = wtile * kTileRows;
-    const bool ragged = slot0 + kTileRows > end || (cur >= slot0 && cur < slot0 + kTileRows);
+    const bool ragged = slot0 + kTileRows > win_end || (win_cur >= slot0 && win_cur < slot0 + kTileRows);
     if (ragged) {   // rows that are not window tokens get zero V so that 0 * garbage cannot make a NaN
       for (int r = 0; r < kTileRows; ++r) {
         const int s = slot0 + r;
-        if ((s >= end || s == cur) && lane < 16)
+        if ((s >= win_end || s == win_cur) && lane < 16)
           *reinterpret_cast<uint4 *>(__cvta_shared_to_generic(Vst + (lane >> 3) * kBoxBytes + r * 128 + (lane & 7) * 16)) =
               make_uint4(0u, 0u, 0u, 0u);
       }
+      fence_async_smem();   // these generic-proxy writes precede the next async-proxy fill of the stage
       __syncwarp();
     }
-    float s[4] = {0.f, 0.f, 0.f, 0.f};
+    float s[4] = {0.f, 0.f, 0.f, 0.f}, s2[4] = {0.f, 0.f, 0.f, 0.f};   // two chains over the feature dimension
     {
       const int r = (lane & 7) + ((lane >> 3) & 1) * 8;
 #pragma unroll
-      for (int ks = 0; ks < KS; ++ks) {
+      for (int ks = 0; ks < KS; ks += 2) {
         const int c = (ks & 3) * 2 + (lane >> 4);
-        uint32_t af[4];
+        uint32_t af[4], ag[4];
         ldmatrix_x4(af, Kst + (ks >> 2) * kBoxBytes + r * 128 + ((c ^ (r & 7)) << 4));
+        ldmatrix_x4(ag, Kst + (ks >> 2) * kBoxBytes + r * 128 + (((c + 2) ^ (r & 7)) << 4));
         mma_bf16(s, af, qb[ks]);
+        mma_bf16(s2, ag, qb[ks + 1]);
       }
     }
 #pragma unroll
-    for (int i = 0; i < 4; ++i) s[i] *= p.scale_log2;
+    for (int i = 0; i < 4; ++i) s[i] = (s[i] + s2[i]) * p.scale_log2;
     if (ragged) {
       const int k0 = slot0 + hrow, k1 = k0 + 8;
-      if (k0 >= end || k0 == cur) s[0] = s[1] = -CUDART_INF_F;
-      if (k1 >= end || k1 == cur) s[2] = s[3] = -CUDART_INF_F;
+      if (k0 >= win_end || k0 == win_cur) s[0] = s[1] = -CUDART_INF_F;
+      if (k1 >= win_end || k1 == win_cur) s[2] = s[3] = -CUDART_INF_F;
     }
     const float mx0 = quad_col_max(fmaxf(s[0], s[2]));
     const float mx1 = quad_col_max(fmaxf(s[1], s[3]));
     const float mn0 = fmaxf(m0, mx0), mn1 = fmaxf(m1, mx1);
-    if (__any_sync(0xffffffffu, mn0 != m0 || mn1 != m1)) {
-      const float c0 = mn0 == -CUDART_INF_F ? 1.f : exp2f(m0 - mn0);
-      const float c1 = mn1 == -CUDART_INF_F ? 1.f : exp2f(m1 - mn1);
+    if (mn0 != m0 || mn1 != m1) {   // lanes of one head column agree; columns may diverge
+      const float c0 = mn0 == -CUDART_INF_F ? 1.f : ex2_approx(m0 - mn0);
+      const float c1 = mn1 == -CUDART_INF_F ? 1.f : ex2_approx(m1 - mn1);
       l0 *= c0;
       l1 *= c1;
 #pragma unroll
@@ -402,11 +493,12 @@ glide_decode_stream_kernel(const DecodeParams p, const StreamParams sp) {
       m0 = mn0;
       m1 = mn1;
     }
+    __syncwarp();
     const float ms0 = m0 == -CUDART_INF_F ? 0.f : m0, ms1 = m1 == -CUDART_INF_F ? 0.f : m1;
     float p0, p1, p2, p3;
     uint32_t pb[2];
-    pb[0] = pack_bf16(exp2f(s[0] - ms0), exp2f(s[1] - ms1), p0, p1);
-    pb[1] = pack_bf16(exp2f(s[2] - ms0), exp2f(s[3] - ms1), p2, p3);
+    pb[0] = pack_bf16(ex2_approx(s[0] - ms0), ex2_approx(s[1] - ms1), p0, p1);
+    pb[1] = pack_bf16(ex2_approx(s[2] - ms0), ex2_approx(s[3] - ms1), p2, p3);
     l0 += p0 + p2;   // the row sum uses the weights as the tensor core sees them
     l1 += p1 + p3;
     pb[0] = movmatrix_trans(pb[0]);
@@ -425,14 +517,14 @@ glide_decode_stream_kernel(const DecodeParams p, const StreamParams sp) {
   };
 
   // ---- state tile: 16 rows of S and z, updated in place and read out ------------------------------
-  auto consume_state = [&](const StreamSegment &sg, int stile, uint32_t stage_addr, uint32_t z_addr) {
+  auto consume_state = [&](const StreamSegment &sg, int stile, const float4 *st, const float *zs) {
     float *Sg = reinterpret_cast<float *>(p.ws + size_t(sg.S_off256) * 256) + size_t(stile) * kTileRows * kD;
     float *zg = reinterpret_cast<float *>(p.ws + size_t(sg.z_off256) * 256) + stile * kTileRows;
     const int src0 = stile * 4;   // lane that holds phi entries of the tile's first row (4 rows per lane)
 #pragma unroll
     for (int r = 0; r < kTileRows; ++r) {
-      float4 s = lds_f32x4(stage_addr + r * (kD * 4) + lane * 16);
-      const float pk = __shfl_sync(0xffffffffu, phik[r & 3], src0 + (r >> 2));
+      float4 s = st[r * (kD / 4) + lane];
+      const float pk = __shfl_sync(0xffffffffu, phi[G][r & 3], src0 + (r >> 2));
       s.x = fmaf(pk, ve[0], s.x);
       s.y = fmaf(pk, ve[1], s.y);
       s.z = fmaf(pk, ve[2], s.z);
@@ -440,7 +532,7 @@ glide_decode_stream_kernel(const DecodeParams p, const StreamParams sp) {
       *reinterpret_cast<float4 *>(Sg + r * kD + lane * 4) = s;
 #pragma unroll
       for (int h = 0; h < G; ++h) {
-        const float f = __shfl_sync(0xffffffffu, phiq[h][r & 3], src0 + (r >> 2));
+        const float f = __shfl_sync(0xffffffffu, phi[h][r & 3], src0 + (r >> 2));
         a[h].x = fmaf(f, s.x, a[h].x);
         a[h].y = fmaf(f, s.y, a[h].y);
         a[h].z = fmaf(f, s.z, a[h].z);
@@ -449,32 +541,30 @@ glide_decode_stream_kernel(const DecodeParams p, const StreamParams sp) {
     }
     // z: lane r < 16 owns row r of the tile
     const int zsrc = src0 + ((lane & 15) >> 2);
-    float pkz = 0.f;
-#pragma unroll
-    for (int j = 0; j < 4; ++j) {
-      const float v = __shfl_sync(0xffffffffu, phik[j], zsrc);
-      if ((lane & 3) == j) pkz = v;
-    }
     float zn = 0.f;
-    if (lane < 16) {
-      zn = lds_f32(z_addr + lane * 4) + pkz;
-      zg[lane] = zn;
-    }
 #pragma unroll
-    for (int h = 0; h < G; ++h) {
-      float fz = 0.f;
+    for (int h = 0; h <= G; ++h) {
+      float f = 0.f;
 #pragma unroll
       for (int j = 0; j < 4; ++j) {
-        const float v = __shfl_sync(0xffffffffu, phiq[h][j], zsrc);
-        if ((lane & 3) == j) fz = v;
+        const float v = __shfl_sync(0xffffffffu, phi[(h + G) % (G + 1)][j], zsrc);   // phi(k_e) first, then the heads
+        if ((lane & 3) == j) f = v;
       }
-      if (lane < 16) bp[h] = fmaf(fz, zn, bp[h]);
+      if (h == 0) {
+        if (lane < 16) {
+          zn = zs[lane] + f;
+          zg[lane] = zn;
+        }
+      } else if (lane < 16) {
+        bp[h - 1] = fmaf(f, zn, bp[h - 1]);
+      }
     }
     had_state = true;
   };
 
   // ---- end of a segment: reduce the 8 warps, finish or hand over the unit -----------------------------
   auto flush = [&](int s) {
+    GLIDE_TRACE_EVENT(6);
     const StreamSegment &sg = sm_segs[s];
     float *rec = sm_rec + warp * L::kRecFloats;
     const bool mine = acc_seg == s;
@@ -505,18 +595,22 @@ glide_decode_stream_kernel(const DecodeParams p, const StreamParams sp) {
       }
       __syncwarp();
       if (had_state) {   // fold the linear readout in as a term with logit 0
-        float mh[G], lh[G];
+        float mh[G], lh[G], bs[G];
 #pragma unroll
         for (int h = 0; h < G; ++h) {
           mh[h] = rec[G * kD + h];
           lh[h] = rec[G * kD + G + h];
+          bs[h] = bp[h];
         }
+#pragma unroll
+        for (int o2 = 16; o2 > 0; o2 >>= 1)
+#pragma unroll
+          for (int h = 0; h < G; ++h) bs[h] += __shfl_xor_sync(0xffffffffu, bs[h], o2);
         __syncwarp();
 #pragma unroll
         for (int h = 0; h < G; ++h) {
-          const float bs = warp_sum(bp[h]);
           const float mn = fmaxf(mh[h], 0.f);
-          const float fo = exp2_or_zero(mh[h], mn), fl = exp2f(-mn);
+          const float fo = exp2_or_zero(mh[h], mn), fl = ex2_approx(-mn);
           float4 *ap = reinterpret_cast<float4 *>(rec + h * kD + lane * 4);
           float4 v = *ap;
           v.x = fmaf(v.x, fo, a[h].x * fl);
@@ -526,7 +620,7 @@ glide_decode_stream_kernel(const DecodeParams p, const StreamParams sp) {
           *ap = v;
           if (lane == 0) {
             rec[G * kD + h] = mn;
-            rec[G * kD + G + h] = fmaf(lh[h], fo, bs * fl);
+            rec[G * kD + G + h] = fmaf(lh[h], fo, bs[h] * fl);
           }
         }
       }
@@ -539,8 +633,9 @@ glide_decode_stream_kernel(const DecodeParams p, const StreamParams sp) {
     }
     // the current token's own logit, one head per warp (needed by whoever finishes the unit)
     const unsigned char *hdr = sm_hdr + size_t(s % kHdrSlots) * L::kHdrBytes;
-    if (warp < G && sg.cap > 0) {
-      if (acc_seg != s) wait_header(s);
+    const bool has_win = sg.cap > 0;
+    if (warp < G && has_win) {
+      if (!mine) wait_header(s);
       float qx[4], kx[4];
       load_elems<bf16, 4>(reinterpret_cast<const bf16 *>(hdr) + warp * kD + lane * 4, qx);
       load_elems<bf16, 4>(reinterpret_cast<const bf16 *>(hdr + G * 256 + 512) + lane * 4, kx);
@@ -561,12 +656,16 @@ glide_decode_stream_kernel(const DecodeParams p, const StreamParams sp) {
 #pragma unroll
     for (int i = 0; i < VPT; ++i) val[i] = 0.f;
     if (active) {
+      float mw[kWarps];
 #pragma unroll
-      for (int w = 0; w < kWarps; ++w) M = fmaxf(M, sm_rec[w * L::kRecFloats + G * kD + h]);
+      for (int w = 0; w < kWarps; ++w) {
+        mw[w] = sm_rec[w * L::kRecFloats + G * kD + h];
+        M = fmaxf(M, mw[w]);
+      }
 #pragma unroll
       for (int w = 0; w < kWarps; ++w) {
         const float *r = sm_rec + w * L::kRecFloats;
-        const float f = exp2_or_zero(r[G * kD + h], M);
+        const float f = exp2_or_zero(mw[w], M);
         lsum = fmaf(r[G * kD + G + h], f, lsum);
 #pragma unroll
         for (int i = 0; i < VPT; ++i) val[i] = fmaf(r[idx0 + i], f, val[i]);
@@ -574,21 +673,26 @@ glide_decode_stream_kernel(const DecodeParams p, const StreamParams sp) {
     }
     const int ub = sg.unit - sg.layer * units_per_layer;
     const int b = ub / p.Hkv, g = ub - b * p.Hkv;
-    const bool has_win = sg.cap > 0;
+    float scur_all[G];   // warp 0 may finish the unit after barrier B, when sm_scur is being rewritten
+#pragma unroll
+    for (int hh = 0; hh < G; ++hh) scur_all[hh] = has_win ? sm_scur[hh] : -CUDART_INF_F;
 
-    // finishes the unit from records (Mr, lr, vr): adds the current token, normalises, writes, appends
-    auto finish = [&](float Mr, float lr, const float (&vr)[VPT]) {
+    if (sg.part < 0) {
+      // the whole unit lives in this CTA: add the current token, normalise, write, append to the ring
       if (active) {
-        const float sc = has_win ? sm_scur[h] : -CUDART_INF_F;
-        const float Mf = fmaxf(fmaxf(Mr, sc), 0.f);
-        const float fr = exp2_or_zero(Mr, Mf), fc = exp2_or_zero(sc, Mf);
-        const float inv = 1.0f / fmaf(lr, fr, fc);
+        float sc = -CUDART_INF_F;
+#pragma unroll
+        for (int hh = 0; hh < G; ++hh)
+          if (hh == h) sc = scur_all[hh];
+        const float Mf = fmaxf(fmaxf(M, sc), 0.f);
+        const float fr = exp2_or_zero(M, Mf), fc = exp2_or_zero(sc, Mf);
+        const float inv = 1.0f / fmaf(lsum, fr, fc);
         const bf16 *vt = reinterpret_cast<const bf16 *>(hdr + G * 256 + 768);
         const int head = p.heads_of[g * G + h];
         bf16 *op = reinterpret_cast<bf16 *>(p.out) + ((size_t(sg.layer) * p.B + b) * p.H + head) * kD + c;
 #pragma unroll
         for (int i = 0; i < VPT; ++i) {
-          const float num = fmaf(vr[i], fr, has_win ? fc * __bfloat162float(vt[c + i]) : 0.f);
+          const float num = fmaf(val[i], fr, has_win ? fc * __bfloat162float(vt[c + i]) : 0.f);
           op[i] = __float2bfloat16_rn(num * inv);
         }
       }
@@ -599,72 +703,102 @@ glide_decode_stream_kernel(const DecodeParams p, const StreamParams sp) {
         uint32_t *dstw = reinterpret_cast<uint32_t *>(reinterpret_cast<bf16 *>(p.ws + (tid < 64 ? ld.ringK : ld.ringV)) + row);
         dstw[tid & 63] = srcw[tid];
       }
-    };
-
-    if (sg.part < 0) {
-      finish(M, lsum, val);
-    } else {
-      // unit cut by a CTA boundary: one global record per CTA, the last ticket merges
+    } else if (active) {
+      // unit cut by a CTA boundary: one global record per CTA
       float *grec = p.partials + (size_t(sg.rec0) + sg.part) * p.rec_floats;
-      if (active) {
 #pragma unroll
-        for (int i = 0; i < VPT; ++i) grec[idx0 + i] = val[i];
-        if (c == 0) {
-          grec[G * kD + h] = M;
-          grec[G * kD + G + h] = lsum;
-        }
-      }
-      __threadfence();
-      __syncthreads();
-      if (tid == 0) sm_flag[0] = atomicAdd(&p.tickets[sg.unit], 1) == sg.n_parts - 1;
-      __syncthreads();
-      if (sm_flag[0]) {
-        __threadfence();
-        float Mg = -CUDART_INF_F, lg = 0.f, vg[VPT];
-#pragma unroll
-        for (int i = 0; i < VPT; ++i) vg[i] = 0.f;
-        if (active) {
-          const float *r0 = p.partials + size_t(sg.rec0) * p.rec_floats;
-          for (int i = 0; i < sg.n_parts; ++i) Mg = fmaxf(Mg, __ldcg(r0 + size_t(i) * p.rec_floats + G * kD + h));
-          for (int i = 0; i < sg.n_parts; ++i) {
-            const float *r = r0 + size_t(i) * p.rec_floats;
-            const float f = exp2_or_zero(__ldcg(r + G * kD + h), Mg);
-            lg = fmaf(__ldcg(r + G * kD + G + h), f, lg);
-#pragma unroll
-            for (int j = 0; j < VPT; ++j) vg[j] = fmaf(__ldcg(r + idx0 + j), f, vg[j]);
-          }
-        }
-        finish(Mg, lg, vg);
-        if (tid == 0) p.tickets[sg.unit] = 0;
+      for (int i = 0; i < VPT; ++i) grec[idx0 + i] = val[i];
+      if (c == 0) {
+        grec[G * kD + h] = M;
+        grec[G * kD + G + h] = lsum;
       }
     }
-    __syncthreads();   // B: record area, logits, flag and this header slot may be reused
+    __syncthreads();   // B: record area and logits may be rewritten; the CTA's global record is complete
+
+    if (sg.part >= 0 && warp == 0) {
+      // Warp 0 takes the unit's ticket while the other warps go on; the last ticket merges the few records.
+      int last = 0;
+      if (lane == 0) {
+        __threadfence();
+        last = atomicAdd(&p.tickets[sg.unit], 1) == sg.n_parts - 1;
+      }
+      last = __shfl_sync(0xffffffffu, last, 0);
+      if (last) {
+        __threadfence();
+        const float *r0 = p.partials + size_t(sg.rec0) * p.rec_floats;
+        const bf16 *vt = reinterpret_cast<const bf16 *>(hdr + G * 256 + 768);
+#pragma unroll
+        for (int hh = 0; hh < G; ++hh) {
+          float Mg = fmaxf(scur_all[hh], 0.f);
+          for (int i = 0; i < sg.n_parts; ++i) Mg = fmaxf(Mg, __ldcg(r0 + size_t(i) * p.rec_floats + G * kD + hh));
+          float lg = 0.f;
+          float4 vg = make_float4(0.f, 0.f, 0.f, 0.f);
+          for (int i = 0; i < sg.n_parts; ++i) {
+            const float *r = r0 + size_t(i) * p.rec_floats;
+            const float f = exp2_or_zero(__ldcg(r + G * kD + hh), Mg);
+            lg = fmaf(__ldcg(r + G * kD + G + hh), f, lg);
+            const float4 av = __ldcg(reinterpret_cast<const float4 *>(r + hh * kD + lane * 4));
+            vg.x = fmaf(av.x, f, vg.x);
+            vg.y = fmaf(av.y, f, vg.y);
+            vg.z = fmaf(av.z, f, vg.z);
+            vg.w = fmaf(av.w, f, vg.w);
+          }
+          const float fc = exp2_or_zero(scur_all[hh], Mg);
+          const float inv = 1.0f / (lg + fc);
+          float vx[4] = {0.f, 0.f, 0.f, 0.f};
+          if (has_win) load_elems<bf16, 4>(vt + lane * 4, vx);
+          const int head = p.heads_of[g * G + hh];
+          const __nv_bfloat162 lo = __floats2bfloat162_rn(fmaf(fc, vx[0], vg.x) * inv, fmaf(fc, vx[1], vg.y) * inv);
+          const __nv_bfloat162 hi = __floats2bfloat162_rn(fmaf(fc, vx[2], vg.z) * inv, fmaf(fc, vx[3], vg.w) * inv);
+          uint2 packed;
+          packed.x = *reinterpret_cast<const uint32_t *>(&lo);
+          packed.y = *reinterpret_cast<const uint32_t *>(&hi);
+          *reinterpret_cast<uint2 *>(reinterpret_cast<bf16 *>(p.out) + ((size_t(sg.layer) * p.B + b) * p.H + head) * kD + lane * 4) = packed;
+        }
+        if (has_win) {
+          const LayerDev &ld = p.layers[sg.layer];
+          const size_t row = (size_t(sg.row_base) + size_t(t % int64_t(sg.cap))) * kD;
+          const uint2 *srcw = reinterpret_cast<const uint2 *>(hdr + G * 256 + 512);
+          reinterpret_cast<uint2 *>(reinterpret_cast<bf16 *>(p.ws + ld.ringK) + row)[lane] = srcw[lane];
+          reinterpret_cast<uint2 *>(reinterpret_cast<bf16 *>(p.ws + ld.ringV) + row)[lane] = srcw[32 + lane];
+        }
+        if (lane == 0) p.tickets[sg.unit] = 0;
+      }
+    }
+    GLIDE_TRACE_EVENT(7);
   };
 
   // ---- main loop --------------------------------------------------------------------------------------
-  Cursor ccur{warp, 0};
+  Cursor ccur;
+  ccur.i = warp;
+  ccur.seg = 0;
+  ccur.tile_end = 0;
+  if (nseg > 0) cursor_load(ccur, sm_segs, t);
   int next_flush = 0;
   TileRef ref;
   while (next_tile(ccur, sm_segs, nseg, ntiles, t, ref)) {
     while (next_flush < ref.seg) flush(next_flush++);
     if (acc_seg != ref.seg) load_unit(ref.seg);
-    const int stage = n_consumed % STAGES;
+    if (ref.is_state && !phi_ready) load_phi(ref.seg);
     if (!failed && !mbar_wait(my_bars + stage * 8, (phases >> stage) & 1u)) failed = true;
     phases ^= 1u << stage;
     failed = __any_sync(0xffffffffu, failed);
+    GLIDE_TRACE_EVENT(ref.is_state ? 4 : 3);
     if (!failed) {
-      const StreamSegment &sg = sm_segs[ref.seg];
       if (ref.is_state)
-        consume_state(sg, ref.index, my_stages + stage * kStageBytes, my_z + stage * 64);
+        consume_state(sm_segs[ref.seg], ref.index, reinterpret_cast<const float4 *>(my_stages_ptr + stage * kStageBytes),
+                      my_z_ptr + stage * 16);
       else
-        consume_window(sg, ref.index, my_stages + stage * kStageBytes);
+        consume_window(ref.index, my_stages + stage * kStageBytes);
     }
-    ++n_consumed;
+    stage = stage + 1 == STAGES ? 0 : stage + 1;
     __syncwarp();   // every lane is done with the stage before it is refilled
     if (!failed) issue_next();
+    GLIDE_TRACE_EVENT(5);
   }
   while (next_flush < nseg) flush(next_flush++);
   if (failed && lane == 0) atomicExch(&p.ctl->status, kDevWaitTimeout);
+  GLIDE_TRACE_EVENT(9);
 
   __syncthreads();
   if (tid == 0) {
@@ -683,7 +817,7 @@ size_t stream_smem_bytes(int max_segs) {
   using L = Layout<G>;
   return 1024 + size_t(kWarps) * STAGES * kStageBytes + size_t(kWarps) * L::kRecFloats * 4 + size_t(kHdrSlots) * L::kHdrBytes +
          size_t(kWarps) * STAGES * 64 + size_t(max_segs) * sizeof(StreamSegment) + size_t(kWarps * STAGES + kHdrSlots) * 8 +
-         8 * 4 + 4 * 4;
+         8 * 4;
 }
 
 template <typename F>
@@ -828,6 +962,12 @@ int stream_decode_setup(glide_ctx *ctx) {
   });
 }
 
+#ifdef GLIDE_TRACE
+extern "C" int glide_debug_set_stream_trace(void *dev_buf) {
+  return cudaMemcpyToSymbol(g_stream_trace, &dev_buf, sizeof(void *)) == cudaSuccess ? 0 : 6;
+}
+#endif
+
 int launch_decode_stream(glide_ctx *ctx, const DecodeParams &p, cudaStream_t stream) {
   StreamParams sp{};
   sp.segs = reinterpret_cast<const StreamSegment *>(ctx->ws + ctx->off_stream_segs);
@@ -835,6 +975,7 @@ int launch_decode_stream(glide_ctx *ctx, const DecodeParams &p, cudaStream_t str
   sp.tmaps = reinterpret_cast<const CUtensorMap_st *>(ctx->ws + ctx->off_tmaps);
   sp.max_segs = ctx->stream_max_segs;
   sp.heads_contiguous = ctx->stream_heads_contiguous ? 1 : 0;
+  sp.kv4d = ctx->tmaps_kv4d ? 1 : 0;
   return dispatch_stream(ctx->G, [&](auto gg, auto ss) -> int {
     constexpr int G = decltype(gg)::value, S = decltype(ss)::value;
     glide_decode_stream_kernel<G, S><<<ctx->decode_grid, kThreads, ctx->stream_smem, stream>>>(p, sp);

@@ -126,7 +126,7 @@ int glide::plan_context(const glide_config *cfg, glide_ctx *ctx, std::vector<Wor
   ctx->off_stream_cta = off;
   off = align_up(off + sizeof(int32_t) * (kMaxStreamCtas + 1), 256);
   ctx->off_tmaps = off;
-  off = align_up(off + size_t(128) * 2 * L, 256);
+  off = align_up(off + size_t(128) * 3 * L, 256);
   ctx->off_phik = off;
   off = align_up(off + sizeof(float) * size_t(L) * units_per_layer * ctx->prefill_chunk * d, 256);
   ctx->off_state = off;

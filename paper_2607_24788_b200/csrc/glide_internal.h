@@ -90,9 +90,10 @@ static_assert(sizeof(StreamSegment) == 64, "StreamSegment is copied as 16-byte c
 struct StreamParams {
   const StreamSegment *segs;
   const int32_t *cta_seg_begin;    // [grid + 1]
-  const struct CUtensorMap_st *tmaps;   // [2 L]: K ring, V ring per layer
+  const struct CUtensorMap_st *tmaps;   // [3 L]: K ring, V ring (2-D), K+V ring (4-D) per layer
   int32_t max_segs;
   int32_t heads_contiguous;
+  int32_t kv4d;                    // the 4-D K+V map exists: one TMA per window tile
 };
 
 struct PrefillParams {
@@ -128,6 +129,7 @@ struct glide_ctx {
   std::vector<int32_t> stream_cta_begin;
   int stream_max_segs = 0;
   bool stream_heads_contiguous = true;
+  bool tmaps_kv4d = false;
   size_t stream_smem = 0;
   size_t stream_seg_capacity = 0, stream_rec_capacity = 0;
   size_t off_stream_segs = 0, off_stream_cta = 0;
