@@ -4,20 +4,21 @@
 // (unit = layer x sequence x KV head, largest first):
 //   state tile  -- 16 rows of the unit's S (8 KiB fp32) plus the 16 matching z entries,
 //   window tile -- 16 ring slots: a 16x128 bf16 K box and V box (8 KiB).
-// The host cuts the stream into one contiguous, equally heavy range per CTA (one CTA per SM) and
-// describes it by a short segment list (one segment per unit the range touches).  Inside a CTA tile
-// i of the range belongs to warp i mod 8.  Every warp owns a ring of TMA stages and keeps it full
-// ACROSS unit boundaries: lane 0 issues cp.async.bulk(.tensor) loads for the warp's next tiles as
-// stages drain, so the memory pipe never empties while a unit is being finished.
+// The host cuts the stream into one contiguous, equally heavy range per WARP (8 warps per CTA, one
+// CTA per SM) and describes each range by a short segment list (one segment per unit it touches).
+// A warp is an autonomous worker: it owns a ring of TMA stages and keeps it full ACROSS unit
+// boundaries (lane 0 issues cp.async.bulk / cp.async.bulk.tensor loads as stages drain), and a small
+// header buffer into which the next unit's q rows, evicted k/v rows and current k/v rows are
+// prefetched while the current unit streams.  There is no CTA-wide barrier after set-up.
 //   window tile: S = K_tile Q^T on the tensor cores (keys on M, query heads on N), online softmax
 //                in the log2 domain, P transposed in registers, O^T += V_tile^T P;
 //   state tile:  S += phi(k_e) v_e^T and z += phi(k_e) in place (fp32), readout phi(q_h)^T S, phi(q_h)^T z.
-// The linear readout is folded into the warp's softmax partial as a term with logit 0 (exact: the
-// shared normaliser's reference m* is max(window max, 0)), so a unit needs ONE (m, l, acc) record per
-// warp.  When a unit's segment ends the 8 warps reduce their records in shared memory; a unit that
-// lies inside one CTA is finished right there (current token's own term, normalise, write, ring
-// append) without touching global scratch.  Only units cut by a CTA boundary go through one global
-// record per CTA and a ticket; the last CTA merges those few records.  No CTA waits for another.
+// The linear readout is folded into the softmax partial as a term with logit 0 (exact: the shared
+// normaliser's reference m* is max(window max, 0)), so a unit needs ONE (m, l, acc) record per warp.
+// A unit that lies inside one warp's range is finished by that warp alone (current token's own term,
+// normalise, write, ring append) without touching global scratch.  Only units cut by a range boundary
+// go through one global record per warp and a ticket; the warp holding the last ticket merges them.
+// No warp waits for another warp; the only waits are on the warp's own mbarriers, and are bounded.
 #include <cuda.h>
 
 #include <algorithm>
@@ -162,58 +163,25 @@ __device__ __forceinline__ void tma_load_4d(uint32_t dst, const void *tmap, int 
 __device__ __forceinline__ bool seg_evicting(const StreamSegment &s, int64_t t) {
   return s.evicts && (s.w == 0 || t >= int64_t(s.w));
 }
-
-// A warp's position in the CTA's tile range with the fields of its current segment cached in registers.
-struct Cursor {
-  int i;         // CTA-relative index of this warp's next candidate tile
-  int seg;       // segment that holds it
-  int tile0, tile_end, n_state, state0, win0;
-  int n_valid_win;   // window tiles of the segment that hold window tokens at this position
-  int evicting;
-};
-struct TileRef {
-  int seg;
-  int index;     // state tile (rows 16*index ..) or window tile (slots 16*index ..) within the unit
-  bool is_state;
-};
-
-__device__ __forceinline__ void cursor_load(Cursor &c, const StreamSegment *segs, int64_t t) {
-  const StreamSegment &s = segs[c.seg];
-  c.tile0 = s.tile0;
-  c.n_state = s.n_state;
-  c.state0 = s.state0;
-  c.win0 = s.win0;
-  c.tile_end = s.tile0 + s.n_state + s.n_win;
+// window tiles of the segment that hold window tokens at position t
+__device__ __forceinline__ int seg_valid_win(const StreamSegment &s, int64_t t) {
   const int64_t lim = t < int64_t(s.cap) ? t : int64_t(s.cap);
-  int nv = int((lim + kTileRows - 1) / kTileRows) - s.win0;
-  c.n_valid_win = nv < 0 ? 0 : (nv > s.n_win ? s.n_win : nv);
-  c.evicting = seg_evicting(s, t) ? 1 : 0;
+  const int nv = int((lim + kTileRows - 1) / kTileRows) - s.win0;
+  return nv < 0 ? 0 : (nv > s.n_win ? s.n_win : nv);
 }
 
-// Next tile of this warp that has work; the issuing lane and the consuming warp walk the same sequence.
-__device__ __forceinline__ bool next_tile(Cursor &c, const StreamSegment *segs, int nseg, int ntiles, int64_t t,
-                                          TileRef &ref) {
-  while (c.i < ntiles) {
-    if (c.i >= c.tile_end) {
-      do { ++c.seg; } while (c.seg + 1 < nseg && c.i >= segs[c.seg].tile0 + segs[c.seg].n_state + segs[c.seg].n_win);
-      cursor_load(c, segs, t);
-    }
-    const int local = c.i - c.tile0;
-    bool valid;
-    if (local < c.n_state) {
-      ref.is_state = true;
-      ref.index = c.state0 + local;
-      valid = c.evicting != 0;
-    } else {
-      ref.is_state = false;
-      ref.index = c.win0 + local - c.n_state;
-      valid = local - c.n_state < c.n_valid_win;
-    }
-    ref.seg = c.seg;
-    c.i += kWarps;
-    if (valid) return true;
-  }
-  return false;
+// A position in the warp's range: segment, tile within the segment, and the segment's tile counts.
+struct Cursor {
+  int seg;
+  int k;          // next tile of the segment: [0, n_state_eff) state tiles, then window tiles
+  int n_state_eff, n_total;
+};
+
+__device__ __forceinline__ void cursor_enter(Cursor &c, const StreamSegment *segs, int64_t t) {
+  const StreamSegment &s = segs[c.seg];
+  c.k = 0;
+  c.n_state_eff = seg_evicting(s, t) ? s.n_state : 0;
+  c.n_total = c.n_state_eff + seg_valid_win(s, t);
 }
 
 template <int G>
@@ -254,6 +222,14 @@ __device__ __forceinline__ void warp_phi_multi(float (&x)[N][4]) {
   }
 }
 
+template <int N>
+__device__ __forceinline__ void warp_sum_multi(float (&x)[N]) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1)
+#pragma unroll
+    for (int n = 0; n < N; ++n) x[n] += __shfl_xor_sync(0xffffffffu, x[n], o);
+}
+
 // ---- the kernel -----------------------------------------------------------------------------
 template <int G, int STAGES>
 __global__ void __launch_bounds__(kThreads, 1)
@@ -261,17 +237,14 @@ glide_decode_stream_kernel(const DecodeParams p, const StreamParams sp) {
   using bf16 = __nv_bfloat16;
   using L = Layout<G>;
   constexpr int KS = kD / 16;
-  constexpr int VPT = (G * kD + kThreads - 1) / kThreads;   // combined values per thread at a flush
 
   extern __shared__ __align__(1024) unsigned char smem_raw[];
   unsigned char *base = reinterpret_cast<unsigned char *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   unsigned char *sm_stages = base;                                                  // [kWarps][STAGES][8 KiB]
-  float *sm_rec = reinterpret_cast<float *>(sm_stages + size_t(kWarps) * STAGES * kStageBytes);   // [kWarps][kRecFloats]
-  unsigned char *sm_hdr = reinterpret_cast<unsigned char *>(sm_rec + kWarps * L::kRecFloats);     // [3][kHdrBytes]
-  float *sm_z = reinterpret_cast<float *>(sm_hdr + kHdrSlots * L::kHdrBytes);                    // [kWarps][STAGES][16]
-  StreamSegment *sm_segs = reinterpret_cast<StreamSegment *>(sm_z + kWarps * STAGES * 16);      // [max_segs]
-  uint64_t *sm_bars = reinterpret_cast<uint64_t *>(sm_segs + sp.max_segs);                        // [kWarps*STAGES + 3]
-  float *sm_scur = reinterpret_cast<float *>(sm_bars + kWarps * STAGES + kHdrSlots);             // [8]
+  unsigned char *sm_hdr = sm_stages + size_t(kWarps) * STAGES * kStageBytes;        // [kWarps][kHdrBytes]
+  float *sm_z = reinterpret_cast<float *>(sm_hdr + kWarps * L::kHdrBytes);           // [kWarps][STAGES][16]
+  StreamSegment *sm_segs = reinterpret_cast<StreamSegment *>(sm_z + kWarps * STAGES * 16);   // [max_segs]
+  uint64_t *sm_bars = reinterpret_cast<uint64_t *>(sm_segs + sp.max_segs);          // [kWarps][STAGES + 1]
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 #ifdef GLIDE_TRACE
@@ -280,91 +253,95 @@ glide_decode_stream_kernel(const DecodeParams p, const StreamParams sp) {
   GLIDE_TRACE_EVENT(1);
   const int64_t t = p.n_dev[0];   // every layer is at the same position (checked by the host)
   const int col2 = (lane & 3) * 2, hrow = lane >> 2;
-  const int seg_begin = sp.cta_seg_begin[blockIdx.x];
-  const int nseg = sp.cta_seg_begin[blockIdx.x + 1] - seg_begin;
-  if (nseg > 0) {
-    const uint4 *src = reinterpret_cast<const uint4 *>(sp.segs + seg_begin);
+  const int range0 = blockIdx.x * kWarps;
+  const int cta_seg_begin = sp.range_seg_begin[range0];
+  const int cta_nseg = sp.range_seg_begin[range0 + kWarps] - cta_seg_begin;
+  const int seg_lo = sp.range_seg_begin[range0 + warp] - cta_seg_begin;       // this warp's segments in the CTA table
+  const int seg_hi = sp.range_seg_begin[range0 + warp + 1] - cta_seg_begin;
+  if (cta_nseg > 0) {
+    const uint4 *src = reinterpret_cast<const uint4 *>(sp.segs + cta_seg_begin);
     uint4 *dst = reinterpret_cast<uint4 *>(sm_segs);
-    for (int i = tid; i < nseg * int(sizeof(StreamSegment) / 16); i += kThreads) dst[i] = src[i];
+    for (int i = tid; i < cta_nseg * int(sizeof(StreamSegment) / 16); i += kThreads) dst[i] = src[i];
   }
-  const uint32_t my_stages = smem_u32(sm_stages + size_t(warp) * STAGES * kStageBytes);
   unsigned char *my_stages_ptr = sm_stages + size_t(warp) * STAGES * kStageBytes;
-  const uint32_t my_bars = smem_u32(sm_bars + warp * STAGES);
-  const uint32_t my_z = smem_u32(sm_z + warp * STAGES * 16);
+  const uint32_t my_stages = smem_u32(my_stages_ptr);
+  unsigned char *my_hdr_ptr = sm_hdr + size_t(warp) * L::kHdrBytes;
+  const uint32_t my_hdr = smem_u32(my_hdr_ptr);
   const float *my_z_ptr = sm_z + warp * STAGES * 16;
-  const uint32_t hdr_bars = smem_u32(sm_bars + kWarps * STAGES);
-  if (lane == 0)
-    for (int s = 0; s < STAGES; ++s) mbar_init(my_bars + s * 8, 1);
-  if (tid == 0)
-    for (int s = 0; s < kHdrSlots; ++s) mbar_init(hdr_bars + s * 8, 1);
-  asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-  fence_async_smem();
-  __syncthreads();
+  const uint32_t my_z = smem_u32(my_z_ptr);
+  const uint32_t my_bars = smem_u32(sm_bars + warp * (STAGES + 1));
+  const uint32_t hdr_bar = my_bars + STAGES * 8;
+  if (lane == 0) {
+    for (int s = 0; s <= STAGES; ++s) mbar_init(my_bars + s * 8, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    fence_async_smem();
+  }
+  __syncthreads();   // segment table and barriers ready; the warps are on their own from here
 
-  const int ntiles = nseg > 0 ? sm_segs[nseg - 1].tile0 + sm_segs[nseg - 1].n_state + sm_segs[nseg - 1].n_win : 0;
   const int units_per_layer = p.B * p.Hkv;
   bool failed = false;
 
-  // ---- header (q rows, evicted k/v, current k/v) of segment s -> slot s % 3, issued by thread 0 -----
+  // ---- header of segment s (q rows | k_e | v_e | k_t | v_t) into this warp's buffer, lane 0 ---------
   auto issue_header = [&](int s) {
-    const StreamSegment &sg = sm_segs[s];
-    const uint32_t bar = hdr_bars + (s % kHdrSlots) * 8;
-    const uint32_t dst = smem_u32(sm_hdr + size_t(s % kHdrSlots) * L::kHdrBytes);
-    const bool ev = seg_evicting(sg, t);
-    const int ub = sg.unit - sg.layer * units_per_layer;
-    const int b = ub / p.Hkv, g = ub - b * p.Hkv;
-    mbar_expect_tx(bar, G * 256 + 512 + (ev ? 512 : 0));
-    const bf16 *qb = reinterpret_cast<const bf16 *>(p.q) + (size_t(sg.layer) * p.B + b) * p.H * kD;
-    if (sp.heads_contiguous) {
-      bulk_load(dst, qb + size_t(p.heads_of[g * G]) * kD, G * 256, bar);
-    } else {
-      for (int h = 0; h < G; ++h) bulk_load(dst + h * 256, qb + size_t(p.heads_of[g * G + h]) * kD, 256, bar);
-    }
-    const bf16 *kt = reinterpret_cast<const bf16 *>(p.k) + size_t(sg.unit) * kD;
-    const bf16 *vt = reinterpret_cast<const bf16 *>(p.v) + size_t(sg.unit) * kD;
-    bulk_load(dst + G * 256 + 512, kt, 256, bar);
-    bulk_load(dst + G * 256 + 768, vt, 256, bar);
-    if (ev) {
-      if (sg.w == 0) {   // no ring: the current token is the one folded into the state
-        bulk_load(dst + G * 256, kt, 256, bar);
-        bulk_load(dst + G * 256 + 256, vt, 256, bar);
+    if (lane == 0) {
+      const StreamSegment &sg = sm_segs[s];
+      const bool ev = seg_evicting(sg, t);
+      const int ub = sg.unit - sg.layer * units_per_layer;
+      const int b = ub / p.Hkv, g = ub - b * p.Hkv;
+      fence_async_smem();
+      mbar_expect_tx(hdr_bar, G * 256 + 512 + (ev ? 512 : 0));
+      const bf16 *qb = reinterpret_cast<const bf16 *>(p.q) + (size_t(sg.layer) * p.B + b) * p.H * kD;
+      if (sp.heads_contiguous) {
+        bulk_load(my_hdr, qb + size_t(p.heads_of[g * G]) * kD, G * 256, hdr_bar);
       } else {
-        const LayerDev &ld = p.layers[sg.layer];
-        const size_t row = (size_t(sg.row_base) + size_t(t % int64_t(sg.cap))) * kD;
-        bulk_load(dst + G * 256, reinterpret_cast<const bf16 *>(p.ws + ld.ringK) + row, 256, bar);
-        bulk_load(dst + G * 256 + 256, reinterpret_cast<const bf16 *>(p.ws + ld.ringV) + row, 256, bar);
+        for (int h = 0; h < G; ++h) bulk_load(my_hdr + h * 256, qb + size_t(p.heads_of[g * G + h]) * kD, 256, hdr_bar);
+      }
+      const bf16 *kt = reinterpret_cast<const bf16 *>(p.k) + size_t(sg.unit) * kD;
+      const bf16 *vt = reinterpret_cast<const bf16 *>(p.v) + size_t(sg.unit) * kD;
+      bulk_load(my_hdr + G * 256 + 512, kt, 256, hdr_bar);
+      bulk_load(my_hdr + G * 256 + 768, vt, 256, hdr_bar);
+      if (ev) {
+        if (sg.w == 0) {   // no ring: the current token is the one folded into the state
+          bulk_load(my_hdr + G * 256, kt, 256, hdr_bar);
+          bulk_load(my_hdr + G * 256 + 256, vt, 256, hdr_bar);
+        } else {
+          const LayerDev &ld = p.layers[sg.layer];
+          const size_t row = (size_t(sg.row_base) + size_t(t % int64_t(sg.cap))) * kD;
+          bulk_load(my_hdr + G * 256, reinterpret_cast<const bf16 *>(p.ws + ld.ringK) + row, 256, hdr_bar);
+          bulk_load(my_hdr + G * 256 + 256, reinterpret_cast<const bf16 *>(p.ws + ld.ringV) + row, 256, hdr_bar);
+        }
       }
     }
   };
-  if (tid == 0) {
-    if (nseg > 0) issue_header(0);
-    if (nseg > 1) issue_header(1);
-  }
+  if (seg_lo < seg_hi) issue_header(seg_lo);
 
-  // ---- tile issue (lane 0 of each warp) ---------------------------------------------------------
+  // ---- tile issue (lane 0) ------------------------------------------------------------------------
   Cursor icur;
-  icur.i = warp;
-  icur.seg = 0;
-  icur.tile_end = 0;
-  if (nseg > 0) cursor_load(icur, sm_segs, t);
+  icur.seg = seg_lo;
+  icur.k = icur.n_state_eff = icur.n_total = 0;
+  if (seg_lo < seg_hi) cursor_enter(icur, sm_segs, t);
   int issue_stage = 0;
   auto issue_next = [&]() {
     if (lane == 0) {
-      TileRef r;
-      if (next_tile(icur, sm_segs, nseg, ntiles, t, r)) {
-        const StreamSegment &sg = sm_segs[r.seg];
+      while (icur.seg < seg_hi && icur.k >= icur.n_total) {
+        if (++icur.seg < seg_hi) cursor_enter(icur, sm_segs, t);
+      }
+      if (icur.seg < seg_hi) {
+        const StreamSegment &sg = sm_segs[icur.seg];
         const uint32_t bar = my_bars + issue_stage * 8;
         const uint32_t dst = my_stages + issue_stage * kStageBytes;
-        if (r.is_state) {
+        if (icur.k < icur.n_state_eff) {
+          const int st = sg.state0 + icur.k;
           mbar_expect_tx(bar, kStageBytes + 64);
-          const float *Sg = reinterpret_cast<const float *>(p.ws + size_t(sg.S_off256) * 256) + size_t(r.index) * kTileRows * kD;
-          const float *zg = reinterpret_cast<const float *>(p.ws + size_t(sg.z_off256) * 256) + r.index * kTileRows;
+          const float *Sg = reinterpret_cast<const float *>(p.ws + size_t(sg.S_off256) * 256) + size_t(st) * kTileRows * kD;
+          const float *zg = reinterpret_cast<const float *>(p.ws + size_t(sg.z_off256) * 256) + st * kTileRows;
           bulk_load(dst, Sg, kStageBytes, bar);
           bulk_load(my_z + issue_stage * 64, zg, 64, bar);
         } else {
+          const int wt = sg.win0 + icur.k - icur.n_state_eff;
           mbar_expect_tx(bar, kStageBytes);
           const CUtensorMap *tk = reinterpret_cast<const CUtensorMap *>(sp.tmaps) + 3 * sg.layer;
-          const int y = sg.row_base + r.index * kTileRows;
+          const int y = sg.row_base + wt * kTileRows;
           if (sp.kv4d) {
             tma_load_4d(dst, tk + 2, 0, y, 0, 0, bar);   // K halves then V halves: [kv][half][row][64]
           } else {
@@ -374,6 +351,7 @@ glide_decode_stream_kernel(const DecodeParams p, const StreamParams sp) {
             tma_load_2d(dst + kTileKV + kBoxBytes, tk + 1, 64, y, bar);
           }
         }
+        ++icur.k;
         issue_stage = issue_stage + 1 == STAGES ? 0 : issue_stage + 1;
       }
     }
@@ -384,61 +362,16 @@ glide_decode_stream_kernel(const DecodeParams p, const StreamParams sp) {
   // ---- per-unit register state ------------------------------------------------------------------
   uint32_t qb[KS][2];
   float o[KS][4];
-  float m0 = -CUDART_INF_F, m1 = -CUDART_INF_F, l0 = 0.f, l1 = 0.f;
+  float m0, m1, l0, l1;
   float phi[G + 1][4];     // phi(q_h) for the G heads, then phi(k_e); lane holds entries 4*lane .. 4*lane+3
   float ve[4];
   float4 a[G];
   float bp[G];
-  bool had_state = false, phi_ready = false;
-  int acc_seg = -1;        // segment the accumulators belong to
+  float scur[G];           // the current token's own logit per head (log2 domain)
+  uint2 kt_bits, vt_bits;  // the current token's k and v entries 4*lane .. 4*lane+3 (bf16)
   int win_end = 0, win_cur = 0;   // window tokens live in slots [0, win_end) except slot win_cur
-  uint32_t phases = 0;     // parity expected by the next wait on each stage
+  uint32_t phases = 0;     // parity expected by the next wait on each stage; bit STAGES: header barrier
   int stage = 0;
-
-  auto wait_header = [&](int s) {
-    if (!mbar_wait(hdr_bars + (s % kHdrSlots) * 8, uint32_t(s / kHdrSlots) & 1u)) failed = true;
-  };
-
-  // q fragments of segment s into registers; accumulators cleared
-  auto load_unit = [&](int s) {
-    const StreamSegment &sg = sm_segs[s];
-    wait_header(s);
-    const uint32_t *hq = reinterpret_cast<const uint32_t *>(sm_hdr + size_t(s % kHdrSlots) * L::kHdrBytes);
-    const bool valid = hrow < G;
-#pragma unroll
-    for (int ks = 0; ks < KS; ++ks) {
-      qb[ks][0] = valid ? hq[hrow * 64 + ks * 8 + (lane & 3)] : 0u;
-      qb[ks][1] = valid ? hq[hrow * 64 + ks * 8 + 4 + (lane & 3)] : 0u;
-    }
-    if (sg.cap > 0) {
-      const int64_t lim = t < int64_t(sg.cap) ? t : int64_t(sg.cap);
-      win_end = int(lim);
-      win_cur = int(t % int64_t(sg.cap));
-    }
-#pragma unroll
-    for (int mt = 0; mt < KS; ++mt) o[mt][0] = o[mt][1] = o[mt][2] = o[mt][3] = 0.f;
-    m0 = m1 = -CUDART_INF_F;
-    l0 = l1 = 0.f;
-#pragma unroll
-    for (int h = 0; h < G; ++h) {
-      a[h] = make_float4(0.f, 0.f, 0.f, 0.f);
-      bp[h] = 0.f;
-    }
-    had_state = false;
-    phi_ready = false;
-    acc_seg = s;
-  };
-
-  // feature maps of the unit's queries and of the evicted key (first state tile of a segment only)
-  auto load_phi = [&](int s) {
-    const bf16 *h0 = reinterpret_cast<const bf16 *>(sm_hdr + size_t(s % kHdrSlots) * L::kHdrBytes);
-#pragma unroll
-    for (int h = 0; h < G; ++h) load_elems<bf16, 4>(h0 + h * kD + lane * 4, phi[h]);
-    load_elems<bf16, 4>(h0 + G * kD + lane * 4, phi[G]);
-    load_elems<bf16, 4>(h0 + (G + 1) * kD + lane * 4, ve);
-    warp_phi_multi<G + 1>(phi);
-    phi_ready = true;
-  };
 
   // ---- window tile ------------------------------------------------------------------------------
   auto consume_window = [&](int wtile, uint32_t stage_addr) {
@@ -559,244 +492,275 @@ glide_decode_stream_kernel(const DecodeParams p, const StreamParams sp) {
         bp[h - 1] = fmaf(f, zn, bp[h - 1]);
       }
     }
-    had_state = true;
   };
 
-  // ---- end of a segment: reduce the 8 warps, finish or hand over the unit -----------------------------
-  auto flush = [&](int s) {
-    GLIDE_TRACE_EVENT(6);
+  // ---- main loop over this warp's segments ------------------------------------------------------------
+  for (int s = seg_lo; s < seg_hi && !failed; ++s) {
     const StreamSegment &sg = sm_segs[s];
-    float *rec = sm_rec + warp * L::kRecFloats;
-    const bool mine = acc_seg == s;
-    // 1. this warp's record (m, l, acc) in shared memory
-    if (mine) {
+    const bool ev = seg_evicting(sg, t);
+    const int n_state_eff = ev ? sg.n_state : 0;
+    const int n_total = n_state_eff + seg_valid_win(sg, t);
+    const bool has_win = sg.cap > 0;
+
+    // -- header: q fragments, current token, feature maps -> registers; then prefetch the next header --
+    GLIDE_TRACE_EVENT(6);
+    if (!mbar_wait(hdr_bar, (phases >> STAGES) & 1u)) failed = true;
+    phases ^= 1u << STAGES;
+    if (__any_sync(0xffffffffu, failed)) {
+      failed = true;
+      break;
+    }
+    {
+      const uint32_t *hq = reinterpret_cast<const uint32_t *>(my_hdr_ptr);
+      const bool valid = hrow < G;
+#pragma unroll
+      for (int ks = 0; ks < KS; ++ks) {
+        qb[ks][0] = valid ? hq[hrow * 64 + ks * 8 + (lane & 3)] : 0u;
+        qb[ks][1] = valid ? hq[hrow * 64 + ks * 8 + 4 + (lane & 3)] : 0u;
+      }
+      const bf16 *h0 = reinterpret_cast<const bf16 *>(my_hdr_ptr);
+      kt_bits = *reinterpret_cast<const uint2 *>(h0 + (G + 2) * kD + lane * 4);
+      vt_bits = *reinterpret_cast<const uint2 *>(h0 + (G + 3) * kD + lane * 4);
+      float kx[4];
+      load_elems<bf16, 4>(h0 + (G + 2) * kD + lane * 4, kx);
+#pragma unroll
+      for (int h = 0; h < G; ++h) {
+        load_elems<bf16, 4>(h0 + h * kD + lane * 4, phi[h]);
+        scur[h] = 0.f;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) scur[h] = fmaf(phi[h][i], kx[i], scur[h]);
+      }
+      warp_sum_multi<G>(scur);
+#pragma unroll
+      for (int h = 0; h < G; ++h) scur[h] = has_win ? scur[h] * p.scale_log2 : -CUDART_INF_F;
+      if (n_state_eff > 0) {
+        load_elems<bf16, 4>(h0 + G * kD + lane * 4, phi[G]);
+        load_elems<bf16, 4>(h0 + (G + 1) * kD + lane * 4, ve);
+        warp_phi_multi<G + 1>(phi);
+      }
+    }
+    __syncwarp();
+    if (s + 1 < seg_hi) issue_header(s + 1);
+    if (has_win) {
+      const int64_t lim = t < int64_t(sg.cap) ? t : int64_t(sg.cap);
+      win_end = int(lim);
+      win_cur = int(t % int64_t(sg.cap));
+    }
+#pragma unroll
+    for (int mt = 0; mt < KS; ++mt) o[mt][0] = o[mt][1] = o[mt][2] = o[mt][3] = 0.f;
+    m0 = m1 = -CUDART_INF_F;
+    l0 = l1 = 0.f;
+#pragma unroll
+    for (int h = 0; h < G; ++h) {
+      a[h] = make_float4(0.f, 0.f, 0.f, 0.f);
+      bp[h] = 0.f;
+    }
+    GLIDE_TRACE_EVENT(7);
+
+    // -- tiles ------------------------------------------------------------------------------------------
+    int last_stage = -1;
+    for (int k = 0; k < n_total; ++k) {
+      if (!mbar_wait(my_bars + stage * 8, (phases >> stage) & 1u)) failed = true;
+      phases ^= 1u << stage;
+      if (__any_sync(0xffffffffu, failed)) {
+        failed = true;
+        break;
+      }
+      GLIDE_TRACE_EVENT(k < n_state_eff ? 4 : 3);
+      if (k < n_state_eff)
+        consume_state(sg, sg.state0 + k, reinterpret_cast<const float4 *>(my_stages_ptr + stage * kStageBytes),
+                      my_z_ptr + stage * 16);
+      else
+        consume_window(sg.win0 + k - n_state_eff, my_stages + stage * kStageBytes);
+      last_stage = stage;
+      stage = stage + 1 == STAGES ? 0 : stage + 1;
+      __syncwarp();   // every lane is done with the stage before it is refilled
+      if (k + 1 < n_total) issue_next();   // the last tile's stage first serves as scratch for the finish
+      GLIDE_TRACE_EVENT(5);
+    }
+    if (failed) break;
+
+    // -- finish: record (m, l, acc) in a common layout: lane holds features 4*lane..4*lane+3 of every head --
+    float mh[G], lh[G];
+    float4 acc[G];
+    if (n_total > n_state_eff) {   // window tiles were processed: move the accumulator fragments through the freed stage
+      float *scr = reinterpret_cast<float *>(my_stages_ptr + last_stage * kStageBytes);
       const float lq0 = quad_col_sum(l0), lq1 = quad_col_sum(l1);
 #pragma unroll
       for (int mt = 0; mt < KS; ++mt) {
         const int d0 = mt * 16 + hrow;
         if (col2 < G) {
-          rec[col2 * kD + d0] = o[mt][0];
-          rec[col2 * kD + d0 + 8] = o[mt][2];
+          scr[col2 * kD + d0] = o[mt][0];
+          scr[col2 * kD + d0 + 8] = o[mt][2];
         }
         if (col2 + 1 < G) {
-          rec[(col2 + 1) * kD + d0] = o[mt][1];
-          rec[(col2 + 1) * kD + d0 + 8] = o[mt][3];
+          scr[(col2 + 1) * kD + d0] = o[mt][1];
+          scr[(col2 + 1) * kD + d0 + 8] = o[mt][3];
         }
       }
       if (hrow == 0) {
         if (col2 < G) {
-          rec[G * kD + col2] = m0;
-          rec[G * kD + G + col2] = lq0;
+          scr[G * kD + col2] = m0;
+          scr[G * kD + G + col2] = lq0;
         }
         if (col2 + 1 < G) {
-          rec[G * kD + col2 + 1] = m1;
-          rec[G * kD + G + col2 + 1] = lq1;
+          scr[G * kD + col2 + 1] = m1;
+          scr[G * kD + G + col2 + 1] = lq1;
         }
       }
       __syncwarp();
-      if (had_state) {   // fold the linear readout in as a term with logit 0
-        float mh[G], lh[G], bs[G];
 #pragma unroll
-        for (int h = 0; h < G; ++h) {
-          mh[h] = rec[G * kD + h];
-          lh[h] = rec[G * kD + G + h];
-          bs[h] = bp[h];
-        }
-#pragma unroll
-        for (int o2 = 16; o2 > 0; o2 >>= 1)
-#pragma unroll
-          for (int h = 0; h < G; ++h) bs[h] += __shfl_xor_sync(0xffffffffu, bs[h], o2);
-        __syncwarp();
-#pragma unroll
-        for (int h = 0; h < G; ++h) {
-          const float mn = fmaxf(mh[h], 0.f);
-          const float fo = exp2_or_zero(mh[h], mn), fl = ex2_approx(-mn);
-          float4 *ap = reinterpret_cast<float4 *>(rec + h * kD + lane * 4);
-          float4 v = *ap;
-          v.x = fmaf(v.x, fo, a[h].x * fl);
-          v.y = fmaf(v.y, fo, a[h].y * fl);
-          v.z = fmaf(v.z, fo, a[h].z * fl);
-          v.w = fmaf(v.w, fo, a[h].w * fl);
-          *ap = v;
-          if (lane == 0) {
-            rec[G * kD + h] = mn;
-            rec[G * kD + G + h] = fmaf(lh[h], fo, bs[h] * fl);
-          }
-        }
+      for (int h = 0; h < G; ++h) {
+        mh[h] = scr[G * kD + h];
+        lh[h] = scr[G * kD + G + h];
+        acc[h] = *reinterpret_cast<const float4 *>(scr + h * kD + lane * 4);
       }
+      fence_async_smem();   // the stage is refilled by the async proxy next
+      __syncwarp();
     } else {
-      for (int i = lane; i < G * kD; i += 32) rec[i] = 0.f;
-      if (lane < G) {
-        rec[G * kD + lane] = -CUDART_INF_F;
-        rec[G * kD + G + lane] = 0.f;
+#pragma unroll
+      for (int h = 0; h < G; ++h) {
+        mh[h] = -CUDART_INF_F;
+        lh[h] = 0.f;
+        acc[h] = make_float4(0.f, 0.f, 0.f, 0.f);
       }
     }
-    // the current token's own logit, one head per warp (needed by whoever finishes the unit)
-    const unsigned char *hdr = sm_hdr + size_t(s % kHdrSlots) * L::kHdrBytes;
-    const bool has_win = sg.cap > 0;
-    if (warp < G && has_win) {
-      if (!mine) wait_header(s);
-      float qx[4], kx[4];
-      load_elems<bf16, 4>(reinterpret_cast<const bf16 *>(hdr) + warp * kD + lane * 4, qx);
-      load_elems<bf16, 4>(reinterpret_cast<const bf16 *>(hdr + G * 256 + 512) + lane * 4, kx);
-      float part = 0.f;
+    if (n_total > 0) issue_next();   // the deferred refill
+    if (n_state_eff > 0) {           // fold the linear readout in as a term with logit 0
+      warp_sum_multi<G>(bp);
 #pragma unroll
-      for (int i = 0; i < 4; ++i) part = fmaf(qx[i], kx[i], part);
-      part = warp_sum(part) * p.scale_log2;
-      if (lane == 0) sm_scur[warp] = part;
-    }
-    __syncthreads();   // A: records and logits visible
-    if (tid == 0 && s + 2 < nseg) issue_header(s + 2);   // slot of segment s-1, fully consumed before A
-
-    // 2. combine the 8 records: thread owns VPT consecutive features of one head
-    const int idx0 = tid * VPT;
-    const bool active = idx0 < G * kD;
-    const int h = active ? idx0 / kD : 0, c = idx0 - h * kD;
-    float M = -CUDART_INF_F, lsum = 0.f, val[VPT];
-#pragma unroll
-    for (int i = 0; i < VPT; ++i) val[i] = 0.f;
-    if (active) {
-      float mw[kWarps];
-#pragma unroll
-      for (int w = 0; w < kWarps; ++w) {
-        mw[w] = sm_rec[w * L::kRecFloats + G * kD + h];
-        M = fmaxf(M, mw[w]);
-      }
-#pragma unroll
-      for (int w = 0; w < kWarps; ++w) {
-        const float *r = sm_rec + w * L::kRecFloats;
-        const float f = exp2_or_zero(mw[w], M);
-        lsum = fmaf(r[G * kD + G + h], f, lsum);
-#pragma unroll
-        for (int i = 0; i < VPT; ++i) val[i] = fmaf(r[idx0 + i], f, val[i]);
+      for (int h = 0; h < G; ++h) {
+        const float mn = fmaxf(mh[h], 0.f);
+        const float fo = exp2_or_zero(mh[h], mn), fl = ex2_approx(-mn);
+        acc[h].x = fmaf(acc[h].x, fo, a[h].x * fl);
+        acc[h].y = fmaf(acc[h].y, fo, a[h].y * fl);
+        acc[h].z = fmaf(acc[h].z, fo, a[h].z * fl);
+        acc[h].w = fmaf(acc[h].w, fo, a[h].w * fl);
+        lh[h] = fmaf(lh[h], fo, bp[h] * fl);
+        mh[h] = mn;
       }
     }
     const int ub = sg.unit - sg.layer * units_per_layer;
     const int b = ub / p.Hkv, g = ub - b * p.Hkv;
-    float scur_all[G];   // warp 0 may finish the unit after barrier B, when sm_scur is being rewritten
-#pragma unroll
-    for (int hh = 0; hh < G; ++hh) scur_all[hh] = has_win ? sm_scur[hh] : -CUDART_INF_F;
-
-    if (sg.part < 0) {
-      // the whole unit lives in this CTA: add the current token, normalise, write, append to the ring
-      if (active) {
-        float sc = -CUDART_INF_F;
-#pragma unroll
-        for (int hh = 0; hh < G; ++hh)
-          if (hh == h) sc = scur_all[hh];
-        const float Mf = fmaxf(fmaxf(M, sc), 0.f);
-        const float fr = exp2_or_zero(M, Mf), fc = exp2_or_zero(sc, Mf);
-        const float inv = 1.0f / fmaf(lsum, fr, fc);
-        const bf16 *vt = reinterpret_cast<const bf16 *>(hdr + G * 256 + 768);
-        const int head = p.heads_of[g * G + h];
-        bf16 *op = reinterpret_cast<bf16 *>(p.out) + ((size_t(sg.layer) * p.B + b) * p.H + head) * kD + c;
-#pragma unroll
-        for (int i = 0; i < VPT; ++i) {
-          const float num = fmaf(val[i], fr, has_win ? fc * __bfloat162float(vt[c + i]) : 0.f);
-          op[i] = __float2bfloat16_rn(num * inv);
-        }
-      }
-      if (has_win && tid < 128) {   // bit copy of the new k,v rows into slot t mod cap
-        const LayerDev &ld = p.layers[sg.layer];
-        const size_t row = (size_t(sg.row_base) + size_t(t % int64_t(sg.cap))) * kD;
-        const uint32_t *srcw = reinterpret_cast<const uint32_t *>(hdr + G * 256 + 512);   // k_t (64 words) | v_t (64 words)
-        uint32_t *dstw = reinterpret_cast<uint32_t *>(reinterpret_cast<bf16 *>(p.ws + (tid < 64 ? ld.ringK : ld.ringV)) + row);
-        dstw[tid & 63] = srcw[tid];
-      }
-    } else if (active) {
-      // unit cut by a CTA boundary: one global record per CTA
+    bool write_out = sg.part < 0;
+    if (sg.part >= 0) {
+      // the unit is cut by a range boundary: this warp's record goes to global scratch, then a ticket
       float *grec = p.partials + (size_t(sg.rec0) + sg.part) * p.rec_floats;
 #pragma unroll
-      for (int i = 0; i < VPT; ++i) grec[idx0 + i] = val[i];
-      if (c == 0) {
-        grec[G * kD + h] = M;
-        grec[G * kD + G + h] = lsum;
+      for (int h = 0; h < G; ++h) {
+        *reinterpret_cast<float4 *>(grec + h * kD + lane * 4) = acc[h];
+        if (lane == 0) {
+          grec[G * kD + h] = mh[h];
+          grec[G * kD + G + h] = lh[h];
+        }
       }
-    }
-    __syncthreads();   // B: record area and logits may be rewritten; the CTA's global record is complete
-
-    if (sg.part >= 0 && warp == 0) {
-      // Warp 0 takes the unit's ticket while the other warps go on; the last ticket merges the few records.
+      __threadfence();
+      __syncwarp();
       int last = 0;
-      if (lane == 0) {
-        __threadfence();
-        last = atomicAdd(&p.tickets[sg.unit], 1) == sg.n_parts - 1;
-      }
+      if (lane == 0) last = atomicAdd(&p.tickets[sg.unit], 1) == sg.n_parts - 1;
       last = __shfl_sync(0xffffffffu, last, 0);
       if (last) {
         __threadfence();
+        // merge the unit's records: maxima and sums first (one (record, head) pair per lane), then the vectors
         const float *r0 = p.partials + size_t(sg.rec0) * p.rec_floats;
-        const bf16 *vt = reinterpret_cast<const bf16 *>(hdr + G * 256 + 768);
+        float Mg[G], lg[G];
 #pragma unroll
-        for (int hh = 0; hh < G; ++hh) {
-          float Mg = fmaxf(scur_all[hh], 0.f);
-          for (int i = 0; i < sg.n_parts; ++i) Mg = fmaxf(Mg, __ldcg(r0 + size_t(i) * p.rec_floats + G * kD + hh));
-          float lg = 0.f;
-          float4 vg = make_float4(0.f, 0.f, 0.f, 0.f);
-          for (int i = 0; i < sg.n_parts; ++i) {
-            const float *r = r0 + size_t(i) * p.rec_floats;
-            const float f = exp2_or_zero(__ldcg(r + G * kD + hh), Mg);
-            lg = fmaf(__ldcg(r + G * kD + G + hh), f, lg);
-            const float4 av = __ldcg(reinterpret_cast<const float4 *>(r + hh * kD + lane * 4));
-            vg.x = fmaf(av.x, f, vg.x);
-            vg.y = fmaf(av.y, f, vg.y);
-            vg.z = fmaf(av.z, f, vg.z);
-            vg.w = fmaf(av.w, f, vg.w);
-          }
-          const float fc = exp2_or_zero(scur_all[hh], Mg);
-          const float inv = 1.0f / (lg + fc);
-          float vx[4] = {0.f, 0.f, 0.f, 0.f};
-          if (has_win) load_elems<bf16, 4>(vt + lane * 4, vx);
-          const int head = p.heads_of[g * G + hh];
-          const __nv_bfloat162 lo = __floats2bfloat162_rn(fmaf(fc, vx[0], vg.x) * inv, fmaf(fc, vx[1], vg.y) * inv);
-          const __nv_bfloat162 hi = __floats2bfloat162_rn(fmaf(fc, vx[2], vg.z) * inv, fmaf(fc, vx[3], vg.w) * inv);
-          uint2 packed;
-          packed.x = *reinterpret_cast<const uint32_t *>(&lo);
-          packed.y = *reinterpret_cast<const uint32_t *>(&hi);
-          *reinterpret_cast<uint2 *>(reinterpret_cast<bf16 *>(p.out) + ((size_t(sg.layer) * p.B + b) * p.H + head) * kD + lane * 4) = packed;
+        for (int h = 0; h < G; ++h) {
+          Mg[h] = -CUDART_INF_F;
+          lg[h] = 0.f;
+          acc[h] = make_float4(0.f, 0.f, 0.f, 0.f);
         }
-        if (has_win) {
-          const LayerDev &ld = p.layers[sg.layer];
-          const size_t row = (size_t(sg.row_base) + size_t(t % int64_t(sg.cap))) * kD;
-          const uint2 *srcw = reinterpret_cast<const uint2 *>(hdr + G * 256 + 512);
-          reinterpret_cast<uint2 *>(reinterpret_cast<bf16 *>(p.ws + ld.ringK) + row)[lane] = srcw[lane];
-          reinterpret_cast<uint2 *>(reinterpret_cast<bf16 *>(p.ws + ld.ringV) + row)[lane] = srcw[32 + lane];
+        constexpr int RPB = 32 / G;   // records per batch
+        for (int i0 = 0; i0 < sg.n_parts; i0 += RPB) {
+          const int ri = i0 + lane / G, rh = lane % G;
+          const bool valid = ri < sg.n_parts;
+          const float me = valid ? __ldcg(r0 + size_t(ri) * p.rec_floats + G * kD + rh) : -CUDART_INF_F;
+          const float le = valid ? __ldcg(r0 + size_t(ri) * p.rec_floats + G * kD + G + rh) : 0.f;
+          // new running maximum per head
+          float Mn[G];
+#pragma unroll
+          for (int h = 0; h < G; ++h) Mn[h] = rh == h ? me : -CUDART_INF_F;
+#pragma unroll
+          for (int o2 = 16; o2 > 0; o2 >>= 1)
+#pragma unroll
+            for (int h = 0; h < G; ++h) Mn[h] = fmaxf(Mn[h], __shfl_xor_sync(0xffffffffu, Mn[h], o2));
+          float fe = 0.f, lpart[G];
+#pragma unroll
+          for (int h = 0; h < G; ++h) {
+            Mn[h] = fmaxf(Mn[h], Mg[h]);
+            const float resc = exp2_or_zero(Mg[h], Mn[h]);
+            lg[h] *= resc;
+            acc[h].x *= resc;
+            acc[h].y *= resc;
+            acc[h].z *= resc;
+            acc[h].w *= resc;
+            Mg[h] = Mn[h];
+            if (rh == h) fe = exp2_or_zero(me, Mn[h]);
+            lpart[h] = rh == h ? le * fe : 0.f;
+          }
+          warp_sum_multi<G>(lpart);
+#pragma unroll
+          for (int h = 0; h < G; ++h) lg[h] += lpart[h];
+          // vectors of this batch: RPB x G independent 16-byte loads per lane
+          const int nb = sg.n_parts - i0 < RPB ? sg.n_parts - i0 : RPB;
+          for (int u0 = 0; u0 < nb; u0 += 4) {
+            float4 vv[4][G];
+#pragma unroll
+            for (int u = 0; u < 4; ++u)
+#pragma unroll
+              for (int h = 0; h < G; ++h)
+                if (u0 + u < nb)
+                  vv[u][h] = __ldcg(reinterpret_cast<const float4 *>(r0 + size_t(i0 + u0 + u) * p.rec_floats + h * kD + lane * 4));
+#pragma unroll
+            for (int u = 0; u < 4; ++u)
+#pragma unroll
+              for (int h = 0; h < G; ++h)
+                if (u0 + u < nb) {
+                  const float f = __shfl_sync(0xffffffffu, fe, (u0 + u) * G + h);
+                  acc[h].x = fmaf(vv[u][h].x, f, acc[h].x);
+                  acc[h].y = fmaf(vv[u][h].y, f, acc[h].y);
+                  acc[h].z = fmaf(vv[u][h].z, f, acc[h].z);
+                  acc[h].w = fmaf(vv[u][h].w, f, acc[h].w);
+                }
+          }
+        }
+#pragma unroll
+        for (int h = 0; h < G; ++h) {
+          mh[h] = Mg[h];
+          lh[h] = lg[h];
         }
         if (lane == 0) p.tickets[sg.unit] = 0;
+        write_out = true;
       }
     }
-    GLIDE_TRACE_EVENT(7);
-  };
-
-  // ---- main loop --------------------------------------------------------------------------------------
-  Cursor ccur;
-  ccur.i = warp;
-  ccur.seg = 0;
-  ccur.tile_end = 0;
-  if (nseg > 0) cursor_load(ccur, sm_segs, t);
-  int next_flush = 0;
-  TileRef ref;
-  while (next_tile(ccur, sm_segs, nseg, ntiles, t, ref)) {
-    while (next_flush < ref.seg) flush(next_flush++);
-    if (acc_seg != ref.seg) load_unit(ref.seg);
-    if (ref.is_state && !phi_ready) load_phi(ref.seg);
-    if (!failed && !mbar_wait(my_bars + stage * 8, (phases >> stage) & 1u)) failed = true;
-    phases ^= 1u << stage;
-    failed = __any_sync(0xffffffffu, failed);
-    GLIDE_TRACE_EVENT(ref.is_state ? 4 : 3);
-    if (!failed) {
-      if (ref.is_state)
-        consume_state(sm_segs[ref.seg], ref.index, reinterpret_cast<const float4 *>(my_stages_ptr + stage * kStageBytes),
-                      my_z_ptr + stage * 16);
-      else
-        consume_window(ref.index, my_stages + stage * kStageBytes);
+    if (write_out) {
+      // the current token's own term, the shared normaliser, the output row and the ring append
+      float vx[4];
+      vx[0] = __uint_as_float(vt_bits.x << 16);
+      vx[1] = __uint_as_float(vt_bits.x & 0xffff0000u);
+      vx[2] = __uint_as_float(vt_bits.y << 16);
+      vx[3] = __uint_as_float(vt_bits.y & 0xffff0000u);
+#pragma unroll
+      for (int h = 0; h < G; ++h) {
+        const float Mf = fmaxf(fmaxf(mh[h], scur[h]), 0.f);
+        const float fr = exp2_or_zero(mh[h], Mf), fc = exp2_or_zero(scur[h], Mf);
+        const float inv = 1.0f / fmaf(lh[h], fr, fc);
+        const int head = p.heads_of[g * G + h];
+        const __nv_bfloat162 lo = __floats2bfloat162_rn(fmaf(acc[h].x, fr, fc * vx[0]) * inv, fmaf(acc[h].y, fr, fc * vx[1]) * inv);
+        const __nv_bfloat162 hi = __floats2bfloat162_rn(fmaf(acc[h].z, fr, fc * vx[2]) * inv, fmaf(acc[h].w, fr, fc * vx[3]) * inv);
+        uint2 packed;
+        packed.x = *reinterpret_cast<const uint32_t *>(&lo);
+        packed.y = *reinterpret_cast<const uint32_t *>(&hi);
+        *reinterpret_cast<uint2 *>(reinterpret_cast<bf16 *>(p.out) + ((size_t(sg.layer) * p.B + b) * p.H + head) * kD + lane * 4) = packed;
+      }
+      if (has_win) {   // every reader of slot t mod cap is done: bit copy of the new rows
+        const LayerDev &ld = p.layers[sg.layer];
+        const size_t row = (size_t(sg.row_base) + size_t(win_cur)) * kD;
+        reinterpret_cast<uint2 *>(reinterpret_cast<bf16 *>(p.ws + ld.ringK) + row)[lane] = kt_bits;
+        reinterpret_cast<uint2 *>(reinterpret_cast<bf16 *>(p.ws + ld.ringV) + row)[lane] = vt_bits;
+      }
     }
-    stage = stage + 1 == STAGES ? 0 : stage + 1;
-    __syncwarp();   // every lane is done with the stage before it is refilled
-    if (!failed) issue_next();
-    GLIDE_TRACE_EVENT(5);
   }
-  while (next_flush < nseg) flush(next_flush++);
   if (failed && lane == 0) atomicExch(&p.ctl->status, kDevWaitTimeout);
   GLIDE_TRACE_EVENT(9);
 
@@ -815,9 +779,8 @@ glide_decode_stream_kernel(const DecodeParams p, const StreamParams sp) {
 template <int G, int STAGES>
 size_t stream_smem_bytes(int max_segs) {
   using L = Layout<G>;
-  return 1024 + size_t(kWarps) * STAGES * kStageBytes + size_t(kWarps) * L::kRecFloats * 4 + size_t(kHdrSlots) * L::kHdrBytes +
-         size_t(kWarps) * STAGES * 64 + size_t(max_segs) * sizeof(StreamSegment) + size_t(kWarps * STAGES + kHdrSlots) * 8 +
-         8 * 4;
+  return 1024 + size_t(kWarps) * STAGES * kStageBytes + size_t(kWarps) * L::kHdrBytes + size_t(kWarps) * STAGES * 64 +
+         size_t(max_segs) * sizeof(StreamSegment) + size_t(kWarps) * (STAGES + 1) * 8;
 }
 
 template <typename F>
@@ -826,16 +789,18 @@ int dispatch_stream(int G, F &&f) {
     case 1: return f(IntTag<1>{}, IntTag<3>{});
     case 2: return f(IntTag<2>{}, IntTag<3>{});
     case 4: return f(IntTag<4>{}, IntTag<3>{});
-    case 8: return f(IntTag<8>{}, IntTag<2>{});
+    case 8: return f(IntTag<8>{}, IntTag<3>{});
     default: return int(GLIDE_ERR_UNSUPPORTED);
   }
 }
 
 }  // namespace
 
-// Cuts the tile stream into `n_ctas` equally heavy ranges (state tiles weigh 2: read + write).
-void build_stream_schedule(const glide_ctx *ctx, int n_ctas, std::vector<StreamSegment> *segs,
-                           std::vector<int32_t> *cta_seg_begin, int *max_segs_per_cta, size_t *n_records) {
+// Cuts the tile stream into `n_ranges` equally heavy contiguous ranges, one per warp.  A state tile weighs
+// 2 (read + write), a window tile 1, and starting a unit costs kUnitWeight (header, feature maps, finish).
+void build_stream_schedule(const glide_ctx *ctx, int n_ranges, std::vector<StreamSegment> *segs,
+                           std::vector<int32_t> *range_seg_begin, int *max_segs_per_cta, size_t *n_records) {
+  constexpr int64_t kUnitWeight = 2;
   const int L = ctx->cfg.n_layers, B = ctx->cfg.batch, Hkv = ctx->cfg.n_kv_heads, d = ctx->cfg.head_dim;
   const int64_t units_per_layer = int64_t(B) * Hkv;
   struct UnitTiles {
@@ -857,36 +822,32 @@ void build_stream_schedule(const glide_ctx *ctx, int n_ctas, std::vector<StreamS
       UnitTiles ut{l, int(int64_t(l) * units_per_layer + u), ld.evicts ? d / kTileRows : 0,
                    int((ld.cap + kTileRows - 1) / kTileRows)};
       units.push_back(ut);
-      total_w += 2 * int64_t(ut.n_state) + ut.n_win;
+      total_w += 2 * int64_t(ut.n_state) + ut.n_win + kUnitWeight;
     }
   }
   segs->clear();
-  cta_seg_begin->assign(size_t(n_ctas) + 1, 0);
-  *max_segs_per_cta = 0;
+  range_seg_begin->assign(size_t(n_ranges) + 1, 0);
   size_t records = 0;
-  // walk the stream; CTA c takes tiles while the cumulative weight stays below (c+1) * total / n_ctas
   size_t ui = 0;
   int st_done = 0, win_done = 0;   // progress inside units[ui]
   int64_t cum = 0;
   std::vector<std::vector<size_t>> unit_segs(units.size());
-  for (int c = 0; c < n_ctas; ++c) {
-    (*cta_seg_begin)[c] = int32_t(segs->size());
-    const int64_t target = (c + 1 == n_ctas) ? total_w : (total_w * (c + 1) + n_ctas - 1) / n_ctas;
-    int tile0 = 0;
+  for (int c = 0; c < n_ranges; ++c) {
+    (*range_seg_begin)[c] = int32_t(segs->size());
+    const int64_t target = (c + 1 == n_ranges) ? total_w : (total_w * (c + 1) + n_ranges - 1) / n_ranges;
     while (ui < units.size() && cum < target) {
       const UnitTiles &ut = units[ui];
       const LayerDev &ld = ctx->layers[ut.layer];
-      int64_t room = target - cum;
+      if (st_done == 0 && win_done == 0) cum += kUnitWeight;
+      int64_t room = std::max<int64_t>(target - cum, 1);
       StreamSegment sg{};
       sg.unit = ut.unit;
       sg.layer = ut.layer;
-      sg.tile0 = tile0;
       sg.state0 = st_done;
       sg.n_state = int(std::min<int64_t>(ut.n_state - st_done, (room + 1) / 2));
       room -= 2 * int64_t(sg.n_state);
       sg.win0 = win_done;
       sg.n_win = (st_done + sg.n_state == ut.n_state) ? int(std::min<int64_t>(ut.n_win - win_done, std::max<int64_t>(room, 0))) : 0;
-      if (sg.n_state == 0 && sg.n_win == 0 && (ut.n_state - st_done > 0 || ut.n_win - win_done > 0)) break;   // range full
       const int64_t ub = ut.unit - int64_t(ut.layer) * units_per_layer;
       sg.row_base = int32_t(ub * ld.cap);
       sg.cap = int32_t(ld.cap);
@@ -897,7 +858,6 @@ void build_stream_schedule(const glide_ctx *ctx, int n_ctas, std::vector<StreamS
       st_done += sg.n_state;
       win_done += sg.n_win;
       cum += 2 * int64_t(sg.n_state) + sg.n_win;
-      tile0 += sg.n_state + sg.n_win;
       unit_segs[ui].push_back(segs->size());
       segs->push_back(sg);
       if (st_done == ut.n_state && win_done == ut.n_win) {
@@ -905,9 +865,11 @@ void build_stream_schedule(const glide_ctx *ctx, int n_ctas, std::vector<StreamS
         st_done = win_done = 0;
       }
     }
-    *max_segs_per_cta = std::max<int>(*max_segs_per_cta, int(segs->size()) - (*cta_seg_begin)[c]);
   }
-  (*cta_seg_begin)[n_ctas] = int32_t(segs->size());
+  (*range_seg_begin)[n_ranges] = int32_t(segs->size());
+  *max_segs_per_cta = 0;
+  for (int c = 0; c + kWarps <= n_ranges; c += kWarps)
+    *max_segs_per_cta = std::max<int>(*max_segs_per_cta, (*range_seg_begin)[c + kWarps] - (*range_seg_begin)[c]);
   for (size_t u = 0; u < units.size(); ++u) {
     const std::vector<size_t> &list = unit_segs[u];
     if (list.size() == 1) {
@@ -934,7 +896,7 @@ int stream_decode_setup(glide_ctx *ctx) {
   const int n_ctas = ctx->sm_count;
   int max_segs = 0;
   size_t n_records = 0;
-  build_stream_schedule(ctx, n_ctas, &ctx->stream_segs, &ctx->stream_cta_begin, &max_segs, &n_records);
+  build_stream_schedule(ctx, n_ctas * kWarps, &ctx->stream_segs, &ctx->stream_cta_begin, &max_segs, &n_records);
   ctx->stream_max_segs = std::max(max_segs, 1);
   if (ctx->stream_segs.size() > ctx->stream_seg_capacity || n_records > ctx->stream_rec_capacity) return GLIDE_ERR_UNSUPPORTED;
   bool contiguous = true;
@@ -971,7 +933,7 @@ extern "C" int glide_debug_set_stream_trace(void *dev_buf) {
 int launch_decode_stream(glide_ctx *ctx, const DecodeParams &p, cudaStream_t stream) {
   StreamParams sp{};
   sp.segs = reinterpret_cast<const StreamSegment *>(ctx->ws + ctx->off_stream_segs);
-  sp.cta_seg_begin = reinterpret_cast<const int32_t *>(ctx->ws + ctx->off_stream_cta);
+  sp.range_seg_begin = reinterpret_cast<const int32_t *>(ctx->ws + ctx->off_stream_cta);
   sp.tmaps = reinterpret_cast<const CUtensorMap_st *>(ctx->ws + ctx->off_tmaps);
   sp.max_segs = ctx->stream_max_segs;
   sp.heads_contiguous = ctx->stream_heads_contiguous ? 1 : 0;

@@ -117,14 +117,14 @@ int glide::plan_context(const glide_config *cfg, glide_ctx *ctx, std::vector<Wor
   ctx->off_tickets = off;
   off = align_up(off + sizeof(int32_t) * size_t(L) * units_per_layer, 256);
   ctx->off_partials = off;
-  ctx->stream_seg_capacity = size_t(L) * units_per_layer + kMaxStreamCtas;
+  ctx->stream_seg_capacity = size_t(L) * units_per_layer + size_t(kMaxStreamCtas) * kStreamWarps;
   ctx->stream_rec_capacity = ctx->stream_seg_capacity;
   part_floats = std::max(part_floats, ctx->stream_rec_capacity * size_t(ctx->rec_floats));
   off = align_up(off + sizeof(float) * part_floats, 256);
   ctx->off_stream_segs = off;
   off = align_up(off + sizeof(StreamSegment) * ctx->stream_seg_capacity, 256);
   ctx->off_stream_cta = off;
-  off = align_up(off + sizeof(int32_t) * (kMaxStreamCtas + 1), 256);
+  off = align_up(off + sizeof(int32_t) * (size_t(kMaxStreamCtas) * kStreamWarps + 1), 256);
   ctx->off_tmaps = off;
   off = align_up(off + size_t(128) * 3 * L, 256);
   ctx->off_phik = off;

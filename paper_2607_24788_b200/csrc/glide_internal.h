@@ -69,14 +69,14 @@ struct DecodeParams {
   float scale_log2;          // softmax_scale * log2(e)
 };
 
-// One segment of the streaming decode kernel's schedule: the part of one unit that falls into one CTA's
+// One segment of the streaming decode kernel's schedule: the part of one unit that falls into one warp's
 // range of the tile stream (state tiles first, then window tiles).  64 bytes.
 struct StreamSegment {
   int32_t unit, layer;
-  int32_t tile0;             // CTA-relative index of the segment's first tile
+  int32_t reserved0;
   int32_t n_state, state0;   // state tiles [state0, state0 + n_state): 16 rows of S each
   int32_t n_win, win0;       // window tiles [win0, win0 + n_win): 16 ring slots each
-  int32_t part;              // this CTA's record among the unit's records, -1 if the whole unit is in this CTA
+  int32_t part;              // this warp's record among the unit's records, -1 if the whole unit is in this range
   int32_t n_parts;           // records of the unit (ticket target)
   int32_t rec0;              // index of the unit's first record in the split-K scratch
   int32_t row_base;          // row of the unit's slot 0 in the layer's [rows][d] ring tensor
@@ -89,7 +89,7 @@ static_assert(sizeof(StreamSegment) == 64, "StreamSegment is copied as 16-byte c
 
 struct StreamParams {
   const StreamSegment *segs;
-  const int32_t *cta_seg_begin;    // [grid + 1]
+  const int32_t *range_seg_begin;  // [8 * grid + 1]: first segment of every warp's range
   const struct CUtensorMap_st *tmaps;   // [3 L]: K ring, V ring (2-D), K+V ring (4-D) per layer
   int32_t max_segs;
   int32_t heads_contiguous;
@@ -161,7 +161,8 @@ int mma_decode_setup(glide_ctx *ctx);         // sizes the grid of the per-item 
 int stream_decode_supported(const glide_ctx *ctx);
 int stream_decode_setup(glide_ctx *ctx);      // builds the static schedule (host copy) and sizes the launch
 int launch_decode_stream(glide_ctx *ctx, const DecodeParams &p, cudaStream_t stream);
-constexpr int kMaxStreamCtas = 1024;          // upper bound on SMs used to size the schedule's workspace
+constexpr int kMaxStreamCtas = 512;           // upper bound on SMs used to size the schedule's workspace
+constexpr int kStreamWarps = 8;               // warps (= ranges of the schedule) per CTA
 int launch_decode_mma(glide_ctx *ctx, const DecodeParams &p, cudaStream_t stream);
 int launch_decode(glide_ctx *ctx, const void *q, const void *k, const void *v, void *out, cudaStream_t stream);
 int decode_occupancy(const glide_ctx *ctx, int *blocks_per_sm);
