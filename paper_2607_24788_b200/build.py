@@ -44,6 +44,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
     os.makedirs(OBJ, exist_ok=True)
     nvcc = _nvcc()
     extra = ["-Xptxas", "-v"] if verbose else []
+    extra += os.environ.get("GLIDE_NVCC_EXTRA", "").split()   # e.g. -DGLIDE_STREAM_STAGES=3 for experiments
 
     def compile_one(src):
         obj = os.path.join(OBJ, os.path.basename(src) + ".o")

@@ -38,6 +38,15 @@ constexpr uint32_t kBoxBytes = kTileRows * 128;            // one 64-column TMA 
 constexpr uint32_t kTileKV = 2 * kBoxBytes;                // K (or V) part of a window stage
 constexpr uint32_t kWaitLimit = 1u << 24;
 constexpr int kHdrSlots = 3;
+#ifndef GLIDE_STREAM_STAGES
+#define GLIDE_STREAM_STAGES 2
+#endif
+// schedule weights: cost of a state tile, a window tile and of starting a unit in a range
+#ifndef GLIDE_W_STATE
+#define GLIDE_W_STATE 7
+#define GLIDE_W_WIN 5
+#define GLIDE_W_UNIT 6
+#endif
 
 // Optional per-warp event trace (debug builds only: -DGLIDE_TRACE).
 #ifdef GLIDE_TRACE
@@ -92,6 +101,12 @@ __device__ __forceinline__ void bulk_load(uint32_t dst, const void *src, uint32_
                "l"(src), "r"(bytes), "r"(bar)
                : "memory");
 }
+__device__ __forceinline__ void bulk_store(void *dst, uint32_t src, uint32_t bytes) {
+  asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(dst), "r"(src), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_read0() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait0() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
 __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 __device__ __forceinline__ void ldmatrix_x4(uint32_t (&r)[4], uint32_t addr) {
   asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
@@ -253,11 +268,9 @@ glide_decode_stream_kernel(const DecodeParams p, const StreamParams sp) {
   GLIDE_TRACE_EVENT(1);
   const int64_t t = p.n_dev[0];   // every layer is at the same position (checked by the host)
   const int col2 = (lane & 3) * 2, hrow = lane >> 2;
-  const int range0 = blockIdx.x * kWarps;
-  const int cta_seg_begin = sp.range_seg_begin[range0];
-  const int cta_nseg = sp.range_seg_begin[range0 + kWarps] - cta_seg_begin;
-  const int seg_lo = sp.range_seg_begin[range0 + warp] - cta_seg_begin;       // this warp's segments in the CTA table
-  const int seg_hi = sp.range_seg_begin[range0 + warp + 1] - cta_seg_begin;
+  // the CTA's slice of the segment list: offsets come with the kernel parameters (no dependent global load)
+  const int cta_seg_begin = sp.cta_seg_begin[blockIdx.x];
+  const int cta_nseg = sp.cta_seg_begin[blockIdx.x + 1] - cta_seg_begin;
   if (cta_nseg > 0) {
     const uint4 *src = reinterpret_cast<const uint4 *>(sp.segs + cta_seg_begin);
     uint4 *dst = reinterpret_cast<uint4 *>(sm_segs);
@@ -267,7 +280,7 @@ glide_decode_stream_kernel(const DecodeParams p, const StreamParams sp) {
   const uint32_t my_stages = smem_u32(my_stages_ptr);
   unsigned char *my_hdr_ptr = sm_hdr + size_t(warp) * L::kHdrBytes;
   const uint32_t my_hdr = smem_u32(my_hdr_ptr);
-  const float *my_z_ptr = sm_z + warp * STAGES * 16;
+  float *my_z_ptr = sm_z + warp * STAGES * 16;
   const uint32_t my_z = smem_u32(my_z_ptr);
   const uint32_t my_bars = smem_u32(sm_bars + warp * (STAGES + 1));
   const uint32_t hdr_bar = my_bars + STAGES * 8;
@@ -277,8 +290,12 @@ glide_decode_stream_kernel(const DecodeParams p, const StreamParams sp) {
     fence_async_smem();
   }
   __syncthreads();   // segment table and barriers ready; the warps are on their own from here
+  // this warp's segments: the run of the CTA's list that carries its index
+  int seg_lo = 0;
+  while (seg_lo < cta_nseg && sm_segs[seg_lo].range < warp) ++seg_lo;
+  int seg_hi = seg_lo;
+  while (seg_hi < cta_nseg && sm_segs[seg_hi].range == warp) ++seg_hi;
 
-  const int units_per_layer = p.B * p.Hkv;
   bool failed = false;
 
   // ---- header of segment s (q rows | k_e | v_e | k_t | v_t) into this warp's buffer, lane 0 ---------
@@ -286,15 +303,14 @@ glide_decode_stream_kernel(const DecodeParams p, const StreamParams sp) {
     if (lane == 0) {
       const StreamSegment &sg = sm_segs[s];
       const bool ev = seg_evicting(sg, t);
-      const int ub = sg.unit - sg.layer * units_per_layer;
-      const int b = ub / p.Hkv, g = ub - b * p.Hkv;
       fence_async_smem();
       mbar_expect_tx(hdr_bar, G * 256 + 512 + (ev ? 512 : 0));
-      const bf16 *qb = reinterpret_cast<const bf16 *>(p.q) + (size_t(sg.layer) * p.B + b) * p.H * kD;
+      const bf16 *qall = reinterpret_cast<const bf16 *>(p.q);
       if (sp.heads_contiguous) {
-        bulk_load(my_hdr, qb + size_t(p.heads_of[g * G]) * kD, G * 256, hdr_bar);
+        bulk_load(my_hdr, qall + size_t(sg.qrow0) * kD, G * 256, hdr_bar);
       } else {
-        for (int h = 0; h < G; ++h) bulk_load(my_hdr + h * 256, qb + size_t(p.heads_of[g * G + h]) * kD, 256, hdr_bar);
+        for (int h = 0; h < G; ++h)
+          bulk_load(my_hdr + h * 256, qall + (size_t(sg.qrow0) + p.heads_of[sg.g * G + h]) * kD, 256, hdr_bar);
       }
       const bf16 *kt = reinterpret_cast<const bf16 *>(p.k) + size_t(sg.unit) * kD;
       const bf16 *vt = reinterpret_cast<const bf16 *>(p.v) + size_t(sg.unit) * kD;
@@ -305,15 +321,13 @@ glide_decode_stream_kernel(const DecodeParams p, const StreamParams sp) {
           bulk_load(my_hdr + G * 256, kt, 256, hdr_bar);
           bulk_load(my_hdr + G * 256 + 256, vt, 256, hdr_bar);
         } else {
-          const LayerDev &ld = p.layers[sg.layer];
           const size_t row = (size_t(sg.row_base) + size_t(t % int64_t(sg.cap))) * kD;
-          bulk_load(my_hdr + G * 256, reinterpret_cast<const bf16 *>(p.ws + ld.ringK) + row, 256, hdr_bar);
-          bulk_load(my_hdr + G * 256 + 256, reinterpret_cast<const bf16 *>(p.ws + ld.ringV) + row, 256, hdr_bar);
+          bulk_load(my_hdr + G * 256, reinterpret_cast<const bf16 *>(p.ws + size_t(sg.ringK_off256) * 256) + row, 256, hdr_bar);
+          bulk_load(my_hdr + G * 256 + 256, reinterpret_cast<const bf16 *>(p.ws + size_t(sg.ringV_off256) * 256) + row, 256, hdr_bar);
         }
       }
     }
   };
-  if (seg_lo < seg_hi) issue_header(seg_lo);
 
   // ---- tile issue (lane 0) ------------------------------------------------------------------------
   Cursor icur;
@@ -356,6 +370,7 @@ glide_decode_stream_kernel(const DecodeParams p, const StreamParams sp) {
       }
     }
   };
+  if (seg_lo < seg_hi) issue_header(seg_lo);   // small and needed first
   for (int s = 0; s < STAGES; ++s) issue_next();
   GLIDE_TRACE_EVENT(2);
 
@@ -372,6 +387,7 @@ glide_decode_stream_kernel(const DecodeParams p, const StreamParams sp) {
   int win_end = 0, win_cur = 0;   // window tokens live in slots [0, win_end) except slot win_cur
   uint32_t phases = 0;     // parity expected by the next wait on each stage; bit STAGES: header barrier
   int stage = 0;
+  int n_pending = 0, pend0 = 0, pend1 = 0;   // segments of this range whose unit is shared with a neighbour (at most two)
 
   // ---- window tile ------------------------------------------------------------------------------
   auto consume_window = [&](int wtile, uint32_t stage_addr) {
@@ -449,10 +465,9 @@ glide_decode_stream_kernel(const DecodeParams p, const StreamParams sp) {
     }
   };
 
-  // ---- state tile: 16 rows of S and z, updated in place and read out ------------------------------
-  auto consume_state = [&](const StreamSegment &sg, int stile, const float4 *st, const float *zs) {
-    float *Sg = reinterpret_cast<float *>(p.ws + size_t(sg.S_off256) * 256) + size_t(stile) * kTileRows * kD;
-    float *zg = reinterpret_cast<float *>(p.ws + size_t(sg.z_off256) * 256) + stile * kTileRows;
+  // ---- state tile: 16 rows of S and z, updated in the stage and stored back by the async proxy ---------
+  // (bulk stores are not ordered by this warp's later fences, so a ticket never waits for state traffic)
+  auto consume_state = [&](const StreamSegment &sg, int stile, float4 *st, float *zs, uint32_t st_addr, uint32_t z_addr) {
     const int src0 = stile * 4;   // lane that holds phi entries of the tile's first row (4 rows per lane)
 #pragma unroll
     for (int r = 0; r < kTileRows; ++r) {
@@ -462,7 +477,7 @@ glide_decode_stream_kernel(const DecodeParams p, const StreamParams sp) {
       s.y = fmaf(pk, ve[1], s.y);
       s.z = fmaf(pk, ve[2], s.z);
       s.w = fmaf(pk, ve[3], s.w);
-      *reinterpret_cast<float4 *>(Sg + r * kD + lane * 4) = s;
+      st[r * (kD / 4) + lane] = s;
 #pragma unroll
       for (int h = 0; h < G; ++h) {
         const float f = __shfl_sync(0xffffffffu, phi[h][r & 3], src0 + (r >> 2));
@@ -486,11 +501,21 @@ glide_decode_stream_kernel(const DecodeParams p, const StreamParams sp) {
       if (h == 0) {
         if (lane < 16) {
           zn = zs[lane] + f;
-          zg[lane] = zn;
+          zs[lane] = zn;
         }
       } else if (lane < 16) {
         bp[h - 1] = fmaf(f, zn, bp[h - 1]);
       }
+    }
+    fence_async_smem();   // the updated rows are read by the async proxy
+    __syncwarp();
+    if (lane == 0) {
+      float *Sg = reinterpret_cast<float *>(p.ws + size_t(sg.S_off256) * 256) + size_t(stile) * kTileRows * kD;
+      float *zg = reinterpret_cast<float *>(p.ws + size_t(sg.z_off256) * 256) + stile * kTileRows;
+      bulk_store(Sg, st_addr, kStageBytes);
+      bulk_store(zg, z_addr, 64);
+      bulk_commit();
+      bulk_wait_read0();   // the stage may be refilled once the store has read it
     }
   };
 
@@ -568,8 +593,8 @@ glide_decode_stream_kernel(const DecodeParams p, const StreamParams sp) {
       }
       GLIDE_TRACE_EVENT(k < n_state_eff ? 4 : 3);
       if (k < n_state_eff)
-        consume_state(sg, sg.state0 + k, reinterpret_cast<const float4 *>(my_stages_ptr + stage * kStageBytes),
-                      my_z_ptr + stage * 16);
+        consume_state(sg, sg.state0 + k, reinterpret_cast<float4 *>(my_stages_ptr + stage * kStageBytes),
+                      my_z_ptr + stage * 16, my_stages + stage * kStageBytes, my_z + stage * 64);
       else
         consume_window(sg.win0 + k - n_state_eff, my_stages + stage * kStageBytes);
       last_stage = stage;
@@ -640,11 +665,9 @@ glide_decode_stream_kernel(const DecodeParams p, const StreamParams sp) {
         mh[h] = mn;
       }
     }
-    const int ub = sg.unit - sg.layer * units_per_layer;
-    const int b = ub / p.Hkv, g = ub - b * p.Hkv;
-    bool write_out = sg.part < 0;
     if (sg.part >= 0) {
-      // the unit is cut by a range boundary: this warp's record goes to global scratch, then a ticket
+      // the unit is cut by a range boundary: this warp's record goes to global scratch; its ticket is taken
+      // at the end of the range, so that the streaming loop never stalls on a fence or an atomic
       float *grec = p.partials + (size_t(sg.rec0) + sg.part) * p.rec_floats;
 #pragma unroll
       for (int h = 0; h < G; ++h) {
@@ -654,87 +677,11 @@ glide_decode_stream_kernel(const DecodeParams p, const StreamParams sp) {
           grec[G * kD + G + h] = lh[h];
         }
       }
-      __threadfence();
-      __syncwarp();
-      int last = 0;
-      if (lane == 0) last = atomicAdd(&p.tickets[sg.unit], 1) == sg.n_parts - 1;
-      last = __shfl_sync(0xffffffffu, last, 0);
-      if (last) {
-        __threadfence();
-        // merge the unit's records: maxima and sums first (one (record, head) pair per lane), then the vectors
-        const float *r0 = p.partials + size_t(sg.rec0) * p.rec_floats;
-        float Mg[G], lg[G];
-#pragma unroll
-        for (int h = 0; h < G; ++h) {
-          Mg[h] = -CUDART_INF_F;
-          lg[h] = 0.f;
-          acc[h] = make_float4(0.f, 0.f, 0.f, 0.f);
-        }
-        constexpr int RPB = 32 / G;   // records per batch
-        for (int i0 = 0; i0 < sg.n_parts; i0 += RPB) {
-          const int ri = i0 + lane / G, rh = lane % G;
-          const bool valid = ri < sg.n_parts;
-          const float me = valid ? __ldcg(r0 + size_t(ri) * p.rec_floats + G * kD + rh) : -CUDART_INF_F;
-          const float le = valid ? __ldcg(r0 + size_t(ri) * p.rec_floats + G * kD + G + rh) : 0.f;
-          // new running maximum per head
-          float Mn[G];
-#pragma unroll
-          for (int h = 0; h < G; ++h) Mn[h] = rh == h ? me : -CUDART_INF_F;
-#pragma unroll
-          for (int o2 = 16; o2 > 0; o2 >>= 1)
-#pragma unroll
-            for (int h = 0; h < G; ++h) Mn[h] = fmaxf(Mn[h], __shfl_xor_sync(0xffffffffu, Mn[h], o2));
-          float fe = 0.f, lpart[G];
-#pragma unroll
-          for (int h = 0; h < G; ++h) {
-            Mn[h] = fmaxf(Mn[h], Mg[h]);
-            const float resc = exp2_or_zero(Mg[h], Mn[h]);
-            lg[h] *= resc;
-            acc[h].x *= resc;
-            acc[h].y *= resc;
-            acc[h].z *= resc;
-            acc[h].w *= resc;
-            Mg[h] = Mn[h];
-            if (rh == h) fe = exp2_or_zero(me, Mn[h]);
-            lpart[h] = rh == h ? le * fe : 0.f;
-          }
-          warp_sum_multi<G>(lpart);
-#pragma unroll
-          for (int h = 0; h < G; ++h) lg[h] += lpart[h];
-          // vectors of this batch: RPB x G independent 16-byte loads per lane
-          const int nb = sg.n_parts - i0 < RPB ? sg.n_parts - i0 : RPB;
-          for (int u0 = 0; u0 < nb; u0 += 4) {
-            float4 vv[4][G];
-#pragma unroll
-            for (int u = 0; u < 4; ++u)
-#pragma unroll
-              for (int h = 0; h < G; ++h)
-                if (u0 + u < nb)
-                  vv[u][h] = __ldcg(reinterpret_cast<const float4 *>(r0 + size_t(i0 + u0 + u) * p.rec_floats + h * kD + lane * 4));
-#pragma unroll
-            for (int u = 0; u < 4; ++u)
-#pragma unroll
-              for (int h = 0; h < G; ++h)
-                if (u0 + u < nb) {
-                  const float f = __shfl_sync(0xffffffffu, fe, (u0 + u) * G + h);
-                  acc[h].x = fmaf(vv[u][h].x, f, acc[h].x);
-                  acc[h].y = fmaf(vv[u][h].y, f, acc[h].y);
-                  acc[h].z = fmaf(vv[u][h].z, f, acc[h].z);
-                  acc[h].w = fmaf(vv[u][h].w, f, acc[h].w);
-                }
-          }
-        }
-#pragma unroll
-        for (int h = 0; h < G; ++h) {
-          mh[h] = Mg[h];
-          lh[h] = lg[h];
-        }
-        if (lane == 0) p.tickets[sg.unit] = 0;
-        write_out = true;
-      }
-    }
-    if (write_out) {
-      // the current token's own term, the shared normaliser, the output row and the ring append
+      if (n_pending == 0) pend0 = s; else pend1 = s;
+      ++n_pending;
+      GLIDE_TRACE_EVENT(10);
+    } else {
+      // the whole unit is in this range: current token's own term, shared normaliser, output row, ring append
       float vx[4];
       vx[0] = __uint_as_float(vt_bits.x << 16);
       vx[1] = __uint_as_float(vt_bits.x & 0xffff0000u);
@@ -745,23 +692,151 @@ glide_decode_stream_kernel(const DecodeParams p, const StreamParams sp) {
         const float Mf = fmaxf(fmaxf(mh[h], scur[h]), 0.f);
         const float fr = exp2_or_zero(mh[h], Mf), fc = exp2_or_zero(scur[h], Mf);
         const float inv = 1.0f / fmaf(lh[h], fr, fc);
-        const int head = p.heads_of[g * G + h];
+        const int orow = sg.qrow0 + (sp.heads_contiguous ? h : p.heads_of[sg.g * G + h]);
         const __nv_bfloat162 lo = __floats2bfloat162_rn(fmaf(acc[h].x, fr, fc * vx[0]) * inv, fmaf(acc[h].y, fr, fc * vx[1]) * inv);
         const __nv_bfloat162 hi = __floats2bfloat162_rn(fmaf(acc[h].z, fr, fc * vx[2]) * inv, fmaf(acc[h].w, fr, fc * vx[3]) * inv);
         uint2 packed;
         packed.x = *reinterpret_cast<const uint32_t *>(&lo);
         packed.y = *reinterpret_cast<const uint32_t *>(&hi);
-        *reinterpret_cast<uint2 *>(reinterpret_cast<bf16 *>(p.out) + ((size_t(sg.layer) * p.B + b) * p.H + head) * kD + lane * 4) = packed;
+        *reinterpret_cast<uint2 *>(reinterpret_cast<bf16 *>(p.out) + size_t(orow) * kD + lane * 4) = packed;
       }
       if (has_win) {   // every reader of slot t mod cap is done: bit copy of the new rows
-        const LayerDev &ld = p.layers[sg.layer];
         const size_t row = (size_t(sg.row_base) + size_t(win_cur)) * kD;
-        reinterpret_cast<uint2 *>(reinterpret_cast<bf16 *>(p.ws + ld.ringK) + row)[lane] = kt_bits;
-        reinterpret_cast<uint2 *>(reinterpret_cast<bf16 *>(p.ws + ld.ringV) + row)[lane] = vt_bits;
+        reinterpret_cast<uint2 *>(reinterpret_cast<bf16 *>(p.ws + size_t(sg.ringK_off256) * 256) + row)[lane] = kt_bits;
+        reinterpret_cast<uint2 *>(reinterpret_cast<bf16 *>(p.ws + size_t(sg.ringV_off256) * 256) + row)[lane] = vt_bits;
       }
     }
   }
+  GLIDE_TRACE_EVENT(14);
+
+  // ---- tickets of the units this range shares with its neighbours; the last ticket of a unit merges -----
+  if (n_pending > 0 && !failed) {
+    __threadfence();
+    __syncwarp();
+    int last = 0;
+    if (lane < n_pending) {
+      const StreamSegment &sg = sm_segs[lane == 0 ? pend0 : pend1];
+      last = atomicAdd(&p.tickets[sg.unit], 1) == sg.n_parts - 1;
+    }
+    const unsigned last_mask = __ballot_sync(0xffffffffu, last != 0);
+    GLIDE_TRACE_EVENT(12);
+    for (int pi = 0; pi < n_pending; ++pi) {
+      if (!((last_mask >> pi) & 1u)) continue;
+      __threadfence();
+      const StreamSegment &sg = sm_segs[pi == 0 ? pend0 : pend1];
+      const bool has_win = sg.cap > 0;
+      // reload the unit's query rows and current token (this warp may have moved on to another unit since)
+      const bf16 *qall = reinterpret_cast<const bf16 *>(p.q);
+      const uint2 ktb = *reinterpret_cast<const uint2 *>(reinterpret_cast<const bf16 *>(p.k) + size_t(sg.unit) * kD + lane * 4);
+      const uint2 vtb = *reinterpret_cast<const uint2 *>(reinterpret_cast<const bf16 *>(p.v) + size_t(sg.unit) * kD + lane * 4);
+      int orow[G];
+      float sc[G];
+      {
+        float kx[4];
+        kx[0] = __uint_as_float(ktb.x << 16);
+        kx[1] = __uint_as_float(ktb.x & 0xffff0000u);
+        kx[2] = __uint_as_float(ktb.y << 16);
+        kx[3] = __uint_as_float(ktb.y & 0xffff0000u);
+#pragma unroll
+        for (int h = 0; h < G; ++h) {
+          orow[h] = sg.qrow0 + (sp.heads_contiguous ? h : p.heads_of[sg.g * G + h]);
+          float qx[4];
+          load_elems<bf16, 4>(qall + size_t(orow[h]) * kD + lane * 4, qx);
+          sc[h] = 0.f;
+#pragma unroll
+          for (int i = 0; i < 4; ++i) sc[h] = fmaf(qx[i], kx[i], sc[h]);
+        }
+        warp_sum_multi<G>(sc);
+#pragma unroll
+        for (int h = 0; h < G; ++h) sc[h] = has_win ? sc[h] * p.scale_log2 : -CUDART_INF_F;
+      }
+      // merge the records: maxima and sums first (one (record, head) pair per lane), then the vectors
+      const float *r0 = p.partials + size_t(sg.rec0) * p.rec_floats;
+      float Mg[G], lg[G];
+      float4 acc[G];
+#pragma unroll
+      for (int h = 0; h < G; ++h) {
+        Mg[h] = -CUDART_INF_F;
+        lg[h] = 0.f;
+        acc[h] = make_float4(0.f, 0.f, 0.f, 0.f);
+      }
+      constexpr int RPB = 32 / G;   // records per batch
+      for (int i0 = 0; i0 < sg.n_parts; i0 += RPB) {
+        const int ri = i0 + lane / G, rh = lane % G;
+        const bool valid = ri < sg.n_parts;
+        const float me = valid ? __ldcg(r0 + size_t(ri) * p.rec_floats + G * kD + rh) : -CUDART_INF_F;
+        const float le = valid ? __ldcg(r0 + size_t(ri) * p.rec_floats + G * kD + G + rh) : 0.f;
+        const int nb = sg.n_parts - i0 < RPB ? sg.n_parts - i0 : RPB;
+        float4 vv[RPB][G];   // the batch's vectors: all loads in flight together with the scalars above
+#pragma unroll
+        for (int u = 0; u < RPB; ++u)
+#pragma unroll
+          for (int h = 0; h < G; ++h)
+            if (u < nb) vv[u][h] = __ldcg(reinterpret_cast<const float4 *>(r0 + size_t(i0 + u) * p.rec_floats + h * kD + lane * 4));
+        float Mn[G];
+#pragma unroll
+        for (int h = 0; h < G; ++h) Mn[h] = rh == h ? me : -CUDART_INF_F;
+#pragma unroll
+        for (int o2 = 16; o2 > 0; o2 >>= 1)
+#pragma unroll
+          for (int h = 0; h < G; ++h) Mn[h] = fmaxf(Mn[h], __shfl_xor_sync(0xffffffffu, Mn[h], o2));
+        float fe = 0.f, lpart[G];
+#pragma unroll
+        for (int h = 0; h < G; ++h) {
+          Mn[h] = fmaxf(Mn[h], Mg[h]);
+          const float resc = exp2_or_zero(Mg[h], Mn[h]);
+          lg[h] *= resc;
+          acc[h].x *= resc;
+          acc[h].y *= resc;
+          acc[h].z *= resc;
+          acc[h].w *= resc;
+          Mg[h] = Mn[h];
+          if (rh == h) fe = exp2_or_zero(me, Mn[h]);
+          lpart[h] = rh == h ? le * fe : 0.f;
+        }
+        warp_sum_multi<G>(lpart);
+#pragma unroll
+        for (int h = 0; h < G; ++h) lg[h] += lpart[h];
+#pragma unroll
+        for (int u = 0; u < RPB; ++u)
+#pragma unroll
+          for (int h = 0; h < G; ++h)
+            if (u < nb) {
+              const float f = __shfl_sync(0xffffffffu, fe, u * G + h);
+              acc[h].x = fmaf(vv[u][h].x, f, acc[h].x);
+              acc[h].y = fmaf(vv[u][h].y, f, acc[h].y);
+              acc[h].z = fmaf(vv[u][h].z, f, acc[h].z);
+              acc[h].w = fmaf(vv[u][h].w, f, acc[h].w);
+            }
+      }
+      float vx[4];
+      vx[0] = __uint_as_float(vtb.x << 16);
+      vx[1] = __uint_as_float(vtb.x & 0xffff0000u);
+      vx[2] = __uint_as_float(vtb.y << 16);
+      vx[3] = __uint_as_float(vtb.y & 0xffff0000u);
+#pragma unroll
+      for (int h = 0; h < G; ++h) {
+        const float Mf = fmaxf(fmaxf(Mg[h], sc[h]), 0.f);
+        const float fr = exp2_or_zero(Mg[h], Mf), fc = exp2_or_zero(sc[h], Mf);
+        const float inv = 1.0f / fmaf(lg[h], fr, fc);
+        const __nv_bfloat162 lo = __floats2bfloat162_rn(fmaf(acc[h].x, fr, fc * vx[0]) * inv, fmaf(acc[h].y, fr, fc * vx[1]) * inv);
+        const __nv_bfloat162 hi = __floats2bfloat162_rn(fmaf(acc[h].z, fr, fc * vx[2]) * inv, fmaf(acc[h].w, fr, fc * vx[3]) * inv);
+        uint2 packed;
+        packed.x = *reinterpret_cast<const uint32_t *>(&lo);
+        packed.y = *reinterpret_cast<const uint32_t *>(&hi);
+        *reinterpret_cast<uint2 *>(reinterpret_cast<bf16 *>(p.out) + size_t(orow[h]) * kD + lane * 4) = packed;
+      }
+      if (has_win) {
+        const size_t row = (size_t(sg.row_base) + size_t(t % int64_t(sg.cap))) * kD;
+        reinterpret_cast<uint2 *>(reinterpret_cast<bf16 *>(p.ws + size_t(sg.ringK_off256) * 256) + row)[lane] = ktb;
+        reinterpret_cast<uint2 *>(reinterpret_cast<bf16 *>(p.ws + size_t(sg.ringV_off256) * 256) + row)[lane] = vtb;
+      }
+      if (lane == 0) p.tickets[sg.unit] = 0;
+      GLIDE_TRACE_EVENT(13);
+    }
+  }
   if (failed && lane == 0) atomicExch(&p.ctl->status, kDevWaitTimeout);
+  if (lane == 0) bulk_wait0();   // this warp's state stores have landed
   GLIDE_TRACE_EVENT(9);
 
   __syncthreads();
@@ -788,7 +863,7 @@ int dispatch_stream(int G, F &&f) {
   switch (G) {
     case 1: return f(IntTag<1>{}, IntTag<3>{});
     case 2: return f(IntTag<2>{}, IntTag<3>{});
-    case 4: return f(IntTag<4>{}, IntTag<3>{});
+    case 4: return f(IntTag<4>{}, IntTag<GLIDE_STREAM_STAGES>{});
     case 8: return f(IntTag<8>{}, IntTag<3>{});
     default: return int(GLIDE_ERR_UNSUPPORTED);
   }
@@ -800,9 +875,13 @@ int dispatch_stream(int G, F &&f) {
 // 2 (read + write), a window tile 1, and starting a unit costs kUnitWeight (header, feature maps, finish).
 void build_stream_schedule(const glide_ctx *ctx, int n_ranges, std::vector<StreamSegment> *segs,
                            std::vector<int32_t> *range_seg_begin, int *max_segs_per_cta, size_t *n_records) {
-  constexpr int64_t kUnitWeight = 2;
+  constexpr int64_t kUnitWeight = GLIDE_W_UNIT, kStateWeight = GLIDE_W_STATE, kWinWeight = GLIDE_W_WIN;
   const int L = ctx->cfg.n_layers, B = ctx->cfg.batch, Hkv = ctx->cfg.n_kv_heads, d = ctx->cfg.head_dim;
   const int64_t units_per_layer = int64_t(B) * Hkv;
+  bool contiguous_heads = true;
+  for (int g = 0; g < Hkv; ++g)
+    for (int i = 1; i < ctx->G; ++i)
+      contiguous_heads = contiguous_heads && ctx->heads_of[size_t(g) * ctx->G + i] == ctx->heads_of[size_t(g) * ctx->G] + i;
   struct UnitTiles {
     int layer, unit;
     int n_state, n_win;
@@ -822,7 +901,7 @@ void build_stream_schedule(const glide_ctx *ctx, int n_ranges, std::vector<Strea
       UnitTiles ut{l, int(int64_t(l) * units_per_layer + u), ld.evicts ? d / kTileRows : 0,
                    int((ld.cap + kTileRows - 1) / kTileRows)};
       units.push_back(ut);
-      total_w += 2 * int64_t(ut.n_state) + ut.n_win + kUnitWeight;
+      total_w += kStateWeight * int64_t(ut.n_state) + kWinWeight * int64_t(ut.n_win) + kUnitWeight;
     }
   }
   segs->clear();
@@ -843,11 +922,14 @@ void build_stream_schedule(const glide_ctx *ctx, int n_ranges, std::vector<Strea
       StreamSegment sg{};
       sg.unit = ut.unit;
       sg.layer = ut.layer;
+      sg.range = c % kWarps;
       sg.state0 = st_done;
-      sg.n_state = int(std::min<int64_t>(ut.n_state - st_done, (room + 1) / 2));
-      room -= 2 * int64_t(sg.n_state);
+      sg.n_state = int(std::min<int64_t>(ut.n_state - st_done, (room + kStateWeight - 1) / kStateWeight));
+      room -= kStateWeight * int64_t(sg.n_state);
       sg.win0 = win_done;
-      sg.n_win = (st_done + sg.n_state == ut.n_state) ? int(std::min<int64_t>(ut.n_win - win_done, std::max<int64_t>(room, 0))) : 0;
+      sg.n_win = (st_done + sg.n_state == ut.n_state)
+                     ? int(std::min<int64_t>(ut.n_win - win_done, (std::max<int64_t>(room, 0) + kWinWeight - 1) / kWinWeight))
+                     : 0;
       const int64_t ub = ut.unit - int64_t(ut.layer) * units_per_layer;
       sg.row_base = int32_t(ub * ld.cap);
       sg.cap = int32_t(ld.cap);
@@ -855,9 +937,17 @@ void build_stream_schedule(const glide_ctx *ctx, int n_ranges, std::vector<Strea
       sg.evicts = ld.evicts;
       sg.S_off256 = int32_t((ld.S + size_t(ub) * d * d * 4) / 256);
       sg.z_off256 = int32_t((ld.z + size_t(ub) * d * 4) / 256);
+      sg.ringK_off256 = int32_t(ld.ringK / 256);
+      sg.ringV_off256 = int32_t(ld.ringV / 256);
+      sg.g = int32_t(ub % Hkv);
+      {
+        const int64_t b = ub / Hkv;
+        const int64_t row = (int64_t(ut.layer) * B + b) * ctx->cfg.n_q_heads;
+        sg.qrow0 = int32_t(row + (contiguous_heads ? ctx->heads_of[size_t(sg.g) * ctx->G] : 0));
+      }
       st_done += sg.n_state;
       win_done += sg.n_win;
-      cum += 2 * int64_t(sg.n_state) + sg.n_win;
+      cum += kStateWeight * int64_t(sg.n_state) + kWinWeight * int64_t(sg.n_win);
       unit_segs[ui].push_back(segs->size());
       segs->push_back(sg);
       if (st_done == ut.n_state && win_done == ut.n_win) {
@@ -893,7 +983,7 @@ int stream_decode_supported(const glide_ctx *ctx) {
 }
 
 int stream_decode_setup(glide_ctx *ctx) {
-  const int n_ctas = ctx->sm_count;
+  const int n_ctas = std::min(ctx->sm_count, kMaxStreamCtas);
   int max_segs = 0;
   size_t n_records = 0;
   build_stream_schedule(ctx, n_ctas * kWarps, &ctx->stream_segs, &ctx->stream_cta_begin, &max_segs, &n_records);
@@ -933,7 +1023,7 @@ extern "C" int glide_debug_set_stream_trace(void *dev_buf) {
 int launch_decode_stream(glide_ctx *ctx, const DecodeParams &p, cudaStream_t stream) {
   StreamParams sp{};
   sp.segs = reinterpret_cast<const StreamSegment *>(ctx->ws + ctx->off_stream_segs);
-  sp.range_seg_begin = reinterpret_cast<const int32_t *>(ctx->ws + ctx->off_stream_cta);
+  for (int c = 0; c <= ctx->decode_grid; ++c) sp.cta_seg_begin[c] = ctx->stream_cta_begin[size_t(c) * kWarps];
   sp.tmaps = reinterpret_cast<const CUtensorMap_st *>(ctx->ws + ctx->off_tmaps);
   sp.max_segs = ctx->stream_max_segs;
   sp.heads_contiguous = ctx->stream_heads_contiguous ? 1 : 0;

@@ -69,11 +69,14 @@ struct DecodeParams {
   float scale_log2;          // softmax_scale * log2(e)
 };
 
+constexpr int kMaxStreamCtas = 192;           // CTAs (one per SM) the streaming decode kernel's schedule can address
+constexpr int kStreamWarps = 8;               // warps (= ranges of the schedule) per CTA
+
 // One segment of the streaming decode kernel's schedule: the part of one unit that falls into one warp's
 // range of the tile stream (state tiles first, then window tiles).  64 bytes.
 struct StreamSegment {
   int32_t unit, layer;
-  int32_t reserved0;
+  int32_t range;             // warp (0..7) of the CTA that owns the segment
   int32_t n_state, state0;   // state tiles [state0, state0 + n_state): 16 rows of S each
   int32_t n_win, win0;       // window tiles [win0, win0 + n_win): 16 ring slots each
   int32_t part;              // this warp's record among the unit's records, -1 if the whole unit is in this range
@@ -83,13 +86,17 @@ struct StreamSegment {
   int32_t cap;               // ring slots
   int32_t w;                 // window (clamped to INT32_MAX)
   int32_t evicts;
-  int32_t S_off256, z_off256;  // workspace byte offsets / 256 of the unit's S and z
+  int32_t S_off256, z_off256;        // workspace byte offsets / 256 of the unit's S and z
+  int32_t ringK_off256, ringV_off256;  // workspace byte offsets / 256 of the layer's K and V rings
+  int32_t qrow0;             // row of the KV head's first query head in the [L*B*H][d] q / out tensors
+  int32_t g;                 // KV head index (for the head table when the groups are not contiguous)
+  int32_t pad_[4];
 };
-static_assert(sizeof(StreamSegment) == 64, "StreamSegment is copied as 16-byte chunks");
+static_assert(sizeof(StreamSegment) == 96, "StreamSegment is copied as 16-byte chunks");
 
 struct StreamParams {
   const StreamSegment *segs;
-  const int32_t *range_seg_begin;  // [8 * grid + 1]: first segment of every warp's range
+  int32_t cta_seg_begin[kMaxStreamCtas + 1];   // first segment of every CTA (its 8 warps' ranges follow each other)
   const struct CUtensorMap_st *tmaps;   // [3 L]: K ring, V ring (2-D), K+V ring (4-D) per layer
   int32_t max_segs;
   int32_t heads_contiguous;
@@ -161,8 +168,6 @@ int mma_decode_setup(glide_ctx *ctx);         // sizes the grid of the per-item 
 int stream_decode_supported(const glide_ctx *ctx);
 int stream_decode_setup(glide_ctx *ctx);      // builds the static schedule (host copy) and sizes the launch
 int launch_decode_stream(glide_ctx *ctx, const DecodeParams &p, cudaStream_t stream);
-constexpr int kMaxStreamCtas = 512;           // upper bound on SMs used to size the schedule's workspace
-constexpr int kStreamWarps = 8;               // warps (= ranges of the schedule) per CTA
 int launch_decode_mma(glide_ctx *ctx, const DecodeParams &p, cudaStream_t stream);
 int launch_decode(glide_ctx *ctx, const void *q, const void *k, const void *v, void *out, cudaStream_t stream);
 int decode_occupancy(const glide_ctx *ctx, int *blocks_per_sm);
