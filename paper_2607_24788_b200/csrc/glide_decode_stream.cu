@@ -43,9 +43,9 @@ constexpr int kHdrSlots = 3;
 #endif
 // schedule weights: cost of a state tile, a window tile and of starting a unit in a range
 #ifndef GLIDE_W_STATE
-#define GLIDE_W_STATE 7
-#define GLIDE_W_WIN 5
-#define GLIDE_W_UNIT 6
+#define GLIDE_W_STATE 15
+#define GLIDE_W_WIN 10
+#define GLIDE_W_UNIT 27
 #endif
 
 // Optional per-warp event trace (debug builds only: -DGLIDE_TRACE).
@@ -221,7 +221,7 @@ __device__ __forceinline__ void warp_phi_multi(float (&x)[N][4]) {
     sm[n] = 0.f;
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
-      x[n][i] = exp2f((x[n][i] - mx[n]) * kLog2e);
+      x[n][i] = ex2_approx((x[n][i] - mx[n]) * kLog2e);
       sm[n] += x[n][i];
     }
   }
@@ -231,7 +231,7 @@ __device__ __forceinline__ void warp_phi_multi(float (&x)[N][4]) {
     for (int n = 0; n < N; ++n) sm[n] += __shfl_xor_sync(0xffffffffu, sm[n], o);
 #pragma unroll
   for (int n = 0; n < N; ++n) {
-    const float inv = 1.0f / sm[n];
+    const float inv = __frcp_rn(sm[n]);
 #pragma unroll
     for (int i = 0; i < 4; ++i) x[n][i] *= inv;
   }
@@ -260,6 +260,8 @@ glide_decode_stream_kernel(const DecodeParams p, const StreamParams sp) {
   float *sm_z = reinterpret_cast<float *>(sm_hdr + kWarps * L::kHdrBytes);           // [kWarps][STAGES][16]
   StreamSegment *sm_segs = reinterpret_cast<StreamSegment *>(sm_z + kWarps * STAGES * 16);   // [max_segs]
   uint64_t *sm_bars = reinterpret_cast<uint64_t *>(sm_segs + sp.max_segs);          // [kWarps][STAGES + 1]
+  int *sm_ctr = reinterpret_cast<int *>(sm_bars + kWarps * (STAGES + 1));             // [kStreamMaxGroups]
+  float *sm_pool = reinterpret_cast<float *>(sm_ctr + kStreamMaxGroups);              // [pool slots][kRecFloats]
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 #ifdef GLIDE_TRACE
@@ -284,6 +286,7 @@ glide_decode_stream_kernel(const DecodeParams p, const StreamParams sp) {
   const uint32_t my_z = smem_u32(my_z_ptr);
   const uint32_t my_bars = smem_u32(sm_bars + warp * (STAGES + 1));
   const uint32_t hdr_bar = my_bars + STAGES * 8;
+  if (tid < kStreamMaxGroups) sm_ctr[tid] = 0;
   if (lane == 0) {
     for (int s = 0; s <= STAGES; ++s) mbar_init(my_bars + s * 8, 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -467,7 +470,16 @@ glide_decode_stream_kernel(const DecodeParams p, const StreamParams sp) {
 
   // ---- state tile: 16 rows of S and z, updated in the stage and stored back by the async proxy ---------
   // (bulk stores are not ordered by this warp's later fences, so a ticket never waits for state traffic)
+#ifdef GLIDE_TRACE
+  long long cyc[6] = {0, 0, 0, 0, 0, 0};
+#define GLIDE_CYC_MARK(var) long long var = clock64()
+#define GLIDE_CYC_ADD(i, var) do { long long n_ = clock64(); cyc[i] += n_ - var; var = n_; } while (0)
+#else
+#define GLIDE_CYC_MARK(var) do { } while (0)
+#define GLIDE_CYC_ADD(i, var) do { } while (0)
+#endif
   auto consume_state = [&](const StreamSegment &sg, int stile, float4 *st, float *zs, uint32_t st_addr, uint32_t z_addr) {
+    GLIDE_CYC_MARK(cm);
     const int src0 = stile * 4;   // lane that holds phi entries of the tile's first row (4 rows per lane)
 #pragma unroll
     for (int r = 0; r < kTileRows; ++r) {
@@ -487,6 +499,7 @@ glide_decode_stream_kernel(const DecodeParams p, const StreamParams sp) {
         a[h].w = fmaf(f, s.w, a[h].w);
       }
     }
+    GLIDE_CYC_ADD(0, cm);
     // z: lane r < 16 owns row r of the tile
     const int zsrc = src0 + ((lane & 15) >> 2);
     float zn = 0.f;
@@ -507,8 +520,10 @@ glide_decode_stream_kernel(const DecodeParams p, const StreamParams sp) {
         bp[h - 1] = fmaf(f, zn, bp[h - 1]);
       }
     }
+    GLIDE_CYC_ADD(1, cm);
     fence_async_smem();   // the updated rows are read by the async proxy
     __syncwarp();
+    GLIDE_CYC_ADD(2, cm);
     if (lane == 0) {
       float *Sg = reinterpret_cast<float *>(p.ws + size_t(sg.S_off256) * 256) + size_t(stile) * kTileRows * kD;
       float *zg = reinterpret_cast<float *>(p.ws + size_t(sg.z_off256) * 256) + stile * kTileRows;
@@ -517,6 +532,7 @@ glide_decode_stream_kernel(const DecodeParams p, const StreamParams sp) {
       bulk_commit();
       bulk_wait_read0();   // the stage may be refilled once the store has read it
     }
+    GLIDE_CYC_ADD(3, cm);
   };
 
   // ---- main loop over this warp's segments ------------------------------------------------------------
@@ -535,6 +551,7 @@ glide_decode_stream_kernel(const DecodeParams p, const StreamParams sp) {
       failed = true;
       break;
     }
+    GLIDE_TRACE_EVENT(15);
     {
       const uint32_t *hq = reinterpret_cast<const uint32_t *>(my_hdr_ptr);
       const bool valid = hrow < G;
@@ -565,6 +582,7 @@ glide_decode_stream_kernel(const DecodeParams p, const StreamParams sp) {
       }
     }
     __syncwarp();
+    GLIDE_TRACE_EVENT(16);
     if (s + 1 < seg_hi) issue_header(s + 1);
     if (has_win) {
       const int64_t lim = t < int64_t(sg.cap) ? t : int64_t(sg.cap);
@@ -605,6 +623,7 @@ glide_decode_stream_kernel(const DecodeParams p, const StreamParams sp) {
     }
     if (failed) break;
 
+    GLIDE_TRACE_EVENT(17);
     // -- finish: record (m, l, acc) in a common layout: lane holds features 4*lane..4*lane+3 of every head --
     float mh[G], lh[G];
     float4 acc[G];
@@ -650,7 +669,9 @@ glide_decode_stream_kernel(const DecodeParams p, const StreamParams sp) {
         acc[h] = make_float4(0.f, 0.f, 0.f, 0.f);
       }
     }
+    GLIDE_TRACE_EVENT(18);
     if (n_total > 0) issue_next();   // the deferred refill
+    GLIDE_TRACE_EVENT(19);
     if (n_state_eff > 0) {           // fold the linear readout in as a term with logit 0
       warp_sum_multi<G>(bp);
 #pragma unroll
@@ -665,8 +686,70 @@ glide_decode_stream_kernel(const DecodeParams p, const StreamParams sp) {
         mh[h] = mn;
       }
     }
+    GLIDE_TRACE_EVENT(20);
+    if (sg.grp_size > 1) {
+      // several warps of this CTA share the unit: records meet in shared memory, the last one to arrive
+      // combines them and carries the unit on
+      float *slot = sm_pool + size_t(sg.grp_slot0 + sg.grp_idx) * L::kRecFloats;
+#pragma unroll
+      for (int h = 0; h < G; ++h) {
+        *reinterpret_cast<float4 *>(slot + h * kD + lane * 4) = acc[h];
+        if (lane == 0) {
+          slot[G * kD + h] = mh[h];
+          slot[G * kD + G + h] = lh[h];
+        }
+      }
+      __syncwarp();
+      int lastc = 0;
+      if (lane == 0) {
+        // shared-memory accesses of one SM are performed in order: the record written above (ordered by the
+        // __syncwarp) is visible to whichever warp sees this arrival
+        // (a relaxed atomic: a fence here would also wait for this warp's outstanding global stores)
+        unsigned old;
+        asm volatile("atom.relaxed.cta.shared.add.u32 %0, [%1], 1;" : "=r"(old) : "r"(smem_u32(&sm_ctr[sg.grp_ctr])) : "memory");
+        lastc = int(old) == sg.grp_size - 1;
+      }
+      lastc = __shfl_sync(0xffffffffu, lastc, 0);
+      GLIDE_TRACE_EVENT(21);
+      if (!lastc) continue;
+      // at most 8 records (one per warp); fully unrolled so that the shared-memory loads overlap
+      const float *g0 = sm_pool + size_t(sg.grp_slot0) * L::kRecFloats;
+      float fr[kWarps][G];
+#pragma unroll
+      for (int h = 0; h < G; ++h) {
+        float Mg = -CUDART_INF_F;
+#pragma unroll
+        for (int i = 0; i < kWarps; ++i) {
+          fr[i][h] = i < sg.grp_size ? g0[size_t(i) * L::kRecFloats + G * kD + h] : -CUDART_INF_F;
+          Mg = fmaxf(Mg, fr[i][h]);
+        }
+        float lg = 0.f;
+#pragma unroll
+        for (int i = 0; i < kWarps; ++i) {
+          fr[i][h] = exp2_or_zero(fr[i][h], Mg);
+          if (i < sg.grp_size) lg = fmaf(g0[size_t(i) * L::kRecFloats + G * kD + G + h], fr[i][h], lg);
+        }
+        mh[h] = Mg;
+        lh[h] = lg;
+        acc[h] = make_float4(0.f, 0.f, 0.f, 0.f);
+      }
+#pragma unroll
+      for (int i = 0; i < kWarps; ++i) {
+        if (i < sg.grp_size) {
+#pragma unroll
+          for (int h = 0; h < G; ++h) {
+            const float4 av = *reinterpret_cast<const float4 *>(g0 + size_t(i) * L::kRecFloats + h * kD + lane * 4);
+            acc[h].x = fmaf(av.x, fr[i][h], acc[h].x);
+            acc[h].y = fmaf(av.y, fr[i][h], acc[h].y);
+            acc[h].z = fmaf(av.z, fr[i][h], acc[h].z);
+            acc[h].w = fmaf(av.w, fr[i][h], acc[h].w);
+          }
+        }
+      }
+      GLIDE_TRACE_EVENT(22);
+    }
     if (sg.part >= 0) {
-      // the unit is cut by a range boundary: this warp's record goes to global scratch; its ticket is taken
+      // the unit is cut by a CTA boundary: this record goes to global scratch; its ticket is taken
       // at the end of the range, so that the streaming loop never stalls on a fence or an atomic
       float *grec = p.partials + (size_t(sg.rec0) + sg.part) * p.rec_floats;
 #pragma unroll
@@ -725,11 +808,33 @@ glide_decode_stream_kernel(const DecodeParams p, const StreamParams sp) {
       __threadfence();
       const StreamSegment &sg = sm_segs[pi == 0 ? pend0 : pend1];
       const bool has_win = sg.cap > 0;
-      // reload the unit's query rows and current token (this warp may have moved on to another unit since)
+      // reload the unit's query rows and current token (this warp may have moved on to another unit since);
+      // every load of the merge's first batch is issued before anything is reduced
       const bf16 *qall = reinterpret_cast<const bf16 *>(p.q);
+      const float *r0 = p.partials + size_t(sg.rec0) * p.rec_floats;
+      constexpr int RPB = 32 / G;   // records per batch
       const uint2 ktb = *reinterpret_cast<const uint2 *>(reinterpret_cast<const bf16 *>(p.k) + size_t(sg.unit) * kD + lane * 4);
       const uint2 vtb = *reinterpret_cast<const uint2 *>(reinterpret_cast<const bf16 *>(p.v) + size_t(sg.unit) * kD + lane * 4);
       int orow[G];
+      uint2 qbits[G];
+#pragma unroll
+      for (int h = 0; h < G; ++h) {
+        orow[h] = sg.qrow0 + (sp.heads_contiguous ? h : p.heads_of[sg.g * G + h]);
+        qbits[h] = *reinterpret_cast<const uint2 *>(qall + size_t(orow[h]) * kD + lane * 4);
+      }
+      float me0, le0;
+      float4 vv0[RPB][G];
+      {
+        const int ri = lane / G, rh = lane % G;
+        const bool valid = ri < sg.n_parts;
+        me0 = valid ? __ldcg(r0 + size_t(ri) * p.rec_floats + G * kD + rh) : -CUDART_INF_F;
+        le0 = valid ? __ldcg(r0 + size_t(ri) * p.rec_floats + G * kD + G + rh) : 0.f;
+#pragma unroll
+        for (int u = 0; u < RPB; ++u)
+#pragma unroll
+          for (int h = 0; h < G; ++h)
+            if (u < sg.n_parts) vv0[u][h] = __ldcg(reinterpret_cast<const float4 *>(r0 + size_t(u) * p.rec_floats + h * kD + lane * 4));
+      }
       float sc[G];
       {
         float kx[4];
@@ -739,19 +844,16 @@ glide_decode_stream_kernel(const DecodeParams p, const StreamParams sp) {
         kx[3] = __uint_as_float(ktb.y & 0xffff0000u);
 #pragma unroll
         for (int h = 0; h < G; ++h) {
-          orow[h] = sg.qrow0 + (sp.heads_contiguous ? h : p.heads_of[sg.g * G + h]);
-          float qx[4];
-          load_elems<bf16, 4>(qall + size_t(orow[h]) * kD + lane * 4, qx);
-          sc[h] = 0.f;
-#pragma unroll
-          for (int i = 0; i < 4; ++i) sc[h] = fmaf(qx[i], kx[i], sc[h]);
+          sc[h] = fmaf(__uint_as_float(qbits[h].x << 16), kx[0], 0.f);
+          sc[h] = fmaf(__uint_as_float(qbits[h].x & 0xffff0000u), kx[1], sc[h]);
+          sc[h] = fmaf(__uint_as_float(qbits[h].y << 16), kx[2], sc[h]);
+          sc[h] = fmaf(__uint_as_float(qbits[h].y & 0xffff0000u), kx[3], sc[h]);
         }
         warp_sum_multi<G>(sc);
 #pragma unroll
         for (int h = 0; h < G; ++h) sc[h] = has_win ? sc[h] * p.scale_log2 : -CUDART_INF_F;
       }
       // merge the records: maxima and sums first (one (record, head) pair per lane), then the vectors
-      const float *r0 = p.partials + size_t(sg.rec0) * p.rec_floats;
       float Mg[G], lg[G];
       float4 acc[G];
 #pragma unroll
@@ -760,19 +862,21 @@ glide_decode_stream_kernel(const DecodeParams p, const StreamParams sp) {
         lg[h] = 0.f;
         acc[h] = make_float4(0.f, 0.f, 0.f, 0.f);
       }
-      constexpr int RPB = 32 / G;   // records per batch
       for (int i0 = 0; i0 < sg.n_parts; i0 += RPB) {
-        const int ri = i0 + lane / G, rh = lane % G;
-        const bool valid = ri < sg.n_parts;
-        const float me = valid ? __ldcg(r0 + size_t(ri) * p.rec_floats + G * kD + rh) : -CUDART_INF_F;
-        const float le = valid ? __ldcg(r0 + size_t(ri) * p.rec_floats + G * kD + G + rh) : 0.f;
+        const int rh = lane % G;
         const int nb = sg.n_parts - i0 < RPB ? sg.n_parts - i0 : RPB;
-        float4 vv[RPB][G];   // the batch's vectors: all loads in flight together with the scalars above
+        float me = me0, le = le0;
+        if (i0 > 0) {   // further batches (units cut into more than RPB records)
+          const int ri = i0 + lane / G;
+          const bool valid = ri < sg.n_parts;
+          me = valid ? __ldcg(r0 + size_t(ri) * p.rec_floats + G * kD + rh) : -CUDART_INF_F;
+          le = valid ? __ldcg(r0 + size_t(ri) * p.rec_floats + G * kD + G + rh) : 0.f;
 #pragma unroll
-        for (int u = 0; u < RPB; ++u)
+          for (int u = 0; u < RPB; ++u)
 #pragma unroll
-          for (int h = 0; h < G; ++h)
-            if (u < nb) vv[u][h] = __ldcg(reinterpret_cast<const float4 *>(r0 + size_t(i0 + u) * p.rec_floats + h * kD + lane * 4));
+            for (int h = 0; h < G; ++h)
+              if (u < nb) vv0[u][h] = __ldcg(reinterpret_cast<const float4 *>(r0 + size_t(i0 + u) * p.rec_floats + h * kD + lane * 4));
+        }
         float Mn[G];
 #pragma unroll
         for (int h = 0; h < G; ++h) Mn[h] = rh == h ? me : -CUDART_INF_F;
@@ -803,10 +907,10 @@ glide_decode_stream_kernel(const DecodeParams p, const StreamParams sp) {
           for (int h = 0; h < G; ++h)
             if (u < nb) {
               const float f = __shfl_sync(0xffffffffu, fe, u * G + h);
-              acc[h].x = fmaf(vv[u][h].x, f, acc[h].x);
-              acc[h].y = fmaf(vv[u][h].y, f, acc[h].y);
-              acc[h].z = fmaf(vv[u][h].z, f, acc[h].z);
-              acc[h].w = fmaf(vv[u][h].w, f, acc[h].w);
+              acc[h].x = fmaf(vv0[u][h].x, f, acc[h].x);
+              acc[h].y = fmaf(vv0[u][h].y, f, acc[h].y);
+              acc[h].z = fmaf(vv0[u][h].z, f, acc[h].z);
+              acc[h].w = fmaf(vv0[u][h].w, f, acc[h].w);
             }
       }
       float vx[4];
@@ -836,6 +940,11 @@ glide_decode_stream_kernel(const DecodeParams p, const StreamParams sp) {
     }
   }
   if (failed && lane == 0) atomicExch(&p.ctl->status, kDevWaitTimeout);
+#ifdef GLIDE_TRACE
+  if (g_stream_trace && lane == 0)
+    for (int i = 0; i < 4; ++i)
+      g_stream_trace[(size_t(blockIdx.x) * kWarps + warp) * 64 + 60 + i] = (static_cast<unsigned long long>(100 + i) << 56) | (unsigned long long)cyc[i];
+#endif
   if (lane == 0) bulk_wait0();   // this warp's state stores have landed
   GLIDE_TRACE_EVENT(9);
 
@@ -855,27 +964,29 @@ template <int G, int STAGES>
 size_t stream_smem_bytes(int max_segs) {
   using L = Layout<G>;
   return 1024 + size_t(kWarps) * STAGES * kStageBytes + size_t(kWarps) * L::kHdrBytes + size_t(kWarps) * STAGES * 64 +
-         size_t(max_segs) * sizeof(StreamSegment) + size_t(kWarps) * (STAGES + 1) * 8;
+         size_t(max_segs) * sizeof(StreamSegment) + size_t(kWarps) * (STAGES + 1) * 8 + size_t(kStreamMaxGroups) * 4 +
+         size_t(kStreamPoolBytes / (L::kRecFloats * 4)) * L::kRecFloats * 4;
 }
 
 template <typename F>
 int dispatch_stream(int G, F &&f) {
   switch (G) {
-    case 1: return f(IntTag<1>{}, IntTag<3>{});
-    case 2: return f(IntTag<2>{}, IntTag<3>{});
+    case 1: return f(IntTag<1>{}, IntTag<GLIDE_STREAM_STAGES>{});
+    case 2: return f(IntTag<2>{}, IntTag<GLIDE_STREAM_STAGES>{});
     case 4: return f(IntTag<4>{}, IntTag<GLIDE_STREAM_STAGES>{});
-    case 8: return f(IntTag<8>{}, IntTag<3>{});
+    case 8: return f(IntTag<8>{}, IntTag<GLIDE_STREAM_STAGES>{});
     default: return int(GLIDE_ERR_UNSUPPORTED);
   }
 }
 
 }  // namespace
 
-// Cuts the tile stream into `n_ranges` equally heavy contiguous ranges, one per warp.  A state tile weighs
-// 2 (read + write), a window tile 1, and starting a unit costs kUnitWeight (header, feature maps, finish).
+// Cuts the tile stream into `n_ranges` equally heavy contiguous ranges, one per warp.  The weights are the
+// measured costs of a state tile, a window tile and of a segment (header, feature maps, finish) relative to
+// each other.
 void build_stream_schedule(const glide_ctx *ctx, int n_ranges, std::vector<StreamSegment> *segs,
                            std::vector<int32_t> *range_seg_begin, int *max_segs_per_cta, size_t *n_records) {
-  constexpr int64_t kUnitWeight = GLIDE_W_UNIT, kStateWeight = GLIDE_W_STATE, kWinWeight = GLIDE_W_WIN;
+  constexpr int64_t kSegWeight = GLIDE_W_UNIT, kStateWeight = GLIDE_W_STATE, kWinWeight = GLIDE_W_WIN;
   const int L = ctx->cfg.n_layers, B = ctx->cfg.batch, Hkv = ctx->cfg.n_kv_heads, d = ctx->cfg.head_dim;
   const int64_t units_per_layer = int64_t(B) * Hkv;
   bool contiguous_heads = true;
@@ -901,7 +1012,7 @@ void build_stream_schedule(const glide_ctx *ctx, int n_ranges, std::vector<Strea
       UnitTiles ut{l, int(int64_t(l) * units_per_layer + u), ld.evicts ? d / kTileRows : 0,
                    int((ld.cap + kTileRows - 1) / kTileRows)};
       units.push_back(ut);
-      total_w += kStateWeight * int64_t(ut.n_state) + kWinWeight * int64_t(ut.n_win) + kUnitWeight;
+      total_w += kStateWeight * int64_t(ut.n_state) + kWinWeight * int64_t(ut.n_win) + kSegWeight;
     }
   }
   segs->clear();
@@ -910,14 +1021,19 @@ void build_stream_schedule(const glide_ctx *ctx, int n_ranges, std::vector<Strea
   size_t ui = 0;
   int st_done = 0, win_done = 0;   // progress inside units[ui]
   int64_t cum = 0;
+  total_w += int64_t(n_ranges) * kSegWeight;   // a range boundary inside a unit adds a segment
   std::vector<std::vector<size_t>> unit_segs(units.size());
   for (int c = 0; c < n_ranges; ++c) {
     (*range_seg_begin)[c] = int32_t(segs->size());
     const int64_t target = (c + 1 == n_ranges) ? total_w : (total_w * (c + 1) + n_ranges - 1) / n_ranges;
+    bool first = true;
     while (ui < units.size() && cum < target) {
+      // opening another segment costs kSegWeight by itself: only worth it if about half of that fits
+      if (!first && c + 1 < n_ranges && target - cum < (kSegWeight + kWinWeight) / 2) break;
+      first = false;
       const UnitTiles &ut = units[ui];
       const LayerDev &ld = ctx->layers[ut.layer];
-      if (st_done == 0 && win_done == 0) cum += kUnitWeight;
+      cum += kSegWeight;   // header, feature maps and finish of a segment
       int64_t room = std::max<int64_t>(target - cum, 1);
       StreamSegment sg{};
       sg.unit = ut.unit;
@@ -960,20 +1076,49 @@ void build_stream_schedule(const glide_ctx *ctx, int n_ranges, std::vector<Strea
   *max_segs_per_cta = 0;
   for (int c = 0; c + kWarps <= n_ranges; c += kWarps)
     *max_segs_per_cta = std::max<int>(*max_segs_per_cta, (*range_seg_begin)[c + kWarps] - (*range_seg_begin)[c]);
+  // Warps of one CTA that share a unit reduce their records in shared memory first (a "group"); only one
+  // record per group goes to global scratch, and a unit that lies inside one group never touches it.
+  const int pool_slots = kStreamPoolBytes / (ctx->rec_floats * 4);
+  std::vector<int> cta_slots(size_t(n_ranges / kWarps) + 1, 0), cta_groups(size_t(n_ranges / kWarps) + 1, 0);
+  std::vector<int> seg_range(segs->size(), 0);
+  for (int c = 0; c < n_ranges; ++c)
+    for (int i = (*range_seg_begin)[c]; i < (*range_seg_begin)[c + 1]; ++i) seg_range[i] = c;
   for (size_t u = 0; u < units.size(); ++u) {
     const std::vector<size_t> &list = unit_segs[u];
-    if (list.size() == 1) {
-      (*segs)[list[0]].part = -1;
-      (*segs)[list[0]].n_parts = 1;
-      (*segs)[list[0]].rec0 = 0;
-    } else {
-      for (size_t i = 0; i < list.size(); ++i) {
-        (*segs)[list[i]].part = int32_t(i);
-        (*segs)[list[i]].n_parts = int32_t(list.size());
-        (*segs)[list[i]].rec0 = int32_t(records);
+    // split the unit's segments (ordered by range) into groups of one CTA each
+    std::vector<std::pair<size_t, size_t>> groups;   // [first, last) into list
+    for (size_t i = 0; i < list.size();) {
+      const int cta = seg_range[list[i]] / kWarps;
+      size_t j = i + 1;
+      while (j < list.size() && seg_range[list[j]] / kWarps == cta) ++j;
+      const int need = int(j - i);
+      if (need >= 2 && cta_slots[cta] + need <= pool_slots && cta_groups[cta] < kStreamMaxGroups) {
+        for (size_t k = i; k < j; ++k) {
+          StreamSegment &sg = (*segs)[list[k]];
+          sg.grp_size = need;
+          sg.grp_slot0 = cta_slots[cta];
+          sg.grp_idx = int(k - i);
+          sg.grp_ctr = cta_groups[cta];
+        }
+        cta_slots[cta] += need;
+        cta_groups[cta] += 1;
+        groups.emplace_back(i, j);
+      } else {   // single warp, or no room left in the CTA's pool: every segment is its own group
+        for (size_t k = i; k < j; ++k) {
+          (*segs)[list[k]].grp_size = 1;
+          groups.emplace_back(k, k + 1);
+        }
       }
-      records += list.size();
+      i = j;
     }
+    for (size_t gi = 0; gi < groups.size(); ++gi)
+      for (size_t k = groups[gi].first; k < groups[gi].second; ++k) {
+        StreamSegment &sg = (*segs)[list[k]];
+        sg.part = groups.size() == 1 ? -1 : int32_t(gi);
+        sg.n_parts = int32_t(groups.size());
+        sg.rec0 = groups.size() == 1 ? 0 : int32_t(records);
+      }
+    if (groups.size() > 1) records += groups.size();
   }
   *n_records = records;
 }

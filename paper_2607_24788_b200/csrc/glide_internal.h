@@ -71,6 +71,8 @@ struct DecodeParams {
 
 constexpr int kMaxStreamCtas = 192;           // CTAs (one per SM) the streaming decode kernel's schedule can address
 constexpr int kStreamWarps = 8;               // warps (= ranges of the schedule) per CTA
+constexpr int kStreamPoolBytes = 56 * 1024;   // shared-memory record slots for the CTA-level reduction
+constexpr int kStreamMaxGroups = 32;          // reduction groups per CTA
 
 // One segment of the streaming decode kernel's schedule: the part of one unit that falls into one warp's
 // range of the tile stream (state tiles first, then window tiles).  64 bytes.
@@ -79,7 +81,7 @@ struct StreamSegment {
   int32_t range;             // warp (0..7) of the CTA that owns the segment
   int32_t n_state, state0;   // state tiles [state0, state0 + n_state): 16 rows of S each
   int32_t n_win, win0;       // window tiles [win0, win0 + n_win): 16 ring slots each
-  int32_t part;              // this warp's record among the unit's records, -1 if the whole unit is in this range
+  int32_t part;              // this group's record among the unit's global records, -1 if the whole unit is in this group
   int32_t n_parts;           // records of the unit (ticket target)
   int32_t rec0;              // index of the unit's first record in the split-K scratch
   int32_t row_base;          // row of the unit's slot 0 in the layer's [rows][d] ring tensor
@@ -90,7 +92,10 @@ struct StreamSegment {
   int32_t ringK_off256, ringV_off256;  // workspace byte offsets / 256 of the layer's K and V rings
   int32_t qrow0;             // row of the KV head's first query head in the [L*B*H][d] q / out tensors
   int32_t g;                 // KV head index (for the head table when the groups are not contiguous)
-  int32_t pad_[4];
+  int32_t grp_size;          // warps of this CTA that share the unit (1: none); they reduce in shared memory first
+  int32_t grp_slot0;         // first shared-memory record slot of the group
+  int32_t grp_idx;           // this segment's slot within the group
+  int32_t grp_ctr;           // the group's arrival counter in shared memory
 };
 static_assert(sizeof(StreamSegment) == 96, "StreamSegment is copied as 16-byte chunks");
 
