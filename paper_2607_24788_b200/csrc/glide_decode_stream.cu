@@ -268,7 +268,9 @@ glide_decode_stream_kernel(const DecodeParams p, const StreamParams sp) {
   int trace_n = 0;
 #endif
   GLIDE_TRACE_EVENT(1);
-  const int64_t t = p.n_dev[0];   // every layer is at the same position (checked by the host)
+  // Programmatic dependent launch: the next launch in the stream may start its prologue on SMs this grid has
+  // left; whatever an earlier kernel wrote is read only after griddepcontrol.wait below.
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   const int col2 = (lane & 3) * 2, hrow = lane >> 2;
   // the CTA's slice of the segment list: offsets come with the kernel parameters (no dependent global load)
   const int cta_seg_begin = sp.cta_seg_begin[blockIdx.x];
@@ -293,6 +295,8 @@ glide_decode_stream_kernel(const DecodeParams p, const StreamParams sp) {
     fence_async_smem();
   }
   __syncthreads();   // segment table and barriers ready; the warps are on their own from here
+  asm volatile("griddepcontrol.wait;" ::: "memory");   // the preceding kernel has completed and its writes are visible
+  const int64_t t = p.n_dev[0];   // every layer is at the same position (checked by the host)
   // this warp's segments: the run of the CTA's list that carries its index
   int seg_lo = 0;
   while (seg_lo < cta_nseg && sm_segs[seg_lo].range < warp) ++seg_lo;
@@ -1175,8 +1179,20 @@ int launch_decode_stream(glide_ctx *ctx, const DecodeParams &p, cudaStream_t str
   sp.kv4d = ctx->tmaps_kv4d ? 1 : 0;
   return dispatch_stream(ctx->G, [&](auto gg, auto ss) -> int {
     constexpr int G = decltype(gg)::value, S = decltype(ss)::value;
-    glide_decode_stream_kernel<G, S><<<ctx->decode_grid, kThreads, ctx->stream_smem, stream>>>(p, sp);
-    if (cudaGetLastError() != cudaSuccess) return GLIDE_ERR_CUDA;
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3(unsigned(ctx->decode_grid));
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = ctx->stream_smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    if (cudaLaunchKernelEx(&cfg, glide_decode_stream_kernel<G, S>, p, sp) != cudaSuccess) {
+      cudaGetLastError();
+      return GLIDE_ERR_CUDA;
+    }
     return GLIDE_OK;
   });
 }
