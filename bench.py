@@ -210,6 +210,21 @@ def build_states(shape, n_replicas: int, extra_tokens: int, device):
     return ctxs, wl
 
 
+def max_over_ranks(values, dist, device):
+    """Replicas only: every rank times its own independent copy of the workload; the job's time is the
+    slowest rank's (max over ranks).  `dist` is torch.distributed or None for a single process."""
+    if dist is None:
+        return [float(v) for v in values]
+    t = torch.tensor([float(v) for v in values], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(x) for x in t.cpu()]
+
+
+def whole_job_tokens_per_s(world: int, batch: int, steps: int, ms: float) -> float:
+    """Aggregate over all replicas: every rank decodes `batch` sequences for `steps` steps in `ms`."""
+    return world * batch * steps / (ms * 1e-3)
+
+
 def run_glide(args, shape):
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -316,10 +331,7 @@ def run_glide(args, shape):
         e2e_ms.append(ev0.elapsed_time(ev1))
     e2e_t = statistics.median(e2e_ms)
 
-    if dist is not None:
-        t = torch.tensor([t_ms, hot_ms, e2e_t], dtype=torch.float64, device=device)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        t_ms, hot_ms, e2e_t = (float(x) for x in t.cpu())
+    t_ms, hot_ms, e2e_t = max_over_ranks([t_ms, hot_ms, e2e_t], dist, device)
 
     if rank == 0:
         peak, peak_kind = load_peaks()
@@ -328,7 +340,7 @@ def run_glide(args, shape):
         info = ctxs[0].glide_decode_launch_info()
         elem = shape.elem_bytes
         line = {
-            "metric": "hybrid-attn decode tokens/s", "value": world * B * K / (t_ms * 1e-3), "unit": "tokens/s",
+            "metric": "hybrid-attn decode tokens/s", "value": whole_job_tokens_per_s(world, B, K, t_ms), "unit": "tokens/s",
             "n_gpus": world, "steps": K, "warmup": max(W, 3), "ms_per_step": t_ms / K, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f32" if shape.dtype == "f32" else "bf16+f32state",
             "data": "synthetic",

@@ -1,0 +1,136 @@
+"""Host-side logic that needs no GPU: the C ABI loads and exports what include/glide.h declares, argument
+checking, workspace sizing, error strings, and the N>1 timing aggregation of the benchmark (gloo, 2 ranks)."""
+import ctypes
+import os
+import re
+import subprocess
+import sys
+
+import pytest
+import torch
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def glide():
+    from paper_2607_24788_b200 import build, glide as g
+    build.build()
+    g.load_library()
+    return g
+
+
+def declared_functions():
+    text = open(os.path.join(ROOT, "include", "glide.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(glide_[a-z_]+)\s*\(", text)))
+
+
+def test_library_exports_every_declared_symbol(glide):
+    lib = ctypes.CDLL(glide.LIB_PATH)
+    names = declared_functions()
+    assert {"glide_create", "glide_prefill", "glide_decode_step", "glide_destroy", "glide_workspace_bytes"} <= set(names)
+    for n in names:
+        assert hasattr(lib, n), f"{n} is declared in include/glide.h but not exported"
+
+
+def test_no_torch_types_in_the_abi():
+    text = open(os.path.join(ROOT, "include", "glide.h")).read()
+    assert "torch" not in text and "at::" not in text and "#include <cuda" not in text
+
+
+def test_strerror(glide):
+    assert glide.strerror(0) == "ok"
+    assert "workspace" in glide.strerror(glide.GLIDE_ERR_WORKSPACE_TOO_SMALL)
+    assert glide.strerror(12345) == "unknown status"
+
+
+def _cfg(glide, **kw):
+    base = dict(windows=[64, 16], batch=2, n_q_heads=8, n_kv_heads=2, head_dim=128, max_tokens=100,
+                dtype=torch.bfloat16)
+    base.update(kw)
+    return glide.make_config(**base)
+
+
+def test_workspace_bytes_scales_with_rings_and_state(glide):
+    cfg, keep = _cfg(glide)
+    small = glide.glide_workspace_bytes(cfg)
+    cfg2, keep2 = _cfg(glide, windows=[64 + 4096, 16])
+    big = glide.glide_workspace_bytes(cfg2)
+    # the first layer's capacity is min(w, max_tokens) = 100: its two rings grow by (100 - 64) slots per unit;
+    # the layer no longer evicts, so its state work items (and their scratch records) go away
+    ring_growth = 2 * 2 * 2 * (100 - 64) * 128 * 2
+    assert abs((big - small) - ring_growth) < (1 << 20) and big > small
+    cfg3, keep3 = _cfg(glide, dtype=torch.float32, head_dim=64)
+    assert glide.glide_workspace_bytes(cfg3) > 0
+
+
+@pytest.mark.parametrize("kw,code", [
+    (dict(head_dim=96), 2), (dict(n_q_heads=6, n_kv_heads=4), 2), (dict(n_q_heads=24, n_kv_heads=2), 2),
+    (dict(windows=[-1, 4]), 1), (dict(max_tokens=0), 1), (dict(prefill_chunk=100), 1), (dict(decode_impl=9), 1),
+    (dict(q_to_kv=[0, 0, 0, 0, 0, 1, 1, 1]), 2), (dict(q_to_kv=[0, 0, 0, 0, 1, 1, 1, 7]), 1),
+    (dict(dtype=torch.float32, decode_impl=3), 2),
+])
+def test_invalid_configurations_are_rejected(glide, kw, code):
+    cfg, keep = _cfg(glide, **kw)
+    out = ctypes.c_size_t(0)
+    assert glide.load_library().glide_workspace_bytes(ctypes.byref(cfg), ctypes.byref(out)) == code
+
+
+def test_create_validates_before_touching_cuda(glide):
+    lib = glide.load_library()
+    cfg, keep = _cfg(glide)
+    handle = ctypes.c_void_p()
+    assert lib.glide_create(ctypes.byref(cfg), None, 1 << 30, None, ctypes.byref(handle)) == glide.GLIDE_ERR_INVALID_ARG
+    assert lib.glide_create(ctypes.byref(cfg), 256, 16, None, ctypes.byref(handle)) == glide.GLIDE_ERR_WORKSPACE_TOO_SMALL
+    assert lib.glide_create(ctypes.byref(cfg), 257, 1 << 40, None, ctypes.byref(handle)) == glide.GLIDE_ERR_INVALID_ARG
+    assert not handle.value
+    assert lib.glide_destroy(None) == glide.GLIDE_ERR_INVALID_ARG
+    assert lib.glide_decode_step(None, None, None, None, None, None) == glide.GLIDE_ERR_INVALID_ARG
+
+
+def test_binding_fails_loudly_without_the_library(glide, monkeypatch):
+    monkeypatch.setattr(glide, "_lib", None)
+    monkeypatch.setattr(glide, "LIB_PATH", "/nonexistent/libglide.so")
+    with pytest.raises(RuntimeError, match="no CPU or PyTorch fallback"):
+        glide.load_library()
+
+
+_RANK_SCRIPT = r"""
+import os, sys, json
+sys.path.insert(0, {root!r})
+import torch, torch.distributed as dist
+import bench
+dist.init_process_group("gloo")
+rank = dist.get_rank()
+vals = bench.max_over_ranks([10.0 + rank, 5.0 - rank, 7.0], dist, torch.device("cpu"))
+if rank == 0:
+    print(json.dumps(dict(vals=vals, value=bench.whole_job_tokens_per_s(dist.get_world_size(), 4, 10, vals[0]))))
+dist.barrier()
+dist.destroy_process_group()
+"""
+
+
+def test_multi_rank_timing_is_max_over_ranks_and_value_sums_replicas(tmp_path):
+    script = tmp_path / "rank.py"
+    script.write_text(_RANK_SCRIPT.format(root=ROOT))
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node=2", "--master-addr", "127.0.0.1",
+           "--master-port", "29731", str(script)]
+    r = subprocess.run(cmd, capture_output=True, text=True, timeout=240)
+    assert r.returncode == 0, r.stderr[-2000:]
+    import json
+    line = [l for l in r.stdout.splitlines() if l.startswith("{")][-1]
+    got = json.loads(line)
+    assert got["vals"] == [11.0, 5.0, 7.0]
+    assert got["value"] == pytest.approx(2 * 4 * 10 / 11e-3)
+
+
+def test_reference_arm_prints_one_json_line_on_cpu():
+    # the reference arm (CPU oracle) on the tiny configuration; also exercises bench.py's argument handling
+    r = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--workload", "c0_tiny_f32",
+                        "--steps", "4", "--warmup", "1"], capture_output=True, text=True, timeout=240)
+    assert r.returncode == 0, r.stderr[-2000:]
+    import json
+    d = json.loads(r.stdout.strip().splitlines()[-1])
+    assert d["impl"] == "reference" and d["unit"] == "tokens/s" and d["value"] > 0
+    assert d["cpu_baseline"]["kind"] == "oracle" and d["e2e"]["h2d_bytes_per_step"] == 0
