@@ -46,7 +46,8 @@ typedef enum {
   GLIDE_ERR_WORKSPACE_TOO_SMALL = 3,
   GLIDE_ERR_CAPACITY = 4,            /* tokens absorbed + T would exceed max_tokens */
   GLIDE_ERR_STATE = 5,               /* decode with layers at different positions */
-  GLIDE_ERR_CUDA = 6                 /* a CUDA runtime call or launch failed */
+  GLIDE_ERR_CUDA = 6,                /* a CUDA runtime call or launch failed */
+  GLIDE_ERR_SCRATCH_LIMIT = 7        /* glide_decode_step_noalloc: the split-K scratch would not fit the static buffer */
 } glide_status;
 
 typedef enum { GLIDE_F32 = 0, GLIDE_BF16 = 1 } glide_dtype;
@@ -126,6 +127,33 @@ int glide_prefill(glide_ctx *ctx, int32_t layer_begin, int32_t layer_count, int6
  * All layers must be at the same position (GLIDE_ERR_STATE otherwise). */
 int glide_decode_step(glide_ctx *ctx, const void *dev_q, const void *dev_k, const void *dev_v, void *dev_out,
                       void *stream);
+
+/* Decode step for callers that must not allocate.  (The paper has no counterpart: this is a deployment
+ * variant of glide_decode_step, not part of the method.)
+ *
+ * Who needs it: a serving process that hands every byte of device memory to its own arena at start-up (KV
+ * cache, weights) and from then on treats cudaMalloc as forbidden -- because it can fail when the arena has
+ * taken the whole GPU, because it synchronises the device, or because the process runs under a budget that
+ * audits allocations.  glide_decode_step itself never allocates either, but it keeps its split-K scratch
+ * (control words, tickets, partial records) in the caller's workspace; a caller that wants the workspace to
+ * hold only persistent state (rings, S, z, tables) and nothing transient can use this call instead: the same
+ * step, computed by the CUDA-core decode kernel (any I/O dtype), with that scratch in a buffer that is part of
+ * the library image: a file-scope `static __device__` array of GLIDE_NOALLOC_SCRATCH_BYTES (8 MiB), which
+ * every GPU that loads the library holds until the process exits.
+ *
+ *   - Same arguments, layouts, state updates and error behaviour as glide_decode_step; results agree with it
+ *     to the tolerance of the I/O dtype (a different kernel may round differently).
+ *   - Configurations whose scratch (256 + 4 * units + 4 * records bytes, a few KiB per work item) exceeds the
+ *     static buffer are refused with GLIDE_ERR_SCRATCH_LIMIT before anything is launched.
+ *   - Calls no cudaMalloc / cudaFree and no allocating library routine.  The first call on each device looks
+ *     the buffer's device address up once (with that device current): make that first call before any stream
+ *     capture begins.
+ *   - All contexts on a device share the one buffer.  It keeps the previous call's contents; the words that
+ *     must start at zero are cleared on `stream` at the start of every call.  Two calls whose kernels overlap
+ *     on the GPU (different streams) race on it: keep calls of this entry point stream-ordered per device. */
+#define GLIDE_NOALLOC_SCRATCH_BYTES (8u << 20)
+int glide_decode_step_noalloc(glide_ctx *ctx, const void *dev_q, const void *dev_k, const void *dev_v, void *dev_out,
+                              void *stream);
 
 /* Free the host context.  Does not touch the workspace. */
 int glide_destroy(glide_ctx *ctx);

@@ -12,6 +12,8 @@
 // the output, stores k,v in the ring slot and clears the ticket.  Nothing ever spins.
 // The last CTA to leave the kernel resets the work counter and advances the position counters,
 // so the step needs no host-side state and no second launch.
+#include <algorithm>
+
 #include "glide_device.cuh"
 
 namespace glide {
@@ -404,6 +406,61 @@ int launch_decode(glide_ctx *ctx, const void *q, const void *k, const void *v, v
     using T = typename decltype(tt)::type;
     constexpr int D = decltype(dd)::value, G = decltype(gg)::value;
     glide_decode_kernel<T, D, G><<<ctx->decode_grid, kDecodeThreads, 0, stream>>>(p);
+    if (cudaGetLastError() != cudaSuccess) return GLIDE_ERR_CUDA;
+    return GLIDE_OK;
+  });
+}
+
+// ---- allocation-free decode variant ---------------------------------------------------------------
+// Split-K scratch of the CUDA-core decode kernel inside the library image instead of the caller's workspace.
+// In host code `g_noalloc_scratch` is only a handle for the symbol, not a device address: the address is
+// looked up once per device with cudaGetSymbolAddress and that pointer is what the kernel receives.
+static __device__ __align__(256) unsigned char g_noalloc_scratch[GLIDE_NOALLOC_SCRATCH_BYTES];
+
+namespace {
+constexpr int kMaxDevices = 64;
+unsigned char *g_noalloc_ptr[kMaxDevices] = {};   // device address of the buffer, per device (nullptr: not looked up yet)
+}  // namespace
+
+int launch_decode_noalloc(glide_ctx *ctx, const void *q, const void *k, const void *v, void *out, cudaStream_t stream) {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) {
+    cudaGetLastError();
+    return GLIDE_ERR_CUDA;
+  }
+  if (dev != ctx->device) return GLIDE_ERR_INVALID_ARG;   // the context lives on another device
+  const size_t units = size_t(ctx->cfg.n_layers) * ctx->cfg.batch * ctx->cfg.n_kv_heads;
+  const size_t tickets_off = 256;
+  const size_t partials_off = tickets_off + (units * sizeof(int32_t) + 255) / 256 * 256;
+  const size_t need = partials_off + ctx->item_part_floats * sizeof(float);
+  if (need > size_t(GLIDE_NOALLOC_SCRATCH_BYTES)) return GLIDE_ERR_SCRATCH_LIMIT;
+  if (!g_noalloc_ptr[dev]) {   // first call on this device: this device is current here
+    void *ptr = nullptr;
+    if (cudaGetSymbolAddress(&ptr, g_noalloc_scratch) != cudaSuccess || !ptr) {
+      cudaGetLastError();
+      return GLIDE_ERR_CUDA;
+    }
+    g_noalloc_ptr[dev] = static_cast<unsigned char *>(ptr);
+  }
+  if (ctx->noalloc_grid == 0) {   // a host-side occupancy query, no allocation
+    int per_sm = 0;
+    if (decode_occupancy(ctx, &per_sm) != GLIDE_OK || per_sm < 1) return GLIDE_ERR_CUDA;
+    ctx->noalloc_grid = std::max(1, std::min(ctx->n_items, ctx->sm_count * per_sm));
+  }
+  unsigned char *scratch = g_noalloc_ptr[dev];
+  // control words and tickets must start at zero; the records are fully written before they are read
+  if (cudaMemsetAsync(scratch, 0, partials_off, stream) != cudaSuccess) {
+    cudaGetLastError();
+    return GLIDE_ERR_CUDA;
+  }
+  DecodeParams p = make_decode_params(ctx, q, k, v, out);
+  p.ctl = reinterpret_cast<Control *>(scratch);
+  p.tickets = reinterpret_cast<int32_t *>(scratch + tickets_off);
+  p.partials = reinterpret_cast<float *>(scratch + partials_off);
+  return dispatch_config(ctx->cfg.io_dtype, ctx->cfg.head_dim, ctx->G, [&](auto tt, auto dd, auto gg) -> int {
+    using T = typename decltype(tt)::type;
+    constexpr int D = decltype(dd)::value, G = decltype(gg)::value;
+    glide_decode_kernel<T, D, G><<<ctx->noalloc_grid, kDecodeThreads, 0, stream>>>(p);
     if (cudaGetLastError() != cudaSuccess) return GLIDE_ERR_CUDA;
     return GLIDE_OK;
   });

@@ -117,6 +117,7 @@ int glide::plan_context(const glide_config *cfg, glide_ctx *ctx, std::vector<Wor
   ctx->off_tickets = off;
   off = align_up(off + sizeof(int32_t) * size_t(L) * units_per_layer, 256);
   ctx->off_partials = off;
+  ctx->item_part_floats = part_floats;
   ctx->stream_seg_capacity = size_t(L) * units_per_layer + size_t(kMaxStreamCtas) * kStreamWarps;
   ctx->stream_rec_capacity = ctx->stream_seg_capacity;
   part_floats = std::max(part_floats, ctx->stream_rec_capacity * size_t(ctx->rec_floats));
@@ -309,6 +310,19 @@ int glide_decode_step(glide_ctx *ctx, const void *q, const void *k, const void *
   return GLIDE_OK;
 }
 
+int glide_decode_step_noalloc(glide_ctx *ctx, const void *q, const void *k, const void *v, void *out, void *stream) {
+  if (!ctx || !q || !k || !v || !out) return GLIDE_ERR_INVALID_ARG;
+  if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out)) return GLIDE_ERR_INVALID_ARG;
+  const int L = ctx->cfg.n_layers;
+  for (int l = 1; l < L; ++l)
+    if (ctx->n_host[l] != ctx->n_host[0]) return GLIDE_ERR_STATE;
+  if (ctx->n_host[0] + 1 > ctx->cfg.max_tokens) return GLIDE_ERR_CAPACITY;
+  int rc = launch_decode_noalloc(ctx, q, k, v, out, as_stream(stream));
+  if (rc) return rc;
+  for (int l = 0; l < L; ++l) ctx->n_host[l] += 1;
+  return GLIDE_OK;
+}
+
 int glide_prefill(glide_ctx *ctx, int32_t layer_begin, int32_t layer_count, int64_t T, const void *q, const void *k,
                   const void *v, void *out, void *stream) {
   if (!ctx || !k || !v || T < 0) return GLIDE_ERR_INVALID_ARG;
@@ -432,6 +446,7 @@ const char *glide_strerror(int code) {
     case GLIDE_ERR_CAPACITY: return "sequence capacity (max_tokens) exceeded";
     case GLIDE_ERR_STATE: return "layers are at different positions";
     case GLIDE_ERR_CUDA: return "CUDA runtime error";
+    case GLIDE_ERR_SCRATCH_LIMIT: return "configuration needs more scratch than the library's built-in static buffer holds";
     default: return "unknown status";
   }
 }

@@ -160,6 +160,8 @@ struct glide_ctx {
   size_t off_ctl = 0, off_ndev = 0, off_layers = 0, off_heads = 0, off_items = 0, off_tickets = 0,
          off_partials = 0, off_tmaps = 0, off_phik = 0, off_state = 0, off_ring = 0, total = 0;
   size_t state_bytes = 0;           // S and z of all layers (contiguous)
+  size_t item_part_floats = 0;      // floats of split-K records the per-item work list needs
+  int noalloc_grid = 0;             // grid of the allocation-free decode variant (0: not sized yet)
 };
 
 namespace glide {
@@ -174,6 +176,7 @@ int stream_decode_supported(const glide_ctx *ctx);
 int stream_decode_setup(glide_ctx *ctx);      // builds the static schedule (host copy) and sizes the launch
 int launch_decode_stream(glide_ctx *ctx, const DecodeParams &p, cudaStream_t stream);
 int launch_decode_mma(glide_ctx *ctx, const DecodeParams &p, cudaStream_t stream);
+int launch_decode_noalloc(glide_ctx *ctx, const void *q, const void *k, const void *v, void *out, cudaStream_t stream);
 int launch_decode(glide_ctx *ctx, const void *q, const void *k, const void *v, void *out, cudaStream_t stream);
 int decode_occupancy(const glide_ctx *ctx, int *blocks_per_sm);
 int launch_prefill(glide_ctx *ctx, int layer_begin, int layer_count, int64_t T, const void *q, const void *k,

@@ -27,6 +27,7 @@ GLIDE_ERR_WORKSPACE_TOO_SMALL = 3
 GLIDE_ERR_CAPACITY = 4
 GLIDE_ERR_STATE = 5
 GLIDE_ERR_CUDA = 6
+GLIDE_ERR_SCRATCH_LIMIT = 7
 
 
 class GlideError(RuntimeError):
@@ -68,6 +69,7 @@ def load_library() -> ctypes.CDLL:
     lib.glide_create.argtypes = [cfgp, vp, ctypes.c_size_t, vp, ctypes.POINTER(vp)]
     lib.glide_prefill.argtypes = [vp, i32, i32, i64, vp, vp, vp, vp, vp]
     lib.glide_decode_step.argtypes = [vp, vp, vp, vp, vp, vp]
+    lib.glide_decode_step_noalloc.argtypes = [vp, vp, vp, vp, vp, vp]
     lib.glide_destroy.argtypes = [vp]
     lib.glide_layer_info.argtypes = [vp, i32, vp, ctypes.POINTER(glide_layer_info_t)]
     lib.glide_export_state.argtypes = [vp, i32, vp, vp, vp, vp, vp]
@@ -78,6 +80,7 @@ def load_library() -> ctypes.CDLL:
     lib.glide_strerror.argtypes = [ctypes.c_int]
     lib.glide_strerror.restype = ctypes.c_char_p
     for name in ("glide_workspace_bytes", "glide_create", "glide_prefill", "glide_decode_step", "glide_destroy",
+                 "glide_decode_step_noalloc",
                  "glide_layer_info", "glide_export_state", "glide_import_state", "glide_reset",
                  "glide_device_status", "glide_decode_launch_info"):
         getattr(lib, name).restype = ctypes.c_int
@@ -173,6 +176,16 @@ class Glide:
         assert q.dtype == k.dtype == v.dtype == out.dtype == self.dtype
         _check(self.lib.glide_decode_step(self._h, _ptr(q), _ptr(k), _ptr(v), _ptr(out), _stream(stream)),
                "glide_decode_step")
+
+    def glide_decode_step_noalloc(self, q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, out: torch.Tensor,
+                                  stream=None) -> None:
+        """glide_decode_step for callers that must not allocate: the step's split-K scratch lives in a static
+        buffer inside the library instead of the workspace (see include/glide.h for the limits)."""
+        assert q.shape == (self.L, self.B, self.H, self.d) and out.shape == q.shape
+        assert k.shape == (self.L, self.B, self.Hkv, self.d) and v.shape == k.shape
+        assert q.dtype == k.dtype == v.dtype == out.dtype == self.dtype
+        _check(self.lib.glide_decode_step_noalloc(self._h, _ptr(q), _ptr(k), _ptr(v), _ptr(out), _stream(stream)),
+               "glide_decode_step_noalloc")
 
     def glide_destroy(self) -> None:
         if getattr(self, "_h", None):
