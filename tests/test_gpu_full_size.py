@@ -1,0 +1,108 @@
+"""Parity at the configurations' full sizes, in the launch configuration bench.py times.
+
+The state is built on the GPU by glide_prefill over the whole synthetic prompt; the oracle rebuilds sampled
+(layer, sequence, KV head) units from the same seeded inputs, one by one, and checks the exported ring rows,
+S, z and counters, a short prefill call with outputs on top of that state, and then decode steps."""
+import numpy as np
+import pytest
+import torch
+
+import bench
+from oracle import glide_oracle as orc
+from paper_2607_24788_b200 import configs as C
+from tests.parity_util import STATE_REL_L2, check_outputs, f32_scale, to_np
+
+pytestmark = pytest.mark.gpu
+
+
+def _unit_inputs(wl, l, b, g, tokens, G):
+    """q [T][G][d], k,v [T][1][d] of one unit as float64 (CPU regeneration of the same seeded values)."""
+    q, k, v = wl.qkv([l], [b], tokens)
+    return (q[0, 0, :, g * G:(g + 1) * G].double().numpy(), k[0, 0, :, g:g + 1].double().numpy(),
+            v[0, 0, :, g:g + 1].double().numpy())
+
+
+def _check(shape, units, extra_prefill=40, n_decode=3):
+    dev = torch.device("cuda", 0)
+    dt = bench.torch_dtype(shape)
+    G = shape.n_q_heads // shape.n_kv_heads
+    d, ctx_len = shape.head_dim, shape.context
+    ctxs, wl = bench.build_states(shape, 1, extra_prefill + n_decode + 8, dev)
+    g = ctxs[0]
+    scale = f32_scale(d)
+    cells = {}
+    for (l, b, kv) in units:
+        cell = orc.Cell(G, 1, d, shape.windows[l], scale)
+        piece = 16384
+        for pos in range(0, ctx_len, piece):
+            _, k, v = _unit_inputs(wl, l, b, kv, range(pos, min(pos + piece, ctx_len)), G)
+            cell.prefill(None, k, v, outputs=False)
+        cells[(l, b, kv)] = cell
+    # state after the full prompt
+    for (l, b, kv), cell in cells.items():
+        info = g.glide_layer_info(l)
+        oi = cell.info()
+        assert (info["n"], info["count"], info["n_evicted"]) == (oi["n"], oi["count"], oi["n_evicted"])
+        rk, rv, S, z = g.glide_export_state(l)
+        ork, orv, oS, oz = cell.export()
+        cap = info["capacity"]
+        tok = cell.slot_tokens()[:cap]
+        valid = np.nonzero(tok >= 0)[0]
+        if len(valid):
+            np.testing.assert_array_equal(to_np(rk[b, kv])[valid], ork[0][valid])
+            np.testing.assert_array_equal(to_np(rv[b, kv])[valid], orv[0][valid])
+        for name, a, r in (("S", to_np(S[b, kv]), oS[0]), ("z", to_np(z[b, kv]), oz[0])):
+            nr = np.linalg.norm(r)
+            if nr:
+                assert np.linalg.norm(a - r) / nr <= STATE_REL_L2, (name, l, b, kv)
+        del rk, rv, S, z
+    # a short prefill call WITH outputs on top of the full-size state
+    pos = ctx_len
+    if extra_prefill:
+        q, k, v = wl.qkv(range(shape.n_layers), range(shape.batch), range(pos, pos + extra_prefill), device=dev)
+        out = torch.full_like(q, float("nan"))
+        g.glide_prefill(q, k, v, out)
+        for (l, b, kv), cell in cells.items():
+            qq, kk, vv = _unit_inputs(wl, l, b, kv, range(pos, pos + extra_prefill), G)
+            ref = cell.prefill(qq, kk, vv)
+            check_outputs(out[l, b, :, kv * G:(kv + 1) * G], ref, dt, f"prefill l{l} b{b} g{kv}")
+        pos += extra_prefill
+        del q, k, v, out
+    # decode steps through the fused kernel
+    for s in range(n_decode):
+        q, k, v = wl.decode_qkv(pos, device=dev)
+        out = torch.full_like(q, float("nan"))
+        g.glide_decode_step(q, k, v, out)
+        assert torch.isfinite(out.float()).all()
+        for (l, b, kv), cell in cells.items():
+            qq, kk, vv = _unit_inputs(wl, l, b, kv, [pos], G)
+            ref = cell.decode(qq[0], kk[0], vv[0])
+            check_outputs(out[l, b, kv * G:(kv + 1) * G], ref, dt, f"decode step {s} l{l} b{b} g{kv}")
+        pos += 1
+    assert g.glide_device_status() == 0
+    for l in range(shape.n_layers):
+        assert g.glide_layer_info(l)["n"] == pos
+
+
+def test_config1_llama_b1_32k_full_size():
+    _check(C.C1, [(0, 0, 0), (3, 0, 7), (5, 0, 2), (11, 0, 5), (12, 0, 1), (23, 0, 6), (24, 0, 0), (31, 0, 7)])
+
+
+def test_config4_mistral_b8_8k_full_size():
+    _check(C.C4, [(0, 0, 0), (1, 7, 3), (9, 3, 6), (17, 5, 1), (26, 2, 4), (31, 7, 7)])
+
+
+def test_config2_llama_b16_16k_full_size():
+    _check(C.C2, [(0, 0, 0), (2, 15, 5), (8, 9, 3), (20, 4, 7), (31, 15, 0)], n_decode=2)
+
+
+def test_config2_uniform_window_control():
+    _check(C.C2_UNIFORM, [(0, 0, 1), (16, 8, 4), (31, 15, 7)], extra_prefill=0, n_decode=2)
+
+
+def test_config3_llama_b4_128k_full_size():
+    _check(C.C3, [(0, 0, 0), (1, 3, 7), (2, 1, 4), (7, 2, 2), (8, 0, 6), (31, 3, 1)], extra_prefill=24, n_decode=2)
+
+
+def test_paper_shaped_blockwise_config_with_linear_only_layers():
+    _check(C.P1, [(0, 0, 3), (9, 0, 0), (10, 0, 7), (21, 0, 2), (22, 0, 5), (31, 0, 1)])
