@@ -47,6 +47,9 @@ constexpr int kHdrSlots = 3;
 #define GLIDE_W_WIN 10
 #define GLIDE_W_UNIT 27
 #endif
+#ifndef GLIDE_W_EDGE
+#define GLIDE_W_EDGE 40
+#endif
 
 // Optional per-warp event trace (debug builds only: -DGLIDE_TRACE).
 #ifdef GLIDE_TRACE
@@ -1026,10 +1029,16 @@ void build_stream_schedule(const glide_ctx *ctx, int n_ranges, std::vector<Strea
   int st_done = 0, win_done = 0;   // progress inside units[ui]
   int64_t cum = 0;
   total_w += int64_t(n_ranges) * kSegWeight;   // a range boundary inside a unit adds a segment
+  // the first and last warp of a CTA usually share a unit with the neighbouring CTA: ticket and merge at the
+  // end of their range cost about kEdgeWeight
+  constexpr int64_t kEdgeWeight = GLIDE_W_EDGE;
+  auto edge_of = [&](int c) -> int64_t { return (c % kWarps == 0 || c % kWarps == kWarps - 1) ? kEdgeWeight : 0; };
+  for (int c = 0; c < n_ranges; ++c) total_w += edge_of(c);
   std::vector<std::vector<size_t>> unit_segs(units.size());
   for (int c = 0; c < n_ranges; ++c) {
     (*range_seg_begin)[c] = int32_t(segs->size());
     const int64_t target = (c + 1 == n_ranges) ? total_w : (total_w * (c + 1) + n_ranges - 1) / n_ranges;
+    cum += edge_of(c);
     bool first = true;
     while (ui < units.size() && cum < target) {
       // opening another segment costs kSegWeight by itself: only worth it if about half of that fits

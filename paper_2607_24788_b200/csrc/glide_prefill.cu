@@ -306,6 +306,7 @@ int launch_prefill(glide_ctx *ctx, int layer_begin, int layer_count, int64_t T, 
   p.Hkv = ctx->cfg.n_kv_heads;
   p.scale_log2 = ctx->scale * kLog2e;
   const int64_t units = int64_t(layer_count) * p.B * p.Hkv;
+  const bool use_mma = prefill_attn_mma_supported(ctx) && ctx->cfg.decode_impl != GLIDE_DECODE_FMA;
   bool any_evicts = false;
   for (int l = layer_begin; l < layer_begin + layer_count; ++l) any_evicts = any_evicts || ctx->layers[l].evicts;
 
@@ -318,7 +319,13 @@ int launch_prefill(glide_ctx *ctx, int layer_begin, int layer_count, int64_t T, 
       const int64_t warps = units * p.C;
       const unsigned warp_blocks = unsigned((warps * 32 + kPrefillThreads - 1) / kPrefillThreads);
       if (any_evicts) prefill_phi_kernel<TT, D><<<warp_blocks, kPrefillThreads, 0, stream>>>(p);
-      if (out) prefill_attn_kernel<TT, D, G><<<warp_blocks, kPrefillThreads, 0, stream>>>(p);
+      if (out) {
+        if (use_mma) {
+          if (launch_prefill_attn_mma(ctx, p, stream) != GLIDE_OK) return GLIDE_ERR_CUDA;
+        } else {
+          prefill_attn_kernel<TT, D, G><<<warp_blocks, kPrefillThreads, 0, stream>>>(p);
+        }
+      }
       if (any_evicts) prefill_state_kernel<TT, D><<<unsigned(units * (D / 16)), kPrefillThreads, 0, stream>>>(p);
       prefill_ring_kernel<TT, D><<<warp_blocks, kPrefillThreads, 0, stream>>>(p);
       if (cudaGetLastError() != cudaSuccess) return GLIDE_ERR_CUDA;
