@@ -242,7 +242,7 @@ def run_glide(args, shape):
     step_bytes = configs.decode_step_bytes(shape, shape.context)
     n_rep = max(1, min(16, math.ceil(8 * L2_BYTES / step_bytes)))
     reps = args.reps
-    extra = math.ceil((max(W, 3) + reps * K + 3 + 3 * K) / n_rep) + 3 * K + 16
+    extra = math.ceil((max(W, 3) + reps * K + 3 + 3 * K) / n_rep) + 3 * K + 16 + 3 * args.prefill_tokens
     ctxs, wl = build_states(shape, n_rep, extra, device)
     L, B, H, Hkv, d = shape.n_layers, shape.batch, shape.n_q_heads, shape.n_kv_heads, shape.head_dim
     dt = torch_dtype(shape)
@@ -363,6 +363,8 @@ def run_glide(args, shape):
             "decode_launch": info,
             "clocks": clocks.summary(),
         }
+        if args.prefill_tokens > 0:
+            line["prefill"] = measure_prefill(ctxs[-1], wl, shape, args.prefill_tokens, device)
         if world == 1 and not args.no_cpu_baseline:
             tok_s, step_s, cores, sample = oracle_decode_rate(shape, 4, 1)
             line["cpu_baseline"] = {"value": tok_s, "unit": "tokens/s", "cores": cores, "kind": "oracle",
@@ -371,6 +373,28 @@ def run_glide(args, shape):
     if dist is not None:
         dist.barrier()
         dist.destroy_process_group()
+
+
+def measure_prefill(ctx, wl, shape, n_tokens, device):
+    """glide_prefill with outputs for n_tokens more tokens on every layer (best of 3, CUDA events)."""
+    L, B, H, d = shape.n_layers, shape.batch, shape.n_q_heads, shape.head_dim
+    n = ctx.glide_layer_info(0)["n"]
+    if n + 3 * n_tokens > ctx.max_tokens:
+        return None
+    q, k, v = wl.qkv(range(L), range(B), range(n, n + n_tokens), device=device)
+    out = torch.empty_like(q)
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    best = None
+    for _ in range(3):
+        ev0.record()
+        ctx.glide_prefill(q, k, v, out)
+        ev1.record()
+        torch.cuda.synchronize()
+        ms = ev0.elapsed_time(ev1)
+        best = ms if best is None else min(best, ms)
+    flops = sum(4.0 * d * H * B * sum(min(w, n + i + 1) for i in range(n_tokens)) for w in shape.windows)
+    return {"tokens": n_tokens, "context_before": n, "ms": best, "tokens_per_s": B * n_tokens / (best * 1e-3),
+            "window_tflops": flops / (best * 1e-3) / 1e12, "note": "glide_prefill with outputs, all layers, chunked"}
 
 
 def main():
@@ -382,6 +406,8 @@ def main():
     ap.add_argument("--workload", default=configs.C1.name, choices=sorted(configs.ALL))
     ap.add_argument("--impl", default="glide", choices=["glide", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--prefill-tokens", type=int, default=1024,
+                    help="tokens appended by glide_prefill WITH outputs after the decode measurement (0: skip)")
     ap.add_argument("--decode-chunk", type=int, default=0, help="window slots per split-K work item (0: library default)")
     ap.add_argument("--state-splits", type=int, default=0, help="row blocks per state update (0: library default)")
     ap.add_argument("--decode-impl", type=int, default=0, help="0 auto, 1 tensor-core/TMA kernel, 2 CUDA-core kernel")
