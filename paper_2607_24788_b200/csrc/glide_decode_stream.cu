@@ -988,133 +988,185 @@ int dispatch_stream(int G, F &&f) {
 
 }  // namespace
 
-// Cuts the tile stream into `n_ranges` equally heavy contiguous ranges, one per warp.  The weights are the
-// measured costs of a state tile, a window tile and of a segment (header, feature maps, finish) relative to
-// each other.
+// Static schedule of the streaming kernel.  Weights are the measured relative costs of a state tile, a window
+// tile and of a segment (header, feature maps, finish).
+//   1. Units (layer x sequence x KV head) are packed whole into CTAs, heaviest first onto the least loaded CTA;
+//      a unit heavier than a CTA's share is first cut into equal pieces.  So almost every unit lives inside one
+//      CTA and is reduced in shared memory; only the oversized ones need global records and a merge.
+//   2. Inside a CTA the list of pieces is cut into 8 contiguous, equally heavy ranges, one per warp.
 void build_stream_schedule(const glide_ctx *ctx, int n_ranges, std::vector<StreamSegment> *segs,
                            std::vector<int32_t> *range_seg_begin, int *max_segs_per_cta, size_t *n_records) {
   constexpr int64_t kSegWeight = GLIDE_W_UNIT, kStateWeight = GLIDE_W_STATE, kWinWeight = GLIDE_W_WIN;
   const int L = ctx->cfg.n_layers, B = ctx->cfg.batch, Hkv = ctx->cfg.n_kv_heads, d = ctx->cfg.head_dim;
+  const int n_ctas = n_ranges / kWarps;
   const int64_t units_per_layer = int64_t(B) * Hkv;
   bool contiguous_heads = true;
   for (int g = 0; g < Hkv; ++g)
     for (int i = 1; i < ctx->G; ++i)
       contiguous_heads = contiguous_heads && ctx->heads_of[size_t(g) * ctx->G + i] == ctx->heads_of[size_t(g) * ctx->G] + i;
-  struct UnitTiles {
-    int layer, unit;
-    int n_state, n_win;
+
+  struct Piece {   // a run of tiles of one unit: state tiles [st0, st0+nst), window tiles [w0, w0+nw)
+    int layer, unit, uidx;
+    int st0, nst, w0, nw;
+    int64_t weight() const { return kStateWeight * nst + kWinWeight * nw + kSegWeight; }
   };
-  std::vector<int> order(L);
-  for (int l = 0; l < L; ++l) order[l] = l;
-  auto layer_weight = [&](int l) -> int64_t {
-    const LayerDev &ld = ctx->layers[l];
-    return (ld.evicts ? 2 * int64_t(d / kTileRows) : 0) + (ld.cap + kTileRows - 1) / kTileRows;
-  };
-  std::stable_sort(order.begin(), order.end(), [&](int x, int y) { return layer_weight(x) > layer_weight(y); });
-  std::vector<UnitTiles> units;
+  std::vector<Piece> pieces;
   int64_t total_w = 0;
-  for (int l : order) {
+  int n_units = 0;
+  for (int l = 0; l < L; ++l) {
     const LayerDev &ld = ctx->layers[l];
     for (int64_t u = 0; u < units_per_layer; ++u) {
-      UnitTiles ut{l, int(int64_t(l) * units_per_layer + u), ld.evicts ? d / kTileRows : 0,
-                   int((ld.cap + kTileRows - 1) / kTileRows)};
-      units.push_back(ut);
-      total_w += kStateWeight * int64_t(ut.n_state) + kWinWeight * int64_t(ut.n_win) + kSegWeight;
+      Piece pc{l, int(int64_t(l) * units_per_layer + u), n_units++, 0, ld.evicts ? d / kTileRows : 0, 0,
+               int((ld.cap + kTileRows - 1) / kTileRows)};
+      pieces.push_back(pc);
+      total_w += pc.weight();
     }
   }
+  const int64_t cta_share = std::max<int64_t>(1, (total_w + n_ctas - 1) / std::max(n_ctas, 1));
+  std::vector<std::vector<size_t>> cta_pieces(size_t(std::max(n_ctas, 1)));
+  std::vector<int64_t> cta_load(size_t(std::max(n_ctas, 1)), 0);
+  // heaviest first
+  std::vector<size_t> order(pieces.size());
+  for (size_t i = 0; i < order.size(); ++i) order[i] = i;
+  std::stable_sort(order.begin(), order.end(), [&](size_t x, size_t y) { return pieces[x].weight() > pieces[y].weight(); });
+  // (a) units heavier than one CTA's share are laid out back to back over the first CTAs and cut exactly at
+  //     the CTA capacity (state tiles first), so those CTAs are full and only these units need global merges
+  size_t oi = 0;
+  {
+    size_t cta = 0;
+    for (; oi < order.size() && pieces[order[oi]].weight() > cta_share; ++oi) {
+      const Piece pc = pieces[order[oi]];
+      int st_done = 0, w_done = 0;
+      while (st_done < pc.nst || w_done < pc.nw) {
+        if (cta + 1 < cta_load.size() && cta_share - cta_load[cta] < kSegWeight + 4 * kWinWeight) ++cta;   // CTA full
+        int64_t room = cta + 1 < cta_load.size() ? cta_share - cta_load[cta] - kSegWeight : INT64_MAX / 4;
+        Piece q = pc;
+        q.st0 = pc.st0 + st_done;
+        q.nst = int(std::min<int64_t>(pc.nst - st_done, std::max<int64_t>(room, 0) / kStateWeight));
+        room -= kStateWeight * int64_t(q.nst);
+        q.w0 = pc.w0 + w_done;
+        q.nw = (st_done + q.nst == pc.nst) ? int(std::min<int64_t>(pc.nw - w_done, std::max<int64_t>(room, 0) / kWinWeight)) : 0;
+        if (q.nst + q.nw == 0) {   // cannot happen with the room check above, but never loop forever
+          q.nst = pc.nst - st_done;
+          q.nw = pc.nw - w_done;
+        }
+        st_done += q.nst;
+        w_done += q.nw;
+        pieces.push_back(q);
+        cta_pieces[cta].push_back(pieces.size() - 1);
+        cta_load[cta] += q.weight();
+      }
+    }
+  }
+  // (b) every other unit goes whole onto the least loaded CTA
+  for (; oi < order.size(); ++oi) {
+    size_t best = 0;
+    for (size_t c = 1; c < cta_load.size(); ++c)
+      if (cta_load[c] < cta_load[best]) best = c;
+    cta_pieces[best].push_back(order[oi]);
+    cta_load[best] += pieces[order[oi]].weight();
+  }
+
   segs->clear();
   range_seg_begin->assign(size_t(n_ranges) + 1, 0);
-  size_t records = 0;
-  size_t ui = 0;
-  int st_done = 0, win_done = 0;   // progress inside units[ui]
-  int64_t cum = 0;
-  total_w += int64_t(n_ranges) * kSegWeight;   // a range boundary inside a unit adds a segment
-  // the first and last warp of a CTA usually share a unit with the neighbouring CTA: ticket and merge at the
-  // end of their range cost about kEdgeWeight
-  constexpr int64_t kEdgeWeight = GLIDE_W_EDGE;
-  auto edge_of = [&](int c) -> int64_t { return (c % kWarps == 0 || c % kWarps == kWarps - 1) ? kEdgeWeight : 0; };
-  for (int c = 0; c < n_ranges; ++c) total_w += edge_of(c);
-  std::vector<std::vector<size_t>> unit_segs(units.size());
-  for (int c = 0; c < n_ranges; ++c) {
-    (*range_seg_begin)[c] = int32_t(segs->size());
-    const int64_t target = (c + 1 == n_ranges) ? total_w : (total_w * (c + 1) + n_ranges - 1) / n_ranges;
-    cum += edge_of(c);
-    bool first = true;
-    while (ui < units.size() && cum < target) {
-      // opening another segment costs kSegWeight by itself: only worth it if about half of that fits
-      if (!first && c + 1 < n_ranges && target - cum < (kSegWeight + kWinWeight) / 2) break;
-      first = false;
-      const UnitTiles &ut = units[ui];
-      const LayerDev &ld = ctx->layers[ut.layer];
-      cum += kSegWeight;   // header, feature maps and finish of a segment
-      int64_t room = std::max<int64_t>(target - cum, 1);
-      StreamSegment sg{};
-      sg.unit = ut.unit;
-      sg.layer = ut.layer;
-      sg.range = c % kWarps;
-      sg.state0 = st_done;
-      sg.n_state = int(std::min<int64_t>(ut.n_state - st_done, (room + kStateWeight - 1) / kStateWeight));
-      room -= kStateWeight * int64_t(sg.n_state);
-      sg.win0 = win_done;
-      sg.n_win = (st_done + sg.n_state == ut.n_state)
-                     ? int(std::min<int64_t>(ut.n_win - win_done, (std::max<int64_t>(room, 0) + kWinWeight - 1) / kWinWeight))
-                     : 0;
-      const int64_t ub = ut.unit - int64_t(ut.layer) * units_per_layer;
-      sg.row_base = int32_t(ub * ld.cap);
-      sg.cap = int32_t(ld.cap);
-      sg.w = int32_t(std::min<int64_t>(ld.w, INT32_MAX));
-      sg.evicts = ld.evicts;
-      sg.S_off256 = int32_t((ld.S + size_t(ub) * d * d * 4) / 256);
-      sg.z_off256 = int32_t((ld.z + size_t(ub) * d * 4) / 256);
-      sg.ringK_off256 = int32_t(ld.ringK / 256);
-      sg.ringV_off256 = int32_t(ld.ringV / 256);
-      sg.g = int32_t(ub % Hkv);
-      {
-        const int64_t b = ub / Hkv;
-        const int64_t row = (int64_t(ut.layer) * B + b) * ctx->cfg.n_q_heads;
-        sg.qrow0 = int32_t(row + (contiguous_heads ? ctx->heads_of[size_t(sg.g) * ctx->G] : 0));
-      }
-      st_done += sg.n_state;
-      win_done += sg.n_win;
-      cum += kStateWeight * int64_t(sg.n_state) + kWinWeight * int64_t(sg.n_win);
-      unit_segs[ui].push_back(segs->size());
-      segs->push_back(sg);
-      if (st_done == ut.n_state && win_done == ut.n_win) {
-        ++ui;
-        st_done = win_done = 0;
+  std::vector<std::vector<size_t>> unit_segs;
+  unit_segs.resize(size_t(n_units));
+  std::vector<int> seg_range;
+  for (int cta = 0; cta < n_ctas; ++cta) {
+    const std::vector<size_t> &list = cta_pieces[size_t(cta)];
+    // the CTA's pieces cut into kWarps contiguous ranges; every range boundary inside a piece adds a segment
+    const int64_t cta_total = cta_load[size_t(cta)] + int64_t(kWarps) * kSegWeight;
+    size_t pi = 0;
+    int st_done = 0, w_done = 0;
+    int64_t cum = 0;
+    for (int wi = 0; wi < kWarps; ++wi) {
+      const int c = cta * kWarps + wi;
+      (*range_seg_begin)[size_t(c)] = int32_t(segs->size());
+      // an equal share of what is left, so that a range that stops short does not load up the last warp
+      const int64_t target = (wi + 1 == kWarps) ? INT64_MAX : cum + (std::max<int64_t>(cta_total - cum, 0) + (kWarps - wi) - 1) / (kWarps - wi);
+      bool first = true;
+      while (pi < list.size() && cum < target) {
+        const Piece &pc = pieces[list[pi]];
+        const LayerDev &ld = ctx->layers[pc.layer];
+        const int64_t rem = kStateWeight * (pc.nst - st_done) + kWinWeight * (pc.nw - w_done);
+        int64_t room = target == INT64_MAX ? INT64_MAX / 4 : target - cum - kSegWeight;
+        StreamSegment sg{};
+        if (rem <= room + cta_total / (kWarps * 8)) {   // finishing the piece here overshoots by little: keep it whole
+          sg.n_state = pc.nst - st_done;
+          sg.n_win = pc.nw - w_done;
+        } else {
+          if (!first && room < 2 * kWinWeight) break;   // not worth opening a segment for a tile or two
+          room = std::max<int64_t>(room, 1);
+          sg.n_state = int(std::min<int64_t>(pc.nst - st_done, (room + kStateWeight - 1) / kStateWeight));
+          room -= kStateWeight * int64_t(sg.n_state);
+          sg.n_win = (st_done + sg.n_state == pc.nst)
+                         ? int(std::min<int64_t>(pc.nw - w_done, (std::max<int64_t>(room, 0) + kWinWeight - 1) / kWinWeight))
+                         : 0;
+        }
+        first = false;
+        sg.unit = pc.unit;
+        sg.layer = pc.layer;
+        sg.range = wi;
+        sg.state0 = pc.st0 + st_done;
+        sg.win0 = pc.w0 + w_done;
+        const int64_t ub = pc.unit - int64_t(pc.layer) * units_per_layer;
+        sg.row_base = int32_t(ub * ld.cap);
+        sg.cap = int32_t(ld.cap);
+        sg.w = int32_t(std::min<int64_t>(ld.w, INT32_MAX));
+        sg.evicts = ld.evicts;
+        sg.S_off256 = int32_t((ld.S + size_t(ub) * d * d * 4) / 256);
+        sg.z_off256 = int32_t((ld.z + size_t(ub) * d * 4) / 256);
+        sg.ringK_off256 = int32_t(ld.ringK / 256);
+        sg.ringV_off256 = int32_t(ld.ringV / 256);
+        sg.g = int32_t(ub % Hkv);
+        {
+          const int64_t b = ub / Hkv;
+          const int64_t row = (int64_t(pc.layer) * B + b) * ctx->cfg.n_q_heads;
+          sg.qrow0 = int32_t(row + (contiguous_heads ? ctx->heads_of[size_t(sg.g) * ctx->G] : 0));
+        }
+        st_done += sg.n_state;
+        w_done += sg.n_win;
+        cum += kSegWeight + kStateWeight * int64_t(sg.n_state) + kWinWeight * int64_t(sg.n_win);
+        unit_segs[size_t(pc.uidx)].push_back(segs->size());
+        seg_range.push_back(c);
+        segs->push_back(sg);
+        if (st_done == pc.nst && w_done == pc.nw) {
+          ++pi;
+          st_done = w_done = 0;
+        }
       }
     }
   }
-  (*range_seg_begin)[n_ranges] = int32_t(segs->size());
+  for (int c = n_ctas * kWarps; c <= n_ranges; ++c) (*range_seg_begin)[size_t(c)] = int32_t(segs->size());
+  (*range_seg_begin)[size_t(n_ranges)] = int32_t(segs->size());
   *max_segs_per_cta = 0;
   for (int c = 0; c + kWarps <= n_ranges; c += kWarps)
-    *max_segs_per_cta = std::max<int>(*max_segs_per_cta, (*range_seg_begin)[c + kWarps] - (*range_seg_begin)[c]);
+    *max_segs_per_cta = std::max<int>(*max_segs_per_cta, (*range_seg_begin)[size_t(c + kWarps)] - (*range_seg_begin)[size_t(c)]);
+
   // Warps of one CTA that share a unit reduce their records in shared memory first (a "group"); only one
   // record per group goes to global scratch, and a unit that lies inside one group never touches it.
+  size_t records = 0;
   const int pool_slots = kStreamPoolBytes / (ctx->rec_floats * 4);
-  std::vector<int> cta_slots(size_t(n_ranges / kWarps) + 1, 0), cta_groups(size_t(n_ranges / kWarps) + 1, 0);
-  std::vector<int> seg_range(segs->size(), 0);
-  for (int c = 0; c < n_ranges; ++c)
-    for (int i = (*range_seg_begin)[c]; i < (*range_seg_begin)[c + 1]; ++i) seg_range[i] = c;
-  for (size_t u = 0; u < units.size(); ++u) {
-    const std::vector<size_t> &list = unit_segs[u];
-    // split the unit's segments (ordered by range) into groups of one CTA each
+  std::vector<int> cta_slots(size_t(n_ctas) + 1, 0), cta_groups(size_t(n_ctas) + 1, 0);
+  for (size_t u = 0; u < unit_segs.size(); ++u) {
+    std::vector<size_t> &list = unit_segs[u];
+    std::stable_sort(list.begin(), list.end(), [&](size_t x, size_t y) { return seg_range[x] < seg_range[y]; });
     std::vector<std::pair<size_t, size_t>> groups;   // [first, last) into list
     for (size_t i = 0; i < list.size();) {
       const int cta = seg_range[list[i]] / kWarps;
       size_t j = i + 1;
       while (j < list.size() && seg_range[list[j]] / kWarps == cta) ++j;
       const int need = int(j - i);
-      if (need >= 2 && cta_slots[cta] + need <= pool_slots && cta_groups[cta] < kStreamMaxGroups) {
+      if (need >= 2 && cta_slots[size_t(cta)] + need <= pool_slots && cta_groups[size_t(cta)] < kStreamMaxGroups) {
         for (size_t k = i; k < j; ++k) {
           StreamSegment &sg = (*segs)[list[k]];
           sg.grp_size = need;
-          sg.grp_slot0 = cta_slots[cta];
+          sg.grp_slot0 = cta_slots[size_t(cta)];
           sg.grp_idx = int(k - i);
-          sg.grp_ctr = cta_groups[cta];
+          sg.grp_ctr = cta_groups[size_t(cta)];
         }
-        cta_slots[cta] += need;
-        cta_groups[cta] += 1;
+        cta_slots[size_t(cta)] += need;
+        cta_groups[size_t(cta)] += 1;
         groups.emplace_back(i, j);
       } else {   // single warp, or no room left in the CTA's pool: every segment is its own group
         for (size_t k = i; k < j; ++k) {
