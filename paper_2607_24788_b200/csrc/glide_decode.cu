@@ -382,6 +382,7 @@ DecodeParams make_decode_params(const glide_ctx *ctx, const void *q, const void 
   p.Hkv = ctx->cfg.n_kv_heads;
   p.rec_floats = ctx->rec_floats;
   p.scale_log2 = ctx->scale * kLog2e;
+  p.t_host = ctx->n_host[0];
   return p;
 }
 

@@ -47,6 +47,9 @@ constexpr int kHdrSlots = 3;
 #define GLIDE_W_WIN 10
 #define GLIDE_W_UNIT 27
 #endif
+#ifndef GLIDE_STREAM_FILL
+#define GLIDE_STREAM_FILL 100
+#endif
 #ifndef GLIDE_W_EDGE
 #define GLIDE_W_EDGE 40
 #endif
@@ -299,7 +302,9 @@ glide_decode_stream_kernel(const DecodeParams p, const StreamParams sp) {
   }
   __syncthreads();   // segment table and barriers ready; the warps are on their own from here
   asm volatile("griddepcontrol.wait;" ::: "memory");   // the preceding kernel has completed and its writes are visible
-  const int64_t t = p.n_dev[0];   // every layer is at the same position (checked by the host)
+  // every layer is at the same position (checked by the host); the host's copy of the counter comes with the
+  // launch, which saves a dependent global load at the head of every warp's critical path
+  const int64_t t = p.t_host;
   // this warp's segments: the run of the CTA's list that carries its index
   int seg_lo = 0;
   while (seg_lo < cta_nseg && sm_segs[seg_lo].range < warp) ++seg_lo;
@@ -1033,13 +1038,15 @@ void build_stream_schedule(const glide_ctx *ctx, int n_ranges, std::vector<Strea
   //     the CTA capacity (state tiles first), so those CTAs are full and only these units need global merges
   size_t oi = 0;
   {
+    // these CTAs end with a ticket + merge chain of a few microseconds: they get less than a full share
+    const int64_t cta_cap = cta_share * GLIDE_STREAM_FILL / 100;
     size_t cta = 0;
     for (; oi < order.size() && pieces[order[oi]].weight() > cta_share; ++oi) {
       const Piece pc = pieces[order[oi]];
       int st_done = 0, w_done = 0;
       while (st_done < pc.nst || w_done < pc.nw) {
-        if (cta + 1 < cta_load.size() && cta_share - cta_load[cta] < kSegWeight + 4 * kWinWeight) ++cta;   // CTA full
-        int64_t room = cta + 1 < cta_load.size() ? cta_share - cta_load[cta] - kSegWeight : INT64_MAX / 4;
+        if (cta + 1 < cta_load.size() && cta_cap - cta_load[cta] < kSegWeight + 4 * kWinWeight) ++cta;   // CTA full
+        int64_t room = cta + 1 < cta_load.size() ? cta_cap - cta_load[cta] - kSegWeight : INT64_MAX / 4;
         Piece q = pc;
         q.st0 = pc.st0 + st_done;
         q.nst = int(std::min<int64_t>(pc.nst - st_done, std::max<int64_t>(room, 0) / kStateWeight));

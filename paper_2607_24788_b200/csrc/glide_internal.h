@@ -67,6 +67,7 @@ struct DecodeParams {
   int32_t L, B, H, Hkv;
   int32_t rec_floats;        // floats per partial record: G * (d + 2) rounded up to 4
   float scale_log2;          // softmax_scale * log2(e)
+  int64_t t_host;            // position of the token being decoded as the host tracks it (= device counter)
 };
 
 constexpr int kMaxStreamCtas = 192;           // CTAs (one per SM) the streaming decode kernel's schedule can address
