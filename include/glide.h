@@ -66,6 +66,10 @@ typedef enum { GLIDE_MERGE_SHARED = 0 } glide_merge;
  * force one kernel (GLIDE_ERR_UNSUPPORTED if it does not apply). */
 typedef enum { GLIDE_DECODE_AUTO = 0, GLIDE_DECODE_MMA = 1, GLIDE_DECODE_FMA = 2, GLIDE_DECODE_STREAM = 3 } glide_decode_impl;
 
+/* Kernel that computes the prefill outputs (bf16 I/O).  AUTO picks the fastest that applies; TCGEN05 needs
+ * head_dim 128; for fp32 I/O only the CUDA-core kernel exists.  State, ring and counters do not depend on it. */
+typedef enum { GLIDE_PREFILL_AUTO = 0, GLIDE_PREFILL_MMA_SYNC = 1, GLIDE_PREFILL_TCGEN05 = 2, GLIDE_PREFILL_FMA = 3 } glide_prefill_impl;
+
 typedef struct {
   int32_t n_layers;        /* L >= 1 */
   int32_t batch;           /* B >= 1 independent sequences of equal length */
@@ -85,6 +89,7 @@ typedef struct {
   int32_t decode_chunk;    /* window slots per split-K work item of the decode kernel; 0 selects automatically */
   int32_t decode_state_splits; /* row blocks the S update/readout of one KV head is split into; 0 selects automatically */
   int32_t decode_impl;     /* glide_decode_impl */
+  int32_t prefill_impl;    /* glide_prefill_impl */
 } glide_config;
 
 typedef struct {

@@ -26,6 +26,11 @@ int validate_config(const glide_config *c) {
   if (c->prefill_chunk < 0 || c->decode_chunk < 0 || c->decode_state_splits < 0) return GLIDE_ERR_INVALID_ARG;
   if (c->prefill_chunk % 16 != 0 || c->prefill_chunk > 1024) return GLIDE_ERR_INVALID_ARG;
   if (c->decode_impl < GLIDE_DECODE_AUTO || c->decode_impl > GLIDE_DECODE_STREAM) return GLIDE_ERR_INVALID_ARG;
+  if (c->prefill_impl < GLIDE_PREFILL_AUTO || c->prefill_impl > GLIDE_PREFILL_FMA) return GLIDE_ERR_INVALID_ARG;
+  if ((c->prefill_impl == GLIDE_PREFILL_MMA_SYNC || c->prefill_impl == GLIDE_PREFILL_TCGEN05) && c->io_dtype != GLIDE_BF16)
+    return GLIDE_ERR_UNSUPPORTED;
+  if ((c->prefill_impl == GLIDE_PREFILL_MMA_SYNC || c->prefill_impl == GLIDE_PREFILL_TCGEN05) && c->head_dim != 128)
+    return GLIDE_ERR_UNSUPPORTED;
   if ((c->decode_impl == GLIDE_DECODE_MMA || c->decode_impl == GLIDE_DECODE_STREAM) && c->io_dtype != GLIDE_BF16)
     return GLIDE_ERR_UNSUPPORTED;
   for (int l = 0; l < c->n_layers; ++l)

@@ -306,7 +306,11 @@ int launch_prefill(glide_ctx *ctx, int layer_begin, int layer_count, int64_t T, 
   p.Hkv = ctx->cfg.n_kv_heads;
   p.scale_log2 = ctx->scale * kLog2e;
   const int64_t units = int64_t(layer_count) * p.B * p.Hkv;
-  const bool use_mma = prefill_attn_mma_supported(ctx) && ctx->cfg.decode_impl != GLIDE_DECODE_FMA;
+  int impl = ctx->cfg.prefill_impl;
+  if (impl == GLIDE_PREFILL_AUTO)
+    impl = (prefill_attn_mma_supported(ctx) && ctx->cfg.decode_impl != GLIDE_DECODE_FMA) ? GLIDE_PREFILL_MMA_SYNC : GLIDE_PREFILL_FMA;
+  const bool use_tc = impl == GLIDE_PREFILL_TCGEN05 && prefill_attn_tc_supported(ctx);
+  const bool use_mma = impl == GLIDE_PREFILL_MMA_SYNC && prefill_attn_mma_supported(ctx);
   bool any_evicts = false;
   for (int l = layer_begin; l < layer_begin + layer_count; ++l) any_evicts = any_evicts || ctx->layers[l].evicts;
 
@@ -320,7 +324,9 @@ int launch_prefill(glide_ctx *ctx, int layer_begin, int layer_count, int64_t T, 
       const unsigned warp_blocks = unsigned((warps * 32 + kPrefillThreads - 1) / kPrefillThreads);
       if (any_evicts) prefill_phi_kernel<TT, D><<<warp_blocks, kPrefillThreads, 0, stream>>>(p);
       if (out) {
-        if (use_mma) {
+        if (use_tc) {
+          if (launch_prefill_attn_tc(ctx, p, stream) != GLIDE_OK) return GLIDE_ERR_CUDA;
+        } else if (use_mma) {
           if (launch_prefill_attn_mma(ctx, p, stream) != GLIDE_OK) return GLIDE_ERR_CUDA;
         } else {
           prefill_attn_kernel<TT, D, G><<<warp_blocks, kPrefillThreads, 0, stream>>>(p);

@@ -44,6 +44,7 @@ class glide_config(ctypes.Structure):
         ("windows", ctypes.POINTER(ctypes.c_int64)), ("q_to_kv", ctypes.POINTER(ctypes.c_int32)),
         ("max_tokens", ctypes.c_int64), ("softmax_scale", ctypes.c_float), ("prefill_chunk", ctypes.c_int32),
         ("decode_chunk", ctypes.c_int32), ("decode_state_splits", ctypes.c_int32), ("decode_impl", ctypes.c_int32),
+        ("prefill_impl", ctypes.c_int32),
     ]
 
 
@@ -112,7 +113,7 @@ def _stream(stream: Optional[torch.cuda.Stream]) -> Optional[int]:
 def make_config(windows: Sequence[int], batch: int, n_q_heads: int, n_kv_heads: int, head_dim: int, max_tokens: int,
                 dtype: torch.dtype = torch.bfloat16, q_to_kv: Optional[Sequence[int]] = None,
                 softmax_scale: float = 0.0, prefill_chunk: int = 0, decode_chunk: int = 0,
-                decode_state_splits: int = 0, decode_impl: int = 0):
+                decode_state_splits: int = 0, decode_impl: int = 0, prefill_impl: int = 0):
     """Returns (glide_config, keepalive) -- keepalive holds the host arrays the struct points to."""
     win = (ctypes.c_int64 * len(windows))(*[int(w) for w in windows])
     qmap = (ctypes.c_int32 * len(q_to_kv))(*[int(x) for x in q_to_kv]) if q_to_kv is not None else None
@@ -126,6 +127,7 @@ def make_config(windows: Sequence[int], batch: int, n_q_heads: int, n_kv_heads: 
     cfg.softmax_scale = float(softmax_scale)
     cfg.prefill_chunk, cfg.decode_chunk, cfg.decode_state_splits = int(prefill_chunk), int(decode_chunk), int(decode_state_splits)
     cfg.decode_impl = int(decode_impl)
+    cfg.prefill_impl = int(prefill_impl)
     return cfg, (win, qmap)
 
 

@@ -118,3 +118,13 @@ def test_errors_and_capacity():
     assert g.glide_layer_info(0)["n"] == 8
     g.glide_reset()
     assert g.glide_layer_info(1) == dict(window=4, capacity=4, n=0, count=0, head_slot=0, n_evicted=0)
+
+
+@pytest.mark.parametrize("impl", [1, 2, 3])   # prefill outputs: mma.sync, tcgen05 + TMEM, CUDA cores
+@pytest.mark.parametrize("G", [1, 4])
+@pytest.mark.parametrize("chunk", [96, 256])
+def test_bf16_prefill_tensor_core_multi_call(impl, G, chunk):
+    # several calls, so window tiles mix ring rows with the call's rows; windows below, at and above the
+    # 128-key tile, one never-evicting layer, one purely linear layer; ragged last query tile
+    run_case([0, 100, 128, 300, 1 << 20], 2, 2 * G, 2, 128, BF16, [130, 257, 61], 4, amp=128 ** -0.5 * 4,
+             seed=chunk + G, prefill_chunk=chunk, prefill_impl=impl)
