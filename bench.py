@@ -115,7 +115,7 @@ def value_scale(shape):
 # ---------------------------------------------------------------------------------------------
 # CPU oracle leg (cpu_baseline and --impl reference)
 # ---------------------------------------------------------------------------------------------
-def oracle_decode_rate(shape, steps: int, warmup: int):
+def oracle_decode_rate(shape, steps: int, warmup: int, single_steps: int = 0):
     """Times the oracle's decode step on the host cores on a bounded sample of the workload: one layer of
     every distinct window size, sequence 0, state built by the oracle's own prefill of the full prompt.
     Per-layer-class times are scaled by the number of layers and sequences of each class."""
@@ -131,6 +131,7 @@ def oracle_decode_rate(shape, steps: int, warmup: int):
     per_class_s = {}
     threads = orc.max_threads()
     used = 1
+    single_s = {}
     for w, layers in classes.items():
         l = layers[0]
         stack = orc.Stack([w], 1, shape.n_q_heads, shape.n_kv_heads, shape.head_dim, scale)
@@ -150,6 +151,17 @@ def oracle_decode_rate(shape, steps: int, warmup: int):
             if s >= warmup:
                 times.append(t1 - t0)
         per_class_s[w] = statistics.median(times)
+        times = []
+        for s in range(single_steps):   # the same stack, one thread
+            q, k, v = wl.qkv([l], [0], [shape.context + warmup + steps + s])
+            q, k, v = (x[:, :, 0].double().numpy() for x in (q, k, v))
+            t0 = time.perf_counter()
+            stack.decode(q, k, v, threads=1)
+            times.append(time.perf_counter() - t0)
+        if times:
+            single_s[w] = statistics.median(times)
+    if single_steps:
+        oracle_decode_rate.single_thread_step_s = sum(single_s[w] * len(layers) for w, layers in classes.items()) * shape.batch
     step_s = sum(per_class_s[w] * len(layers) for w, layers in classes.items()) * shape.batch
     sample = (f"layers {sorted(v[0] for v in classes.values())} (one per distinct window), sequence 0, "
               f"{steps} decode steps each after the oracle's own {shape.context}-token prefill; "
@@ -242,7 +254,7 @@ def run_glide(args, shape):
     step_bytes = configs.decode_step_bytes(shape, shape.context)
     n_rep = max(1, min(16, math.ceil(8 * L2_BYTES / step_bytes)))
     reps = args.reps
-    extra = math.ceil((max(W, 3) + reps * K + 3 + 3 * K) / n_rep) + 3 * K + 16 + 3 * args.prefill_tokens
+    extra = math.ceil((max(W, 3) + (reps + 1) * K + 3 + 3 * K) / n_rep) + 6 * K + 32 + 3 * args.prefill_tokens
     ctxs, wl = build_states(shape, n_rep, extra, device)
     L, B, H, Hkv, d = shape.n_layers, shape.batch, shape.n_q_heads, shape.n_kv_heads, shape.head_dim
     dt = torch_dtype(shape)
@@ -292,6 +304,18 @@ def run_glide(args, shape):
             times_ms.append(ev0.elapsed_time(ev1))
     t_ms = statistics.median(times_ms)
 
+    # every step on its own pair of events (rotating state copies as above): the spread of the step latency;
+    # an event between two launches keeps the next launch from overlapping the previous one's tail
+    lat_us = []
+    evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(K)]
+    barrier()
+    for i in range(K):
+        evs[i][0].record()
+        one_step(dev_in[i % n_in])
+        evs[i][1].record()
+    barrier()
+    lat_us = sorted(a.elapsed_time(b) * 1e3 for a, b in evs)
+
     # same context every step: window and state of the previous step may still sit in L2
     hot_ms = []
     for _ in range(3):
@@ -331,6 +355,10 @@ def run_glide(args, shape):
         e2e_ms.append(ev0.elapsed_time(ev1))
     e2e_t = statistics.median(e2e_ms)
 
+    per_layer = None
+    if world == 1 and step_bytes <= (8 << 30):
+        per_layer = measure_per_layer_launch(ctxs[0], shape, views(dev_in[0]), outs[0], K, device)
+
     t_ms, hot_ms, e2e_t = max_over_ranks([t_ms, hot_ms, e2e_t], dist, device)
 
     if rank == 0:
@@ -354,6 +382,9 @@ def run_glide(args, shape):
                          "kernel": "glide_decode_kernel", "algorithmic_bytes_per_launch": step_bytes,
                          "frac_of_nominal_8TBps": achieved / 8000.0},
             "per_step_attention_latency_us": launch_s * 1e6,
+            "step_latency_us": {"median": lat_us[len(lat_us) // 2], "p10": lat_us[len(lat_us) // 10],
+                                "p90": lat_us[(len(lat_us) * 9) // 10], "steps": len(lat_us),
+                                "note": "each step between its own two events (no overlap with the neighbours), rank 0"},
             "hot_l2": {"tokens_per_s": world * B * K / (hot_ms * 1e-3), "us_per_step": hot_ms * 1e3 / K,
                        "note": "same sequence state every step (L2 may hold part of it)"},
             "e2e": {"value": world * B * e2e_steps / (e2e_t * 1e-3), "unit": "tokens/s",
@@ -363,16 +394,95 @@ def run_glide(args, shape):
             "decode_launch": info,
             "clocks": clocks.summary(),
         }
+        if per_layer is not None:
+            per_layer["vs_one_launch_hot_l2"] = per_layer["us_per_step"] / (hot_ms * 1e3 / K)
+            line["per_layer_launch"] = per_layer
         if args.prefill_tokens > 0:
             line["prefill"] = measure_prefill(ctxs[-1], wl, shape, args.prefill_tokens, device)
         if world == 1 and not args.no_cpu_baseline:
-            tok_s, step_s, cores, sample = oracle_decode_rate(shape, 4, 1)
+            tok_s, step_s, cores, sample = oracle_decode_rate(shape, 4, 1, single_steps=2)
             line["cpu_baseline"] = {"value": tok_s, "unit": "tokens/s", "cores": cores, "kind": "oracle",
                                     "sample": sample, "ms_per_step": step_s * 1e3}
+            step1 = oracle_decode_rate.single_thread_step_s
+            line["cpu_baseline"]["single_thread"] = {"value": B / step1, "unit": "tokens/s", "cores": 1,
+                                                     "ms_per_step": step1 * 1e3}
         print(json.dumps(line))
     if dist is not None:
         dist.barrier()
         dist.destroy_process_group()
+
+
+def measure_per_layer_launch(g0, shape, qkv, out, steps, device):
+    """The same decode step issued as one launch per layer (L one-layer contexts holding copies of the layers'
+    state) instead of one launch for the whole stack: what the per-launch overhead costs when the windows are
+    small.  Same sequence state every step, so it compares with the one-launch `hot_l2` figure."""
+    from paper_2607_24788_b200 import glide
+    L = shape.n_layers
+    dt = torch_dtype(shape)
+    n = g0.glide_layer_info(0)["n"]
+    layer_ctx = []
+    for l in range(L):
+        g = glide.Glide([shape.windows[l]], shape.batch, shape.n_q_heads, shape.n_kv_heads, shape.head_dim,
+                        g0.max_tokens, dtype=dt, device=device, **KERNEL_KNOBS)   # same capacity: same ring size
+        rk, rv, S, z = g0.glide_export_state(l)
+        cap = g.capacity(0)
+        g.glide_import_state(0, n, rk if cap else None, rv if cap else None, S, z)
+        layer_ctx.append(g)
+    torch.cuda.synchronize()
+    q, k, v = qkv
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+
+    # the C entry point with pointers resolved once: the binding's per-call argument checks (tens of microseconds)
+    # would otherwise be what is measured
+    import ctypes
+    vp = ctypes.c_void_p
+    sptr = vp(torch.cuda.current_stream().cuda_stream or None)
+    calls = [(g.lib.glide_decode_step, g._h, vp(q[l].data_ptr()), vp(k[l].data_ptr()), vp(v[l].data_ptr()),
+              vp(out[l].data_ptr())) for l, g in enumerate(layer_ctx)]
+
+    def launch(l):
+        fn, h, a, b, c, o = calls[l]
+        if fn(h, a, b, c, o, sptr) != 0:
+            raise RuntimeError("glide_decode_step failed in per-layer mode")
+
+    def step():
+        for l in range(L):
+            launch(l)
+
+    for _ in range(3):
+        step()
+    torch.cuda.synchronize()
+    res = []
+    host_us = []
+    for _ in range(3):
+        ev0.record()
+        h0 = time.perf_counter()
+        for _ in range(steps):
+            step()
+        h1 = time.perf_counter()
+        ev1.record()
+        torch.cuda.synchronize()
+        res.append(ev0.elapsed_time(ev1) * 1e3 / steps)
+        host_us.append((h1 - h0) * 1e6 / steps)
+    # every layer's launch alone between two events (what a model that runs other kernels between the layers'
+    # attention calls sees on the GPU), summed over the layers
+    isolated = 0.0
+    for l in range(L):
+        one = []
+        for _ in range(12):
+            ev0.record()
+            launch(l)
+            ev1.record()
+            torch.cuda.synchronize()
+            one.append(ev0.elapsed_time(ev1) * 1e3)
+        isolated += statistics.median(one)
+    del layer_ctx
+    return {"us_per_step": statistics.median(res), "launches_per_step": L,
+            "host_issue_us_per_step": statistics.median(host_us),
+            "sum_of_isolated_launches_us": isolated,
+            "note": "one glide_decode_step per layer on one-layer contexts, issued back to back; when "
+                    "host_issue_us_per_step is about us_per_step the figure is bound by the host issuing launches; "
+                    "sum_of_isolated_launches_us adds up each layer's launch timed alone between two events"}
 
 
 def measure_prefill(ctx, wl, shape, n_tokens, device):
@@ -410,11 +520,13 @@ def main():
                     help="tokens appended by glide_prefill WITH outputs after the decode measurement (0: skip)")
     ap.add_argument("--decode-chunk", type=int, default=0, help="window slots per split-K work item (0: library default)")
     ap.add_argument("--state-splits", type=int, default=0, help="row blocks per state update (0: library default)")
-    ap.add_argument("--decode-impl", type=int, default=0, help="0 auto, 1 tensor-core/TMA kernel, 2 CUDA-core kernel")
+    ap.add_argument("--decode-impl", type=int, default=0,
+                    help="0 auto, 1 per-item tensor-core/TMA kernel, 2 CUDA-core kernel, 3 streaming tensor-core/TMA kernel")
+    ap.add_argument("--prefill-impl", type=int, default=0, help="0 auto, 1 mma.sync, 2 tcgen05 + TMEM, 3 CUDA cores")
     args = ap.parse_args()
     shape = configs.ALL[args.workload]
     KERNEL_KNOBS.update(decode_chunk=args.decode_chunk, decode_state_splits=args.state_splits,
-                        decode_impl=args.decode_impl)
+                        decode_impl=args.decode_impl, prefill_impl=args.prefill_impl)
     if args.impl == "reference":
         run_reference(args, shape)
     else:

@@ -50,6 +50,9 @@ constexpr int kHdrSlots = 3;
 #ifndef GLIDE_STREAM_FILL
 #define GLIDE_STREAM_FILL 100
 #endif
+#ifndef GLIDE_W_MIN_CTA
+#define GLIDE_W_MIN_CTA 128   // least weight worth a CTA of its own (about ten tiles)
+#endif
 #ifndef GLIDE_W_EDGE
 #define GLIDE_W_EDGE 40
 #endif
@@ -305,6 +308,10 @@ glide_decode_stream_kernel(const DecodeParams p, const StreamParams sp) {
   // every layer is at the same position (checked by the host); the host's copy of the counter comes with the
   // launch, which saves a dependent global load at the head of every warp's critical path
   const int64_t t = p.t_host;
+  // the device counters are not read by this kernel; one thread moves them on (no grid-wide completion count,
+  // which would put an atomic round trip at the end of every CTA)
+  if (blockIdx.x == 0)
+    for (int l = tid; l < p.L; l += kThreads) p.n_dev[l] = t + 1;
   // this warp's segments: the run of the CTA's list that carries its index
   int seg_lo = 0;
   while (seg_lo < cta_nseg && sm_segs[seg_lo].range < warp) ++seg_lo;
@@ -960,16 +967,6 @@ glide_decode_stream_kernel(const DecodeParams p, const StreamParams sp) {
   if (lane == 0) bulk_wait0();   // this warp's state stores have landed
   GLIDE_TRACE_EVENT(9);
 
-  __syncthreads();
-  if (tid == 0) {
-    __threadfence();
-    if (atomicAdd(&p.ctl->done_counter, 1) == int(gridDim.x) - 1) {
-      p.ctl->work_counter = 0;
-      p.ctl->done_counter = 0;
-      for (int l = 0; l < p.L; ++l) p.n_dev[l] += 1;
-      __threadfence();
-    }
-  }
 }
 
 template <int G, int STAGES>
@@ -1027,44 +1024,67 @@ void build_stream_schedule(const glide_ctx *ctx, int n_ranges, std::vector<Strea
       total_w += pc.weight();
     }
   }
-  const int64_t cta_share = std::max<int64_t>(1, (total_w + n_ctas - 1) / std::max(n_ctas, 1));
+  // Small problems (one layer, a short window, a small batch) do not have work for every CTA: below about ten
+  // tiles per CTA the per-segment overheads and the number of records per merge grow faster than the streaming
+  // time shrinks.  Units that are small themselves are then kept whole.
+  constexpr int64_t kMinCtaWeight = GLIDE_W_MIN_CTA;
+  int64_t max_unit_w = 0;
+  for (const Piece &pc : pieces) max_unit_w = std::max(max_unit_w, pc.weight());
+  const int n_used = int(std::max<int64_t>(1, std::min<int64_t>(n_ctas, total_w / kMinCtaWeight)));
+  int64_t cta_share = std::max<int64_t>(1, (total_w + n_used - 1) / n_used);
+  if (n_used < n_ctas && max_unit_w <= 2 * kMinCtaWeight) cta_share = std::max(cta_share, max_unit_w);
   std::vector<std::vector<size_t>> cta_pieces(size_t(std::max(n_ctas, 1)));
   std::vector<int64_t> cta_load(size_t(std::max(n_ctas, 1)), 0);
   // heaviest first
   std::vector<size_t> order(pieces.size());
   for (size_t i = 0; i < order.size(); ++i) order[i] = i;
   std::stable_sort(order.begin(), order.end(), [&](size_t x, size_t y) { return pieces[x].weight() > pieces[y].weight(); });
-  // (a) units heavier than one CTA's share are laid out back to back over the first CTAs and cut exactly at
-  //     the CTA capacity (state tiles first), so those CTAs are full and only these units need global merges
+  // (a) units heavier than one CTA's share are laid out back to back over the first CTAs (state tiles first) and
+  //     cut at cumulative targets, so that what one CTA leaves unused goes to the next one instead of piling up
+  //     on the last; only these units need global records and a merge
   size_t oi = 0;
   {
-    // these CTAs end with a ticket + merge chain of a few microseconds: they get less than a full share
-    const int64_t cta_cap = cta_share * GLIDE_STREAM_FILL / 100;
-    size_t cta = 0;
-    for (; oi < order.size() && pieces[order[oi]].weight() > cta_share; ++oi) {
+    int64_t heavy_w = 0;
+    size_t n_heavy = 0;
+    while (n_heavy < order.size() && pieces[order[n_heavy]].weight() > cta_share) heavy_w += pieces[order[n_heavy++]].weight();
+    const int n_h = int(std::max<int64_t>(1, std::min<int64_t>(n_used, (heavy_w + cta_share / 2) / cta_share)));
+    // every CTA boundary inside a unit opens one more piece with its own fixed cost
+    const int64_t target = (heavy_w + int64_t(n_h) * kSegWeight) * GLIDE_STREAM_FILL / 100 / n_h + 1;
+    int cta = 0;
+    int64_t cum = 0;   // weight laid out so far over all heavy CTAs
+    for (; oi < n_heavy; ++oi) {
       const Piece pc = pieces[order[oi]];
       int st_done = 0, w_done = 0;
       while (st_done < pc.nst || w_done < pc.nw) {
-        if (cta + 1 < cta_load.size() && cta_cap - cta_load[cta] < kSegWeight + 4 * kWinWeight) ++cta;   // CTA full
-        int64_t room = cta + 1 < cta_load.size() ? cta_cap - cta_load[cta] - kSegWeight : INT64_MAX / 4;
+        const bool last_cta = cta + 1 >= n_h;
+        int64_t room = last_cta ? INT64_MAX / 4 : int64_t(cta + 1) * target - cum - kSegWeight;
+        if (!last_cta && room < 4 * kWinWeight) {   // not worth a piece: this CTA is full
+          ++cta;
+          continue;
+        }
         Piece q = pc;
         q.st0 = pc.st0 + st_done;
-        q.nst = int(std::min<int64_t>(pc.nst - st_done, std::max<int64_t>(room, 0) / kStateWeight));
+        q.nst = int(std::min<int64_t>(pc.nst - st_done, room / kStateWeight));
         room -= kStateWeight * int64_t(q.nst);
         q.w0 = pc.w0 + w_done;
         q.nw = (st_done + q.nst == pc.nst) ? int(std::min<int64_t>(pc.nw - w_done, std::max<int64_t>(room, 0) / kWinWeight)) : 0;
-        if (q.nst + q.nw == 0) {   // cannot happen with the room check above, but never loop forever
+        // a remainder of a few tiles is not worth a piece of its own either
+        const int64_t rest = kStateWeight * int64_t(pc.nst - st_done - q.nst) + kWinWeight * int64_t(pc.nw - w_done - q.nw);
+        if (q.nst + q.nw == 0 || rest < 4 * kWinWeight) {
           q.nst = pc.nst - st_done;
           q.nw = pc.nw - w_done;
         }
         st_done += q.nst;
         w_done += q.nw;
         pieces.push_back(q);
-        cta_pieces[cta].push_back(pieces.size() - 1);
-        cta_load[cta] += q.weight();
+        cta_pieces[size_t(cta)].push_back(pieces.size() - 1);
+        cta_load[size_t(cta)] += q.weight();
+        cum += q.weight();
       }
     }
   }
+  // CTAs beyond n_used stay empty
+  for (size_t c = size_t(n_used); c < cta_load.size(); ++c) cta_load[c] = INT64_MAX / 2;
   // (b) every other unit goes whole onto the least loaded CTA
   for (; oi < order.size(); ++oi) {
     size_t best = 0;
@@ -1073,6 +1093,7 @@ void build_stream_schedule(const glide_ctx *ctx, int n_ranges, std::vector<Strea
     cta_pieces[best].push_back(order[oi]);
     cta_load[best] += pieces[order[oi]].weight();
   }
+  for (size_t c = size_t(n_used); c < cta_load.size(); ++c) cta_load[c] = 0;
 
   segs->clear();
   range_seg_begin->assign(size_t(n_ranges) + 1, 0);
@@ -1221,7 +1242,9 @@ int stream_decode_setup(glide_ctx *ctx) {
     }
     if (smem > size_t(dev_max)) return GLIDE_ERR_UNSUPPORTED;   // too many segments per CTA for the table
     auto kern = glide_decode_stream_kernel<G, S>;
-    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem)) != cudaSuccess) {
+    // the attribute belongs to the kernel, not to the context: ask for the device maximum so that contexts with
+    // different schedules (different table sizes) can be alive together
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, dev_max) != cudaSuccess) {
       cudaGetLastError();
       return GLIDE_ERR_CUDA;
     }
@@ -1256,7 +1279,11 @@ int launch_decode_stream(glide_ctx *ctx, const DecodeParams &p, cudaStream_t str
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
+#ifdef GLIDE_NO_PDL
+    cfg.numAttrs = 0;
+#else
     cfg.numAttrs = 1;
+#endif
     if (cudaLaunchKernelEx(&cfg, glide_decode_stream_kernel<G, S>, p, sp) != cudaSuccess) {
       cudaGetLastError();
       return GLIDE_ERR_CUDA;

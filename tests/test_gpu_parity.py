@@ -128,3 +128,24 @@ def test_bf16_prefill_tensor_core_multi_call(impl, G, chunk):
     # 128-key tile, one never-evicting layer, one purely linear layer; ragged last query tile
     run_case([0, 100, 128, 300, 1 << 20], 2, 2 * G, 2, 128, BF16, [130, 257, 61], 4, amp=128 ** -0.5 * 4,
              seed=chunk + G, prefill_chunk=chunk, prefill_impl=impl)
+
+
+def test_contexts_with_different_schedules_coexist():
+    # two live contexts whose streaming schedules need different amounts of shared memory; the one created first
+    # must still launch after the second was created
+    import numpy as np
+    from paper_2607_24788_b200 import glide, synth
+    from oracle import glide_oracle as orc
+    from tests.parity_util import f32_scale, to_np, check_outputs
+    d, B, H, Hkv = 128, 1, 8, 2
+    shapes = [[48] * 24, [48]]
+    wls = [synth.Workload(5 + i, len(w), B, H, Hkv, d, BF16, d ** -0.5 * 4) for i, w in enumerate(shapes)]
+    gs = [glide.Glide(w, B, H, Hkv, d, 64, dtype=BF16, softmax_scale=f32_scale(d)) for w in shapes]
+    stacks = [orc.Stack(w, B, H, Hkv, d, f32_scale(d)) for w in shapes]
+    for t in range(6):
+        for g, wl, st, w in zip(gs, wls, stacks, shapes):
+            q, k, v = wl.decode_qkv(t, "cuda")
+            out = torch.empty_like(q)
+            g.glide_decode_step(q, k, v, out)
+            ref = st.decode(to_np(q), to_np(k), to_np(v))
+            check_outputs(out, ref, BF16, f"L={len(w)} step {t}")
