@@ -1047,9 +1047,11 @@ void build_stream_schedule(const glide_ctx *ctx, int n_ranges, std::vector<Strea
     int64_t heavy_w = 0;
     size_t n_heavy = 0;
     while (n_heavy < order.size() && pieces[order[n_heavy]].weight() > cta_share) heavy_w += pieces[order[n_heavy++]].weight();
-    const int n_h = int(std::max<int64_t>(1, std::min<int64_t>(n_used, (heavy_w + cta_share / 2) / cta_share)));
+    // these CTAs end with a ticket + merge chain of a few microseconds: they get less than a full share
+    const int64_t heavy_share = std::max<int64_t>(1, cta_share * GLIDE_STREAM_FILL / 100);
+    const int n_h = int(std::max<int64_t>(1, std::min<int64_t>(n_used, (heavy_w + heavy_share / 2) / heavy_share)));
     // every CTA boundary inside a unit opens one more piece with its own fixed cost
-    const int64_t target = (heavy_w + int64_t(n_h) * kSegWeight) * GLIDE_STREAM_FILL / 100 / n_h + 1;
+    const int64_t target = (heavy_w + int64_t(n_h) * kSegWeight) / n_h + 1;
     int cta = 0;
     int64_t cum = 0;   // weight laid out so far over all heavy CTAs
     for (; oi < n_heavy; ++oi) {
