@@ -50,6 +50,9 @@ constexpr int kHdrSlots = 3;
 #ifndef GLIDE_STREAM_FILL
 #define GLIDE_STREAM_FILL 100
 #endif
+#ifndef GLIDE_STREAM_TMAP_PREFETCH
+#define GLIDE_STREAM_TMAP_PREFETCH 1
+#endif
 #ifndef GLIDE_W_MIN_CTA
 #define GLIDE_W_MIN_CTA 128   // least weight worth a CTA of its own (about ten tiles)
 #endif
@@ -168,6 +171,9 @@ __device__ __forceinline__ float4 lds_f32x4(uint32_t addr) {
   float4 v;
   asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(addr));
   return v;
+}
+__device__ __forceinline__ void prefetch_tensormap(const void *tmap) {
+  asm volatile("prefetch.tensormap [%0];" ::"l"(tmap) : "memory");
 }
 // ---- schedule walking ------------------------------------------------------------------------
 __device__ __forceinline__ float ex2_approx(float x) {   // 2^x, 2 ulp, 2^-inf = 0
@@ -304,6 +310,12 @@ glide_decode_stream_kernel(const DecodeParams p, const StreamParams sp) {
     fence_async_smem();
   }
   __syncthreads();   // segment table and barriers ready; the warps are on their own from here
+#if GLIDE_STREAM_TMAP_PREFETCH
+  // the ring descriptors are written when the context is created, never by a kernel: fetch the ones this
+  // CTA's segments use before waiting for the preceding kernel
+  if (tid < cta_nseg && sm_segs[tid].cap > 0)
+    prefetch_tensormap(reinterpret_cast<const CUtensorMap *>(sp.tmaps) + 3 * sm_segs[tid].layer + (sp.kv4d ? 2 : 0));
+#endif
   asm volatile("griddepcontrol.wait;" ::: "memory");   // the preceding kernel has completed and its writes are visible
   // every layer is at the same position (checked by the host); the host's copy of the counter comes with the
   // launch, which saves a dependent global load at the head of every warp's critical path
