@@ -208,13 +208,20 @@ __global__ void __launch_bounds__(kPrefillThreads) prefill_attn_kernel(const Pre
   }
 }
 
-// 3. S += phi(K'_c)^T V'_c ; z += sum phi(K'_c): one CTA per (unit, block of RB state rows)
+// 3. S += phi(K'_c)^T V'_c ; z += sum phi(K'_c) in fp32 on the CUDA cores (the carry keeps fp32 precision, which
+// a bf16 or tf32 tensor-core product of phi(K') would not).  One CTA per (unit, block of 64 state rows): the
+// chunk's phi(K') columns and V' rows are staged through shared memory 32 tokens at a time and every thread
+// accumulates an 8 x (D/16) register tile of rank-1 updates (rows ty*4..+3 and 32+ty*4..+3, columns tx*4..+3 and,
+// for D = 128, 64+tx*4..+3: 16-byte shared-memory reads without bank conflicts).
+constexpr int kStateRows = 64;    // state rows per CTA
+constexpr int kStateTok = 32;     // tokens per shared-memory stage
 template <typename T, int D>
 __global__ void __launch_bounds__(kPrefillThreads) prefill_state_kernel(const PrefillParams p) {
-  constexpr int RB = 16;                          // state rows per CTA
-  constexpr int NRS = kPrefillThreads / D > 0 ? kPrefillThreads / D : 1;  // row sub-groups (1 for D=128, 2 for D=64)
-  constexpr int RPT = RB / NRS;                   // rows per thread
-  const int blocks_per_unit = D / RB;
+  static_assert(kPrefillThreads == 128, "8 x 16 thread grid");
+  constexpr int CG = D / 64;                      // column groups of 4 per thread
+  __shared__ __align__(16) float sphi[kStateTok][kStateRows];
+  __shared__ __align__(16) float sv[kStateTok][D];
+  const int blocks_per_unit = D / kStateRows;
   const int64_t u = blockIdx.x / blocks_per_unit;
   const int rb = blockIdx.x % blocks_per_unit;
   const int g = int(u % p.Hkv);
@@ -223,32 +230,77 @@ __global__ void __launch_bounds__(kPrefillThreads) prefill_state_kernel(const Pr
   const LayerDev ld = p.layers[p.layer_begin + lrel];
   if (!ld.evicts) return;
   const int64_t first = p.n0 + p.c0 - ld.w;       // delayed token of chunk index 0
-  int i_lo = first < 0 ? int(first < -int64_t(p.C) ? p.C : -first) : 0;
+  const int i_lo = first < 0 ? int(first < -int64_t(p.C) ? p.C : -first) : 0;
   if (i_lo >= p.C) return;
   const RowSource<T> src = make_source<T, D>(p, ld, lrel, b, g);
   const int ub = b * p.Hkv + g;
-  const int c = threadIdx.x % D, rs = threadIdx.x / D;
-  const int r0 = rb * RB + rs * RPT;
-  const float *pk = p.phik + size_t(u) * p.Cmax * D;
-  if (rs < NRS) {
-    float acc[RPT];
+  const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
+  const float *pk = p.phik + size_t(u) * p.Cmax * D + rb * kStateRows;
+  float acc[8][4 * CG];
 #pragma unroll
-    for (int r = 0; r < RPT; ++r) acc[r] = 0.f;
-    for (int i = i_lo; i < p.C; ++i) {
-      const float vv = to_f32(src.v(first + i, D)[c]);
-      const float *f = pk + size_t(i) * D + r0;
+  for (int r = 0; r < 8; ++r)
 #pragma unroll
-      for (int r = 0; r < RPT; ++r) acc[r] = fmaf(f[r], vv, acc[r]);
+    for (int c = 0; c < 4 * CG; ++c) acc[r][c] = 0.f;
+  float zacc = 0.f;   // threads 0..63: z of row rb*64 + tid
+  for (int i0 = i_lo; i0 < p.C; i0 += kStateTok) {
+    const int nt = min(kStateTok, p.C - i0);
+    // stage: phi columns of this row block (fp32) and the delayed tokens' V rows (converted to fp32)
+    for (int e = tid; e < kStateTok * (kStateRows / 4); e += kPrefillThreads) {
+      const int i = e / (kStateRows / 4), c4 = e % (kStateRows / 4);
+      float4 f = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (i < nt) f = *reinterpret_cast<const float4 *>(pk + size_t(i0 + i) * D + c4 * 4);
+      *reinterpret_cast<float4 *>(&sphi[i][c4 * 4]) = f;
     }
-    float *Sb = reinterpret_cast<float *>(p.ws + ld.S) + size_t(ub) * D * D;
+    for (int e = tid; e < kStateTok * (D / 4); e += kPrefillThreads) {
+      const int i = e / (D / 4), c4 = e % (D / 4);
+      float x[4] = {0.f, 0.f, 0.f, 0.f};
+      if (i < nt) load_elems<T, 4>(src.v(first + i0 + i, D) + c4 * 4, x);
+      *reinterpret_cast<float4 *>(&sv[i][c4 * 4]) = make_float4(x[0], x[1], x[2], x[3]);
+    }
+    __syncthreads();
+#pragma unroll 4
+    for (int i = 0; i < kStateTok; ++i) {
+      const float4 fa = *reinterpret_cast<const float4 *>(&sphi[i][ty * 4]);
+      const float4 fb = *reinterpret_cast<const float4 *>(&sphi[i][32 + ty * 4]);
+      const float fr[8] = {fa.x, fa.y, fa.z, fa.w, fb.x, fb.y, fb.z, fb.w};
+      float vc[4 * CG];
 #pragma unroll
-    for (int r = 0; r < RPT; ++r) Sb[size_t(r0 + r) * D + c] += acc[r];
+      for (int cg = 0; cg < CG; ++cg) {
+        const float4 vv = *reinterpret_cast<const float4 *>(&sv[i][cg * 64 + tx * 4]);
+        vc[cg * 4 + 0] = vv.x;
+        vc[cg * 4 + 1] = vv.y;
+        vc[cg * 4 + 2] = vv.z;
+        vc[cg * 4 + 3] = vv.w;
+      }
+#pragma unroll
+      for (int r = 0; r < 8; ++r)
+#pragma unroll
+        for (int c = 0; c < 4 * CG; ++c) acc[r][c] = fmaf(fr[r], vc[c], acc[r][c]);
+    }
+    if (tid < kStateRows) {
+#pragma unroll 8
+      for (int i = 0; i < kStateTok; ++i) zacc += sphi[i][tid];
+    }
+    __syncthreads();
   }
-  if (rb == 0 && threadIdx.x < D) {
-    float zs = 0.f;
-    for (int i = i_lo; i < p.C; ++i) zs += pk[size_t(i) * D + threadIdx.x];
-    float *zb = reinterpret_cast<float *>(p.ws + ld.z) + size_t(ub) * D;
-    zb[threadIdx.x] += zs;
+  float *Sb = reinterpret_cast<float *>(p.ws + ld.S) + size_t(ub) * D * D + size_t(rb) * kStateRows * D;
+#pragma unroll
+  for (int r = 0; r < 8; ++r) {
+    const int row = (r >> 2) * 32 + ty * 4 + (r & 3);
+#pragma unroll
+    for (int cg = 0; cg < CG; ++cg) {
+      float4 *dst = reinterpret_cast<float4 *>(Sb + size_t(row) * D + cg * 64 + tx * 4);
+      float4 cur = *dst;
+      cur.x += acc[r][cg * 4 + 0];
+      cur.y += acc[r][cg * 4 + 1];
+      cur.z += acc[r][cg * 4 + 2];
+      cur.w += acc[r][cg * 4 + 3];
+      *dst = cur;
+    }
+  }
+  if (tid < kStateRows) {
+    float *zb = reinterpret_cast<float *>(p.ws + ld.z) + size_t(ub) * D + rb * kStateRows;
+    zb[tid] += zacc;
   }
 }
 
@@ -332,7 +384,7 @@ int launch_prefill(glide_ctx *ctx, int layer_begin, int layer_count, int64_t T, 
           prefill_attn_kernel<TT, D, G><<<warp_blocks, kPrefillThreads, 0, stream>>>(p);
         }
       }
-      if (any_evicts) prefill_state_kernel<TT, D><<<unsigned(units * (D / 16)), kPrefillThreads, 0, stream>>>(p);
+      if (any_evicts) prefill_state_kernel<TT, D><<<unsigned(units * (D / kStateRows)), kPrefillThreads, 0, stream>>>(p);
       prefill_ring_kernel<TT, D><<<warp_blocks, kPrefillThreads, 0, stream>>>(p);
       if (cudaGetLastError() != cudaSuccess) return GLIDE_ERR_CUDA;
     }
