@@ -1,22 +1,28 @@
-// GLIDE prefill outputs on the 5th-generation tensor cores (tcgen05 + TMEM), bf16 I/O, head_dim 128.
+// GLIDE prefill outputs on the 5th-generation tensor cores (tcgen05 + TMEM + TMA), bf16 I/O, head_dim 128.
 //
-// One CTA (128 threads) owns 128 query rows of one (layer, sequence, KV head) unit -- 128/G consecutive
-// tokens of the chunk times the G query heads (row = token * G + head) -- and thread r owns row r, which
-// is also TMEM lane r.
-//   window part   128-key tiles of the sliding window (ring rows for tokens older than the call, the call's
-//                 own rows otherwise) are staged with cp.async into the 128-byte-swizzled K-major / MN-major
-//                 layouts tcgen05.mma reads.  One elected thread issues S = Q K^T (8 x m128n128k16) into TMEM
-//                 columns [0,128); every thread reads its row with tcgen05.ld, masks, takes the row maximum
-//                 without any shuffle, writes P = 2^(s - m_ref) as bf16 into the swizzled A-operand layout,
-//                 and the elected thread issues O += P V into TMEM columns [128,256).  The reference m_ref is
-//                 lazy: O is rescaled in TMEM (tcgen05.ld / tcgen05.st) only when a row's maximum grows by
-//                 more than 2^8.  K tiles are prefetched two tiles ahead, V tiles one.
-//   linear part   with m* = max(m_ref, 0) per row: phi(Q) 2^-m* (bf16, K-major) times a bf16 copy of the state
-//                 (inter-chunk), and C = phi(Q) phi(K')^T masked to j' <= i, then C V' (intra-chunk), through the
-//                 same two MMAs; l accumulates the matching sums.
-//   out = O / l, bf16, one contiguous 256-byte row per thread.
-// Every mbarrier wait is bounded; on a time-out the CTA records kDevWaitTimeout, skips the remaining work,
-// frees its TMEM columns and returns.
+// One CTA (10 warps) owns 256 query rows of one (layer, sequence, KV head) unit: two row tiles X = A, B of 128
+// rows each, a row being (token, query head of the group), row = token * G + head.
+//   warps 0-3   softmax of tile A: thread r owns row r = TMEM lane r
+//   warps 4-7   softmax of tile B
+//   warp 8      one elected thread issues every tcgen05.mma
+//   warp 9      one elected thread issues the TMA loads of the K and V tiles
+// Window part, per 128-key tile t (keys are tokens j0 + 0..127, j0 a multiple of 16):
+//   loader    K_t and V_t as 16-token boxes (ring rows for tokens older than the call, the call's rows otherwise)
+//             into a ring of three 32 KiB buffers, 128-byte swizzle, completion on an mbarrier
+//   MMA       S_X = Q_X K_t^T into TMEM (8 x m128n128k16), committed to an mbarrier the softmax warps wait on
+//   softmax   tcgen05.ld of the own row, mask, row maximum without any shuffle, P = 2^(s - m_ref) as bf16 into
+//             the swizzled A-operand layout in shared memory; the reference m_ref is lazy: O is rescaled in
+//             TMEM only when the maximum grows by more than 2^8
+//   MMA       O_X += P_X V_t (V as the MN-major B operand), then S_X of the next tile: while one row tile is
+//             in its softmax the tensor core works for the other
+// TMEM columns: S_A [0,128) S_B [128,256) O_A [256,384) O_B [384,512).
+// Linear part (after the window tiles, the whole CTA in step): with m* = max(m_ref, 0) per row, phi(Q) 2^-m* as
+// bf16 times a bf16 copy of the state (inter-chunk), and C = phi(Q) phi(K')^T masked to j' <= i, then C V'
+// (intra-chunk), through the same MMAs; l accumulates the matching sums.  out = O / l.
+// Every mbarrier wait is bounded; on a time-out the CTA records kDevWaitTimeout, leaves its loops, frees its TMEM
+// columns and returns.
+#include <cuda.h>
+
 #include <algorithm>
 
 #include "glide_device.cuh"
@@ -26,13 +32,18 @@ namespace glide {
 namespace {
 
 constexpr int kD = 128;
-constexpr int kRows = 128;
-constexpr int kKT = 128;             // keys per tile
-constexpr int kThreads = 128;
+constexpr int kRows = 128;            // rows per row tile
+constexpr int kKT = 128;              // keys per tile
+constexpr int kGroup = 16;            // tokens per TMA box
+constexpr int kSoftmaxThreads = 256;
+constexpr int kThreads = 320;
+constexpr int kMmaWarp = 8, kLoadWarp = 9;
 constexpr uint32_t kTileBytes = 32768;   // [2 boxes][128 rows][64 bf16]
 constexpr uint32_t kBoxBytes = 16384;
+constexpr uint32_t kGroupBytes = kGroup * 128;   // one 16-token box of 64 columns
 constexpr uint32_t kWaitLimit = 1u << 20;
-constexpr float kLazy = 8.0f;        // rescale O only when the row maximum grows by more than 2^8
+constexpr float kLazy = 8.0f;         // rescale O only when the row maximum grows by more than 2^8
+constexpr int kStages = 3;
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return uint32_t(__cvta_generic_to_shared(p)); }
 // byte offset of 16-byte chunk c16 (0..15) of row `row` inside a [2][128][64] bf16 tile with 128-byte swizzle
@@ -44,10 +55,7 @@ __device__ __forceinline__ void cp_async16(uint32_t dst, const void *src, bool v
   asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(bytes) : "memory");
 }
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
-template <int N>
-__device__ __forceinline__ void cp_async_wait() {
-  asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
-}
+__device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_group 0;" ::: "memory"); }
 __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
@@ -55,6 +63,11 @@ __device__ __forceinline__ float ex2(float x) {
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
+}
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
+  uint32_t r;
+  asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+  return r;
 }
 // shared-memory matrix descriptor, 128-byte swizzle
 __device__ __forceinline__ uint64_t make_desc(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
@@ -77,17 +90,54 @@ __device__ __forceinline__ void mma_f16(uint32_t tmem_d, uint64_t adesc, uint64_
       "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
       : "memory");
 }
+// 8 MMAs of one 128 x 128 x 128 product; B K-major (D = A B^T) or MN-major (D (+)= A B)
+__device__ __forceinline__ void issue_mma(uint32_t tmem_d, uint32_t a_tile, uint32_t b_tile, bool b_mn, bool accumulate) {
+  const uint32_t idesc = make_idesc(b_mn);
+#pragma unroll
+  for (int ks = 0; ks < 8; ++ks) {
+    const uint64_t adesc = make_desc(a_tile + (ks >> 2) * kBoxBytes + (ks & 3) * 32, 16, 1024);
+    const uint64_t bdesc = b_mn ? make_desc(b_tile + ks * 2048, kBoxBytes, 1024)
+                                : make_desc(b_tile + (ks >> 2) * kBoxBytes + (ks & 3) * 32, 16, 1024);
+    mma_f16(tmem_d, adesc, bdesc, idesc, (accumulate || ks > 0) ? 1u : 0u);
+  }
+}
 __device__ __forceinline__ void mma_commit(uint32_t bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
-  uint32_t ok = 0;
-  for (uint32_t spin = 0; spin < kWaitLimit && !ok; ++spin)
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+// Bounded wait; gives up early when another thread of the CTA has already timed out.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *failed) {
+  for (uint32_t spin = 0; spin < kWaitLimit; ++spin) {
+    uint32_t ok;
     asm volatile("{.reg .pred p; mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2; selp.u32 %0, 1, 0, p;}"
                  : "=r"(ok)
                  : "r"(bar), "r"(parity)
                  : "memory");
-  return ok != 0;
+    if (ok) return true;
+    if ((spin & 1023u) == 1023u && *failed) return false;
+  }
+  *failed = 1;
+  return false;
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const void *tmap, int x, int y, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(dst),
+      "l"(tmap), "r"(x), "r"(y), "r"(bar)
+      : "memory");
+}
+__device__ __forceinline__ void tma_load_4d(uint32_t dst, const void *tmap, int c0, int c1, int c2, int c3, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5}], [%6];" ::"r"(dst),
+      "l"(tmap), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(bar)
+      : "memory");
 }
 __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
   asm volatile(
@@ -113,110 +163,110 @@ __device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32
 }
 
 struct Smem {
-  unsigned char q[kTileBytes];       // Q, later phi(Q) 2^-m*
-  unsigned char p[kTileBytes];       // P (or C): A operand of the second MMA
-  unsigned char k[2][kTileBytes];    // K tiles / phi(K') tile
-  unsigned char v[2][kTileBytes];    // V tiles / bf16 state / V' tile
+  unsigned char q[2][kTileBytes];        // Q_A, Q_B; later phi(Q) 2^-m*
+  unsigned char p[2][kTileBytes];        // P_A, P_B (or C): A operand of the second MMA
+  unsigned char kv[kStages][kTileBytes]; // K and V tiles in turn; linear part: bf16 state, phi(K') tile, V' tile
   float z[kD];
-  uint64_t bar;                      // completion of the MMAs issued so far
+  uint64_t bar_full[kStages];            // TMA bytes of the buffer have landed
+  uint64_t bar_free[kStages];            // the MMAs that read the buffer have completed
+  uint64_t bar_q[2];                     // Q_X staged (128 arrivals)
+  uint64_t bar_s[2];                     // S_X of the current tile is in TMEM
+  uint64_t bar_p[2];                     // P_X of the current tile is in shared memory (128 arrivals)
+  uint64_t bar_done;                     // every window MMA has completed
+  uint64_t bar_lin;                      // linear part: the MMAs issued so far have completed
   uint32_t tmem_base;
   int failed;
 };
+static_assert(sizeof(Smem) + 1024 <= 232448, "shared memory of one CTA");
 
+// the call's K (or V) rows as a 4-D tensor {d, Hkv, T, layers x sequences}: boxes of 16 tokens x 64 columns of one KV head
+struct CallMaps {
+  CUtensorMap k, v;
+};
 
 template <int G>
-__global__ void __launch_bounds__(kThreads, 1) prefill_attn_tc_kernel(const PrefillParams p) {
+__global__ void __launch_bounds__(kThreads, 1)
+prefill_attn_tc_kernel(const PrefillParams p, const CUtensorMap *ring_maps, const __grid_constant__ CallMaps cm) {
   using bf16 = __nv_bfloat16;
-  constexpr int TOK = kRows / G;
+  constexpr int TOKT = kRows / G;    // tokens per row tile
+  constexpr int TOKC = 2 * TOKT;     // tokens per CTA
   extern __shared__ __align__(1024) unsigned char smem_raw[];
   Smem &sm = *reinterpret_cast<Smem *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-  const int tid = threadIdx.x, warp = tid >> 5;
-  const int tiles_per_chunk = (p.C + TOK - 1) / TOK;
-  const int64_t u = blockIdx.x / tiles_per_chunk;
-  const int tok0 = int(blockIdx.x % tiles_per_chunk) * TOK;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int ctas_per_chunk = (p.C + TOKC - 1) / TOKC;
+  const int64_t u = blockIdx.x / ctas_per_chunk;
+  const int tok0 = int(blockIdx.x % ctas_per_chunk) * TOKC;
   const int g = int(u % p.Hkv);
   const int b = int((u / p.Hkv) % p.B);
   const int lrel = int(u / (int64_t(p.Hkv) * p.B));
-  const LayerDev ld = p.layers[p.layer_begin + lrel];
-  const int ntok = min(TOK, p.C - tok0);
+  const int layer = p.layer_begin + lrel;
+  const LayerDev ld = p.layers[layer];
+  const int ntok = min(TOKC, p.C - tok0);
+  const int ntokA = min(TOKT, ntok), ntokB = ntok - ntokA;
+  const bool hasB = ntokB > 0;
   const int64_t tq0 = p.n0 + p.c0 + tok0;
   const int64_t tq_last = tq0 + ntok - 1;
   const int64_t w = ld.w;
   const uint32_t cap = ld.cap > 0 ? uint32_t(ld.cap) : 1u;
-
   const size_t unit_rows = (size_t(b) * p.Hkv + g) * size_t(ld.cap);
-  const bf16 *ringK = reinterpret_cast<const bf16 *>(p.ws + ld.ringK) + unit_rows * kD;
-  const bf16 *ringV = reinterpret_cast<const bf16 *>(p.ws + ld.ringV) + unit_rows * kD;
   const size_t seq = (size_t(lrel) * p.B + b) * size_t(p.T);
-  const bf16 *callK = reinterpret_cast<const bf16 *>(p.k) + (seq * p.Hkv + g) * kD;
-  const bf16 *callV = reinterpret_cast<const bf16 *>(p.v) + (seq * p.Hkv + g) * kD;
-  const int64_t call_stride = int64_t(p.Hkv) * kD;
+  volatile int *failed = &sm.failed;
 
   // a time-out recorded by an earlier CTA ends the launch quickly
   if (*reinterpret_cast<volatile int32_t *>(&p.ctl->status) == kDevWaitTimeout) return;
 
-  const uint32_t sQ = smem_u32(sm.q), sP = smem_u32(sm.p);
-  const uint32_t sK[2] = {smem_u32(sm.k[0]), smem_u32(sm.k[1])};
-  const uint32_t sV[2] = {smem_u32(sm.v[0]), smem_u32(sm.v[1])};
-  const uint32_t bar = smem_u32(&sm.bar);
+  const bool has_window = w > 0;
+  int64_t j_lo = tq0 - w + 1;
+  if (j_lo < 0) j_lo = 0;
+  j_lo &= ~int64_t(kGroup - 1);   // key tiles start at a multiple of the TMA box
+  const int n_tiles = has_window ? int((tq_last - j_lo) / kKT) + 1 : 0;
 
   if (tid == 0) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(bar));
+    for (int s = 0; s < kStages; ++s) {
+      mbar_init(smem_u32(&sm.bar_full[s]), 1);
+      mbar_init(smem_u32(&sm.bar_free[s]), 1);
+    }
+    for (int x = 0; x < 2; ++x) {
+      mbar_init(smem_u32(&sm.bar_q[x]), kRows);
+      mbar_init(smem_u32(&sm.bar_s[x]), 1);
+      mbar_init(smem_u32(&sm.bar_p[x]), kRows);
+    }
+    mbar_init(smem_u32(&sm.bar_done), 1);
+    mbar_init(smem_u32(&sm.bar_lin), 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     sm.failed = 0;
   }
   if (warp == 0) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], 256;" ::"r"(smem_u32(&sm.tmem_base)) : "memory");
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], 512;" ::"r"(smem_u32(&sm.tmem_base)) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
+  // K/V buffers start at zero: token groups past the CTA's last token are never loaded, and what a masked key's
+  // V row holds is multiplied by a zero weight, so it has to be finite
+  for (int i = tid; i < int(kStages * kTileBytes / 16); i += kThreads)
+    reinterpret_cast<uint4 *>(&sm.kv[0][0])[i] = make_uint4(0u, 0u, 0u, 0u);
+  fence_async_smem();
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = sm.tmem_base;
-  const uint32_t tS = tmem + (uint32_t(warp * 32) << 16);         // this warp's lanes, columns [0,128): S / C
-  const uint32_t tO = tS + 128;                                    // columns [128,256): O
-  uint32_t phase = 0;
-  bool failed = false;
+  const uint32_t sQ[2] = {smem_u32(sm.q[0]), smem_u32(sm.q[1])};
+  const uint32_t sP[2] = {smem_u32(sm.p[0]), smem_u32(sm.p[1])};
+  const uint32_t sKV[kStages] = {smem_u32(sm.kv[0]), smem_u32(sm.kv[1]), smem_u32(sm.kv[2])};
 
-  // rows of tokens j0 .. j0+127 (absolute) of K or V -> swizzled tile; tokens outside [0, j_max] are zero-filled
-  auto load_rows = [&](uint32_t dst, bool is_v, int64_t j0, int64_t j_max) {
-    const bf16 *ring = is_v ? ringV : ringK;
-    const bf16 *call = is_v ? callV : callK;
-#pragma unroll 4
-    for (int i = 0; i < kKT * 16 / kThreads; ++i) {
-      const int id = tid + kThreads * i;
-      const int r = id >> 4, c = id & 15;
-      const int64_t j = j0 + r;
-      const bool valid = j >= 0 && j <= j_max;
-      const int64_t jj = valid ? j : 0;
-      const bool from_call = jj >= p.n0;
-      const bf16 *src = from_call ? call + size_t(jj - p.n0) * call_stride : ring + size_t(uint32_t(jj) % cap) * kD;
-      cp_async16(dst + sw128(r, c), src + c * 8, valid);
-    }
-  };
-  // 8 MMAs of one 128 x 128 x 128 product; B K-major (S = A B^T) or MN-major (O += A B)
-  auto issue_mma = [&](uint32_t tmem_d, uint32_t a_tile, uint32_t b_tile, bool b_mn, bool accumulate) {
-    const uint32_t idesc = make_idesc(b_mn);
-#pragma unroll
-    for (int ks = 0; ks < 8; ++ks) {
-      const uint64_t adesc = make_desc(a_tile + (ks >> 2) * kBoxBytes + (ks & 3) * 32, 16, 1024);
-      const uint64_t bdesc = b_mn ? make_desc(b_tile + ks * 2048, kBoxBytes, 1024)
-                                  : make_desc(b_tile + (ks >> 2) * kBoxBytes + (ks & 3) * 32, 16, 1024);
-      mma_f16(tmem_d, adesc, bdesc, idesc, (accumulate || ks > 0) ? 1u : 0u);
-    }
-  };
-  // all threads wait for the MMAs committed so far; `failed` stays uniform over the warp
-  auto wait_mma = [&]() {
-    __syncwarp();
-    bool bad = failed;
-    if (!bad && !mbar_wait(bar, phase & 1u)) {
-      bad = true;
-      sm.failed = 1;
-    }
-    failed = __any_sync(0xffffffffu, bad);
-    ++phase;
-    tc_fence_after();
-  };
+  // ---- softmax threads: per-row state that lives across the window and the linear part ----------------------
+  const int X = (tid >> 7) & 1;                   // row tile of this thread (softmax warps only)
+  const int row = tid & 127;
+  const int tok_r = row / G, hh = row - tok_r * G;
+  const int ntokX = X ? ntokB : ntokA;
+  const bool activeX = tid < kSoftmaxThreads && ntokX > 0;
+  const int tl = tok0 + X * TOKT + tok_r;         // chunk-relative token of this row
+  const int64_t tok_abs = p.n0 + p.c0 + tl;
+  const uint32_t tS = tmem + (uint32_t((warp & 3) * 32) << 16) + uint32_t(X) * 128u;
+  const uint32_t tO = tS + 256u;
+  float m_ref = -CUDART_INF_F, l_sum = 0.f;
+  const bf16 *qrow = reinterpret_cast<const bf16 *>(p.q) +
+                     ((seq + size_t(p.c0 + (tok_r < ntokX ? tl : tok0))) * p.H + p.heads_of[g * G + hh]) * kD;
+
   // multiply this thread's O row by f (warp-collective TMEM read-modify-write)
   auto scale_o = [&](float f) {
 #pragma unroll 1
@@ -228,132 +278,199 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_attn_tc_kernel(const Pref
       tmem_st32(tO + c0, r);
     }
   };
-
-  const int row = tid;
-  const int tok_r = row / G, hh = row - tok_r * G;
-  const int64_t tok_abs = tq0 + tok_r;
-
-  // ---- prologue: Q and the first tiles ---------------------------------------------------------------
-  const bool has_window = w > 0;
-  int64_t j_lo = tq0 - w + 1;
-  if (j_lo < 0) j_lo = 0;
-  const int n_wtiles = has_window ? int((tq_last - j_lo) / kKT) + 1 : 0;
-  {
-    const bf16 *qbase = reinterpret_cast<const bf16 *>(p.q) + (seq + size_t(p.c0 + tok0)) * p.H * kD;
-#pragma unroll 4
-    for (int i = 0; i < kRows * 16 / kThreads; ++i) {
-      const int id = tid + kThreads * i;
-      const int r = id >> 4, c = id & 15;
-      const int tk = r / G, h2 = r - tk * G;
-      const bool valid = tk < ntok;
-      cp_async16(sQ + sw128(r, c), qbase + (size_t(valid ? tk : 0) * p.H + p.heads_of[g * G + h2]) * kD + c * 8, valid);
-    }
-    if (n_wtiles > 0) load_rows(sK[0], false, j_lo, tq_last);
-    cp_async_commit();
-    if (n_wtiles > 1) load_rows(sK[1], false, j_lo + kKT, tq_last);
-    if (n_wtiles > 0) load_rows(sV[0], true, j_lo, tq_last);
-    cp_async_commit();
-  }
-  bool o_init = false;   // O holds a valid accumulation (uniform over the CTA)
-  if (n_wtiles > 0) {
-    cp_async_wait<1>();
-    fence_async_smem();
-    tc_fence_before();
-    __syncthreads();
-    if (tid == 0) {
-      tc_fence_after();
-      issue_mma(tmem, sQ, sK[0], false, false);
-      mma_commit(bar);
-    }
-  }
-
-  float m_ref = -CUDART_INF_F, l_sum = 0.f;
-  // ---- window part -------------------------------------------------------------------------------------
-  for (int t = 0; t < n_wtiles; ++t) {
-    wait_mma();   // S(t) is in TMEM, O += P V of tile t-1 has finished
-    if (t + 2 < n_wtiles) load_rows(sK[t & 1], false, j_lo + int64_t(t + 2) * kKT, tq_last);
-    if (t + 1 < n_wtiles) load_rows(sV[(t + 1) & 1], true, j_lo + int64_t(t + 1) * kKT, tq_last);
-    cp_async_commit();
-    const int64_t j0 = j_lo + int64_t(t) * kKT;
-    const bool interior = j0 + kKT - 1 <= tq0 && j0 > tq_last - w;
-    if (!failed) {
-      // pass 1: row maximum of the masked, scaled logits
-      float mx = -CUDART_INF_F;
+  // weights of one S row against reference mr (log2 domain) -> bf16 P row in the swizzled A layout; returns their sum
+  auto write_p = [&](auto masked, int lo, int hi, float mr, float scale) -> float {
+    constexpr bool kMasked = decltype(masked)::value;
+    float sum0 = 0.f, sum1 = 0.f;
+    unsigned char *prow = sm.p[X];
 #pragma unroll 1
-      for (int c0 = 0; c0 < kKT; c0 += 32) {
-        uint32_t r[32];
-        tmem_ld32(tS + c0, r);
+    for (int c0 = 0; c0 < kKT; c0 += 32) {
+      uint32_t r[32];
+      tmem_ld32(tS + c0, r);
 #pragma unroll
-        for (int i = 0; i < 32; ++i) {
-          const int64_t j = j0 + c0 + i;
-          const bool ok = interior || (j <= tok_abs && j > tok_abs - w);
-          if (ok) mx = fmaxf(mx, __uint_as_float(r[i]) * p.scale_log2);
-        }
-      }
-      // lazy reference: move it (and rescale O, l) only when the maximum grows by more than 2^kLazy
-      float f = 1.f;
-      if (mx > m_ref + kLazy || (m_ref == -CUDART_INF_F && mx > -CUDART_INF_F)) {
-        f = m_ref == -CUDART_INF_F ? 0.f : ex2(m_ref - mx);
-        m_ref = mx;
-      }
-      if (o_init && __any_sync(0xffffffffu, f != 1.f)) scale_o(f);
-      l_sum *= f;
-      const float mr = m_ref == -CUDART_INF_F ? 0.f : m_ref;
-      // pass 2: P = 2^(s - m_ref) as bf16 into the swizzled A-operand layout; the row sum uses the rounded weights
-#pragma unroll 1
-      for (int c0 = 0; c0 < kKT; c0 += 32) {
-        uint32_t r[32];
-        tmem_ld32(tS + c0, r);
+      for (int q4 = 0; q4 < 4; ++q4) {
+        uint32_t pk[4];
 #pragma unroll
-        for (int q4 = 0; q4 < 4; ++q4) {
-          uint32_t pk[4];
-#pragma unroll
-          for (int e = 0; e < 4; ++e) {
-            float pv[2];
-#pragma unroll
-            for (int z2 = 0; z2 < 2; ++z2) {
-              const int i = q4 * 8 + e * 2 + z2;
-              const int64_t j = j0 + c0 + i;
-              const bool ok = interior || (j <= tok_abs && j > tok_abs - w);
-              pv[z2] = ok ? ex2(__uint_as_float(r[i]) * p.scale_log2 - mr) : 0.f;
-            }
-            const __nv_bfloat162 h2 = __floats2bfloat162_rn(pv[0], pv[1]);
-            l_sum += __low2float(h2) + __high2float(h2);
-            pk[e] = *reinterpret_cast<const uint32_t *>(&h2);
+        for (int e = 0; e < 4; ++e) {
+          const int i = q4 * 8 + e * 2;
+          float a0 = ex2(fmaf(__uint_as_float(r[i]), scale, -mr));
+          float a1 = ex2(fmaf(__uint_as_float(r[i + 1]), scale, -mr));
+          if (kMasked) {
+            if (c0 + i < lo || c0 + i > hi) a0 = 0.f;
+            if (c0 + i + 1 < lo || c0 + i + 1 > hi) a1 = 0.f;
           }
-          *reinterpret_cast<uint4 *>(sm.p + sw128(row, (c0 >> 3) + q4)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+          pk[e] = pack_bf16x2(a0, a1);
+          sum0 += __uint_as_float(pk[e] << 16);          // the sum uses the weights as the tensor core sees them
+          sum1 += __uint_as_float(pk[e] & 0xffff0000u);
+        }
+        *reinterpret_cast<uint4 *>(prow + sw128(row, (c0 >> 3) + q4)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+      }
+    }
+    return sum0 + sum1;
+  };
+
+  // =========================== window part: warp-specialised ===========================
+  if (tid < kSoftmaxThreads) {
+    if (activeX) {
+      // Q_X: 128 rows x 16 chunks by the 128 threads of the row tile
+      const bf16 *qbase = reinterpret_cast<const bf16 *>(p.q) + (seq + size_t(p.c0 + tok0 + X * TOKT)) * p.H * kD;
+#pragma unroll 4
+      for (int i = 0; i < kRows * 16 / kRows; ++i) {
+        const int id = row + kRows * i;
+        const int r = id >> 4, c = id & 15;
+        const int tk = r / G, h2 = r - tk * G;
+        const bool valid = tk < ntokX;
+        cp_async16(sQ[X] + sw128(r, c), qbase + (size_t(valid ? tk : 0) * p.H + p.heads_of[g * G + h2]) * kD + c * 8, valid);
+      }
+      cp_async_commit();
+      cp_async_wait_all();
+      fence_async_smem();
+      mbar_arrive(smem_u32(&sm.bar_q[X]));
+
+      const int64_t tqX0 = tq0 + X * TOKT, tqX_last = tqX0 + ntokX - 1;
+      bool o_written = false;   // a P V product has been accumulated into O_X (uniform over the row tile)
+      for (int t = 0; t < n_tiles; ++t) {
+        const bool got = mbar_wait(smem_u32(&sm.bar_s[X]), uint32_t(t) & 1u, failed);
+        if (!__all_sync(0xffffffffu, got)) break;   // warp-uniform: the collectives below need every lane
+        tc_fence_after();
+        const int64_t j0 = j_lo + int64_t(t) * kKT;
+        const bool interior = j0 + kKT - 1 <= tqX0 && j0 > tqX_last - w;
+        // valid columns of this row: lo <= c <= hi
+        int64_t lo64 = tok_abs - w + 1 - j0, hi64 = tok_abs - j0;
+        const int lo = int(lo64 < 0 ? 0 : (lo64 > kKT ? kKT : lo64));
+        const int hi = int(hi64 < -1 ? -1 : (hi64 > kKT - 1 ? kKT - 1 : hi64));
+        // pass 1: row maximum of the valid raw scores (the scale is positive: it is applied to the maximum)
+        float mx = -CUDART_INF_F;
+#pragma unroll 1
+        for (int c0 = 0; c0 < kKT; c0 += 32) {
+          uint32_t r[32];
+          tmem_ld32(tS + c0, r);
+          float m4[4] = {-CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F};
+          if (interior) {
+#pragma unroll
+            for (int i = 0; i < 32; ++i) m4[i & 3] = fmaxf(m4[i & 3], __uint_as_float(r[i]));
+          } else {
+#pragma unroll
+            for (int i = 0; i < 32; ++i)
+              if (c0 + i >= lo && c0 + i <= hi) m4[i & 3] = fmaxf(m4[i & 3], __uint_as_float(r[i]));
+          }
+          mx = fmaxf(mx, fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3])));
+        }
+        mx *= p.scale_log2;
+        // lazy reference: move it (and rescale O, l) only when the maximum grows by more than 2^kLazy
+        float f = 1.f;
+        if (mx > m_ref + kLazy || (m_ref == -CUDART_INF_F && mx > -CUDART_INF_F)) {
+          f = m_ref == -CUDART_INF_F ? 0.f : ex2(m_ref - mx);
+          m_ref = mx;
+        }
+        if (o_written && __any_sync(0xffffffffu, f != 1.f)) scale_o(f);
+        l_sum *= f;
+        const float mr = m_ref == -CUDART_INF_F ? 0.f : m_ref;
+        if (interior) l_sum += write_p(IntTag<0>{}, lo, hi, mr, p.scale_log2);
+        else l_sum += write_p(IntTag<1>{}, lo, hi, mr, p.scale_log2);
+        fence_async_smem();     // P is read by the tensor core (async proxy)
+        tc_fence_before();      // this thread's TMEM reads of S_X precede the MMA that overwrites it
+        mbar_arrive(smem_u32(&sm.bar_p[X]));
+        o_written = true;
+      }
+    }
+    if (n_tiles > 0) mbar_wait(smem_u32(&sm.bar_done), 0u, failed);
+    tc_fence_after();
+  } else if (warp == kMmaWarp) {
+    if (lane == 0 && n_tiles > 0) {
+      bool ok = mbar_wait(smem_u32(&sm.bar_q[0]), 0u, failed);
+      if (ok && hasB) ok = mbar_wait(smem_u32(&sm.bar_q[1]), 0u, failed);
+      if (ok) ok = mbar_wait(smem_u32(&sm.bar_full[0]), 0u, failed);   // K_0
+      if (ok) {
+        tc_fence_after();
+        issue_mma(tmem, sQ[0], sKV[0], false, false);
+        mma_commit(smem_u32(&sm.bar_s[0]));
+        if (hasB) {
+          issue_mma(tmem + 128, sQ[1], sKV[0], false, false);
+          mma_commit(smem_u32(&sm.bar_s[1]));
+        }
+        mma_commit(smem_u32(&sm.bar_free[0]));
+      }
+      for (int t = 0; t < n_tiles && ok; ++t) {
+        const int seqV = 2 * t + 1, seqK = 2 * t + 2;
+        const bool more = t + 1 < n_tiles;
+        ok = mbar_wait(smem_u32(&sm.bar_full[seqV % kStages]), uint32_t(seqV / kStages) & 1u, failed);
+        if (ok && more) ok = mbar_wait(smem_u32(&sm.bar_full[seqK % kStages]), uint32_t(seqK / kStages) & 1u, failed);
+        for (int x = 0; x < 2 && ok; ++x) {
+          if (x == 1 && !hasB) break;
+          ok = mbar_wait(smem_u32(&sm.bar_p[x]), uint32_t(t) & 1u, failed);
+          if (!ok) break;
+          tc_fence_after();
+          issue_mma(tmem + 256 + x * 128, sP[x], sKV[seqV % kStages], true, t > 0);
+          if (more) {
+            issue_mma(tmem + x * 128, sQ[x], sKV[seqK % kStages], false, false);
+            mma_commit(smem_u32(&sm.bar_s[x]));
+          }
+        }
+        if (ok) {
+          mma_commit(smem_u32(&sm.bar_free[seqV % kStages]));
+          if (more) mma_commit(smem_u32(&sm.bar_free[seqK % kStages]));
+        }
+      }
+      if (ok) mma_commit(smem_u32(&sm.bar_done));
+    }
+  } else if (warp == kLoadWarp) {
+    if (lane == 0 && n_tiles > 0) {
+      const CUtensorMap *ringK = ring_maps + 3 * layer, *ringV = ringK + 1;
+      bool ok = true;
+      for (int sq = 0; sq < 2 * n_tiles && ok; ++sq) {
+        const int t = sq >> 1, slot = sq % kStages;
+        const bool is_v = sq & 1;
+        if (sq >= kStages) ok = mbar_wait(smem_u32(&sm.bar_free[slot]), uint32_t(sq / kStages - 1) & 1u, failed);
+        if (!ok) break;
+        const int64_t j0 = j_lo + int64_t(t) * kKT;
+        int ngroups = 0;
+        for (int gi = 0; gi < kKT / kGroup; ++gi)
+          if (j0 + gi * kGroup <= tq_last) ++ngroups;
+        const uint32_t bar = smem_u32(&sm.bar_full[slot]);
+        mbar_expect_tx(bar, uint32_t(ngroups) * 2u * kGroupBytes);
+        for (int gi = 0; gi < ngroups; ++gi) {
+          const int64_t j = j0 + gi * kGroup;
+          const uint32_t dst = sKV[slot] + uint32_t(gi) * kGroupBytes;
+          if (j >= p.n0) {      // the call's own rows
+            const CUtensorMap *m = is_v ? &cm.v : &cm.k;
+            tma_load_4d(dst, m, 0, g, int(j - p.n0), lrel * p.B + b, bar);
+            tma_load_4d(dst + kBoxBytes, m, 64, g, int(j - p.n0), lrel * p.B + b, bar);
+          } else {              // ring rows: a 16-token group never wraps (ring sizes are multiples of 16 where rings wrap)
+            const CUtensorMap *m = is_v ? ringV : ringK;
+            const int y = int(unit_rows + size_t(uint64_t(j) % cap));
+            tma_load_2d(dst, m, 0, y, bar);
+            tma_load_2d(dst + kBoxBytes, m, 64, y, bar);
+          }
         }
       }
     }
-    cp_async_wait<1>();
-    fence_async_smem();
-    tc_fence_before();
-    __syncthreads();
-    if (tid == 0) {
-      tc_fence_after();
-      issue_mma(tmem + 128, sP, sV[t & 1], true, o_init);
-      if (t + 1 < n_wtiles) issue_mma(tmem, sQ, sK[(t + 1) & 1], false, false);
-      mma_commit(bar);
-    }
-    o_init = true;
   }
-  if (n_wtiles > 0) wait_mma();
-  cp_async_wait<0>();
-  __syncthreads();   // every thread's copies into the Q tile have landed before rows are overwritten
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
 
-  // ---- linear part --------------------------------------------------------------------------------------
+  // =========================== linear part: the whole CTA in step ===========================
+  // (no early exits from here on: every thread passes the same __syncthreads; after a time-out the waits return
+  // at once and the results are discarded)
   const bool linear = ld.evicts && tq_last >= w;
+  bool o_init = n_tiles > 0;   // O_X holds a valid accumulation (uniform over the CTA)
+  uint32_t lin_phase = 0;
+  const int mma_tid = kMmaWarp * 32;
+  auto wait_lin = [&]() {
+    mbar_wait(smem_u32(&sm.bar_lin), lin_phase & 1u, failed);
+    ++lin_phase;
+    tc_fence_after();
+  };
   if (linear) {
-    const float M = fmaxf(m_ref, 0.f);
-    const float fw = m_ref == -CUDART_INF_F ? 0.f : ex2(m_ref - M);
-    const float fl = ex2(-M);
-    if (o_init && !failed && __any_sync(0xffffffffu, fw != 1.f)) scale_o(fw);
-    l_sum *= fw;
-    // phi(q) of this thread's row, times 2^-m*, as bf16 (kept packed in registers and written to the Q tile)
-    uint32_t phq[kD / 2];
-    {
-      const bf16 *qrow = reinterpret_cast<const bf16 *>(p.q) +
-                         ((seq + size_t(p.c0 + tok0 + (tok_r < ntok ? tok_r : 0))) * p.H + p.heads_of[g * G + hh]) * kD;
+    const int64_t folded = p.n0 + p.c0 - w;   // tokens below this index are in S, z at the start of the chunk
+    uint32_t phq[kD / 2];                      // phi(q) 2^-m* of this row, packed bf16
+    if (activeX) {
+      const float M = fmaxf(m_ref, 0.f);
+      const float fw = m_ref == -CUDART_INF_F ? 0.f : ex2(m_ref - M);
+      const float fl = ex2(-M);
+      if (o_init && __any_sync(0xffffffffu, fw != 1.f)) scale_o(fw);
+      l_sum *= fw;
 #pragma unroll
       for (int i = 0; i < kD / 8; ++i) {
         const uint4 v4 = *reinterpret_cast<const uint4 *>(qrow + i * 8);
@@ -372,93 +489,93 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_attn_tc_kernel(const Pref
         sum += ex2((__uint_as_float(phq[i] << 16) - mx) * kLog2e) + ex2((__uint_as_float(phq[i] & 0xffff0000u) - mx) * kLog2e);
       const float sc = fl * __frcp_rn(sum);
 #pragma unroll
-      for (int i = 0; i < kD / 2; ++i) {
-        const __nv_bfloat162 h2 = __floats2bfloat162_rn(ex2((__uint_as_float(phq[i] << 16) - mx) * kLog2e) * sc,
-                                                        ex2((__uint_as_float(phq[i] & 0xffff0000u) - mx) * kLog2e) * sc);
-        phq[i] = *reinterpret_cast<const uint32_t *>(&h2);
-      }
+      for (int i = 0; i < kD / 2; ++i)
+        phq[i] = pack_bf16x2(ex2((__uint_as_float(phq[i] << 16) - mx) * kLog2e) * sc,
+                             ex2((__uint_as_float(phq[i] & 0xffff0000u) - mx) * kLog2e) * sc);
 #pragma unroll
       for (int c = 0; c < 16; ++c)
-        *reinterpret_cast<uint4 *>(sm.q + sw128(row, c)) = make_uint4(phq[c * 4], phq[c * 4 + 1], phq[c * 4 + 2], phq[c * 4 + 3]);
+        *reinterpret_cast<uint4 *>(sm.q[X] + sw128(row, c)) = make_uint4(phq[c * 4], phq[c * 4 + 1], phq[c * 4 + 2], phq[c * 4 + 3]);
     }
     const int ub = b * p.Hkv + g;
-    const int64_t folded = p.n0 + p.c0 - w;   // tokens below this index are in S, z at the start of the chunk
-    if (folded > 0) {
-      // inter-chunk: O += (phi(Q) 2^-m*) S with a bf16 copy of the state as the MN-major B tile
+    if (folded > 0 && tid < kSoftmaxThreads) {
+      // bf16 copy of the state as the MN-major B tile of the inter-chunk product
       const float *Sg = reinterpret_cast<const float *>(p.ws + ld.S) + size_t(ub) * kD * kD;
-      const float *zg = reinterpret_cast<const float *>(p.ws + ld.z) + size_t(ub) * kD;
 #pragma unroll 4
-      for (int i = 0; i < kD * 16 / kThreads; ++i) {
-        const int id = tid + kThreads * i;
+      for (int i = 0; i < kD * 16 / kSoftmaxThreads; ++i) {
+        const int id = tid + kSoftmaxThreads * i;
         const int r = id >> 4, c = id & 15;
         const float4 f0 = *reinterpret_cast<const float4 *>(Sg + size_t(r) * kD + c * 8);
         const float4 f1 = *reinterpret_cast<const float4 *>(Sg + size_t(r) * kD + c * 8 + 4);
-        const __nv_bfloat162 h0 = __floats2bfloat162_rn(f0.x, f0.y), h1 = __floats2bfloat162_rn(f0.z, f0.w);
-        const __nv_bfloat162 h2 = __floats2bfloat162_rn(f1.x, f1.y), h3 = __floats2bfloat162_rn(f1.z, f1.w);
-        *reinterpret_cast<uint4 *>(sm.v[0] + sw128(r, c)) =
-            make_uint4(*reinterpret_cast<const uint32_t *>(&h0), *reinterpret_cast<const uint32_t *>(&h1),
-                       *reinterpret_cast<const uint32_t *>(&h2), *reinterpret_cast<const uint32_t *>(&h3));
+        *reinterpret_cast<uint4 *>(sm.kv[0] + sw128(r, c)) =
+            make_uint4(pack_bf16x2(f0.x, f0.y), pack_bf16x2(f0.z, f0.w), pack_bf16x2(f1.x, f1.y), pack_bf16x2(f1.z, f1.w));
       }
-      sm.z[tid] = zg[tid];
-      fence_async_smem();
-      tc_fence_before();
-      __syncthreads();
-      if (tid == 0) {
-        tc_fence_after();
-        issue_mma(tmem + 128, sQ, sV[0], true, o_init);
-        mma_commit(bar);
-      }
-      o_init = true;
-      float dot = 0.f;
-#pragma unroll
-      for (int i = 0; i < kD / 2; ++i)
-        dot += __uint_as_float(phq[i] << 16) * sm.z[2 * i] + __uint_as_float(phq[i] & 0xffff0000u) * sm.z[2 * i + 1];
-      l_sum += dot;
-      wait_mma();
-    } else {
-      fence_async_smem();
-      __syncthreads();
+      if (tid < kD) sm.z[tid] = (reinterpret_cast<const float *>(p.ws + ld.z) + size_t(ub) * kD)[tid];
     }
-    // intra-chunk: delayed tokens of this chunk up to the tile's last token, 128 at a time
+    fence_async_smem();
+    tc_fence_before();
+    __syncthreads();
+    if (folded > 0) {
+      if (tid == mma_tid) {
+        tc_fence_after();
+        issue_mma(tmem + 256, sQ[0], sKV[0], true, o_init);
+        if (hasB) issue_mma(tmem + 384, sQ[1], sKV[0], true, o_init);
+        mma_commit(smem_u32(&sm.bar_lin));
+      }
+      if (activeX) {
+        float dot = 0.f;
+#pragma unroll
+        for (int i = 0; i < kD / 2; ++i)
+          dot += __uint_as_float(phq[i] << 16) * sm.z[2 * i] + __uint_as_float(phq[i] & 0xffff0000u) * sm.z[2 * i + 1];
+        l_sum += dot;
+      }
+      wait_lin();
+      o_init = true;
+    }
+    // intra-chunk: delayed tokens of this chunk up to the CTA's last token, 128 at a time
     const int i_lo = folded < 0 ? int(-folded < int64_t(p.C) ? -folded : int64_t(p.C)) : 0;
     const int i_hi = tok0 + ntok - 1;
-    const int tl = tok0 + tok_r;   // chunk-relative token of this row
     const float *pkp = p.phik + size_t(u) * p.Cmax * kD;
+    const bf16 *ringV = reinterpret_cast<const bf16 *>(p.ws + ld.ringV) + unit_rows * kD;
+    const bf16 *callV = reinterpret_cast<const bf16 *>(p.v) + (seq * p.Hkv + g) * kD;
+    const int64_t call_stride = int64_t(p.Hkv) * kD;
     for (int i0 = i_lo & ~(kKT - 1); i0 <= i_hi; i0 += kKT) {
-      // phi(K') tile (fp32 scratch -> bf16, K-major) and the delayed tokens' V rows (MN-major)
+      if (tid < kSoftmaxThreads) {
+        // phi(K') tile (fp32 scratch -> bf16, K-major) and the delayed tokens' V rows (MN-major)
 #pragma unroll 4
-      for (int i = 0; i < kKT * 16 / kThreads; ++i) {
-        const int id = tid + kThreads * i;
-        const int r = id >> 4, c = id & 15;
-        const int ii = i0 + r;
-        uint4 pkd = make_uint4(0u, 0u, 0u, 0u);
-        if (ii >= i_lo && ii <= i_hi) {
-          const float4 f0 = *reinterpret_cast<const float4 *>(pkp + size_t(ii) * kD + c * 8);
-          const float4 f1 = *reinterpret_cast<const float4 *>(pkp + size_t(ii) * kD + c * 8 + 4);
-          const __nv_bfloat162 h0 = __floats2bfloat162_rn(f0.x, f0.y), h1 = __floats2bfloat162_rn(f0.z, f0.w);
-          const __nv_bfloat162 h2 = __floats2bfloat162_rn(f1.x, f1.y), h3 = __floats2bfloat162_rn(f1.z, f1.w);
-          pkd = make_uint4(*reinterpret_cast<const uint32_t *>(&h0), *reinterpret_cast<const uint32_t *>(&h1),
-                           *reinterpret_cast<const uint32_t *>(&h2), *reinterpret_cast<const uint32_t *>(&h3));
+        for (int i = 0; i < kKT * 16 / kSoftmaxThreads; ++i) {
+          const int id = tid + kSoftmaxThreads * i;
+          const int r = id >> 4, c = id & 15;
+          const int ii = i0 + r;
+          const bool valid = ii >= i_lo && ii <= i_hi;
+          uint4 pkd = make_uint4(0u, 0u, 0u, 0u);
+          if (valid) {
+            const float4 f0 = *reinterpret_cast<const float4 *>(pkp + size_t(ii) * kD + c * 8);
+            const float4 f1 = *reinterpret_cast<const float4 *>(pkp + size_t(ii) * kD + c * 8 + 4);
+            pkd = make_uint4(pack_bf16x2(f0.x, f0.y), pack_bf16x2(f0.z, f0.w), pack_bf16x2(f1.x, f1.y), pack_bf16x2(f1.z, f1.w));
+          }
+          *reinterpret_cast<uint4 *>(sm.kv[1] + sw128(r, c)) = pkd;
+          const int64_t jj = valid ? p.n0 + p.c0 - w + ii : 0;
+          const bool from_call = jj >= p.n0;
+          const bf16 *src = from_call ? callV + size_t(jj - p.n0) * call_stride : ringV + size_t(uint64_t(jj) % cap) * kD;
+          cp_async16(sKV[2] + sw128(r, c), src + c * 8, valid);
         }
-        *reinterpret_cast<uint4 *>(sm.k[0] + sw128(r, c)) = pkd;
-        const bool valid = ii >= i_lo && ii <= i_hi;
-        const int64_t jj = valid ? p.n0 + p.c0 - w + ii : 0;
-        const bool from_call = jj >= p.n0;
-        const bf16 *src = from_call ? callV + size_t(jj - p.n0) * call_stride : ringV + size_t(uint32_t(jj) % cap) * kD;
-        cp_async16(sV[1] + sw128(r, c), src + c * 8, valid);
+        cp_async_commit();
+        cp_async_wait_all();
       }
-      cp_async_commit();
-      cp_async_wait<0>();
       fence_async_smem();
       tc_fence_before();
       __syncthreads();
-      if (tid == 0) {
+      if (tid == mma_tid) {
         tc_fence_after();
-        issue_mma(tmem, sQ, sK[0], false, false);   // C = (phi(Q) 2^-m*) phi(K')^T
-        mma_commit(bar);
+        issue_mma(tmem, sQ[0], sKV[1], false, false);   // C_X = (phi(Q_X) 2^-m*) phi(K')^T
+        if (hasB) issue_mma(tmem + 128, sQ[1], sKV[1], false, false);
+        mma_commit(smem_u32(&sm.bar_lin));
       }
-      wait_mma();
-      if (!failed) {
+      wait_lin();
+      if (activeX) {
+        // C row -> bf16, masked to delayed tokens j' <= i of this row (the values already carry 2^-m*)
+        float sum0 = 0.f, sum1 = 0.f;
+        const int lo = i_lo - i0, hi = tl - i0;
 #pragma unroll 1
         for (int c0 = 0; c0 < kKT; c0 += 32) {
           uint32_t r[32];
@@ -468,42 +585,42 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_attn_tc_kernel(const Pref
             uint32_t pk[4];
 #pragma unroll
             for (int e = 0; e < 4; ++e) {
-              float pv[2];
-#pragma unroll
-              for (int z2 = 0; z2 < 2; ++z2) {
-                const int i = q4 * 8 + e * 2 + z2;
-                const int ii = i0 + c0 + i;
-                pv[z2] = (ii <= tl && ii >= i_lo) ? __uint_as_float(r[i]) : 0.f;
-              }
-              const __nv_bfloat162 h2 = __floats2bfloat162_rn(pv[0], pv[1]);
-              l_sum += __low2float(h2) + __high2float(h2);
-              pk[e] = *reinterpret_cast<const uint32_t *>(&h2);
+              const int i = c0 + q4 * 8 + e * 2;
+              const float a0 = (i >= lo && i <= hi) ? __uint_as_float(r[i - c0]) : 0.f;
+              const float a1 = (i + 1 >= lo && i + 1 <= hi) ? __uint_as_float(r[i + 1 - c0]) : 0.f;
+              pk[e] = pack_bf16x2(a0, a1);
+              sum0 += __uint_as_float(pk[e] << 16);
+              sum1 += __uint_as_float(pk[e] & 0xffff0000u);
             }
-            *reinterpret_cast<uint4 *>(sm.p + sw128(row, (c0 >> 3) + q4)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+            *reinterpret_cast<uint4 *>(sm.p[X] + sw128(row, (c0 >> 3) + q4)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
           }
         }
+        l_sum += sum0 + sum1;
       }
       fence_async_smem();
       tc_fence_before();
       __syncthreads();
-      if (tid == 0) {
+      if (tid == mma_tid) {
         tc_fence_after();
-        issue_mma(tmem + 128, sP, sV[1], true, o_init);
-        mma_commit(bar);
+        issue_mma(tmem + 256, sP[0], sKV[2], true, o_init);
+        if (hasB) issue_mma(tmem + 384, sP[1], sKV[2], true, o_init);
+        mma_commit(smem_u32(&sm.bar_lin));
       }
+      wait_lin();
       o_init = true;
-      wait_mma();
     }
   }
 
   // ---- shared normaliser and store: one contiguous 256-byte row per thread ------------------------------------
   __syncthreads();
-  if (sm.failed) {
+  const bool bad = sm.failed != 0;
+  if (bad) {
     if (tid == 0) atomicExch(&p.ctl->status, kDevWaitTimeout);
-  } else if (o_init) {
-    const bool store = tok_r < ntok;   // the TMEM loads below are warp-collective: only the store is per row
+  } else if (activeX && o_init) {
+    const bool store = tok_r < ntokX;   // the TMEM loads below are warp-collective: only the store is per row
     const float inv = store ? 1.0f / l_sum : 0.f;
-    bf16 *op = reinterpret_cast<bf16 *>(p.out) + ((seq + size_t(p.c0 + tok0 + (store ? tok_r : 0))) * p.H + p.heads_of[g * G + hh]) * kD;
+    bf16 *op = reinterpret_cast<bf16 *>(p.out) +
+               ((seq + size_t(p.c0 + (store ? tl : tok0))) * p.H + p.heads_of[g * G + hh]) * kD;
 #pragma unroll 1
     for (int c0 = 0; c0 < kD; c0 += 32) {
       uint32_t r[32];
@@ -512,38 +629,80 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_attn_tc_kernel(const Pref
       for (int q4 = 0; q4 < 4; ++q4) {
         uint32_t pk[4];
 #pragma unroll
-        for (int e = 0; e < 4; ++e) {
-          const __nv_bfloat162 h2 = __floats2bfloat162_rn(__uint_as_float(r[q4 * 8 + e * 2]) * inv, __uint_as_float(r[q4 * 8 + e * 2 + 1]) * inv);
-          pk[e] = *reinterpret_cast<const uint32_t *>(&h2);
-        }
+        for (int e = 0; e < 4; ++e)
+          pk[e] = pack_bf16x2(__uint_as_float(r[q4 * 8 + e * 2]) * inv, __uint_as_float(r[q4 * 8 + e * 2 + 1]) * inv);
         if (store) *reinterpret_cast<uint4 *>(op + c0 + q4 * 8) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
       }
     }
   }
   tc_fence_before();
   __syncthreads();
-  if (warp == 0) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 256;" ::"r"(tmem) : "memory");
+  if (warp == 0) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 512;" ::"r"(tmem) : "memory");
 }
 
 }  // namespace
 
-bool prefill_attn_tc_supported(const glide_ctx *ctx) {
-  return ctx->cfg.io_dtype == GLIDE_BF16 && ctx->cfg.head_dim == kD;
+// The kernel needs the ring descriptors made for the tensor-core decode kernels, 16-token TMA boxes that never
+// straddle the call boundary (tokens absorbed so far a multiple of 16) or a ring wrap (ring sizes of evicting
+// layers multiples of 16).
+bool prefill_attn_tc_supported(const glide_ctx *ctx, int layer_begin, int layer_count, int64_t n0) {
+  if (ctx->cfg.io_dtype != GLIDE_BF16 || ctx->cfg.head_dim != kD || ctx->decode_kind < 1) return false;
+  if (n0 % kGroup != 0 || ctx->prefill_chunk % kGroup != 0) return false;
+  for (int l = layer_begin; l < layer_begin + layer_count; ++l) {
+    const LayerDev &ld = ctx->layers[size_t(l)];
+    if (ld.cap > 0 && ld.evicts && ld.cap % kGroup != 0) return false;
+  }
+  return true;
 }
 
+namespace {
+typedef CUresult (*EncodeFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *, const cuuint64_t *,
+                             const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave, CUtensorMapSwizzle,
+                             CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+EncodeFn tensor_map_encoder() {
+  static EncodeFn fn = [] {
+    void *f = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &f, cudaEnableDefault, &q) != cudaSuccess || !f ||
+        q != cudaDriverEntryPointSuccess) {
+      cudaGetLastError();
+      f = nullptr;
+    }
+    return reinterpret_cast<EncodeFn>(f);
+  }();
+  return fn;
+}
+}  // namespace
+
 int launch_prefill_attn_tc(glide_ctx *ctx, const PrefillParams &p, cudaStream_t stream) {
+  EncodeFn encode = tensor_map_encoder();
+  if (!encode) return GLIDE_ERR_CUDA;
+  CallMaps cm;
+  {
+    const cuuint64_t dims[4] = {cuuint64_t(kD), cuuint64_t(p.Hkv), cuuint64_t(p.T), cuuint64_t(p.layer_count) * cuuint64_t(p.B)};
+    const cuuint64_t strides[3] = {cuuint64_t(kD) * 2, cuuint64_t(p.Hkv) * kD * 2, cuuint64_t(p.T) * p.Hkv * kD * 2};
+    const cuuint32_t box[4] = {64, 1, kGroup, 1};
+    const cuuint32_t estr[4] = {1, 1, 1, 1};
+    for (int kv = 0; kv < 2; ++kv) {
+      CUresult r = encode(kv == 0 ? &cm.k : &cm.v, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void *>(kv == 0 ? p.k : p.v), dims,
+                          strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                          CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+      if (r != CUDA_SUCCESS) return GLIDE_ERR_UNSUPPORTED;
+    }
+  }
+  const CUtensorMap *ring_maps = reinterpret_cast<const CUtensorMap *>(ctx->ws + ctx->off_tmaps);
   const int64_t units = int64_t(p.layer_count) * p.B * p.Hkv;
   auto launch = [&](auto gg) -> int {
     constexpr int G = decltype(gg)::value;
-    constexpr int TOK = kRows / G;
+    constexpr int TOKC = 2 * kRows / G;
     auto kern = prefill_attn_tc_kernel<G>;
     const size_t smem = sizeof(Smem) + 1024;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem)) != cudaSuccess) {
       cudaGetLastError();
       return GLIDE_ERR_CUDA;
     }
-    const int64_t blocks = units * ((p.C + TOK - 1) / TOK);
-    kern<<<unsigned(blocks), kThreads, smem, stream>>>(p);
+    const int64_t blocks = units * ((p.C + TOKC - 1) / TOKC);
+    kern<<<unsigned(blocks), kThreads, smem, stream>>>(p, ring_maps, cm);
     return cudaGetLastError() == cudaSuccess ? GLIDE_OK : GLIDE_ERR_CUDA;
   };
   switch (ctx->G) {

@@ -149,3 +149,17 @@ def test_contexts_with_different_schedules_coexist():
             g.glide_decode_step(q, k, v, out)
             ref = st.decode(to_np(q), to_np(k), to_np(v))
             check_outputs(out, ref, BF16, f"L={len(w)} step {t}")
+
+
+@pytest.mark.parametrize("G", [1, 2, 4, 8])
+@pytest.mark.parametrize("chunk", [96, 256])
+def test_bf16_prefill_tcgen05_aligned_calls(G, chunk):
+    # the tcgen05 kernel runs when every call starts at a multiple of 16 tokens and wrapping rings are multiples
+    # of 16: windows below, at and above the 128-key tile, a ring that wraps several times, a never-evicting
+    # layer whose ring size is not a multiple of 16, a purely linear layer; one and two row tiles per CTA
+    run_case([0, 16, 64, 128, 304, 1 << 20], 2, 2 * G, 2, 128, BF16, [144, 256, 48, 16], 5, amp=128 ** -0.5 * 4,
+             seed=chunk + G, prefill_chunk=chunk, prefill_impl=2)
+
+
+def test_bf16_prefill_tcgen05_large_logits():
+    run_case([48, 208], 1, 8, 2, 128, BF16, [256], 6, amp=128 ** -0.5 * 12, prefill_impl=2)
