@@ -43,7 +43,7 @@ constexpr uint32_t kBoxBytes = 16384;
 constexpr uint32_t kGroupBytes = kGroup * 128;   // one 16-token box of 64 columns
 constexpr uint32_t kWaitLimit = 1u << 20;
 constexpr float kLazy = 8.0f;         // rescale O only when the row maximum grows by more than 2^8
-constexpr int kStages = 3;
+constexpr int kStages = 5;
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return uint32_t(__cvta_generic_to_shared(p)); }
 // byte offset of 16-byte chunk c16 (0..15) of row `row` inside a [2][128][64] bf16 tile with 128-byte swizzle
@@ -101,6 +101,21 @@ __device__ __forceinline__ void issue_mma(uint32_t tmem_d, uint32_t a_tile, uint
     mma_f16(tmem_d, adesc, bdesc, idesc, (accumulate || ks > 0) ? 1u : 0u);
   }
 }
+// the same product with the A operand in TMEM: lane = row, 32-bit column c = elements 2c (low half) and 2c+1 of
+// the row, 8 columns per k16 step; B MN-major in shared memory
+__device__ __forceinline__ void issue_mma_ts(uint32_t tmem_d, uint32_t tmem_a, uint32_t b_tile, bool accumulate) {
+  const uint32_t idesc = make_idesc(true);
+#pragma unroll
+  for (int ks = 0; ks < 8; ++ks) {
+    const uint64_t bdesc = make_desc(b_tile + ks * 2048, kBoxBytes, 1024);
+    const uint32_t acc = (accumulate || ks > 0) ? 1u : 0u;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}" ::"r"(tmem_d),
+        "r"(tmem_a + ks * 8), "l"(bdesc), "r"(idesc), "r"(acc)
+        : "memory");
+  }
+}
 __device__ __forceinline__ void mma_commit(uint32_t bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
@@ -150,6 +165,19 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
       : "r"(taddr));
   asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 }
+// the same load without the wait: the registers are valid only after tmem_wait_ld()
+__device__ __forceinline__ void tmem_ld32_nowait(uint32_t taddr, uint32_t (&r)[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]), "=r"(r[9]),
+        "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]), "=r"(r[17]), "=r"(r[18]),
+        "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]),
+        "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr));
+}
+__device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32]) {
   asm volatile(
       "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
@@ -162,16 +190,35 @@ __device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32
   asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
 }
 
+#ifdef GLIDE_TC_PROFILE
+__device__ long long g_tc_prof[16];
+#define TC_MARK() long long tc_t_ = clock64(); long long tc_acc_[16] = {0,0,0,0,0,0,0,0,0,0,0,0,0,0,0,0}
+#define TC_ADD(i) do { long long n_ = clock64(); tc_acc_[i] += n_ - tc_t_; tc_t_ = n_; } while (0)
+#define TC_FLUSH(lo, hi) do { if (blockIdx.x == GLIDE_TC_PROFILE) for (int i_ = lo; i_ < hi; ++i_) atomicAdd(reinterpret_cast<unsigned long long *>(&g_tc_prof[i_]), (unsigned long long)tc_acc_[i_]); } while (0)
+#else
+#define TC_MARK() do { } while (0)
+#define TC_ADD(i) do { } while (0)
+#define TC_FLUSH(lo, hi) do { } while (0)
+#endif
+
+// (no wait: the caller issues tmem_wait_st() once after its last store)
+__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&r)[16]) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};" ::"r"(taddr),
+      "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]), "r"(r[9]), "r"(r[10]),
+      "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
+      : "memory");
+}
+
 struct Smem {
   unsigned char q[2][kTileBytes];        // Q_A, Q_B; later phi(Q) 2^-m*
-  unsigned char p[2][kTileBytes];        // P_A, P_B (or C): A operand of the second MMA
   unsigned char kv[kStages][kTileBytes]; // K and V tiles in turn; linear part: bf16 state, phi(K') tile, V' tile
   float z[kD];
   uint64_t bar_full[kStages];            // TMA bytes of the buffer have landed
   uint64_t bar_free[kStages];            // the MMAs that read the buffer have completed
   uint64_t bar_q[2];                     // Q_X staged (128 arrivals)
   uint64_t bar_s[2];                     // S_X of the current tile is in TMEM
-  uint64_t bar_p[2];                     // P_X of the current tile is in shared memory (128 arrivals)
+  uint64_t bar_p[2];                     // P_X of the current tile is in TMEM (128 arrivals)
   uint64_t bar_done;                     // every window MMA has completed
   uint64_t bar_lin;                      // linear part: the MMAs issued so far have completed
   uint32_t tmem_base;
@@ -211,6 +258,7 @@ prefill_attn_tc_kernel(const PrefillParams p, const CUtensorMap *ring_maps, cons
   const size_t unit_rows = (size_t(b) * p.Hkv + g) * size_t(ld.cap);
   const size_t seq = (size_t(lrel) * p.B + b) * size_t(p.T);
   volatile int *failed = &sm.failed;
+  TC_MARK();
 
   // a time-out recorded by an earlier CTA ends the launch quickly
   if (*reinterpret_cast<volatile int32_t *>(&p.ctl->status) == kDevWaitTimeout) return;
@@ -250,8 +298,8 @@ prefill_attn_tc_kernel(const PrefillParams p, const CUtensorMap *ring_maps, cons
   tc_fence_after();
   const uint32_t tmem = sm.tmem_base;
   const uint32_t sQ[2] = {smem_u32(sm.q[0]), smem_u32(sm.q[1])};
-  const uint32_t sP[2] = {smem_u32(sm.p[0]), smem_u32(sm.p[1])};
-  const uint32_t sKV[kStages] = {smem_u32(sm.kv[0]), smem_u32(sm.kv[1]), smem_u32(sm.kv[2])};
+  const uint32_t sKV0 = smem_u32(sm.kv[0]);
+  auto kv_addr = [&](int slot) { return sKV0 + uint32_t(slot) * kTileBytes; };
 
   // ---- softmax threads: per-row state that lives across the window and the linear part ----------------------
   const int X = (tid >> 7) & 1;                   // row tile of this thread (softmax warps only)
@@ -282,33 +330,37 @@ prefill_attn_tc_kernel(const PrefillParams p, const CUtensorMap *ring_maps, cons
   auto write_p = [&](auto masked, int lo, int hi, float mr, float scale) -> float {
     constexpr bool kMasked = decltype(masked)::value;
     float sum0 = 0.f, sum1 = 0.f;
-    unsigned char *prow = sm.p[X];
-#pragma unroll 1
+    uint32_t ra[32], rb[32];
+    tmem_ld32_nowait(tS, ra);
+#pragma unroll
     for (int c0 = 0; c0 < kKT; c0 += 32) {
-      uint32_t r[32];
-      tmem_ld32(tS + c0, r);
+      uint32_t (&r)[32] = ((c0 >> 5) & 1) ? rb : ra;
+      uint32_t pk[16];
+      tmem_wait_ld();
+      // the next 32 columns are on their way while these are turned into weights; the store below touches
+      // columns [c0/2, c0/2+16), which lie below c0+32 only when they have been read already
+      if (c0 + 32 < kKT) tmem_ld32_nowait(tS + c0 + 32, ((c0 >> 5) & 1) ? ra : rb);
 #pragma unroll
-      for (int q4 = 0; q4 < 4; ++q4) {
-        uint32_t pk[4];
-#pragma unroll
-        for (int e = 0; e < 4; ++e) {
-          const int i = q4 * 8 + e * 2;
-          float a0 = ex2(fmaf(__uint_as_float(r[i]), scale, -mr));
-          float a1 = ex2(fmaf(__uint_as_float(r[i + 1]), scale, -mr));
-          if (kMasked) {
-            if (c0 + i < lo || c0 + i > hi) a0 = 0.f;
-            if (c0 + i + 1 < lo || c0 + i + 1 > hi) a1 = 0.f;
-          }
-          pk[e] = pack_bf16x2(a0, a1);
-          sum0 += __uint_as_float(pk[e] << 16);          // the sum uses the weights as the tensor core sees them
-          sum1 += __uint_as_float(pk[e] & 0xffff0000u);
+      for (int e = 0; e < 16; ++e) {
+        const int i = e * 2;
+        float a0 = ex2(fmaf(__uint_as_float(r[i]), scale, -mr));
+        float a1 = ex2(fmaf(__uint_as_float(r[i + 1]), scale, -mr));
+        if (kMasked) {
+          if (c0 + i < lo || c0 + i > hi) a0 = 0.f;
+          if (c0 + i + 1 < lo || c0 + i + 1 > hi) a1 = 0.f;
         }
-        *reinterpret_cast<uint4 *>(prow + sw128(row, (c0 >> 3) + q4)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+        pk[e] = pack_bf16x2(a0, a1);
+        sum0 += __uint_as_float(pk[e] << 16);          // the sum uses the weights as the tensor core sees them
+        sum1 += __uint_as_float(pk[e] & 0xffff0000u);
       }
+      // P overwrites the S columns this thread has already consumed: keys c0..c0+31 -> columns c0/2..c0/2+15
+      tmem_st16(tS + (c0 >> 1), pk);
     }
+    tmem_wait_st();
     return sum0 + sum1;
   };
 
+  TC_ADD(7);
   // =========================== window part: warp-specialised ===========================
   if (tid < kSoftmaxThreads) {
     if (activeX) {
@@ -326,12 +378,14 @@ prefill_attn_tc_kernel(const PrefillParams p, const CUtensorMap *ring_maps, cons
       cp_async_wait_all();
       fence_async_smem();
       mbar_arrive(smem_u32(&sm.bar_q[X]));
+      TC_ADD(11);
 
       const int64_t tqX0 = tq0 + X * TOKT, tqX_last = tqX0 + ntokX - 1;
       bool o_written = false;   // a P V product has been accumulated into O_X (uniform over the row tile)
       for (int t = 0; t < n_tiles; ++t) {
         const bool got = mbar_wait(smem_u32(&sm.bar_s[X]), uint32_t(t) & 1u, failed);
         if (!__all_sync(0xffffffffu, got)) break;   // warp-uniform: the collectives below need every lane
+        TC_ADD(0);
         tc_fence_after();
         const int64_t j0 = j_lo + int64_t(t) * kKT;
         const bool interior = j0 + kKT - 1 <= tqX0 && j0 > tqX_last - w;
@@ -357,6 +411,7 @@ prefill_attn_tc_kernel(const PrefillParams p, const CUtensorMap *ring_maps, cons
           mx = fmaxf(mx, fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3])));
         }
         mx *= p.scale_log2;
+        TC_ADD(1);
         // lazy reference: move it (and rescale O, l) only when the maximum grows by more than 2^kLazy
         float f = 1.f;
         if (mx > m_ref + kLazy || (m_ref == -CUDART_INF_F && mx > -CUDART_INF_F)) {
@@ -364,18 +419,20 @@ prefill_attn_tc_kernel(const PrefillParams p, const CUtensorMap *ring_maps, cons
           m_ref = mx;
         }
         if (o_written && __any_sync(0xffffffffu, f != 1.f)) scale_o(f);
+        TC_ADD(2);
         l_sum *= f;
         const float mr = m_ref == -CUDART_INF_F ? 0.f : m_ref;
         if (interior) l_sum += write_p(IntTag<0>{}, lo, hi, mr, p.scale_log2);
         else l_sum += write_p(IntTag<1>{}, lo, hi, mr, p.scale_log2);
-        fence_async_smem();     // P is read by the tensor core (async proxy)
-        tc_fence_before();      // this thread's TMEM reads of S_X precede the MMA that overwrites it
+        tc_fence_before();      // this thread's TMEM accesses precede the MMAs that read P and overwrite S
         mbar_arrive(smem_u32(&sm.bar_p[X]));
+        TC_ADD(3);
         o_written = true;
       }
     }
     if (n_tiles > 0) mbar_wait(smem_u32(&sm.bar_done), 0u, failed);
     tc_fence_after();
+    TC_ADD(4);
   } else if (warp == kMmaWarp) {
     if (lane == 0 && n_tiles > 0) {
       bool ok = mbar_wait(smem_u32(&sm.bar_q[0]), 0u, failed);
@@ -383,10 +440,10 @@ prefill_attn_tc_kernel(const PrefillParams p, const CUtensorMap *ring_maps, cons
       if (ok) ok = mbar_wait(smem_u32(&sm.bar_full[0]), 0u, failed);   // K_0
       if (ok) {
         tc_fence_after();
-        issue_mma(tmem, sQ[0], sKV[0], false, false);
+        issue_mma(tmem, sQ[0], kv_addr(0), false, false);
         mma_commit(smem_u32(&sm.bar_s[0]));
         if (hasB) {
-          issue_mma(tmem + 128, sQ[1], sKV[0], false, false);
+          issue_mma(tmem + 128, sQ[1], kv_addr(0), false, false);
           mma_commit(smem_u32(&sm.bar_s[1]));
         }
         mma_commit(smem_u32(&sm.bar_free[0]));
@@ -396,16 +453,19 @@ prefill_attn_tc_kernel(const PrefillParams p, const CUtensorMap *ring_maps, cons
         const bool more = t + 1 < n_tiles;
         ok = mbar_wait(smem_u32(&sm.bar_full[seqV % kStages]), uint32_t(seqV / kStages) & 1u, failed);
         if (ok && more) ok = mbar_wait(smem_u32(&sm.bar_full[seqK % kStages]), uint32_t(seqK / kStages) & 1u, failed);
+        TC_ADD(12);
         for (int x = 0; x < 2 && ok; ++x) {
           if (x == 1 && !hasB) break;
           ok = mbar_wait(smem_u32(&sm.bar_p[x]), uint32_t(t) & 1u, failed);
           if (!ok) break;
+          TC_ADD(13);
           tc_fence_after();
-          issue_mma(tmem + 256 + x * 128, sP[x], sKV[seqV % kStages], true, t > 0);
+          issue_mma_ts(tmem + 256 + x * 128, tmem + x * 128, kv_addr(seqV % kStages), t > 0);
           if (more) {
-            issue_mma(tmem + x * 128, sQ[x], sKV[seqK % kStages], false, false);
+            issue_mma(tmem + x * 128, sQ[x], kv_addr(seqK % kStages), false, false);
             mma_commit(smem_u32(&sm.bar_s[x]));
           }
+          TC_ADD(14);
         }
         if (ok) {
           mma_commit(smem_u32(&sm.bar_free[seqV % kStages]));
@@ -415,30 +475,34 @@ prefill_attn_tc_kernel(const PrefillParams p, const CUtensorMap *ring_maps, cons
       if (ok) mma_commit(smem_u32(&sm.bar_done));
     }
   } else if (warp == kLoadWarp) {
-    if (lane == 0 && n_tiles > 0) {
+    // lane gi issues the two boxes (column halves) of token group gi of the tile: the address arithmetic of the
+    // eight groups runs in parallel instead of as one long dependent chain
+    if (n_tiles > 0) {
       const CUtensorMap *ringK = ring_maps + 3 * layer, *ringV = ringK + 1;
+      const int gi = lane;
       bool ok = true;
-      for (int sq = 0; sq < 2 * n_tiles && ok; ++sq) {
+      for (int sq = 0; sq < 2 * n_tiles; ++sq) {
         const int t = sq >> 1, slot = sq % kStages;
         const bool is_v = sq & 1;
         if (sq >= kStages) ok = mbar_wait(smem_u32(&sm.bar_free[slot]), uint32_t(sq / kStages - 1) & 1u, failed);
-        if (!ok) break;
+        if (!__all_sync(0xffffffffu, ok)) break;
         const int64_t j0 = j_lo + int64_t(t) * kKT;
-        int ngroups = 0;
-        for (int gi = 0; gi < kKT / kGroup; ++gi)
-          if (j0 + gi * kGroup <= tq_last) ++ngroups;
+        const int64_t left = tq_last - j0;                       // >= 0: the tile holds at least one valid token
+        const int ngroups = left >= kKT - 1 ? kKT / kGroup : int(left / kGroup) + 1;
         const uint32_t bar = smem_u32(&sm.bar_full[slot]);
-        mbar_expect_tx(bar, uint32_t(ngroups) * 2u * kGroupBytes);
-        for (int gi = 0; gi < ngroups; ++gi) {
+        if (lane == 0) mbar_expect_tx(bar, uint32_t(ngroups) * 2u * kGroupBytes);
+        __syncwarp();
+        if (gi < ngroups) {
           const int64_t j = j0 + gi * kGroup;
-          const uint32_t dst = sKV[slot] + uint32_t(gi) * kGroupBytes;
+          const uint32_t dst = kv_addr(slot) + uint32_t(gi) * kGroupBytes;
           if (j >= p.n0) {      // the call's own rows
             const CUtensorMap *m = is_v ? &cm.v : &cm.k;
             tma_load_4d(dst, m, 0, g, int(j - p.n0), lrel * p.B + b, bar);
             tma_load_4d(dst + kBoxBytes, m, 64, g, int(j - p.n0), lrel * p.B + b, bar);
           } else {              // ring rows: a 16-token group never wraps (ring sizes are multiples of 16 where rings wrap)
             const CUtensorMap *m = is_v ? ringV : ringK;
-            const int y = int(unit_rows + size_t(uint64_t(j) % cap));
+            const uint32_t slot_row = (j >> 32) == 0 ? uint32_t(j) % cap : uint32_t(uint64_t(j) % cap);
+            const int y = int(unit_rows + slot_row);
             tma_load_2d(dst, m, 0, y, bar);
             tma_load_2d(dst + kBoxBytes, m, 64, y, bar);
           }
@@ -449,6 +513,7 @@ prefill_attn_tc_kernel(const PrefillParams p, const CUtensorMap *ring_maps, cons
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
+  TC_ADD(8);
 
   // =========================== linear part: the whole CTA in step ===========================
   // (no early exits from here on: every thread passes the same __syncthreads; after a time-out the waits return
@@ -517,8 +582,8 @@ prefill_attn_tc_kernel(const PrefillParams p, const CUtensorMap *ring_maps, cons
     if (folded > 0) {
       if (tid == mma_tid) {
         tc_fence_after();
-        issue_mma(tmem + 256, sQ[0], sKV[0], true, o_init);
-        if (hasB) issue_mma(tmem + 384, sQ[1], sKV[0], true, o_init);
+        issue_mma(tmem + 256, sQ[0], kv_addr(0), true, o_init);
+        if (hasB) issue_mma(tmem + 384, sQ[1], kv_addr(0), true, o_init);
         mma_commit(smem_u32(&sm.bar_lin));
       }
       if (activeX) {
@@ -557,7 +622,7 @@ prefill_attn_tc_kernel(const PrefillParams p, const CUtensorMap *ring_maps, cons
           const int64_t jj = valid ? p.n0 + p.c0 - w + ii : 0;
           const bool from_call = jj >= p.n0;
           const bf16 *src = from_call ? callV + size_t(jj - p.n0) * call_stride : ringV + size_t(uint64_t(jj) % cap) * kD;
-          cp_async16(sKV[2] + sw128(r, c), src + c * 8, valid);
+          cp_async16(kv_addr(2) + sw128(r, c), src + c * 8, valid);
         }
         cp_async_commit();
         cp_async_wait_all();
@@ -567,8 +632,8 @@ prefill_attn_tc_kernel(const PrefillParams p, const CUtensorMap *ring_maps, cons
       __syncthreads();
       if (tid == mma_tid) {
         tc_fence_after();
-        issue_mma(tmem, sQ[0], sKV[1], false, false);   // C_X = (phi(Q_X) 2^-m*) phi(K')^T
-        if (hasB) issue_mma(tmem + 128, sQ[1], sKV[1], false, false);
+        issue_mma(tmem, sQ[0], kv_addr(1), false, false);   // C_X = (phi(Q_X) 2^-m*) phi(K')^T
+        if (hasB) issue_mma(tmem + 128, sQ[1], kv_addr(1), false, false);
         mma_commit(smem_u32(&sm.bar_lin));
       }
       wait_lin();
@@ -578,32 +643,28 @@ prefill_attn_tc_kernel(const PrefillParams p, const CUtensorMap *ring_maps, cons
         const int lo = i_lo - i0, hi = tl - i0;
 #pragma unroll 1
         for (int c0 = 0; c0 < kKT; c0 += 32) {
-          uint32_t r[32];
+          uint32_t r[32], pk[16];
           tmem_ld32(tS + c0, r);
 #pragma unroll
-          for (int q4 = 0; q4 < 4; ++q4) {
-            uint32_t pk[4];
-#pragma unroll
-            for (int e = 0; e < 4; ++e) {
-              const int i = c0 + q4 * 8 + e * 2;
-              const float a0 = (i >= lo && i <= hi) ? __uint_as_float(r[i - c0]) : 0.f;
-              const float a1 = (i + 1 >= lo && i + 1 <= hi) ? __uint_as_float(r[i + 1 - c0]) : 0.f;
-              pk[e] = pack_bf16x2(a0, a1);
-              sum0 += __uint_as_float(pk[e] << 16);
-              sum1 += __uint_as_float(pk[e] & 0xffff0000u);
-            }
-            *reinterpret_cast<uint4 *>(sm.p[X] + sw128(row, (c0 >> 3) + q4)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+          for (int e = 0; e < 16; ++e) {
+            const int i = c0 + e * 2;
+            const float a0 = (i >= lo && i <= hi) ? __uint_as_float(r[e * 2]) : 0.f;
+            const float a1 = (i + 1 >= lo && i + 1 <= hi) ? __uint_as_float(r[e * 2 + 1]) : 0.f;
+            pk[e] = pack_bf16x2(a0, a1);
+            sum0 += __uint_as_float(pk[e] << 16);
+            sum1 += __uint_as_float(pk[e] & 0xffff0000u);
           }
+          tmem_st16(tS + (c0 >> 1), pk);
         }
+        tmem_wait_st();
         l_sum += sum0 + sum1;
       }
-      fence_async_smem();
       tc_fence_before();
       __syncthreads();
       if (tid == mma_tid) {
         tc_fence_after();
-        issue_mma(tmem + 256, sP[0], sKV[2], true, o_init);
-        if (hasB) issue_mma(tmem + 384, sP[1], sKV[2], true, o_init);
+        issue_mma_ts(tmem + 256, tmem, kv_addr(2), o_init);
+        if (hasB) issue_mma_ts(tmem + 384, tmem + 128, kv_addr(2), o_init);
         mma_commit(smem_u32(&sm.bar_lin));
       }
       wait_lin();
@@ -613,6 +674,7 @@ prefill_attn_tc_kernel(const PrefillParams p, const CUtensorMap *ring_maps, cons
 
   // ---- shared normaliser and store: one contiguous 256-byte row per thread ------------------------------------
   __syncthreads();
+  TC_ADD(5);
   const bool bad = sm.failed != 0;
   if (bad) {
     if (tid == 0) atomicExch(&p.ctl->status, kDevWaitTimeout);
@@ -635,12 +697,26 @@ prefill_attn_tc_kernel(const PrefillParams p, const CUtensorMap *ring_maps, cons
       }
     }
   }
+  TC_ADD(6);
+  if (tid == 0) { TC_FLUSH(0, 12); }
+  if (tid == kMmaWarp * 32) { TC_FLUSH(12, 16); }
   tc_fence_before();
   __syncthreads();
   if (warp == 0) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 512;" ::"r"(tmem) : "memory");
 }
 
 }  // namespace
+
+#ifdef GLIDE_TC_PROFILE
+extern "C" int glide_debug_tc_profile(long long *out16, int reset) {
+  if (cudaMemcpyFromSymbol(out16, g_tc_prof, sizeof(long long) * 16) != cudaSuccess) return 6;
+  if (reset) {
+    long long z[16] = {};
+    if (cudaMemcpyToSymbol(g_tc_prof, z, sizeof(z)) != cudaSuccess) return 6;
+  }
+  return 0;
+}
+#endif
 
 // The kernel needs the ring descriptors made for the tensor-core decode kernels, 16-token TMA boxes that never
 // straddle the call boundary (tokens absorbed so far a multiple of 16) or a ring wrap (ring sizes of evicting
