@@ -27,6 +27,12 @@
  *           z = sum_E phi(k_j) (Sec. II recurrences), with decode() (one token,
  *           incremental fold) and prefill() (many tokens, explicit sums).
  *
+ * Alternative merges (appendix "(b) Retention-based SWA", the two hybrid equations): merge = 1 adds the
+ * separately normalised linear term over the evicted tokens and the separately normalised window softmax,
+ *   O_t = phi(q) S_{t-w} / phi(q) z_{t-w} + sum_W a_j v_j / sum_W a_j ;
+ * merge = 2 is the same sum with the state holding every token up to t (S_t, z_t).  A term whose token set is
+ * empty is taken as zero (the paper is silent; its quotient would be 0/0).  merge = 0 is the shared normaliser.
+ *
  * Parity pins (tests, CPU only): form A vs form B; w >= n vs a library causal
  * softmax attention; w = 0 vs matrix-form linear attention; the closed form for
  * q = k = 0; convexity; decode == prefill.  Random-input output VALUES have no
@@ -61,18 +67,38 @@ static double dot(const double *a, const double *b, int d) {
   return s;
 }
 
+/* The merge of the two parts.  numw/denw: window sums already multiplied by exp(-M); numl/denl: linear sums.
+ * merge 0: one shared normaliser (Sec. III-B); merge 1, 2: the sum of the two separately normalised terms
+ * (appendix hybrid equations), an empty term counting as zero. */
+static void combine(int merge, int d, double M, const double *numw, double denw, const double *numl,
+                    double denl, double *o) {
+  if (merge == 0) {
+    double eM = exp(-M);
+    for (int c = 0; c < d; ++c) o[c] = (numw[c] + eM * numl[c]) / (denw + eM * denl);
+    return;
+  }
+  for (int c = 0; c < d; ++c) {
+    double x = 0.0;
+    if (denw > 0.0) x += numw[c] / denw;
+    if (denl > 0.0) x += numl[c] / denl;
+    o[c] = x;
+  }
+}
+
 /* ------------------------------------------------------------------------- */
 /* Form B: brute force over the full history.                                 */
 /* q [T][H][d], k,v [T][Hkv][d], out [n_sel][H][d]; sel = positions to        */
 /* evaluate (NULL: all T positions, n_sel ignored).                           */
 /* ------------------------------------------------------------------------- */
-void glide_oracle_bruteforce(int64_t T, int H, int Hkv, int d, int64_t w, double scale,
+void glide_oracle_bruteforce(int64_t T, int H, int Hkv, int d, int64_t w, double scale, int merge,
                              const int32_t *q_to_kv, const double *q, const double *k,
                              const double *v, int64_t n_sel, const int64_t *sel, double *out) {
   int64_t count = sel ? n_sel : T;
+  int64_t delay = merge == 2 ? 0 : w; /* the linear term covers tokens j <= t - delay */
   double *phiq = (double *)malloc(sizeof(double) * d);
   double *phik = (double *)malloc(sizeof(double) * d);
   double *num = (double *)malloc(sizeof(double) * d);
+  double *numl = (double *)malloc(sizeof(double) * d);
   for (int64_t si = 0; si < count; ++si) {
     int64_t t = sel ? sel[si] : si;
     for (int h = 0; h < H; ++h) {
@@ -97,22 +123,23 @@ void glide_oracle_bruteforce(int64_t T, int H, int Hkv, int d, int64_t w, double
         for (int c = 0; c < d; ++c) num[c] += a * vj[c];
       }
       phi_softmax(qt, d, phiq);
-      double eM = exp(-M);
-      for (int64_t j = 0; j <= t - w; ++j) { /* empty when t < w */
+      double denl = 0.0;
+      for (int c = 0; c < d; ++c) numl[c] = 0.0;
+      for (int64_t j = 0; j <= t - delay; ++j) { /* empty when t < delay */
         const double *kj = k + ((size_t)j * Hkv + g) * d;
         const double *vj = v + ((size_t)j * Hkv + g) * d;
         phi_softmax(kj, d, phik);
-        double c_j = dot(phiq, phik, d) * eM;
-        den += c_j;
-        for (int c = 0; c < d; ++c) num[c] += c_j * vj[c];
+        double c_j = dot(phiq, phik, d);
+        denl += c_j;
+        for (int c = 0; c < d; ++c) numl[c] += c_j * vj[c];
       }
-      double *o = out + ((size_t)si * H + h) * d;
-      for (int c = 0; c < d; ++c) o[c] = num[c] / den;
+      combine(merge, d, M, num, den, numl, denl, out + ((size_t)si * H + h) * d);
     }
   }
   free(phiq);
   free(phik);
   free(num);
+  free(numl);
 }
 
 /* ------------------------------------------------------------------------- */
@@ -121,6 +148,8 @@ void glide_oracle_bruteforce(int64_t T, int H, int Hkv, int d, int64_t w, double
 typedef struct glide_oracle_cell {
   int H, Hkv, d;
   int64_t w;     /* window; ring capacity is exactly w (0: no ring) */
+  int merge;     /* 0 shared normaliser, 1 / 2 the appendix' sums of two normalised terms */
+  int64_t delay; /* a token enters the state `delay` steps after it arrives: w, or 0 for merge 2 */
   double scale;
   int32_t *q_to_kv;
   int64_t n;     /* tokens absorbed so far */
@@ -130,13 +159,15 @@ typedef struct glide_oracle_cell {
   double *z;     /* [Hkv][d] */
 } glide_oracle_cell;
 
-glide_oracle_cell *glide_oracle_cell_new(int H, int Hkv, int d, int64_t w, double scale,
+glide_oracle_cell *glide_oracle_cell_new(int H, int Hkv, int d, int64_t w, double scale, int merge,
                                          const int32_t *q_to_kv) {
   glide_oracle_cell *c = (glide_oracle_cell *)calloc(1, sizeof(*c));
   c->H = H;
   c->Hkv = Hkv;
   c->d = d;
   c->w = w;
+  c->merge = merge;
+  c->delay = merge == 2 ? 0 : w;
   c->scale = scale;
   c->q_to_kv = (int32_t *)malloc(sizeof(int32_t) * H);
   memcpy(c->q_to_kv, q_to_kv, sizeof(int32_t) * H);
@@ -185,14 +216,12 @@ static void append_token(glide_oracle_cell *c, int g, int64_t t, const double *k
                          const double *v, double *phik) {
   int d = c->d;
   int64_t w = c->w;
-  if (w == 0) { /* no ring: the token goes straight to the state */
-    fold(c, g, k, v, phik);
-    return;
-  }
+  if (c->delay == 0) fold(c, g, k, v, phik); /* no ring (w = 0) or the all-token state: token t enters the state now */
+  if (w == 0) return;
   int64_t slot = t % w;
   double *Kslot = c->Kr + ((size_t)g * w + slot) * d;
   double *Vslot = c->Vr + ((size_t)g * w + slot) * d;
-  if (t >= w) fold(c, g, Kslot, Vslot, phik); /* that slot holds token t-w, which leaves the window */
+  if (c->delay > 0 && t >= w) fold(c, g, Kslot, Vslot, phik); /* that slot holds token t-w, which leaves the window */
   memcpy(Kslot, k, sizeof(double) * d);
   memcpy(Vslot, v, sizeof(double) * d);
 }
@@ -221,16 +250,19 @@ static void readout(const glide_oracle_cell *c, int h, int64_t t, const double *
     den += a;
     for (int col = 0; col < d; ++col) num[col] += a * vj[col];
   }
-  /* linear part: phi(q) S and phi(q) z on the state that already holds E_t */
+  /* linear part: phi(q) S and phi(q) z on the state that already holds its token set */
   phi_softmax(qt, d, phiq);
   const double *S = c->S + (size_t)g * d * d;
   const double *z = c->z + (size_t)g * d;
-  double eM = exp(-M);
+  double *numl = (double *)malloc(sizeof(double) * d);
+  double denl = 0.0;
+  for (int col = 0; col < d; ++col) numl[col] = 0.0;
   for (int r = 0; r < d; ++r) {
-    den += eM * phiq[r] * z[r];
-    for (int col = 0; col < d; ++col) num[col] += eM * phiq[r] * S[(size_t)r * d + col];
+    denl += phiq[r] * z[r];
+    for (int col = 0; col < d; ++col) numl[col] += phiq[r] * S[(size_t)r * d + col];
   }
-  for (int col = 0; col < d; ++col) o[col] = num[col] / den;
+  combine(c->merge, d, M, num, den, numl, denl, o);
+  free(numl);
 }
 
 /* One decode step for the heads of KV head g only (used for threading). */
@@ -305,11 +337,12 @@ void glide_oracle_cell_prefill(glide_oracle_cell *c, int64_t T, const double *q,
                                const double *k, const double *v, int64_t n_sel,
                                const int64_t *sel, double *out) {
   int d = c->d, H = c->H, Hkv = c->Hkv;
-  int64_t w = c->w, n0 = c->n;
+  int64_t w = c->w, n0 = c->n, delay = c->delay;
   int64_t count = (sel == NULL && n_sel < 0) ? T : n_sel;
   double *phiq = (double *)malloc(sizeof(double) * d);
   double *phik = (double *)malloc(sizeof(double) * d);
   double *num = (double *)malloc(sizeof(double) * d);
+  double *numl = (double *)malloc(sizeof(double) * d);
 
 /* token j (absolute index) of KV head g: from the call if j >= n0, else from the ring */
 #define TOK_K(j, g) ((j) >= n0 ? k + ((size_t)((j)-n0) * Hkv + (g)) * d \
@@ -339,35 +372,35 @@ void glide_oracle_cell_prefill(glide_oracle_cell *c, int64_t T, const double *q,
         for (int col = 0; col < d; ++col) num[col] += a * vj[col];
       }
       phi_softmax(qt, d, phiq);
-      double eM = exp(-M);
-      /* evicted before the call started: held by the state */
+      /* in the state before the call started */
       const double *S = c->S + (size_t)g * d * d;
       const double *z = c->z + (size_t)g * d;
+      double denl = 0.0;
+      for (int col = 0; col < d; ++col) numl[col] = 0.0;
       for (int r = 0; r < d; ++r) {
-        den += eM * phiq[r] * z[r];
-        for (int col = 0; col < d; ++col) num[col] += eM * phiq[r] * S[(size_t)r * d + col];
+        denl += phiq[r] * z[r];
+        for (int col = 0; col < d; ++col) numl[col] += phiq[r] * S[(size_t)r * d + col];
       }
-      /* evicted since the call started: tokens max(0, n0-w) .. t-w, explicit */
-      int64_t e_lo = n0 - w;
+      /* entered the state since the call started: tokens max(0, n0-delay) .. t-delay, explicit */
+      int64_t e_lo = n0 - delay;
       if (e_lo < 0) e_lo = 0;
-      for (int64_t j = e_lo; j <= t - w; ++j) {
+      for (int64_t j = e_lo; j <= t - delay; ++j) {
         phi_softmax(TOK_K(j, g), d, phik);
-        double c_j = eM * dot(phiq, phik, d);
+        double c_j = dot(phiq, phik, d);
         const double *vj = TOK_V(j, g);
-        den += c_j;
-        for (int col = 0; col < d; ++col) num[col] += c_j * vj[col];
+        denl += c_j;
+        for (int col = 0; col < d; ++col) numl[col] += c_j * vj[col];
       }
-      double *o = out + ((size_t)si * H + h) * d;
-      for (int col = 0; col < d; ++col) o[col] = num[col] / den;
+      combine(c->merge, d, M, num, den, numl, denl, out + ((size_t)si * H + h) * d);
     }
   }
 
-  /* state by definition: fold tokens [max(0,n0-w), n0+T-w) in order ... */
+  /* state by definition: fold tokens [max(0,n0-delay), n0+T-delay) in order ... */
   int64_t n1 = n0 + T;
   for (int g = 0; g < Hkv; ++g) {
-    int64_t e_lo = n0 - w;
+    int64_t e_lo = n0 - delay;
     if (e_lo < 0) e_lo = 0;
-    for (int64_t j = e_lo; j < n1 - w; ++j) fold(c, g, TOK_K(j, g), TOK_V(j, g), phik);
+    for (int64_t j = e_lo; j < n1 - delay; ++j) fold(c, g, TOK_K(j, g), TOK_V(j, g), phik);
   }
   /* ... then the ring: slot s holds the newest token j < n1 with j mod w == s.
    * Only call tokens need writing; older survivors are already in place. */
@@ -388,6 +421,7 @@ void glide_oracle_cell_prefill(glide_oracle_cell *c, int64_t T, const double *q,
   free(phiq);
   free(phik);
   free(num);
+  free(numl);
 }
 
 /* Bookkeeping that the GPU path must reproduce bit-exactly. */

@@ -38,11 +38,11 @@ def _load():
         return _lib
     lib = ctypes.CDLL(build())
     lib.glide_oracle_bruteforce.argtypes = [
-        ctypes.c_int64, ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_int64, ctypes.c_double,
+        ctypes.c_int64, ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_int64, ctypes.c_double, ctypes.c_int,
         _i32p, _f64p, _f64p, _f64p, ctypes.c_int64, _i64p, _f64p]
     lib.glide_oracle_bruteforce.restype = None
     lib.glide_oracle_cell_new.argtypes = [ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_int64,
-                                          ctypes.c_double, _i32p]
+                                          ctypes.c_double, ctypes.c_int, _i32p]
     lib.glide_oracle_cell_new.restype = ctypes.c_void_p
     lib.glide_oracle_cell_free.argtypes = [ctypes.c_void_p]
     lib.glide_oracle_cell_free.restype = None
@@ -86,8 +86,10 @@ def max_threads() -> int:
     return int(_load().glide_oracle_max_threads())
 
 
-def bruteforce(q, k, v, w: int, scale: float, q_to_kv=None, sel: Optional[Sequence[int]] = None) -> np.ndarray:
-    """Form B: the defining sums over the full history.
+def bruteforce(q, k, v, w: int, scale: float, q_to_kv=None, sel: Optional[Sequence[int]] = None,
+               merge: int = 0) -> np.ndarray:
+    """Form B: the defining sums over the full history (merge: 0 shared normaliser, 1 / 2 the appendix' sums of
+    two separately normalised terms with the evicted-token / all-token state).
 
     q [T][H][d], k,v [T][Hkv][d] -> out [T or len(sel)][H][d] (float64)."""
     lib = _load()
@@ -97,12 +99,12 @@ def bruteforce(q, k, v, w: int, scale: float, q_to_kv=None, sel: Optional[Sequen
     m = default_q_to_kv(H, Hkv) if q_to_kv is None else np.ascontiguousarray(q_to_kv, dtype=np.int32)
     if sel is None:
         out = np.empty((T, H, d), dtype=np.float64)
-        lib.glide_oracle_bruteforce(T, H, Hkv, d, int(w), float(scale), _ptr(m, _i32p), _ptr(q), _ptr(k),
+        lib.glide_oracle_bruteforce(T, H, Hkv, d, int(w), float(scale), int(merge), _ptr(m, _i32p), _ptr(q), _ptr(k),
                                     _ptr(v), 0, None, _ptr(out))
     else:
         s = np.ascontiguousarray(sel, dtype=np.int64)
         out = np.empty((len(s), H, d), dtype=np.float64)
-        lib.glide_oracle_bruteforce(T, H, Hkv, d, int(w), float(scale), _ptr(m, _i32p), _ptr(q), _ptr(k),
+        lib.glide_oracle_bruteforce(T, H, Hkv, d, int(w), float(scale), int(merge), _ptr(m, _i32p), _ptr(q), _ptr(k),
                                     _ptr(v), len(s), _ptr(s, _i64p), _ptr(out))
     return out
 
@@ -110,11 +112,12 @@ def bruteforce(q, k, v, w: int, scale: float, q_to_kv=None, sel: Optional[Sequen
 class Cell:
     """Form A for one (layer, sequence): ring of the last w tokens + S/z state."""
 
-    def __init__(self, H: int, Hkv: int, d: int, w: int, scale: float, q_to_kv=None):
+    def __init__(self, H: int, Hkv: int, d: int, w: int, scale: float, q_to_kv=None, merge: int = 0):
         self._lib = _load()
+        self.merge = int(merge)
         self.H, self.Hkv, self.d, self.w, self.scale = H, Hkv, d, int(w), float(scale)
         self.q_to_kv = default_q_to_kv(H, Hkv) if q_to_kv is None else np.ascontiguousarray(q_to_kv, dtype=np.int32)
-        self._h = ctypes.c_void_p(self._lib.glide_oracle_cell_new(H, Hkv, d, int(w), float(scale),
+        self._h = ctypes.c_void_p(self._lib.glide_oracle_cell_new(H, Hkv, d, int(w), float(scale), int(merge),
                                                                    _ptr(self.q_to_kv, _i32p)))
 
     def __del__(self):
@@ -180,10 +183,11 @@ class Stack:
     decode: q [L][B][H][d], k,v [L][B][Hkv][d] -> out [L][B][H][d]
     prefill (layers lb..lb+lc): q [lc][B][T][H][d], k,v [lc][B][T][Hkv][d]."""
 
-    def __init__(self, windows: Sequence[int], batch: int, H: int, Hkv: int, d: int, scale: float, q_to_kv=None):
+    def __init__(self, windows: Sequence[int], batch: int, H: int, Hkv: int, d: int, scale: float, q_to_kv=None,
+                 merge: int = 0):
         self.L, self.B, self.H, self.Hkv, self.d = len(windows), batch, H, Hkv, d
         self.windows = [int(w) for w in windows]
-        self.cells = [[Cell(H, Hkv, d, w, scale, q_to_kv) for _ in range(batch)] for w in self.windows]
+        self.cells = [[Cell(H, Hkv, d, w, scale, q_to_kv, merge) for _ in range(batch)] for w in self.windows]
         flat = [c._h for row in self.cells for c in row]
         self._handles = (ctypes.c_void_p * len(flat))(*flat)
         self._lib = _load()
