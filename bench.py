@@ -134,7 +134,7 @@ def oracle_decode_rate(shape, steps: int, warmup: int, single_steps: int = 0):
     single_s = {}
     for w, layers in classes.items():
         l = layers[0]
-        stack = orc.Stack([w], 1, shape.n_q_heads, shape.n_kv_heads, shape.head_dim, scale)
+        stack = orc.Stack([w], 1, shape.n_q_heads, shape.n_kv_heads, shape.head_dim, scale, merge=KERNEL_KNOBS.get("merge", 0))
         # only the tokens that can still matter are absorbed one piece at a time
         piece = 2048
         for pos in range(0, shape.context, piece):
@@ -180,7 +180,8 @@ def run_reference(args, shape):
         "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup, "ms_per_step": step_s * 1e3,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
         "config": {"workload": shape.name, "batch": shape.batch, "context": shape.context,
-                   "sum_windows": sum(shape.windows), "timed_oracle_steps_per_layer_class": steps},
+                   "sum_windows": sum(shape.windows), "timed_oracle_steps_per_layer_class": steps,
+                   "merge": KERNEL_KNOBS.get("merge", 0)},
         "cpu_baseline": {"value": tok_s, "unit": "tokens/s", "cores": cores, "kind": "oracle", "sample": sample},
         "e2e": {"value": tok_s, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
@@ -220,6 +221,16 @@ def build_states(shape, n_replicas: int, extra_tokens: int, device):
             g.glide_import_state(l, shape.context, rk if cap else None, rv if cap else None, S, z)
         torch.cuda.synchronize()
     return ctxs, wl
+
+
+def decode_kernel_name(shape) -> str:
+    """The kernel glide_create selects for this shape and these knobs (see include/glide.h)."""
+    impl, merge = KERNEL_KNOBS.get("decode_impl", 0), KERNEL_KNOBS.get("merge", 0)
+    if shape.dtype == "f32" or impl == 2 or merge != 0:
+        return "glide_decode_kernel"
+    if shape.head_dim == 128 and impl in (0, 3):
+        return "glide_decode_stream_kernel"
+    return "glide_decode_mma_kernel"
 
 
 def max_over_ranks(values, dist, device):
@@ -376,10 +387,10 @@ def run_glide(args, shape):
                        "sum_windows": sum(shape.windows), "q_heads": H, "kv_heads": Hkv, "head_dim": d,
                        "l2": f"steps rotate over {n_rep} independent state copies ({n_rep * step_bytes / 1e6:.0f} MB per "
                              f"rotation > 126 MB L2); median of {reps} repetitions of K steps",
-                       "multi_gpu": "replicas only"},
+                       "multi_gpu": "replicas only", "merge": KERNEL_KNOBS.get("merge", 0)},
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                          "traffic": NCU_TRAFFIC_BYTES.get(shape.name), "peak_kind": f"of {peak_kind}",
-                         "kernel": "glide_decode_kernel", "algorithmic_bytes_per_launch": step_bytes,
+                         "kernel": decode_kernel_name(shape), "algorithmic_bytes_per_launch": step_bytes,
                          "frac_of_nominal_8TBps": achieved / 8000.0},
             "per_step_attention_latency_us": launch_s * 1e6,
             "step_latency_us": {"median": lat_us[len(lat_us) // 2], "p10": lat_us[len(lat_us) // 10],
@@ -529,10 +540,13 @@ def main():
     ap.add_argument("--decode-impl", type=int, default=0,
                     help="0 auto, 1 per-item tensor-core/TMA kernel, 2 CUDA-core kernel, 3 streaming tensor-core/TMA kernel")
     ap.add_argument("--prefill-impl", type=int, default=0, help="0 auto, 1 mma.sync, 2 tcgen05 + TMEM, 3 CUDA cores")
+    ap.add_argument("--merge", type=int, default=0,
+                    help="0 shared normaliser (the paper's default), 1 / 2 the appendix' sums of two normalised terms "
+                         "(evicted-token / all-token state; CUDA-core kernels)")
     args = ap.parse_args()
     shape = configs.ALL[args.workload]
     KERNEL_KNOBS.update(decode_chunk=args.decode_chunk, decode_state_splits=args.state_splits,
-                        decode_impl=args.decode_impl, prefill_impl=args.prefill_impl)
+                        decode_impl=args.decode_impl, prefill_impl=args.prefill_impl, merge=args.merge)
     if args.impl == "reference":
         run_reference(args, shape)
     else:

@@ -58,8 +58,14 @@ typedef enum { GLIDE_F32 = 0, GLIDE_BF16 = 1 } glide_dtype;
 typedef enum { GLIDE_PHI_SOFTMAX = 0 } glide_phi;
 
 /* How the window part and the linear part are merged (Sec. III-B "(+)"; appendix
- * "Retention-based SWA").  GLIDE_MERGE_SHARED is the shared normaliser above. */
-typedef enum { GLIDE_MERGE_SHARED = 0 } glide_merge;
+ * "Retention-based SWA").  GLIDE_MERGE_SHARED is the shared normaliser above.  The other two are the appendix'
+ * hybrid equations, a plain sum of two separately normalised terms:
+ *   GLIDE_MERGE_SUM_EVICTED   phi(q) S / phi(q) z over the evicted tokens  +  window softmax
+ *   GLIDE_MERGE_SUM_ALL       the same with a state that holds every token up to the current one (a token is
+ *                             folded when it arrives, not when it leaves the window)
+ * A term whose token set is empty counts as zero.  These two run on the CUDA-core kernels only (decode_impl and
+ * prefill_impl must be AUTO or FMA). */
+typedef enum { GLIDE_MERGE_SHARED = 0, GLIDE_MERGE_SUM_EVICTED = 1, GLIDE_MERGE_SUM_ALL = 2 } glide_merge;
 
 /* Decode kernel selection.  AUTO: for bf16 I/O the statically scheduled streaming tensor-core/TMA kernel
  * (head_dim 128) or the per-item tensor-core/TMA kernel; for fp32 I/O the CUDA-core kernel.  The others

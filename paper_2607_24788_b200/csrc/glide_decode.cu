@@ -37,6 +37,7 @@ struct DecodeSmem {
   float scur[G];
   float M[G];
   float inv[G];
+  float invl[G];   // sum-of-terms merges: 1 / (phi(q) z), or 0 while the state is empty
   int item;
   int last;
 };
@@ -134,10 +135,10 @@ __device__ __forceinline__ void state_item(const DecodeParams &p, const WorkItem
   constexpr int TPR = D / 4;                   // threads per state row (float4 each)
   constexpr int RPI = kDecodeThreads / TPR;    // rows per iteration
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  if (!(ld.w == 0 || t >= ld.w)) return;       // nothing leaves the window yet: S,z are still zero
+  if (t < ld.wlin) return;                     // nothing has reached the state yet: S,z are still zero
   const int ub = b * p.Hkv + g;
   const T *ke, *ve;
-  if (ld.w == 0) {  // no ring: the current token goes straight to the state
+  if (ld.wlin == 0) {  // no ring, or a state that holds every token: the current token is folded now
     ke = reinterpret_cast<const T *>(p.k) + size_t(it.unit) * D;
     ve = reinterpret_cast<const T *>(p.v) + size_t(it.unit) * D;
   } else {          // slot t mod cap holds token t - w
@@ -236,7 +237,7 @@ __device__ __forceinline__ void merge_unit(const DecodeParams &p, const WorkItem
   const int per_unit = ld.n_win_items + ld.n_state_items;
   const float *rec0 = p.partials + ld.part_base + size_t(ub) * per_unit * p.rec_floats;
   const bool has_win = ld.cap > 0;
-  const bool has_state = ld.n_state_items > 0 && (ld.w == 0 || t >= ld.w);
+  const bool has_state = ld.n_state_items > 0 && t >= ld.wlin;
   const T *kt = reinterpret_cast<const T *>(p.k) + size_t(it.unit) * D;
   const T *vt = reinterpret_cast<const T *>(p.v) + size_t(it.unit) * D;
 
@@ -257,7 +258,10 @@ __device__ __forceinline__ void merge_unit(const DecodeParams &p, const WorkItem
   __syncthreads();
   if (tid < G) {
     const int h = tid;
-    float M = 0.f;  // m* = max(window max, 0): the linear terms carry the factor exp(-m*) <= 1
+    // shared normaliser: m* = max(window max, 0), the linear terms carry the factor exp(-m*) <= 1;
+    // sum of two normalised terms: the window is normalised on its own, against its own maximum
+    const bool shared = ld.merge == GLIDE_MERGE_SHARED;
+    float M = shared ? 0.f : -CUDART_INF_F;
     for (int i = 0; i < ld.n_win_items; ++i) M = fmaxf(M, __ldcg(rec0 + size_t(i) * p.rec_floats + G * D + h));
     if (has_win) M = fmaxf(M, sm.scur[h]);
     float den = 0.f;
@@ -267,14 +271,17 @@ __device__ __forceinline__ void merge_unit(const DecodeParams &p, const WorkItem
       den = fmaf(__ldcg(r + G * D + G + h), exp2f(mi - M), den);
     }
     if (has_win) den += exp2f(sm.scur[h] - M);
+    float invl = 0.f;
     if (has_state) {
       float bsum = 0.f;
       for (int i = 0; i < ld.n_state_items; ++i)
         bsum += __ldcg(rec0 + size_t(ld.n_win_items + i) * p.rec_floats + G * D + h);
-      den = fmaf(exp2f(-M), bsum, den);
+      if (shared) den = fmaf(exp2f(-M), bsum, den);
+      else invl = bsum > 0.f ? 1.0f / bsum : 0.f;
     }
     sm.M[h] = M;
-    sm.inv[h] = 1.0f / den;
+    sm.inv[h] = den > 0.f ? 1.0f / den : 0.f;   // den = 0 only for a sum-of-terms layer without a window
+    sm.invl[h] = invl;
   }
   __syncthreads();
   T *outp = reinterpret_cast<T *>(p.out);
@@ -287,13 +294,15 @@ __device__ __forceinline__ void merge_unit(const DecodeParams &p, const WorkItem
       num = fmaf(__ldcg(r + idx), exp2f(__ldcg(r + G * D + h) - M), num);
     }
     if (has_win) num = fmaf(exp2f(sm.scur[h] - M), to_f32(vt[c]), num);
+    float lin = 0.f;
     if (has_state) {
       float asum = 0.f;
       for (int i = 0; i < ld.n_state_items; ++i) asum += __ldcg(rec0 + size_t(ld.n_win_items + i) * p.rec_floats + idx);
-      num = fmaf(exp2f(-M), asum, num);
+      if (ld.merge == GLIDE_MERGE_SHARED) num = fmaf(exp2f(-M), asum, num);
+      else lin = asum * sm.invl[h];
     }
     const int head = p.heads_of[g * G + h];
-    from_f32(outp + ((size_t(it.layer) * p.B + b) * p.H + head) * D + c, num * sm.inv[h]);
+    from_f32(outp + ((size_t(it.layer) * p.B + b) * p.H + head) * D + c, fmaf(num, sm.inv[h], lin));
   }
   if (has_win) {  // every reader of slot t mod cap has finished: store the new row
     const size_t row = (size_t(ub) * size_t(ld.cap) + size_t(t % ld.cap)) * D;

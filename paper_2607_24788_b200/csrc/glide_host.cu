@@ -35,7 +35,12 @@ int validate_config(const glide_config *c) {
     return GLIDE_ERR_UNSUPPORTED;
   for (int l = 0; l < c->n_layers; ++l)
     if (c->windows[l] < 0) return GLIDE_ERR_INVALID_ARG;
-  if (c->phi != GLIDE_PHI_SOFTMAX || c->merge != GLIDE_MERGE_SHARED) return GLIDE_ERR_UNSUPPORTED;
+  if (c->phi != GLIDE_PHI_SOFTMAX) return GLIDE_ERR_UNSUPPORTED;
+  if (c->merge < GLIDE_MERGE_SHARED || c->merge > GLIDE_MERGE_SUM_ALL) return GLIDE_ERR_INVALID_ARG;
+  if (c->merge != GLIDE_MERGE_SHARED &&
+      (c->decode_impl == GLIDE_DECODE_MMA || c->decode_impl == GLIDE_DECODE_STREAM ||
+       c->prefill_impl == GLIDE_PREFILL_MMA_SYNC || c->prefill_impl == GLIDE_PREFILL_TCGEN05))
+    return GLIDE_ERR_UNSUPPORTED;   // the sum-of-terms merges exist on the CUDA-core kernels only
   if (c->head_dim != 64 && c->head_dim != 128) return GLIDE_ERR_UNSUPPORTED;
   if (c->n_q_heads % c->n_kv_heads != 0) return GLIDE_ERR_UNSUPPORTED;
   int G = c->n_q_heads / c->n_kv_heads;
@@ -95,7 +100,9 @@ int glide::plan_context(const glide_config *cfg, glide_ctx *ctx, std::vector<Wor
     LayerDev &ld = ctx->layers[l];
     ld.w = ctx->windows[l];
     ld.cap = std::min<int64_t>(ld.w, cfg->max_tokens);
-    ld.evicts = ld.w < cfg->max_tokens ? 1 : 0;
+    ld.merge = cfg->merge;
+    ld.wlin = cfg->merge == GLIDE_MERGE_SUM_ALL ? 0 : ld.w;
+    ld.evicts = ld.wlin < cfg->max_tokens ? 1 : 0;
     const int chunk = chunk_of(ld.cap);
     ld.n_win_items = int((ld.cap + chunk - 1) / chunk);
     ld.n_state_items = ld.evicts ? splits : 0;
@@ -244,7 +251,7 @@ int glide_create(const glide_config *cfg, void *dev_workspace, size_t workspace_
   int per_sm = 0;
   // kernel choice: fp32 -> CUDA cores; bf16 -> streaming tensor-core kernel when it applies, else per-item one
   ctx->decode_kind = 0;
-  if (ok && cfg->io_dtype == GLIDE_BF16 && cfg->decode_impl != GLIDE_DECODE_FMA) {
+  if (ok && cfg->io_dtype == GLIDE_BF16 && cfg->decode_impl != GLIDE_DECODE_FMA && cfg->merge == GLIDE_MERGE_SHARED) {
     ok = build_ring_tensor_maps(ctx) == GLIDE_OK;
     const bool want_stream = cfg->decode_impl == GLIDE_DECODE_AUTO || cfg->decode_impl == GLIDE_DECODE_STREAM;
     if (ok && want_stream && stream_decode_supported(ctx) && ctx->sm_count <= kMaxStreamCtas) {

@@ -24,8 +24,9 @@ struct LayerDev {
   size_t part_base;     // float index into the split-K scratch of this layer's first unit
   int32_t n_win_items;  // window work items per unit
   int32_t n_state_items;// state work items per unit (0 if the layer never evicts)
-  int32_t evicts;       // 1 if w < max_tokens
-  int32_t pad_;
+  int32_t evicts;       // 1 if the layer has a state that ever receives tokens: wlin < max_tokens
+  int32_t merge;        // glide_merge
+  int64_t wlin;         // a token enters the state wlin steps after it arrives: w, or 0 when the state holds all tokens
 };
 
 // One work item of the decode kernel.

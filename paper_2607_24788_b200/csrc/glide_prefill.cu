@@ -65,7 +65,7 @@ __global__ void __launch_bounds__(kPrefillThreads) prefill_phi_kernel(const Pref
   const int lrel = int(u / (int64_t(p.Hkv) * p.B));
   const LayerDev ld = p.layers[p.layer_begin + lrel];
   if (!ld.evicts) return;
-  const int64_t j = p.n0 + p.c0 + i - ld.w;  // delayed token
+  const int64_t j = p.n0 + p.c0 + i - ld.wlin;  // delayed token
   if (j < 0) return;
   const RowSource<T> src = make_source<T, D>(p, ld, lrel, b, g);
   float x[E];
@@ -146,8 +146,8 @@ __global__ void __launch_bounds__(kPrefillThreads) prefill_attn_kernel(const Pre
 #pragma unroll
     for (int e = 0; e < E; ++e) lin[h][e] = 0.f;
   }
-  if (ld.evicts && tq >= ld.w) {
-    const int64_t folded_at_chunk_start = p.n0 + p.c0 - ld.w;  // tokens < this are in S,z
+  if (ld.evicts && tq >= ld.wlin) {
+    const int64_t folded_at_chunk_start = p.n0 + p.c0 - ld.wlin;  // tokens < this are in S,z
     if (folded_at_chunk_start > 0) {
       const float *Sb = reinterpret_cast<const float *>(p.ws + ld.S) + size_t(ub) * D * D;
       const float *zb = reinterpret_cast<const float *>(p.ws + ld.z) + size_t(ub) * D;
@@ -176,7 +176,7 @@ __global__ void __launch_bounds__(kPrefillThreads) prefill_attn_kernel(const Pre
     int i_lo = 0;
     if (folded_at_chunk_start < 0) i_lo = int(-folded_at_chunk_start);  // delayed index < 0 does not exist
     for (int ii = i_lo; ii <= i; ++ii) {
-      const int64_t j = p.n0 + p.c0 + ii - ld.w;
+      const int64_t j = p.n0 + p.c0 + ii - ld.wlin;
       float fk[E], vx[E];
       load_elems<float, E>(pk + size_t(ii) * D + lane * E, fk);
       load_elems<T, E>(src.v(j, D) + lane * E, vx);
@@ -193,8 +193,18 @@ __global__ void __launch_bounds__(kPrefillThreads) prefill_attn_kernel(const Pre
     }
   }
 
-  // shared normaliser
+  // shared normaliser, or the sum of the two separately normalised terms (an empty term counts as zero)
   T *obase = reinterpret_cast<T *>(p.out) + ((size_t(lrel) * p.B + b) * size_t(p.T) + size_t(p.c0 + i)) * p.H * D;
+  if (ld.merge != GLIDE_MERGE_SHARED) {
+#pragma unroll
+    for (int h = 0; h < G; ++h) {
+      const float iw = l[h] > 0.f ? 1.0f / l[h] : 0.f, il = bl[h] > 0.f ? 1.0f / bl[h] : 0.f;
+      const int head = p.heads_of[g * G + h];
+#pragma unroll
+      for (int e = 0; e < E; ++e) from_f32(obase + size_t(head) * D + lane * E + e, fmaf(acc[h][e], iw, lin[h][e] * il));
+    }
+    return;
+  }
 #pragma unroll
   for (int h = 0; h < G; ++h) {
     const float M = fmaxf(m[h], 0.f);
@@ -229,7 +239,7 @@ __global__ void __launch_bounds__(kPrefillThreads) prefill_state_kernel(const Pr
   const int lrel = int(u / (int64_t(p.Hkv) * p.B));
   const LayerDev ld = p.layers[p.layer_begin + lrel];
   if (!ld.evicts) return;
-  const int64_t first = p.n0 + p.c0 - ld.w;       // delayed token of chunk index 0
+  const int64_t first = p.n0 + p.c0 - ld.wlin;    // delayed token of chunk index 0
   const int i_lo = first < 0 ? int(first < -int64_t(p.C) ? p.C : -first) : 0;
   if (i_lo >= p.C) return;
   const RowSource<T> src = make_source<T, D>(p, ld, lrel, b, g);
@@ -360,7 +370,8 @@ int launch_prefill(glide_ctx *ctx, int layer_begin, int layer_count, int64_t T, 
   const int64_t units = int64_t(layer_count) * p.B * p.Hkv;
   int impl = ctx->cfg.prefill_impl;
   if (impl == GLIDE_PREFILL_AUTO)
-    impl = (prefill_attn_mma_supported(ctx) && ctx->cfg.decode_impl != GLIDE_DECODE_FMA) ? GLIDE_PREFILL_TCGEN05 : GLIDE_PREFILL_FMA;
+    impl = (prefill_attn_mma_supported(ctx) && ctx->cfg.decode_impl != GLIDE_DECODE_FMA && ctx->cfg.merge == GLIDE_MERGE_SHARED)
+               ? GLIDE_PREFILL_TCGEN05 : GLIDE_PREFILL_FMA;
   // the tcgen05 kernel has alignment conditions that depend on the call; where they do not hold the call falls
   // back to the mma.sync kernel
   const bool use_tc = impl == GLIDE_PREFILL_TCGEN05 && prefill_attn_tc_supported(ctx, layer_begin, layer_count, p.n0);

@@ -17,7 +17,7 @@ LIB_PATH = os.path.join(_PKG, "libglide.so")
 
 GLIDE_F32, GLIDE_BF16 = 0, 1
 GLIDE_PHI_SOFTMAX = 0
-GLIDE_MERGE_SHARED = 0
+GLIDE_MERGE_SHARED, GLIDE_MERGE_SUM_EVICTED, GLIDE_MERGE_SUM_ALL = 0, 1, 2
 GLIDE_DECODE_AUTO, GLIDE_DECODE_MMA, GLIDE_DECODE_FMA, GLIDE_DECODE_STREAM = 0, 1, 2, 3
 
 GLIDE_OK = 0
@@ -113,14 +113,14 @@ def _stream(stream: Optional[torch.cuda.Stream]) -> Optional[int]:
 def make_config(windows: Sequence[int], batch: int, n_q_heads: int, n_kv_heads: int, head_dim: int, max_tokens: int,
                 dtype: torch.dtype = torch.bfloat16, q_to_kv: Optional[Sequence[int]] = None,
                 softmax_scale: float = 0.0, prefill_chunk: int = 0, decode_chunk: int = 0,
-                decode_state_splits: int = 0, decode_impl: int = 0, prefill_impl: int = 0):
+                decode_state_splits: int = 0, decode_impl: int = 0, prefill_impl: int = 0, merge: int = 0):
     """Returns (glide_config, keepalive) -- keepalive holds the host arrays the struct points to."""
     win = (ctypes.c_int64 * len(windows))(*[int(w) for w in windows])
     qmap = (ctypes.c_int32 * len(q_to_kv))(*[int(x) for x in q_to_kv]) if q_to_kv is not None else None
     cfg = glide_config()
     cfg.n_layers, cfg.batch, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim = len(windows), batch, n_q_heads, n_kv_heads, head_dim
     cfg.io_dtype = {torch.float32: GLIDE_F32, torch.bfloat16: GLIDE_BF16}[dtype]
-    cfg.phi, cfg.merge = GLIDE_PHI_SOFTMAX, GLIDE_MERGE_SHARED
+    cfg.phi, cfg.merge = GLIDE_PHI_SOFTMAX, int(merge)
     cfg.windows = ctypes.cast(win, ctypes.POINTER(ctypes.c_int64))
     cfg.q_to_kv = ctypes.cast(qmap, ctypes.POINTER(ctypes.c_int32)) if qmap is not None else None
     cfg.max_tokens = int(max_tokens)

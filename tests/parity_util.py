@@ -78,7 +78,8 @@ def run_case(windows: Sequence[int], B: int, H: int, Hkv: int, d: int, dtype: to
     wl = synth.Workload(seed, L, B, H, Hkv, d, dtype, amp)
     g = glide.Glide(windows, B, H, Hkv, d, max_tokens, dtype=dtype, device=dev, q_to_kv=q_to_kv, softmax_scale=scale,
                     **cfg_kw)
-    stack = orc.Stack(windows, B, H, Hkv, d, scale, q_to_kv=None if q_to_kv is None else np.asarray(q_to_kv, np.int32))
+    stack = orc.Stack(windows, B, H, Hkv, d, scale, q_to_kv=None if q_to_kv is None else np.asarray(q_to_kv, np.int32),
+                      merge=cfg_kw.get("merge", 0))
     pos = 0
     worst = 0.0
     for T in prompt_calls:

@@ -163,3 +163,19 @@ def test_bf16_prefill_tcgen05_aligned_calls(G, chunk):
 
 def test_bf16_prefill_tcgen05_large_logits():
     run_case([48, 208], 1, 8, 2, 128, BF16, [256], 6, amp=128 ** -0.5 * 12, prefill_impl=2)
+
+
+@pytest.mark.parametrize("merge", [1, 2])   # appendix hybrid equations: evicted-token state / all-token state
+@pytest.mark.parametrize("dtype,d", [(F32, 64), (BF16, 128)])
+def test_sum_of_terms_merges(merge, dtype, d):
+    amp = 1.0 if dtype == F32 else d ** -0.5 * 4
+    run_case([0, 1, 5, 40, 1000], 2, 4, 2, d, dtype, [70, 33], 24, amp=amp, seed=merge, prefill_chunk=32, decode_chunk=16,
+             merge=merge)
+
+
+def test_sum_of_terms_merges_need_the_cuda_core_kernels():
+    from paper_2607_24788_b200 import glide
+    with pytest.raises(glide.GlideError):
+        glide.Glide([64], 1, 8, 2, 128, 256, dtype=BF16, merge=1, decode_impl=3)
+    with pytest.raises(glide.GlideError):
+        glide.Glide([64], 1, 8, 2, 128, 256, dtype=BF16, merge=2, prefill_impl=2)
