@@ -424,37 +424,35 @@ def run_glide(args, shape):
 
 
 def measure_per_layer_launch(g0, shape, qkv, out, steps, device):
-    """The same decode step issued as one launch per layer (L one-layer contexts holding copies of the layers'
-    state) instead of one launch for the whole stack: what the per-launch overhead costs when the windows are
-    small.  Same sequence state every step, so it compares with the one-launch `hot_l2` figure."""
+    """The same decode step issued layer by layer through glide_decode_step_layers (one launch per layer, each with
+    its own schedule) instead of one launch for the whole stack: what a model pays whose layers depend on each
+    other, and what the per-launch overhead costs when the windows are small.  Same sequence state every step,
+    so it compares with the one-launch `hot_l2` figure."""
     from paper_2607_24788_b200 import glide
+    import ctypes
     L = shape.n_layers
     dt = torch_dtype(shape)
     n = g0.glide_layer_info(0)["n"]
-    layer_ctx = []
+    g = glide.Glide(shape.windows, shape.batch, shape.n_q_heads, shape.n_kv_heads, shape.head_dim, g0.max_tokens,
+                    dtype=dt, device=device, prefill_chunk=shape.prefill_chunk, **KERNEL_KNOBS)
     for l in range(L):
-        g = glide.Glide([shape.windows[l]], shape.batch, shape.n_q_heads, shape.n_kv_heads, shape.head_dim,
-                        g0.max_tokens, dtype=dt, device=device, **KERNEL_KNOBS)   # same capacity: same ring size
         rk, rv, S, z = g0.glide_export_state(l)
-        cap = g.capacity(0)
-        g.glide_import_state(0, n, rk if cap else None, rv if cap else None, S, z)
-        layer_ctx.append(g)
+        cap = g.capacity(l)
+        g.glide_import_state(l, n, rk if cap else None, rv if cap else None, S, z)
     torch.cuda.synchronize()
     q, k, v = qkv
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-
     # the C entry point with pointers resolved once: the binding's per-call argument checks (tens of microseconds)
     # would otherwise be what is measured
-    import ctypes
     vp = ctypes.c_void_p
     sptr = vp(torch.cuda.current_stream().cuda_stream or None)
-    calls = [(g.lib.glide_decode_step, g._h, vp(q[l].data_ptr()), vp(k[l].data_ptr()), vp(v[l].data_ptr()),
-              vp(out[l].data_ptr())) for l, g in enumerate(layer_ctx)]
+    fn = g.lib.glide_decode_step_layers
+    calls = [(l, vp(q[l].data_ptr()), vp(k[l].data_ptr()), vp(v[l].data_ptr()), vp(out[l].data_ptr())) for l in range(L)]
 
     def launch(l):
-        fn, h, a, b, c, o = calls[l]
-        if fn(h, a, b, c, o, sptr) != 0:
-            raise RuntimeError("glide_decode_step failed in per-layer mode")
+        _, a, b, c, o = calls[l]
+        if fn(g._h, l, 1, a, b, c, o, sptr) != 0:
+            raise RuntimeError("glide_decode_step_layers failed in per-layer mode")
 
     def step():
         for l in range(L):
@@ -475,25 +473,11 @@ def measure_per_layer_launch(g0, shape, qkv, out, steps, device):
         torch.cuda.synchronize()
         res.append(ev0.elapsed_time(ev1) * 1e3 / steps)
         host_us.append((h1 - h0) * 1e6 / steps)
-    # every layer's launch alone between two events (what a model that runs other kernels between the layers'
-    # attention calls sees on the GPU), summed over the layers
-    isolated = 0.0
-    for l in range(L):
-        one = []
-        for _ in range(12):
-            ev0.record()
-            launch(l)
-            ev1.record()
-            torch.cuda.synchronize()
-            one.append(ev0.elapsed_time(ev1) * 1e3)
-        isolated += statistics.median(one)
-    del layer_ctx
+    del g
     return {"us_per_step": statistics.median(res), "launches_per_step": L,
             "host_issue_us_per_step": statistics.median(host_us),
-            "sum_of_isolated_launches_us": isolated,
-            "note": "one glide_decode_step per layer on one-layer contexts, issued back to back; when "
-                    "host_issue_us_per_step is about us_per_step the figure is bound by the host issuing launches; "
-                    "sum_of_isolated_launches_us adds up each layer's launch timed alone between two events"}
+            "note": "glide_decode_step_layers, one layer per call, issued back to back; when host_issue_us_per_step is "
+                    "about us_per_step the figure is bound by the host issuing launches"}
 
 
 def measure_prefill(ctx, wl, shape, n_tokens, device):

@@ -115,7 +115,8 @@ typedef struct {
 int glide_workspace_bytes(const glide_config *cfg, size_t *bytes_out);
 
 /* Build a context over caller-owned device memory `dev_workspace` (>= glide_workspace_bytes,
- * 256-byte aligned).  Sets the GQA head mapping and the per-layer windows, uploads the static
+ * 256-byte aligned; a 2 MiB-aligned base is worth about 2 % on the smallest decode steps, because the library
+ * places the streamed arrays on 2 MiB multiples of its offsets).  Sets the GQA head mapping and the per-layer windows, uploads the static
  * work lists and zeroes rings' bookkeeping, S and z on `stream`.  The workspace must stay
  * alive and untouched by the caller until glide_destroy. */
 int glide_create(const glide_config *cfg, void *dev_workspace, size_t workspace_bytes, void *stream,
@@ -141,6 +142,16 @@ int glide_prefill(glide_ctx *ctx, int32_t layer_begin, int32_t layer_count, int6
  * All layers must be at the same position (GLIDE_ERR_STATE otherwise). */
 int glide_decode_step(glide_ctx *ctx, const void *dev_q, const void *dev_k, const void *dev_v, void *dev_out,
                       void *stream);
+
+/* The same step for the layers [layer_begin, layer_begin + layer_count) only: what a model needs whose layer l + 1
+ * computes its q, k, v from layer l's output (the setting of the paper's experiments, whose "Limitations & Future
+ * Works" section names the kernel-launch overhead of small windows).  Tensors are those of the range:
+ *   dev_q, dev_out [layer_count][B][H][d];  dev_k, dev_v [layer_count][B][H_kv][d].
+ * The layers of the range must be at the same position; other layers are not touched, and glide_decode_step
+ * needs all layers level again.  On the streaming kernel a range other than the whole stack is one launch per
+ * layer (each with its own schedule); on the other kernels it is one launch. */
+int glide_decode_step_layers(glide_ctx *ctx, int32_t layer_begin, int32_t layer_count, const void *dev_q,
+                             const void *dev_k, const void *dev_v, void *dev_out, void *stream);
 
 /* Decode step for callers that must not allocate.  (The paper has no counterpart: this is a deployment
  * variant of glide_decode_step, not part of the method.)

@@ -331,6 +331,7 @@ __global__ void __launch_bounds__(kDecodeThreads) glide_decode_kernel(const Deco
       if (tid == 0) atomicExch(&p.ctl->status, kDevBadItem);
       continue;
     }
+    if (it.layer < p.layer_begin || it.layer >= p.layer_begin + p.layer_count) continue;   // not a layer of this launch
     const LayerDev ld = p.layers[it.layer];
     const int64_t t = p.n_dev[it.layer];
     const int ub = it.unit - it.layer * units_per_layer;
@@ -357,7 +358,7 @@ __global__ void __launch_bounds__(kDecodeThreads) glide_decode_kernel(const Deco
       // every CTA has drained the list: re-arm it and advance the positions
       p.ctl->work_counter = 0;
       p.ctl->done_counter = 0;
-      for (int l = 0; l < p.L; ++l) p.n_dev[l] += 1;
+      for (int l = 0; l < p.layer_count; ++l) p.n_dev[p.layer_begin + l] += 1;
       __threadfence();
     }
   }
@@ -370,8 +371,19 @@ __global__ void glide_advance_kernel(int64_t *n_dev, int layer_begin, int layer_
 
 }  // namespace
 
-DecodeParams make_decode_params(const glide_ctx *ctx, const void *q, const void *k, const void *v, void *out) {
+// q, k, v, out are the tensors of the layer range [layer_begin, layer_begin + layer_count).  The per-item kernels
+// index them with the absolute layer, so they get base pointers moved back by layer_begin layers (never
+// dereferenced below the range); the streaming kernel's per-range schedules are numbered from the range's start.
+DecodeParams make_decode_params(const glide_ctx *ctx, int layer_begin, int layer_count, const void *q, const void *k,
+                                const void *v, void *out) {
   DecodeParams p{};
+  if (ctx->decode_kind != 2 && layer_begin > 0) {
+    const size_t row = size_t(ctx->cfg.head_dim) * ctx->elem * size_t(ctx->cfg.batch) * size_t(layer_begin);
+    q = static_cast<const unsigned char *>(q) - row * ctx->cfg.n_q_heads;
+    out = static_cast<unsigned char *>(out) - row * ctx->cfg.n_q_heads;
+    k = static_cast<const unsigned char *>(k) - row * ctx->cfg.n_kv_heads;
+    v = static_cast<const unsigned char *>(v) - row * ctx->cfg.n_kv_heads;
+  }
   p.ws = ctx->ws;
   p.layers = reinterpret_cast<const LayerDev *>(ctx->ws + ctx->off_layers);
   p.items = reinterpret_cast<const WorkItem *>(ctx->ws + ctx->off_items);
@@ -391,7 +403,9 @@ DecodeParams make_decode_params(const glide_ctx *ctx, const void *q, const void 
   p.Hkv = ctx->cfg.n_kv_heads;
   p.rec_floats = ctx->rec_floats;
   p.scale_log2 = ctx->scale * kLog2e;
-  p.t_host = ctx->n_host[0];
+  p.t_host = ctx->n_host[size_t(layer_begin)];
+  p.layer_begin = layer_begin;
+  p.layer_count = layer_count;
   return p;
 }
 
@@ -408,9 +422,25 @@ int decode_occupancy(const glide_ctx *ctx, int *blocks_per_sm) {
   });
 }
 
-int launch_decode(glide_ctx *ctx, const void *q, const void *k, const void *v, void *out, cudaStream_t stream) {
-  const DecodeParams p = make_decode_params(ctx, q, k, v, out);
-  if (ctx->decode_kind == 2) return launch_decode_stream(ctx, p, stream);
+int launch_decode(glide_ctx *ctx, int layer_begin, int layer_count, const void *q, const void *k, const void *v, void *out,
+                  cudaStream_t stream) {
+  const int L = ctx->cfg.n_layers;
+  if (ctx->decode_kind == 2 && layer_count != L) {
+    // the streaming kernel has a schedule for the whole stack and one per layer: a partial range is one launch per layer
+    const size_t qrow = size_t(ctx->cfg.head_dim) * ctx->elem * size_t(ctx->cfg.batch) * ctx->cfg.n_q_heads;
+    const size_t krow = size_t(ctx->cfg.head_dim) * ctx->elem * size_t(ctx->cfg.batch) * ctx->cfg.n_kv_heads;
+    for (int i = 0; i < layer_count; ++i) {
+      const DecodeParams pl = make_decode_params(ctx, layer_begin + i, 1, static_cast<const unsigned char *>(q) + qrow * i,
+                                                 static_cast<const unsigned char *>(k) + krow * i,
+                                                 static_cast<const unsigned char *>(v) + krow * i,
+                                                 static_cast<unsigned char *>(out) + qrow * i);
+      const int rc = launch_decode_stream(ctx, pl, 1 + layer_begin + i, stream);
+      if (rc) return rc;
+    }
+    return GLIDE_OK;
+  }
+  const DecodeParams p = make_decode_params(ctx, layer_begin, layer_count, q, k, v, out);
+  if (ctx->decode_kind == 2) return launch_decode_stream(ctx, p, 0, stream);
   if (ctx->decode_kind == 1) return launch_decode_mma(ctx, p, stream);
   return dispatch_config(ctx->cfg.io_dtype, ctx->cfg.head_dim, ctx->G, [&](auto tt, auto dd, auto gg) -> int {
     using T = typename decltype(tt)::type;
@@ -463,7 +493,7 @@ int launch_decode_noalloc(glide_ctx *ctx, const void *q, const void *k, const vo
     cudaGetLastError();
     return GLIDE_ERR_CUDA;
   }
-  DecodeParams p = make_decode_params(ctx, q, k, v, out);
+  DecodeParams p = make_decode_params(ctx, 0, ctx->cfg.n_layers, q, k, v, out);
   p.ctl = reinterpret_cast<Control *>(scratch);
   p.tickets = reinterpret_cast<int32_t *>(scratch + tickets_off);
   p.partials = reinterpret_cast<float *>(scratch + partials_off);

@@ -593,6 +593,7 @@ __global__ void __launch_bounds__(WARPS * 32, 1) glide_decode_mma_kernel(const D
       if (lane == 0) atomicExch(&p.ctl->status, kDevBadItem);
       continue;
     }
+    if (it.layer < p.layer_begin || it.layer >= p.layer_begin + p.layer_count) continue;   // not a layer of this launch
     const LayerDev ld = p.layers[it.layer];
     const int64_t t = p.n_dev[it.layer];
     const int ub = it.unit - it.layer * units_per_layer;
@@ -631,7 +632,7 @@ __global__ void __launch_bounds__(WARPS * 32, 1) glide_decode_mma_kernel(const D
     if (atomicAdd(&p.ctl->done_counter, 1) == int(gridDim.x) - 1) {
       p.ctl->work_counter = 0;
       p.ctl->done_counter = 0;
-      for (int l = 0; l < p.L; ++l) p.n_dev[l] += 1;
+      for (int l = 0; l < p.layer_count; ++l) p.n_dev[p.layer_begin + l] += 1;
       __threadfence();
     }
   }

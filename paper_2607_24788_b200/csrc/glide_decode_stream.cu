@@ -323,7 +323,7 @@ glide_decode_stream_kernel(const DecodeParams p, const StreamParams sp) {
   // the device counters are not read by this kernel; one thread moves them on (no grid-wide completion count,
   // which would put an atomic round trip at the end of every CTA)
   if (blockIdx.x == 0)
-    for (int l = tid; l < p.L; l += kThreads) p.n_dev[l] = t + 1;
+    for (int l = tid; l < p.layer_count; l += kThreads) p.n_dev[p.layer_begin + l] = t + 1;
   // this warp's segments: the run of the CTA's list that carries its index
   int seg_lo = 0;
   while (seg_lo < cta_nseg && sm_segs[seg_lo].range < warp) ++seg_lo;
@@ -1008,10 +1008,13 @@ int dispatch_stream(int G, F &&f) {
 //      a unit heavier than a CTA's share is first cut into equal pieces.  So almost every unit lives inside one
 //      CTA and is reduced in shared memory; only the oversized ones need global records and a merge.
 //   2. Inside a CTA the list of pieces is cut into 8 contiguous, equally heavy ranges, one per warp.
-void build_stream_schedule(const glide_ctx *ctx, int n_ranges, std::vector<StreamSegment> *segs,
+// Schedule for the layers [layer_begin, layer_begin + layer_count).  Units and query rows are numbered relative to
+// the first layer of the range (that is how a launch for the range addresses q, k, v, out and the tickets); the
+// layer index itself stays absolute (descriptors, layer table).
+void build_stream_schedule(const glide_ctx *ctx, int layer_begin, int layer_count, int n_ranges, std::vector<StreamSegment> *segs,
                            std::vector<int32_t> *range_seg_begin, int *max_segs_per_cta, size_t *n_records) {
   constexpr int64_t kSegWeight = GLIDE_W_UNIT, kStateWeight = GLIDE_W_STATE, kWinWeight = GLIDE_W_WIN;
-  const int L = ctx->cfg.n_layers, B = ctx->cfg.batch, Hkv = ctx->cfg.n_kv_heads, d = ctx->cfg.head_dim;
+  const int B = ctx->cfg.batch, Hkv = ctx->cfg.n_kv_heads, d = ctx->cfg.head_dim;
   const int n_ctas = n_ranges / kWarps;
   const int64_t units_per_layer = int64_t(B) * Hkv;
   bool contiguous_heads = true;
@@ -1027,10 +1030,10 @@ void build_stream_schedule(const glide_ctx *ctx, int n_ranges, std::vector<Strea
   std::vector<Piece> pieces;
   int64_t total_w = 0;
   int n_units = 0;
-  for (int l = 0; l < L; ++l) {
+  for (int l = layer_begin; l < layer_begin + layer_count; ++l) {
     const LayerDev &ld = ctx->layers[l];
     for (int64_t u = 0; u < units_per_layer; ++u) {
-      Piece pc{l, int(int64_t(l) * units_per_layer + u), n_units++, 0, ld.evicts ? d / kTileRows : 0, 0,
+      Piece pc{l, int(int64_t(l - layer_begin) * units_per_layer + u), n_units++, 0, ld.evicts ? d / kTileRows : 0, 0,
                int((ld.cap + kTileRows - 1) / kTileRows)};
       pieces.push_back(pc);
       total_w += pc.weight();
@@ -1151,7 +1154,7 @@ void build_stream_schedule(const glide_ctx *ctx, int n_ranges, std::vector<Strea
         sg.range = wi;
         sg.state0 = pc.st0 + st_done;
         sg.win0 = pc.w0 + w_done;
-        const int64_t ub = pc.unit - int64_t(pc.layer) * units_per_layer;
+        const int64_t ub = pc.unit - int64_t(pc.layer - layer_begin) * units_per_layer;
         sg.row_base = int32_t(ub * ld.cap);
         sg.cap = int32_t(ld.cap);
         sg.w = int32_t(std::min<int64_t>(ld.w, INT32_MAX));
@@ -1163,7 +1166,7 @@ void build_stream_schedule(const glide_ctx *ctx, int n_ranges, std::vector<Strea
         sg.g = int32_t(ub % Hkv);
         {
           const int64_t b = ub / Hkv;
-          const int64_t row = (int64_t(pc.layer) * B + b) * ctx->cfg.n_q_heads;
+          const int64_t row = (int64_t(pc.layer - layer_begin) * B + b) * ctx->cfg.n_q_heads;
           sg.qrow0 = int32_t(row + (contiguous_heads ? ctx->heads_of[size_t(sg.g) * ctx->G] : 0));
         }
         st_done += sg.n_state;
@@ -1236,11 +1239,26 @@ int stream_decode_supported(const glide_ctx *ctx) {
 
 int stream_decode_setup(glide_ctx *ctx) {
   const int n_ctas = std::min(ctx->sm_count, kMaxStreamCtas);
-  int max_segs = 0;
-  size_t n_records = 0;
-  build_stream_schedule(ctx, n_ctas * kWarps, &ctx->stream_segs, &ctx->stream_cta_begin, &max_segs, &n_records);
-  ctx->stream_max_segs = std::max(max_segs, 1);
-  if (ctx->stream_segs.size() > ctx->stream_seg_capacity || n_records > ctx->stream_rec_capacity) return GLIDE_ERR_UNSUPPORTED;
+  const int L = ctx->cfg.n_layers;
+  ctx->stream_scheds.clear();
+  ctx->stream_segs.clear();
+  ctx->stream_max_segs = 1;
+  // [0]: all layers in one launch; [1 + l]: layer l alone, for callers that run other kernels between the layers
+  const int n_sched = L > 1 ? L + 1 : 1;
+  for (int si = 0; si < n_sched; ++si) {
+    std::vector<StreamSegment> segs;
+    glide_ctx::StreamSchedule sc;
+    int max_segs = 0;
+    size_t n_records = 0;
+    build_stream_schedule(ctx, si == 0 ? 0 : si - 1, si == 0 ? L : 1, n_ctas * kWarps, &segs, &sc.range_begin, &max_segs, &n_records);
+    if (n_records > ctx->stream_rec_capacity) return GLIDE_ERR_UNSUPPORTED;
+    sc.seg_base = ctx->stream_segs.size();
+    sc.n_segs = segs.size();
+    ctx->stream_segs.insert(ctx->stream_segs.end(), segs.begin(), segs.end());
+    ctx->stream_max_segs = std::max(ctx->stream_max_segs, max_segs);
+    ctx->stream_scheds.push_back(std::move(sc));
+  }
+  if (ctx->stream_segs.size() > ctx->stream_seg_capacity) return GLIDE_ERR_UNSUPPORTED;
   bool contiguous = true;
   for (int g = 0; g < ctx->cfg.n_kv_heads; ++g)
     for (int i = 1; i < ctx->G; ++i)
@@ -1274,10 +1292,12 @@ extern "C" int glide_debug_set_stream_trace(void *dev_buf) {
 }
 #endif
 
-int launch_decode_stream(glide_ctx *ctx, const DecodeParams &p, cudaStream_t stream) {
+int launch_decode_stream(glide_ctx *ctx, const DecodeParams &p, int schedule, cudaStream_t stream) {
+  if (schedule < 0 || size_t(schedule) >= ctx->stream_scheds.size()) return GLIDE_ERR_INVALID_ARG;
+  const glide_ctx::StreamSchedule &sc = ctx->stream_scheds[size_t(schedule)];
   StreamParams sp{};
-  sp.segs = reinterpret_cast<const StreamSegment *>(ctx->ws + ctx->off_stream_segs);
-  for (int c = 0; c <= ctx->decode_grid; ++c) sp.cta_seg_begin[c] = ctx->stream_cta_begin[size_t(c) * kWarps];
+  sp.segs = reinterpret_cast<const StreamSegment *>(ctx->ws + ctx->off_stream_segs) + sc.seg_base;
+  for (int c = 0; c <= ctx->decode_grid; ++c) sp.cta_seg_begin[c] = sc.range_begin[size_t(c) * kWarps];
   sp.tmaps = reinterpret_cast<const CUtensorMap_st *>(ctx->ws + ctx->off_tmaps);
   sp.max_segs = ctx->stream_max_segs;
   sp.heads_contiguous = ctx->stream_heads_contiguous ? 1 : 0;

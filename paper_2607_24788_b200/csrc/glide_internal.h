@@ -69,6 +69,7 @@ struct DecodeParams {
   int32_t rec_floats;        // floats per partial record: G * (d + 2) rounded up to 4
   float scale_log2;          // softmax_scale * log2(e)
   int64_t t_host;            // position of the token being decoded as the host tracks it (= device counter)
+  int32_t layer_begin, layer_count;   // layers of this launch; q, k, v, out are indexed with the absolute layer
 };
 
 constexpr int kMaxStreamCtas = 192;           // CTAs (one per SM) the streaming decode kernel's schedule can address
@@ -139,8 +140,14 @@ struct glide_ctx {
   std::vector<int64_t> n_host;      // mirror of the device counters
   std::vector<unsigned char> tmaps_host;  // TMA descriptors of the rings (bf16 tensor-core decode kernel)
   int decode_kind = 0;              // 0 CUDA-core kernel, 1 per-item tensor-core kernel, 2 streaming tensor-core kernel
-  std::vector<glide::StreamSegment> stream_segs;
-  std::vector<int32_t> stream_cta_begin;
+  // schedules of the streaming kernel: [0] all layers; [1 + l] layer l alone (built when L > 1)
+  struct StreamSchedule {
+    size_t seg_base = 0;                 // index of its first segment in the device array
+    size_t n_segs = 0;
+    std::vector<int32_t> range_begin;    // first segment of every warp range, relative to seg_base
+  };
+  std::vector<StreamSchedule> stream_scheds;
+  std::vector<glide::StreamSegment> stream_segs;   // all schedules, concatenated (host copy of the device array)
   int stream_max_segs = 0;
   bool stream_heads_contiguous = true;
   bool tmaps_kv4d = false;
@@ -171,15 +178,17 @@ namespace glide {
 // Layout planning shared by glide_workspace_bytes and glide_create (host only).
 int plan_context(const glide_config *cfg, glide_ctx *ctx, std::vector<WorkItem> *items);
 
-DecodeParams make_decode_params(const glide_ctx *ctx, const void *q, const void *k, const void *v, void *out);
+DecodeParams make_decode_params(const glide_ctx *ctx, int layer_begin, int layer_count, const void *q, const void *k,
+                                const void *v, void *out);
 int build_ring_tensor_maps(glide_ctx *ctx);   // TMA descriptors of every layer's K and V ring (host copy)
 int mma_decode_setup(glide_ctx *ctx);         // sizes the grid of the per-item tensor-core kernel
 int stream_decode_supported(const glide_ctx *ctx);
 int stream_decode_setup(glide_ctx *ctx);      // builds the static schedule (host copy) and sizes the launch
-int launch_decode_stream(glide_ctx *ctx, const DecodeParams &p, cudaStream_t stream);
+int launch_decode_stream(glide_ctx *ctx, const DecodeParams &p, int schedule, cudaStream_t stream);
 int launch_decode_mma(glide_ctx *ctx, const DecodeParams &p, cudaStream_t stream);
 int launch_decode_noalloc(glide_ctx *ctx, const void *q, const void *k, const void *v, void *out, cudaStream_t stream);
-int launch_decode(glide_ctx *ctx, const void *q, const void *k, const void *v, void *out, cudaStream_t stream);
+int launch_decode(glide_ctx *ctx, int layer_begin, int layer_count, const void *q, const void *k, const void *v, void *out,
+                  cudaStream_t stream);
 int decode_occupancy(const glide_ctx *ctx, int *blocks_per_sm);
 int launch_prefill(glide_ctx *ctx, int layer_begin, int layer_count, int64_t T, const void *q, const void *k,
                    const void *v, void *out, cudaStream_t stream);

@@ -71,6 +71,7 @@ def load_library() -> ctypes.CDLL:
     lib.glide_prefill.argtypes = [vp, i32, i32, i64, vp, vp, vp, vp, vp]
     lib.glide_decode_step.argtypes = [vp, vp, vp, vp, vp, vp]
     lib.glide_decode_step_noalloc.argtypes = [vp, vp, vp, vp, vp, vp]
+    lib.glide_decode_step_layers.argtypes = [vp, i32, i32, vp, vp, vp, vp, vp]
     lib.glide_destroy.argtypes = [vp]
     lib.glide_layer_info.argtypes = [vp, i32, vp, ctypes.POINTER(glide_layer_info_t)]
     lib.glide_export_state.argtypes = [vp, i32, vp, vp, vp, vp, vp]
@@ -81,7 +82,7 @@ def load_library() -> ctypes.CDLL:
     lib.glide_strerror.argtypes = [ctypes.c_int]
     lib.glide_strerror.restype = ctypes.c_char_p
     for name in ("glide_workspace_bytes", "glide_create", "glide_prefill", "glide_decode_step", "glide_destroy",
-                 "glide_decode_step_noalloc",
+                 "glide_decode_step_noalloc", "glide_decode_step_layers",
                  "glide_layer_info", "glide_export_state", "glide_import_state", "glide_reset",
                  "glide_device_status", "glide_decode_launch_info"):
         getattr(lib, name).restype = ctypes.c_int
@@ -151,9 +152,12 @@ class Glide:
         self.cfg, self._keep = make_config(windows, batch, n_q_heads, n_kv_heads, head_dim, max_tokens, dtype, **kw)
         self.workspace_bytes = glide_workspace_bytes(self.cfg)
         with torch.cuda.device(self.device):
-            self.workspace = torch.empty(self.workspace_bytes + 256, dtype=torch.uint8, device=self.device)
+            # 256-byte alignment is required; 2 MiB keeps the library's own 2 MiB-aligned offsets of the streamed
+            # arrays aligned in device memory as well
+            align = 2 << 20
+            self.workspace = torch.empty(self.workspace_bytes + align, dtype=torch.uint8, device=self.device)
             base = self.workspace.data_ptr()
-            self._ws_ptr = (base + 255) // 256 * 256
+            self._ws_ptr = (base + align - 1) // align * align
             handle = ctypes.c_void_p()
             _check(self.lib.glide_create(ctypes.byref(self.cfg), self._ws_ptr, self.workspace_bytes, _stream(None),
                                          ctypes.byref(handle)), "glide_create")
@@ -178,6 +182,15 @@ class Glide:
         assert q.dtype == k.dtype == v.dtype == out.dtype == self.dtype
         _check(self.lib.glide_decode_step(self._h, _ptr(q), _ptr(k), _ptr(v), _ptr(out), _stream(stream)),
                "glide_decode_step")
+
+    def glide_decode_step_layers(self, q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, out: torch.Tensor,
+                                 layer_begin: int, layer_count: int, stream=None) -> None:
+        """glide_decode_step for the layers [layer_begin, layer_begin + layer_count); tensors are the range's."""
+        assert q.shape == (layer_count, self.B, self.H, self.d) and out.shape == q.shape
+        assert k.shape == (layer_count, self.B, self.Hkv, self.d) and v.shape == k.shape
+        assert q.dtype == k.dtype == v.dtype == out.dtype == self.dtype
+        _check(self.lib.glide_decode_step_layers(self._h, int(layer_begin), int(layer_count), _ptr(q), _ptr(k), _ptr(v),
+                                                 _ptr(out), _stream(stream)), "glide_decode_step_layers")
 
     def glide_decode_step_noalloc(self, q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, out: torch.Tensor,
                                   stream=None) -> None:

@@ -179,3 +179,39 @@ def test_sum_of_terms_merges_need_the_cuda_core_kernels():
         glide.Glide([64], 1, 8, 2, 128, 256, dtype=BF16, merge=1, decode_impl=3)
     with pytest.raises(glide.GlideError):
         glide.Glide([64], 1, 8, 2, 128, 256, dtype=BF16, merge=2, prefill_impl=2)
+
+
+@pytest.mark.parametrize("dtype,d,impl", [(BF16, 128, 0), (BF16, 128, 1), (BF16, 64, 0), (F32, 64, 0)])
+def test_decode_step_layers(dtype, d, impl):
+    # layer by layer, in ranges, and for the whole stack, interleaved: every path against the oracle, and the
+    # positions of the layers bit-exact afterwards (streaming kernel, per-item tensor-core kernel, CUDA-core kernel)
+    import numpy as np
+    from paper_2607_24788_b200 import glide, synth
+    from oracle import glide_oracle as orc
+    from tests.parity_util import f32_scale, to_np, check_outputs, check_state
+    windows, B, H, Hkv = [40, 0, 16, 300, 1 << 20], 2, 8, 2
+    L = len(windows)
+    amp = 1.0 if dtype == F32 else d ** -0.5 * 4
+    wl = synth.Workload(3, L, B, H, Hkv, d, dtype, amp)
+    g = glide.Glide(windows, B, H, Hkv, d, 128, dtype=dtype, softmax_scale=f32_scale(d), decode_impl=impl)
+    stack = orc.Stack(windows, B, H, Hkv, d, f32_scale(d))
+    q, k, v = wl.qkv(range(L), range(B), range(0, 50), device="cuda")
+    g.glide_prefill(None, k, v, None)
+    stack.prefill(None, to_np(k), to_np(v), outputs=False)
+    for t in range(50, 62):
+        q, k, v = wl.decode_qkv(t, "cuda")
+        out = torch.full_like(q, float("nan"))
+        ref = stack.decode(to_np(q), to_np(k), to_np(v))
+        if t % 3 == 0:
+            g.glide_decode_step(q, k, v, out)
+        elif t % 3 == 1:
+            for l in range(L):
+                g.glide_decode_step_layers(q[l:l + 1], k[l:l + 1], v[l:l + 1], out[l:l + 1], l, 1)
+        else:
+            g.glide_decode_step_layers(q[3:5], k[3:5], v[3:5], out[3:5], 3, 2)
+            with pytest.raises(glide.GlideError):      # layers 3, 4 are ahead of the others now
+                g.glide_decode_step(q, k, v, out)
+            g.glide_decode_step_layers(q[0:3], k[0:3], v[0:3], out[0:3], 0, 3)
+        check_outputs(out, ref, dtype, f"step {t}")
+    check_state(g, stack, "after mixed steps")
+    assert g.glide_device_status() == 0
