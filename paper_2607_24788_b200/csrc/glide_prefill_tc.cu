@@ -288,10 +288,19 @@ prefill_attn_tc_kernel(const PrefillParams p, const CUtensorMap *ring_maps, cons
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], 512;" ::"r"(smem_u32(&sm.tmem_base)) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
-  // K/V buffers start at zero: token groups past the CTA's last token are never loaded, and what a masked key's
-  // V row holds is multiplied by a zero weight, so it has to be finite
-  for (int i = tid; i < int(kStages * kTileBytes / 16); i += kThreads)
-    reinterpret_cast<uint4 *>(&sm.kv[0][0])[i] = make_uint4(0u, 0u, 0u, 0u);
+  // Token groups past the CTA's last token are never loaded (only the last tile has such groups), and what a
+  // masked key's V row holds is multiplied by a zero weight, so it has to be finite: those rows of the buffer that
+  // will hold the last V tile start at zero (earlier tiles that pass through the buffer leave real rows behind).
+  if (n_tiles > 0) {
+    const int last_slot = (2 * (n_tiles - 1) + 1) % kStages;
+    const int64_t j0_last = j_lo + int64_t(n_tiles - 1) * kKT;
+    const int first_skipped = int((tq_last - j0_last) / kGroup) + 1;   // groups [first_skipped, 8) are not loaded
+    const int n16 = (kKT / kGroup - first_skipped) * int(kGroupBytes / 16);
+    for (int half = 0; half < 2; ++half) {
+      uint4 *dst = reinterpret_cast<uint4 *>(&sm.kv[last_slot][half * kBoxBytes + first_skipped * kGroupBytes]);
+      for (int i = tid; i < n16; i += kThreads) dst[i] = make_uint4(0u, 0u, 0u, 0u);
+    }
+  }
   fence_async_smem();
   tc_fence_before();
   __syncthreads();
@@ -312,8 +321,6 @@ prefill_attn_tc_kernel(const PrefillParams p, const CUtensorMap *ring_maps, cons
   const uint32_t tS = tmem + (uint32_t((warp & 3) * 32) << 16) + uint32_t(X) * 128u;
   const uint32_t tO = tS + 256u;
   float m_ref = -CUDART_INF_F, l_sum = 0.f;
-  const bf16 *qrow = reinterpret_cast<const bf16 *>(p.q) +
-                     ((seq + size_t(p.c0 + (tok_r < ntokX ? tl : tok0))) * p.H + p.heads_of[g * G + hh]) * kD;
 
   // multiply this thread's O row by f (warp-collective TMEM read-modify-write)
   auto scale_o = [&](float f) {
@@ -536,9 +543,10 @@ prefill_attn_tc_kernel(const PrefillParams p, const CUtensorMap *ring_maps, cons
       const float fl = ex2(-M);
       if (o_init && __any_sync(0xffffffffu, fw != 1.f)) scale_o(fw);
       l_sum *= fw;
+      // this row of Q is still in the shared tile (every S product has completed)
 #pragma unroll
       for (int i = 0; i < kD / 8; ++i) {
-        const uint4 v4 = *reinterpret_cast<const uint4 *>(qrow + i * 8);
+        const uint4 v4 = *reinterpret_cast<const uint4 *>(sm.q[X] + sw128(row, i));
         phq[i * 4 + 0] = v4.x;
         phq[i * 4 + 1] = v4.y;
         phq[i * 4 + 2] = v4.z;
@@ -548,15 +556,21 @@ prefill_attn_tc_kernel(const PrefillParams p, const CUtensorMap *ring_maps, cons
 #pragma unroll
       for (int i = 0; i < kD / 2; ++i)
         mx = fmaxf(mx, fmaxf(__uint_as_float(phq[i] << 16), __uint_as_float(phq[i] & 0xffff0000u)));
-      float sum = 0.f;
+      // one pass of exponentials: kept as packed bf16, normalised by the sum of the unrounded values afterwards
+      float sum0 = 0.f, sum1 = 0.f;
+      const float mxl = mx * kLog2e;
+#pragma unroll
+      for (int i = 0; i < kD / 2; ++i) {
+        const float e0 = ex2(fmaf(__uint_as_float(phq[i] << 16), kLog2e, -mxl));
+        const float e1 = ex2(fmaf(__uint_as_float(phq[i] & 0xffff0000u), kLog2e, -mxl));
+        sum0 += e0;
+        sum1 += e1;
+        phq[i] = pack_bf16x2(e0, e1);
+      }
+      const float sc = fl * __frcp_rn(sum0 + sum1);
 #pragma unroll
       for (int i = 0; i < kD / 2; ++i)
-        sum += ex2((__uint_as_float(phq[i] << 16) - mx) * kLog2e) + ex2((__uint_as_float(phq[i] & 0xffff0000u) - mx) * kLog2e);
-      const float sc = fl * __frcp_rn(sum);
-#pragma unroll
-      for (int i = 0; i < kD / 2; ++i)
-        phq[i] = pack_bf16x2(ex2((__uint_as_float(phq[i] << 16) - mx) * kLog2e) * sc,
-                             ex2((__uint_as_float(phq[i] & 0xffff0000u) - mx) * kLog2e) * sc);
+        phq[i] = pack_bf16x2(__uint_as_float(phq[i] << 16) * sc, __uint_as_float(phq[i] & 0xffff0000u) * sc);
 #pragma unroll
       for (int c = 0; c < 16; ++c)
         *reinterpret_cast<uint4 *>(sm.q[X] + sw128(row, c)) = make_uint4(phq[c * 4], phq[c * 4 + 1], phq[c * 4 + 2], phq[c * 4 + 3]);
