@@ -484,12 +484,6 @@ def measure_prefill(ctx, wl, shape, n_tokens, device):
     """glide_prefill with outputs for n_tokens more tokens on every layer (best of 3, CUDA events)."""
     L, B, H, d = shape.n_layers, shape.batch, shape.n_q_heads, shape.head_dim
     n = ctx.glide_layer_info(0)["n"]
-    # chunked prefill in serving starts on chunk boundaries; the tcgen05 kernel wants a multiple of 16 tokens, so a
-    # few more decode steps bring this context there
-    while n % 16:
-        qd, kd, vd = wl.decode_qkv(n, device)
-        ctx.glide_decode_step(qd, kd, vd, torch.empty_like(qd))
-        n += 1
     if n + 3 * n_tokens > ctx.max_tokens:
         return None
     q, k, v = wl.qkv(range(L), range(B), range(n, n + n_tokens), device=device)

@@ -73,10 +73,8 @@ typedef enum { GLIDE_MERGE_SHARED = 0, GLIDE_MERGE_SUM_EVICTED = 1, GLIDE_MERGE_
 typedef enum { GLIDE_DECODE_AUTO = 0, GLIDE_DECODE_MMA = 1, GLIDE_DECODE_FMA = 2, GLIDE_DECODE_STREAM = 3 } glide_decode_impl;
 
 /* Kernel that computes the prefill outputs (bf16 I/O).  AUTO picks the fastest that applies.  MMA_SYNC and
- * TCGEN05 need head_dim 128; TCGEN05 also needs, per call, a start position (tokens absorbed so far) that is a
- * multiple of 16 and ring sizes of the evicting layers that are multiples of 16, and falls back to MMA_SYNC for
- * a call where that does not hold.  For fp32 I/O only the CUDA-core kernel exists.  State, ring and counters do
- * not depend on the choice. */
+ * TCGEN05 need head_dim 128.  For fp32 I/O only the CUDA-core kernel exists.  State, ring and counters do not
+ * depend on the choice. */
 typedef enum { GLIDE_PREFILL_AUTO = 0, GLIDE_PREFILL_MMA_SYNC = 1, GLIDE_PREFILL_TCGEN05 = 2, GLIDE_PREFILL_FMA = 3 } glide_prefill_impl;
 
 typedef struct {

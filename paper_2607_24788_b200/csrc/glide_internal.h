@@ -192,7 +192,7 @@ int launch_decode(glide_ctx *ctx, int layer_begin, int layer_count, const void *
 int decode_occupancy(const glide_ctx *ctx, int *blocks_per_sm);
 int launch_prefill(glide_ctx *ctx, int layer_begin, int layer_count, int64_t T, const void *q, const void *k,
                    const void *v, void *out, cudaStream_t stream);
-bool prefill_attn_tc_supported(const glide_ctx *ctx, int layer_begin, int layer_count, int64_t n0);
+bool prefill_attn_tc_supported(const glide_ctx *ctx);
 int launch_prefill_attn_tc(glide_ctx *ctx, const PrefillParams &p, cudaStream_t stream);
 bool prefill_attn_mma_supported(const glide_ctx *ctx);
 int launch_prefill_attn_mma(glide_ctx *ctx, const PrefillParams &p, cudaStream_t stream);

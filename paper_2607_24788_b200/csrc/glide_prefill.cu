@@ -372,9 +372,9 @@ int launch_prefill(glide_ctx *ctx, int layer_begin, int layer_count, int64_t T, 
   if (impl == GLIDE_PREFILL_AUTO)
     impl = (prefill_attn_mma_supported(ctx) && ctx->cfg.decode_impl != GLIDE_DECODE_FMA && ctx->cfg.merge == GLIDE_MERGE_SHARED)
                ? GLIDE_PREFILL_TCGEN05 : GLIDE_PREFILL_FMA;
-  // the tcgen05 kernel has alignment conditions that depend on the call; where they do not hold the call falls
-  // back to the mma.sync kernel
-  const bool use_tc = impl == GLIDE_PREFILL_TCGEN05 && prefill_attn_tc_supported(ctx, layer_begin, layer_count, p.n0);
+  // the tcgen05 kernel needs the ring descriptors of the tensor-core decode kernels (absent when decode_impl asks
+  // for the CUDA-core kernel); without them the call uses the mma.sync kernel
+  const bool use_tc = impl == GLIDE_PREFILL_TCGEN05 && prefill_attn_tc_supported(ctx);
   const bool use_mma = (impl == GLIDE_PREFILL_MMA_SYNC || (impl == GLIDE_PREFILL_TCGEN05 && !use_tc)) && prefill_attn_mma_supported(ctx);
   bool any_evicts = false;
   for (int l = layer_begin; l < layer_begin + layer_count; ++l) any_evicts = any_evicts || ctx->layers[l].evicts;

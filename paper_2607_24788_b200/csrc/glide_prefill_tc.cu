@@ -271,7 +271,7 @@ prefill_attn_tc_kernel(const PrefillParams p, const CUtensorMap *ring_maps, cons
 
   if (tid == 0) {
     for (int s = 0; s < kStages; ++s) {
-      mbar_init(smem_u32(&sm.bar_full[s]), 1);
+      mbar_init(smem_u32(&sm.bar_full[s]), 2);
       mbar_init(smem_u32(&sm.bar_free[s]), 1);
     }
     for (int x = 0; x < 2; ++x) {
@@ -482,10 +482,18 @@ prefill_attn_tc_kernel(const PrefillParams p, const CUtensorMap *ring_maps, cons
       if (ok) mma_commit(smem_u32(&sm.bar_done));
     }
   } else if (warp == kLoadWarp) {
-    // lane gi issues the two boxes (column halves) of token group gi of the tile: the address arithmetic of the
-    // eight groups runs in parallel instead of as one long dependent chain
+    // A 128-key tile is eight groups of 16 tokens.  A group that lies in one source (ring or call) and is contiguous
+    // there is fetched by TMA, lane gi issuing the two boxes (column halves) of group gi so that the address
+    // arithmetic of the groups runs in parallel.  A group that straddles the call boundary or a ring wrap is copied
+    // row by row by the whole warp (at most a few per tile).  Each buffer's barrier takes two arrivals: the
+    // expect-tx one before the TMA boxes are issued and a plain one after the row copies.
     if (n_tiles > 0) {
       const CUtensorMap *ringK = ring_maps + 3 * layer, *ringV = ringK + 1;
+      const bf16 *ringKp = reinterpret_cast<const bf16 *>(p.ws + ld.ringK) + unit_rows * kD;
+      const bf16 *ringVp = reinterpret_cast<const bf16 *>(p.ws + ld.ringV) + unit_rows * kD;
+      const bf16 *callKp = reinterpret_cast<const bf16 *>(p.k) + (seq * p.Hkv + g) * kD;
+      const bf16 *callVp = reinterpret_cast<const bf16 *>(p.v) + (seq * p.Hkv + g) * kD;
+      const int64_t call_stride = int64_t(p.Hkv) * kD;
       const int gi = lane;
       bool ok = true;
       for (int sq = 0; sq < 2 * n_tiles; ++sq) {
@@ -497,23 +505,49 @@ prefill_attn_tc_kernel(const PrefillParams p, const CUtensorMap *ring_maps, cons
         const int64_t left = tq_last - j0;                       // >= 0: the tile holds at least one valid token
         const int ngroups = left >= kKT - 1 ? kKT / kGroup : int(left / kGroup) + 1;
         const uint32_t bar = smem_u32(&sm.bar_full[slot]);
-        if (lane == 0) mbar_expect_tx(bar, uint32_t(ngroups) * 2u * kGroupBytes);
+        // this lane's group: where it comes from and whether one box covers it
+        const int64_t j = j0 + gi * kGroup;
+        const bool mine = gi < ngroups;
+        const bool from_call = j >= p.n0;
+        const uint32_t slot_row = (j >> 32) == 0 ? uint32_t(j) % cap : uint32_t(uint64_t(j) % cap);
+        const bool boxed = mine && (from_call || (j + kGroup <= p.n0 && slot_row + kGroup <= cap));
+        const unsigned boxed_mask = __ballot_sync(0xffffffffu, boxed);
+        const unsigned manual_mask = __ballot_sync(0xffffffffu, mine && !boxed);
+        if (lane == 0) mbar_expect_tx(bar, uint32_t(__popc(boxed_mask)) * 2u * kGroupBytes);
         __syncwarp();
-        if (gi < ngroups) {
-          const int64_t j = j0 + gi * kGroup;
+        if (boxed) {
           const uint32_t dst = kv_addr(slot) + uint32_t(gi) * kGroupBytes;
-          if (j >= p.n0) {      // the call's own rows
+          if (from_call) {
             const CUtensorMap *m = is_v ? &cm.v : &cm.k;
             tma_load_4d(dst, m, 0, g, int(j - p.n0), lrel * p.B + b, bar);
             tma_load_4d(dst + kBoxBytes, m, 64, g, int(j - p.n0), lrel * p.B + b, bar);
-          } else {              // ring rows: a 16-token group never wraps (ring sizes are multiples of 16 where rings wrap)
+          } else {
             const CUtensorMap *m = is_v ? ringV : ringK;
-            const uint32_t slot_row = (j >> 32) == 0 ? uint32_t(j) % cap : uint32_t(uint64_t(j) % cap);
             const int y = int(unit_rows + slot_row);
             tma_load_2d(dst, m, 0, y, bar);
             tma_load_2d(dst + kBoxBytes, m, 64, y, bar);
           }
         }
+        for (unsigned mm = manual_mask; mm; mm &= mm - 1) {
+          const int gm = __ffs(int(mm)) - 1;
+          unsigned char *tile = sm.kv[slot];
+#pragma unroll
+          for (int i = 0; i < kGroup * 16 / 32; ++i) {
+            const int id = lane + 32 * i;
+            const int r = id >> 4, c = id & 15;
+            const int64_t jj = j0 + gm * kGroup + r;
+            uint4 val = make_uint4(0u, 0u, 0u, 0u);
+            if (jj <= tq_last) {
+              const bf16 *src = jj >= p.n0 ? (is_v ? callVp : callKp) + size_t(jj - p.n0) * call_stride
+                                           : (is_v ? ringVp : ringKp) + size_t(uint64_t(jj) % cap) * kD;
+              val = *reinterpret_cast<const uint4 *>(src + c * 8);
+            }
+            *reinterpret_cast<uint4 *>(tile + sw128(gm * kGroup + r, c)) = val;
+          }
+        }
+        fence_async_smem();   // the row copies are read by the tensor core (async proxy)
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar);
       }
     }
   }
@@ -732,17 +766,9 @@ extern "C" int glide_debug_tc_profile(long long *out16, int reset) {
 }
 #endif
 
-// The kernel needs the ring descriptors made for the tensor-core decode kernels, 16-token TMA boxes that never
-// straddle the call boundary (tokens absorbed so far a multiple of 16) or a ring wrap (ring sizes of evicting
-// layers multiples of 16).
-bool prefill_attn_tc_supported(const glide_ctx *ctx, int layer_begin, int layer_count, int64_t n0) {
-  if (ctx->cfg.io_dtype != GLIDE_BF16 || ctx->cfg.head_dim != kD || ctx->decode_kind < 1) return false;
-  if (n0 % kGroup != 0 || ctx->prefill_chunk % kGroup != 0) return false;
-  for (int l = layer_begin; l < layer_begin + layer_count; ++l) {
-    const LayerDev &ld = ctx->layers[size_t(l)];
-    if (ld.cap > 0 && ld.evicts && ld.cap % kGroup != 0) return false;
-  }
-  return true;
+// The kernel needs the ring descriptors made for the tensor-core decode kernels.
+bool prefill_attn_tc_supported(const glide_ctx *ctx) {
+  return ctx->cfg.io_dtype == GLIDE_BF16 && ctx->cfg.head_dim == kD && ctx->decode_kind >= 1;
 }
 
 namespace {

@@ -215,3 +215,31 @@ def test_decode_step_layers(dtype, d, impl):
         check_outputs(out, ref, dtype, f"step {t}")
     check_state(g, stack, "after mixed steps")
     assert g.glide_device_status() == 0
+
+
+def test_bf16_prefill_tcgen05_after_decode_steps():
+    # a prompt, a few decode steps, then another prompt (a second turn): the second call starts at a position that
+    # is not a multiple of 16 and its first key tiles mix ring rows, wrapped ring rows and the call's rows
+    from paper_2607_24788_b200 import glide, synth
+    from oracle import glide_oracle as orc
+    from tests.parity_util import f32_scale, to_np, check_outputs, check_state
+    windows, B, H, Hkv, d = [24, 100, 150, 1 << 20, 0], 2, 8, 2, 128
+    L = len(windows)
+    wl = synth.Workload(17, L, B, H, Hkv, d, BF16, d ** -0.5 * 4)
+    g = glide.Glide(windows, B, H, Hkv, d, 600, dtype=BF16, softmax_scale=f32_scale(d), prefill_impl=2)
+    stack = orc.Stack(windows, B, H, Hkv, d, f32_scale(d))
+    pos = 0
+    for T, n_dec in ((173, 5), (140, 3), (64, 0)):
+        q, k, v = wl.qkv(range(L), range(B), range(pos, pos + T), device="cuda")
+        out = torch.full_like(q, float("nan"))
+        g.glide_prefill(q, k, v, out)
+        check_outputs(out, stack.prefill(to_np(q), to_np(k), to_np(v)), BF16, f"prefill@{pos}+{T}")
+        pos += T
+        for _ in range(n_dec):
+            q, k, v = wl.decode_qkv(pos, "cuda")
+            out = torch.empty_like(q)
+            g.glide_decode_step(q, k, v, out)
+            check_outputs(out, stack.decode(to_np(q), to_np(k), to_np(v)), BF16, f"decode@{pos}")
+            pos += 1
+    check_state(g, stack, "after two turns")
+    assert g.glide_device_status() == 0
