@@ -97,6 +97,7 @@ int glide::plan_context(const glide_config *cfg, glide_ctx *ctx, std::vector<Wor
   const int splits = cfg->decode_state_splits ? std::min<int>(cfg->decode_state_splits, d) : (d == 128 ? 4 : 2);
   const int64_t units_per_layer = int64_t(B) * Hkv;
 
+  if (int64_t(L) * units_per_layer > (int64_t(1) << 30)) return GLIDE_ERR_UNSUPPORTED;   // unit indices are 32-bit
   ctx->layers.assign(L, LayerDev{});
   size_t part_floats = 0;
   int64_t n_items = 0;
@@ -104,6 +105,8 @@ int glide::plan_context(const glide_config *cfg, glide_ctx *ctx, std::vector<Wor
     LayerDev &ld = ctx->layers[l];
     ld.w = ctx->windows[l];
     ld.cap = std::min<int64_t>(ld.w, cfg->max_tokens);
+    // ring rows of a layer are addressed with 32-bit TMA coordinates and 32-bit row indices in the schedules
+    if (units_per_layer * ld.cap > int64_t(INT32_MAX) - 1024) return GLIDE_ERR_UNSUPPORTED;
     ld.merge = cfg->merge;
     ld.wlin = cfg->merge == GLIDE_MERGE_SUM_ALL ? 0 : ld.w;
     ld.evicts = ld.wlin < cfg->max_tokens ? 1 : 0;
