@@ -9,6 +9,12 @@
 
 using namespace glide;
 
+#ifndef GLIDE_RING_SKEW_BYTES
+#define GLIDE_RING_SKEW_BYTES 66816          // 65 KiB + 1280 B
+#endif
+#ifndef GLIDE_RING_SKEW_MIN_BYTES
+#define GLIDE_RING_SKEW_MIN_BYTES (size_t(1) << 30)
+#endif
 #ifndef GLIDE_STATE_ALIGN
 #define GLIDE_STATE_ALIGN (2u << 20)
 #endif
@@ -164,6 +170,14 @@ int glide::plan_context(const glide_config *cfg, glide_ctx *ctx, std::vector<Wor
   }
   ctx->state_bytes = off - ctx->off_state;
   off = align_up(off, 256);
+  {
+    // Where the rings start relative to the 2 MiB-aligned state is worth 1-2 % of the decode bandwidth, in opposite
+    // directions for small and large contexts (measured: B = 1 / 115 MB of rings is 1.5 % faster with the rings
+    // aligned, B = 16 / 1.8 GB and B = 4 / 4.2 GB are 0.8 % and 2 % faster with them 65 KiB + 1280 B further on).
+    size_t ring_total = 0;
+    for (int l = 0; l < L; ++l) ring_total += 2 * size_t(units_per_layer) * size_t(ctx->layers[l].cap) * d * ctx->elem;
+    if (ring_total >= GLIDE_RING_SKEW_MIN_BYTES) off += size_t(GLIDE_RING_SKEW_BYTES);
+  }
   ctx->off_ring = off;
   for (int l = 0; l < L; ++l) {
     size_t bytes = align_up(size_t(units_per_layer) * size_t(ctx->layers[l].cap) * d * ctx->elem, 256);
