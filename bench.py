@@ -226,11 +226,11 @@ def build_states(shape, n_replicas: int, extra_tokens: int, device):
 def decode_kernel_name(shape) -> str:
     """The kernel glide_create selects for this shape and these knobs (see include/glide.h)."""
     impl, merge = KERNEL_KNOBS.get("decode_impl", 0), KERNEL_KNOBS.get("merge", 0)
-    if shape.dtype == "f32" or impl == 2 or merge != 0:
+    if shape.dtype == "f32" or impl == 2:
         return "glide_decode_kernel"
     if shape.head_dim == 128 and impl in (0, 3):
         return "glide_decode_stream_kernel"
-    return "glide_decode_mma_kernel"
+    return "glide_decode_mma_kernel" if merge == 0 else "glide_decode_kernel"
 
 
 def max_over_ranks(values, dist, device):
@@ -520,7 +520,7 @@ def main():
     ap.add_argument("--prefill-impl", type=int, default=0, help="0 auto, 1 mma.sync, 2 tcgen05 + TMEM, 3 CUDA cores")
     ap.add_argument("--merge", type=int, default=0,
                     help="0 shared normaliser (the paper's default), 1 / 2 the appendix' sums of two normalised terms "
-                         "(evicted-token / all-token state; CUDA-core kernels)")
+                         "(evicted-token / all-token state)")
     args = ap.parse_args()
     shape = configs.ALL[args.workload]
     KERNEL_KNOBS.update(decode_chunk=args.decode_chunk, decode_state_splits=args.state_splits,

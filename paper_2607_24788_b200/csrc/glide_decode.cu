@@ -401,7 +401,7 @@ DecodeParams make_decode_params(const glide_ctx *ctx, int layer_begin, int layer
   p.B = ctx->cfg.batch;
   p.H = ctx->cfg.n_q_heads;
   p.Hkv = ctx->cfg.n_kv_heads;
-  p.rec_floats = ctx->rec_floats;
+  p.rec_floats = ctx->decode_kind == 2 ? ctx->stream_rec_floats : ctx->rec_floats;
   p.scale_log2 = ctx->scale * kLog2e;
   p.t_host = ctx->n_host[size_t(layer_begin)];
   p.layer_begin = layer_begin;
@@ -497,6 +497,7 @@ int launch_decode_noalloc(glide_ctx *ctx, const void *q, const void *k, const vo
   p.ctl = reinterpret_cast<Control *>(scratch);
   p.tickets = reinterpret_cast<int32_t *>(scratch + tickets_off);
   p.partials = reinterpret_cast<float *>(scratch + partials_off);
+  p.rec_floats = ctx->rec_floats;   // this variant always runs the CUDA-core kernel and its record layout
   return dispatch_config(ctx->cfg.io_dtype, ctx->cfg.head_dim, ctx->G, [&](auto tt, auto dd, auto gg) -> int {
     using T = typename decltype(tt)::type;
     constexpr int D = decltype(dd)::value, G = decltype(gg)::value;

@@ -191,7 +191,9 @@ __device__ __forceinline__ void tma_load_4d(uint32_t dst, const void *tmap, int 
 }
 
 __device__ __forceinline__ bool seg_evicting(const StreamSegment &s, int64_t t) {
-  return s.evicts && (s.w == 0 || t >= int64_t(s.w));
+  // evicts bit 0: the layer has a state; bit 1: the token folded at a step is the current one (no ring, or a state
+  // that holds every token), otherwise the one that leaves the window
+  return (s.evicts & 1) && ((s.evicts & 2) || t >= int64_t(s.w));
 }
 // window tiles of the segment that hold window tokens at position t
 __device__ __forceinline__ int seg_valid_win(const StreamSegment &s, int64_t t) {
@@ -214,9 +216,13 @@ __device__ __forceinline__ void cursor_enter(Cursor &c, const StreamSegment *seg
   c.n_total = c.n_state_eff + seg_valid_win(s, t);
 }
 
-template <int G>
+// Records.  Shared normaliser: (acc[G][d], m[G], l[G]) with the linear readout already folded in as a term with
+// logit 0.  Sum of two normalised terms (SUM): the window part as above and, kRecW floats further on, the linear
+// part (a[G][d], b[G]) kept apart.
+template <int G, bool SUM = false>
 struct Layout {
-  static constexpr int kRecFloats = (G * kD + 2 * G + 3) / 4 * 4;
+  static constexpr int kRecW = (G * kD + 2 * G + 3) / 4 * 4;
+  static constexpr int kRecFloats = SUM ? 2 * kRecW : kRecW;
   static constexpr uint32_t kHdrBytes = G * 256 + 4 * 256;   // q rows | k_e | v_e | k_t | v_t
 };
 
@@ -261,11 +267,11 @@ __device__ __forceinline__ void warp_sum_multi(float (&x)[N]) {
 }
 
 // ---- the kernel -----------------------------------------------------------------------------
-template <int G, int STAGES>
+template <int G, int STAGES, bool SUM>
 __global__ void __launch_bounds__(kThreads, 1)
 glide_decode_stream_kernel(const DecodeParams p, const StreamParams sp) {
   using bf16 = __nv_bfloat16;
-  using L = Layout<G>;
+  using L = Layout<G, SUM>;
   constexpr int KS = kD / 16;
 
   extern __shared__ __align__(1024) unsigned char smem_raw[];
@@ -351,7 +357,7 @@ glide_decode_stream_kernel(const DecodeParams p, const StreamParams sp) {
       bulk_load(my_hdr + G * 256 + 512, kt, 256, hdr_bar);
       bulk_load(my_hdr + G * 256 + 768, vt, 256, hdr_bar);
       if (ev) {
-        if (sg.w == 0) {   // no ring: the current token is the one folded into the state
+        if (sg.evicts & 2) {   // the current token is the one folded into the state
           bulk_load(my_hdr + G * 256, kt, 256, hdr_bar);
           bulk_load(my_hdr + G * 256 + 256, vt, 256, hdr_bar);
         } else {
@@ -703,8 +709,8 @@ glide_decode_stream_kernel(const DecodeParams p, const StreamParams sp) {
     GLIDE_TRACE_EVENT(18);
     if (n_total > 0) issue_next();   // the deferred refill
     GLIDE_TRACE_EVENT(19);
-    if (n_state_eff > 0) {           // fold the linear readout in as a term with logit 0
-      warp_sum_multi<G>(bp);
+    if (n_state_eff > 0) warp_sum_multi<G>(bp);
+    if (!SUM && n_state_eff > 0) {   // fold the linear readout in as a term with logit 0
 #pragma unroll
       for (int h = 0; h < G; ++h) {
         const float mn = fmaxf(mh[h], 0.f);
@@ -725,9 +731,11 @@ glide_decode_stream_kernel(const DecodeParams p, const StreamParams sp) {
 #pragma unroll
       for (int h = 0; h < G; ++h) {
         *reinterpret_cast<float4 *>(slot + h * kD + lane * 4) = acc[h];
+        if (SUM) *reinterpret_cast<float4 *>(slot + L::kRecW + h * kD + lane * 4) = a[h];
         if (lane == 0) {
           slot[G * kD + h] = mh[h];
           slot[G * kD + G + h] = lh[h];
+          if (SUM) slot[L::kRecW + G * kD + h] = bp[h];
         }
       }
       __syncwarp();
@@ -777,6 +785,27 @@ glide_decode_stream_kernel(const DecodeParams p, const StreamParams sp) {
           }
         }
       }
+      if (SUM) {   // the linear parts of the group's records simply add up
+#pragma unroll
+        for (int h = 0; h < G; ++h) {
+          a[h] = make_float4(0.f, 0.f, 0.f, 0.f);
+          bp[h] = 0.f;
+        }
+#pragma unroll
+        for (int i = 0; i < kWarps; ++i) {
+          if (i < sg.grp_size) {
+#pragma unroll
+            for (int h = 0; h < G; ++h) {
+              const float4 av = *reinterpret_cast<const float4 *>(g0 + size_t(i) * L::kRecFloats + L::kRecW + h * kD + lane * 4);
+              a[h].x += av.x;
+              a[h].y += av.y;
+              a[h].z += av.z;
+              a[h].w += av.w;
+              bp[h] += g0[size_t(i) * L::kRecFloats + L::kRecW + G * kD + h];
+            }
+          }
+        }
+      }
       GLIDE_TRACE_EVENT(22);
     }
     if (sg.part >= 0) {
@@ -786,9 +815,11 @@ glide_decode_stream_kernel(const DecodeParams p, const StreamParams sp) {
 #pragma unroll
       for (int h = 0; h < G; ++h) {
         *reinterpret_cast<float4 *>(grec + h * kD + lane * 4) = acc[h];
+        if (SUM) *reinterpret_cast<float4 *>(grec + L::kRecW + h * kD + lane * 4) = a[h];
         if (lane == 0) {
           grec[G * kD + h] = mh[h];
           grec[G * kD + G + h] = lh[h];
+          if (SUM) grec[L::kRecW + G * kD + h] = bp[h];
         }
       }
       if (n_pending == 0) pend0 = s; else pend1 = s;
@@ -803,12 +834,18 @@ glide_decode_stream_kernel(const DecodeParams p, const StreamParams sp) {
       vx[3] = __uint_as_float(vt_bits.y & 0xffff0000u);
 #pragma unroll
       for (int h = 0; h < G; ++h) {
-        const float Mf = fmaxf(fmaxf(mh[h], scur[h]), 0.f);
+        // shared normaliser: reference max(window max, 0); sum of terms: the window against its own maximum, the
+        // linear term a / b added (an empty term counts as zero)
+        const float Mf = SUM ? fmaxf(mh[h], scur[h]) : fmaxf(fmaxf(mh[h], scur[h]), 0.f);
         const float fr = exp2_or_zero(mh[h], Mf), fc = exp2_or_zero(scur[h], Mf);
-        const float inv = 1.0f / fmaf(lh[h], fr, fc);
+        const float den = fmaf(lh[h], fr, fc);
+        const float inv = (!SUM || den > 0.f) ? 1.0f / den : 0.f;
+        const float il = (SUM && bp[h] > 0.f) ? 1.0f / bp[h] : 0.f;
         const int orow = sg.qrow0 + (sp.heads_contiguous ? h : p.heads_of[sg.g * G + h]);
-        const __nv_bfloat162 lo = __floats2bfloat162_rn(fmaf(acc[h].x, fr, fc * vx[0]) * inv, fmaf(acc[h].y, fr, fc * vx[1]) * inv);
-        const __nv_bfloat162 hi = __floats2bfloat162_rn(fmaf(acc[h].z, fr, fc * vx[2]) * inv, fmaf(acc[h].w, fr, fc * vx[3]) * inv);
+        const __nv_bfloat162 lo = __floats2bfloat162_rn(fmaf(fmaf(acc[h].x, fr, fc * vx[0]), inv, SUM ? a[h].x * il : 0.f),
+                                                        fmaf(fmaf(acc[h].y, fr, fc * vx[1]), inv, SUM ? a[h].y * il : 0.f));
+        const __nv_bfloat162 hi = __floats2bfloat162_rn(fmaf(fmaf(acc[h].z, fr, fc * vx[2]), inv, SUM ? a[h].z * il : 0.f),
+                                                        fmaf(fmaf(acc[h].w, fr, fc * vx[3]), inv, SUM ? a[h].w * il : 0.f));
         uint2 packed;
         packed.x = *reinterpret_cast<const uint32_t *>(&lo);
         packed.y = *reinterpret_cast<const uint32_t *>(&hi);
@@ -950,12 +987,37 @@ glide_decode_stream_kernel(const DecodeParams p, const StreamParams sp) {
       vx[2] = __uint_as_float(vtb.y << 16);
       vx[3] = __uint_as_float(vtb.y & 0xffff0000u);
 #pragma unroll
+      float4 al[G];
+      float bl[G];
+      if (SUM) {   // linear parts of all records: plain sums
+#pragma unroll
+        for (int h = 0; h < G; ++h) {
+          al[h] = make_float4(0.f, 0.f, 0.f, 0.f);
+          bl[h] = 0.f;
+        }
+        for (int i = 0; i < sg.n_parts; ++i) {
+#pragma unroll
+          for (int h = 0; h < G; ++h) {
+            const float4 av = __ldcg(reinterpret_cast<const float4 *>(r0 + size_t(i) * p.rec_floats + L::kRecW + h * kD + lane * 4));
+            al[h].x += av.x;
+            al[h].y += av.y;
+            al[h].z += av.z;
+            al[h].w += av.w;
+            bl[h] += __ldcg(r0 + size_t(i) * p.rec_floats + L::kRecW + G * kD + h);
+          }
+        }
+      }
+#pragma unroll
       for (int h = 0; h < G; ++h) {
-        const float Mf = fmaxf(fmaxf(Mg[h], sc[h]), 0.f);
+        const float Mf = SUM ? fmaxf(Mg[h], sc[h]) : fmaxf(fmaxf(Mg[h], sc[h]), 0.f);
         const float fr = exp2_or_zero(Mg[h], Mf), fc = exp2_or_zero(sc[h], Mf);
-        const float inv = 1.0f / fmaf(lg[h], fr, fc);
-        const __nv_bfloat162 lo = __floats2bfloat162_rn(fmaf(acc[h].x, fr, fc * vx[0]) * inv, fmaf(acc[h].y, fr, fc * vx[1]) * inv);
-        const __nv_bfloat162 hi = __floats2bfloat162_rn(fmaf(acc[h].z, fr, fc * vx[2]) * inv, fmaf(acc[h].w, fr, fc * vx[3]) * inv);
+        const float den = fmaf(lg[h], fr, fc);
+        const float inv = (!SUM || den > 0.f) ? 1.0f / den : 0.f;
+        const float il = (SUM && bl[h] > 0.f) ? 1.0f / bl[h] : 0.f;
+        const __nv_bfloat162 lo = __floats2bfloat162_rn(fmaf(fmaf(acc[h].x, fr, fc * vx[0]), inv, SUM ? al[h].x * il : 0.f),
+                                                        fmaf(fmaf(acc[h].y, fr, fc * vx[1]), inv, SUM ? al[h].y * il : 0.f));
+        const __nv_bfloat162 hi = __floats2bfloat162_rn(fmaf(fmaf(acc[h].z, fr, fc * vx[2]), inv, SUM ? al[h].z * il : 0.f),
+                                                        fmaf(fmaf(acc[h].w, fr, fc * vx[3]), inv, SUM ? al[h].w * il : 0.f));
         uint2 packed;
         packed.x = *reinterpret_cast<const uint32_t *>(&lo);
         packed.y = *reinterpret_cast<const uint32_t *>(&hi);
@@ -981,23 +1043,29 @@ glide_decode_stream_kernel(const DecodeParams p, const StreamParams sp) {
 
 }
 
-template <int G, int STAGES>
+template <int G, int STAGES, bool SUM>
 size_t stream_smem_bytes(int max_segs) {
-  using L = Layout<G>;
+  using L = Layout<G, SUM>;
   return 1024 + size_t(kWarps) * STAGES * kStageBytes + size_t(kWarps) * L::kHdrBytes + size_t(kWarps) * STAGES * 64 +
          size_t(max_segs) * sizeof(StreamSegment) + size_t(kWarps) * (STAGES + 1) * 8 + size_t(kStreamMaxGroups) * 4 +
          size_t(kStreamPoolBytes / (L::kRecFloats * 4)) * L::kRecFloats * 4;
 }
 
+// f(group size, stages, sum-of-terms merge)
 template <typename F>
-int dispatch_stream(int G, F &&f) {
+int dispatch_stream(int G, bool sum, F &&f) {
+#define GLIDE_STREAM_CASE(GG)                                                        \
+  case GG:                                                                           \
+    return sum ? f(IntTag<GG>{}, IntTag<GLIDE_STREAM_STAGES>{}, IntTag<1>{})         \
+               : f(IntTag<GG>{}, IntTag<GLIDE_STREAM_STAGES>{}, IntTag<0>{});
   switch (G) {
-    case 1: return f(IntTag<1>{}, IntTag<GLIDE_STREAM_STAGES>{});
-    case 2: return f(IntTag<2>{}, IntTag<GLIDE_STREAM_STAGES>{});
-    case 4: return f(IntTag<4>{}, IntTag<GLIDE_STREAM_STAGES>{});
-    case 8: return f(IntTag<8>{}, IntTag<GLIDE_STREAM_STAGES>{});
+    GLIDE_STREAM_CASE(1)
+    GLIDE_STREAM_CASE(2)
+    GLIDE_STREAM_CASE(4)
+    GLIDE_STREAM_CASE(8)
     default: return int(GLIDE_ERR_UNSUPPORTED);
   }
+#undef GLIDE_STREAM_CASE
 }
 
 }  // namespace
@@ -1158,7 +1226,7 @@ void build_stream_schedule(const glide_ctx *ctx, int layer_begin, int layer_coun
         sg.row_base = int32_t(ub * ld.cap);
         sg.cap = int32_t(ld.cap);
         sg.w = int32_t(std::min<int64_t>(ld.w, INT32_MAX));
-        sg.evicts = ld.evicts;
+        sg.evicts = ld.evicts ? (ld.wlin == 0 ? 3 : 1) : 0;
         sg.S_off256 = int32_t((ld.S + size_t(ub) * d * d * 4) / 256);
         sg.z_off256 = int32_t((ld.z + size_t(ub) * d * 4) / 256);
         sg.ringK_off256 = int32_t(ld.ringK / 256);
@@ -1191,7 +1259,7 @@ void build_stream_schedule(const glide_ctx *ctx, int layer_begin, int layer_coun
   // Warps of one CTA that share a unit reduce their records in shared memory first (a "group"); only one
   // record per group goes to global scratch, and a unit that lies inside one group never touches it.
   size_t records = 0;
-  const int pool_slots = kStreamPoolBytes / (ctx->rec_floats * 4);
+  const int pool_slots = kStreamPoolBytes / (ctx->stream_rec_floats * 4);
   std::vector<int> cta_slots(size_t(n_ctas) + 1, 0), cta_groups(size_t(n_ctas) + 1, 0);
   for (size_t u = 0; u < unit_segs.size(); ++u) {
     std::vector<size_t> &list = unit_segs[u];
@@ -1264,16 +1332,17 @@ int stream_decode_setup(glide_ctx *ctx) {
     for (int i = 1; i < ctx->G; ++i)
       contiguous = contiguous && ctx->heads_of[size_t(g) * ctx->G + i] == ctx->heads_of[size_t(g) * ctx->G] + i;
   ctx->stream_heads_contiguous = contiguous;
-  return dispatch_stream(ctx->G, [&](auto gg, auto ss) -> int {
+  return dispatch_stream(ctx->G, ctx->cfg.merge != GLIDE_MERGE_SHARED, [&](auto gg, auto ss, auto mm) -> int {
     constexpr int G = decltype(gg)::value, S = decltype(ss)::value;
-    const size_t smem = stream_smem_bytes<G, S>(ctx->stream_max_segs);
+    constexpr bool SUM = decltype(mm)::value != 0;
+    const size_t smem = stream_smem_bytes<G, S, SUM>(ctx->stream_max_segs);
     int dev_max = 0;
     if (cudaDeviceGetAttribute(&dev_max, cudaDevAttrMaxSharedMemoryPerBlockOptin, ctx->device) != cudaSuccess) {
       cudaGetLastError();
       return GLIDE_ERR_CUDA;
     }
     if (smem > size_t(dev_max)) return GLIDE_ERR_UNSUPPORTED;   // too many segments per CTA for the table
-    auto kern = glide_decode_stream_kernel<G, S>;
+    auto kern = glide_decode_stream_kernel<G, S, SUM>;
     // the attribute belongs to the kernel, not to the context: ask for the device maximum so that contexts with
     // different schedules (different table sizes) can be alive together
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, dev_max) != cudaSuccess) {
@@ -1302,8 +1371,9 @@ int launch_decode_stream(glide_ctx *ctx, const DecodeParams &p, int schedule, cu
   sp.max_segs = ctx->stream_max_segs;
   sp.heads_contiguous = ctx->stream_heads_contiguous ? 1 : 0;
   sp.kv4d = ctx->tmaps_kv4d ? 1 : 0;
-  return dispatch_stream(ctx->G, [&](auto gg, auto ss) -> int {
+  return dispatch_stream(ctx->G, ctx->cfg.merge != GLIDE_MERGE_SHARED, [&](auto gg, auto ss, auto mm) -> int {
     constexpr int G = decltype(gg)::value, S = decltype(ss)::value;
+    constexpr bool SUM = decltype(mm)::value != 0;
     cudaLaunchConfig_t cfg{};
     cfg.gridDim = dim3(unsigned(ctx->decode_grid));
     cfg.blockDim = dim3(kThreads);
@@ -1318,7 +1388,7 @@ int launch_decode_stream(glide_ctx *ctx, const DecodeParams &p, int schedule, cu
 #else
     cfg.numAttrs = 1;
 #endif
-    if (cudaLaunchKernelEx(&cfg, glide_decode_stream_kernel<G, S>, p, sp) != cudaSuccess) {
+    if (cudaLaunchKernelEx(&cfg, glide_decode_stream_kernel<G, S, SUM>, p, sp) != cudaSuccess) {
       cudaGetLastError();
       return GLIDE_ERR_CUDA;
     }

@@ -48,9 +48,9 @@ int validate_config(const glide_config *c) {
   if (c->phi != GLIDE_PHI_SOFTMAX) return GLIDE_ERR_UNSUPPORTED;
   if (c->merge < GLIDE_MERGE_SHARED || c->merge > GLIDE_MERGE_SUM_ALL) return GLIDE_ERR_INVALID_ARG;
   if (c->merge != GLIDE_MERGE_SHARED &&
-      (c->decode_impl == GLIDE_DECODE_MMA || c->decode_impl == GLIDE_DECODE_STREAM ||
-       c->prefill_impl == GLIDE_PREFILL_MMA_SYNC || c->prefill_impl == GLIDE_PREFILL_TCGEN05))
-    return GLIDE_ERR_UNSUPPORTED;   // the sum-of-terms merges exist on the CUDA-core kernels only
+      (c->decode_impl == GLIDE_DECODE_MMA || c->prefill_impl == GLIDE_PREFILL_MMA_SYNC ||
+       c->prefill_impl == GLIDE_PREFILL_TCGEN05))
+    return GLIDE_ERR_UNSUPPORTED;   // sum-of-terms merges: streaming or CUDA-core decode kernel, CUDA-core prefill
   if (c->head_dim != 64 && c->head_dim != 128) return GLIDE_ERR_UNSUPPORTED;
   if (c->n_q_heads % c->n_kv_heads != 0) return GLIDE_ERR_UNSUPPORTED;
   int G = c->n_q_heads / c->n_kv_heads;
@@ -96,6 +96,7 @@ int glide::plan_context(const glide_config *cfg, glide_ctx *ctx, std::vector<Wor
   ctx->cfg.q_to_kv = nullptr;
   ctx->n_host.assign(L, 0);
   ctx->rec_floats = int(align_up(size_t(ctx->G) * (d + 2), 4));
+  ctx->stream_rec_floats = ctx->rec_floats * (cfg->merge == GLIDE_MERGE_SHARED ? 1 : 2);
 
   // window slots per split-K item: fixed by the caller, or 128 (512 for very long windows, to bound the
   // number of partials one merge has to read)
@@ -146,7 +147,7 @@ int glide::plan_context(const glide_config *cfg, glide_ctx *ctx, std::vector<Wor
   // the all-layer schedule plus one schedule per layer (glide_decode_step_layers)
   ctx->stream_rec_capacity = size_t(L) * units_per_layer + size_t(kMaxStreamCtas) * kStreamWarps;
   ctx->stream_seg_capacity = 2 * size_t(L) * units_per_layer + size_t(L + 1) * kMaxStreamCtas * kStreamWarps;
-  part_floats = std::max(part_floats, ctx->stream_rec_capacity * size_t(ctx->rec_floats));
+  part_floats = std::max(part_floats, ctx->stream_rec_capacity * size_t(ctx->stream_rec_floats));
   off = align_up(off + sizeof(float) * part_floats, 256);
   ctx->off_stream_segs = off;
   off = align_up(off + sizeof(StreamSegment) * ctx->stream_seg_capacity, 256);
@@ -276,7 +277,7 @@ int glide_create(const glide_config *cfg, void *dev_workspace, size_t workspace_
   int per_sm = 0;
   // kernel choice: fp32 -> CUDA cores; bf16 -> streaming tensor-core kernel when it applies, else per-item one
   ctx->decode_kind = 0;
-  if (ok && cfg->io_dtype == GLIDE_BF16 && cfg->decode_impl != GLIDE_DECODE_FMA && cfg->merge == GLIDE_MERGE_SHARED) {
+  if (ok && cfg->io_dtype == GLIDE_BF16 && cfg->decode_impl != GLIDE_DECODE_FMA) {
     ok = build_ring_tensor_maps(ctx) == GLIDE_OK;
     const bool want_stream = cfg->decode_impl == GLIDE_DECODE_AUTO || cfg->decode_impl == GLIDE_DECODE_STREAM;
     if (ok && want_stream && stream_decode_supported(ctx) && ctx->sm_count <= kMaxStreamCtas) {
@@ -289,15 +290,18 @@ int glide_create(const glide_config *cfg, void *dev_workspace, size_t workspace_
         delete ctx;
         return GLIDE_ERR_UNSUPPORTED;
       }
-      ok = mma_decode_setup(ctx) == GLIDE_OK;
-      ctx->decode_kind = 1;
+      if (cfg->merge == GLIDE_MERGE_SHARED) {
+        ok = mma_decode_setup(ctx) == GLIDE_OK;
+        ctx->decode_kind = 1;
+      }   // the per-item tensor-core kernel has the shared normaliser only: other merges use the CUDA-core kernel
     }
-  } else if (ok) {
+  }
+  if (ok && ctx->decode_kind == 0) {
     ok = decode_occupancy(ctx, &per_sm) == GLIDE_OK && per_sm > 0;
     if (ok) ctx->decode_grid = std::max(1, std::min(ctx->n_items, ctx->sm_count * per_sm));
   }
   if (ok) {
-    if (ctx->decode_kind >= 1)
+    if (!ctx->tmaps_host.empty())
       ok = cudaMemcpyAsync(ctx->ws + ctx->off_tmaps, ctx->tmaps_host.data(), ctx->tmaps_host.size(),
                            cudaMemcpyHostToDevice, st) == cudaSuccess;
     if (ok && ctx->decode_kind == 2) {

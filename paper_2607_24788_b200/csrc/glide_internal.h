@@ -160,6 +160,7 @@ struct glide_ctx {
   int decode_grid = 0;
   int n_items = 0;
   int rec_floats = 0;
+  int stream_rec_floats = 0;        // record size of the streaming kernel (twice as large for the sum-of-terms merges)
   int prefill_chunk = 0;
   float scale = 0.f;
   size_t elem = 0;

@@ -173,10 +173,20 @@ def test_sum_of_terms_merges(merge, dtype, d):
              merge=merge)
 
 
-def test_sum_of_terms_merges_need_the_cuda_core_kernels():
+@pytest.mark.parametrize("merge", [1, 2])
+@pytest.mark.parametrize("G", [1, 4, 8])
+def test_sum_of_terms_merges_streaming_kernel(merge, G):
+    # bf16, d = 128: decode on the streaming tensor-core kernel (units inside one warp, shared-memory groups and
+    # units cut across CTAs all occur with these windows), prefill on the CUDA-core kernel
+    run_case([700, 300, 64, 16, 0, 0, 48, 1 << 20], 2, 2 * G, 2, 128, BF16, [720], 12, amp=128 ** -0.5 * 4, seed=merge + G,
+             decode_impl=3, merge=merge)
+    run_case([0, 5, 40], 3, 2 * G, 2, 128, BF16, [30], 30, amp=128 ** -0.5 * 8, seed=merge, decode_impl=3, merge=merge)
+
+
+def test_sum_of_terms_merges_kernel_limits():
     from paper_2607_24788_b200 import glide
     with pytest.raises(glide.GlideError):
-        glide.Glide([64], 1, 8, 2, 128, 256, dtype=BF16, merge=1, decode_impl=3)
+        glide.Glide([64], 1, 8, 2, 128, 256, dtype=BF16, merge=1, decode_impl=1)   # per-item tensor-core kernel
     with pytest.raises(glide.GlideError):
         glide.Glide([64], 1, 8, 2, 128, 256, dtype=BF16, merge=2, prefill_impl=2)
 
