@@ -142,6 +142,11 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
   *failed = 1;
   return false;
 }
+__device__ __forceinline__ void bulk_load(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
+               "l"(src), "r"(bytes), "r"(bar)
+               : "memory");
+}
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const void *tmap, int x, int y, uint32_t bar) {
   asm volatile(
       "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(dst),
@@ -191,8 +196,8 @@ __device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32
 }
 
 #ifdef GLIDE_TC_PROFILE
-__device__ long long g_tc_prof[16];
-#define TC_MARK() long long tc_t_ = clock64(); long long tc_acc_[16] = {0,0,0,0,0,0,0,0,0,0,0,0,0,0,0,0}
+__device__ long long g_tc_prof[24];
+#define TC_MARK() long long tc_t_ = clock64(); long long tc_acc_[24] = {0,0,0,0,0,0,0,0,0,0,0,0,0,0,0,0,0,0,0,0,0,0,0,0}
 #define TC_ADD(i) do { long long n_ = clock64(); tc_acc_[i] += n_ - tc_t_; tc_t_ = n_; } while (0)
 #define TC_FLUSH(lo, hi) do { if (blockIdx.x == GLIDE_TC_PROFILE) for (int i_ = lo; i_ < hi; ++i_) atomicAdd(reinterpret_cast<unsigned long long *>(&g_tc_prof[i_]), (unsigned long long)tc_acc_[i_]); } while (0)
 #else
@@ -221,6 +226,7 @@ struct Smem {
   uint64_t bar_p[2];                     // P_X of the current tile is in TMEM (128 arrivals)
   uint64_t bar_done;                     // every window MMA has completed
   uint64_t bar_lin;                      // linear part: the MMAs issued so far have completed
+  uint64_t bar_state;                    // S (fp32) and z of the unit have landed
   uint32_t tmem_base;
   int failed;
 };
@@ -281,6 +287,7 @@ prefill_attn_tc_kernel(const PrefillParams p, const CUtensorMap *ring_maps, cons
     }
     mbar_init(smem_u32(&sm.bar_done), 1);
     mbar_init(smem_u32(&sm.bar_lin), 1);
+    mbar_init(smem_u32(&sm.bar_state), 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     sm.failed = 0;
   }
@@ -309,6 +316,14 @@ prefill_attn_tc_kernel(const PrefillParams p, const CUtensorMap *ring_maps, cons
   const uint32_t sQ[2] = {smem_u32(sm.q[0]), smem_u32(sm.q[1])};
   const uint32_t sKV0 = smem_u32(sm.kv[0]);
   auto kv_addr = [&](int slot) { return sKV0 + uint32_t(slot) * kTileBytes; };
+  // Roles of the five buffers after the window loop, by the order in which the loop stops using them (load number
+  // 2 n_tiles - 5 + k; a negative number is a buffer the loop never used): the two that come free first receive the
+  // unit's fp32 state (64 KiB, bulk-copied while the last key tiles are still being processed), the others hold the
+  // bf16 state tile, the phi(K') tile and the V' tile of the linear part.
+  auto late_seq = [&](int k) { return 2 * n_tiles - kStages + k; };
+  auto late_slot = [&](int k) { const int sq = late_seq(k); return sq >= 0 ? sq % kStages : sq + kStages; };
+  const int slotS0 = late_slot(0), slotS1 = late_slot(1), slotSb = late_slot(2), slotPk = late_slot(3), slotV = late_slot(4);
+  const bool need_state = ld.evicts && tq_last >= w && p.n0 + p.c0 - w > 0;
 
   // ---- softmax threads: per-row state that lives across the window and the linear part ----------------------
   const int X = (tid >> 7) & 1;                   // row tile of this thread (softmax warps only)
@@ -550,6 +565,23 @@ prefill_attn_tc_kernel(const PrefillParams p, const CUtensorMap *ring_maps, cons
         if (lane == 0) mbar_arrive(bar);
       }
     }
+    if (lane == 0 && need_state && !*failed) {
+      // S (fp32) and z as they are at the start of the chunk, into the two buffers the window loop leaves first
+      bool ok = true;
+      for (int k = 0; k < 2 && ok; ++k) {
+        const int sq = late_seq(k);
+        if (sq >= 0) ok = mbar_wait(smem_u32(&sm.bar_free[sq % kStages]), uint32_t(sq / kStages) & 1u, failed);
+      }
+      if (ok) {
+        const int ub = b * p.Hkv + g;
+        const unsigned char *Sg = p.ws + ld.S + size_t(ub) * kD * kD * sizeof(float);
+        const uint32_t bar = smem_u32(&sm.bar_state);
+        mbar_expect_tx(bar, uint32_t(kD * kD * sizeof(float) + kD * sizeof(float)));
+        for (int i = 0; i < 4; ++i)
+          bulk_load(kv_addr(i < 2 ? slotS0 : slotS1) + uint32_t(i & 1) * 16384u, Sg + size_t(i) * 16384, 16384u, bar);
+        bulk_load(smem_u32(sm.z), p.ws + ld.z + size_t(ub) * kD * sizeof(float), uint32_t(kD * sizeof(float)), bar);
+      }
+    }
   }
   tc_fence_before();
   __syncthreads();
@@ -572,7 +604,10 @@ prefill_attn_tc_kernel(const PrefillParams p, const CUtensorMap *ring_maps, cons
     const int64_t folded = p.n0 + p.c0 - w;   // tokens below this index are in S, z at the start of the chunk
     uint32_t phq[kD / 2];                      // phi(q) 2^-m* of this row, packed bf16
     if (activeX) {
-      const float M = fmaxf(m_ref, 0.f);
+      // Any common reference M >= m_ref gives the same quotient O / l.  M = max(m_ref, 0) would rescale O for every
+      // row whose window maximum is negative; a floor of -64 keeps 2^-M and everything scaled by it far inside the
+      // fp32 / bf16 range (phi <= 1) and makes that rescale a rarity.
+      const float M = fmaxf(m_ref, -64.f);
       const float fw = m_ref == -CUDART_INF_F ? 0.f : ex2(m_ref - M);
       const float fl = ex2(-M);
       if (o_init && __any_sync(0xffffffffu, fw != 1.f)) scale_o(fw);
@@ -609,20 +644,20 @@ prefill_attn_tc_kernel(const PrefillParams p, const CUtensorMap *ring_maps, cons
       for (int c = 0; c < 16; ++c)
         *reinterpret_cast<uint4 *>(sm.q[X] + sw128(row, c)) = make_uint4(phq[c * 4], phq[c * 4 + 1], phq[c * 4 + 2], phq[c * 4 + 3]);
     }
-    const int ub = b * p.Hkv + g;
+    TC_ADD(9);
     if (folded > 0 && tid < kSoftmaxThreads) {
       // bf16 copy of the state as the MN-major B tile of the inter-chunk product
-      const float *Sg = reinterpret_cast<const float *>(p.ws + ld.S) + size_t(ub) * kD * kD;
+      mbar_wait(smem_u32(&sm.bar_state), 0u, failed);
 #pragma unroll 4
       for (int i = 0; i < kD * 16 / kSoftmaxThreads; ++i) {
         const int id = tid + kSoftmaxThreads * i;
         const int r = id >> 4, c = id & 15;
-        const float4 f0 = *reinterpret_cast<const float4 *>(Sg + size_t(r) * kD + c * 8);
-        const float4 f1 = *reinterpret_cast<const float4 *>(Sg + size_t(r) * kD + c * 8 + 4);
-        *reinterpret_cast<uint4 *>(sm.kv[0] + sw128(r, c)) =
+        const float *Sg = reinterpret_cast<const float *>(sm.kv[r < 64 ? slotS0 : slotS1]) + size_t(r & 63) * kD;
+        const float4 f0 = *reinterpret_cast<const float4 *>(Sg + c * 8);
+        const float4 f1 = *reinterpret_cast<const float4 *>(Sg + c * 8 + 4);
+        *reinterpret_cast<uint4 *>(sm.kv[slotSb] + sw128(r, c)) =
             make_uint4(pack_bf16x2(f0.x, f0.y), pack_bf16x2(f0.z, f0.w), pack_bf16x2(f1.x, f1.y), pack_bf16x2(f1.z, f1.w));
       }
-      if (tid < kD) sm.z[tid] = (reinterpret_cast<const float *>(p.ws + ld.z) + size_t(ub) * kD)[tid];
     }
     fence_async_smem();
     tc_fence_before();
@@ -630,8 +665,8 @@ prefill_attn_tc_kernel(const PrefillParams p, const CUtensorMap *ring_maps, cons
     if (folded > 0) {
       if (tid == mma_tid) {
         tc_fence_after();
-        issue_mma(tmem + 256, sQ[0], kv_addr(0), true, o_init);
-        if (hasB) issue_mma(tmem + 384, sQ[1], kv_addr(0), true, o_init);
+        issue_mma(tmem + 256, sQ[0], kv_addr(slotSb), true, o_init);
+        if (hasB) issue_mma(tmem + 384, sQ[1], kv_addr(slotSb), true, o_init);
         mma_commit(smem_u32(&sm.bar_lin));
       }
       if (activeX) {
@@ -644,6 +679,7 @@ prefill_attn_tc_kernel(const PrefillParams p, const CUtensorMap *ring_maps, cons
       wait_lin();
       o_init = true;
     }
+    TC_ADD(10);
     // intra-chunk: delayed tokens of this chunk up to the CTA's last token, 128 at a time
     const int i_lo = folded < 0 ? int(-folded < int64_t(p.C) ? -folded : int64_t(p.C)) : 0;
     const int i_hi = tok0 + ntok - 1;
@@ -666,39 +702,57 @@ prefill_attn_tc_kernel(const PrefillParams p, const CUtensorMap *ring_maps, cons
             const float4 f1 = *reinterpret_cast<const float4 *>(pkp + size_t(ii) * kD + c * 8 + 4);
             pkd = make_uint4(pack_bf16x2(f0.x, f0.y), pack_bf16x2(f0.z, f0.w), pack_bf16x2(f1.x, f1.y), pack_bf16x2(f1.z, f1.w));
           }
-          *reinterpret_cast<uint4 *>(sm.kv[1] + sw128(r, c)) = pkd;
+          *reinterpret_cast<uint4 *>(sm.kv[slotPk] + sw128(r, c)) = pkd;
           const int64_t jj = valid ? p.n0 + p.c0 - w + ii : 0;
           const bool from_call = jj >= p.n0;
-          const bf16 *src = from_call ? callV + size_t(jj - p.n0) * call_stride : ringV + size_t(uint64_t(jj) % cap) * kD;
-          cp_async16(kv_addr(2) + sw128(r, c), src + c * 8, valid);
+          const uint32_t slot_row = (jj >> 32) == 0 ? uint32_t(jj) % cap : uint32_t(uint64_t(jj) % cap);
+          const bf16 *src = from_call ? callV + size_t(jj - p.n0) * call_stride : ringV + size_t(slot_row) * kD;
+          cp_async16(kv_addr(slotV) + sw128(r, c), src + c * 8, valid);
         }
         cp_async_commit();
+        TC_ADD(16);
         cp_async_wait_all();
       }
       fence_async_smem();
       tc_fence_before();
       __syncthreads();
+      TC_ADD(17);
       if (tid == mma_tid) {
         tc_fence_after();
-        issue_mma(tmem, sQ[0], kv_addr(1), false, false);   // C_X = (phi(Q_X) 2^-m*) phi(K')^T
-        if (hasB) issue_mma(tmem + 128, sQ[1], kv_addr(1), false, false);
+        issue_mma(tmem, sQ[0], kv_addr(slotPk), false, false);   // C_X = (phi(Q_X) 2^-m*) phi(K')^T
+        if (hasB) issue_mma(tmem + 128, sQ[1], kv_addr(slotPk), false, false);
         mma_commit(smem_u32(&sm.bar_lin));
       }
       wait_lin();
+      TC_ADD(18);
       if (activeX) {
         // C row -> bf16, masked to delayed tokens j' <= i of this row (the values already carry 2^-m*)
         float sum0 = 0.f, sum1 = 0.f;
         const int lo = i_lo - i0, hi = tl - i0;
-#pragma unroll 1
+        // a tile that lies wholly before the row tile's first token (and after the first delayed token) needs no mask
+        const bool whole = i0 + kKT - 1 <= tok0 + X * TOKT && i0 >= i_lo;
+        uint32_t ra[32], rb[32];
+        tmem_ld32_nowait(tS, ra);
+#pragma unroll
         for (int c0 = 0; c0 < kKT; c0 += 32) {
-          uint32_t r[32], pk[16];
-          tmem_ld32(tS + c0, r);
+          uint32_t (&r)[32] = ((c0 >> 5) & 1) ? rb : ra;
+          uint32_t pk[16];
+          tmem_wait_ld();
+          if (c0 + 32 < kKT) tmem_ld32_nowait(tS + c0 + 32, ((c0 >> 5) & 1) ? ra : rb);
+          if (whole) {
+#pragma unroll
+            for (int e = 0; e < 16; ++e) pk[e] = pack_bf16x2(__uint_as_float(r[e * 2]), __uint_as_float(r[e * 2 + 1]));
+          } else {
+#pragma unroll
+            for (int e = 0; e < 16; ++e) {
+              const int i = c0 + e * 2;
+              const float a0 = (i >= lo && i <= hi) ? __uint_as_float(r[e * 2]) : 0.f;
+              const float a1 = (i + 1 >= lo && i + 1 <= hi) ? __uint_as_float(r[e * 2 + 1]) : 0.f;
+              pk[e] = pack_bf16x2(a0, a1);
+            }
+          }
 #pragma unroll
           for (int e = 0; e < 16; ++e) {
-            const int i = c0 + e * 2;
-            const float a0 = (i >= lo && i <= hi) ? __uint_as_float(r[e * 2]) : 0.f;
-            const float a1 = (i + 1 >= lo && i + 1 <= hi) ? __uint_as_float(r[e * 2 + 1]) : 0.f;
-            pk[e] = pack_bf16x2(a0, a1);
             sum0 += __uint_as_float(pk[e] << 16);
             sum1 += __uint_as_float(pk[e] & 0xffff0000u);
           }
@@ -707,22 +761,24 @@ prefill_attn_tc_kernel(const PrefillParams p, const CUtensorMap *ring_maps, cons
         tmem_wait_st();
         l_sum += sum0 + sum1;
       }
+      TC_ADD(19);
       tc_fence_before();
       __syncthreads();
       if (tid == mma_tid) {
         tc_fence_after();
-        issue_mma_ts(tmem + 256, tmem, kv_addr(2), o_init);
-        if (hasB) issue_mma_ts(tmem + 384, tmem + 128, kv_addr(2), o_init);
+        issue_mma_ts(tmem + 256, tmem, kv_addr(slotV), o_init);
+        if (hasB) issue_mma_ts(tmem + 384, tmem + 128, kv_addr(slotV), o_init);
         mma_commit(smem_u32(&sm.bar_lin));
       }
       wait_lin();
+      TC_ADD(20);
       o_init = true;
     }
   }
 
   // ---- shared normaliser and store: one contiguous 256-byte row per thread ------------------------------------
   __syncthreads();
-  TC_ADD(5);
+  TC_ADD(15);
   const bool bad = sm.failed != 0;
   if (bad) {
     if (tid == 0) atomicExch(&p.ctl->status, kDevWaitTimeout);
@@ -746,7 +802,7 @@ prefill_attn_tc_kernel(const PrefillParams p, const CUtensorMap *ring_maps, cons
     }
   }
   TC_ADD(6);
-  if (tid == 0) { TC_FLUSH(0, 12); }
+  if (tid == 0) { TC_FLUSH(0, 12); TC_FLUSH(15, 24); }
   if (tid == kMmaWarp * 32) { TC_FLUSH(12, 16); }
   tc_fence_before();
   __syncthreads();
@@ -756,10 +812,10 @@ prefill_attn_tc_kernel(const PrefillParams p, const CUtensorMap *ring_maps, cons
 }  // namespace
 
 #ifdef GLIDE_TC_PROFILE
-extern "C" int glide_debug_tc_profile(long long *out16, int reset) {
-  if (cudaMemcpyFromSymbol(out16, g_tc_prof, sizeof(long long) * 16) != cudaSuccess) return 6;
+extern "C" int glide_debug_tc_profile(long long *out24, int reset) {
+  if (cudaMemcpyFromSymbol(out24, g_tc_prof, sizeof(long long) * 24) != cudaSuccess) return 6;
   if (reset) {
-    long long z[16] = {};
+    long long z[24] = {};
     if (cudaMemcpyToSymbol(g_tc_prof, z, sizeof(z)) != cudaSuccess) return 6;
   }
   return 0;
