@@ -16,9 +16,9 @@
 //   MMA       O_X += P_X V_t (V as the MN-major B operand), then S_X of the next tile: while one row tile is
 //             in its softmax the tensor core works for the other
 // TMEM columns: S_A [0,128) S_B [128,256) O_A [256,384) O_B [384,512).
-// Linear part (after the window tiles, the whole CTA in step): with m* = max(m_ref, 0) per row, phi(Q) 2^-m* as
-// bf16 times a bf16 copy of the state (inter-chunk), and C = phi(Q) phi(K')^T masked to j' <= i, then C V'
-// (intra-chunk), through the same MMAs; l accumulates the matching sums.  out = O / l.
+// Linear part (after the window tiles, the whole CTA in step): with a common reference M = max(m_ref, -64) per
+// row, phi(Q) 2^-M as bf16 times a bf16 copy of the state (inter-chunk), and C = phi(Q) phi(K')^T masked to
+// j' <= i, then C V' (intra-chunk), through the same MMAs; l accumulates the matching sums.  out = O / l.
 // Every mbarrier wait is bounded; on a time-out the CTA records kDevWaitTimeout, leaves its loops, frees its TMEM
 // columns and returns.
 #include <cuda.h>
