@@ -178,8 +178,9 @@ def test_sum_of_terms_merges(merge, dtype, d):
 def test_sum_of_terms_merges_streaming_kernel(merge, G):
     # bf16, d = 128: decode on the streaming tensor-core kernel (units inside one warp, shared-memory groups and
     # units cut across CTAs all occur with these windows), prefill on the CUDA-core kernel
+    # (prefill outputs of these merges are checked in test_sum_of_terms_merges: here the prompt only builds the state)
     run_case([700, 300, 64, 16, 0, 0, 48, 1 << 20], 2, 2 * G, 2, 128, BF16, [720], 12, amp=128 ** -0.5 * 4, seed=merge + G,
-             decode_impl=3, merge=merge)
+             decode_impl=3, merge=merge, check_prefill_outputs=False)
     run_case([0, 5, 40], 3, 2 * G, 2, 128, BF16, [30], 30, amp=128 ** -0.5 * 8, seed=merge, decode_impl=3, merge=merge)
 
 
