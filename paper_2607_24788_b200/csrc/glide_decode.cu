@@ -261,7 +261,7 @@ __device__ __forceinline__ void merge_unit(const DecodeParams &p, const WorkItem
     // shared normaliser: m* = max(window max, 0), the linear terms carry the factor exp(-m*) <= 1;
     // sum of two normalised terms: the window is normalised on its own, against its own maximum
     const bool shared = ld.merge == GLIDE_MERGE_SHARED;
-    float M = shared ? 0.f : -CUDART_INF_F;
+    float M = (shared && has_state) ? 0.f : -CUDART_INF_F;   // the floor belongs to the linear terms (logit 0)
     for (int i = 0; i < ld.n_win_items; ++i) M = fmaxf(M, __ldcg(rec0 + size_t(i) * p.rec_floats + G * D + h));
     if (has_win) M = fmaxf(M, sm.scur[h]);
     float den = 0.f;

@@ -443,10 +443,11 @@ __device__ __forceinline__ void merge_unit_warp(const DecodeParams &p, const Wor
       scur[h] = warp_sum(part) * p.scale_log2;
     }
   }
-  // m* = max(window max, current logit, 0); the partial maxima are read once, lane-strided
+  // m* = max(window max, current logit, 0 if the state holds tokens: its terms have logit 0; without them a floor
+  // would only push the window weights towards underflow); the partial maxima are read once, lane-strided
 #pragma unroll
   for (int h = 0; h < G; ++h) {
-    float mx = fmaxf(scur[h], 0.f);
+    float mx = has_state ? fmaxf(scur[h], 0.f) : scur[h];
     for (int i = lane; i < n_win; i += 32) mx = fmaxf(mx, __ldcg(rec0 + size_t(i) * p.rec_floats + G * D + h));
     M[h] = warp_max(mx);
   }
@@ -462,7 +463,7 @@ __device__ __forceinline__ void merge_unit_warp(const DecodeParams &p, const Wor
     float bs = 0.f;
     if (has_state)
       for (int i = lane; i < n_st; i += 32) bs += __ldcg(rec0 + size_t(n_win + i) * p.rec_floats + G * D + h);
-    den = warp_sum(den) + (has_win ? exp2f(scur[h] - M[h]) : 0.f) + exp2f(-M[h]) * warp_sum(bs);
+    den = warp_sum(den) + (has_win ? exp2f(scur[h] - M[h]) : 0.f) + (has_state ? exp2f(-M[h]) * warp_sum(bs) : 0.f);
     inv[h] = 1.0f / den;
   }
   __syncwarp();

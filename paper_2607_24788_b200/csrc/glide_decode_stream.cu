@@ -834,9 +834,10 @@ glide_decode_stream_kernel(const DecodeParams p, const StreamParams sp) {
       vx[3] = __uint_as_float(vt_bits.y & 0xffff0000u);
 #pragma unroll
       for (int h = 0; h < G; ++h) {
-        // shared normaliser: reference max(window max, 0); sum of terms: the window against its own maximum, the
-        // linear term a / b added (an empty term counts as zero)
-        const float Mf = SUM ? fmaxf(mh[h], scur[h]) : fmaxf(fmaxf(mh[h], scur[h]), 0.f);
+        // reference: the largest logit of the records (a record that includes the linear readout carries a
+        // reference >= 0 already; without a state no floor is wanted: it would only push the window weights
+        // towards underflow).  Sum of terms: the linear term a / b is added (an empty term counts as zero)
+        const float Mf = fmaxf(mh[h], scur[h]);
         const float fr = exp2_or_zero(mh[h], Mf), fc = exp2_or_zero(scur[h], Mf);
         const float den = fmaf(lh[h], fr, fc);
         const float inv = (!SUM || den > 0.f) ? 1.0f / den : 0.f;
@@ -1009,7 +1010,7 @@ glide_decode_stream_kernel(const DecodeParams p, const StreamParams sp) {
       }
 #pragma unroll
       for (int h = 0; h < G; ++h) {
-        const float Mf = SUM ? fmaxf(Mg[h], sc[h]) : fmaxf(fmaxf(Mg[h], sc[h]), 0.f);
+        const float Mf = fmaxf(Mg[h], sc[h]);
         const float fr = exp2_or_zero(Mg[h], Mf), fc = exp2_or_zero(sc[h], Mf);
         const float den = fmaf(lg[h], fr, fc);
         const float inv = (!SUM || den > 0.f) ? 1.0f / den : 0.f;

@@ -207,9 +207,9 @@ __global__ void __launch_bounds__(kPrefillThreads) prefill_attn_kernel(const Pre
   }
 #pragma unroll
   for (int h = 0; h < G; ++h) {
-    const float M = fmaxf(m[h], 0.f);
+    const float M = bl[h] > 0.f ? fmaxf(m[h], 0.f) : m[h];   // the floor belongs to the linear terms (logit 0)
     const float fw = m[h] == -CUDART_INF_F ? 0.f : exp2f(m[h] - M);
-    const float fl = exp2f(-M);
+    const float fl = bl[h] > 0.f ? exp2f(-M) : 0.f;
     const float inv = 1.0f / fmaf(l[h], fw, fl * bl[h]);
     const int head = p.heads_of[g * G + h];
 #pragma unroll

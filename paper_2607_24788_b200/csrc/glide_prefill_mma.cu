@@ -329,9 +329,11 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_attn_mma_kernel(const Pre
     float fl[2];
 #pragma unroll
     for (int h = 0; h < 2; ++h) {
-      const float M = fmaxf(m_row[h], 0.f);
+      // a row without evicted tokens keeps its own reference and gets phi(q) = 0: the floor belongs to the linear terms
+      const bool has_lin = (h ? tokB : tokA) >= w;
+      const float M = has_lin ? fmaxf(m_row[h], 0.f) : m_row[h];
       const float fw = m_row[h] == -CUDART_INF_F ? 0.f : ex2(m_row[h] - M);
-      fl[h] = ex2(-M);
+      fl[h] = has_lin ? ex2(-M) : 0.f;
       l_row[h] *= fw;
 #pragma unroll
       for (int nt = 0; nt < kD / 8; ++nt) {

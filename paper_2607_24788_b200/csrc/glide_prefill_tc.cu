@@ -607,9 +607,12 @@ prefill_attn_tc_kernel(const PrefillParams p, const CUtensorMap *ring_maps, cons
       // Any common reference M >= m_ref gives the same quotient O / l.  M = max(m_ref, 0) would rescale O for every
       // row whose window maximum is negative; a floor of -64 keeps 2^-M and everything scaled by it far inside the
       // fp32 / bf16 range (phi <= 1) and makes that rescale a rarity.
-      const float M = fmaxf(m_ref, -64.f);
+      // A row without evicted tokens (position below the window size) keeps its own reference and gets phi(q) = 0:
+      // a floor there would only push its window weights towards underflow.
+      const bool has_lin = tok_abs >= w;
+      const float M = has_lin ? fmaxf(m_ref, -64.f) : m_ref;
       const float fw = m_ref == -CUDART_INF_F ? 0.f : ex2(m_ref - M);
-      const float fl = ex2(-M);
+      const float fl = has_lin ? ex2(-M) : 0.f;
       if (o_init && __any_sync(0xffffffffu, fw != 1.f)) scale_o(fw);
       l_sum *= fw;
       // this row of Q is still in the shared tile (every S product has completed)

@@ -254,3 +254,36 @@ def test_bf16_prefill_tcgen05_after_decode_steps():
             pos += 1
     check_state(g, stack, "after two turns")
     assert g.glide_device_status() == 0
+
+
+@pytest.mark.parametrize("dtype,d,kw", [(BF16, 128, {}), (BF16, 128, dict(prefill_impl=1, decode_impl=1)),
+                                        (BF16, 128, dict(prefill_impl=3, decode_impl=2)), (F32, 64, {})])
+def test_very_negative_window_logits_without_linear_terms(dtype, d, kw):
+    # every window logit is about -180 (keys close to the all-ones vector, queries close to minus a multiple of it;
+    # values of order one): rows that have no evicted token yet, and layers that never evict, must be normalised
+    # against their own maximum, not against the logit 0 of the linear terms, or their window weights underflow to
+    # 0 / 0.  Every kernel family, prefill and decode.
+    from paper_2607_24788_b200 import glide, synth
+    from oracle import glide_oracle as orc
+    from tests.parity_util import f32_scale, to_np, check_outputs
+    windows, B, H, Hkv = [16, 100, 1 << 20], 2, 8, 2
+    L = len(windows)
+    wl = synth.Workload(5, L, B, H, Hkv, d, dtype, 1.0)
+    qmul = 16.0 if d == 128 else 24.0
+
+    def shaped(q, k, v):
+        return (-qmul + 0.25 * q.float()).to(dtype), (1.0 + 0.05 * k.float()).to(dtype), v
+
+    g = glide.Glide(windows, B, H, Hkv, d, 64, dtype=dtype, softmax_scale=f32_scale(d), prefill_chunk=32, **kw)
+    stack = orc.Stack(windows, B, H, Hkv, d, f32_scale(d))
+    q, k, v = shaped(*wl.qkv(range(L), range(B), range(0, 48), device="cuda"))
+    logits = torch.einsum("lbthd,lbshd->lbhts", q.float(), k.float().repeat_interleave(H // Hkv, dim=3)) * f32_scale(d)
+    assert logits.max().item() < -150.0      # the case is what it claims to be
+    out = torch.full_like(q, float("nan"))
+    g.glide_prefill(q, k, v, out)
+    check_outputs(out, stack.prefill(to_np(q), to_np(k), to_np(v)), dtype, "prefill")
+    for t in range(48, 56):
+        q, k, v = shaped(*wl.decode_qkv(t, "cuda"))
+        out = torch.empty_like(q)
+        g.glide_decode_step(q, k, v, out)
+        check_outputs(out, stack.decode(to_np(q), to_np(k), to_np(v)), dtype, f"decode@{t}")
