@@ -192,8 +192,9 @@ def test_sum_of_terms_merges_kernel_limits():
         glide.Glide([64], 1, 8, 2, 128, 256, dtype=BF16, merge=2, prefill_impl=2)
 
 
-@pytest.mark.parametrize("dtype,d,impl", [(BF16, 128, 0), (BF16, 128, 1), (BF16, 64, 0), (F32, 64, 0)])
-def test_decode_step_layers(dtype, d, impl):
+@pytest.mark.parametrize("dtype,d,impl,merge", [(BF16, 128, 0, 0), (BF16, 128, 1, 0), (BF16, 64, 0, 0), (F32, 64, 0, 0),
+                                               (BF16, 128, 0, 2), (F32, 64, 0, 1)])
+def test_decode_step_layers(dtype, d, impl, merge):
     # layer by layer, in ranges, and for the whole stack, interleaved: every path against the oracle, and the
     # positions of the layers bit-exact afterwards (streaming kernel, per-item tensor-core kernel, CUDA-core kernel)
     import numpy as np
@@ -204,8 +205,8 @@ def test_decode_step_layers(dtype, d, impl):
     L = len(windows)
     amp = 1.0 if dtype == F32 else d ** -0.5 * 4
     wl = synth.Workload(3, L, B, H, Hkv, d, dtype, amp)
-    g = glide.Glide(windows, B, H, Hkv, d, 128, dtype=dtype, softmax_scale=f32_scale(d), decode_impl=impl)
-    stack = orc.Stack(windows, B, H, Hkv, d, f32_scale(d))
+    g = glide.Glide(windows, B, H, Hkv, d, 128, dtype=dtype, softmax_scale=f32_scale(d), decode_impl=impl, merge=merge)
+    stack = orc.Stack(windows, B, H, Hkv, d, f32_scale(d), merge=merge)
     q, k, v = wl.qkv(range(L), range(B), range(0, 50), device="cuda")
     g.glide_prefill(None, k, v, None)
     stack.prefill(None, to_np(k), to_np(v), outputs=False)
