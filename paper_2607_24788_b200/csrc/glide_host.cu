@@ -48,9 +48,8 @@ int validate_config(const glide_config *c) {
   if (c->phi != GLIDE_PHI_SOFTMAX) return GLIDE_ERR_UNSUPPORTED;
   if (c->merge < GLIDE_MERGE_SHARED || c->merge > GLIDE_MERGE_SUM_ALL) return GLIDE_ERR_INVALID_ARG;
   if (c->merge != GLIDE_MERGE_SHARED &&
-      (c->decode_impl == GLIDE_DECODE_MMA || c->prefill_impl == GLIDE_PREFILL_MMA_SYNC ||
-       c->prefill_impl == GLIDE_PREFILL_TCGEN05))
-    return GLIDE_ERR_UNSUPPORTED;   // sum-of-terms merges: streaming or CUDA-core decode kernel, CUDA-core prefill
+      (c->decode_impl == GLIDE_DECODE_MMA || c->prefill_impl == GLIDE_PREFILL_MMA_SYNC))
+    return GLIDE_ERR_UNSUPPORTED;   // sum-of-terms merges: not on the per-item tensor-core decode kernel nor on mma.sync
   if (c->head_dim != 64 && c->head_dim != 128) return GLIDE_ERR_UNSUPPORTED;
   if (c->n_q_heads % c->n_kv_heads != 0) return GLIDE_ERR_UNSUPPORTED;
   int G = c->n_q_heads / c->n_kv_heads;
@@ -157,6 +156,9 @@ int glide::plan_context(const glide_config *cfg, glide_ctx *ctx, std::vector<Wor
   off = align_up(off + size_t(128) * 3 * L, 256);
   ctx->off_phik = off;
   off = align_up(off + sizeof(float) * size_t(L) * units_per_layer * ctx->prefill_chunk * d, 256);
+  ctx->off_zcum = off;   // running sums of phi(K') over the chunk: only the sum-of-terms merges use them
+  if (cfg->merge != GLIDE_MERGE_SHARED)
+    off = align_up(off + sizeof(float) * size_t(L) * units_per_layer * ctx->prefill_chunk * d, 256);
   // the streamed arrays start on a 2 MiB boundary of the workspace whatever the sizes of the small tables before
   // them (measured on the B = 1 decode step: 31.5 us against 32.1 us with 64 KiB or 256 B alignment)
   off = align_up(off, size_t(GLIDE_STATE_ALIGN));

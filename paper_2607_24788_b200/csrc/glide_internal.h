@@ -117,6 +117,8 @@ struct PrefillParams {
   const int32_t *heads_of;
   Control *ctl;
   float *phik;               // chunk scratch: [layer_count][B][Hkv][C][d] fp32, phi of the delayed keys
+  float *zcum;               // sum-of-terms merges on the tcgen05 kernel: running sums of phik over the chunk, same shape
+  int32_t merge;             // glide_merge
   const void *q, *k, *v;     // the call's inputs
   void *out;
   int64_t n0;                // tokens absorbed before this call (all layers of the call)
@@ -168,7 +170,7 @@ struct glide_ctx {
   size_t ws_bytes = 0;
   // workspace regions (byte offsets)
   size_t off_ctl = 0, off_ndev = 0, off_layers = 0, off_heads = 0, off_items = 0, off_tickets = 0,
-         off_partials = 0, off_tmaps = 0, off_phik = 0, off_state = 0, off_ring = 0, total = 0;
+         off_partials = 0, off_tmaps = 0, off_phik = 0, off_zcum = 0, off_state = 0, off_ring = 0, total = 0;
   size_t state_bytes = 0;           // S and z of all layers (contiguous)
   size_t item_part_floats = 0;      // floats of split-K records the per-item work list needs
   int noalloc_grid = 0;             // grid of the allocation-free decode variant (0: not sized yet)

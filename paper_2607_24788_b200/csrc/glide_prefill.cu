@@ -314,6 +314,30 @@ __global__ void __launch_bounds__(kPrefillThreads) prefill_state_kernel(const Pr
   }
 }
 
+// 1b. (sum-of-terms merges on the tcgen05 kernel) running sums of phi(K') over the chunk: zcum[i] = sum over the valid
+// delayed indices ii <= i of phi(k'_ii); a row's linear normaliser is then phi(q) . (z + zcum[own index]).
+// One thread per (unit, feature), sequential over the chunk (C <= 1024).
+template <int D>
+__global__ void __launch_bounds__(kPrefillThreads) prefill_zcum_kernel(const PrefillParams p) {
+  const int64_t idx = int64_t(blockIdx.x) * kPrefillThreads + threadIdx.x;
+  const int64_t units = int64_t(p.layer_count) * p.B * p.Hkv;
+  if (idx >= units * D) return;
+  const int r = int(idx % D);
+  const int64_t u = idx / D;
+  const int lrel = int(u / (int64_t(p.Hkv) * p.B));
+  const LayerDev ld = p.layers[p.layer_begin + lrel];
+  if (!ld.evicts) return;
+  const int64_t first = p.n0 + p.c0 - ld.wlin;
+  const int i_lo = first < 0 ? int(first < -int64_t(p.C) ? p.C : -first) : 0;
+  const float *pk = p.phik + size_t(u) * p.Cmax * D + r;
+  float *zc = p.zcum + size_t(u) * p.Cmax * D + r;
+  float run = 0.f;
+  for (int i = 0; i < p.C; ++i) {
+    if (i >= i_lo) run += pk[size_t(i) * D];
+    zc[size_t(i) * D] = run;
+  }
+}
+
 // 4. ring fill: the chunk's newest min(C, cap) tokens
 template <typename T, int D>
 __global__ void __launch_bounds__(kPrefillThreads) prefill_ring_kernel(const PrefillParams p) {
@@ -353,6 +377,8 @@ int launch_prefill(glide_ctx *ctx, int layer_begin, int layer_count, int64_t T, 
   p.heads_of = reinterpret_cast<const int32_t *>(ctx->ws + ctx->off_heads);
   p.ctl = reinterpret_cast<Control *>(ctx->ws + ctx->off_ctl);
   p.phik = reinterpret_cast<float *>(ctx->ws + ctx->off_phik);
+  p.zcum = reinterpret_cast<float *>(ctx->ws + ctx->off_zcum);
+  p.merge = ctx->cfg.merge;
   p.q = q;
   p.k = k;
   p.v = v;
@@ -370,12 +396,13 @@ int launch_prefill(glide_ctx *ctx, int layer_begin, int layer_count, int64_t T, 
   const int64_t units = int64_t(layer_count) * p.B * p.Hkv;
   int impl = ctx->cfg.prefill_impl;
   if (impl == GLIDE_PREFILL_AUTO)
-    impl = (prefill_attn_mma_supported(ctx) && ctx->cfg.decode_impl != GLIDE_DECODE_FMA && ctx->cfg.merge == GLIDE_MERGE_SHARED)
-               ? GLIDE_PREFILL_TCGEN05 : GLIDE_PREFILL_FMA;
+    impl = (prefill_attn_mma_supported(ctx) && ctx->cfg.decode_impl != GLIDE_DECODE_FMA) ? GLIDE_PREFILL_TCGEN05 : GLIDE_PREFILL_FMA;
   // the tcgen05 kernel needs the ring descriptors of the tensor-core decode kernels (absent when decode_impl asks
   // for the CUDA-core kernel); without them the call uses the mma.sync kernel
   const bool use_tc = impl == GLIDE_PREFILL_TCGEN05 && prefill_attn_tc_supported(ctx);
-  const bool use_mma = (impl == GLIDE_PREFILL_MMA_SYNC || (impl == GLIDE_PREFILL_TCGEN05 && !use_tc)) && prefill_attn_mma_supported(ctx);
+  // (the mma.sync kernel has the shared normaliser only: the other merges fall through to the CUDA-core kernel)
+  const bool use_mma = (impl == GLIDE_PREFILL_MMA_SYNC || (impl == GLIDE_PREFILL_TCGEN05 && !use_tc)) &&
+                       prefill_attn_mma_supported(ctx) && ctx->cfg.merge == GLIDE_MERGE_SHARED;
   bool any_evicts = false;
   for (int l = layer_begin; l < layer_begin + layer_count; ++l) any_evicts = any_evicts || ctx->layers[l].evicts;
 
@@ -390,6 +417,8 @@ int launch_prefill(glide_ctx *ctx, int layer_begin, int layer_count, int64_t T, 
       if (any_evicts) prefill_phi_kernel<TT, D><<<warp_blocks, kPrefillThreads, 0, stream>>>(p);
       if (out) {
         if (use_tc) {
+          if (any_evicts && p.merge != GLIDE_MERGE_SHARED)
+            prefill_zcum_kernel<D><<<unsigned((units * D + kPrefillThreads - 1) / kPrefillThreads), kPrefillThreads, 0, stream>>>(p);
           if (launch_prefill_attn_tc(ctx, p, stream) != GLIDE_OK) return GLIDE_ERR_CUDA;
         } else if (use_mma) {
           if (launch_prefill_attn_mma(ctx, p, stream) != GLIDE_OK) return GLIDE_ERR_CUDA;

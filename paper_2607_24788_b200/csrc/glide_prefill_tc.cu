@@ -260,6 +260,8 @@ prefill_attn_tc_kernel(const PrefillParams p, const CUtensorMap *ring_maps, cons
   const int64_t tq0 = p.n0 + p.c0 + tok0;
   const int64_t tq_last = tq0 + ntok - 1;
   const int64_t w = ld.w;
+  const int64_t wl = ld.wlin;                      // delay of the linear stream: w, or 0 when the state holds every token
+  const bool sum_terms = p.merge != GLIDE_MERGE_SHARED;
   const uint32_t cap = ld.cap > 0 ? uint32_t(ld.cap) : 1u;
   const size_t unit_rows = (size_t(b) * p.Hkv + g) * size_t(ld.cap);
   const size_t seq = (size_t(lrel) * p.B + b) * size_t(p.T);
@@ -323,7 +325,7 @@ prefill_attn_tc_kernel(const PrefillParams p, const CUtensorMap *ring_maps, cons
   auto late_seq = [&](int k) { return 2 * n_tiles - kStages + k; };
   auto late_slot = [&](int k) { const int sq = late_seq(k); return sq >= 0 ? sq % kStages : sq + kStages; };
   const int slotS0 = late_slot(0), slotS1 = late_slot(1), slotSb = late_slot(2), slotPk = late_slot(3), slotV = late_slot(4);
-  const bool need_state = ld.evicts && tq_last >= w && p.n0 + p.c0 - w > 0;
+  const bool need_state = ld.evicts && tq_last >= wl && p.n0 + p.c0 - wl > 0;
 
   // ---- softmax threads: per-row state that lives across the window and the linear part ----------------------
   const int X = (tid >> 7) & 1;                   // row tile of this thread (softmax warps only)
@@ -591,7 +593,7 @@ prefill_attn_tc_kernel(const PrefillParams p, const CUtensorMap *ring_maps, cons
   // =========================== linear part: the whole CTA in step ===========================
   // (no early exits from here on: every thread passes the same __syncthreads; after a time-out the waits return
   // at once and the results are discarded)
-  const bool linear = ld.evicts && tq_last >= w;
+  const bool linear = ld.evicts && tq_last >= wl;
   bool o_init = n_tiles > 0;   // O_X holds a valid accumulation (uniform over the CTA)
   uint32_t lin_phase = 0;
   const int mma_tid = kMmaWarp * 32;
@@ -601,7 +603,7 @@ prefill_attn_tc_kernel(const PrefillParams p, const CUtensorMap *ring_maps, cons
     tc_fence_after();
   };
   if (linear) {
-    const int64_t folded = p.n0 + p.c0 - w;   // tokens below this index are in S, z at the start of the chunk
+    const int64_t folded = p.n0 + p.c0 - wl;   // tokens below this index are in S, z at the start of the chunk
     uint32_t phq[kD / 2];                      // phi(q) 2^-m* of this row, packed bf16
     if (activeX) {
       // Any common reference M >= m_ref gives the same quotient O / l.  M = max(m_ref, 0) would rescale O for every
@@ -609,12 +611,17 @@ prefill_attn_tc_kernel(const PrefillParams p, const CUtensorMap *ring_maps, cons
       // fp32 / bf16 range (phi <= 1) and makes that rescale a rarity.
       // A row without evicted tokens (position below the window size) keeps its own reference and gets phi(q) = 0:
       // a floor there would only push its window weights towards underflow.
-      const bool has_lin = tok_abs >= w;
+      // Sum of two normalised terms instead: the window part is normalised now (O / l), and phi(q) is divided by the
+      // row's linear normaliser phi(q) . (z + running sum of phi(K') up to the row's own delayed token), so that what
+      // the linear products add to O is the normalised linear term; the final division is by 1.
+      const bool has_lin = tok_abs >= wl;
       const float M = has_lin ? fmaxf(m_ref, -64.f) : m_ref;
-      const float fw = m_ref == -CUDART_INF_F ? 0.f : ex2(m_ref - M);
+      float fw = m_ref == -CUDART_INF_F ? 0.f : ex2(m_ref - M);
       const float fl = has_lin ? ex2(-M) : 0.f;
+      if (sum_terms) fw = l_sum > 0.f ? 1.0f / l_sum : 0.f;
       if (o_init && __any_sync(0xffffffffu, fw != 1.f)) scale_o(fw);
-      l_sum *= fw;
+      l_sum = sum_terms ? 1.f : l_sum * fw;
+      if (sum_terms && need_state) mbar_wait(smem_u32(&sm.bar_state), 0u, failed);   // z is needed for the normaliser
       // this row of Q is still in the shared tile (every S product has completed)
 #pragma unroll
       for (int i = 0; i < kD / 8; ++i) {
@@ -629,17 +636,35 @@ prefill_attn_tc_kernel(const PrefillParams p, const CUtensorMap *ring_maps, cons
       for (int i = 0; i < kD / 2; ++i)
         mx = fmaxf(mx, fmaxf(__uint_as_float(phq[i] << 16), __uint_as_float(phq[i] & 0xffff0000u)));
       // one pass of exponentials: kept as packed bf16, normalised by the sum of the unrounded values afterwards
-      float sum0 = 0.f, sum1 = 0.f;
+      float sum0 = 0.f, sum1 = 0.f, dz0 = 0.f, dz1 = 0.f;
       const float mxl = mx * kLog2e;
+      const float4 *zrow = reinterpret_cast<const float4 *>(p.zcum + (size_t(u) * p.Cmax + size_t(tok_r < ntokX ? tl : tok0)) * kD);
 #pragma unroll
-      for (int i = 0; i < kD / 2; ++i) {
-        const float e0 = ex2(fmaf(__uint_as_float(phq[i] << 16), kLog2e, -mxl));
-        const float e1 = ex2(fmaf(__uint_as_float(phq[i] & 0xffff0000u), kLog2e, -mxl));
-        sum0 += e0;
-        sum1 += e1;
-        phq[i] = pack_bf16x2(e0, e1);
+      for (int i4 = 0; i4 < kD / 4; ++i4) {
+        float zz[4] = {0.f, 0.f, 0.f, 0.f};
+        if (sum_terms) {
+          const float4 zc = __ldg(zrow + i4);
+          zz[0] = zc.x, zz[1] = zc.y, zz[2] = zc.z, zz[3] = zc.w;
+          if (need_state) {
+#pragma unroll
+            for (int e = 0; e < 4; ++e) zz[e] += sm.z[i4 * 4 + e];
+          }
+        }
+#pragma unroll
+        for (int hf = 0; hf < 2; ++hf) {
+          const int i = i4 * 2 + hf;
+          const float e0 = ex2(fmaf(__uint_as_float(phq[i] << 16), kLog2e, -mxl));
+          const float e1 = ex2(fmaf(__uint_as_float(phq[i] & 0xffff0000u), kLog2e, -mxl));
+          sum0 += e0;
+          sum1 += e1;
+          dz0 = fmaf(e0, zz[hf * 2], dz0);
+          dz1 = fmaf(e1, zz[hf * 2 + 1], dz1);
+          phq[i] = pack_bf16x2(e0, e1);
+        }
       }
-      const float sc = fl * __frcp_rn(sum0 + sum1);
+      // shared normaliser: phi(q) 2^-M;  sum of terms: phi(q) / (phi(q) . z_row) = e / (e . z_row)
+      const float dz = dz0 + dz1;
+      const float sc = sum_terms ? ((has_lin && dz > 0.f) ? 1.0f / dz : 0.f) : fl * __frcp_rn(sum0 + sum1);
 #pragma unroll
       for (int i = 0; i < kD / 2; ++i)
         phq[i] = pack_bf16x2(__uint_as_float(phq[i] << 16) * sc, __uint_as_float(phq[i] & 0xffff0000u) * sc);
@@ -677,7 +702,7 @@ prefill_attn_tc_kernel(const PrefillParams p, const CUtensorMap *ring_maps, cons
 #pragma unroll
         for (int i = 0; i < kD / 2; ++i)
           dot += __uint_as_float(phq[i] << 16) * sm.z[2 * i] + __uint_as_float(phq[i] & 0xffff0000u) * sm.z[2 * i + 1];
-        l_sum += dot;
+        if (!sum_terms) l_sum += dot;
       }
       wait_lin();
       o_init = true;
@@ -706,7 +731,7 @@ prefill_attn_tc_kernel(const PrefillParams p, const CUtensorMap *ring_maps, cons
             pkd = make_uint4(pack_bf16x2(f0.x, f0.y), pack_bf16x2(f0.z, f0.w), pack_bf16x2(f1.x, f1.y), pack_bf16x2(f1.z, f1.w));
           }
           *reinterpret_cast<uint4 *>(sm.kv[slotPk] + sw128(r, c)) = pkd;
-          const int64_t jj = valid ? p.n0 + p.c0 - w + ii : 0;
+          const int64_t jj = valid ? p.n0 + p.c0 - wl + ii : 0;
           const bool from_call = jj >= p.n0;
           const uint32_t slot_row = (jj >> 32) == 0 ? uint32_t(jj) % cap : uint32_t(uint64_t(jj) % cap);
           const bf16 *src = from_call ? callV + size_t(jj - p.n0) * call_stride : ringV + size_t(slot_row) * kD;
@@ -762,7 +787,7 @@ prefill_attn_tc_kernel(const PrefillParams p, const CUtensorMap *ring_maps, cons
           tmem_st16(tS + (c0 >> 1), pk);
         }
         tmem_wait_st();
-        l_sum += sum0 + sum1;
+        if (!sum_terms) l_sum += sum0 + sum1;
       }
       TC_ADD(19);
       tc_fence_before();

@@ -166,11 +166,21 @@ def test_bf16_prefill_tcgen05_large_logits():
 
 
 @pytest.mark.parametrize("merge", [1, 2])   # appendix hybrid equations: evicted-token state / all-token state
-@pytest.mark.parametrize("dtype,d", [(F32, 64), (BF16, 128)])
-def test_sum_of_terms_merges(merge, dtype, d):
+@pytest.mark.parametrize("dtype,d,kw", [(F32, 64, {}), (BF16, 128, {}), (BF16, 128, dict(prefill_impl=3, decode_impl=2)),
+                                        (BF16, 64, {})])
+def test_sum_of_terms_merges(merge, dtype, d, kw):
+    # bf16 / d = 128 default: tcgen05 prefill + streaming decode; forced CUDA-core kernels; d = 64; fp32
     amp = 1.0 if dtype == F32 else d ** -0.5 * 4
     run_case([0, 1, 5, 40, 1000], 2, 4, 2, d, dtype, [70, 33], 24, amp=amp, seed=merge, prefill_chunk=32, decode_chunk=16,
-             merge=merge)
+             merge=merge, **kw)
+
+
+@pytest.mark.parametrize("merge", [1, 2])
+@pytest.mark.parametrize("G,chunk", [(1, 96), (4, 256), (8, 32)])
+def test_sum_of_terms_merges_tcgen05_prefill(merge, G, chunk):
+    # several calls (aligned and not), windows below / at / above the key tile, a purely linear and a never-evicting layer
+    run_case([0, 16, 100, 128, 304, 1 << 20], 2, 2 * G, 2, 128, BF16, [144, 130, 61], 4, amp=128 ** -0.5 * 4,
+             seed=merge + G, prefill_chunk=chunk, prefill_impl=2, merge=merge)
 
 
 @pytest.mark.parametrize("merge", [1, 2])
@@ -189,7 +199,7 @@ def test_sum_of_terms_merges_kernel_limits():
     with pytest.raises(glide.GlideError):
         glide.Glide([64], 1, 8, 2, 128, 256, dtype=BF16, merge=1, decode_impl=1)   # per-item tensor-core kernel
     with pytest.raises(glide.GlideError):
-        glide.Glide([64], 1, 8, 2, 128, 256, dtype=BF16, merge=2, prefill_impl=2)
+        glide.Glide([64], 1, 8, 2, 128, 256, dtype=BF16, merge=2, prefill_impl=1)   # mma.sync prefill kernel
 
 
 @pytest.mark.parametrize("dtype,d,impl,merge", [(BF16, 128, 0, 0), (BF16, 128, 1, 0), (BF16, 64, 0, 0), (F32, 64, 0, 0),

@@ -70,7 +70,7 @@ def test_workspace_bytes_scales_with_rings_and_state(glide):
     (dict(windows=[-1, 4]), 1), (dict(max_tokens=0), 1), (dict(prefill_chunk=100), 1), (dict(decode_impl=9), 1),
     (dict(q_to_kv=[0, 0, 0, 0, 0, 1, 1, 1]), 2), (dict(q_to_kv=[0, 0, 0, 0, 1, 1, 1, 7]), 1),
     (dict(dtype=torch.float32, decode_impl=3), 2),
-    (dict(merge=3), 1), (dict(merge=1, decode_impl=1), 2), (dict(merge=2, prefill_impl=2), 2), (dict(prefill_impl=7), 1),
+    (dict(merge=3), 1), (dict(merge=1, decode_impl=1), 2), (dict(merge=2, prefill_impl=1), 2), (dict(prefill_impl=7), 1),
     (dict(dtype=torch.float32, prefill_impl=2), 2),
     # ring rows of one layer must fit 32-bit indices: 4096 sequences x 2 KV heads x 2^20 slots
     (dict(batch=4096, windows=[1 << 20, 16], max_tokens=1 << 20), 2),
