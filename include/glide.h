@@ -63,9 +63,9 @@ typedef enum { GLIDE_PHI_SOFTMAX = 0 } glide_phi;
  *   GLIDE_MERGE_SUM_EVICTED   phi(q) S / phi(q) z over the evicted tokens  +  window softmax
  *   GLIDE_MERGE_SUM_ALL       the same with a state that holds every token up to the current one (a token is
  *                             folded when it arrives, not when it leaves the window)
- * A term whose token set is empty counts as zero.  Decode runs them on the streaming tensor-core kernel (bf16,
- * head_dim 128) or the CUDA-core kernel, prefill on the CUDA-core kernels (decode_impl must not be MMA,
- * prefill_impl must be AUTO or FMA). */
+ * A term whose token set is empty counts as zero.  With bf16 I/O and head_dim 128 they run on the streaming decode
+ * kernel and the tcgen05 prefill kernel, otherwise on the CUDA-core kernels (decode_impl must not be MMA,
+ * prefill_impl must not be MMA_SYNC). */
 typedef enum { GLIDE_MERGE_SHARED = 0, GLIDE_MERGE_SUM_EVICTED = 1, GLIDE_MERGE_SUM_ALL = 2 } glide_merge;
 
 /* Decode kernel selection.  AUTO: for bf16 I/O the statically scheduled streaming tensor-core/TMA kernel
