@@ -30,7 +30,7 @@ namespace glide {
 namespace {
 
 constexpr int kD = 128;
-constexpr int kWarps = 8;
+constexpr int kWarps = kStreamWarps;
 constexpr int kThreads = kWarps * 32;
 constexpr int kTileRows = 16;
 constexpr uint32_t kStageBytes = 2 * kTileRows * kD * 2;   // 8 KiB: K box + V box, or 16 fp32 state rows
@@ -268,7 +268,7 @@ __device__ __forceinline__ void warp_sum_multi(float (&x)[N]) {
 
 // ---- the kernel -----------------------------------------------------------------------------
 template <int G, int STAGES, bool SUM>
-__global__ void __launch_bounds__(kThreads, 1)
+__global__ void __launch_bounds__(kThreads, GLIDE_STREAM_CTAS_PER_SM)
 glide_decode_stream_kernel(const DecodeParams p, const StreamParams sp) {
   using bf16 = __nv_bfloat16;
   using L = Layout<G, SUM>;
@@ -1307,7 +1307,7 @@ int stream_decode_supported(const glide_ctx *ctx) {
 }
 
 int stream_decode_setup(glide_ctx *ctx) {
-  const int n_ctas = std::min(ctx->sm_count, kMaxStreamCtas);
+  const int n_ctas = std::min(ctx->sm_count * GLIDE_STREAM_CTAS_PER_SM, kMaxStreamCtas);
   const int L = ctx->cfg.n_layers;
   ctx->stream_scheds.clear();
   ctx->stream_segs.clear();

@@ -282,7 +282,7 @@ int glide_create(const glide_config *cfg, void *dev_workspace, size_t workspace_
   if (ok && cfg->io_dtype == GLIDE_BF16 && cfg->decode_impl != GLIDE_DECODE_FMA) {
     ok = build_ring_tensor_maps(ctx) == GLIDE_OK;
     const bool want_stream = cfg->decode_impl == GLIDE_DECODE_AUTO || cfg->decode_impl == GLIDE_DECODE_STREAM;
-    if (ok && want_stream && stream_decode_supported(ctx) && ctx->sm_count <= kMaxStreamCtas) {
+    if (ok && want_stream && stream_decode_supported(ctx) && ctx->sm_count * GLIDE_STREAM_CTAS_PER_SM <= kMaxStreamCtas) {
       int rc2 = stream_decode_setup(ctx);
       if (rc2 == GLIDE_OK) ctx->decode_kind = 2;
       else if (rc2 != GLIDE_ERR_UNSUPPORTED) ok = false;

@@ -72,9 +72,18 @@ struct DecodeParams {
   int32_t layer_begin, layer_count;   // layers of this launch; q, k, v, out are indexed with the absolute layer
 };
 
-constexpr int kMaxStreamCtas = 192;           // CTAs (one per SM) the streaming decode kernel's schedule can address
-constexpr int kStreamWarps = 8;               // warps (= ranges of the schedule) per CTA
-constexpr int kStreamPoolBytes = 56 * 1024;   // shared-memory record slots for the CTA-level reduction
+#ifndef GLIDE_STREAM_WARPS
+#define GLIDE_STREAM_WARPS 8
+#endif
+#ifndef GLIDE_STREAM_CTAS_PER_SM
+#define GLIDE_STREAM_CTAS_PER_SM 1
+#endif
+#ifndef GLIDE_STREAM_POOL_KB
+#define GLIDE_STREAM_POOL_KB 56
+#endif
+constexpr int kMaxStreamCtas = 192 * GLIDE_STREAM_CTAS_PER_SM;   // CTAs the streaming decode kernel's schedule can address
+constexpr int kStreamWarps = GLIDE_STREAM_WARPS;                 // warps (= ranges of the schedule) per CTA
+constexpr int kStreamPoolBytes = GLIDE_STREAM_POOL_KB * 1024;    // shared-memory record slots for the CTA-level reduction
 constexpr int kStreamMaxGroups = 32;          // reduction groups per CTA
 
 // One segment of the streaming decode kernel's schedule: the part of one unit that falls into one warp's
