@@ -1045,11 +1045,11 @@ glide_decode_stream_kernel(const DecodeParams p, const StreamParams sp) {
 }
 
 template <int G, int STAGES, bool SUM>
-size_t stream_smem_bytes(int max_segs) {
+size_t stream_smem_bytes(int max_segs, int pool_slots) {
   using L = Layout<G, SUM>;
   return 1024 + size_t(kWarps) * STAGES * kStageBytes + size_t(kWarps) * L::kHdrBytes + size_t(kWarps) * STAGES * 64 +
          size_t(max_segs) * sizeof(StreamSegment) + size_t(kWarps) * (STAGES + 1) * 8 + size_t(kStreamMaxGroups) * 4 +
-         size_t(kStreamPoolBytes / (L::kRecFloats * 4)) * L::kRecFloats * 4;
+         size_t(pool_slots) * L::kRecFloats * 4;
 }
 
 // f(group size, stages, sum-of-terms merge)
@@ -1080,8 +1080,9 @@ int dispatch_stream(int G, bool sum, F &&f) {
 // Schedule for the layers [layer_begin, layer_begin + layer_count).  Units and query rows are numbered relative to
 // the first layer of the range (that is how a launch for the range addresses q, k, v, out and the tickets); the
 // layer index itself stays absolute (descriptors, layer table).
-void build_stream_schedule(const glide_ctx *ctx, int layer_begin, int layer_count, int n_ranges, std::vector<StreamSegment> *segs,
-                           std::vector<int32_t> *range_seg_begin, int *max_segs_per_cta, size_t *n_records) {
+void build_stream_schedule(const glide_ctx *ctx, int layer_begin, int layer_count, int n_ranges, int pool_slots,
+                           std::vector<StreamSegment> *segs, std::vector<int32_t> *range_seg_begin, int *max_segs_per_cta,
+                           size_t *n_records) {
   constexpr int64_t kSegWeight = GLIDE_W_UNIT, kStateWeight = GLIDE_W_STATE, kWinWeight = GLIDE_W_WIN;
   const int B = ctx->cfg.batch, Hkv = ctx->cfg.n_kv_heads, d = ctx->cfg.head_dim;
   const int n_ctas = n_ranges / kWarps;
@@ -1260,7 +1261,6 @@ void build_stream_schedule(const glide_ctx *ctx, int layer_begin, int layer_coun
   // Warps of one CTA that share a unit reduce their records in shared memory first (a "group"); only one
   // record per group goes to global scratch, and a unit that lies inside one group never touches it.
   size_t records = 0;
-  const int pool_slots = kStreamPoolBytes / (ctx->stream_rec_floats * 4);
   std::vector<int> cta_slots(size_t(n_ctas) + 1, 0), cta_groups(size_t(n_ctas) + 1, 0);
   for (size_t u = 0; u < unit_segs.size(); ++u) {
     std::vector<size_t> &list = unit_segs[u];
@@ -1309,25 +1309,11 @@ int stream_decode_supported(const glide_ctx *ctx) {
 int stream_decode_setup(glide_ctx *ctx) {
   const int n_ctas = std::min(ctx->sm_count * GLIDE_STREAM_CTAS_PER_SM, kMaxStreamCtas);
   const int L = ctx->cfg.n_layers;
-  ctx->stream_scheds.clear();
-  ctx->stream_segs.clear();
-  ctx->stream_max_segs = 1;
-  // [0]: all layers in one launch; [1 + l]: layer l alone, for callers that run other kernels between the layers
-  const int n_sched = L > 1 ? L + 1 : 1;
-  for (int si = 0; si < n_sched; ++si) {
-    std::vector<StreamSegment> segs;
-    glide_ctx::StreamSchedule sc;
-    int max_segs = 0;
-    size_t n_records = 0;
-    build_stream_schedule(ctx, si == 0 ? 0 : si - 1, si == 0 ? L : 1, n_ctas * kWarps, &segs, &sc.range_begin, &max_segs, &n_records);
-    if (n_records > ctx->stream_rec_capacity) return GLIDE_ERR_UNSUPPORTED;
-    sc.seg_base = ctx->stream_segs.size();
-    sc.n_segs = segs.size();
-    ctx->stream_segs.insert(ctx->stream_segs.end(), segs.begin(), segs.end());
-    ctx->stream_max_segs = std::max(ctx->stream_max_segs, max_segs);
-    ctx->stream_scheds.push_back(std::move(sc));
+  int dev_max = 0;
+  if (cudaDeviceGetAttribute(&dev_max, cudaDevAttrMaxSharedMemoryPerBlockOptin, ctx->device) != cudaSuccess) {
+    cudaGetLastError();
+    return GLIDE_ERR_CUDA;
   }
-  if (ctx->stream_segs.size() > ctx->stream_seg_capacity) return GLIDE_ERR_UNSUPPORTED;
   bool contiguous = true;
   for (int g = 0; g < ctx->cfg.n_kv_heads; ++g)
     for (int i = 1; i < ctx->G; ++i)
@@ -1336,13 +1322,36 @@ int stream_decode_setup(glide_ctx *ctx) {
   return dispatch_stream(ctx->G, ctx->cfg.merge != GLIDE_MERGE_SHARED, [&](auto gg, auto ss, auto mm) -> int {
     constexpr int G = decltype(gg)::value, S = decltype(ss)::value;
     constexpr bool SUM = decltype(mm)::value != 0;
-    const size_t smem = stream_smem_bytes<G, S, SUM>(ctx->stream_max_segs);
-    int dev_max = 0;
-    if (cudaDeviceGetAttribute(&dev_max, cudaDevAttrMaxSharedMemoryPerBlockOptin, ctx->device) != cudaSuccess) {
-      cudaGetLastError();
-      return GLIDE_ERR_CUDA;
+    // The record pool for the shared-memory groups takes what the segment table leaves, up to kStreamPoolBytes: with
+    // many small units per CTA (large batches) the table is large and hardly any unit is shared between warps.
+    const int rec_bytes = ctx->stream_rec_floats * 4;
+    int pool_slots = kStreamPoolBytes / rec_bytes;
+    for (int attempt = 0;; ++attempt) {
+      ctx->stream_scheds.clear();
+      ctx->stream_segs.clear();
+      ctx->stream_max_segs = 1;
+      // [0]: all layers in one launch; [1 + l]: layer l alone, for callers that run other kernels between the layers
+      const int n_sched = L > 1 ? L + 1 : 1;
+      for (int si = 0; si < n_sched; ++si) {
+        std::vector<StreamSegment> segs;
+        glide_ctx::StreamSchedule sc;
+        int max_segs = 0;
+        size_t n_records = 0;
+        build_stream_schedule(ctx, si == 0 ? 0 : si - 1, si == 0 ? L : 1, n_ctas * kWarps, pool_slots, &segs, &sc.range_begin,
+                              &max_segs, &n_records);
+        if (n_records > ctx->stream_rec_capacity) return GLIDE_ERR_UNSUPPORTED;
+        sc.seg_base = ctx->stream_segs.size();
+        sc.n_segs = segs.size();
+        ctx->stream_segs.insert(ctx->stream_segs.end(), segs.begin(), segs.end());
+        ctx->stream_max_segs = std::max(ctx->stream_max_segs, max_segs);
+        ctx->stream_scheds.push_back(std::move(sc));
+      }
+      if (ctx->stream_segs.size() > ctx->stream_seg_capacity) return GLIDE_ERR_UNSUPPORTED;
+      if (stream_smem_bytes<G, S, SUM>(ctx->stream_max_segs, pool_slots) <= size_t(dev_max)) break;
+      const size_t without_pool = stream_smem_bytes<G, S, SUM>(ctx->stream_max_segs, 0);
+      if (attempt > 0 || without_pool > size_t(dev_max)) return GLIDE_ERR_UNSUPPORTED;   // the table alone does not fit
+      pool_slots = int((size_t(dev_max) - without_pool) / size_t(rec_bytes));
     }
-    if (smem > size_t(dev_max)) return GLIDE_ERR_UNSUPPORTED;   // too many segments per CTA for the table
     auto kern = glide_decode_stream_kernel<G, S, SUM>;
     // the attribute belongs to the kernel, not to the context: ask for the device maximum so that contexts with
     // different schedules (different table sizes) can be alive together
@@ -1350,7 +1359,7 @@ int stream_decode_setup(glide_ctx *ctx) {
       cudaGetLastError();
       return GLIDE_ERR_CUDA;
     }
-    ctx->stream_smem = smem;
+    ctx->stream_smem = stream_smem_bytes<G, S, SUM>(ctx->stream_max_segs, pool_slots);
     ctx->decode_grid = n_ctas;
     return GLIDE_OK;
   });

@@ -298,3 +298,9 @@ def test_very_negative_window_logits_without_linear_terms(dtype, d, kw):
         out = torch.empty_like(q)
         g.glide_decode_step(q, k, v, out)
         check_outputs(out, stack.decode(to_np(q), to_np(k), to_np(v)), dtype, f"decode@{t}")
+
+
+def test_streaming_kernel_with_hundreds_of_units_per_cta():
+    # 32 768 small units: the segment table of a CTA takes over most of the shared-memory record pool; the streaming
+    # kernel (asked for explicitly) must still apply and agree with the oracle
+    run_case([0, 1] * 16, 128, 8, 8, 128, BF16, [], 3, amp=128 ** -0.5 * 4, seed=3, decode_impl=3, state_checks=False)
