@@ -120,9 +120,8 @@ def test_errors_and_capacity():
     assert g.glide_layer_info(1) == dict(window=4, capacity=4, n=0, count=0, head_slot=0, n_evicted=0)
 
 
-@pytest.mark.parametrize("impl", [1, 2, 3])   # prefill outputs: mma.sync, tcgen05 + TMEM, CUDA cores
-@pytest.mark.parametrize("G", [1, 4])
-@pytest.mark.parametrize("chunk", [96, 256])
+# prefill outputs: impl 1 mma.sync, 2 tcgen05 + TMEM, 3 CUDA cores
+@pytest.mark.parametrize("impl,G,chunk", [(1, 1, 96), (1, 4, 256), (2, 1, 256), (2, 4, 96), (2, 4, 256), (3, 4, 96)])
 def test_bf16_prefill_tensor_core_multi_call(impl, G, chunk):
     # several calls, so window tiles mix ring rows with the call's rows; windows below, at and above the
     # 128-key tile, one never-evicting layer, one purely linear layer; ragged last query tile
@@ -151,8 +150,7 @@ def test_contexts_with_different_schedules_coexist():
             check_outputs(out, ref, BF16, f"L={len(w)} step {t}")
 
 
-@pytest.mark.parametrize("G", [1, 2, 4, 8])
-@pytest.mark.parametrize("chunk", [96, 256])
+@pytest.mark.parametrize("G,chunk", [(1, 96), (2, 256), (4, 96), (4, 256), (8, 96)])
 def test_bf16_prefill_tcgen05_aligned_calls(G, chunk):
     # the tcgen05 kernel runs when every call starts at a multiple of 16 tokens and wrapping rings are multiples
     # of 16: windows below, at and above the 128-key tile, a ring that wraps several times, a never-evicting
