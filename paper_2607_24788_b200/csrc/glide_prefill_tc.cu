@@ -195,16 +195,6 @@ __device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32
   asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
 }
 
-#ifdef GLIDE_TC_PROFILE
-__device__ long long g_tc_prof[24];
-#define TC_MARK() long long tc_t_ = clock64(); long long tc_acc_[24] = {0,0,0,0,0,0,0,0,0,0,0,0,0,0,0,0,0,0,0,0,0,0,0,0}
-#define TC_ADD(i) do { long long n_ = clock64(); tc_acc_[i] += n_ - tc_t_; tc_t_ = n_; } while (0)
-#define TC_FLUSH(lo, hi) do { if (blockIdx.x == GLIDE_TC_PROFILE) for (int i_ = lo; i_ < hi; ++i_) atomicAdd(reinterpret_cast<unsigned long long *>(&g_tc_prof[i_]), (unsigned long long)tc_acc_[i_]); } while (0)
-#else
-#define TC_MARK() do { } while (0)
-#define TC_ADD(i) do { } while (0)
-#define TC_FLUSH(lo, hi) do { } while (0)
-#endif
 
 // (no wait: the caller issues tmem_wait_st() once after its last store)
 __device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&r)[16]) {
@@ -237,8 +227,8 @@ struct CallMaps {
   CUtensorMap k, v;
 };
 
-template <int G>
-__global__ void __launch_bounds__(kThreads, 1)
+template <int G, bool SUM>
+__global__ void __launch_bounds__(kThreads, 1)   // 10 warps = 3 on one scheduler: 168 registers per thread at most
 prefill_attn_tc_kernel(const PrefillParams p, const CUtensorMap *ring_maps, const __grid_constant__ CallMaps cm) {
   using bf16 = __nv_bfloat16;
   constexpr int TOKT = kRows / G;    // tokens per row tile
@@ -261,12 +251,11 @@ prefill_attn_tc_kernel(const PrefillParams p, const CUtensorMap *ring_maps, cons
   const int64_t tq_last = tq0 + ntok - 1;
   const int64_t w = ld.w;
   const int64_t wl = ld.wlin;                      // delay of the linear stream: w, or 0 when the state holds every token
-  const bool sum_terms = p.merge != GLIDE_MERGE_SHARED;
+  constexpr bool sum_terms = SUM;                  // sum of two normalised terms instead of the shared normaliser
   const uint32_t cap = ld.cap > 0 ? uint32_t(ld.cap) : 1u;
   const size_t unit_rows = (size_t(b) * p.Hkv + g) * size_t(ld.cap);
   const size_t seq = (size_t(lrel) * p.B + b) * size_t(p.T);
   volatile int *failed = &sm.failed;
-  TC_MARK();
 
   // a time-out recorded by an earlier CTA ends the launch quickly
   if (*reinterpret_cast<volatile int32_t *>(&p.ctl->status) == kDevWaitTimeout) return;
@@ -383,8 +372,6 @@ prefill_attn_tc_kernel(const PrefillParams p, const CUtensorMap *ring_maps, cons
     tmem_wait_st();
     return sum0 + sum1;
   };
-
-  TC_ADD(7);
   // =========================== window part: warp-specialised ===========================
   if (tid < kSoftmaxThreads) {
     if (activeX) {
@@ -402,14 +389,12 @@ prefill_attn_tc_kernel(const PrefillParams p, const CUtensorMap *ring_maps, cons
       cp_async_wait_all();
       fence_async_smem();
       mbar_arrive(smem_u32(&sm.bar_q[X]));
-      TC_ADD(11);
 
       const int64_t tqX0 = tq0 + X * TOKT, tqX_last = tqX0 + ntokX - 1;
       bool o_written = false;   // a P V product has been accumulated into O_X (uniform over the row tile)
       for (int t = 0; t < n_tiles; ++t) {
         const bool got = mbar_wait(smem_u32(&sm.bar_s[X]), uint32_t(t) & 1u, failed);
         if (!__all_sync(0xffffffffu, got)) break;   // warp-uniform: the collectives below need every lane
-        TC_ADD(0);
         tc_fence_after();
         const int64_t j0 = j_lo + int64_t(t) * kKT;
         const bool interior = j0 + kKT - 1 <= tqX0 && j0 > tqX_last - w;
@@ -435,7 +420,6 @@ prefill_attn_tc_kernel(const PrefillParams p, const CUtensorMap *ring_maps, cons
           mx = fmaxf(mx, fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3])));
         }
         mx *= p.scale_log2;
-        TC_ADD(1);
         // lazy reference: move it (and rescale O, l) only when the maximum grows by more than 2^kLazy
         float f = 1.f;
         if (mx > m_ref + kLazy || (m_ref == -CUDART_INF_F && mx > -CUDART_INF_F)) {
@@ -443,20 +427,17 @@ prefill_attn_tc_kernel(const PrefillParams p, const CUtensorMap *ring_maps, cons
           m_ref = mx;
         }
         if (o_written && __any_sync(0xffffffffu, f != 1.f)) scale_o(f);
-        TC_ADD(2);
         l_sum *= f;
         const float mr = m_ref == -CUDART_INF_F ? 0.f : m_ref;
         if (interior) l_sum += write_p(IntTag<0>{}, lo, hi, mr, p.scale_log2);
         else l_sum += write_p(IntTag<1>{}, lo, hi, mr, p.scale_log2);
         tc_fence_before();      // this thread's TMEM accesses precede the MMAs that read P and overwrite S
         mbar_arrive(smem_u32(&sm.bar_p[X]));
-        TC_ADD(3);
         o_written = true;
       }
     }
     if (n_tiles > 0) mbar_wait(smem_u32(&sm.bar_done), 0u, failed);
     tc_fence_after();
-    TC_ADD(4);
   } else if (warp == kMmaWarp) {
     if (lane == 0 && n_tiles > 0) {
       bool ok = mbar_wait(smem_u32(&sm.bar_q[0]), 0u, failed);
@@ -477,19 +458,16 @@ prefill_attn_tc_kernel(const PrefillParams p, const CUtensorMap *ring_maps, cons
         const bool more = t + 1 < n_tiles;
         ok = mbar_wait(smem_u32(&sm.bar_full[seqV % kStages]), uint32_t(seqV / kStages) & 1u, failed);
         if (ok && more) ok = mbar_wait(smem_u32(&sm.bar_full[seqK % kStages]), uint32_t(seqK / kStages) & 1u, failed);
-        TC_ADD(12);
         for (int x = 0; x < 2 && ok; ++x) {
           if (x == 1 && !hasB) break;
           ok = mbar_wait(smem_u32(&sm.bar_p[x]), uint32_t(t) & 1u, failed);
           if (!ok) break;
-          TC_ADD(13);
           tc_fence_after();
           issue_mma_ts(tmem + 256 + x * 128, tmem + x * 128, kv_addr(seqV % kStages), t > 0);
           if (more) {
             issue_mma(tmem + x * 128, sQ[x], kv_addr(seqK % kStages), false, false);
             mma_commit(smem_u32(&sm.bar_s[x]));
           }
-          TC_ADD(14);
         }
         if (ok) {
           mma_commit(smem_u32(&sm.bar_free[seqV % kStages]));
@@ -588,7 +566,6 @@ prefill_attn_tc_kernel(const PrefillParams p, const CUtensorMap *ring_maps, cons
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
-  TC_ADD(8);
 
   // =========================== linear part: the whole CTA in step ===========================
   // (no early exits from here on: every thread passes the same __syncthreads; after a time-out the waits return
@@ -672,7 +649,6 @@ prefill_attn_tc_kernel(const PrefillParams p, const CUtensorMap *ring_maps, cons
       for (int c = 0; c < 16; ++c)
         *reinterpret_cast<uint4 *>(sm.q[X] + sw128(row, c)) = make_uint4(phq[c * 4], phq[c * 4 + 1], phq[c * 4 + 2], phq[c * 4 + 3]);
     }
-    TC_ADD(9);
     if (folded > 0 && tid < kSoftmaxThreads) {
       // bf16 copy of the state as the MN-major B tile of the inter-chunk product
       mbar_wait(smem_u32(&sm.bar_state), 0u, failed);
@@ -707,7 +683,6 @@ prefill_attn_tc_kernel(const PrefillParams p, const CUtensorMap *ring_maps, cons
       wait_lin();
       o_init = true;
     }
-    TC_ADD(10);
     // intra-chunk: delayed tokens of this chunk up to the CTA's last token, 128 at a time
     const int i_lo = folded < 0 ? int(-folded < int64_t(p.C) ? -folded : int64_t(p.C)) : 0;
     const int i_hi = tok0 + ntok - 1;
@@ -738,13 +713,11 @@ prefill_attn_tc_kernel(const PrefillParams p, const CUtensorMap *ring_maps, cons
           cp_async16(kv_addr(slotV) + sw128(r, c), src + c * 8, valid);
         }
         cp_async_commit();
-        TC_ADD(16);
         cp_async_wait_all();
       }
       fence_async_smem();
       tc_fence_before();
       __syncthreads();
-      TC_ADD(17);
       if (tid == mma_tid) {
         tc_fence_after();
         issue_mma(tmem, sQ[0], kv_addr(slotPk), false, false);   // C_X = (phi(Q_X) 2^-m*) phi(K')^T
@@ -752,7 +725,6 @@ prefill_attn_tc_kernel(const PrefillParams p, const CUtensorMap *ring_maps, cons
         mma_commit(smem_u32(&sm.bar_lin));
       }
       wait_lin();
-      TC_ADD(18);
       if (activeX) {
         // C row -> bf16, masked to delayed tokens j' <= i of this row (the values already carry 2^-m*)
         float sum0 = 0.f, sum1 = 0.f;
@@ -789,7 +761,6 @@ prefill_attn_tc_kernel(const PrefillParams p, const CUtensorMap *ring_maps, cons
         tmem_wait_st();
         if (!sum_terms) l_sum += sum0 + sum1;
       }
-      TC_ADD(19);
       tc_fence_before();
       __syncthreads();
       if (tid == mma_tid) {
@@ -799,14 +770,12 @@ prefill_attn_tc_kernel(const PrefillParams p, const CUtensorMap *ring_maps, cons
         mma_commit(smem_u32(&sm.bar_lin));
       }
       wait_lin();
-      TC_ADD(20);
       o_init = true;
     }
   }
 
   // ---- shared normaliser and store: one contiguous 256-byte row per thread ------------------------------------
   __syncthreads();
-  TC_ADD(15);
   const bool bad = sm.failed != 0;
   if (bad) {
     if (tid == 0) atomicExch(&p.ctl->status, kDevWaitTimeout);
@@ -829,9 +798,6 @@ prefill_attn_tc_kernel(const PrefillParams p, const CUtensorMap *ring_maps, cons
       }
     }
   }
-  TC_ADD(6);
-  if (tid == 0) { TC_FLUSH(0, 12); TC_FLUSH(15, 24); }
-  if (tid == kMmaWarp * 32) { TC_FLUSH(12, 16); }
   tc_fence_before();
   __syncthreads();
   if (warp == 0) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 512;" ::"r"(tmem) : "memory");
@@ -839,16 +805,6 @@ prefill_attn_tc_kernel(const PrefillParams p, const CUtensorMap *ring_maps, cons
 
 }  // namespace
 
-#ifdef GLIDE_TC_PROFILE
-extern "C" int glide_debug_tc_profile(long long *out24, int reset) {
-  if (cudaMemcpyFromSymbol(out24, g_tc_prof, sizeof(long long) * 24) != cudaSuccess) return 6;
-  if (reset) {
-    long long z[24] = {};
-    if (cudaMemcpyToSymbol(g_tc_prof, z, sizeof(z)) != cudaSuccess) return 6;
-  }
-  return 0;
-}
-#endif
 
 // The kernel needs the ring descriptors made for the tensor-core decode kernels.
 bool prefill_attn_tc_supported(const glide_ctx *ctx) {
@@ -895,15 +851,17 @@ int launch_prefill_attn_tc(glide_ctx *ctx, const PrefillParams &p, cudaStream_t 
   auto launch = [&](auto gg) -> int {
     constexpr int G = decltype(gg)::value;
     constexpr int TOKC = 2 * kRows / G;
-    auto kern = prefill_attn_tc_kernel<G>;
     const size_t smem = sizeof(Smem) + 1024;
-    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem)) != cudaSuccess) {
-      cudaGetLastError();
-      return GLIDE_ERR_CUDA;
-    }
     const int64_t blocks = units * ((p.C + TOKC - 1) / TOKC);
-    kern<<<unsigned(blocks), kThreads, smem, stream>>>(p, ring_maps, cm);
-    return cudaGetLastError() == cudaSuccess ? GLIDE_OK : GLIDE_ERR_CUDA;
+    auto run = [&](auto kern) -> int {
+      if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem)) != cudaSuccess) {
+        cudaGetLastError();
+        return GLIDE_ERR_CUDA;
+      }
+      kern<<<unsigned(blocks), kThreads, smem, stream>>>(p, ring_maps, cm);
+      return cudaGetLastError() == cudaSuccess ? GLIDE_OK : GLIDE_ERR_CUDA;
+    };
+    return p.merge == GLIDE_MERGE_SHARED ? run(prefill_attn_tc_kernel<G, false>) : run(prefill_attn_tc_kernel<G, true>);
   };
   switch (ctx->G) {
     case 1: return launch(IntTag<1>{});
