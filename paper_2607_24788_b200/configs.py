@@ -106,3 +106,32 @@ def theoretical_speedup(alpha: float, w: float, d: float) -> float:
 def blockwise_cost(L: int, w: float, d: float, alpha: float) -> float:
     """Per-token cost of the (0, alpha*w, w) allocation with three equal blocks: Lwd/3 + Lw(1-alpha)d/3 + Ld^2."""
     return L * w * d / 3.0 + L * w * (1.0 - alpha) * d / 3.0 + L * d * d
+
+
+def three_block_split(n_layers: int) -> List[int]:
+    """Split of Algorithm 1: early, middle and last block of contiguous layers, as equal as the layer count allows
+    (a remainder goes to the earlier blocks, which keep the larger windows)."""
+    base, rem = divmod(n_layers, 3)
+    return [base + (1 if b < rem else 0) for b in range(3)]
+
+
+def blockwise_delta_candidates(w: int) -> List[int]:
+    """The search space of Algorithm 1 for the middle block: delta in {0, w/2, 15w/16, w}."""
+    return [0, w // 2, (15 * w) // 16, w]
+
+
+def blockwise_allocate(n_layers: int, w: int, task_acc_eval, split: Sequence[int] = None):
+    """Block-wise delta allocation (Algorithm 1).  The early block keeps delta = 0 (window w), the last block gets
+    delta = w (window 0: linear attention only); each candidate delta of the middle block is scored by
+    `task_acc_eval(windows) -> float` (the caller's task accuracy of the model run with these per-layer windows) and
+    the best one is kept.  Among equal scores the larger delta wins: it reads less of the cache for the same accuracy.
+    Returns (windows, delta_mid, {delta: score})."""
+    split = list(split) if split is not None else three_block_split(n_layers)
+    if len(split) != 3 or sum(split) != n_layers or min(split) < 0:
+        raise ValueError("split must give three block sizes that add up to n_layers")
+    scores = {}
+    for delta in blockwise_delta_candidates(w):
+        if delta not in scores:
+            scores[delta] = float(task_acc_eval(blockwise_windows(w, (0, delta, w), split)))
+    best = max(scores, key=lambda dl: (scores[dl], dl))
+    return blockwise_windows(w, (0, best, w), split), best, scores

@@ -59,3 +59,26 @@ def test_decode_step_bytes():
     assert C.decode_step_bytes(s, 3) == 2 * 4 * 4 * 64 * 4 + 2 * 4 * 64 * 4 + (8 + 8) * 64 * 4
     # n = 8 >= w: 8 slots + state read/write
     assert C.decode_step_bytes(s, 8) == 2 * 8 * 4 * 64 * 4 + 2 * (4 * 64 * 64 + 4 * 64) * 4 + 2 * 4 * 64 * 4 + 16 * 64 * 4
+
+
+def test_blockwise_allocation_search():
+    # Algorithm 1: early block delta 0, last block delta w, the middle block's delta picked by the caller's score
+    assert C.three_block_split(32) == [11, 11, 10] and C.three_block_split(30) == [10, 10, 10]
+    assert C.blockwise_delta_candidates(1024) == [0, 512, 960, 1024]
+    seen = []
+
+    def acc(windows):
+        seen.append(list(windows))
+        return {1024: 0.70, 512: 0.69, 64: 0.71, 0: 0.40}[windows[15]]
+
+    windows, delta, scores = C.blockwise_allocate(32, 1024, acc, split=(10, 12, 10))
+    assert delta == 960 and windows == [1024] * 10 + [64] * 12 + [0] * 10
+    assert scores == {0: 0.70, 512: 0.69, 960: 0.71, 1024: 0.40}
+    assert len(seen) == 4 and all(s[:10] == [1024] * 10 and s[22:] == [0] * 10 for s in seen)
+    # equal scores: the allocation that reads less of the cache
+    _, delta, _ = C.blockwise_allocate(30, 1024, lambda ws: 1.0)
+    assert delta == 1024
+    # the chosen row reproduces the KV I/O the table prints for it (0, 15w/16, w): 43 MiB
+    assert round(C.kv_io_bytes_per_token(windows) / MiB) == 43
+    with pytest.raises(ValueError):
+        C.blockwise_allocate(32, 1024, acc, split=(10, 10, 10))
