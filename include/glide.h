@@ -179,13 +179,36 @@ int glide_decode_step_layers(glide_ctx *ctx, int32_t layer_begin, int32_t layer_
 int glide_decode_step_noalloc(glide_ctx *ctx, const void *dev_q, const void *dev_k, const void *dev_v, void *dev_out,
                               void *stream);
 
+/* ---- sequences of different lengths (continuous batching) -----------------------------------------
+ * The method is defined per sequence (Sec. II "KV Cache", Sec. III-B): nothing couples the B sequences of a
+ * context, so each slot b may hold a sequence of its own length.  The position of slot b at layer l is the layer's
+ * counter (moved by glide_prefill and the decode steps, which advance every slot together) plus an offset of the
+ * slot, which the three calls below change.  They act on all layers and need all layers level (GLIDE_ERR_STATE
+ * otherwise).  A decode step always advances every slot by one token: a slot that holds no live sequence is
+ * stepped along with whatever its input rows contain (finite values keep its state finite) and is reset before it
+ * is used again; the capacity check of a step is against the longest slot.  glide_prefill for all slots at once
+ * needs them at one position. */
+
+/* Slot b starts an empty sequence: position 0, S and z zeroed (ring rows need no clearing).  Other slots are
+ * untouched.  Stream-ordered. */
+int glide_reset_seq(glide_ctx *ctx, int32_t b, void *stream);
+
+/* glide_prefill for slot b alone, all layers: appends T tokens to that sequence.
+ *   dev_q, dev_out [L][T][H][d] (dev_out NULL: state only);  dev_k, dev_v [L][T][H_kv][d]. */
+int glide_prefill_seq(glide_ctx *ctx, int32_t b, int64_t T, const void *dev_q, const void *dev_k, const void *dev_v,
+                      void *dev_out, void *stream);
+
+/* Tokens slot b holds, as the host tracks them (no device access). */
+int glide_seq_tokens(glide_ctx *ctx, int32_t b, int64_t *n_out);
+
 /* Free the host context.  Does not touch the workspace. */
 int glide_destroy(glide_ctx *ctx);
 
 /* ---- test / benchmark support -------------------------------------------------------------- */
 
-/* Bookkeeping of one layer, read back from the device counters (synchronises `stream`). */
+/* Bookkeeping of one layer, read back from the device counters (synchronises `stream`): slot 0, or slot b. */
 int glide_layer_info(glide_ctx *ctx, int32_t layer, void *stream, glide_layer_info_t *out);
+int glide_seq_layer_info(glide_ctx *ctx, int32_t layer, int32_t b, void *stream, glide_layer_info_t *out);
 
 /* Copy one layer's state to caller DEVICE buffers (any may be NULL):
  *   dev_ringK, dev_ringV [B][H_kv][capacity][d] in the I/O dtype (slot order);
@@ -194,11 +217,11 @@ int glide_export_state(glide_ctx *ctx, int32_t layer, void *dev_ringK, void *dev
                        float *dev_z, void *stream);
 
 /* Overwrite one layer's state from caller DEVICE buffers (same layouts; NULL leaves that part
- * as it is) and set its position to n (0 <= n <= max_tokens). */
+ * as it is) and set the layer's counter to n (0 <= n <= max_tokens; slot offsets stay as they are). */
 int glide_import_state(glide_ctx *ctx, int32_t layer, int64_t n, const void *dev_ringK, const void *dev_ringV,
                        const float *dev_S, const float *dev_z, void *stream);
 
-/* Back to the empty state: counters, S and z zeroed (rings need no clearing). */
+/* Back to the empty state: counters, slot offsets, S and z zeroed (rings need no clearing). */
 int glide_reset(glide_ctx *ctx, void *stream);
 
 /* Status word written by device-side range checks (0 = none tripped).  Synchronises `stream`. */

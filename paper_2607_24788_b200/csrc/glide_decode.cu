@@ -333,9 +333,9 @@ __global__ void __launch_bounds__(kDecodeThreads) glide_decode_kernel(const Deco
     }
     if (it.layer < p.layer_begin || it.layer >= p.layer_begin + p.layer_count) continue;   // not a layer of this launch
     const LayerDev ld = p.layers[it.layer];
-    const int64_t t = p.n_dev[it.layer];
     const int ub = it.unit - it.layer * units_per_layer;
     const int b = ub / p.Hkv, g = ub - b * p.Hkv;
+    const int64_t t = p.n_dev[it.layer] + (p.seq_off ? p.seq_off[b] : 0);   // position of this sequence
     const int per_unit = ld.n_win_items + ld.n_state_items;
     float *rec = p.partials + ld.part_base + (size_t(ub) * per_unit + it.part) * p.rec_floats;
     if (it.kind == kItemWindow)
@@ -392,6 +392,7 @@ DecodeParams make_decode_params(const glide_ctx *ctx, int layer_begin, int layer
   p.tickets = reinterpret_cast<int32_t *>(ctx->ws + ctx->off_tickets);
   p.partials = reinterpret_cast<float *>(ctx->ws + ctx->off_partials);
   p.n_dev = reinterpret_cast<int64_t *>(ctx->ws + ctx->off_ndev);
+  p.seq_off = ctx->ragged ? reinterpret_cast<const int64_t *>(ctx->ws + ctx->off_seqoff) : nullptr;
   p.q = q;
   p.k = k;
   p.v = v;

@@ -596,9 +596,9 @@ __global__ void __launch_bounds__(WARPS * 32, 1) glide_decode_mma_kernel(const D
     }
     if (it.layer < p.layer_begin || it.layer >= p.layer_begin + p.layer_count) continue;   // not a layer of this launch
     const LayerDev ld = p.layers[it.layer];
-    const int64_t t = p.n_dev[it.layer];
     const int ub = it.unit - it.layer * units_per_layer;
     const int b = ub / p.Hkv, g = ub - b * p.Hkv;
+    const int64_t t = p.n_dev[it.layer] + (p.seq_off ? p.seq_off[b] : 0);   // position of this sequence
     const int per_unit = ld.n_win_items + ld.n_state_items;
     float *rec = p.partials + ld.part_base + (size_t(ub) * per_unit + it.part) * p.rec_floats;
     GLIDE_TRACE_EVENT(it.kind == kItemWindow ? 3 : 4);

@@ -190,13 +190,15 @@ __device__ __forceinline__ void tma_load_4d(uint32_t dst, const void *tmap, int 
       : "memory");
 }
 
-__device__ __forceinline__ bool seg_evicting(const StreamSegment &s, int64_t t) {
+__device__ __forceinline__ bool seg_evicting(const StreamSegment &s) {
+  const int64_t t = s.t;
   // evicts bit 0: the layer has a state; bit 1: the token folded at a step is the current one (no ring, or a state
   // that holds every token), otherwise the one that leaves the window
   return (s.evicts & 1) && ((s.evicts & 2) || t >= int64_t(s.w));
 }
 // window tiles of the segment that hold window tokens at position t
-__device__ __forceinline__ int seg_valid_win(const StreamSegment &s, int64_t t) {
+__device__ __forceinline__ int seg_valid_win(const StreamSegment &s) {
+  const int64_t t = s.t;
   const int64_t lim = t < int64_t(s.cap) ? t : int64_t(s.cap);
   const int nv = int((lim + kTileRows - 1) / kTileRows) - s.win0;
   return nv < 0 ? 0 : (nv > s.n_win ? s.n_win : nv);
@@ -209,11 +211,11 @@ struct Cursor {
   int n_state_eff, n_total;
 };
 
-__device__ __forceinline__ void cursor_enter(Cursor &c, const StreamSegment *segs, int64_t t) {
+__device__ __forceinline__ void cursor_enter(Cursor &c, const StreamSegment *segs) {
   const StreamSegment &s = segs[c.seg];
   c.k = 0;
-  c.n_state_eff = seg_evicting(s, t) ? s.n_state : 0;
-  c.n_total = c.n_state_eff + seg_valid_win(s, t);
+  c.n_state_eff = seg_evicting(s) ? s.n_state : 0;
+  c.n_total = c.n_state_eff + seg_valid_win(s);
 }
 
 // Records.  Shared normaliser: (acc[G][d], m[G], l[G]) with the linear readout already folded in as a term with
@@ -299,7 +301,20 @@ glide_decode_stream_kernel(const DecodeParams p, const StreamParams sp) {
   if (cta_nseg > 0) {
     const uint4 *src = reinterpret_cast<const uint4 *>(sp.segs + cta_seg_begin);
     uint4 *dst = reinterpret_cast<uint4 *>(sm_segs);
-    for (int i = tid; i < cta_nseg * int(sizeof(StreamSegment) / 16); i += kThreads) dst[i] = src[i];
+    // A sequence's position is the layers' common counter plus the sequence's own offset (zero unless sequences
+    // were reset or prefilled one by one; written by copies from the host, never by a kernel, so it may be read
+    // before the preceding kernel has completed).  The position goes into the last 16 bytes of every segment of
+    // the CTA's shared copy: {b, pad, t}.
+    constexpr int kChunks = int(sizeof(StreamSegment) / 16);
+    for (int i = tid; i < cta_nseg * kChunks; i += kThreads) {
+      uint4 c = src[i];
+      if (i % kChunks == kChunks - 1) {
+        const int64_t t = p.t_host + (p.seq_off ? p.seq_off[c.x] : 0);
+        c.z = uint32_t(uint64_t(t));
+        c.w = uint32_t(uint64_t(t) >> 32);
+      }
+      dst[i] = c;
+    }
   }
   unsigned char *my_stages_ptr = sm_stages + size_t(warp) * STAGES * kStageBytes;
   const uint32_t my_stages = smem_u32(my_stages_ptr);
@@ -325,11 +340,10 @@ glide_decode_stream_kernel(const DecodeParams p, const StreamParams sp) {
   asm volatile("griddepcontrol.wait;" ::: "memory");   // the preceding kernel has completed and its writes are visible
   // every layer is at the same position (checked by the host); the host's copy of the counter comes with the
   // launch, which saves a dependent global load at the head of every warp's critical path
-  const int64_t t = p.t_host;
   // the device counters are not read by this kernel; one thread moves them on (no grid-wide completion count,
   // which would put an atomic round trip at the end of every CTA)
   if (blockIdx.x == 0)
-    for (int l = tid; l < p.layer_count; l += kThreads) p.n_dev[p.layer_begin + l] = t + 1;
+    for (int l = tid; l < p.layer_count; l += kThreads) p.n_dev[p.layer_begin + l] = p.t_host + 1;
   // this warp's segments: the run of the CTA's list that carries its index
   int seg_lo = 0;
   while (seg_lo < cta_nseg && sm_segs[seg_lo].range < warp) ++seg_lo;
@@ -342,7 +356,8 @@ glide_decode_stream_kernel(const DecodeParams p, const StreamParams sp) {
   auto issue_header = [&](int s) {
     if (lane == 0) {
       const StreamSegment &sg = sm_segs[s];
-      const bool ev = seg_evicting(sg, t);
+      const int64_t t = sg.t;
+      const bool ev = seg_evicting(sg);
       fence_async_smem();
       mbar_expect_tx(hdr_bar, G * 256 + 512 + (ev ? 512 : 0));
       const bf16 *qall = reinterpret_cast<const bf16 *>(p.q);
@@ -373,12 +388,12 @@ glide_decode_stream_kernel(const DecodeParams p, const StreamParams sp) {
   Cursor icur;
   icur.seg = seg_lo;
   icur.k = icur.n_state_eff = icur.n_total = 0;
-  if (seg_lo < seg_hi) cursor_enter(icur, sm_segs, t);
+  if (seg_lo < seg_hi) cursor_enter(icur, sm_segs);
   int issue_stage = 0;
   auto issue_next = [&]() {
     if (lane == 0) {
       while (icur.seg < seg_hi && icur.k >= icur.n_total) {
-        if (++icur.seg < seg_hi) cursor_enter(icur, sm_segs, t);
+        if (++icur.seg < seg_hi) cursor_enter(icur, sm_segs);
       }
       if (icur.seg < seg_hi) {
         const StreamSegment &sg = sm_segs[icur.seg];
@@ -575,9 +590,10 @@ glide_decode_stream_kernel(const DecodeParams p, const StreamParams sp) {
   // ---- main loop over this warp's segments ------------------------------------------------------------
   for (int s = seg_lo; s < seg_hi && !failed; ++s) {
     const StreamSegment &sg = sm_segs[s];
-    const bool ev = seg_evicting(sg, t);
+    const int64_t t = sg.t;
+    const bool ev = seg_evicting(sg);
     const int n_state_eff = ev ? sg.n_state : 0;
-    const int n_total = n_state_eff + seg_valid_win(sg, t);
+    const int n_total = n_state_eff + seg_valid_win(sg);
     const bool has_win = sg.cap > 0;
 
     // -- header: q fragments, current token, feature maps -> registers; then prefetch the next header --
@@ -1025,7 +1041,7 @@ glide_decode_stream_kernel(const DecodeParams p, const StreamParams sp) {
         *reinterpret_cast<uint2 *>(reinterpret_cast<bf16 *>(p.out) + size_t(orow[h]) * kD + lane * 4) = packed;
       }
       if (has_win) {
-        const size_t row = (size_t(sg.row_base) + size_t(t % int64_t(sg.cap))) * kD;
+        const size_t row = (size_t(sg.row_base) + size_t(sg.t % int64_t(sg.cap))) * kD;
         reinterpret_cast<uint2 *>(reinterpret_cast<bf16 *>(p.ws + size_t(sg.ringK_off256) * 256) + row)[lane] = ktb;
         reinterpret_cast<uint2 *>(reinterpret_cast<bf16 *>(p.ws + size_t(sg.ringV_off256) * 256) + row)[lane] = vtb;
       }
@@ -1234,6 +1250,8 @@ void build_stream_schedule(const glide_ctx *ctx, int layer_begin, int layer_coun
         sg.ringK_off256 = int32_t(ld.ringK / 256);
         sg.ringV_off256 = int32_t(ld.ringV / 256);
         sg.g = int32_t(ub % Hkv);
+        sg.b = int32_t(ub / Hkv);
+        sg.t = 0;
         {
           const int64_t b = ub / Hkv;
           const int64_t row = (int64_t(pc.layer - layer_begin) * B + b) * ctx->cfg.n_q_heads;

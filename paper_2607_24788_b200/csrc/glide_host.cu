@@ -94,6 +94,7 @@ int glide::plan_context(const glide_config *cfg, glide_ctx *ctx, std::vector<Wor
   ctx->cfg.windows = nullptr;
   ctx->cfg.q_to_kv = nullptr;
   ctx->n_host.assign(L, 0);
+  ctx->seq_off.assign(size_t(cfg->batch), 0);
   ctx->rec_floats = int(align_up(size_t(ctx->G) * (d + 2), 4));
   ctx->stream_rec_floats = ctx->rec_floats * (cfg->merge == GLIDE_MERGE_SHARED ? 1 : 2);
 
@@ -133,6 +134,8 @@ int glide::plan_context(const glide_config *cfg, glide_ctx *ctx, std::vector<Wor
   off = align_up(off + sizeof(Control), 256);
   ctx->off_ndev = off;
   off = align_up(off + sizeof(int64_t) * L, 256);
+  ctx->off_seqoff = off;   // per-sequence position offsets (zeroed with the counters)
+  off = align_up(off + sizeof(int64_t) * size_t(cfg->batch), 256);
   ctx->off_layers = off;
   off = align_up(off + sizeof(LayerDev) * L, 256);
   ctx->off_heads = off;
@@ -339,6 +342,32 @@ int glide_destroy(glide_ctx *ctx) {
   return GLIDE_OK;
 }
 
+namespace {
+int64_t max_seq_off(const glide_ctx *ctx) {
+  int64_t m = ctx->seq_off.empty() ? 0 : ctx->seq_off[0];
+  for (int64_t o : ctx->seq_off) m = std::max(m, o);
+  return m;
+}
+bool layers_level(const glide_ctx *ctx) {
+  for (size_t l = 1; l < ctx->n_host.size(); ++l)
+    if (ctx->n_host[l] != ctx->n_host[0]) return false;
+  return true;
+}
+// new offset of sequence b, on the host and (ordered on the stream) on the device
+int set_seq_off(glide_ctx *ctx, int b, int64_t off, cudaStream_t st) {
+  // pageable 8-byte source: the runtime stages it before returning
+  if (cudaMemcpyAsync(ctx->ws + ctx->off_seqoff + sizeof(int64_t) * size_t(b), &off, sizeof(int64_t),
+                      cudaMemcpyHostToDevice, st) != cudaSuccess) {
+    cudaGetLastError();
+    return GLIDE_ERR_CUDA;
+  }
+  ctx->seq_off[size_t(b)] = off;
+  ctx->ragged = false;
+  for (int64_t o : ctx->seq_off) ctx->ragged = ctx->ragged || o != 0;
+  return GLIDE_OK;
+}
+}  // namespace
+
 int glide_decode_step_layers(glide_ctx *ctx, int32_t layer_begin, int32_t layer_count, const void *q, const void *k,
                              const void *v, void *out, void *stream) {
   if (!ctx || !q || !k || !v || !out) return GLIDE_ERR_INVALID_ARG;
@@ -346,7 +375,7 @@ int glide_decode_step_layers(glide_ctx *ctx, int32_t layer_begin, int32_t layer_
   if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out)) return GLIDE_ERR_INVALID_ARG;
   for (int l = layer_begin + 1; l < layer_begin + layer_count; ++l)
     if (ctx->n_host[l] != ctx->n_host[layer_begin]) return GLIDE_ERR_STATE;
-  if (ctx->n_host[layer_begin] + 1 > ctx->cfg.max_tokens) return GLIDE_ERR_CAPACITY;
+  if (ctx->n_host[layer_begin] + max_seq_off(ctx) + 1 > ctx->cfg.max_tokens) return GLIDE_ERR_CAPACITY;
   int rc = launch_decode(ctx, layer_begin, layer_count, q, k, v, out, as_stream(stream));
   if (rc) return rc;
   for (int l = layer_begin; l < layer_begin + layer_count; ++l) ctx->n_host[l] += 1;
@@ -364,7 +393,7 @@ int glide_decode_step_noalloc(glide_ctx *ctx, const void *q, const void *k, cons
   const int L = ctx->cfg.n_layers;
   for (int l = 1; l < L; ++l)
     if (ctx->n_host[l] != ctx->n_host[0]) return GLIDE_ERR_STATE;
-  if (ctx->n_host[0] + 1 > ctx->cfg.max_tokens) return GLIDE_ERR_CAPACITY;
+  if (ctx->n_host[0] + max_seq_off(ctx) + 1 > ctx->cfg.max_tokens) return GLIDE_ERR_CAPACITY;
   int rc = launch_decode_noalloc(ctx, q, k, v, out, as_stream(stream));
   if (rc) return rc;
   for (int l = 0; l < L; ++l) ctx->n_host[l] += 1;
@@ -380,24 +409,70 @@ int glide_prefill(glide_ctx *ctx, int32_t layer_begin, int32_t layer_count, int6
   if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out)) return GLIDE_ERR_INVALID_ARG;
   for (int l = layer_begin + 1; l < layer_begin + layer_count; ++l)
     if (ctx->n_host[l] != ctx->n_host[layer_begin]) return GLIDE_ERR_STATE;
-  if (ctx->n_host[layer_begin] + T > ctx->cfg.max_tokens) return GLIDE_ERR_CAPACITY;
+  // one call for all sequences needs them at one position
+  for (int64_t o : ctx->seq_off)
+    if (o != ctx->seq_off[0]) return GLIDE_ERR_STATE;
+  if (ctx->n_host[layer_begin] + ctx->seq_off[0] + T > ctx->cfg.max_tokens) return GLIDE_ERR_CAPACITY;
   if (T == 0) return GLIDE_OK;
-  int rc = launch_prefill(ctx, layer_begin, layer_count, T, q, k, v, out, as_stream(stream));
+  int rc = launch_prefill(ctx, layer_begin, layer_count, T, q, k, v, out, -1, ctx->n_host[layer_begin] + ctx->seq_off[0],
+                          as_stream(stream));
   if (rc) return rc;
   for (int l = layer_begin; l < layer_begin + layer_count; ++l) ctx->n_host[l] += T;
   return GLIDE_OK;
 }
 
-int glide_layer_info(glide_ctx *ctx, int32_t layer, void *stream, glide_layer_info_t *out) {
-  if (!ctx || !out || layer < 0 || layer >= ctx->cfg.n_layers) return GLIDE_ERR_INVALID_ARG;
-  int64_t n = 0;
+int glide_prefill_seq(glide_ctx *ctx, int32_t b, int64_t T, const void *q, const void *k, const void *v, void *out,
+                      void *stream) {
+  if (!ctx || !k || !v || T < 0 || b < 0 || b >= ctx->cfg.batch) return GLIDE_ERR_INVALID_ARG;
+  if (out && !q) return GLIDE_ERR_INVALID_ARG;
+  if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out)) return GLIDE_ERR_INVALID_ARG;
+  if (!layers_level(ctx)) return GLIDE_ERR_STATE;
+  const int64_t n0 = ctx->n_host[0] + ctx->seq_off[size_t(b)];
+  if (n0 + T > ctx->cfg.max_tokens) return GLIDE_ERR_CAPACITY;
+  if (T == 0) return GLIDE_OK;
+  int rc = launch_prefill(ctx, 0, ctx->cfg.n_layers, T, q, k, v, out, b, n0, as_stream(stream));
+  if (rc) return rc;
+  return set_seq_off(ctx, b, ctx->seq_off[size_t(b)] + T, as_stream(stream));
+}
+
+int glide_reset_seq(glide_ctx *ctx, int32_t b, void *stream) {
+  if (!ctx || b < 0 || b >= ctx->cfg.batch) return GLIDE_ERR_INVALID_ARG;
+  if (!layers_level(ctx)) return GLIDE_ERR_STATE;
+  cudaStream_t st = as_stream(stream);
+  // S and z of the slot start at zero; ring rows need no clearing (slots at or beyond the position are never read)
+  const size_t d = size_t(ctx->cfg.head_dim), Hkv = size_t(ctx->cfg.n_kv_heads);
+  bool ok = true;
+  for (const LayerDev &ld : ctx->layers) {
+    ok = ok && cudaMemsetAsync(ctx->ws + ld.S + size_t(b) * Hkv * d * d * 4, 0, Hkv * d * d * 4, st) == cudaSuccess;
+    ok = ok && cudaMemsetAsync(ctx->ws + ld.z + size_t(b) * Hkv * d * 4, 0, Hkv * d * 4, st) == cudaSuccess;
+  }
+  if (!ok) {
+    cudaGetLastError();
+    return GLIDE_ERR_CUDA;
+  }
+  return set_seq_off(ctx, b, -ctx->n_host[0], st);
+}
+
+int glide_seq_tokens(glide_ctx *ctx, int32_t b, int64_t *n_out) {
+  if (!ctx || !n_out || b < 0 || b >= ctx->cfg.batch) return GLIDE_ERR_INVALID_ARG;
+  if (!layers_level(ctx)) return GLIDE_ERR_STATE;
+  *n_out = ctx->n_host[0] + ctx->seq_off[size_t(b)];
+  return GLIDE_OK;
+}
+
+int glide_seq_layer_info(glide_ctx *ctx, int32_t layer, int32_t b, void *stream, glide_layer_info_t *out) {
+  if (!ctx || !out || layer < 0 || layer >= ctx->cfg.n_layers || b < 0 || b >= ctx->cfg.batch) return GLIDE_ERR_INVALID_ARG;
+  int64_t n = 0, off = 0;
   cudaStream_t st = as_stream(stream);
   if (cudaMemcpyAsync(&n, ctx->ws + ctx->off_ndev + sizeof(int64_t) * layer, sizeof(int64_t), cudaMemcpyDeviceToHost,
                       st) != cudaSuccess ||
+      cudaMemcpyAsync(&off, ctx->ws + ctx->off_seqoff + sizeof(int64_t) * size_t(b), sizeof(int64_t),
+                      cudaMemcpyDeviceToHost, st) != cudaSuccess ||
       cudaStreamSynchronize(st) != cudaSuccess) {
     cudaGetLastError();
     return GLIDE_ERR_CUDA;
   }
+  n += off;
   const LayerDev &ld = ctx->layers[layer];
   out->window = ld.w;
   out->capacity = ld.cap;
@@ -406,6 +481,10 @@ int glide_layer_info(glide_ctx *ctx, int32_t layer, void *stream, glide_layer_in
   out->head_slot = ld.cap > 0 ? n % ld.cap : 0;
   out->n_evicted = std::max<int64_t>(0, n - ld.w);
   return GLIDE_OK;
+}
+
+int glide_layer_info(glide_ctx *ctx, int32_t layer, void *stream, glide_layer_info_t *out) {
+  return glide_seq_layer_info(ctx, layer, 0, stream, out);
 }
 
 int glide_export_state(glide_ctx *ctx, int32_t layer, void *ringK, void *ringV, float *S, float *z, void *stream) {
@@ -461,6 +540,8 @@ int glide_reset(glide_ctx *ctx, void *stream) {
     return GLIDE_ERR_CUDA;
   }
   std::fill(ctx->n_host.begin(), ctx->n_host.end(), 0);
+  std::fill(ctx->seq_off.begin(), ctx->seq_off.end(), 0);
+  ctx->ragged = false;
   return GLIDE_OK;
 }
 

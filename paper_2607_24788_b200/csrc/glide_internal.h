@@ -2,6 +2,7 @@
 #pragma once
 
 #include <cuda_runtime.h>
+#include <stddef.h>
 #include <stdint.h>
 
 #include <vector>
@@ -62,6 +63,7 @@ struct DecodeParams {
   int32_t *tickets;          // [units]
   float *partials;
   int64_t *n_dev;            // [L]
+  const int64_t *seq_off;    // [B] position of sequence b minus the layer's counter; null when every offset is zero
   const void *q, *k, *v;
   void *out;
   int32_t n_items;
@@ -108,8 +110,12 @@ struct StreamSegment {
   int32_t grp_slot0;         // first shared-memory record slot of the group
   int32_t grp_idx;           // this segment's slot within the group
   int32_t grp_ctr;           // the group's arrival counter in shared memory
+  int32_t b;                 // sequence of the unit
+  int32_t pad_;
+  int64_t t;                 // position of the unit's sequence at this step: written into the CTA's shared copy by the kernel
 };
-static_assert(sizeof(StreamSegment) == 96, "StreamSegment is copied as 16-byte chunks");
+static_assert(sizeof(StreamSegment) == 112, "StreamSegment is copied as 16-byte chunks");
+static_assert(offsetof(StreamSegment, b) == 96 && offsetof(StreamSegment, t) == 104, "the last chunk is {b, pad, t}");
 
 struct StreamParams {
   const StreamSegment *segs;
@@ -136,7 +142,8 @@ struct PrefillParams {
   int32_t C;                 // tokens in the current chunk
   int32_t Cmax;              // scratch stride (prefill_chunk)
   int32_t layer_begin, layer_count;
-  int32_t L, B, H, Hkv;
+  int32_t L, B, H, Hkv;      // B: sequences of the call's tensors
+  int32_t b0;                // sequence slot of the context that the call's sequence 0 is (0 unless one sequence is prefilled)
   float scale_log2;
 };
 
@@ -149,6 +156,8 @@ struct glide_ctx {
   std::vector<int32_t> heads_of;    // [Hkv][G]
   std::vector<glide::LayerDev> layers;
   std::vector<int64_t> n_host;      // mirror of the device counters
+  std::vector<int64_t> seq_off;     // [B] mirror of the per-sequence offsets: sequence b of layer l is at n_host[l] + seq_off[b]
+  bool ragged = false;              // some offset is not zero
   std::vector<unsigned char> tmaps_host;  // TMA descriptors of the rings (bf16 tensor-core decode kernel)
   int decode_kind = 0;              // 0 CUDA-core kernel, 1 per-item tensor-core kernel, 2 streaming tensor-core kernel
   // schedules of the streaming kernel: [0] all layers; [1 + l] layer l alone (built when L > 1)
@@ -178,7 +187,7 @@ struct glide_ctx {
   unsigned char *ws = nullptr;
   size_t ws_bytes = 0;
   // workspace regions (byte offsets)
-  size_t off_ctl = 0, off_ndev = 0, off_layers = 0, off_heads = 0, off_items = 0, off_tickets = 0,
+  size_t off_ctl = 0, off_ndev = 0, off_seqoff = 0, off_layers = 0, off_heads = 0, off_items = 0, off_tickets = 0,
          off_partials = 0, off_tmaps = 0, off_phik = 0, off_zcum = 0, off_state = 0, off_ring = 0, total = 0;
   size_t state_bytes = 0;           // S and z of all layers (contiguous)
   size_t item_part_floats = 0;      // floats of split-K records the per-item work list needs
@@ -202,8 +211,10 @@ int launch_decode_noalloc(glide_ctx *ctx, const void *q, const void *k, const vo
 int launch_decode(glide_ctx *ctx, int layer_begin, int layer_count, const void *q, const void *k, const void *v, void *out,
                   cudaStream_t stream);
 int decode_occupancy(const glide_ctx *ctx, int *blocks_per_sm);
+// seq < 0: the call's tensors hold all B sequences, the layers' counters advance; otherwise they hold sequence slot
+// `seq` alone ([layer_count][1][T]...), which is at position n0, and no counter is touched
 int launch_prefill(glide_ctx *ctx, int layer_begin, int layer_count, int64_t T, const void *q, const void *k,
-                   const void *v, void *out, cudaStream_t stream);
+                   const void *v, void *out, int seq, int64_t n0, cudaStream_t stream);
 bool prefill_attn_tc_supported(const glide_ctx *ctx);
 int launch_prefill_attn_tc(glide_ctx *ctx, const PrefillParams &p, cudaStream_t stream);
 bool prefill_attn_mma_supported(const glide_ctx *ctx);

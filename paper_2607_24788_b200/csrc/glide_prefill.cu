@@ -38,7 +38,7 @@ struct RowSource {
 template <typename T, int D>
 __device__ __forceinline__ RowSource<T> make_source(const PrefillParams &p, const LayerDev &ld, int lrel, int b, int g) {
   RowSource<T> s;
-  const size_t unit_rows = (size_t(b) * p.Hkv + g) * size_t(ld.cap);
+  const size_t unit_rows = (size_t(b + p.b0) * p.Hkv + g) * size_t(ld.cap);   // b + b0: the sequence's slot in the context
   s.ringK = reinterpret_cast<const T *>(p.ws + ld.ringK) + unit_rows * D;
   s.ringV = reinterpret_cast<const T *>(p.ws + ld.ringV) + unit_rows * D;
   const size_t seq = (size_t(lrel) * p.B + b) * size_t(p.T) * p.Hkv * D + size_t(g) * D;
@@ -94,7 +94,7 @@ __global__ void __launch_bounds__(kPrefillThreads) prefill_attn_kernel(const Pre
   const LayerDev ld = p.layers[p.layer_begin + lrel];
   const RowSource<T> src = make_source<T, D>(p, ld, lrel, b, g);
   const int64_t tq = p.n0 + p.c0 + i;  // absolute position of the query
-  const int ub = b * p.Hkv + g;
+  const int ub = (b + p.b0) * p.Hkv + g;
 
   float qr[G][E];
   const T *qbase = reinterpret_cast<const T *>(p.q) + ((size_t(lrel) * p.B + b) * size_t(p.T) + size_t(p.c0 + i)) * p.H * D;
@@ -243,7 +243,7 @@ __global__ void __launch_bounds__(kPrefillThreads) prefill_state_kernel(const Pr
   const int i_lo = first < 0 ? int(first < -int64_t(p.C) ? p.C : -first) : 0;
   if (i_lo >= p.C) return;
   const RowSource<T> src = make_source<T, D>(p, ld, lrel, b, g);
-  const int ub = b * p.Hkv + g;
+  const int ub = (b + p.b0) * p.Hkv + g;
   const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
   const float *pk = p.phik + size_t(u) * p.Cmax * D + rb * kStateRows;
   float acc[8][4 * CG];
@@ -355,7 +355,7 @@ __global__ void __launch_bounds__(kPrefillThreads) prefill_ring_kernel(const Pre
   if (ld.cap == 0 || int64_t(i) < int64_t(p.C) - ld.cap) return;  // older tokens of the chunk are overwritten anyway
   const int64_t j = p.n0 + p.c0 + i;
   const size_t src = (((size_t(lrel) * p.B + b) * size_t(p.T) + size_t(p.c0 + i)) * p.Hkv + g) * D + lane * E;
-  const size_t dst = ((size_t(b) * p.Hkv + g) * size_t(ld.cap) + size_t(j % ld.cap)) * D + lane * E;
+  const size_t dst = ((size_t(b + p.b0) * p.Hkv + g) * size_t(ld.cap) + size_t(j % ld.cap)) * D + lane * E;
   const T *ks = reinterpret_cast<const T *>(p.k) + src;
   const T *vs = reinterpret_cast<const T *>(p.v) + src;
   T *kd = reinterpret_cast<T *>(p.ws + ld.ringK) + dst;
@@ -370,7 +370,7 @@ __global__ void __launch_bounds__(kPrefillThreads) prefill_ring_kernel(const Pre
 }  // namespace
 
 int launch_prefill(glide_ctx *ctx, int layer_begin, int layer_count, int64_t T, const void *q, const void *k,
-                   const void *v, void *out, cudaStream_t stream) {
+                   const void *v, void *out, int seq, int64_t n0, cudaStream_t stream) {
   PrefillParams p{};
   p.ws = ctx->ws;
   p.layers = reinterpret_cast<const LayerDev *>(ctx->ws + ctx->off_layers);
@@ -383,13 +383,14 @@ int launch_prefill(glide_ctx *ctx, int layer_begin, int layer_count, int64_t T, 
   p.k = k;
   p.v = v;
   p.out = out;
-  p.n0 = ctx->n_host[layer_begin];
+  p.n0 = n0;
   p.T = T;
   p.Cmax = ctx->prefill_chunk;
   p.layer_begin = layer_begin;
   p.layer_count = layer_count;
   p.L = ctx->cfg.n_layers;
-  p.B = ctx->cfg.batch;
+  p.B = seq < 0 ? ctx->cfg.batch : 1;
+  p.b0 = seq < 0 ? 0 : seq;
   p.H = ctx->cfg.n_q_heads;
   p.Hkv = ctx->cfg.n_kv_heads;
   p.scale_log2 = ctx->scale * kLog2e;
@@ -433,7 +434,7 @@ int launch_prefill(glide_ctx *ctx, int layer_begin, int layer_count, int64_t T, 
     return GLIDE_OK;
   });
   if (rc) return rc;
-  return launch_advance(ctx, layer_begin, layer_count, T, stream);
+  return seq < 0 ? launch_advance(ctx, layer_begin, layer_count, T, stream) : GLIDE_OK;
 }
 
 }  // namespace glide

@@ -105,7 +105,7 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_attn_mma_kernel(const Pre
   const int64_t w = ld.w;
   const int64_t cap = ld.cap > 0 ? ld.cap : 1;
 
-  const size_t unit_rows = (size_t(b) * p.Hkv + g) * size_t(ld.cap);
+  const size_t unit_rows = (size_t(b + p.b0) * p.Hkv + g) * size_t(ld.cap);
   const bf16 *ringK = reinterpret_cast<const bf16 *>(p.ws + ld.ringK) + unit_rows * kD;
   const bf16 *ringV = reinterpret_cast<const bf16 *>(p.ws + ld.ringV) + unit_rows * kD;
   const size_t seq = (size_t(lrel) * p.B + b) * size_t(p.T);
@@ -353,7 +353,7 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_attn_mma_kernel(const Pre
         qf[ks][3] = scale2(qf[ks][3], fl[1]);
       }
     }
-    const int ub = b * p.Hkv + g;
+    const int ub = (b + p.b0) * p.Hkv + g;
     const int64_t folded = p.n0 + p.c0 - w;   // tokens below this index are in S, z at the start of the chunk
     if (folded > 0) {
       // inter-chunk: the state as a bf16 "V tile" (features on the key axis), two halves of 64 rows

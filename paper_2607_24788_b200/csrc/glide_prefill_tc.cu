@@ -253,7 +253,7 @@ prefill_attn_tc_kernel(const PrefillParams p, const CUtensorMap *ring_maps, cons
   const int64_t wl = ld.wlin;                      // delay of the linear stream: w, or 0 when the state holds every token
   constexpr bool sum_terms = SUM;                  // sum of two normalised terms instead of the shared normaliser
   const uint32_t cap = ld.cap > 0 ? uint32_t(ld.cap) : 1u;
-  const size_t unit_rows = (size_t(b) * p.Hkv + g) * size_t(ld.cap);
+  const size_t unit_rows = (size_t(b + p.b0) * p.Hkv + g) * size_t(ld.cap);   // b + b0: the sequence's slot in the context
   const size_t seq = (size_t(lrel) * p.B + b) * size_t(p.T);
   volatile int *failed = &sm.failed;
 
@@ -553,7 +553,7 @@ prefill_attn_tc_kernel(const PrefillParams p, const CUtensorMap *ring_maps, cons
         if (sq >= 0) ok = mbar_wait(smem_u32(&sm.bar_free[sq % kStages]), uint32_t(sq / kStages) & 1u, failed);
       }
       if (ok) {
-        const int ub = b * p.Hkv + g;
+        const int ub = (b + p.b0) * p.Hkv + g;
         const unsigned char *Sg = p.ws + ld.S + size_t(ub) * kD * kD * sizeof(float);
         const uint32_t bar = smem_u32(&sm.bar_state);
         mbar_expect_tx(bar, uint32_t(kD * kD * sizeof(float) + kD * sizeof(float)));

@@ -19,6 +19,7 @@ GLIDE_F32, GLIDE_BF16 = 0, 1
 GLIDE_PHI_SOFTMAX = 0
 GLIDE_MERGE_SHARED, GLIDE_MERGE_SUM_EVICTED, GLIDE_MERGE_SUM_ALL = 0, 1, 2
 GLIDE_DECODE_AUTO, GLIDE_DECODE_MMA, GLIDE_DECODE_FMA, GLIDE_DECODE_STREAM = 0, 1, 2, 3
+GLIDE_PREFILL_AUTO, GLIDE_PREFILL_MMA_SYNC, GLIDE_PREFILL_TCGEN05, GLIDE_PREFILL_FMA = 0, 1, 2, 3
 
 GLIDE_OK = 0
 GLIDE_ERR_INVALID_ARG = 1
@@ -72,6 +73,10 @@ def load_library() -> ctypes.CDLL:
     lib.glide_decode_step.argtypes = [vp, vp, vp, vp, vp, vp]
     lib.glide_decode_step_noalloc.argtypes = [vp, vp, vp, vp, vp, vp]
     lib.glide_decode_step_layers.argtypes = [vp, i32, i32, vp, vp, vp, vp, vp]
+    lib.glide_reset_seq.argtypes = [vp, i32, vp]
+    lib.glide_prefill_seq.argtypes = [vp, i32, i64, vp, vp, vp, vp, vp]
+    lib.glide_seq_tokens.argtypes = [vp, i32, ctypes.POINTER(i64)]
+    lib.glide_seq_layer_info.argtypes = [vp, i32, i32, vp, ctypes.POINTER(glide_layer_info_t)]
     lib.glide_destroy.argtypes = [vp]
     lib.glide_layer_info.argtypes = [vp, i32, vp, ctypes.POINTER(glide_layer_info_t)]
     lib.glide_export_state.argtypes = [vp, i32, vp, vp, vp, vp, vp]
@@ -201,6 +206,32 @@ class Glide:
         assert q.dtype == k.dtype == v.dtype == out.dtype == self.dtype
         _check(self.lib.glide_decode_step_noalloc(self._h, _ptr(q), _ptr(k), _ptr(v), _ptr(out), _stream(stream)),
                "glide_decode_step_noalloc")
+
+    # -- sequences of different lengths: every slot of the batch has its own position ---------------
+    def glide_reset_seq(self, b: int, stream=None) -> None:
+        """Slot b starts an empty sequence; the other slots are untouched."""
+        _check(self.lib.glide_reset_seq(self._h, int(b), _stream(stream)), "glide_reset_seq")
+
+    def glide_prefill_seq(self, b: int, q: Optional[torch.Tensor], k: torch.Tensor, v: torch.Tensor,
+                          out: Optional[torch.Tensor] = None, stream=None) -> None:
+        """glide_prefill for slot b alone, all layers: q, out [L][T][H][d]; k, v [L][T][H_kv][d]."""
+        T = k.shape[1]
+        assert k.shape == (self.L, T, self.Hkv, self.d) and v.shape == k.shape and k.dtype == self.dtype
+        if out is not None:
+            assert q is not None and q.shape == (self.L, T, self.H, self.d) and out.shape == q.shape
+        _check(self.lib.glide_prefill_seq(self._h, int(b), T, _ptr(q), _ptr(k), _ptr(v), _ptr(out), _stream(stream)),
+               "glide_prefill_seq")
+
+    def glide_seq_tokens(self, b: int) -> int:
+        n = ctypes.c_int64(0)
+        _check(self.lib.glide_seq_tokens(self._h, int(b), ctypes.byref(n)), "glide_seq_tokens")
+        return int(n.value)
+
+    def glide_seq_layer_info(self, layer: int, b: int) -> dict:
+        info = glide_layer_info_t()
+        _check(self.lib.glide_seq_layer_info(self._h, layer, int(b), _stream(None), ctypes.byref(info)),
+               "glide_seq_layer_info")
+        return {n: int(getattr(info, n)) for n, _ in glide_layer_info_t._fields_}
 
     def glide_destroy(self) -> None:
         if getattr(self, "_h", None):

@@ -1,0 +1,194 @@
+"""Sequences of different lengths in one context (continuous batching) against the CPU oracle.
+
+Every slot of the batch holds its own sequence: slots are prefilled one by one with prompts of different lengths,
+decoded together, reset and refilled while the others keep going.  The oracle side is one independent cell per
+(layer, live sequence), so nothing but the per-sequence definition of the method enters the expected values.
+"""
+import numpy as np
+import pytest
+import torch
+
+from oracle import glide_oracle as orc
+from paper_2607_24788_b200 import glide, synth
+from tests.parity_util import STATE_REL_L2, check_outputs, f32_scale, to_np
+
+pytestmark = pytest.mark.gpu
+
+N_IDS = 64   # logical sequences of the synthetic workload (slots draw fresh ids from it)
+
+
+class Ragged:
+    """The CUDA context and, per slot, the oracle cells of the sequence that lives there."""
+
+    def __init__(self, windows, B, H, Hkv, d, dtype, max_tokens, seed=0, amp=1.0, **cfg_kw):
+        self.L, self.B, self.H, self.Hkv, self.d, self.dtype = len(windows), B, H, Hkv, d, dtype
+        self.windows, self.merge = list(windows), cfg_kw.get("merge", 0)
+        self.scale = f32_scale(d)
+        self.wl = synth.Workload(seed, self.L, N_IDS, H, Hkv, d, dtype, amp)
+        self.g = glide.Glide(windows, B, H, Hkv, d, max_tokens, dtype=dtype, device="cuda", softmax_scale=self.scale,
+                             **cfg_kw)
+        self.next_id = 0
+        self.ids, self.pos, self.cells = [0] * B, [0] * B, [None] * B
+        for b in range(B):
+            self.new_sequence(b, reset=False)
+        self.worst = 0.0
+
+    def new_sequence(self, b, reset=True):
+        self.ids[b], self.pos[b] = self.next_id, 0
+        self.next_id += 1
+        self.cells[b] = [orc.Cell(self.H, self.Hkv, self.d, w, self.scale, merge=self.merge) for w in self.windows]
+        if reset:
+            self.g.glide_reset_seq(b)
+
+    def prefill_seq(self, b, T, outputs=True):
+        q, k, v = self.wl.qkv(range(self.L), [self.ids[b]], range(self.pos[b], self.pos[b] + T), device="cuda")
+        q, k, v = q[:, 0].contiguous(), k[:, 0].contiguous(), v[:, 0].contiguous()
+        out = torch.full_like(q, float("nan")) if outputs else None
+        self.g.glide_prefill_seq(b, q if outputs else None, k, v, out)
+        for l in range(self.L):
+            ref = self.cells[b][l].prefill(to_np(q[l]), to_np(k[l]), to_np(v[l]), outputs=outputs)
+            if outputs:
+                self.worst = max(self.worst, check_outputs(out[l], ref, self.dtype, f"prefill slot {b} layer {l} @{self.pos[b]}+{T}"))
+        self.pos[b] += T
+        assert self.g.glide_seq_tokens(b) == self.pos[b]
+
+    def _step_inputs(self):
+        parts = [self.wl.qkv(range(self.L), [self.ids[b]], [self.pos[b]], device="cuda") for b in range(self.B)]
+        return [torch.cat([p[i][:, :, 0] for p in parts], dim=1).contiguous() for i in range(3)]
+
+    def decode(self, steps=1, by_layer=False):
+        for _ in range(steps):
+            q, k, v = self._step_inputs()
+            out = torch.full_like(q, float("nan"))
+            if by_layer:
+                for l in range(self.L):
+                    self.g.glide_decode_step_layers(q[l:l + 1], k[l:l + 1], v[l:l + 1], out[l:l + 1], l, 1)
+            else:
+                self.g.glide_decode_step(q, k, v, out)
+            for b in range(self.B):
+                ref = np.stack([self.cells[b][l].decode(to_np(q[l, b]), to_np(k[l, b]), to_np(v[l, b])) for l in range(self.L)])
+                self.worst = max(self.worst, check_outputs(out[:, b], ref, self.dtype, f"decode slot {b} t={self.pos[b]}"))
+                self.pos[b] += 1
+
+    def check_state(self, what=""):
+        g = self.g
+        for l in range(self.L):
+            rk, rv, S, z = g.glide_export_state(l)
+            for b in range(self.B):
+                cell = self.cells[b][l]
+                info, oi = g.glide_seq_layer_info(l, b), cell.info()
+                assert (info["n"], info["count"], info["n_evicted"]) == (oi["n"], oi["count"], oi["n_evicted"]), (what, l, b, info, oi)
+                cap = info["capacity"]
+                if cap:
+                    assert info["head_slot"] == oi["n"] % cap
+                ork, orv, oS, oz = cell.export()
+                tok = cell.slot_tokens()
+                valid = np.nonzero(tok[:cap] >= 0)[0] if cap else np.array([], dtype=np.int64)
+                if len(valid):
+                    np.testing.assert_array_equal(to_np(rk[b])[:, valid], ork[:, valid], err_msg=f"{what} ringK l{l} b{b}")
+                    np.testing.assert_array_equal(to_np(rv[b])[:, valid], orv[:, valid], err_msg=f"{what} ringV l{l} b{b}")
+                for name, a, r in (("S", to_np(S[b]), oS), ("z", to_np(z[b]), oz)):
+                    nr = np.linalg.norm(r)
+                    if nr == 0:
+                        assert np.abs(a).max() == 0, f"{what} {name} l{l} b{b} should be zero"
+                    else:
+                        assert np.linalg.norm(a - r) / nr <= STATE_REL_L2, f"{what} {name} l{l} b{b}"
+        assert g.glide_device_status() == 0
+
+
+def scenario(r: Ragged, prompts, by_layer=False):
+    """prompts of different lengths, joint decode, one slot reset and refilled in two calls, joint decode again"""
+    for b, T in enumerate(prompts):
+        if T:
+            r.prefill_seq(b, T)
+    r.check_state("after the prompts")
+    r.decode(5, by_layer=by_layer)
+    r.check_state("after the first decode steps")
+    victim = 1 % r.B
+    r.new_sequence(victim)
+    r.check_state("after resetting a slot")
+    r.prefill_seq(victim, 40)
+    r.prefill_seq(victim, 27, outputs=False)
+    r.decode(6, by_layer=by_layer)
+    # a slot that was never prefilled decodes from position 0 on; another reset right before a step
+    r.new_sequence(0)
+    r.decode(3, by_layer=by_layer)
+    r.check_state("at the end")
+    r.g.glide_destroy()
+    return r.worst
+
+
+@pytest.mark.parametrize("merge", [0, 1, 2])
+def test_ragged_fp32_cuda_cores(merge):
+    r = Ragged([48, 16, 0, 200], 3, 4, 2, 64, torch.float32, 400, seed=3, amp=1.5, merge=merge, prefill_chunk=32)
+    scenario(r, [37, 5, 150])
+
+
+@pytest.mark.parametrize("merge", [0, 1, 2])
+def test_ragged_bf16_streaming_and_tcgen05(merge):
+    # (the sum of two normalised terms is up to twice as large as one: smaller values keep bf16 output rounding
+    # inside the absolute tolerance)
+    r = Ragged([64, 16, 0, 300, 128], 4, 8, 2, 128, torch.bfloat16, 600, seed=4, amp=1.0 if merge == 0 else 0.5,
+               merge=merge, prefill_chunk=64)
+    scenario(r, [130, 0, 333, 17])
+
+
+def test_ragged_bf16_layer_by_layer():
+    r = Ragged([64, 0, 160], 3, 8, 2, 128, torch.bfloat16, 500, seed=5, prefill_chunk=64)
+    scenario(r, [100, 7, 261], by_layer=True)
+
+
+def test_ragged_bf16_per_item_mma_and_mma_sync_prefill():
+    r = Ragged([64, 16, 0, 300], 3, 8, 2, 128, torch.bfloat16, 600, seed=6, prefill_chunk=64,
+               decode_impl=glide.GLIDE_DECODE_MMA, prefill_impl=glide.GLIDE_PREFILL_MMA_SYNC)
+    scenario(r, [130, 2, 333])
+
+
+def test_ragged_noalloc_step():
+    r = Ragged([32, 0, 100], 2, 4, 2, 64, torch.float32, 300, seed=7)
+    r.prefill_seq(0, 120)
+    r.prefill_seq(1, 9)
+    for _ in range(4):
+        q, k, v = r._step_inputs()
+        out = torch.full_like(q, float("nan"))
+        r.g.glide_decode_step_noalloc(q, k, v, out)
+        for b in range(r.B):
+            ref = np.stack([r.cells[b][l].decode(to_np(q[l, b]), to_np(k[l, b]), to_np(v[l, b])) for l in range(r.L)])
+            check_outputs(out[:, b], ref, r.dtype, f"noalloc slot {b}")
+            r.pos[b] += 1
+    r.check_state("noalloc")
+    r.g.glide_destroy()
+
+
+def test_joint_prefill_needs_level_slots_and_capacity_follows_the_longest_slot():
+    L, B, H, Hkv, d = 2, 2, 4, 2, 64
+    r = Ragged([16, 0], B, H, Hkv, d, torch.float32, 64, seed=8)
+    r.prefill_seq(0, 50)
+    q, k, v = r.wl.qkv(range(L), [0, 1], range(0, 4), device="cuda")
+    with pytest.raises(glide.GlideError) as e:
+        r.g.glide_prefill(q, k, v, torch.empty_like(q))
+    assert e.value.code == glide.GLIDE_ERR_STATE
+    with pytest.raises(glide.GlideError) as e:
+        r.prefill_seq(0, 15)                      # 50 + 15 > 64
+    assert e.value.code == glide.GLIDE_ERR_CAPACITY
+    r.decode(14)                                   # slot 0 reaches 64 tokens
+    q, k, v = r._step_inputs()
+    with pytest.raises(glide.GlideError) as e:
+        r.g.glide_decode_step(q, k, v, torch.empty_like(q))
+    assert e.value.code == glide.GLIDE_ERR_CAPACITY
+    # every slot reset: level again (all offsets equal), a joint prefill works and matches fresh sequences
+    for b in range(B):
+        r.new_sequence(b)
+    q, k, v = r.wl.qkv(range(L), r.ids, range(0, 20), device="cuda")
+    out = torch.full_like(q, float("nan"))
+    r.g.glide_prefill(q, k, v, out)
+    for b in range(B):
+        for l in range(L):
+            ref = r.cells[b][l].prefill(to_np(q[l, b]), to_np(k[l, b]), to_np(v[l, b]))
+            check_outputs(out[l, b], ref, r.dtype, "joint prefill after resets")
+        r.pos[b] += 20
+    r.decode(3)
+    r.check_state("after joint prefill")
+    r.g.glide_reset()
+    assert [r.g.glide_seq_tokens(b) for b in range(B)] == [0, 0]
+    r.g.glide_destroy()
