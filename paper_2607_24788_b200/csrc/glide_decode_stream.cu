@@ -190,15 +190,13 @@ __device__ __forceinline__ void tma_load_4d(uint32_t dst, const void *tmap, int 
       : "memory");
 }
 
-__device__ __forceinline__ bool seg_evicting(const StreamSegment &s) {
-  const int64_t t = s.t;
+__device__ __forceinline__ bool seg_evicting(const StreamSegment &s, int64_t t) {
   // evicts bit 0: the layer has a state; bit 1: the token folded at a step is the current one (no ring, or a state
   // that holds every token), otherwise the one that leaves the window
   return (s.evicts & 1) && ((s.evicts & 2) || t >= int64_t(s.w));
 }
 // window tiles of the segment that hold window tokens at position t
-__device__ __forceinline__ int seg_valid_win(const StreamSegment &s) {
-  const int64_t t = s.t;
+__device__ __forceinline__ int seg_valid_win(const StreamSegment &s, int64_t t) {
   const int64_t lim = t < int64_t(s.cap) ? t : int64_t(s.cap);
   const int nv = int((lim + kTileRows - 1) / kTileRows) - s.win0;
   return nv < 0 ? 0 : (nv > s.n_win ? s.n_win : nv);
@@ -211,11 +209,11 @@ struct Cursor {
   int n_state_eff, n_total;
 };
 
-__device__ __forceinline__ void cursor_enter(Cursor &c, const StreamSegment *segs) {
+__device__ __forceinline__ void cursor_enter(Cursor &c, const StreamSegment *segs, int64_t t) {
   const StreamSegment &s = segs[c.seg];
   c.k = 0;
-  c.n_state_eff = seg_evicting(s) ? s.n_state : 0;
-  c.n_total = c.n_state_eff + seg_valid_win(s);
+  c.n_state_eff = seg_evicting(s, t) ? s.n_state : 0;
+  c.n_total = c.n_state_eff + seg_valid_win(s, t);
 }
 
 // Records.  Shared normaliser: (acc[G][d], m[G], l[G]) with the linear readout already folded in as a term with
@@ -269,7 +267,7 @@ __device__ __forceinline__ void warp_sum_multi(float (&x)[N]) {
 }
 
 // ---- the kernel -----------------------------------------------------------------------------
-template <int G, int STAGES, bool SUM>
+template <int G, int STAGES, bool SUM, bool RAGGED>
 __global__ void __launch_bounds__(kThreads, GLIDE_STREAM_CTAS_PER_SM)
 glide_decode_stream_kernel(const DecodeParams p, const StreamParams sp) {
   using bf16 = __nv_bfloat16;
@@ -285,6 +283,7 @@ glide_decode_stream_kernel(const DecodeParams p, const StreamParams sp) {
   uint64_t *sm_bars = reinterpret_cast<uint64_t *>(sm_segs + sp.max_segs);          // [kWarps][STAGES + 1]
   int *sm_ctr = reinterpret_cast<int *>(sm_bars + kWarps * (STAGES + 1));             // [kStreamMaxGroups]
   float *sm_pool = reinterpret_cast<float *>(sm_ctr + kStreamMaxGroups);              // [pool slots][kRecFloats]
+  int64_t *sm_t = reinterpret_cast<int64_t *>(base + sp.t_off);                       // [max_segs], behind the pool
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 #ifdef GLIDE_TRACE
@@ -301,20 +300,7 @@ glide_decode_stream_kernel(const DecodeParams p, const StreamParams sp) {
   if (cta_nseg > 0) {
     const uint4 *src = reinterpret_cast<const uint4 *>(sp.segs + cta_seg_begin);
     uint4 *dst = reinterpret_cast<uint4 *>(sm_segs);
-    // A sequence's position is the layers' common counter plus the sequence's own offset (zero unless sequences
-    // were reset or prefilled one by one; written by copies from the host, never by a kernel, so it may be read
-    // before the preceding kernel has completed).  The position goes into the last 16 bytes of every segment of
-    // the CTA's shared copy: {b, pad, t}.
-    constexpr int kChunks = int(sizeof(StreamSegment) / 16);
-    for (int i = tid; i < cta_nseg * kChunks; i += kThreads) {
-      uint4 c = src[i];
-      if (i % kChunks == kChunks - 1) {
-        const int64_t t = p.t_host + (p.seq_off ? p.seq_off[c.x] : 0);
-        c.z = uint32_t(uint64_t(t));
-        c.w = uint32_t(uint64_t(t) >> 32);
-      }
-      dst[i] = c;
-    }
+    for (int i = tid; i < cta_nseg * int(sizeof(StreamSegment) / 16); i += kThreads) dst[i] = src[i];
   }
   unsigned char *my_stages_ptr = sm_stages + size_t(warp) * STAGES * kStageBytes;
   const uint32_t my_stages = smem_u32(my_stages_ptr);
@@ -330,7 +316,17 @@ glide_decode_stream_kernel(const DecodeParams p, const StreamParams sp) {
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     fence_async_smem();
   }
-  __syncthreads();   // segment table and barriers ready; the warps are on their own from here
+  __syncthreads();   // segment table and barriers ready
+  // A sequence's position is the layers' common counter, which comes with the launch, plus the sequence's own offset
+  // (zero unless sequences were reset or prefilled one by one; written by copies from the host, never by a kernel,
+  // so it may be read before the preceding kernel has completed).  Level batches (RAGGED false: an instantiation of
+  // its own, so that the B = 1 step carries none of this) take the position from the launch parameters.
+  constexpr bool ragged = RAGGED;
+  if (ragged) {
+    for (int i = tid; i < cta_nseg; i += kThreads) sm_t[i] = p.t_host + p.seq_off[(sm_segs[i].unit / p.Hkv) % p.B];
+    __syncthreads();
+  }
+  auto pos_of = [&](int s) -> int64_t { return ragged ? sm_t[s] : p.t_host; };
 #if GLIDE_STREAM_TMAP_PREFETCH
   // the ring descriptors are written when the context is created, never by a kernel: fetch the ones this
   // CTA's segments use before waiting for the preceding kernel
@@ -356,8 +352,8 @@ glide_decode_stream_kernel(const DecodeParams p, const StreamParams sp) {
   auto issue_header = [&](int s) {
     if (lane == 0) {
       const StreamSegment &sg = sm_segs[s];
-      const int64_t t = sg.t;
-      const bool ev = seg_evicting(sg);
+      const int64_t t = pos_of(s);
+      const bool ev = seg_evicting(sg, t);
       fence_async_smem();
       mbar_expect_tx(hdr_bar, G * 256 + 512 + (ev ? 512 : 0));
       const bf16 *qall = reinterpret_cast<const bf16 *>(p.q);
@@ -388,12 +384,12 @@ glide_decode_stream_kernel(const DecodeParams p, const StreamParams sp) {
   Cursor icur;
   icur.seg = seg_lo;
   icur.k = icur.n_state_eff = icur.n_total = 0;
-  if (seg_lo < seg_hi) cursor_enter(icur, sm_segs);
+  if (seg_lo < seg_hi) cursor_enter(icur, sm_segs, pos_of(icur.seg));
   int issue_stage = 0;
   auto issue_next = [&]() {
     if (lane == 0) {
       while (icur.seg < seg_hi && icur.k >= icur.n_total) {
-        if (++icur.seg < seg_hi) cursor_enter(icur, sm_segs);
+        if (++icur.seg < seg_hi) cursor_enter(icur, sm_segs, pos_of(icur.seg));
       }
       if (icur.seg < seg_hi) {
         const StreamSegment &sg = sm_segs[icur.seg];
@@ -590,10 +586,10 @@ glide_decode_stream_kernel(const DecodeParams p, const StreamParams sp) {
   // ---- main loop over this warp's segments ------------------------------------------------------------
   for (int s = seg_lo; s < seg_hi && !failed; ++s) {
     const StreamSegment &sg = sm_segs[s];
-    const int64_t t = sg.t;
-    const bool ev = seg_evicting(sg);
+    const int64_t t = pos_of(s);
+    const bool ev = seg_evicting(sg, t);
     const int n_state_eff = ev ? sg.n_state : 0;
-    const int n_total = n_state_eff + seg_valid_win(sg);
+    const int n_total = n_state_eff + seg_valid_win(sg, t);
     const bool has_win = sg.cap > 0;
 
     // -- header: q fragments, current token, feature maps -> registers; then prefetch the next header --
@@ -1041,7 +1037,7 @@ glide_decode_stream_kernel(const DecodeParams p, const StreamParams sp) {
         *reinterpret_cast<uint2 *>(reinterpret_cast<bf16 *>(p.out) + size_t(orow[h]) * kD + lane * 4) = packed;
       }
       if (has_win) {
-        const size_t row = (size_t(sg.row_base) + size_t(sg.t % int64_t(sg.cap))) * kD;
+        const size_t row = (size_t(sg.row_base) + size_t(pos_of(pi == 0 ? pend0 : pend1) % int64_t(sg.cap))) * kD;
         reinterpret_cast<uint2 *>(reinterpret_cast<bf16 *>(p.ws + size_t(sg.ringK_off256) * 256) + row)[lane] = ktb;
         reinterpret_cast<uint2 *>(reinterpret_cast<bf16 *>(p.ws + size_t(sg.ringV_off256) * 256) + row)[lane] = vtb;
       }
@@ -1065,7 +1061,7 @@ size_t stream_smem_bytes(int max_segs, int pool_slots) {
   using L = Layout<G, SUM>;
   return 1024 + size_t(kWarps) * STAGES * kStageBytes + size_t(kWarps) * L::kHdrBytes + size_t(kWarps) * STAGES * 64 +
          size_t(max_segs) * sizeof(StreamSegment) + size_t(kWarps) * (STAGES + 1) * 8 + size_t(kStreamMaxGroups) * 4 +
-         size_t(pool_slots) * L::kRecFloats * 4;
+         size_t(pool_slots) * L::kRecFloats * 4 + size_t(max_segs) * 8;
 }
 
 // f(group size, stages, sum-of-terms merge)
@@ -1250,8 +1246,6 @@ void build_stream_schedule(const glide_ctx *ctx, int layer_begin, int layer_coun
         sg.ringK_off256 = int32_t(ld.ringK / 256);
         sg.ringV_off256 = int32_t(ld.ringV / 256);
         sg.g = int32_t(ub % Hkv);
-        sg.b = int32_t(ub / Hkv);
-        sg.t = 0;
         {
           const int64_t b = ub / Hkv;
           const int64_t row = (int64_t(pc.layer - layer_begin) * B + b) * ctx->cfg.n_q_heads;
@@ -1370,10 +1364,12 @@ int stream_decode_setup(glide_ctx *ctx) {
       if (attempt > 0 || without_pool > size_t(dev_max)) return GLIDE_ERR_UNSUPPORTED;   // the table alone does not fit
       pool_slots = int((size_t(dev_max) - without_pool) / size_t(rec_bytes));
     }
-    auto kern = glide_decode_stream_kernel<G, S, SUM>;
     // the attribute belongs to the kernel, not to the context: ask for the device maximum so that contexts with
     // different schedules (different table sizes) can be alive together
-    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, dev_max) != cudaSuccess) {
+    if (cudaFuncSetAttribute(glide_decode_stream_kernel<G, S, SUM, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             dev_max) != cudaSuccess ||
+        cudaFuncSetAttribute(glide_decode_stream_kernel<G, S, SUM, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             dev_max) != cudaSuccess) {
       cudaGetLastError();
       return GLIDE_ERR_CUDA;
     }
@@ -1399,6 +1395,7 @@ int launch_decode_stream(glide_ctx *ctx, const DecodeParams &p, int schedule, cu
   sp.max_segs = ctx->stream_max_segs;
   sp.heads_contiguous = ctx->stream_heads_contiguous ? 1 : 0;
   sp.kv4d = ctx->tmaps_kv4d ? 1 : 0;
+  sp.t_off = int32_t(ctx->stream_smem - 1024 - size_t(ctx->stream_max_segs) * 8);
   return dispatch_stream(ctx->G, ctx->cfg.merge != GLIDE_MERGE_SHARED, [&](auto gg, auto ss, auto mm) -> int {
     constexpr int G = decltype(gg)::value, S = decltype(ss)::value;
     constexpr bool SUM = decltype(mm)::value != 0;
@@ -1416,7 +1413,9 @@ int launch_decode_stream(glide_ctx *ctx, const DecodeParams &p, int schedule, cu
 #else
     cfg.numAttrs = 1;
 #endif
-    if (cudaLaunchKernelEx(&cfg, glide_decode_stream_kernel<G, S, SUM>, p, sp) != cudaSuccess) {
+    const cudaError_t err = p.seq_off ? cudaLaunchKernelEx(&cfg, glide_decode_stream_kernel<G, S, SUM, true>, p, sp)
+                                      : cudaLaunchKernelEx(&cfg, glide_decode_stream_kernel<G, S, SUM, false>, p, sp);
+    if (err != cudaSuccess) {
       cudaGetLastError();
       return GLIDE_ERR_CUDA;
     }

@@ -134,8 +134,6 @@ int glide::plan_context(const glide_config *cfg, glide_ctx *ctx, std::vector<Wor
   off = align_up(off + sizeof(Control), 256);
   ctx->off_ndev = off;
   off = align_up(off + sizeof(int64_t) * L, 256);
-  ctx->off_seqoff = off;   // per-sequence position offsets (zeroed with the counters)
-  off = align_up(off + sizeof(int64_t) * size_t(cfg->batch), 256);
   ctx->off_layers = off;
   off = align_up(off + sizeof(LayerDev) * L, 256);
   ctx->off_heads = off;
@@ -162,6 +160,8 @@ int glide::plan_context(const glide_config *cfg, glide_ctx *ctx, std::vector<Wor
   ctx->off_zcum = off;   // running sums of phi(K') over the chunk: only the sum-of-terms merges use them
   if (cfg->merge != GLIDE_MERGE_SHARED)
     off = align_up(off + sizeof(float) * size_t(L) * units_per_layer * ctx->prefill_chunk * d, 256);
+  ctx->off_seqoff = off;   // per-sequence position offsets
+  off = align_up(off + sizeof(int64_t) * size_t(cfg->batch), 256);
   // the streamed arrays start on a 2 MiB boundary of the workspace whatever the sizes of the small tables before
   // them (measured on the B = 1 decode step: 31.5 us against 32.1 us with 64 KiB or 256 B alignment)
   off = align_up(off, size_t(GLIDE_STATE_ALIGN));
@@ -316,6 +316,7 @@ int glide_create(const glide_config *cfg, void *dev_workspace, size_t workspace_
     }
     // control words, counters, tickets, S and z start at zero
     ok = ok && cudaMemsetAsync(ctx->ws, 0, ctx->off_layers, st) == cudaSuccess &&
+         cudaMemsetAsync(ctx->ws + ctx->off_seqoff, 0, sizeof(int64_t) * size_t(ctx->cfg.batch), st) == cudaSuccess &&
          cudaMemsetAsync(ctx->ws + ctx->off_tickets, 0, ctx->off_partials - ctx->off_tickets, st) == cudaSuccess &&
          cudaMemsetAsync(ctx->ws + ctx->off_state, 0, ctx->state_bytes, st) == cudaSuccess;
     ok = ok && cudaMemcpyAsync(ctx->ws + ctx->off_layers, ctx->layers.data(), sizeof(LayerDev) * ctx->layers.size(),
@@ -533,6 +534,7 @@ int glide_reset(glide_ctx *ctx, void *stream) {
   if (!ctx) return GLIDE_ERR_INVALID_ARG;
   cudaStream_t st = as_stream(stream);
   bool ok = cudaMemsetAsync(ctx->ws, 0, ctx->off_layers, st) == cudaSuccess &&
+            cudaMemsetAsync(ctx->ws + ctx->off_seqoff, 0, sizeof(int64_t) * size_t(ctx->cfg.batch), st) == cudaSuccess &&
             cudaMemsetAsync(ctx->ws + ctx->off_tickets, 0, ctx->off_partials - ctx->off_tickets, st) == cudaSuccess &&
             cudaMemsetAsync(ctx->ws + ctx->off_state, 0, ctx->state_bytes, st) == cudaSuccess;
   if (!ok) {

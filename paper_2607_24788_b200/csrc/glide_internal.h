@@ -110,12 +110,8 @@ struct StreamSegment {
   int32_t grp_slot0;         // first shared-memory record slot of the group
   int32_t grp_idx;           // this segment's slot within the group
   int32_t grp_ctr;           // the group's arrival counter in shared memory
-  int32_t b;                 // sequence of the unit
-  int32_t pad_;
-  int64_t t;                 // position of the unit's sequence at this step: written into the CTA's shared copy by the kernel
 };
-static_assert(sizeof(StreamSegment) == 112, "StreamSegment is copied as 16-byte chunks");
-static_assert(offsetof(StreamSegment, b) == 96 && offsetof(StreamSegment, t) == 104, "the last chunk is {b, pad, t}");
+static_assert(sizeof(StreamSegment) == 96, "StreamSegment is copied as 16-byte chunks");
 
 struct StreamParams {
   const StreamSegment *segs;
@@ -124,6 +120,7 @@ struct StreamParams {
   int32_t max_segs;
   int32_t heads_contiguous;
   int32_t kv4d;                    // the 4-D K+V map exists: one TMA per window tile
+  int32_t t_off;                   // byte offset in the CTA's shared memory of the per-segment positions (int64 each)
 };
 
 struct PrefillParams {
