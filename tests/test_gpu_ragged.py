@@ -192,3 +192,36 @@ def test_joint_prefill_needs_level_slots_and_capacity_follows_the_longest_slot()
     r.g.glide_reset()
     assert [r.g.glide_seq_tokens(b) for b in range(B)] == [0, 0]
     r.g.glide_destroy()
+
+
+@pytest.mark.parametrize("seed", range(8))
+def test_ragged_random_schedules(seed):
+    """Seeded random configurations and random sequences of per-slot prefills, joint decode steps and resets."""
+    rng = np.random.default_rng(1000 + seed)
+    bf16 = bool(rng.integers(0, 2))
+    dtype, d = (torch.bfloat16, 128) if bf16 else (torch.float32, int(rng.choice([64, 128])))
+    Hkv = int(rng.choice([1, 2, 4]))
+    H = Hkv * int(rng.choice([1, 2, 4]))
+    B = int(rng.integers(1, 6))
+    L = int(rng.integers(1, 5))
+    windows = [int(rng.choice([0, 1, 7, 16, 33, 64, 150, 400])) for _ in range(L)]
+    merge = int(rng.integers(0, 3))
+    kw = dict(merge=merge, prefill_chunk=int(rng.choice([16, 64, 256])))
+    if bf16 and rng.integers(0, 3) == 0:
+        kw.update(decode_impl=glide.GLIDE_DECODE_FMA, prefill_impl=glide.GLIDE_PREFILL_FMA)
+    max_tokens = 700
+    r = Ragged(windows, B, H, Hkv, d, dtype, max_tokens, seed=seed, amp=0.5 if merge else 1.0, **kw)
+    for _ in range(int(rng.integers(6, 12))):
+        op = int(rng.integers(0, 4))
+        b = int(rng.integers(0, B))
+        if op == 0:
+            T = int(rng.choice([1, 3, 17, 64, 130, 260]))
+            if r.pos[b] + T <= max_tokens - 40:
+                r.prefill_seq(b, T, outputs=bool(rng.integers(0, 4)))
+        elif op == 1:
+            r.new_sequence(b)
+        else:
+            r.decode(int(rng.integers(1, 4)), by_layer=bool(rng.integers(0, 4) == 0))
+    r.decode(2)
+    r.check_state(f"seed {seed}")
+    r.g.glide_destroy()
