@@ -679,7 +679,7 @@ int build_ring_tensor_maps(glide_ctx *ctx) {
   }
   EncodeFn encode = reinterpret_cast<EncodeFn>(fn);
   const int L = ctx->cfg.n_layers, D = ctx->cfg.head_dim;
-  ctx->tmaps_host.assign(size_t(L) * 3 * sizeof(CUtensorMap), 0);
+  ctx->tmaps_host.assign(size_t(L) * 5 * sizeof(CUtensorMap), 0);
   ctx->tmaps_kv4d = D == 128;
   CUtensorMap *maps = reinterpret_cast<CUtensorMap *>(ctx->tmaps_host.data());
   for (int l = 0; l < L; ++l) {
@@ -696,6 +696,15 @@ int build_ring_tensor_maps(glide_ctx *ctx) {
                           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
       if (r != CUDA_SUCCESS) return GLIDE_ERR_CUDA;
+      // the same ring with boxes of a whole 128-key tile (prefill: tiles that neither wrap nor cross into the call);
+      // these maps follow the 3 L maps of the decode kernels
+      if (D == 128 && ld.cap >= 128) {
+        const cuuint32_t box128[2] = {64, 128};
+        r = encode(&maps[3 * L + 2 * l + kv], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, gptr, dims, strides, box128, estr,
+                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+        if (r != CUDA_SUCCESS) return GLIDE_ERR_CUDA;
+      }
     }
     if (D == 128 && ctx->tmaps_kv4d) {
       // K and V rings of the layer as one 4-D tensor [kv][half][row][64]: a single TMA then fills a whole

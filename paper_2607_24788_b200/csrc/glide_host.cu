@@ -154,7 +154,7 @@ int glide::plan_context(const glide_config *cfg, glide_ctx *ctx, std::vector<Wor
   ctx->off_stream_cta = off;
   off = align_up(off + sizeof(int32_t) * (size_t(kMaxStreamCtas) * kStreamWarps + 1), 256);
   ctx->off_tmaps = off;
-  off = align_up(off + size_t(128) * 3 * L, 256);
+  off = align_up(off + size_t(128) * 5 * L, 256);   // per layer 3 maps of 16-row boxes, then (from 3 L on) 2 of 128-row boxes
   ctx->off_phik = off;
   off = align_up(off + sizeof(float) * size_t(L) * units_per_layer * ctx->prefill_chunk * d, 256);
   ctx->off_zcum = off;   // running sums of phi(K') over the chunk: only the sum-of-terms merges use them

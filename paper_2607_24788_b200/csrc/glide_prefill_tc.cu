@@ -22,6 +22,7 @@
 // Every mbarrier wait is bounded; on a time-out the CTA records kDevWaitTimeout, leaves its loops, frees its TMEM
 // columns and returns.
 #include <cuda.h>
+#include <cstring>
 
 #include <algorithm>
 
@@ -224,7 +225,8 @@ static_assert(sizeof(Smem) + 1024 <= 232448, "shared memory of one CTA");
 
 // the call's K (or V) rows as a 4-D tensor {d, Hkv, T, layers x sequences}: boxes of 16 tokens x 64 columns of one KV head
 struct CallMaps {
-  CUtensorMap k, v;
+  CUtensorMap k, v;         // boxes of 16 tokens
+  CUtensorMap k128, v128;   // boxes of a whole 128-key tile
 };
 
 template <int G, bool SUM>
@@ -484,6 +486,7 @@ prefill_attn_tc_kernel(const PrefillParams p, const CUtensorMap *ring_maps, cons
     // expect-tx one before the TMA boxes are issued and a plain one after the row copies.
     if (n_tiles > 0) {
       const CUtensorMap *ringK = ring_maps + 3 * layer, *ringV = ringK + 1;
+      const CUtensorMap *ringK128 = ring_maps + 3 * p.L + 2 * layer, *ringV128 = ringK128 + 1;
       const bf16 *ringKp = reinterpret_cast<const bf16 *>(p.ws + ld.ringK) + unit_rows * kD;
       const bf16 *ringVp = reinterpret_cast<const bf16 *>(p.ws + ld.ringV) + unit_rows * kD;
       const bf16 *callKp = reinterpret_cast<const bf16 *>(p.k) + (seq * p.Hkv + g) * kD;
@@ -500,6 +503,32 @@ prefill_attn_tc_kernel(const PrefillParams p, const CUtensorMap *ring_maps, cons
         const int64_t left = tq_last - j0;                       // >= 0: the tile holds at least one valid token
         const int ngroups = left >= kKT - 1 ? kKT / kGroup : int(left / kGroup) + 1;
         const uint32_t bar = smem_u32(&sm.bar_full[slot]);
+        // A full tile that lies in one source without a wrap takes two boxes of 128 rows (the layout in shared memory
+        // is that of eight 16-row boxes).  Tiles that reach past the CTA's last token keep the 16-row path, which
+        // never loads a later token's row.
+        {
+          const uint32_t slot_row0 = (j0 >> 32) == 0 ? uint32_t(j0) % cap : uint32_t(uint64_t(j0) % cap);
+          const bool all_call = j0 >= p.n0;
+          const bool all_ring = j0 + kKT <= p.n0 && slot_row0 + kKT <= cap;
+          if (ngroups == kKT / kGroup && (all_call || all_ring)) {
+            if (lane == 0) {
+              mbar_expect_tx(bar, kTileBytes);
+              const uint32_t dst = kv_addr(slot);
+              if (all_call) {
+                const CUtensorMap *m = is_v ? &cm.v128 : &cm.k128;
+                tma_load_4d(dst, m, 0, g, int(j0 - p.n0), lrel * p.B + b, bar);
+                tma_load_4d(dst + kBoxBytes, m, 64, g, int(j0 - p.n0), lrel * p.B + b, bar);
+              } else {
+                const CUtensorMap *m = is_v ? ringV128 : ringK128;
+                const int y = int(unit_rows + slot_row0);
+                tma_load_2d(dst, m, 0, y, bar);
+                tma_load_2d(dst + kBoxBytes, m, 64, y, bar);
+              }
+              mbar_arrive(bar);   // the barrier's second arrival (after the row copies on the other path)
+            }
+            continue;
+          }
+        }
         // this lane's group: where it comes from and whether one box covers it
         const int64_t j = j0 + gi * kGroup;
         const bool mine = gi < ngroups;
@@ -837,11 +866,14 @@ int launch_prefill_attn_tc(glide_ctx *ctx, const PrefillParams &p, cudaStream_t 
   {
     const cuuint64_t dims[4] = {cuuint64_t(kD), cuuint64_t(p.Hkv), cuuint64_t(p.T), cuuint64_t(p.layer_count) * cuuint64_t(p.B)};
     const cuuint64_t strides[3] = {cuuint64_t(kD) * 2, cuuint64_t(p.Hkv) * kD * 2, cuuint64_t(p.T) * p.Hkv * kD * 2};
-    const cuuint32_t box[4] = {64, 1, kGroup, 1};
+    const cuuint32_t box[4] = {64, 1, kGroup, 1}, box128[4] = {64, 1, kKT, 1};
     const cuuint32_t estr[4] = {1, 1, 1, 1};
-    for (int kv = 0; kv < 2; ++kv) {
-      CUresult r = encode(kv == 0 ? &cm.k : &cm.v, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void *>(kv == 0 ? p.k : p.v), dims,
-                          strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+    memset(&cm, 0, sizeof(cm));
+    // (a whole-tile box is used only for tiles that lie inside the call: calls shorter than a tile never need it)
+    for (int kv = 0; kv < (p.T >= kKT ? 4 : 2); ++kv) {
+      CUtensorMap *m = kv == 0 ? &cm.k : kv == 1 ? &cm.v : kv == 2 ? &cm.k128 : &cm.v128;
+      CUresult r = encode(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void *>((kv & 1) == 0 ? p.k : p.v), dims,
+                          strides, kv < 2 ? box : box128, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                           CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
       if (r != CUDA_SUCCESS) return GLIDE_ERR_UNSUPPORTED;
     }
