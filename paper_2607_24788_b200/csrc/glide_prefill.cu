@@ -21,6 +21,15 @@ namespace {
 
 constexpr int kPrefillThreads = 128;
 
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return uint32_t(__cvta_generic_to_shared(p)); }
+// 16 bytes global -> shared; a false `valid` writes zeros and reads nothing
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void *src, bool valid) {
+  const int bytes = valid ? 16 : 0;
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_group 0;" ::: "memory"); }
+
 template <typename T>
 struct RowSource {
   const T *ringK, *ringV;   // unit base: [cap][D]
@@ -50,30 +59,41 @@ __device__ __forceinline__ RowSource<T> make_source(const PrefillParams &p, cons
   return s;
 }
 
-// 1. phi of the delayed keys of this chunk: one warp per (unit, chunk token)
+// 1. phi of the delayed keys of this chunk: one warp per (unit, kTokPerWarp consecutive chunk tokens), the rows'
+// loads issued together (with one row per warp the kernel was bound by the latency of its single load)
+constexpr int kTokPerWarp = 4;
 template <typename T, int D>
 __global__ void __launch_bounds__(kPrefillThreads) prefill_phi_kernel(const PrefillParams p) {
   constexpr int E = D / 32;
   const int lane = threadIdx.x & 31;
   const int64_t wid = (int64_t(blockIdx.x) * kPrefillThreads + threadIdx.x) >> 5;
   const int64_t units = int64_t(p.layer_count) * p.B * p.Hkv;
-  if (wid >= units * p.C) return;
-  const int i = int(wid % p.C);
-  const int64_t u = wid / p.C;
+  const int groups = (p.C + kTokPerWarp - 1) / kTokPerWarp;
+  if (wid >= units * groups) return;
+  const int i0 = int(wid % groups) * kTokPerWarp;
+  const int64_t u = wid / groups;
   const int g = int(u % p.Hkv);
   const int b = int((u / p.Hkv) % p.B);
   const int lrel = int(u / (int64_t(p.Hkv) * p.B));
   const LayerDev ld = p.layers[p.layer_begin + lrel];
   if (!ld.evicts) return;
-  const int64_t j = p.n0 + p.c0 + i - ld.wlin;  // delayed token
-  if (j < 0) return;
   const RowSource<T> src = make_source<T, D>(p, ld, lrel, b, g);
-  float x[E];
-  load_elems<T, E>(src.k(j, D) + lane * E, x);
-  warp_phi<E>(x);
-  float *dst = p.phik + (size_t(u) * p.Cmax + i) * D + lane * E;
+  float x[kTokPerWarp][E];
+  bool valid[kTokPerWarp];
 #pragma unroll
-  for (int e = 0; e < E; ++e) dst[e] = x[e];
+  for (int r = 0; r < kTokPerWarp; ++r) {
+    const int64_t j = p.n0 + p.c0 + i0 + r - ld.wlin;  // delayed token
+    valid[r] = i0 + r < p.C && j >= 0;
+    if (valid[r]) load_elems<T, E>(src.k(j, D) + lane * E, x[r]);
+  }
+#pragma unroll
+  for (int r = 0; r < kTokPerWarp; ++r) {
+    if (!valid[r]) continue;   // warp-uniform
+    warp_phi<E>(x[r]);
+    float *dst = p.phik + (size_t(u) * p.Cmax + i0 + r) * D + lane * E;
+#pragma unroll
+    for (int e = 0; e < E; ++e) dst[e] = x[r][e];
+  }
 }
 
 // 2. outputs: one warp per (unit, query token), G heads at once
@@ -225,12 +245,25 @@ __global__ void __launch_bounds__(kPrefillThreads) prefill_attn_kernel(const Pre
 // for D = 128, 64+tx*4..+3: 16-byte shared-memory reads without bank conflicts).
 constexpr int kStateRows = 64;    // state rows per CTA
 constexpr int kStateTok = 32;     // tokens per shared-memory stage
+// V values of one shared-memory row chunk as fp32 (the stage holds the rows in the I/O dtype)
+__device__ __forceinline__ void stage_v4(const float *p, float (&x)[4]) {
+  const float4 v = *reinterpret_cast<const float4 *>(p);
+  x[0] = v.x, x[1] = v.y, x[2] = v.z, x[3] = v.w;
+}
+__device__ __forceinline__ void stage_v4(const __nv_bfloat16 *p, float (&x)[4]) {
+  const uint2 v = *reinterpret_cast<const uint2 *>(p);
+  x[0] = __uint_as_float(v.x << 16), x[1] = __uint_as_float(v.x & 0xffff0000u);
+  x[2] = __uint_as_float(v.y << 16), x[3] = __uint_as_float(v.y & 0xffff0000u);
+}
 template <typename T, int D>
 __global__ void __launch_bounds__(kPrefillThreads) prefill_state_kernel(const PrefillParams p) {
   static_assert(kPrefillThreads == 128, "8 x 16 thread grid");
   constexpr int CG = D / 64;                      // column groups of 4 per thread
-  __shared__ __align__(16) float sphi[kStateTok][kStateRows];
-  __shared__ __align__(16) float sv[kStateTok][D];
+  // two stages, filled by cp.async while the other one is consumed: phi columns (fp32), then V' rows (I/O dtype)
+  constexpr int kPhiBytes = kStateTok * kStateRows * 4;
+  constexpr int kVBytes = kStateTok * D * int(sizeof(T));
+  constexpr int kVChunks = D * int(sizeof(T)) / 16;   // 16-byte chunks per V row
+  __shared__ __align__(16) unsigned char stage[2][kPhiBytes + kVBytes];
   const int blocks_per_unit = D / kStateRows;
   const int64_t u = blockIdx.x / blocks_per_unit;
   const int rb = blockIdx.x % blocks_per_unit;
@@ -252,35 +285,44 @@ __global__ void __launch_bounds__(kPrefillThreads) prefill_state_kernel(const Pr
 #pragma unroll
     for (int c = 0; c < 4 * CG; ++c) acc[r][c] = 0.f;
   float zacc = 0.f;   // threads 0..63: z of row rb*64 + tid
-  for (int i0 = i_lo; i0 < p.C; i0 += kStateTok) {
+  // tokens past the chunk's end are filled with zeros (cp.async with a source size of 0)
+  auto issue = [&](int buf, int i0) {
     const int nt = min(kStateTok, p.C - i0);
-    // stage: phi columns of this row block (fp32) and the delayed tokens' V rows (converted to fp32)
+    const uint32_t sphi = smem_u32(stage[buf]), sv = sphi + kPhiBytes;
     for (int e = tid; e < kStateTok * (kStateRows / 4); e += kPrefillThreads) {
       const int i = e / (kStateRows / 4), c4 = e % (kStateRows / 4);
-      float4 f = make_float4(0.f, 0.f, 0.f, 0.f);
-      if (i < nt) f = *reinterpret_cast<const float4 *>(pk + size_t(i0 + i) * D + c4 * 4);
-      *reinterpret_cast<float4 *>(&sphi[i][c4 * 4]) = f;
+      cp_async16(sphi + uint32_t(i * kStateRows + c4 * 4) * 4u, pk + size_t(i0 + (i < nt ? i : 0)) * D + c4 * 4, i < nt);
     }
-    for (int e = tid; e < kStateTok * (D / 4); e += kPrefillThreads) {
-      const int i = e / (D / 4), c4 = e % (D / 4);
-      float x[4] = {0.f, 0.f, 0.f, 0.f};
-      if (i < nt) load_elems<T, 4>(src.v(first + i0 + i, D) + c4 * 4, x);
-      *reinterpret_cast<float4 *>(&sv[i][c4 * 4]) = make_float4(x[0], x[1], x[2], x[3]);
+    for (int e = tid; e < kStateTok * kVChunks; e += kPrefillThreads) {
+      const int i = e / kVChunks, c = e % kVChunks;
+      const unsigned char *row = reinterpret_cast<const unsigned char *>(src.v(first + i0 + (i < nt ? i : 0), D));
+      cp_async16(sv + uint32_t(i * kVChunks + c) * 16u, row + c * 16, i < nt);
+    }
+    cp_async_commit();
+  };
+  issue(0, i_lo);
+  int buf = 0;
+  for (int i0 = i_lo; i0 < p.C; i0 += kStateTok, buf ^= 1) {
+    if (i0 + kStateTok < p.C) {
+      issue(buf ^ 1, i0 + kStateTok);
+      asm volatile("cp.async.wait_group 1;" ::: "memory");
+    } else {
+      cp_async_wait_all();
     }
     __syncthreads();
+    const float *sphi = reinterpret_cast<const float *>(stage[buf]);
+    const T *sv = reinterpret_cast<const T *>(stage[buf] + kPhiBytes);
 #pragma unroll 4
     for (int i = 0; i < kStateTok; ++i) {
-      const float4 fa = *reinterpret_cast<const float4 *>(&sphi[i][ty * 4]);
-      const float4 fb = *reinterpret_cast<const float4 *>(&sphi[i][32 + ty * 4]);
+      const float4 fa = *reinterpret_cast<const float4 *>(sphi + i * kStateRows + ty * 4);
+      const float4 fb = *reinterpret_cast<const float4 *>(sphi + i * kStateRows + 32 + ty * 4);
       const float fr[8] = {fa.x, fa.y, fa.z, fa.w, fb.x, fb.y, fb.z, fb.w};
       float vc[4 * CG];
 #pragma unroll
       for (int cg = 0; cg < CG; ++cg) {
-        const float4 vv = *reinterpret_cast<const float4 *>(&sv[i][cg * 64 + tx * 4]);
-        vc[cg * 4 + 0] = vv.x;
-        vc[cg * 4 + 1] = vv.y;
-        vc[cg * 4 + 2] = vv.z;
-        vc[cg * 4 + 3] = vv.w;
+        float x[4];
+        stage_v4(sv + i * D + cg * 64 + tx * 4, x);
+        vc[cg * 4 + 0] = x[0], vc[cg * 4 + 1] = x[1], vc[cg * 4 + 2] = x[2], vc[cg * 4 + 3] = x[3];
       }
 #pragma unroll
       for (int r = 0; r < 8; ++r)
@@ -289,9 +331,9 @@ __global__ void __launch_bounds__(kPrefillThreads) prefill_state_kernel(const Pr
     }
     if (tid < kStateRows) {
 #pragma unroll 8
-      for (int i = 0; i < kStateTok; ++i) zacc += sphi[i][tid];
+      for (int i = 0; i < kStateTok; ++i) zacc += sphi[i * kStateRows + tid];
     }
-    __syncthreads();
+    __syncthreads();   // the stage is refilled by the next iteration's issue
   }
   float *Sb = reinterpret_cast<float *>(p.ws + ld.S) + size_t(ub) * D * D + size_t(rb) * kStateRows * D;
 #pragma unroll
@@ -338,32 +380,51 @@ __global__ void __launch_bounds__(kPrefillThreads) prefill_zcum_kernel(const Pre
   }
 }
 
-// 4. ring fill: the chunk's newest min(C, cap) tokens
+// 4. ring fill: the chunk's newest min(C, cap) tokens; one warp per (unit, kTokPerWarp consecutive chunk tokens)
 template <typename T, int D>
 __global__ void __launch_bounds__(kPrefillThreads) prefill_ring_kernel(const PrefillParams p) {
   constexpr int E = D / 32;
   const int lane = threadIdx.x & 31;
   const int64_t wid = (int64_t(blockIdx.x) * kPrefillThreads + threadIdx.x) >> 5;
   const int64_t units = int64_t(p.layer_count) * p.B * p.Hkv;
-  if (wid >= units * p.C) return;
-  const int i = int(wid % p.C);
-  const int64_t u = wid / p.C;
+  const int groups = (p.C + kTokPerWarp - 1) / kTokPerWarp;
+  if (wid >= units * groups) return;
+  const int i0 = int(wid % groups) * kTokPerWarp;
+  const int64_t u = wid / groups;
   const int g = int(u % p.Hkv);
   const int b = int((u / p.Hkv) % p.B);
   const int lrel = int(u / (int64_t(p.Hkv) * p.B));
   const LayerDev ld = p.layers[p.layer_begin + lrel];
-  if (ld.cap == 0 || int64_t(i) < int64_t(p.C) - ld.cap) return;  // older tokens of the chunk are overwritten anyway
-  const int64_t j = p.n0 + p.c0 + i;
-  const size_t src = (((size_t(lrel) * p.B + b) * size_t(p.T) + size_t(p.c0 + i)) * p.Hkv + g) * D + lane * E;
-  const size_t dst = ((size_t(b + p.b0) * p.Hkv + g) * size_t(ld.cap) + size_t(j % ld.cap)) * D + lane * E;
-  const T *ks = reinterpret_cast<const T *>(p.k) + src;
-  const T *vs = reinterpret_cast<const T *>(p.v) + src;
-  T *kd = reinterpret_cast<T *>(p.ws + ld.ringK) + dst;
-  T *vd = reinterpret_cast<T *>(p.ws + ld.ringV) + dst;
+  if (ld.cap == 0) return;
+  T kx[kTokPerWarp][E], vx[kTokPerWarp][E];
+  bool valid[kTokPerWarp];
 #pragma unroll
-  for (int e = 0; e < E; ++e) {
-    kd[e] = ks[e];
-    vd[e] = vs[e];
+  for (int r = 0; r < kTokPerWarp; ++r) {
+    const int i = i0 + r;
+    valid[r] = i < p.C && int64_t(i) >= int64_t(p.C) - ld.cap;   // older tokens of the chunk are overwritten anyway
+    if (valid[r]) {
+      const size_t src = (((size_t(lrel) * p.B + b) * size_t(p.T) + size_t(p.c0 + i)) * p.Hkv + g) * D + lane * E;
+      const T *ks = reinterpret_cast<const T *>(p.k) + src;
+      const T *vs = reinterpret_cast<const T *>(p.v) + src;
+#pragma unroll
+      for (int e = 0; e < E; ++e) {
+        kx[r][e] = ks[e];
+        vx[r][e] = vs[e];
+      }
+    }
+  }
+#pragma unroll
+  for (int r = 0; r < kTokPerWarp; ++r) {
+    if (!valid[r]) continue;
+    const int64_t j = p.n0 + p.c0 + i0 + r;
+    const size_t dst = ((size_t(b + p.b0) * p.Hkv + g) * size_t(ld.cap) + size_t(j % ld.cap)) * D + lane * E;
+    T *kd = reinterpret_cast<T *>(p.ws + ld.ringK) + dst;
+    T *vd = reinterpret_cast<T *>(p.ws + ld.ringV) + dst;
+#pragma unroll
+    for (int e = 0; e < E; ++e) {
+      kd[e] = kx[r][e];
+      vd[e] = vx[r][e];
+    }
   }
 }
 
@@ -415,7 +476,9 @@ int launch_prefill(glide_ctx *ctx, int layer_begin, int layer_count, int64_t T, 
       p.C = int(std::min<int64_t>(p.Cmax, T - c0));
       const int64_t warps = units * p.C;
       const unsigned warp_blocks = unsigned((warps * 32 + kPrefillThreads - 1) / kPrefillThreads);
-      if (any_evicts) prefill_phi_kernel<TT, D><<<warp_blocks, kPrefillThreads, 0, stream>>>(p);
+      const int64_t warps4 = units * ((p.C + kTokPerWarp - 1) / kTokPerWarp);
+      const unsigned warp4_blocks = unsigned((warps4 * 32 + kPrefillThreads - 1) / kPrefillThreads);
+      if (any_evicts) prefill_phi_kernel<TT, D><<<warp4_blocks, kPrefillThreads, 0, stream>>>(p);
       if (out) {
         if (use_tc) {
           if (any_evicts && p.merge != GLIDE_MERGE_SHARED)
@@ -428,7 +491,7 @@ int launch_prefill(glide_ctx *ctx, int layer_begin, int layer_count, int64_t T, 
         }
       }
       if (any_evicts) prefill_state_kernel<TT, D><<<unsigned(units * (D / kStateRows)), kPrefillThreads, 0, stream>>>(p);
-      prefill_ring_kernel<TT, D><<<warp_blocks, kPrefillThreads, 0, stream>>>(p);
+      prefill_ring_kernel<TT, D><<<warp4_blocks, kPrefillThreads, 0, stream>>>(p);
       if (cudaGetLastError() != cudaSuccess) return GLIDE_ERR_CUDA;
     }
     return GLIDE_OK;
