@@ -216,6 +216,8 @@ bool prefill_attn_tc_supported(const glide_ctx *ctx);
 int launch_prefill_attn_tc(glide_ctx *ctx, const PrefillParams &p, cudaStream_t stream);
 bool prefill_attn_mma_supported(const glide_ctx *ctx);
 int launch_prefill_attn_mma(glide_ctx *ctx, const PrefillParams &p, cudaStream_t stream);
+bool prefill_state_mma_supported(const glide_ctx *ctx);
+int launch_prefill_state_mma(glide_ctx *ctx, const PrefillParams &p, cudaStream_t stream);
 int launch_advance(glide_ctx *ctx, int layer_begin, int layer_count, int64_t T, cudaStream_t stream);
 
 }  // namespace glide

@@ -465,6 +465,9 @@ int launch_prefill(glide_ctx *ctx, int layer_begin, int layer_count, int64_t T, 
   // (the mma.sync kernel has the shared normaliser only: the other merges fall through to the CUDA-core kernel)
   const bool use_mma = (impl == GLIDE_PREFILL_MMA_SYNC || (impl == GLIDE_PREFILL_TCGEN05 && !use_tc)) &&
                        prefill_attn_mma_supported(ctx) && ctx->cfg.merge == GLIDE_MERGE_SHARED;
+  // carry of the chunk scan: tensor cores with an error-free three-way bf16 split of phi(K') (bf16, d = 128), or the
+  // CUDA-core kernel (fp32 I/O, d = 64, and whenever the CUDA-core prefill is asked for)
+  const bool state_mma = prefill_state_mma_supported(ctx) && impl != GLIDE_PREFILL_FMA;
   bool any_evicts = false;
   for (int l = layer_begin; l < layer_begin + layer_count; ++l) any_evicts = any_evicts || ctx->layers[l].evicts;
 
@@ -490,7 +493,13 @@ int launch_prefill(glide_ctx *ctx, int layer_begin, int layer_count, int64_t T, 
           prefill_attn_kernel<TT, D, G><<<warp_blocks, kPrefillThreads, 0, stream>>>(p);
         }
       }
-      if (any_evicts) prefill_state_kernel<TT, D><<<unsigned(units * (D / kStateRows)), kPrefillThreads, 0, stream>>>(p);
+      if (any_evicts) {
+        if (state_mma) {
+          if (launch_prefill_state_mma(ctx, p, stream) != GLIDE_OK) return GLIDE_ERR_CUDA;
+        } else {
+          prefill_state_kernel<TT, D><<<unsigned(units * (D / kStateRows)), kPrefillThreads, 0, stream>>>(p);
+        }
+      }
       prefill_ring_kernel<TT, D><<<warp4_blocks, kPrefillThreads, 0, stream>>>(p);
       if (cudaGetLastError() != cudaSuccess) return GLIDE_ERR_CUDA;
     }

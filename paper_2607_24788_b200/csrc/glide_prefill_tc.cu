@@ -510,7 +510,9 @@ prefill_attn_tc_kernel(const PrefillParams p, const CUtensorMap *ring_maps, cons
           const uint32_t slot_row0 = (j0 >> 32) == 0 ? uint32_t(j0) % cap : uint32_t(uint64_t(j0) % cap);
           const bool all_call = j0 >= p.n0;
           const bool all_ring = j0 + kKT <= p.n0 && slot_row0 + kKT <= cap;
-          if (ngroups == kKT / kGroup && (all_call || all_ring)) {
+          // (left >= kKT - 1: every row of the tile is a token up to the CTA's last one; eight groups alone would also
+          // admit a last group that is only partly valid)
+          if (left >= kKT - 1 && (all_call || all_ring)) {
             if (lane == 0) {
               mbar_expect_tx(bar, kTileBytes);
               const uint32_t dst = kv_addr(slot);

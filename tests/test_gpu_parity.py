@@ -302,3 +302,27 @@ def test_streaming_kernel_with_hundreds_of_units_per_cta():
     # 32 768 small units: the segment table of a CTA takes over most of the shared-memory record pool; the streaming
     # kernel (asked for explicitly) must still apply and agree with the oracle
     run_case([0, 1] * 16, 128, 8, 8, 128, BF16, [], 3, amp=128 ** -0.5 * 4, seed=3, decode_impl=3, state_checks=False)
+
+
+@pytest.mark.parametrize("impl", [2, 3])
+def test_chunk_scan_carry_stays_fp32_accurate_over_a_long_prompt(impl):
+    """16 chunks of carry: the tensor-core state kernel (prefill_impl 2: phi(K') split into three bf16 terms, exact
+    products, fp32 accumulation) and the CUDA-core one (prefill_impl 3) both stay well inside the 1e-5 state tolerance."""
+    import numpy as np
+    from oracle import glide_oracle as orc
+    from paper_2607_24788_b200 import glide, synth
+    from tests.parity_util import f32_scale, to_np
+    L, B, H, Hkv, d, T = 2, 1, 8, 2, 128, 4096
+    windows = [64, 0]
+    wl = synth.Workload(11, L, B, H, Hkv, d, BF16, 2.0)
+    g = glide.Glide(windows, B, H, Hkv, d, T + 8, dtype=BF16, softmax_scale=f32_scale(d), prefill_impl=impl)
+    stack = orc.Stack(windows, B, H, Hkv, d, f32_scale(d))
+    q, k, v = wl.qkv(range(L), range(B), range(T), device="cuda")
+    g.glide_prefill(None, k, v, None)
+    stack.prefill(to_np(q), to_np(k), to_np(v), outputs=False)
+    for l in range(L):
+        _, _, S, z = g.glide_export_state(l)
+        _, _, oS, oz = stack.cells[l][0].export()
+        assert np.linalg.norm(to_np(S[0]) - oS) / np.linalg.norm(oS) <= 3e-6
+        assert np.linalg.norm(to_np(z[0]) - oz) / np.linalg.norm(oz) <= 3e-6
+    g.glide_destroy()
