@@ -225,3 +225,46 @@ def test_ragged_random_schedules(seed):
     r.decode(2)
     r.check_state(f"seed {seed}")
     r.g.glide_destroy()
+
+
+def test_ragged_llama_shape_long_sequences_sampled_layers():
+    """Config-1 shapes (32 layers, H = 32, H_kv = 8, d = 128) with four sequences of very different lengths: heavy
+    units are cut across CTAs and merged through tickets while every sequence sits at its own position.  The oracle
+    follows one layer of every window size."""
+    from paper_2607_24788_b200 import configs as C
+    windows = list(C.C1.windows)
+    L, B, H, Hkv, d = len(windows), 4, 32, 8, 128
+    lengths = [9000, 4100, 17, 6500]
+    layers = [0, 5, 13, 31]                       # windows 4096, 1024, 256, 64
+    scale = f32_scale(d)
+    wl = synth.Workload(21, L, N_IDS, H, Hkv, d, torch.bfloat16, d ** -0.5 * 4)
+    g = glide.Glide(windows, B, H, Hkv, d, 10000, dtype=torch.bfloat16, device="cuda", softmax_scale=scale)
+    cells = {(l, b): orc.Cell(H, Hkv, d, windows[l], scale) for l in layers for b in range(B)}
+    for b, T in enumerate(lengths):
+        pos = 0
+        while pos < T:
+            n = min(4096, T - pos)
+            k, v = wl.kv(range(L), [b], range(pos, pos + n), device="cuda")
+            g.glide_prefill_seq(b, None, k[:, 0].contiguous(), v[:, 0].contiguous(), None)
+            for l in layers:
+                cells[(l, b)].prefill(None, to_np(k[l, 0]), to_np(v[l, 0]), outputs=False)
+            pos += n
+        assert g.glide_seq_tokens(b) == T
+    pos = list(lengths)
+    for step in range(3):
+        parts = [wl.qkv(range(L), [b], [pos[b]], device="cuda") for b in range(B)]
+        q, k, v = [torch.cat([p[i][:, :, 0] for p in parts], dim=1).contiguous() for i in range(3)]
+        out = torch.full_like(q, float("nan"))
+        g.glide_decode_step(q, k, v, out)
+        assert torch.isfinite(out.float()).all()
+        for l in layers:
+            for b in range(B):
+                ref = cells[(l, b)].decode(to_np(q[l, b]), to_np(k[l, b]), to_np(v[l, b]))
+                check_outputs(out[l, b], ref, torch.bfloat16, f"step {step} layer {l} slot {b} t={pos[b]}")
+        pos = [x + 1 for x in pos]
+    for l in layers:
+        for b in range(B):
+            info, oi = g.glide_seq_layer_info(l, b), cells[(l, b)].info()
+            assert (info["n"], info["count"], info["n_evicted"]) == (oi["n"], oi["count"], oi["n_evicted"])
+    assert g.glide_device_status() == 0
+    g.glide_destroy()
