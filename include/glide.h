@@ -184,10 +184,8 @@ int glide_decode_step_noalloc(glide_ctx *ctx, const void *dev_q, const void *dev
  * context, so each slot b may hold a sequence of its own length.  The position of slot b at layer l is the layer's
  * counter (moved by glide_prefill and the decode steps, which advance every slot together) plus an offset of the
  * slot, which the three calls below change.  They act on all layers and need all layers level (GLIDE_ERR_STATE
- * otherwise).  A decode step always advances every slot by one token: a slot that holds no live sequence is
- * stepped along with whatever its input rows contain (finite values keep its state finite) and is reset before it
- * is used again; the capacity check of a step is against the longest slot.  glide_prefill for all slots at once
- * needs them at one position. */
+ * otherwise).  A decode step advances every slot that is not parked by one token; the capacity check of a step is
+ * against the longest such slot.  glide_prefill for all slots at once needs them at one position and none parked. */
 
 /* Slot b starts an empty sequence: position 0, S and z zeroed (ring rows need no clearing).  Other slots are
  * untouched.  Stream-ordered. */
@@ -198,7 +196,13 @@ int glide_reset_seq(glide_ctx *ctx, int32_t b, void *stream);
 int glide_prefill_seq(glide_ctx *ctx, int32_t b, int64_t T, const void *dev_q, const void *dev_k, const void *dev_v,
                       void *dev_out, void *stream);
 
-/* Tokens slot b holds, as the host tracks them (no device access). */
+/* Slot b holds no sequence from now on: decode steps skip it (its rows of q, k, v are not read, its rows of out
+ * and its ring, S and z are not written), so an idle slot costs no memory traffic.  glide_reset_seq starts a new
+ * sequence in it; glide_prefill_seq and glide_seq_layer_info on a parked slot return GLIDE_ERR_STATE.  May be
+ * called between the layer-range calls of a step.  Stream-ordered. */
+int glide_park_seq(glide_ctx *ctx, int32_t b, void *stream);
+
+/* Tokens slot b holds, as the host tracks them (no device access); -1 for a parked slot. */
 int glide_seq_tokens(glide_ctx *ctx, int32_t b, int64_t *n_out);
 
 /* Free the host context.  Does not touch the workspace. */

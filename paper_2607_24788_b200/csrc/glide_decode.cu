@@ -336,6 +336,7 @@ __global__ void __launch_bounds__(kDecodeThreads) glide_decode_kernel(const Deco
     const int ub = it.unit - it.layer * units_per_layer;
     const int b = ub / p.Hkv, g = ub - b * p.Hkv;
     const int64_t t = p.n_dev[it.layer] + (p.seq_off ? p.seq_off[b] : 0);   // position of this sequence
+    if (t < 0) continue;   // parked slot: nothing is read or written for it (every item of the unit takes this branch)
     const int per_unit = ld.n_win_items + ld.n_state_items;
     float *rec = p.partials + ld.part_base + (size_t(ub) * per_unit + it.part) * p.rec_floats;
     if (it.kind == kItemWindow)

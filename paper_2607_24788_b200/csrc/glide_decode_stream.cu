@@ -190,13 +190,19 @@ __device__ __forceinline__ void tma_load_4d(uint32_t dst, const void *tmap, int 
       : "memory");
 }
 
+// (PARKABLE: the launch has slot offsets, so a position may be negative = a parked slot; the instantiation for level
+// batches carries none of the checks)
+template <bool PARKABLE>
 __device__ __forceinline__ bool seg_evicting(const StreamSegment &s, int64_t t) {
   // evicts bit 0: the layer has a state; bit 1: the token folded at a step is the current one (no ring, or a state
   // that holds every token), otherwise the one that leaves the window
+  if (PARKABLE && t < 0) return false;
   return (s.evicts & 1) && ((s.evicts & 2) || t >= int64_t(s.w));
 }
 // window tiles of the segment that hold window tokens at position t
+template <bool PARKABLE>
 __device__ __forceinline__ int seg_valid_win(const StreamSegment &s, int64_t t) {
+  if (PARKABLE && t < 0) return 0;
   const int64_t lim = t < int64_t(s.cap) ? t : int64_t(s.cap);
   const int nv = int((lim + kTileRows - 1) / kTileRows) - s.win0;
   return nv < 0 ? 0 : (nv > s.n_win ? s.n_win : nv);
@@ -209,11 +215,12 @@ struct Cursor {
   int n_state_eff, n_total;
 };
 
+template <bool PARKABLE>
 __device__ __forceinline__ void cursor_enter(Cursor &c, const StreamSegment *segs, int64_t t) {
   const StreamSegment &s = segs[c.seg];
   c.k = 0;
-  c.n_state_eff = seg_evicting(s, t) ? s.n_state : 0;
-  c.n_total = c.n_state_eff + seg_valid_win(s, t);
+  c.n_state_eff = seg_evicting<PARKABLE>(s, t) ? s.n_state : 0;
+  c.n_total = c.n_state_eff + seg_valid_win<PARKABLE>(s, t);
 }
 
 // Records.  Shared normaliser: (acc[G][d], m[G], l[G]) with the linear readout already folded in as a term with
@@ -353,7 +360,7 @@ glide_decode_stream_kernel(const DecodeParams p, const StreamParams sp) {
     if (lane == 0) {
       const StreamSegment &sg = sm_segs[s];
       const int64_t t = pos_of(s);
-      const bool ev = seg_evicting(sg, t);
+      const bool ev = seg_evicting<RAGGED>(sg, t);
       fence_async_smem();
       mbar_expect_tx(hdr_bar, G * 256 + 512 + (ev ? 512 : 0));
       const bf16 *qall = reinterpret_cast<const bf16 *>(p.q);
@@ -384,12 +391,12 @@ glide_decode_stream_kernel(const DecodeParams p, const StreamParams sp) {
   Cursor icur;
   icur.seg = seg_lo;
   icur.k = icur.n_state_eff = icur.n_total = 0;
-  if (seg_lo < seg_hi) cursor_enter(icur, sm_segs, pos_of(icur.seg));
+  if (seg_lo < seg_hi) cursor_enter<RAGGED>(icur, sm_segs, pos_of(icur.seg));
   int issue_stage = 0;
   auto issue_next = [&]() {
     if (lane == 0) {
       while (icur.seg < seg_hi && icur.k >= icur.n_total) {
-        if (++icur.seg < seg_hi) cursor_enter(icur, sm_segs, pos_of(icur.seg));
+        if (++icur.seg < seg_hi) cursor_enter<RAGGED>(icur, sm_segs, pos_of(icur.seg));
       }
       if (icur.seg < seg_hi) {
         const StreamSegment &sg = sm_segs[icur.seg];
@@ -587,9 +594,9 @@ glide_decode_stream_kernel(const DecodeParams p, const StreamParams sp) {
   for (int s = seg_lo; s < seg_hi && !failed; ++s) {
     const StreamSegment &sg = sm_segs[s];
     const int64_t t = pos_of(s);
-    const bool ev = seg_evicting(sg, t);
+    const bool ev = seg_evicting<RAGGED>(sg, t);
     const int n_state_eff = ev ? sg.n_state : 0;
-    const int n_total = n_state_eff + seg_valid_win(sg, t);
+    const int n_total = n_state_eff + seg_valid_win<RAGGED>(sg, t);
     const bool has_win = sg.cap > 0;
 
     // -- header: q fragments, current token, feature maps -> registers; then prefetch the next header --
@@ -633,6 +640,10 @@ glide_decode_stream_kernel(const DecodeParams p, const StreamParams sp) {
     __syncwarp();
     GLIDE_TRACE_EVENT(16);
     if (s + 1 < seg_hi) issue_header(s + 1);
+    // A parked slot (negative position; only batches with slot offsets have them) goes through the header hand-over
+    // like every segment and then leaves: it has no tiles, and nothing of it is reduced or written.  All segments
+    // of a unit share the position, so its group counters and tickets stay untouched as well.
+    if (RAGGED && t < 0) continue;
     if (has_win) {
       const int64_t lim = t < int64_t(sg.cap) ? t : int64_t(sg.cap);
       win_end = int(lim);

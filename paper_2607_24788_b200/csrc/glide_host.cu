@@ -95,6 +95,7 @@ int glide::plan_context(const glide_config *cfg, glide_ctx *ctx, std::vector<Wor
   ctx->cfg.q_to_kv = nullptr;
   ctx->n_host.assign(L, 0);
   ctx->seq_off.assign(size_t(cfg->batch), 0);
+  ctx->parked.assign(size_t(cfg->batch), 0);
   ctx->rec_floats = int(align_up(size_t(ctx->G) * (d + 2), 4));
   ctx->stream_rec_floats = ctx->rec_floats * (cfg->merge == GLIDE_MERGE_SHARED ? 1 : 2);
 
@@ -344,9 +345,11 @@ int glide_destroy(glide_ctx *ctx) {
 }
 
 namespace {
+// largest offset among the slots that hold a sequence (the parked ones are never stepped)
 int64_t max_seq_off(const glide_ctx *ctx) {
-  int64_t m = ctx->seq_off.empty() ? 0 : ctx->seq_off[0];
-  for (int64_t o : ctx->seq_off) m = std::max(m, o);
+  int64_t m = kParkedOffset;
+  for (size_t b = 0; b < ctx->seq_off.size(); ++b)
+    if (!ctx->parked[b]) m = std::max(m, ctx->seq_off[b]);
   return m;
 }
 bool layers_level(const glide_ctx *ctx) {
@@ -411,8 +414,8 @@ int glide_prefill(glide_ctx *ctx, int32_t layer_begin, int32_t layer_count, int6
   for (int l = layer_begin + 1; l < layer_begin + layer_count; ++l)
     if (ctx->n_host[l] != ctx->n_host[layer_begin]) return GLIDE_ERR_STATE;
   // one call for all sequences needs them at one position
-  for (int64_t o : ctx->seq_off)
-    if (o != ctx->seq_off[0]) return GLIDE_ERR_STATE;
+  for (size_t b = 0; b < ctx->seq_off.size(); ++b)
+    if (ctx->seq_off[b] != ctx->seq_off[0] || ctx->parked[b]) return GLIDE_ERR_STATE;
   if (ctx->n_host[layer_begin] + ctx->seq_off[0] + T > ctx->cfg.max_tokens) return GLIDE_ERR_CAPACITY;
   if (T == 0) return GLIDE_OK;
   int rc = launch_prefill(ctx, layer_begin, layer_count, T, q, k, v, out, -1, ctx->n_host[layer_begin] + ctx->seq_off[0],
@@ -428,6 +431,7 @@ int glide_prefill_seq(glide_ctx *ctx, int32_t b, int64_t T, const void *q, const
   if (out && !q) return GLIDE_ERR_INVALID_ARG;
   if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out)) return GLIDE_ERR_INVALID_ARG;
   if (!layers_level(ctx)) return GLIDE_ERR_STATE;
+  if (ctx->parked[size_t(b)]) return GLIDE_ERR_STATE;   // a parked slot starts again with glide_reset_seq
   const int64_t n0 = ctx->n_host[0] + ctx->seq_off[size_t(b)];
   if (n0 + T > ctx->cfg.max_tokens) return GLIDE_ERR_CAPACITY;
   if (T == 0) return GLIDE_OK;
@@ -451,18 +455,30 @@ int glide_reset_seq(glide_ctx *ctx, int32_t b, void *stream) {
     cudaGetLastError();
     return GLIDE_ERR_CUDA;
   }
+  ctx->parked[size_t(b)] = 0;
   return set_seq_off(ctx, b, -ctx->n_host[0], st);
+}
+
+int glide_park_seq(glide_ctx *ctx, int32_t b, void *stream) {
+  if (!ctx || b < 0 || b >= ctx->cfg.batch) return GLIDE_ERR_INVALID_ARG;
+  ctx->parked[size_t(b)] = 1;
+  return set_seq_off(ctx, b, kParkedOffset, as_stream(stream));
 }
 
 int glide_seq_tokens(glide_ctx *ctx, int32_t b, int64_t *n_out) {
   if (!ctx || !n_out || b < 0 || b >= ctx->cfg.batch) return GLIDE_ERR_INVALID_ARG;
   if (!layers_level(ctx)) return GLIDE_ERR_STATE;
+  if (ctx->parked[size_t(b)]) {
+    *n_out = -1;
+    return GLIDE_OK;
+  }
   *n_out = ctx->n_host[0] + ctx->seq_off[size_t(b)];
   return GLIDE_OK;
 }
 
 int glide_seq_layer_info(glide_ctx *ctx, int32_t layer, int32_t b, void *stream, glide_layer_info_t *out) {
   if (!ctx || !out || layer < 0 || layer >= ctx->cfg.n_layers || b < 0 || b >= ctx->cfg.batch) return GLIDE_ERR_INVALID_ARG;
+  if (ctx->parked[size_t(b)]) return GLIDE_ERR_STATE;   // a parked slot has no position
   int64_t n = 0, off = 0;
   cudaStream_t st = as_stream(stream);
   if (cudaMemcpyAsync(&n, ctx->ws + ctx->off_ndev + sizeof(int64_t) * layer, sizeof(int64_t), cudaMemcpyDeviceToHost,
@@ -543,6 +559,7 @@ int glide_reset(glide_ctx *ctx, void *stream) {
   }
   std::fill(ctx->n_host.begin(), ctx->n_host.end(), 0);
   std::fill(ctx->seq_off.begin(), ctx->seq_off.end(), 0);
+  std::fill(ctx->parked.begin(), ctx->parked.end(), 0);
   ctx->ragged = false;
   return GLIDE_OK;
 }

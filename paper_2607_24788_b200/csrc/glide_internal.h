@@ -13,6 +13,7 @@ namespace glide {
 
 constexpr int kDecodeThreads = 128;   // 4 warps per CTA
 constexpr int kMaxGroup = 8;          // query heads per KV head
+constexpr int64_t kParkedOffset = -(int64_t(1) << 61);   // slot offset of a parked slot: position < 0 at any counter
 
 // Per-layer constants, resident in the workspace (device) and mirrored on the host.
 struct LayerDev {
@@ -155,6 +156,7 @@ struct glide_ctx {
   std::vector<int64_t> n_host;      // mirror of the device counters
   std::vector<int64_t> seq_off;     // [B] mirror of the per-sequence offsets: sequence b of layer l is at n_host[l] + seq_off[b]
   bool ragged = false;              // some offset is not zero
+  std::vector<char> parked;         // [B] slot holds no sequence: its offset makes every position negative
   std::vector<unsigned char> tmaps_host;  // TMA descriptors of the rings (bf16 tensor-core decode kernel)
   int decode_kind = 0;              // 0 CUDA-core kernel, 1 per-item tensor-core kernel, 2 streaming tensor-core kernel
   // schedules of the streaming kernel: [0] all layers; [1 + l] layer l alone (built when L > 1)

@@ -74,6 +74,7 @@ def load_library() -> ctypes.CDLL:
     lib.glide_decode_step_noalloc.argtypes = [vp, vp, vp, vp, vp, vp]
     lib.glide_decode_step_layers.argtypes = [vp, i32, i32, vp, vp, vp, vp, vp]
     lib.glide_reset_seq.argtypes = [vp, i32, vp]
+    lib.glide_park_seq.argtypes = [vp, i32, vp]
     lib.glide_prefill_seq.argtypes = [vp, i32, i64, vp, vp, vp, vp, vp]
     lib.glide_seq_tokens.argtypes = [vp, i32, ctypes.POINTER(i64)]
     lib.glide_seq_layer_info.argtypes = [vp, i32, i32, vp, ctypes.POINTER(glide_layer_info_t)]
@@ -211,6 +212,10 @@ class Glide:
     def glide_reset_seq(self, b: int, stream=None) -> None:
         """Slot b starts an empty sequence; the other slots are untouched."""
         _check(self.lib.glide_reset_seq(self._h, int(b), _stream(stream)), "glide_reset_seq")
+
+    def glide_park_seq(self, b: int, stream=None) -> None:
+        """Slot b holds no sequence: decode steps skip it until glide_reset_seq starts a new one there."""
+        _check(self.lib.glide_park_seq(self._h, int(b), _stream(stream)), "glide_park_seq")
 
     def glide_prefill_seq(self, b: int, q: Optional[torch.Tensor], k: torch.Tensor, v: torch.Tensor,
                           out: Optional[torch.Tensor] = None, stream=None) -> None:

@@ -29,6 +29,7 @@ class Ragged:
                              **cfg_kw)
         self.next_id = 0
         self.ids, self.pos, self.cells = [0] * B, [0] * B, [None] * B
+        self.parked = set()
         for b in range(B):
             self.new_sequence(b, reset=False)
         self.worst = 0.0
@@ -37,8 +38,13 @@ class Ragged:
         self.ids[b], self.pos[b] = self.next_id, 0
         self.next_id += 1
         self.cells[b] = [orc.Cell(self.H, self.Hkv, self.d, w, self.scale, merge=self.merge) for w in self.windows]
+        self.parked.discard(b)
         if reset:
             self.g.glide_reset_seq(b)
+
+    def park(self, b):
+        self.parked.add(b)
+        self.g.glide_park_seq(b)
 
     def prefill_seq(self, b, T, outputs=True):
         q, k, v = self.wl.qkv(range(self.L), [self.ids[b]], range(self.pos[b], self.pos[b] + T), device="cuda")
@@ -66,6 +72,9 @@ class Ragged:
             else:
                 self.g.glide_decode_step(q, k, v, out)
             for b in range(self.B):
+                if b in self.parked:
+                    assert torch.isnan(out[:, b].float()).all(), "a parked slot's output rows were written"
+                    continue
                 ref = np.stack([self.cells[b][l].decode(to_np(q[l, b]), to_np(k[l, b]), to_np(v[l, b])) for l in range(self.L)])
                 self.worst = max(self.worst, check_outputs(out[:, b], ref, self.dtype, f"decode slot {b} t={self.pos[b]}"))
                 self.pos[b] += 1
@@ -75,6 +84,8 @@ class Ragged:
         for l in range(self.L):
             rk, rv, S, z = g.glide_export_state(l)
             for b in range(self.B):
+                if b in self.parked:
+                    continue
                 cell = self.cells[b][l]
                 info, oi = g.glide_seq_layer_info(l, b), cell.info()
                 assert (info["n"], info["count"], info["n_evicted"]) == (oi["n"], oi["count"], oi["n_evicted"]), (what, l, b, info, oi)
@@ -196,7 +207,8 @@ def test_joint_prefill_needs_level_slots_and_capacity_follows_the_longest_slot()
 
 @pytest.mark.parametrize("seed", range(8))
 def test_ragged_random_schedules(seed):
-    """Seeded random configurations and random sequences of per-slot prefills, joint decode steps and resets."""
+    """Seeded random configurations and random sequences of per-slot prefills, joint decode steps, resets and
+    parked slots."""
     rng = np.random.default_rng(1000 + seed)
     bf16 = bool(rng.integers(0, 2))
     dtype, d = (torch.bfloat16, 128) if bf16 else (torch.float32, int(rng.choice([64, 128])))
@@ -212,9 +224,13 @@ def test_ragged_random_schedules(seed):
     max_tokens = 700
     r = Ragged(windows, B, H, Hkv, d, dtype, max_tokens, seed=seed, amp=0.5 if merge else 1.0, **kw)
     for _ in range(int(rng.integers(6, 12))):
-        op = int(rng.integers(0, 4))
+        op = int(rng.integers(0, 5))
         b = int(rng.integers(0, B))
-        if op == 0:
+        if op == 4:
+            r.park(b)
+        elif op == 0:
+            if b in r.parked:
+                r.new_sequence(b)
             T = int(rng.choice([1, 3, 17, 64, 130, 260]))
             if r.pos[b] + T <= max_tokens - 40:
                 r.prefill_seq(b, T, outputs=bool(rng.integers(0, 4)))
@@ -268,3 +284,82 @@ def test_ragged_llama_shape_long_sequences_sampled_layers():
             assert (info["n"], info["count"], info["n_evicted"]) == (oi["n"], oi["count"], oi["n_evicted"])
     assert g.glide_device_status() == 0
     g.glide_destroy()
+
+
+def _snapshot(g, b):
+    """ring, S, z of slot b for every layer (device copies)"""
+    snap = []
+    for l in range(g.L):
+        rk, rv, S, z = g.glide_export_state(l)
+        snap.append(tuple(x[b].clone() for x in (rk, rv, S, z)))
+    return snap
+
+
+@pytest.mark.parametrize("kind", ["f32", "bf16_stream", "bf16_stream_by_layer", "bf16_mma", "bf16_sum"])
+def test_parked_slot_is_skipped(kind):
+    """A parked slot is not stepped: its outputs stay as the caller left them, its ring, S, z do not change (bit for
+    bit), whatever its input rows hold (NaN here); the other slots are unaffected; a reset starts a new sequence."""
+    kw, by_layer = {}, False
+    if kind == "f32":
+        dtype, d, H, Hkv = torch.float32, 64, 4, 2
+    else:
+        dtype, d, H, Hkv = torch.bfloat16, 128, 8, 2
+        if kind == "bf16_mma":
+            kw = dict(decode_impl=glide.GLIDE_DECODE_MMA)
+        if kind == "bf16_sum":
+            kw = dict(merge=1)
+        by_layer = kind == "bf16_stream_by_layer"
+    r = Ragged([48, 0, 300, 16], 3, H, Hkv, d, dtype, 600, seed=12, amp=0.5 if kw.get("merge") else 1.0, **kw)
+    for b, T in enumerate([200, 350, 31]):
+        r.prefill_seq(b, T)
+    r.decode(2, by_layer=by_layer)
+    victim = 1
+    r.g.glide_park_seq(victim)
+    assert r.g.glide_seq_tokens(victim) == -1
+    before = _snapshot(r.g, victim)
+    live = [b for b in range(r.B) if b != victim]
+    for _ in range(4):
+        q, k, v = r._step_inputs()
+        q[:, victim], k[:, victim], v[:, victim] = float("nan"), float("nan"), float("nan")
+        out = torch.full_like(q, 7.0)
+        if by_layer:
+            for l in range(r.L):
+                r.g.glide_decode_step_layers(q[l:l + 1], k[l:l + 1], v[l:l + 1], out[l:l + 1], l, 1)
+        else:
+            r.g.glide_decode_step(q, k, v, out)
+        assert (out[:, victim] == 7.0).all()
+        for b in live:
+            ref = np.stack([r.cells[b][l].decode(to_np(q[l, b]), to_np(k[l, b]), to_np(v[l, b])) for l in range(r.L)])
+            check_outputs(out[:, b], ref, r.dtype, f"slot {b} beside a parked slot")
+            r.pos[b] += 1
+    after = _snapshot(r.g, victim)
+    for l in range(r.L):
+        for x, y in zip(before[l], after[l]):
+            assert torch.equal(x, y)
+    with pytest.raises(glide.GlideError) as e:
+        r.prefill_seq(victim, 4)
+    assert e.value.code == glide.GLIDE_ERR_STATE
+    r.new_sequence(victim)          # glide_reset_seq: the slot is live again, at position 0
+    r.prefill_seq(victim, 70)
+    r.decode(3, by_layer=by_layer)
+    r.check_state("after the parked slot was reused")
+    r.g.glide_destroy()
+
+
+def test_parked_slots_do_not_count_for_capacity_and_all_parked_is_a_no_op():
+    r = Ragged([16, 0], 2, 4, 2, 64, torch.float32, 40, seed=13)
+    r.prefill_seq(0, 39)
+    r.g.glide_park_seq(0)
+    for _ in range(5):             # slot 0 would be past max_tokens by now
+        q, k, v = r._step_inputs()
+        out = torch.full_like(q, 3.0)
+        r.g.glide_decode_step(q, k, v, out)
+        ref = np.stack([r.cells[1][l].decode(to_np(q[l, 1]), to_np(k[l, 1]), to_np(v[l, 1])) for l in range(r.L)])
+        check_outputs(out[:, 1], ref, r.dtype, "live slot")
+        r.pos[1] += 1
+    r.g.glide_park_seq(1)
+    q, k, v = r._step_inputs()
+    out = torch.full_like(q, 3.0)
+    r.g.glide_decode_step_noalloc(q, k, v, out)
+    assert (out == 3.0).all() and r.g.glide_device_status() == 0
+    r.g.glide_destroy()
