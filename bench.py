@@ -9,10 +9,14 @@ and the shared-normaliser merge.  The state the steps start from is built (untim
 glide_prefill over the synthetic prompt.  Default workload: Llama-3-8B-shaped stack, batch 1,
 32K context (configs.C1).  Prints ONE JSON line.
 
-Timing: CUDA events on the launching stream around exactly K steps, repeated a few times while
-NVML samples the clocks; the median repetition is reported.  Consecutive steps rotate over
-several independent copies of the sequence state (total footprint well above the 126 MB L2), so
-no step finds its window or state in L2 from the step before.
+Timing: CUDA events on the launching stream around exactly K steps, repeated until at least half a
+second of timed work has accumulated while NVML samples the clocks; the median repetition is
+reported.  Consecutive steps rotate over several independent copies of the sequence state (total
+footprint well above the 126 MB L2), so no step finds its window or state in L2 from the step
+before.  `value` is the back-to-back throughput (the launches of consecutive steps overlap by
+programmatic dependent launch); `per_step_attention_latency_us` is the median of steps timed one
+by one between their own events.  After the headline workload the other configurations and the two
+controls (uniform window, full-KV softmax) are timed the same way and reported under `workloads`.
 
 N > 1 (torchrun): the path does not shard -- every rank runs an independent replica of the
 workload on its own GPU, no collective on the data path; value = tokens of all ranks / max time.
@@ -39,6 +43,8 @@ L2_BYTES = 126e6
 # dram__bytes_read.sum + dram__bytes_write.sum per decode launch from the committed ncu capture
 # (profiles/), keyed by workload name; None until a capture exists for that workload.
 NCU_TRAFFIC_BYTES = {"c1_llama8b_b1_32k": 143.1e6}   # profiles/decode_stream_c1.md
+MIN_TIMED_S = 0.5     # the K-step region is repeated until this much timed work has accumulated
+MAX_REPS = 4000
 KERNEL_KNOBS = {}   # tuning overrides from the command line (decode_chunk, decode_state_splits, decode_impl)
 
 
@@ -169,6 +175,16 @@ def oracle_decode_rate(shape, steps: int, warmup: int, single_steps: int = 0):
     return shape.batch / step_s, step_s, used, sample
 
 
+def workload_config(shape, extra=None):
+    """The `config` object of a bench line: what was run, the same keys for both arms."""
+    cfg = {"workload": shape.name, "batch": shape.batch, "context": shape.context, "n_layers": shape.n_layers,
+           "sum_windows": sum(shape.windows), "q_heads": shape.n_q_heads, "kv_heads": shape.n_kv_heads,
+           "head_dim": shape.head_dim, "multi_gpu": "replicas only", "merge": KERNEL_KNOBS.get("merge", 0)}
+    if extra:
+        cfg.update(extra)
+    return cfg
+
+
 def run_reference(args, shape):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
@@ -179,9 +195,8 @@ def run_reference(args, shape):
         "impl": "reference", "metric": "hybrid-attn decode tokens/s", "value": tok_s, "unit": "tokens/s",
         "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup, "ms_per_step": step_s * 1e3,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": shape.name, "batch": shape.batch, "context": shape.context,
-                   "sum_windows": sum(shape.windows), "timed_oracle_steps_per_layer_class": steps,
-                   "merge": KERNEL_KNOBS.get("merge", 0)},
+        "config": workload_config(shape, {"l2": "host memory (the oracle runs on the host cores)",
+                                          "timing": f"{steps} oracle steps per distinct window size, see cpu_baseline.sample"}),
         "cpu_baseline": {"value": tok_s, "unit": "tokens/s", "cores": cores, "kind": "oracle", "sample": sample},
         "e2e": {"value": tok_s, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
@@ -248,6 +263,156 @@ def whole_job_tokens_per_s(world: int, batch: int, steps: int, ms: float) -> flo
     return world * batch * steps / (ms * 1e-3)
 
 
+def roofline_bytes(shape):
+    """(the benchmark spec's bytes, bytes with the step's own q/k/v/out rows and the ring append) of one decode step."""
+    return configs.decode_step_stream_bytes(shape, shape.context), configs.decode_step_bytes(shape, shape.context)
+
+
+class DecodeBench:
+    """The decode-step measurement of one workload: state copies built by glide_prefill, inputs resident in HBM,
+    K back-to-back steps between two CUDA events, repeated; steps rotate over the state copies."""
+
+    def __init__(self, shape, K, W, device, dist, prefill_tokens=0):
+        self.shape, self.K, self.W, self.device, self.dist = shape, K, max(W, 3), device, dist
+        self.bytes_stream, self.bytes_io = roofline_bytes(shape)
+        self.prefill_tokens = prefill_tokens
+        free_b, _ = torch.cuda.mem_get_info(device)
+        n_rep = max(1, min(16, math.ceil(8 * L2_BYTES / self.bytes_io)))
+        # positions a state copy may advance before it is rewound (and room for the prefill measurement at the end)
+        self.slack = max(256, 6 * K + 64) + 3 * prefill_tokens
+        cfg_probe = self._workspace_bytes(shape, self.slack)
+        n_rep = max(1, min(n_rep, int(0.8 * free_b // max(cfg_probe, 1))))
+        self.n_rep = n_rep
+        self.ctxs, self.wl = build_states(shape, n_rep, self.slack, device)
+        L, B, H, Hkv, d = shape.n_layers, shape.batch, shape.n_q_heads, shape.n_kv_heads, shape.head_dim
+        self.dt = torch_dtype(shape)
+        # inputs of the timed steps, resident in HBM: one buffer per step holding q | k | v
+        self.n_in = min(K, 64)
+        self.nq, self.nk = L * B * H * d, L * B * Hkv * d
+        self.dev_in = torch.empty((self.n_in, self.nq + 2 * self.nk), dtype=self.dt, device=device)
+        for i in range(self.n_in):
+            q, k, v = self.wl.decode_qkv(shape.context + i, device)
+            self.dev_in[i, :self.nq] = q.reshape(-1)
+            self.dev_in[i, self.nq:self.nq + self.nk] = k.reshape(-1)
+            self.dev_in[i, self.nq + self.nk:] = v.reshape(-1)
+        self.outs = [torch.empty((L, B, H, d), dtype=self.dt, device=device) for _ in range(2)]
+        self.step_no = 0
+        self.advanced = [0] * n_rep              # steps each copy has taken since it was last rewound
+
+    @staticmethod
+    def _workspace_bytes(shape, slack):
+        from paper_2607_24788_b200 import glide
+        cfg, keep = glide.make_config(shape.windows, shape.batch, shape.n_q_heads, shape.n_kv_heads, shape.head_dim,
+                                      shape.context + slack, dtype=torch_dtype(shape), prefill_chunk=shape.prefill_chunk,
+                                      **KERNEL_KNOBS)
+        return glide.glide_workspace_bytes(cfg)
+
+    def views(self, buf):
+        L, B, H, Hkv, d = (self.shape.n_layers, self.shape.batch, self.shape.n_q_heads, self.shape.n_kv_heads,
+                           self.shape.head_dim)
+        nq, nk = self.nq, self.nk
+        return (buf[:nq].view(L, B, H, d), buf[nq:nq + nk].view(L, B, Hkv, d), buf[nq + nk:].view(L, B, Hkv, d))
+
+    def one_step(self, buf, ctx_index=None):
+        i = self.step_no
+        self.step_no += 1
+        c = i % self.n_rep if ctx_index is None else ctx_index
+        q, k, v = self.views(buf)
+        self.ctxs[c].glide_decode_step(q, k, v, self.outs[i & 1])
+        self.advanced[c] += 1
+
+    def make_room(self, steps_per_ctx):
+        """Rewinds the position counters of copies that could not take `steps_per_ctx` more steps (untimed; ring, S
+        and z stay as they are: the time of a step does not depend on the values)."""
+        for c in range(len(self.ctxs)):
+            if self.advanced[c] + steps_per_ctx + 2 > self.slack - 3 * self.prefill_tokens:
+                self.rewind(c)
+
+    def rewind(self, c):
+        for l in range(self.shape.n_layers):
+            self.ctxs[c].glide_import_state(l, self.shape.context, None, None, None, None)
+        self.advanced[c] = 0
+
+    def barrier(self):
+        torch.cuda.synchronize()
+        if self.dist is not None:
+            self.dist.barrier()
+            torch.cuda.synchronize()
+
+    def warm_up(self):
+        for i in range(self.W):
+            self.one_step(self.dev_in[i % self.n_in])
+        self.barrier()
+
+    def back_to_back(self, reps, local_rank):
+        """Median time of K back-to-back steps; repeated `reps` times at least and until MIN_TIMED_S of timed work."""
+        K = self.K
+        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        times_ms, total = [], 0.0
+        per_ctx = math.ceil(K / self.n_rep) + 1
+        with ClockSampler(local_rank) as clocks:
+            while len(times_ms) < reps or (total < MIN_TIMED_S * 1e3 and len(times_ms) < MAX_REPS):
+                self.make_room(per_ctx)
+                self.barrier()
+                ev0.record()
+                for i in range(K):
+                    self.one_step(self.dev_in[i % self.n_in])
+                ev1.record()
+                self.barrier()
+                times_ms.append(ev0.elapsed_time(ev1))
+                total += times_ms[-1]
+        return statistics.median(times_ms), len(times_ms), clocks.summary()
+
+    def isolated(self, n_steps):
+        """Every step between its own pair of events (rotating state copies as above): an event between two launches
+        keeps the next launch from overlapping the previous one's tail.  Sorted microseconds."""
+        self.make_room(math.ceil(n_steps / self.n_rep) + 1)
+        evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(n_steps)]
+        self.barrier()
+        for i in range(n_steps):
+            evs[i][0].record()
+            self.one_step(self.dev_in[i % self.n_in])
+            evs[i][1].record()
+        self.barrier()
+        return sorted(a.elapsed_time(b) * 1e3 for a, b in evs)
+
+    def close(self):
+        self.ctxs, self.dev_in, self.outs = None, None, None
+        torch.cuda.empty_cache()
+
+
+def latency_summary(lat_us):
+    return {"median": lat_us[len(lat_us) // 2], "p10": lat_us[len(lat_us) // 10], "p90": lat_us[(len(lat_us) * 9) // 10],
+            "steps": len(lat_us),
+            "note": "each step between its own two events (no overlap with the neighbours), rank 0"}
+
+
+def side_workload(shape, K, W, device, local_rank, prefill_tokens=0):
+    """One entry of `workloads`: the same decode measurement on another configuration or control."""
+    peak, peak_kind = load_peaks()
+    b = DecodeBench(shape, K, W, device, None, prefill_tokens)
+    b.warm_up()
+    t_ms, n_reps, clocks = b.back_to_back(3, local_rank)
+    lat = b.isolated(max(K, 16))
+    us = t_ms * 1e3 / K
+    entry = {"us_per_step": us, "tokens_per_s": shape.batch / (us * 1e-6), "isolated_step_us": latency_summary(lat)["median"],
+             "algorithmic_bytes_per_launch": b.bytes_stream, "algorithmic_bytes_incl_io": b.bytes_io,
+             "achieved_gbs": b.bytes_stream / (us * 1e-6) / 1e9, "frac": b.bytes_stream / (us * 1e-6) / 1e9 / peak,
+             "frac_incl_io": b.bytes_io / (us * 1e-6) / 1e9 / peak, "peak_kind": f"of {peak_kind}",
+             "state_copies": b.n_rep, "repetitions": n_reps, "steps_per_repetition": K, "clocks": clocks,
+             "kernel": decode_kernel_name(shape), "sum_windows": sum(shape.windows), "batch": shape.batch,
+             "context": shape.context}
+    if prefill_tokens > 0:
+        b.rewind(b.n_rep - 1)
+        entry["prefill"] = measure_prefill(b.ctxs[-1], b.wl, shape, prefill_tokens, device)
+    b.close()
+    return entry
+
+
+SIDE_WORKLOADS = ("c2_llama8b_b16_16k", "c2_control_uniform_w1024", "c3_llama8b_b4_128k", "c3_control_full_kv",
+                  "c4_mistral7b_b8_8k_chunked", "p1_blockwise_0_half_w")
+
+
 def run_glide(args, shape):
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -262,140 +427,91 @@ def run_glide(args, shape):
         dist.init_process_group("nccl", device_id=device)
 
     K, W = args.steps, args.warmup
-    step_bytes = configs.decode_step_bytes(shape, shape.context)
-    n_rep = max(1, min(16, math.ceil(8 * L2_BYTES / step_bytes)))
-    reps = args.reps
-    extra = math.ceil((max(W, 3) + (reps + 1) * K + 3 + 3 * K) / n_rep) + 6 * K + 32 + 3 * args.prefill_tokens
-    ctxs, wl = build_states(shape, n_rep, extra, device)
+    b = DecodeBench(shape, K, W, device, dist, args.prefill_tokens)
     L, B, H, Hkv, d = shape.n_layers, shape.batch, shape.n_q_heads, shape.n_kv_heads, shape.head_dim
-    dt = torch_dtype(shape)
-
-    # inputs of the timed steps, resident in HBM: one buffer per step holding q | k | v
-    n_in = min(K, 64)
-    nq, nk = L * B * H * d, L * B * Hkv * d
-    dev_in = torch.empty((n_in, nq + 2 * nk), dtype=dt, device=device)
-    for i in range(n_in):
-        q, k, v = wl.decode_qkv(shape.context + i, device)
-        dev_in[i, :nq] = q.reshape(-1)
-        dev_in[i, nq:nq + nk] = k.reshape(-1)
-        dev_in[i, nq + nk:] = v.reshape(-1)
-    outs = [torch.empty((L, B, H, d), dtype=dt, device=device) for _ in range(2)]
-
-    def views(buf):
-        return (buf[:nq].view(L, B, H, d), buf[nq:nq + nk].view(L, B, Hkv, d), buf[nq + nk:].view(L, B, Hkv, d))
-
-    step_no = [0]
-
-    def one_step(buf):
-        i = step_no[0]
-        step_no[0] += 1
-        q, k, v = views(buf)
-        ctxs[i % n_rep].glide_decode_step(q, k, v, outs[i & 1])
-
-    def barrier():
-        torch.cuda.synchronize()
-        if dist is not None:
-            dist.barrier()
-            torch.cuda.synchronize()
-
-    for i in range(max(W, 3)):
-        one_step(dev_in[i % n_in])
-    barrier()
-
-    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    times_ms = []
-    with ClockSampler(local_rank) as clocks:
-        for _ in range(reps):
-            barrier()
-            ev0.record()
-            for i in range(K):
-                one_step(dev_in[i % n_in])
-            ev1.record()
-            barrier()
-            times_ms.append(ev0.elapsed_time(ev1))
-    t_ms = statistics.median(times_ms)
-
-    # every step on its own pair of events (rotating state copies as above): the spread of the step latency;
-    # an event between two launches keeps the next launch from overlapping the previous one's tail
-    lat_us = []
-    evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(K)]
-    barrier()
-    for i in range(K):
-        evs[i][0].record()
-        one_step(dev_in[i % n_in])
-        evs[i][1].record()
-    barrier()
-    lat_us = sorted(a.elapsed_time(b) * 1e3 for a, b in evs)
+    dt, nq, nk, n_in = b.dt, b.nq, b.nk, b.n_in
+    b.warm_up()
+    t_ms, n_reps, clocks = b.back_to_back(args.reps, local_rank)
+    lat_us = b.isolated(max(K, 32))
 
     # same context every step: window and state of the previous step may still sit in L2
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     hot_ms = []
-    for _ in range(3):
-        barrier()
+    for _ in range(5):
+        b.make_room(K + 1)
+        b.barrier()
         ev0.record()
         for i in range(K):
-            q, k, v = views(dev_in[i % n_in])
-            ctxs[0].glide_decode_step(q, k, v, outs[i & 1])
+            b.one_step(b.dev_in[i % n_in], ctx_index=0)
         ev1.record()
-        barrier()
+        b.barrier()
         hot_ms.append(ev0.elapsed_time(ev1))
     hot_ms = statistics.median(hot_ms)
 
     # end to end through the public call with HOST buffers: pinned q|k|v -> device, step, out -> pinned host
     host_in = torch.empty((n_in, nq + 2 * nk), dtype=dt).pin_memory()
-    host_in.copy_(dev_in.cpu())
+    host_in.copy_(b.dev_in.cpu())
     host_out = torch.empty((L, B, H, d), dtype=dt).pin_memory()
     stage = torch.empty((nq + 2 * nk,), dtype=dt, device=device)
     e2e_steps = K
 
     def e2e_step(i):
         stage.copy_(host_in[i % n_in], non_blocking=True)
-        one_step(stage)
-        host_out.copy_(outs[(step_no[0] - 1) & 1], non_blocking=True)
+        b.one_step(stage)
+        host_out.copy_(b.outs[(b.step_no - 1) & 1], non_blocking=True)
         torch.cuda.current_stream().synchronize()   # the next token depends on this result
 
+    b.make_room(3)
     for i in range(3):
         e2e_step(i)
     e2e_ms = []
-    for _ in range(3):
-        barrier()
+    for _ in range(5):
+        b.make_room(math.ceil(e2e_steps / b.n_rep) + 1)
+        b.barrier()
         ev0.record()
         for i in range(e2e_steps):
             e2e_step(i)
         ev1.record()
-        barrier()
+        b.barrier()
         e2e_ms.append(ev0.elapsed_time(ev1))
     e2e_t = statistics.median(e2e_ms)
 
     per_layer = None
-    if world == 1 and step_bytes <= (8 << 30):
-        per_layer = measure_per_layer_launch(ctxs[0], shape, views(dev_in[0]), outs[0], K, device)
+    if world == 1 and b.bytes_io <= (8 << 30):
+        b.make_room(1)
+        per_layer = measure_per_layer_launch(b.ctxs[0], shape, b.views(b.dev_in[0]), b.outs[0], K, device)
 
     t_ms, hot_ms, e2e_t = max_over_ranks([t_ms, hot_ms, e2e_t], dist, device)
 
     if rank == 0:
         peak, peak_kind = load_peaks()
         launch_s = t_ms * 1e-3 / K
-        achieved = step_bytes / launch_s / 1e9
-        info = ctxs[0].glide_decode_launch_info()
+        achieved = b.bytes_stream / launch_s / 1e9
+        info = b.ctxs[0].glide_decode_launch_info()
         elem = shape.elem_bytes
+        lat = latency_summary(lat_us)
         line = {
             "metric": "hybrid-attn decode tokens/s", "value": whole_job_tokens_per_s(world, B, K, t_ms), "unit": "tokens/s",
-            "n_gpus": world, "steps": K, "warmup": max(W, 3), "ms_per_step": t_ms / K, "higher_is_better": True,
+            "n_gpus": world, "steps": K, "warmup": b.W, "ms_per_step": t_ms / K, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f32" if shape.dtype == "f32" else "bf16+f32state",
             "data": "synthetic",
-            "config": {"workload": shape.name, "batch": B, "context": shape.context, "n_layers": L,
-                       "sum_windows": sum(shape.windows), "q_heads": H, "kv_heads": Hkv, "head_dim": d,
-                       "l2": f"steps rotate over {n_rep} independent state copies ({n_rep * step_bytes / 1e6:.0f} MB per "
-                             f"rotation > 126 MB L2); median of {reps} repetitions of K steps",
-                       "multi_gpu": "replicas only", "merge": KERNEL_KNOBS.get("merge", 0)},
+            "config": workload_config(shape, {
+                "l2": f"steps rotate over {b.n_rep} independent state copies ({b.n_rep * b.bytes_io / 1e6:.0f} MB per "
+                      f"rotation > 126 MB L2)",
+                "timing": f"value = back-to-back throughput: K steps between two events, consecutive launches overlap by "
+                          f"programmatic dependent launch; median of {n_reps} repetitions (>= {MIN_TIMED_S} s of timed "
+                          f"work); the isolated-step latency is per_step_attention_latency_us"}),
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                          "traffic": NCU_TRAFFIC_BYTES.get(shape.name), "peak_kind": f"of {peak_kind}",
-                         "kernel": decode_kernel_name(shape), "algorithmic_bytes_per_launch": step_bytes,
-                         "frac_of_nominal_8TBps": achieved / 8000.0},
-            "per_step_attention_latency_us": launch_s * 1e6,
-            "step_latency_us": {"median": lat_us[len(lat_us) // 2], "p10": lat_us[len(lat_us) // 10],
-                                "p90": lat_us[(len(lat_us) * 9) // 10], "steps": len(lat_us),
-                                "note": "each step between its own two events (no overlap with the neighbours), rank 0"},
+                         "kernel": decode_kernel_name(shape), "algorithmic_bytes_per_launch": b.bytes_stream,
+                         "bytes_formula": "sum over layers and sequences of 2 w H_kv d 2B (window) + S,z read and written",
+                         "algorithmic_bytes_incl_io": b.bytes_io,
+                         "frac_incl_io": b.bytes_io / launch_s / 1e9 / peak,
+                         "frac_of_nominal_8TBps": achieved / 8000.0,
+                         "isolated_step_frac": b.bytes_stream / (lat["median"] * 1e-6) / 1e9 / peak},
+            "per_step_attention_latency_us": lat["median"],
+            "back_to_back_us_per_step": launch_s * 1e6,
+            "step_latency_us": lat,
             "hot_l2": {"tokens_per_s": world * B * K / (hot_ms * 1e-3), "us_per_step": hot_ms * 1e3 / K,
                        "note": "same sequence state every step (L2 may hold part of it)"},
             "e2e": {"value": world * B * e2e_steps / (e2e_t * 1e-3), "unit": "tokens/s",
@@ -403,13 +519,27 @@ def run_glide(args, shape):
                     "us_per_step": e2e_t * 1e3 / e2e_steps},
             "gpu_launches": K * info["launches"],
             "decode_launch": info,
-            "clocks": clocks.summary(),
+            "clocks": clocks,
         }
         if per_layer is not None:
             per_layer["vs_one_launch_hot_l2"] = per_layer["us_per_step"] / (hot_ms * 1e3 / K)
             line["per_layer_launch"] = per_layer
         if args.prefill_tokens > 0:
-            line["prefill"] = measure_prefill(ctxs[-1], wl, shape, args.prefill_tokens, device)
+            b.rewind(b.n_rep - 1)
+            line["prefill"] = measure_prefill(b.ctxs[-1], b.wl, shape, args.prefill_tokens, device)
+        b.close()
+        if world == 1 and args.side_workloads != "none":
+            names = SIDE_WORKLOADS if args.side_workloads == "all" else tuple(args.side_workloads.split(","))
+            line["workloads"] = {}
+            for name in names:
+                if name == shape.name:
+                    continue
+                try:
+                    line["workloads"][name] = side_workload(configs.ALL[name], K, W, device, local_rank,
+                                                            prefill_tokens=256 if name.startswith("c3_llama") else 0)
+                except torch.OutOfMemoryError as e:   # a device with less memory than the control needs
+                    line["workloads"][name] = {"skipped": f"out of device memory: {str(e)[:80]}"}
+                    torch.cuda.empty_cache()
         if world == 1 and not args.no_cpu_baseline:
             tok_s, step_s, cores, sample = oracle_decode_rate(shape, 4, 1, single_steps=2)
             line["cpu_baseline"] = {"value": tok_s, "unit": "tokens/s", "cores": cores, "kind": "oracle",
@@ -507,7 +637,12 @@ def main():
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=256)
     ap.add_argument("--warmup", type=int, default=20)
-    ap.add_argument("--reps", type=int, default=15, help="repetitions of the K-step timed region (median reported)")
+    ap.add_argument("--reps", type=int, default=15,
+                    help="least number of repetitions of the K-step timed region (median reported; repeated further "
+                         "until half a second of timed work has accumulated)")
+    ap.add_argument("--side-workloads", default="all",
+                    help="'all', 'none' or a comma-separated list: the other configurations and controls timed after "
+                         "the headline workload (one GPU only)")
     ap.add_argument("--workload", default=configs.C1.name, choices=sorted(configs.ALL))
     ap.add_argument("--impl", default="glide", choices=["glide", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")

@@ -234,6 +234,17 @@ int glide_device_status(glide_ctx *ctx, void *stream, int32_t *status_out);
 /* Kernels one glide_decode_step launches and work items it processes (for launch accounting). */
 int glide_decode_launch_info(glide_ctx *ctx, int32_t *n_launches, int32_t *n_work_items, int32_t *grid_size);
 
+/* The streaming decode kernel's static schedule of one all-layer step (Sec. III-B: one unit of work per layer, sequence
+ * and KV head: its window of w_l ring slots and its d x d state), as glide_create would build it on a device with
+ * n_sms SMs and smem_limit bytes of shared memory per CTA.  Host only, no CUDA calls.  *n_rows receives the number
+ * of segments; the first min(*n_rows, max_rows) are described in rows_out, 12 int32 each: {CTA, warp of the CTA,
+ * unit, layer, state tiles, first state tile, window tiles, first window tile, warps of the CTA that share the unit
+ * (1: none), the segment's shared-memory record slot (-1: none), index of the CTA's global record (-1: the unit lies
+ * in one CTA), global records of the unit}.  A tile is 16 rows of S or 16 ring slots.  GLIDE_ERR_UNSUPPORTED when
+ * the configuration does not run on that kernel. */
+int glide_stream_schedule(const glide_config *cfg, int32_t n_sms, int64_t smem_limit, int32_t *rows_out, int32_t max_rows,
+                          int32_t *n_rows);
+
 /* Static, NUL-terminated description of a status code. */
 const char *glide_strerror(int code);
 

@@ -97,6 +97,18 @@ def decode_step_bytes(shape: GlideShape, n: int) -> int:
     return total * shape.batch
 
 
+def decode_step_stream_bytes(shape: GlideShape, n: int) -> int:
+    """The roofline bytes of one decode step as the task states them: per layer and sequence the window's K and V rows,
+    2 w H_kv d elem, plus the recurrent state S, z read and written once the layer evicts (all sequences)."""
+    Hkv, d, eb = shape.n_kv_heads, shape.head_dim, shape.elem_bytes
+    total = 0
+    for w in shape.windows:
+        total += 2 * min(w, n + 1) * Hkv * d * eb
+        if n >= w:
+            total += 2 * (Hkv * d * d + Hkv * d) * 4
+    return total * shape.batch
+
+
 def theoretical_speedup(alpha: float, w: float, d: float) -> float:
     """Per-token speedup of a three-equal-block (0, alpha*w, w) allocation over the (0,0,0) hybrid
     (Sec. III-C): S = 1 + (1 + alpha) / ((2 + 3d/w) - alpha)."""

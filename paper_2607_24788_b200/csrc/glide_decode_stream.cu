@@ -24,6 +24,7 @@
 #include <algorithm>
 
 #include "glide_device.cuh"
+#include "glide_trace.cuh"
 
 namespace glide {
 
@@ -58,22 +59,6 @@ constexpr int kHdrSlots = 3;
 #endif
 #ifndef GLIDE_W_EDGE
 #define GLIDE_W_EDGE 40
-#endif
-
-// Optional per-warp event trace (debug builds only: -DGLIDE_TRACE).
-#ifdef GLIDE_TRACE
-__device__ unsigned long long *g_stream_trace = nullptr;   // [warps][64] of (code << 56 | globaltimer ns)
-#define GLIDE_TRACE_EVENT(code)                                                                        \
-  do {                                                                                                 \
-    if (g_stream_trace && lane == 0 && trace_n < 64) {                                                 \
-      unsigned long long now;                                                                          \
-      asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(now));                                          \
-      g_stream_trace[(size_t(blockIdx.x) * kWarps + (threadIdx.x >> 5)) * 64 + trace_n++] =            \
-          (static_cast<unsigned long long>(code) << 56) | (now & 0x00ffffffffffffffull);               \
-    }                                                                                                  \
-  } while (0)
-#else
-#define GLIDE_TRACE_EVENT(code) do { } while (0)
 #endif
 
 // ---- PTX wrappers --------------------------------------------------------------------------
@@ -293,9 +278,7 @@ glide_decode_stream_kernel(const DecodeParams p, const StreamParams sp) {
   int64_t *sm_t = reinterpret_cast<int64_t *>(base + sp.t_off);                       // [max_segs], behind the pool
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-#ifdef GLIDE_TRACE
-  int trace_n = 0;
-#endif
+  GLIDE_TRACE_DECL;
   GLIDE_TRACE_EVENT(1);
   // Programmatic dependent launch: the next launch in the stream may start its prologue on SMs this grid has
   // left; whatever an earlier kernel wrote is read only after griddepcontrol.wait below.
@@ -525,16 +508,7 @@ glide_decode_stream_kernel(const DecodeParams p, const StreamParams sp) {
 
   // ---- state tile: 16 rows of S and z, updated in the stage and stored back by the async proxy ---------
   // (bulk stores are not ordered by this warp's later fences, so a ticket never waits for state traffic)
-#ifdef GLIDE_TRACE
-  long long cyc[6] = {0, 0, 0, 0, 0, 0};
-#define GLIDE_CYC_MARK(var) long long var = clock64()
-#define GLIDE_CYC_ADD(i, var) do { long long n_ = clock64(); cyc[i] += n_ - var; var = n_; } while (0)
-#else
-#define GLIDE_CYC_MARK(var) do { } while (0)
-#define GLIDE_CYC_ADD(i, var) do { } while (0)
-#endif
   auto consume_state = [&](const StreamSegment &sg, int stile, float4 *st, float *zs, uint32_t st_addr, uint32_t z_addr) {
-    GLIDE_CYC_MARK(cm);
     const int src0 = stile * 4;   // lane that holds phi entries of the tile's first row (4 rows per lane)
 #pragma unroll
     for (int r = 0; r < kTileRows; ++r) {
@@ -554,7 +528,6 @@ glide_decode_stream_kernel(const DecodeParams p, const StreamParams sp) {
         a[h].w = fmaf(f, s.w, a[h].w);
       }
     }
-    GLIDE_CYC_ADD(0, cm);
     // z: lane r < 16 owns row r of the tile
     const int zsrc = src0 + ((lane & 15) >> 2);
     float zn = 0.f;
@@ -575,10 +548,8 @@ glide_decode_stream_kernel(const DecodeParams p, const StreamParams sp) {
         bp[h - 1] = fmaf(f, zn, bp[h - 1]);
       }
     }
-    GLIDE_CYC_ADD(1, cm);
     fence_async_smem();   // the updated rows are read by the async proxy
     __syncwarp();
-    GLIDE_CYC_ADD(2, cm);
     if (lane == 0) {
       float *Sg = reinterpret_cast<float *>(p.ws + size_t(sg.S_off256) * 256) + size_t(stile) * kTileRows * kD;
       float *zg = reinterpret_cast<float *>(p.ws + size_t(sg.z_off256) * 256) + stile * kTileRows;
@@ -587,7 +558,6 @@ glide_decode_stream_kernel(const DecodeParams p, const StreamParams sp) {
       bulk_commit();
       bulk_wait_read0();   // the stage may be refilled once the store has read it
     }
-    GLIDE_CYC_ADD(3, cm);
   };
 
   // ---- main loop over this warp's segments ------------------------------------------------------------
@@ -607,7 +577,6 @@ glide_decode_stream_kernel(const DecodeParams p, const StreamParams sp) {
       failed = true;
       break;
     }
-    GLIDE_TRACE_EVENT(15);
     {
       const uint32_t *hq = reinterpret_cast<const uint32_t *>(my_hdr_ptr);
       const bool valid = hrow < G;
@@ -638,7 +607,6 @@ glide_decode_stream_kernel(const DecodeParams p, const StreamParams sp) {
       }
     }
     __syncwarp();
-    GLIDE_TRACE_EVENT(16);
     if (s + 1 < seg_hi) issue_header(s + 1);
     // A parked slot (negative position; only batches with slot offsets have them) goes through the header hand-over
     // like every segment and then leaves: it has no tiles, and nothing of it is reduced or written.  All segments
@@ -658,7 +626,6 @@ glide_decode_stream_kernel(const DecodeParams p, const StreamParams sp) {
       a[h] = make_float4(0.f, 0.f, 0.f, 0.f);
       bp[h] = 0.f;
     }
-    GLIDE_TRACE_EVENT(7);
 
     // -- tiles ------------------------------------------------------------------------------------------
     int last_stage = -1;
@@ -679,11 +646,8 @@ glide_decode_stream_kernel(const DecodeParams p, const StreamParams sp) {
       stage = stage + 1 == STAGES ? 0 : stage + 1;
       __syncwarp();   // every lane is done with the stage before it is refilled
       if (k + 1 < n_total) issue_next();   // the last tile's stage first serves as scratch for the finish
-      GLIDE_TRACE_EVENT(5);
     }
     if (failed) break;
-
-    GLIDE_TRACE_EVENT(17);
     // -- finish: record (m, l, acc) in a common layout: lane holds features 4*lane..4*lane+3 of every head --
     float mh[G], lh[G];
     float4 acc[G];
@@ -729,9 +693,7 @@ glide_decode_stream_kernel(const DecodeParams p, const StreamParams sp) {
         acc[h] = make_float4(0.f, 0.f, 0.f, 0.f);
       }
     }
-    GLIDE_TRACE_EVENT(18);
     if (n_total > 0) issue_next();   // the deferred refill
-    GLIDE_TRACE_EVENT(19);
     if (n_state_eff > 0) warp_sum_multi<G>(bp);
     if (!SUM && n_state_eff > 0) {   // fold the linear readout in as a term with logit 0
 #pragma unroll
@@ -746,7 +708,6 @@ glide_decode_stream_kernel(const DecodeParams p, const StreamParams sp) {
         mh[h] = mn;
       }
     }
-    GLIDE_TRACE_EVENT(20);
     if (sg.grp_size > 1) {
       // several warps of this CTA share the unit: records meet in shared memory, the last one to arrive
       // combines them and carries the unit on
@@ -847,7 +808,6 @@ glide_decode_stream_kernel(const DecodeParams p, const StreamParams sp) {
       }
       if (n_pending == 0) pend0 = s; else pend1 = s;
       ++n_pending;
-      GLIDE_TRACE_EVENT(10);
     } else {
       // the whole unit is in this range: current token's own term, shared normaliser, output row, ring append
       float vx[4];
@@ -1057,11 +1017,6 @@ glide_decode_stream_kernel(const DecodeParams p, const StreamParams sp) {
     }
   }
   if (failed && lane == 0) atomicExch(&p.ctl->status, kDevWaitTimeout);
-#ifdef GLIDE_TRACE
-  if (g_stream_trace && lane == 0)
-    for (int i = 0; i < 4; ++i)
-      g_stream_trace[(size_t(blockIdx.x) * kWarps + warp) * 64 + 60 + i] = (static_cast<unsigned long long>(100 + i) << 56) | (unsigned long long)cyc[i];
-#endif
   if (lane == 0) bulk_wait0();   // this warp's state stores have landed
   GLIDE_TRACE_EVENT(9);
 
@@ -1329,14 +1284,10 @@ int stream_decode_supported(const glide_ctx *ctx) {
   return ctx->cfg.io_dtype == GLIDE_BF16 && ctx->cfg.head_dim == kD;
 }
 
-int stream_decode_setup(glide_ctx *ctx) {
-  const int n_ctas = std::min(ctx->sm_count * GLIDE_STREAM_CTAS_PER_SM, kMaxStreamCtas);
+// Host-only part of the set-up: every schedule of the context for a device with n_ctas SMs and smem_limit bytes of
+// shared memory per CTA; sizes the record pool so that stages, tables and pool fit.
+int stream_decode_plan(glide_ctx *ctx, int n_ctas, size_t smem_limit) {
   const int L = ctx->cfg.n_layers;
-  int dev_max = 0;
-  if (cudaDeviceGetAttribute(&dev_max, cudaDevAttrMaxSharedMemoryPerBlockOptin, ctx->device) != cudaSuccess) {
-    cudaGetLastError();
-    return GLIDE_ERR_CUDA;
-  }
   bool contiguous = true;
   for (int g = 0; g < ctx->cfg.n_kv_heads; ++g)
     for (int i = 1; i < ctx->G; ++i)
@@ -1370,11 +1321,29 @@ int stream_decode_setup(glide_ctx *ctx) {
         ctx->stream_scheds.push_back(std::move(sc));
       }
       if (ctx->stream_segs.size() > ctx->stream_seg_capacity) return GLIDE_ERR_UNSUPPORTED;
-      if (stream_smem_bytes<G, S, SUM>(ctx->stream_max_segs, pool_slots) <= size_t(dev_max)) break;
+      if (stream_smem_bytes<G, S, SUM>(ctx->stream_max_segs, pool_slots) <= smem_limit) break;
       const size_t without_pool = stream_smem_bytes<G, S, SUM>(ctx->stream_max_segs, 0);
-      if (attempt > 0 || without_pool > size_t(dev_max)) return GLIDE_ERR_UNSUPPORTED;   // the table alone does not fit
-      pool_slots = int((size_t(dev_max) - without_pool) / size_t(rec_bytes));
+      if (attempt > 0 || without_pool > smem_limit) return GLIDE_ERR_UNSUPPORTED;   // the table alone does not fit
+      pool_slots = int((smem_limit - without_pool) / size_t(rec_bytes));
     }
+    ctx->stream_smem = stream_smem_bytes<G, S, SUM>(ctx->stream_max_segs, pool_slots);
+    ctx->decode_grid = n_ctas;
+    return GLIDE_OK;
+  });
+}
+
+int stream_decode_setup(glide_ctx *ctx) {
+  const int n_ctas = std::min(ctx->sm_count * GLIDE_STREAM_CTAS_PER_SM, kMaxStreamCtas);
+  int dev_max = 0;
+  if (cudaDeviceGetAttribute(&dev_max, cudaDevAttrMaxSharedMemoryPerBlockOptin, ctx->device) != cudaSuccess) {
+    cudaGetLastError();
+    return GLIDE_ERR_CUDA;
+  }
+  const int rc = stream_decode_plan(ctx, n_ctas, size_t(dev_max));
+  if (rc) return rc;
+  return dispatch_stream(ctx->G, ctx->cfg.merge != GLIDE_MERGE_SHARED, [&](auto gg, auto ss, auto mm) -> int {
+    constexpr int G = decltype(gg)::value, S = decltype(ss)::value;
+    constexpr bool SUM = decltype(mm)::value != 0;
     // the attribute belongs to the kernel, not to the context: ask for the device maximum so that contexts with
     // different schedules (different table sizes) can be alive together
     if (cudaFuncSetAttribute(glide_decode_stream_kernel<G, S, SUM, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -1384,17 +1353,9 @@ int stream_decode_setup(glide_ctx *ctx) {
       cudaGetLastError();
       return GLIDE_ERR_CUDA;
     }
-    ctx->stream_smem = stream_smem_bytes<G, S, SUM>(ctx->stream_max_segs, pool_slots);
-    ctx->decode_grid = n_ctas;
     return GLIDE_OK;
   });
 }
-
-#ifdef GLIDE_TRACE
-extern "C" int glide_debug_set_stream_trace(void *dev_buf) {
-  return cudaMemcpyToSymbol(g_stream_trace, &dev_buf, sizeof(void *)) == cudaSuccess ? 0 : 6;
-}
-#endif
 
 int launch_decode_stream(glide_ctx *ctx, const DecodeParams &p, int schedule, cudaStream_t stream) {
   if (schedule < 0 || size_t(schedule) >= ctx->stream_scheds.size()) return GLIDE_ERR_INVALID_ARG;

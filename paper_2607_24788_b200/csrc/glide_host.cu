@@ -585,6 +585,32 @@ int glide_decode_launch_info(glide_ctx *ctx, int32_t *n_launches, int32_t *n_wor
   return GLIDE_OK;
 }
 
+int glide_stream_schedule(const glide_config *cfg, int32_t n_sms, int64_t smem_limit, int32_t *rows_out, int32_t max_rows,
+                          int32_t *n_rows) {
+  if (!n_rows || n_sms < 1 || n_sms * GLIDE_STREAM_CTAS_PER_SM > kMaxStreamCtas || smem_limit < 0 || max_rows < 0 ||
+      (max_rows > 0 && !rows_out))
+    return GLIDE_ERR_INVALID_ARG;
+  glide_ctx ctx;
+  int rc = plan_context(cfg, &ctx, nullptr);
+  if (rc) return rc;
+  if (!stream_decode_supported(&ctx) || cfg->decode_impl == GLIDE_DECODE_FMA || cfg->decode_impl == GLIDE_DECODE_MMA)
+    return GLIDE_ERR_UNSUPPORTED;
+  const int n_ctas = n_sms * GLIDE_STREAM_CTAS_PER_SM;
+  rc = stream_decode_plan(&ctx, n_ctas, size_t(smem_limit));
+  if (rc) return rc;
+  const glide_ctx::StreamSchedule &sc = ctx.stream_scheds[0];
+  *n_rows = int32_t(sc.n_segs);
+  for (int c = 0; c < n_ctas; ++c)
+    for (int i = sc.range_begin[size_t(c) * kStreamWarps]; i < sc.range_begin[size_t(c + 1) * kStreamWarps] && i < max_rows; ++i) {
+      const StreamSegment &sg = ctx.stream_segs[sc.seg_base + size_t(i)];
+      int32_t *r = rows_out + size_t(i) * 12;
+      r[0] = c; r[1] = sg.range; r[2] = sg.unit; r[3] = sg.layer; r[4] = sg.n_state; r[5] = sg.state0; r[6] = sg.n_win;
+      r[7] = sg.win0; r[8] = sg.grp_size; r[9] = sg.grp_size > 1 ? sg.grp_slot0 + sg.grp_idx : -1; r[10] = sg.part;
+      r[11] = sg.n_parts;
+    }
+  return GLIDE_OK;
+}
+
 const char *glide_strerror(int code) {
   switch (code) {
     case GLIDE_OK: return "ok";

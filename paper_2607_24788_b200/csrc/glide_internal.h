@@ -203,6 +203,7 @@ DecodeParams make_decode_params(const glide_ctx *ctx, int layer_begin, int layer
 int build_ring_tensor_maps(glide_ctx *ctx);   // TMA descriptors of every layer's K and V ring (host copy)
 int mma_decode_setup(glide_ctx *ctx);         // sizes the grid of the per-item tensor-core kernel
 int stream_decode_supported(const glide_ctx *ctx);
+int stream_decode_plan(glide_ctx *ctx, int n_ctas, size_t smem_limit);   // every schedule of the context (host only)
 int stream_decode_setup(glide_ctx *ctx);      // builds the static schedule (host copy) and sizes the launch
 int launch_decode_stream(glide_ctx *ctx, const DecodeParams &p, int schedule, cudaStream_t stream);
 int launch_decode_mma(glide_ctx *ctx, const DecodeParams &p, cudaStream_t stream);

@@ -85,6 +85,8 @@ def load_library() -> ctypes.CDLL:
     lib.glide_reset.argtypes = [vp, vp]
     lib.glide_device_status.argtypes = [vp, vp, ctypes.POINTER(i32)]
     lib.glide_decode_launch_info.argtypes = [vp, ctypes.POINTER(i32), ctypes.POINTER(i32), ctypes.POINTER(i32)]
+    lib.glide_stream_schedule.argtypes = [cfgp, i32, i64, ctypes.POINTER(i32), i32, ctypes.POINTER(i32)]
+    lib.glide_stream_schedule.restype = ctypes.c_int
     lib.glide_strerror.argtypes = [ctypes.c_int]
     lib.glide_strerror.restype = ctypes.c_char_p
     for name in ("glide_workspace_bytes", "glide_create", "glide_prefill", "glide_decode_step", "glide_destroy",
@@ -98,6 +100,21 @@ def load_library() -> ctypes.CDLL:
 
 def strerror(code: int) -> str:
     return load_library().glide_strerror(int(code)).decode()
+
+
+def glide_stream_schedule(cfg, n_sms: int = 148, smem_limit: int = 232448):
+    """The streaming decode kernel's all-layer schedule for `cfg` (host only): an int32 array [segments][12], see
+    include/glide.h."""
+    import numpy as np
+    lib = load_library()
+    n = ctypes.c_int32(0)
+    _check(lib.glide_stream_schedule(ctypes.byref(cfg), n_sms, smem_limit, None, 0, ctypes.byref(n)), "glide_stream_schedule")
+    rows = np.zeros((n.value, 12), dtype=np.int32)
+    if n.value:
+        _check(lib.glide_stream_schedule(ctypes.byref(cfg), n_sms, smem_limit,
+                                         rows.ctypes.data_as(ctypes.POINTER(ctypes.c_int32)), n.value, ctypes.byref(n)),
+               "glide_stream_schedule")
+    return rows
 
 
 def _check(code: int, where: str):

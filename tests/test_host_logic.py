@@ -138,3 +138,62 @@ def test_reference_arm_prints_one_json_line_on_cpu():
     d = json.loads(r.stdout.strip().splitlines()[-1])
     assert d["impl"] == "reference" and d["unit"] == "tokens/s" and d["value"] > 0
     assert d["cpu_baseline"]["kind"] == "oracle" and d["e2e"]["h2d_bytes_per_step"] == 0
+
+
+@pytest.mark.parametrize("windows,batch,max_tokens,n_sms", [
+    ([4096] * 4 + [1024] * 8 + [256] * 12 + [64] * 8, 1, 32768 + 64, 148),     # config 1: units heavier than a CTA's share
+    ([4096] * 4 + [1024] * 8 + [256] * 12 + [64] * 8, 16, 16384 + 64, 148),    # config 2: hundreds of whole units per CTA
+    ([1024, 512, 0, 48, 100000], 3, 5000, 148),                                # linear-only, ragged and never-evicting layers
+    ([64], 1, 256, 148), ([200, 17], 2, 300, 20),
+])
+def test_stream_schedule_covers_every_tile_exactly_once(glide, windows, batch, max_tokens, n_sms):
+    """The static schedule of the streaming decode kernel (host logic, no GPU): every 16-row tile of every unit's state
+    and window is in exactly one segment, shared-memory groups and global records are numbered consistently."""
+    import numpy as np
+    hkv, d = 8, 128
+    cfg, keep = glide.make_config(windows, batch, 32, hkv, d, max_tokens, dtype=torch.bfloat16)
+    rows = glide.glide_stream_schedule(cfg, n_sms=n_sms)
+    assert rows.shape[1] == 12 and len(rows) > 0
+    n_units = len(windows) * batch * hkv
+    seen_state = [np.zeros(d // 16, dtype=np.int32) for _ in range(n_units)]
+    seen_win = {}
+    for cta, warp, unit, layer, nst, st0, nw, w0, gsz, slot, part, nparts in rows.tolist():
+        assert 0 <= cta < n_sms and 0 <= warp < 8 and 0 <= unit < n_units and layer == unit // (batch * hkv)
+        cap = min(windows[layer], max_tokens)
+        tiles = (cap + 15) // 16
+        evicts = windows[layer] < max_tokens
+        assert nst >= 0 and nw >= 0 and st0 + nst <= (d // 16 if evicts else 0) and w0 + nw <= tiles
+        seen_state[unit][st0:st0 + nst] += 1
+        seen_win.setdefault(unit, np.zeros(tiles, dtype=np.int32))[w0:w0 + nw] += 1
+    for unit in range(n_units):
+        layer = unit // (batch * hkv)
+        evicts = windows[layer] < max_tokens
+        assert unit in seen_win, f"unit {unit} has no segment"
+        assert (seen_win[unit] == 1).all(), f"window tiles of unit {unit}"
+        assert (seen_state[unit] == (1 if evicts else 0)).all(), f"state tiles of unit {unit}"
+    # groups: the segments of one unit inside one CTA carry its size and distinct slots; records: 0 .. n_parts - 1
+    by_cta_unit, by_unit = {}, {}
+    for r in rows.tolist():
+        by_cta_unit.setdefault((r[0], r[2]), []).append(r)
+        by_unit.setdefault(r[2], []).append(r)
+    for (cta, unit), rs in by_cta_unit.items():
+        sizes = {r[8] for r in rs}
+        if sizes != {1}:
+            assert sizes == {len(rs)} and len({r[9] for r in rs}) == len(rs) and min(r[9] for r in rs) >= 0
+        assert len({r[1] for r in rs}) == len(rs) or sizes == {1}, "one segment per warp in a group"
+    for cta in {r[0] for r in rows.tolist()}:
+        slots = [r[9] for r in rows.tolist() if r[0] == cta and r[9] >= 0]
+        assert len(slots) == len(set(slots)), "record slots of a CTA are distinct"
+    for unit, rs in by_unit.items():
+        nparts = {r[11] for r in rs}
+        assert len(nparts) == 1
+        n = nparts.pop()
+        parts = sorted({r[10] for r in rs})
+        assert parts == ([-1] if n == 1 else list(range(n)))
+
+
+def test_stream_schedule_refuses_what_the_kernel_does_not_run(glide):
+    cfg, keep = glide.make_config([64], 1, 4, 4, 64, 128, dtype=torch.bfloat16)
+    with pytest.raises(glide.GlideError) as e:
+        glide.glide_stream_schedule(cfg)
+    assert e.value.code == glide.GLIDE_ERR_UNSUPPORTED
