@@ -115,7 +115,17 @@ def torch_dtype(shape):
 
 
 def value_scale(shape):
+    """Standard deviation of the q and k entries."""
+    if shape.value_scales is not None:
+        return shape.value_scales[0]
     return synth.default_value_scale(shape.head_dim, shape.unit_variance)
+
+
+def make_workload(shape):
+    """The seeded input generator of a configuration."""
+    return synth.Workload(shape.seed, shape.n_layers, shape.batch, shape.n_q_heads, shape.n_kv_heads, shape.head_dim,
+                          torch_dtype(shape), value_scale(shape),
+                          v_scale=None if shape.value_scales is None else shape.value_scales[1])
 
 
 # ---------------------------------------------------------------------------------------------
@@ -128,8 +138,7 @@ def oracle_decode_rate(shape, steps: int, warmup: int, single_steps: int = 0):
     from oracle import glide_oracle as orc
     import numpy as np
     dt = torch_dtype(shape)
-    wl = synth.Workload(shape.seed, shape.n_layers, shape.batch, shape.n_q_heads, shape.n_kv_heads, shape.head_dim, dt,
-                        value_scale(shape))
+    wl = make_workload(shape)
     scale = float(np.float32(1.0) / np.sqrt(np.float32(shape.head_dim)))
     classes = {}
     for l, w in enumerate(shape.windows):
@@ -210,8 +219,7 @@ def run_reference(args, shape):
 def build_states(shape, n_replicas: int, extra_tokens: int, device):
     from paper_2607_24788_b200 import glide
     dt = torch_dtype(shape)
-    wl = synth.Workload(shape.seed, shape.n_layers, shape.batch, shape.n_q_heads, shape.n_kv_heads, shape.head_dim, dt,
-                        value_scale(shape))
+    wl = make_workload(shape)
     max_tokens = shape.context + extra_tokens
     ctxs = [glide.Glide(shape.windows, shape.batch, shape.n_q_heads, shape.n_kv_heads, shape.head_dim, max_tokens,
                         dtype=dt, device=device, prefill_chunk=shape.prefill_chunk, **KERNEL_KNOBS)

@@ -24,7 +24,15 @@
  *     and every q/k/v/out buffer.  The library owns only the small host-side context.
  *   - Every call returns a glide_status code (0 = success).  Arguments are validated
  *     before anything is launched; a failing call changes no state.  Device code never
- *     traps: internal range checks record a code in a status word (glide_device_status).
+ *     traps: internal range checks and bounded waits record a code in a status word
+ *     (glide_device_status).  Once that word is not zero the step that set it may have
+ *     left a unit unfinished (outputs not written, a reduction counter not returned to
+ *     zero): call glide_reset, or glide_import_state for every layer, before the context
+ *     is used again.
+ *   - The host context tracks every layer's position and hands it to each launch, and it
+ *     advances its own bookkeeping per call.  A launch that is recorded once and replayed
+ *     (a CUDA graph) would run again at the recorded position: issue every prefill and
+ *     decode step through these calls.
  *   - Not thread-safe per context; different contexts are independent.
  */
 #ifndef GLIDE_H_
@@ -113,7 +121,11 @@ typedef struct {
  * split-K scratch, work lists, chunk-scan scratch).  Host only, no CUDA calls. */
 int glide_workspace_bytes(const glide_config *cfg, size_t *bytes_out);
 
-/* Build a context over caller-owned device memory `dev_workspace` (>= glide_workspace_bytes,
+/* Set up the per-layer hybrid attention of Sec. III-B (Eq. 7: window softmax over the newest w_l = w - delta_l
+ * tokens of layer l, linear state for the rest; the layer-wise allocation delta_l is the caller's, Sec. III-C) with
+ * the KV cache of Sec. II "KV Cache" reduced to one ring of w_l slots per layer plus the state S, z of Sec. II
+ * "Linearized Attention".
+ * Build a context over caller-owned device memory `dev_workspace` (>= glide_workspace_bytes,
  * 256-byte aligned; a 2 MiB-aligned base is worth about 2 % on the smallest decode steps, because the library
  * places the streamed arrays on 2 MiB multiples of its offsets).  Sets the GQA head mapping and the per-layer windows, uploads the static
  * work lists and zeroes rings' bookkeeping, S and z on `stream`.  The workspace must stay
@@ -133,7 +145,9 @@ int glide_create(const glide_config *cfg, void *dev_workspace, size_t workspace_
 int glide_prefill(glide_ctx *ctx, int32_t layer_begin, int32_t layer_count, int64_t T, const void *dev_q,
                   const void *dev_k, const void *dev_v, void *dev_out, void *stream);
 
-/* Decode stage: one token for every layer and sequence, one fused launch.
+/* Decode stage (Sec. II "KV Cache", decode; Sec. III-B Eq. 7 with its two component equations; the state fold is
+ * Sec. II "Linearized Attention", S_i = S_{i-1} + phi(k_i)^T v_i, z_i = z_{i-1} + phi(k_i)^T): one token for every
+ * layer and sequence, one fused launch.
  *   dev_q, dev_out [L][B][H][d];  dev_k, dev_v [L][B][H_kv][d].
  * Per layer: the token leaving the window (if any) is folded into S,z in place, the window is
  * streamed once for all query heads of a KV head, the linear readout uses the updated state, and
@@ -166,12 +180,14 @@ int glide_decode_step_layers(glide_ctx *ctx, int32_t layer_begin, int32_t layer_
  * every GPU that loads the library holds until the process exits.
  *
  *   - Same arguments, layouts, state updates and error behaviour as glide_decode_step; results agree with it
- *     to the tolerance of the I/O dtype (a different kernel may round differently).
+ *     to the tolerance of the I/O dtype (a different kernel may round differently).  The status word of the
+ *     device-side checks stays in the context's own workspace, as for every other call (glide_device_status);
+ *     only the step's counters, tickets and partial records live in the static buffer.
  *   - Configurations whose scratch (256 + 4 * units + 4 * records bytes, a few KiB per work item) exceeds the
  *     static buffer are refused with GLIDE_ERR_SCRATCH_LIMIT before anything is launched.
  *   - Calls no cudaMalloc / cudaFree and no allocating library routine.  The first call on each device looks
- *     the buffer's device address up once (with that device current): make that first call before any stream
- *     capture begins.
+ *     the buffer's device address up once (with that device current): make that first call outside any stream
+ *     capture.
  *   - All contexts on a device share the one buffer.  It keeps the previous call's contents; the words that
  *     must start at zero are cleared on `stream` at the start of every call.  Two calls whose kernels overlap
  *     on the GPU (different streams) race on it: keep calls of this entry point stream-ordered per device. */
@@ -196,8 +212,9 @@ int glide_reset_seq(glide_ctx *ctx, int32_t b, void *stream);
 int glide_prefill_seq(glide_ctx *ctx, int32_t b, int64_t T, const void *dev_q, const void *dev_k, const void *dev_v,
                       void *dev_out, void *stream);
 
-/* Slot b holds no sequence from now on: decode steps skip it (its rows of q, k, v are not read, its rows of out
- * and its ring, S and z are not written), so an idle slot costs no memory traffic.  glide_reset_seq starts a new
+/* Slot b holds no sequence from now on: decode steps skip it (its rows of q, k, v may be fetched but are not used --
+ * they must stay addressable --, its rows of out and its ring, S and z are not written), so an idle slot costs no
+ * window or state traffic.  glide_reset_seq starts a new
  * sequence in it; glide_prefill_seq and glide_seq_layer_info on a parked slot return GLIDE_ERR_STATE.  May be
  * called between the layer-range calls of a step.  Stream-ordered. */
 int glide_park_seq(glide_ctx *ctx, int32_t b, void *stream);
@@ -205,7 +222,8 @@ int glide_park_seq(glide_ctx *ctx, int32_t b, void *stream);
 /* Tokens slot b holds, as the host tracks them (no device access); -1 for a parked slot. */
 int glide_seq_tokens(glide_ctx *ctx, int32_t b, int64_t *n_out);
 
-/* Free the host context.  Does not touch the workspace. */
+/* Free the host context (the end of a sequence batch's life: the cache of Sec. II "KV Cache" is the caller's
+ * workspace, which this call does not touch). */
 int glide_destroy(glide_ctx *ctx);
 
 /* ---- test / benchmark support -------------------------------------------------------------- */

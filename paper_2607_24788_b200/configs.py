@@ -25,6 +25,7 @@ class GlideShape:
     unit_variance: bool = False   # q,k,v ~ N(0,1) (True) or N(0,1)/sqrt(d)
     prefill_chunk: int = 0
     seed: int = 0
+    value_scales: tuple = None    # (std of q and k entries, std of v entries) when the defaults above are not wanted
 
     @property
     def max_tokens(self) -> int:

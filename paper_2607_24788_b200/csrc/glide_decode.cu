@@ -328,13 +328,16 @@ __global__ void __launch_bounds__(kDecodeThreads) glide_decode_kernel(const Deco
     if (idx >= p.n_items) break;
     const WorkItem it = p.items[idx];
     if (it.layer < 0 || it.layer >= p.L || it.unit < 0) {  // corrupted list: record and skip
-      if (tid == 0) atomicExch(&p.ctl->status, kDevBadItem);
+      if (tid == 0) atomicExch(p.status, kDevBadItem);
       continue;
     }
     if (it.layer < p.layer_begin || it.layer >= p.layer_begin + p.layer_count) continue;   // not a layer of this launch
     const LayerDev ld = p.layers[it.layer];
     const int ub = it.unit - it.layer * units_per_layer;
     const int b = ub / p.Hkv, g = ub - b * p.Hkv;
+    GLIDE_CHECK_OR(ub >= 0 && ub < units_per_layer && it.begin >= 0 && it.count >= 0 &&
+                       it.begin + it.count <= (it.kind == kItemWindow ? ld.cap : int64_t(D)),
+                   p.status, continue);   // (uniform over the CTA: every thread sees the same item)
     const int64_t t = p.n_dev[it.layer] + (p.seq_off ? p.seq_off[b] : 0);   // position of this sequence
     if (t < 0) continue;   // parked slot: nothing is read or written for it (every item of the unit takes this branch)
     const int per_unit = ld.n_win_items + ld.n_state_items;
@@ -390,6 +393,7 @@ DecodeParams make_decode_params(const glide_ctx *ctx, int layer_begin, int layer
   p.items = reinterpret_cast<const WorkItem *>(ctx->ws + ctx->off_items);
   p.heads_of = reinterpret_cast<const int32_t *>(ctx->ws + ctx->off_heads);
   p.ctl = reinterpret_cast<Control *>(ctx->ws + ctx->off_ctl);
+  p.status = &p.ctl->status;
   p.tickets = reinterpret_cast<int32_t *>(ctx->ws + ctx->off_tickets);
   p.partials = reinterpret_cast<float *>(ctx->ws + ctx->off_partials);
   p.n_dev = reinterpret_cast<int64_t *>(ctx->ws + ctx->off_ndev);
@@ -496,7 +500,7 @@ int launch_decode_noalloc(glide_ctx *ctx, const void *q, const void *k, const vo
     return GLIDE_ERR_CUDA;
   }
   DecodeParams p = make_decode_params(ctx, 0, ctx->cfg.n_layers, q, k, v, out);
-  p.ctl = reinterpret_cast<Control *>(scratch);
+  p.ctl = reinterpret_cast<Control *>(scratch);   // counters only: p.status stays the context's own word
   p.tickets = reinterpret_cast<int32_t *>(scratch + tickets_off);
   p.partials = reinterpret_cast<float *>(scratch + partials_off);
   p.rec_floats = ctx->rec_floats;   // this variant always runs the CUDA-core kernel and its record layout

@@ -591,7 +591,7 @@ __global__ void __launch_bounds__(WARPS * 32, 1) glide_decode_mma_kernel(const D
     if (idx >= p.n_items) break;
     const WorkItem it = p.items[idx];
     if (it.layer < 0 || it.layer >= p.L || it.unit < 0) {
-      if (lane == 0) atomicExch(&p.ctl->status, kDevBadItem);
+      if (lane == 0) atomicExch(p.status, kDevBadItem);
       continue;
     }
     if (it.layer < p.layer_begin || it.layer >= p.layer_begin + p.layer_count) continue;   // not a layer of this launch
@@ -606,7 +606,7 @@ __global__ void __launch_bounds__(WARPS * 32, 1) glide_decode_mma_kernel(const D
     if (it.kind == kItemWindow) {
       window_item_mma<D, G, STAGES>(p, tmaps + 3 * it.layer, tmaps + 3 * it.layer + 1, it, ld, t, b, g, rec, pipe, lane);
       if (pipe.failed) {  // a TMA never completed: record it and stop taking work
-        if (lane == 0) atomicExch(&p.ctl->status, kDevWaitTimeout);
+        if (lane == 0) atomicExch(p.status, kDevWaitTimeout);
         break;
       }
     } else {

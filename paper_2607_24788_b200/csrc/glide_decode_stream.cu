@@ -385,6 +385,9 @@ glide_decode_stream_kernel(const DecodeParams p, const StreamParams sp) {
         const StreamSegment &sg = sm_segs[icur.seg];
         const uint32_t bar = my_bars + issue_stage * 8;
         const uint32_t dst = my_stages + issue_stage * kStageBytes;
+        GLIDE_CHECK_OR(icur.k < icur.n_state_eff ? (sg.state0 + icur.k) * kTileRows < kD
+                                                 : (sg.win0 + icur.k - icur.n_state_eff) * kTileRows < sg.cap,
+                       p.status, (void)0);
         if (icur.k < icur.n_state_eff) {
           const int st = sg.state0 + icur.k;
           mbar_expect_tx(bar, kStageBytes + 64);
@@ -1016,7 +1019,7 @@ glide_decode_stream_kernel(const DecodeParams p, const StreamParams sp) {
       GLIDE_TRACE_EVENT(13);
     }
   }
-  if (failed && lane == 0) atomicExch(&p.ctl->status, kDevWaitTimeout);
+  if (failed && lane == 0) atomicExch(p.status, kDevWaitTimeout);
   if (lane == 0) bulk_wait0();   // this warp's state stores have landed
   GLIDE_TRACE_EVENT(9);
 

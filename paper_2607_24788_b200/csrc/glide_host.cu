@@ -5,6 +5,8 @@
 #include <cstring>
 #include <new>
 
+#include <nvtx3/nvToolsExt.h>
+
 #include "glide_internal.h"
 
 using namespace glide;
@@ -20,6 +22,15 @@ using namespace glide;
 #endif
 
 namespace {
+
+// A named range around a call of the library, for timelines of profilers that follow NVTX (a no-op when none is
+// attached: the header-only NVTX loader finds no tool and returns at once).
+struct Range {
+  explicit Range(const char *name) { nvtxRangePushA(name); }
+  ~Range() { nvtxRangePop(); }
+  Range(const Range &) = delete;
+  Range &operator=(const Range &) = delete;
+};
 
 size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
@@ -258,6 +269,7 @@ int glide_workspace_bytes(const glide_config *cfg, size_t *bytes_out) {
 int glide_create(const glide_config *cfg, void *dev_workspace, size_t workspace_bytes, void *stream,
                  glide_ctx **ctx_out) {
   if (!ctx_out) return GLIDE_ERR_INVALID_ARG;
+  Range range("glide_create");
   *ctx_out = nullptr;
   glide_ctx *ctx = new (std::nothrow) glide_ctx;
   if (!ctx) return GLIDE_ERR_INVALID_ARG;
@@ -375,6 +387,7 @@ int set_seq_off(glide_ctx *ctx, int b, int64_t off, cudaStream_t st) {
 int glide_decode_step_layers(glide_ctx *ctx, int32_t layer_begin, int32_t layer_count, const void *q, const void *k,
                              const void *v, void *out, void *stream) {
   if (!ctx || !q || !k || !v || !out) return GLIDE_ERR_INVALID_ARG;
+  Range range("glide_decode_step");
   if (layer_begin < 0 || layer_count < 1 || layer_begin + layer_count > ctx->cfg.n_layers) return GLIDE_ERR_INVALID_ARG;
   if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out)) return GLIDE_ERR_INVALID_ARG;
   for (int l = layer_begin + 1; l < layer_begin + layer_count; ++l)
@@ -393,6 +406,7 @@ int glide_decode_step(glide_ctx *ctx, const void *q, const void *k, const void *
 
 int glide_decode_step_noalloc(glide_ctx *ctx, const void *q, const void *k, const void *v, void *out, void *stream) {
   if (!ctx || !q || !k || !v || !out) return GLIDE_ERR_INVALID_ARG;
+  Range range("glide_decode_step_noalloc");
   if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out)) return GLIDE_ERR_INVALID_ARG;
   const int L = ctx->cfg.n_layers;
   for (int l = 1; l < L; ++l)
@@ -407,6 +421,7 @@ int glide_decode_step_noalloc(glide_ctx *ctx, const void *q, const void *k, cons
 int glide_prefill(glide_ctx *ctx, int32_t layer_begin, int32_t layer_count, int64_t T, const void *q, const void *k,
                   const void *v, void *out, void *stream) {
   if (!ctx || !k || !v || T < 0) return GLIDE_ERR_INVALID_ARG;
+  Range range("glide_prefill");
   if (out && !q) return GLIDE_ERR_INVALID_ARG;
   if (layer_begin < 0 || layer_count < 1 || layer_begin + layer_count > ctx->cfg.n_layers)
     return GLIDE_ERR_INVALID_ARG;
@@ -428,6 +443,7 @@ int glide_prefill(glide_ctx *ctx, int32_t layer_begin, int32_t layer_count, int6
 int glide_prefill_seq(glide_ctx *ctx, int32_t b, int64_t T, const void *q, const void *k, const void *v, void *out,
                       void *stream) {
   if (!ctx || !k || !v || T < 0 || b < 0 || b >= ctx->cfg.batch) return GLIDE_ERR_INVALID_ARG;
+  Range range("glide_prefill_seq");
   if (out && !q) return GLIDE_ERR_INVALID_ARG;
   if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out)) return GLIDE_ERR_INVALID_ARG;
   if (!layers_level(ctx)) return GLIDE_ERR_STATE;

@@ -47,6 +47,20 @@ enum : int { kItemWindow = 0, kItemState = 1 };
 // Device status codes (glide_device_status).
 enum : int { kDevOk = 0, kDevBadSlot = 1, kDevBadItem = 2, kDevWaitTimeout = 3 };
 
+// Range checks of a debug build (-DGLIDE_CHECKS): a ring slot, state row or unit index outside its bounds records
+// kDevBadSlot in the status word and the access is skipped; nothing traps.  Absent from normal builds.
+#ifdef GLIDE_CHECKS
+#define GLIDE_CHECK_OR(cond, status_ptr, action)                 \
+  do {                                                           \
+    if (!(cond)) {                                               \
+      atomicExch((status_ptr), glide::kDevBadSlot);              \
+      action;                                                    \
+    }                                                            \
+  } while (0)
+#else
+#define GLIDE_CHECK_OR(cond, status_ptr, action) do { } while (0)
+#endif
+
 // Control words at the start of the workspace.
 struct Control {
   int32_t work_counter;
@@ -60,7 +74,8 @@ struct DecodeParams {
   const LayerDev *layers;
   const WorkItem *items;
   const int32_t *heads_of;   // [Hkv][G] query heads of each KV head
-  Control *ctl;
+  Control *ctl;              // work and completion counters (the allocation-free step keeps them in the static buffer)
+  int32_t *status;           // the context's status word, in its workspace for every entry point (glide_device_status)
   int32_t *tickets;          // [units]
   float *partials;
   int64_t *n_dev;            // [L]

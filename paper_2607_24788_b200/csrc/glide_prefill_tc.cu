@@ -8,7 +8,7 @@
 //   warp 9      one elected thread issues the TMA loads of the K and V tiles
 // Window part, per 128-key tile t (keys are tokens j0 + 0..127, j0 a multiple of 16):
 //   loader    K_t and V_t as 16-token boxes (ring rows for tokens older than the call, the call's rows otherwise)
-//             into a ring of three 32 KiB buffers, 128-byte swizzle, completion on an mbarrier
+//             into a ring of five 32 KiB buffers (kStages), 128-byte swizzle, completion on an mbarrier
 //   MMA       S_X = Q_X K_t^T into TMEM (8 x m128n128k16), committed to an mbarrier the softmax warps wait on
 //   softmax   tcgen05.ld of the own row, mask, row maximum without any shuffle, P = 2^(s - m_ref) as bf16 into
 //             the swizzled A-operand layout in shared memory; the reference m_ref is lazy: O is rescaled in

@@ -78,13 +78,15 @@ class Workload:
     """Addressable synthetic q/k/v for one configuration."""
 
     def __init__(self, seed: int, n_layers: int, batch: int, H: int, Hkv: int, d: int, dtype: torch.dtype,
-                 scale: float):
+                 scale: float, v_scale: float = None):
+        """scale: standard deviation of the q and k entries (and of v unless v_scale gives its own)."""
         self.seed, self.L, self.B, self.H, self.Hkv, self.d = seed, n_layers, batch, H, Hkv, d
         self.dtype, self.scale = dtype, scale
+        self.v_scale = scale if v_scale is None else v_scale
 
     def _gen(self, tensor, layers, batches, tokens, heads, device):
         return generate(self.seed, tensor, layers, batches, tokens, heads, self.d, n_layers=self.L, batch=self.B,
-                        scale=self.scale, dtype=self.dtype, device=device)
+                        scale=self.v_scale if tensor == V else self.scale, dtype=self.dtype, device=device)
 
     def qkv(self, layers, batches, tokens, device="cpu"):
         """(q [l][b][t][H][d], k [l][b][t][Hkv][d], v likewise)."""

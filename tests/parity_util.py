@@ -12,6 +12,11 @@ from paper_2607_24788_b200 import glide, synth
 
 TOL = {torch.float32: dict(max_abs=1e-4, rel_l2=None), torch.bfloat16: dict(max_abs=2e-2, rel_l2=1e-2)}
 STATE_REL_L2 = 1e-5
+# bf16: the relative-L2 bound also holds for every output row on its own (the d values of one layer, sequence,
+# token and head), so that an error confined to one head, one token or one layer with small outputs cannot hide
+# behind the rest of the tensor.  Rows whose reference norm is below the floor are left to the max-abs bound: a
+# row that small is dominated by the bf16 rounding of outputs near zero, not by the attention arithmetic.
+ROW_NORM_FLOOR = 1e-6
 
 
 def f32_scale(d: int) -> float:
@@ -33,6 +38,14 @@ def check_outputs(got: torch.Tensor, ref: np.ndarray, dtype: torch.dtype, what: 
     if tol["rel_l2"] is not None and g.size:
         rel = np.linalg.norm(g - ref) / max(np.linalg.norm(ref), 1e-30)
         assert rel <= tol["rel_l2"], f"{what}: rel-L2 {rel:.3e} > {tol['rel_l2']}"
+        row_ref = np.linalg.norm(ref, axis=-1)
+        row_err = np.linalg.norm(g - ref, axis=-1)
+        live = row_ref >= ROW_NORM_FLOOR
+        if live.any():
+            row_rel = np.where(live, row_err / np.maximum(row_ref, ROW_NORM_FLOOR), 0.0)
+            worst = np.unravel_index(np.argmax(row_rel), row_rel.shape)
+            assert row_rel[worst] <= tol["rel_l2"], (f"{what}: row {tuple(int(i) for i in worst)} rel-L2 "
+                                                     f"{row_rel[worst]:.3e} > {tol['rel_l2']} (row norm {row_ref[worst]:.3e})")
     return err
 
 

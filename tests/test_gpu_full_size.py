@@ -88,6 +88,14 @@ def test_config1_llama_b1_32k_full_size():
     _check(C.C1, [(0, 0, 0), (3, 0, 7), (5, 0, 2), (11, 0, 5), (12, 0, 1), (23, 0, 6), (24, 0, 0), (31, 0, 7)])
 
 
+def test_config1_shape_with_unit_scale_values():
+    """Config 1's shapes with v ~ N(0,1) and q, k ~ N(0, 16/d): outputs are of order 0.02 .. 0.1 instead of 1e-3, so
+    that the absolute bound of the bf16 tolerance means something at 32K context, and phi is not almost uniform."""
+    from dataclasses import replace
+    shape = replace(C.C1, name="c1_unit_scale_values", value_scales=(4.0 / C.C1.head_dim ** 0.5, 1.0), seed=3)
+    _check(shape, [(1, 0, 4), (7, 0, 0), (15, 0, 3), (28, 0, 6)])
+
+
 def test_config4_mistral_b8_8k_full_size():
     _check(C.C4, [(0, 0, 0), (1, 7, 3), (9, 3, 6), (17, 5, 1), (26, 2, 4), (31, 7, 7)])
 
