@@ -62,8 +62,15 @@ typedef enum { GLIDE_F32 = 0, GLIDE_BF16 = 1 } glide_dtype;
 
 /* Feature map of the linear part.  GLIDE_PHI_SOFTMAX is the paper's default
  * (Sec. III-B): phi(x) = softmax over the head_dim entries of x, no parameters,
- * feature dimension = head_dim. */
-typedef enum { GLIDE_PHI_SOFTMAX = 0 } glide_phi;
+ * feature dimension = head_dim.
+ * GLIDE_PHI_PROJ_SOFTMAX2 is the learned map of the Hedgehog / LoLCATs line that the appendix' "Linear Attention"
+ * lists among the kernels the method accepts (the paper prints no formula for it; this is the library's reading):
+ * with one d x d matrix W per head, y = W^T x (y_j = sum_i x_i W[i][j]),
+ *   phi_W(x) = [ softmax(y) ; softmax(-y) ],   feature dimension 2 * head_dim,
+ * a matrix per layer and query head for the queries (phi_wq) and per layer and KV head for the keys (phi_wk).
+ * S is then [2d][d] and z [2d] per KV head.  It runs on the CUDA-core kernels and, for bf16 I/O with head_dim 128,
+ * the decode step on the streaming kernel (decode_impl AUTO, FMA or STREAM; prefill_impl AUTO or FMA). */
+typedef enum { GLIDE_PHI_SOFTMAX = 0, GLIDE_PHI_PROJ_SOFTMAX2 = 1 } glide_phi;
 
 /* How the window part and the linear part are merged (Sec. III-B "(+)"; appendix
  * "Retention-based SWA").  GLIDE_MERGE_SHARED is the shared normaliser above.  The other two are the appendix'
@@ -106,6 +113,16 @@ typedef struct {
   int32_t decode_state_splits; /* row blocks the S update/readout of one KV head is split into; 0 selects automatically */
   int32_t decode_impl;     /* glide_decode_impl */
   int32_t prefill_impl;    /* glide_prefill_impl */
+  const void *phi_wq;      /* GLIDE_PHI_PROJ_SOFTMAX2: device [n_layers][n_q_heads][d][d] in the I/O dtype, row i column j
+                              = W[i][j]; borrowed, must stay alive and unchanged until glide_destroy.  Else NULL. */
+  const void *phi_wk;      /* likewise [n_layers][n_kv_heads][d][d] for the keys */
+  int32_t gated;           /* 1: gated recurrence (Sec. III-B "GLA-style gating mechanisms"; the paper gives no formula,
+                              the library's reading): every token brings a decay gamma in (0, 1] per KV head, which
+                              waits in the ring with its key and value, and the state decays by the gate of the token
+                              that enters it: S <- gamma S + phi(k) v^T, z <- gamma z + phi(k).  Gates are passed to
+                              glide_prefill_gated / glide_decode_step_gated; the calls without gates use gamma = 1.
+                              Runs on the CUDA-core kernels (decode_impl AUTO or FMA, prefill_impl AUTO or FMA). */
+  int32_t reserved_;       /* must be 0 */
 } glide_config;
 
 typedef struct {
@@ -155,6 +172,15 @@ int glide_prefill(glide_ctx *ctx, int32_t layer_begin, int32_t layer_count, int6
  * All layers must be at the same position (GLIDE_ERR_STATE otherwise). */
 int glide_decode_step(glide_ctx *ctx, const void *dev_q, const void *dev_k, const void *dev_v, void *dev_out,
                       void *stream);
+
+/* glide_prefill and glide_decode_step of a context created with gated = 1 (GLIDE_ERR_INVALID_ARG otherwise), with
+ * the tokens' gates: dev_gate fp32 [layer_count][B][T][H_kv] (prefill) or [L][B][H_kv] (decode), each in (0, 1];
+ * NULL stands for gates of 1.  The gate of a token decays the state at the step the token enters it (Sec. III-B
+ * "GLA-style gating mechanisms", see glide_config.gated). */
+int glide_prefill_gated(glide_ctx *ctx, int32_t layer_begin, int32_t layer_count, int64_t T, const void *dev_q,
+                        const void *dev_k, const void *dev_v, const float *dev_gate, void *dev_out, void *stream);
+int glide_decode_step_gated(glide_ctx *ctx, const void *dev_q, const void *dev_k, const void *dev_v,
+                            const float *dev_gate, void *dev_out, void *stream);
 
 /* The same step for the layers [layer_begin, layer_begin + layer_count) only: what a model needs whose layer l + 1
  * computes its q, k, v from layer l's output (the setting of the paper's experiments, whose "Limitations & Future
@@ -234,7 +260,8 @@ int glide_seq_layer_info(glide_ctx *ctx, int32_t layer, int32_t b, void *stream,
 
 /* Copy one layer's state to caller DEVICE buffers (any may be NULL):
  *   dev_ringK, dev_ringV [B][H_kv][capacity][d] in the I/O dtype (slot order);
- *   dev_S [B][H_kv][d][d] fp32 with S[r][c] = sum phi(k)_r v_c;  dev_z [B][H_kv][d] fp32. */
+ *   dev_S [B][H_kv][D_phi][d] fp32 with S[r][c] = sum phi(k)_r v_c;  dev_z [B][H_kv][D_phi] fp32
+ *   (D_phi = d, or 2d with GLIDE_PHI_PROJ_SOFTMAX2). */
 int glide_export_state(glide_ctx *ctx, int32_t layer, void *dev_ringK, void *dev_ringV, float *dev_S,
                        float *dev_z, void *stream);
 
@@ -242,6 +269,11 @@ int glide_export_state(glide_ctx *ctx, int32_t layer, void *dev_ringK, void *dev
  * as it is) and set the layer's counter to n (0 <= n <= max_tokens; slot offsets stay as they are). */
 int glide_import_state(glide_ctx *ctx, int32_t layer, int64_t n, const void *dev_ringK, const void *dev_ringV,
                        const float *dev_S, const float *dev_z, void *stream);
+
+/* The gates of a gated context's ring, one layer: dev_gates fp32 [B][H_kv][capacity] (slot order), copied out or in
+ * like the ring rows above (glide_import_gates leaves the counter alone: call it beside glide_import_state). */
+int glide_export_gates(glide_ctx *ctx, int32_t layer, float *dev_gates, void *stream);
+int glide_import_gates(glide_ctx *ctx, int32_t layer, const float *dev_gates, void *stream);
 
 /* Back to the empty state: counters, slot offsets, S and z zeroed (rings need no clearing). */
 int glide_reset(glide_ctx *ctx, void *stream);

@@ -22,17 +22,17 @@ namespace {
 
 template <int D, int G>
 constexpr int scratch_floats() {
-  // window items: [warps][G][D+2]; state items: [row groups][G][D]
+  // window items: [warps][G][D+2]; state items: [row groups][G][D]; feature kernel: [D] + reductions
   constexpr int NW = kDecodeThreads / 32;
   constexpr int RPI = kDecodeThreads / (D / 4);
   return (NW * G * (D + 2) > RPI * G * D) ? NW * G * (D + 2) : RPI * G * D;
 }
 
-template <typename T, int D, int G>
+template <typename T, int D, int G, int DP = D>
 struct DecodeSmem {
   float scratch[scratch_floats<D, G>()];
-  float phiq[G][D];
-  float phik[D];
+  float phiq[G][DP];
+  float phik[DP];
   float ve[D];
   float scur[G];
   float M[G];
@@ -43,9 +43,9 @@ struct DecodeSmem {
 };
 
 // ---- window item ---------------------------------------------------------------------------
-template <typename T, int D, int G>
+template <typename T, int D, int G, int DP>
 __device__ __forceinline__ void window_item(const DecodeParams &p, const WorkItem &it, const LayerDev &ld,
-                                            int64_t t, int b, int g, float *rec, DecodeSmem<T, D, G> &sm) {
+                                            int64_t t, int b, int g, float *rec, DecodeSmem<T, D, G, DP> &sm) {
   constexpr int E = D / 32;
   constexpr int NW = kDecodeThreads / 32;
   constexpr int U = 4;
@@ -127,9 +127,12 @@ __device__ __forceinline__ void window_item(const DecodeParams &p, const WorkIte
 }
 
 // ---- state item ----------------------------------------------------------------------------
-template <typename T, int D, int G>
+// DP: the feature dimension (rows of S): D for the parameter-free map, 2 D for the learned map, whose phi(k_e) and
+// phi(q_h) were written by the feature kernel in front of this launch (p.phit).  A gated context decays the rows by
+// the gate of the token that enters the state.
+template <typename T, int D, int G, int DP>
 __device__ __forceinline__ void state_item(const DecodeParams &p, const WorkItem &it, const LayerDev &ld, int64_t t,
-                                           int b, int g, float *rec, DecodeSmem<T, D, G> &sm) {
+                                           int b, int g, float *rec, DecodeSmem<T, D, G, DP> &sm) {
   constexpr int E = D / 32;
   constexpr int NW = kDecodeThreads / 32;
   constexpr int TPR = D / 4;                   // threads per state row (float4 each)
@@ -138,38 +141,52 @@ __device__ __forceinline__ void state_item(const DecodeParams &p, const WorkItem
   if (t < ld.wlin) return;                     // nothing has reached the state yet: S,z are still zero
   const int ub = b * p.Hkv + g;
   const T *ke, *ve;
+  float gamma = 1.f;                           // gate of the token that enters the state
   if (ld.wlin == 0) {  // no ring, or a state that holds every token: the current token is folded now
     ke = reinterpret_cast<const T *>(p.k) + size_t(it.unit) * D;
     ve = reinterpret_cast<const T *>(p.v) + size_t(it.unit) * D;
+    if (p.gated && p.gate) gamma = p.gate[it.unit];
   } else {          // slot t mod cap holds token t - w
-    const size_t row = (size_t(ub) * size_t(ld.cap) + size_t(t % ld.cap)) * D;
-    ke = reinterpret_cast<const T *>(p.ws + ld.ringK) + row;
-    ve = reinterpret_cast<const T *>(p.ws + ld.ringV) + row;
+    const size_t slot = size_t(ub) * size_t(ld.cap) + size_t(t % ld.cap);
+    ke = reinterpret_cast<const T *>(p.ws + ld.ringK) + slot * D;
+    ve = reinterpret_cast<const T *>(p.ws + ld.ringV) + slot * D;
+    if (p.gated) gamma = reinterpret_cast<const float *>(p.ws + ld.ringG)[slot];
   }
-  if (warp == 0) {
-    float x[E], y[E];
-    load_elems<T, E>(ke + lane * E, x);
-    load_elems<T, E>(ve + lane * E, y);
-    warp_phi<E>(x);
+  const int r_end = it.begin + it.count;
+  if constexpr (DP == D) {
+    if (warp == 0) {
+      float x[E], y[E];
+      load_elems<T, E>(ke + lane * E, x);
+      load_elems<T, E>(ve + lane * E, y);
+      warp_phi<E>(x);
 #pragma unroll
-    for (int i = 0; i < E; ++i) {
-      sm.phik[lane * E + i] = x[i];
-      sm.ve[lane * E + i] = y[i];
+      for (int i = 0; i < E; ++i) {
+        sm.phik[lane * E + i] = x[i];
+        sm.ve[lane * E + i] = y[i];
+      }
     }
-  }
-  for (int h = warp; h < G; h += NW) {
-    const int head = p.heads_of[g * G + h];
-    float x[E];
-    load_elems<T, E>(reinterpret_cast<const T *>(p.q) + ((size_t(it.layer) * p.B + b) * p.H + head) * D + lane * E, x);
-    warp_phi<E>(x);
+    for (int h = warp; h < G; h += NW) {
+      const int head = p.heads_of[g * G + h];
+      float x[E];
+      load_elems<T, E>(reinterpret_cast<const T *>(p.q) + ((size_t(it.layer) * p.B + b) * p.H + head) * D + lane * E, x);
+      warp_phi<E>(x);
 #pragma unroll
-    for (int i = 0; i < E; ++i) sm.phiq[h][lane * E + i] = x[i];
+      for (int i = 0; i < E; ++i) sm.phiq[h][lane * E + i] = x[i];
+    }
+  } else {
+    // the rows of this item from the feature kernel's output: [unit][DP / 16][G + 1][16]
+    const float *ph = p.phit + size_t(it.unit - p.layer_begin * p.B * p.Hkv) * DP * (G + 1);
+    for (int idx = tid; idx < (G + 1) * it.count; idx += kDecodeThreads) {
+      const int h = idx / it.count, r = it.begin + idx % it.count;
+      const float val = ph[(size_t(r >> 4) * (G + 1) + h) * 16 + (r & 15)];
+      if (h < G) sm.phiq[h][r] = val; else sm.phik[r] = val;
+    }
+    for (int c = tid; c < D; c += kDecodeThreads) sm.ve[c] = to_f32(ve[c]);
   }
   __syncthreads();
 
   const int c4 = tid % TPR, rsub = tid / TPR;
-  const int r_end = it.begin + it.count;
-  float *Sb = reinterpret_cast<float *>(p.ws + ld.S) + size_t(ub) * D * D;
+  float *Sb = reinterpret_cast<float *>(p.ws + ld.S) + size_t(ub) * DP * D;
   const float4 v4 = *reinterpret_cast<const float4 *>(&sm.ve[c4 * 4]);
   float4 a[G];
 #pragma unroll
@@ -179,10 +196,10 @@ __device__ __forceinline__ void state_item(const DecodeParams &p, const WorkItem
     float4 *sp = reinterpret_cast<float4 *>(Sb + size_t(r) * D + c4 * 4);
     float4 s = *sp;
     const float pk = sm.phik[r];
-    s.x = fmaf(pk, v4.x, s.x);
-    s.y = fmaf(pk, v4.y, s.y);
-    s.z = fmaf(pk, v4.z, s.z);
-    s.w = fmaf(pk, v4.w, s.w);
+    s.x = fmaf(pk, v4.x, gamma * s.x);
+    s.y = fmaf(pk, v4.y, gamma * s.y);
+    s.z = fmaf(pk, v4.z, gamma * s.z);
+    s.w = fmaf(pk, v4.w, gamma * s.w);
     *sp = s;
 #pragma unroll
     for (int h = 0; h < G; ++h) {
@@ -195,12 +212,12 @@ __device__ __forceinline__ void state_item(const DecodeParams &p, const WorkItem
   }
   // z rows of this block and the b_h readout: warp 0
   if (warp == 0) {
-    float *zb = reinterpret_cast<float *>(p.ws + ld.z) + size_t(ub) * D;
+    float *zb = reinterpret_cast<float *>(p.ws + ld.z) + size_t(ub) * DP;
     float bp[G];
 #pragma unroll
     for (int h = 0; h < G; ++h) bp[h] = 0.f;
     for (int r = it.begin + lane; r < r_end; r += 32) {
-      const float zn = zb[r] + sm.phik[r];
+      const float zn = fmaf(gamma, zb[r], sm.phik[r]);
       zb[r] = zn;
 #pragma unroll
       for (int h = 0; h < G; ++h) bp[h] = fmaf(sm.phiq[h][r], zn, bp[h]);
@@ -227,9 +244,9 @@ __device__ __forceinline__ void state_item(const DecodeParams &p, const WorkItem
 }
 
 // ---- merge (last ticket of a unit) -----------------------------------------------------------
-template <typename T, int D, int G>
+template <typename T, int D, int G, int DP>
 __device__ __forceinline__ void merge_unit(const DecodeParams &p, const WorkItem &it, const LayerDev &ld, int64_t t,
-                                           int b, int g, DecodeSmem<T, D, G> &sm) {
+                                           int b, int g, DecodeSmem<T, D, G, DP> &sm) {
   constexpr int E = D / 32;
   constexpr int NW = kDecodeThreads / 32;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -312,12 +329,15 @@ __device__ __forceinline__ void merge_unit(const DecodeParams &p, const WorkItem
       Kd[c] = kt[c];
       Vd[c] = vt[c];
     }
+    if (p.gated && tid == 0)   // the token's gate waits in the ring with it
+      reinterpret_cast<float *>(p.ws + ld.ringG)[size_t(ub) * size_t(ld.cap) + size_t(t % ld.cap)] =
+          p.gate ? p.gate[it.unit] : 1.f;
   }
 }
 
-template <typename T, int D, int G>
+template <typename T, int D, int G, int DP>
 __global__ void __launch_bounds__(kDecodeThreads) glide_decode_kernel(const DecodeParams p) {
-  __shared__ DecodeSmem<T, D, G> sm;
+  __shared__ DecodeSmem<T, D, G, DP> sm;
   const int tid = threadIdx.x;
   const int units_per_layer = p.B * p.Hkv;
   for (;;) {
@@ -336,23 +356,23 @@ __global__ void __launch_bounds__(kDecodeThreads) glide_decode_kernel(const Deco
     const int ub = it.unit - it.layer * units_per_layer;
     const int b = ub / p.Hkv, g = ub - b * p.Hkv;
     GLIDE_CHECK_OR(ub >= 0 && ub < units_per_layer && it.begin >= 0 && it.count >= 0 &&
-                       it.begin + it.count <= (it.kind == kItemWindow ? ld.cap : int64_t(D)),
+                       it.begin + it.count <= (it.kind == kItemWindow ? ld.cap : int64_t(DP)),
                    p.status, continue);   // (uniform over the CTA: every thread sees the same item)
     const int64_t t = p.n_dev[it.layer] + (p.seq_off ? p.seq_off[b] : 0);   // position of this sequence
     if (t < 0) continue;   // parked slot: nothing is read or written for it (every item of the unit takes this branch)
     const int per_unit = ld.n_win_items + ld.n_state_items;
     float *rec = p.partials + ld.part_base + (size_t(ub) * per_unit + it.part) * p.rec_floats;
     if (it.kind == kItemWindow)
-      window_item<T, D, G>(p, it, ld, t, b, g, rec, sm);
+      window_item<T, D, G, DP>(p, it, ld, t, b, g, rec, sm);
     else
-      state_item<T, D, G>(p, it, ld, t, b, g, rec, sm);
+      state_item<T, D, G, DP>(p, it, ld, t, b, g, rec, sm);
     __threadfence();
     __syncthreads();
     if (tid == 0) sm.last = atomicAdd(&p.tickets[it.unit], 1) == per_unit - 1;
     __syncthreads();
     if (sm.last) {
       __threadfence();
-      merge_unit<T, D, G>(p, it, ld, t, b, g, sm);
+      merge_unit<T, D, G, DP>(p, it, ld, t, b, g, sm);
       if (tid == 0) p.tickets[it.unit] = 0;
     }
   }
@@ -364,6 +384,113 @@ __global__ void __launch_bounds__(kDecodeThreads) glide_decode_kernel(const Deco
       p.ctl->done_counter = 0;
       for (int l = 0; l < p.layer_count; ++l) p.n_dev[p.layer_begin + l] += 1;
       __threadfence();
+    }
+  }
+}
+
+// ---- learned feature map of one decode step ------------------------------------------------------
+// phi_W(x) = [softmax(W^T x); softmax(-W^T x)] of the step's queries and of the key that enters the state, for every
+// unit of the launch, into p.phit [unit][DP / 16][G + 1][16] (row G: the key).  One CTA of D threads per (layer, KV
+// head, row of the group): thread j owns output j; the d x d matrix of the head is read once, coalesced over j, for
+// all sequences of the batch (kPhiSeqs at a time in registers).
+constexpr int kPhiSeqs = 8;
+template <typename T, int D, int G>
+__global__ void __launch_bounds__(D) glide_decode_phi_kernel(const DecodeParams p) {
+  constexpr int DP = 2 * D;
+  __shared__ float sx[kPhiSeqs][D];
+  __shared__ float red[kPhiSeqs][2][D / 32];
+  const int j = threadIdx.x, warp = j >> 5, lane = j & 31;
+  const int row = blockIdx.x % (G + 1);
+  const int g = (blockIdx.x / (G + 1)) % p.Hkv;
+  const int lrel = blockIdx.x / ((G + 1) * p.Hkv);
+  const int layer = p.layer_begin + lrel;
+  const LayerDev ld = p.layers[layer];
+  if (row == G && !ld.evicts) return;
+  const int head = row < G ? p.heads_of[g * G + row] : 0;
+  const T *W = row < G ? reinterpret_cast<const T *>(p.wq) + (size_t(layer) * p.H + head) * D * D
+                       : reinterpret_cast<const T *>(p.wk) + (size_t(layer) * p.Hkv + g) * D * D;
+  for (int b0 = 0; b0 < p.B; b0 += kPhiSeqs) {
+    const int nb = min(kPhiSeqs, p.B - b0);
+    bool live[kPhiSeqs];
+    __syncthreads();
+#pragma unroll
+    for (int bi = 0; bi < kPhiSeqs; ++bi) {
+      live[bi] = false;
+      if (bi >= nb) continue;
+      const int b = b0 + bi;
+      const int64_t t = p.n_dev[layer] + (p.seq_off ? p.seq_off[b] : 0);
+      if (t < 0) continue;   // parked slot
+      const int ub = b * p.Hkv + g;
+      const T *x;
+      // the per-item kernels index q, k, v with the absolute layer (their base pointers are moved back)
+      const int lq = p.tensors_absolute ? layer : lrel;
+      if (row < G) {
+        x = reinterpret_cast<const T *>(p.q) + ((size_t(lq) * p.B + b) * p.H + head) * D;
+      } else if (t < ld.wlin) {
+        continue;            // nothing enters the state at this step
+      } else if (ld.wlin == 0) {
+        x = reinterpret_cast<const T *>(p.k) + (size_t(lq) * p.B * p.Hkv + ub) * D;
+      } else {
+        x = reinterpret_cast<const T *>(p.ws + ld.ringK) + (size_t(ub) * size_t(ld.cap) + size_t(t % ld.cap)) * D;
+      }
+      live[bi] = true;
+      sx[bi][j] = to_f32(x[j]);
+    }
+    __syncthreads();
+    float y[kPhiSeqs];
+#pragma unroll
+    for (int bi = 0; bi < kPhiSeqs; ++bi) y[bi] = 0.f;
+#pragma unroll 8
+    for (int i = 0; i < D; ++i) {
+      const float w = to_f32(W[size_t(i) * D + j]);
+#pragma unroll
+      for (int bi = 0; bi < kPhiSeqs; ++bi) y[bi] = fmaf(sx[bi][i], w, y[bi]);
+    }
+    // the two softmax halves over the D outputs: maxima of y and -y, then the sums
+    float e0[kPhiSeqs], e1[kPhiSeqs];
+#pragma unroll
+    for (int bi = 0; bi < kPhiSeqs; ++bi) {
+      const float mx = warp_max(y[bi]), mn = warp_max(-y[bi]);
+      if (lane == 0) {
+        red[bi][0][warp] = mx;
+        red[bi][1][warp] = mn;
+      }
+    }
+    __syncthreads();
+#pragma unroll
+    for (int bi = 0; bi < kPhiSeqs; ++bi) {
+      float mx = red[bi][0][0], mn = red[bi][1][0];
+#pragma unroll
+      for (int w = 1; w < D / 32; ++w) {
+        mx = fmaxf(mx, red[bi][0][w]);
+        mn = fmaxf(mn, red[bi][1][w]);
+      }
+      e0[bi] = exp2f((y[bi] - mx) * kLog2e);
+      e1[bi] = exp2f((-y[bi] - mn) * kLog2e);
+    }
+    __syncthreads();
+#pragma unroll
+    for (int bi = 0; bi < kPhiSeqs; ++bi) {
+      const float s0 = warp_sum(e0[bi]), s1 = warp_sum(e1[bi]);
+      if (lane == 0) {
+        red[bi][0][warp] = s0;
+        red[bi][1][warp] = s1;
+      }
+    }
+    __syncthreads();
+#pragma unroll
+    for (int bi = 0; bi < kPhiSeqs; ++bi) {
+      if (!live[bi]) continue;
+      float s0 = 0.f, s1 = 0.f;
+#pragma unroll
+      for (int w = 0; w < D / 32; ++w) {
+        s0 += red[bi][0][w];
+        s1 += red[bi][1][w];
+      }
+      const size_t unit = (size_t(lrel) * p.B + (b0 + bi)) * p.Hkv + g;
+      float *ph = p.phit + unit * DP * (G + 1);
+      ph[(size_t(j >> 4) * (G + 1) + row) * 16 + (j & 15)] = e0[bi] / s0;
+      ph[(size_t((D + j) >> 4) * (G + 1) + row) * 16 + (j & 15)] = e1[bi] / s1;
     }
   }
 }
@@ -398,6 +525,13 @@ DecodeParams make_decode_params(const glide_ctx *ctx, int layer_begin, int layer
   p.partials = reinterpret_cast<float *>(ctx->ws + ctx->off_partials);
   p.n_dev = reinterpret_cast<int64_t *>(ctx->ws + ctx->off_ndev);
   p.seq_off = ctx->ragged ? reinterpret_cast<const int64_t *>(ctx->ws + ctx->off_seqoff) : nullptr;
+  p.phit = ctx->cfg.phi == GLIDE_PHI_PROJ_SOFTMAX2 ? reinterpret_cast<float *>(ctx->ws + ctx->off_phit) : nullptr;
+  p.wq = ctx->cfg.phi_wq;
+  p.wk = ctx->cfg.phi_wk;
+  p.dp = ctx->dp;
+  p.gated = ctx->cfg.gated;
+  p.gate = nullptr;
+  p.tensors_absolute = ctx->decode_kind != 2;
   p.q = q;
   p.k = k;
   p.v = v;
@@ -415,11 +549,23 @@ DecodeParams make_decode_params(const glide_ctx *ctx, int layer_begin, int layer
   return p;
 }
 
-int decode_occupancy(const glide_ctx *ctx, int *blocks_per_sm) {
+namespace {
+// f(TypeTag<T>, IntTag<D>, IntTag<G>, IntTag<DP>) for the configured dtype, head_dim, group size and feature dimension
+template <typename F>
+int dispatch_decode(const glide_ctx *ctx, F &&f) {
   return dispatch_config(ctx->cfg.io_dtype, ctx->cfg.head_dim, ctx->G, [&](auto tt, auto dd, auto gg) -> int {
+    constexpr int D = decltype(dd)::value;
+    if (ctx->dp == D) return f(tt, dd, gg, IntTag<D>{});
+    return f(tt, dd, gg, IntTag<2 * D>{});
+  });
+}
+}  // namespace
+
+int decode_occupancy(const glide_ctx *ctx, int *blocks_per_sm) {
+  return dispatch_decode(ctx, [&](auto tt, auto dd, auto gg, auto pp) -> int {
     using T = typename decltype(tt)::type;
-    constexpr int D = decltype(dd)::value, G = decltype(gg)::value;
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(blocks_per_sm, glide_decode_kernel<T, D, G>, kDecodeThreads,
+    constexpr int D = decltype(dd)::value, G = decltype(gg)::value, DP = decltype(pp)::value;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(blocks_per_sm, glide_decode_kernel<T, D, G, DP>, kDecodeThreads,
                                                       0) != cudaSuccess) {
       cudaGetLastError();
       return GLIDE_ERR_CUDA;
@@ -428,8 +574,21 @@ int decode_occupancy(const glide_ctx *ctx, int *blocks_per_sm) {
   });
 }
 
-int launch_decode(glide_ctx *ctx, int layer_begin, int layer_count, const void *q, const void *k, const void *v, void *out,
-                  cudaStream_t stream) {
+// the step's learned features, in front of the decode kernel of the same layers
+int launch_decode_phi(glide_ctx *ctx, const DecodeParams &p, cudaStream_t stream) {
+  if (ctx->cfg.phi != GLIDE_PHI_PROJ_SOFTMAX2) return GLIDE_OK;
+  return dispatch_config(ctx->cfg.io_dtype, ctx->cfg.head_dim, ctx->G, [&](auto tt, auto dd, auto gg) -> int {
+    using T = typename decltype(tt)::type;
+    constexpr int D = decltype(dd)::value, G = decltype(gg)::value;
+    const unsigned grid = unsigned(p.layer_count) * unsigned(p.Hkv) * unsigned(G + 1);
+    glide_decode_phi_kernel<T, D, G><<<grid, D, 0, stream>>>(p);
+    if (cudaGetLastError() != cudaSuccess) return GLIDE_ERR_CUDA;
+    return GLIDE_OK;
+  });
+}
+
+int launch_decode(glide_ctx *ctx, int layer_begin, int layer_count, const void *q, const void *k, const void *v,
+                  const float *gate, void *out, cudaStream_t stream) {
   const int L = ctx->cfg.n_layers;
   if (ctx->decode_kind == 2 && layer_count != L) {
     // the streaming kernel has a schedule for the whole stack and one per layer: a partial range is one launch per layer
@@ -440,18 +599,23 @@ int launch_decode(glide_ctx *ctx, int layer_begin, int layer_count, const void *
                                                  static_cast<const unsigned char *>(k) + krow * i,
                                                  static_cast<const unsigned char *>(v) + krow * i,
                                                  static_cast<unsigned char *>(out) + qrow * i);
-      const int rc = launch_decode_stream(ctx, pl, 1 + layer_begin + i, stream);
+      int rc = launch_decode_phi(ctx, pl, stream);
+      if (rc) return rc;
+      rc = launch_decode_stream(ctx, pl, 1 + layer_begin + i, stream);
       if (rc) return rc;
     }
     return GLIDE_OK;
   }
-  const DecodeParams p = make_decode_params(ctx, layer_begin, layer_count, q, k, v, out);
+  DecodeParams p = make_decode_params(ctx, layer_begin, layer_count, q, k, v, out);
+  p.gate = gate;
+  const int rc = launch_decode_phi(ctx, p, stream);
+  if (rc) return rc;
   if (ctx->decode_kind == 2) return launch_decode_stream(ctx, p, 0, stream);
   if (ctx->decode_kind == 1) return launch_decode_mma(ctx, p, stream);
-  return dispatch_config(ctx->cfg.io_dtype, ctx->cfg.head_dim, ctx->G, [&](auto tt, auto dd, auto gg) -> int {
+  return dispatch_decode(ctx, [&](auto tt, auto dd, auto gg, auto pp) -> int {
     using T = typename decltype(tt)::type;
-    constexpr int D = decltype(dd)::value, G = decltype(gg)::value;
-    glide_decode_kernel<T, D, G><<<ctx->decode_grid, kDecodeThreads, 0, stream>>>(p);
+    constexpr int D = decltype(dd)::value, G = decltype(gg)::value, DP = decltype(pp)::value;
+    glide_decode_kernel<T, D, G, DP><<<ctx->decode_grid, kDecodeThreads, 0, stream>>>(p);
     if (cudaGetLastError() != cudaSuccess) return GLIDE_ERR_CUDA;
     return GLIDE_OK;
   });
@@ -504,10 +668,13 @@ int launch_decode_noalloc(glide_ctx *ctx, const void *q, const void *k, const vo
   p.tickets = reinterpret_cast<int32_t *>(scratch + tickets_off);
   p.partials = reinterpret_cast<float *>(scratch + partials_off);
   p.rec_floats = ctx->rec_floats;   // this variant always runs the CUDA-core kernel and its record layout
-  return dispatch_config(ctx->cfg.io_dtype, ctx->cfg.head_dim, ctx->G, [&](auto tt, auto dd, auto gg) -> int {
+  p.tensors_absolute = 1;
+  const int rc = launch_decode_phi(ctx, p, stream);
+  if (rc) return rc;
+  return dispatch_decode(ctx, [&](auto tt, auto dd, auto gg, auto pp) -> int {
     using T = typename decltype(tt)::type;
-    constexpr int D = decltype(dd)::value, G = decltype(gg)::value;
-    glide_decode_kernel<T, D, G><<<ctx->noalloc_grid, kDecodeThreads, 0, stream>>>(p);
+    constexpr int D = decltype(dd)::value, G = decltype(gg)::value, DP = decltype(pp)::value;
+    glide_decode_kernel<T, D, G, DP><<<ctx->noalloc_grid, kDecodeThreads, 0, stream>>>(p);
     if (cudaGetLastError() != cudaSuccess) return GLIDE_ERR_CUDA;
     return GLIDE_OK;
   });

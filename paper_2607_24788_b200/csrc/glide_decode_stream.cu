@@ -1284,7 +1284,7 @@ void build_stream_schedule(const glide_ctx *ctx, int layer_begin, int layer_coun
 }
 
 int stream_decode_supported(const glide_ctx *ctx) {
-  return ctx->cfg.io_dtype == GLIDE_BF16 && ctx->cfg.head_dim == kD;
+  return ctx->cfg.io_dtype == GLIDE_BF16 && ctx->cfg.head_dim == kD && ctx->cfg.phi == GLIDE_PHI_SOFTMAX && !ctx->cfg.gated;
 }
 
 // Host-only part of the set-up: every schedule of the context for a device with n_ctas SMs and smem_limit bytes of

@@ -56,7 +56,21 @@ int validate_config(const glide_config *c) {
     return GLIDE_ERR_UNSUPPORTED;
   for (int l = 0; l < c->n_layers; ++l)
     if (c->windows[l] < 0) return GLIDE_ERR_INVALID_ARG;
-  if (c->phi != GLIDE_PHI_SOFTMAX) return GLIDE_ERR_UNSUPPORTED;
+  if (c->phi != GLIDE_PHI_SOFTMAX && c->phi != GLIDE_PHI_PROJ_SOFTMAX2) return GLIDE_ERR_INVALID_ARG;
+  if (c->gated != 0 && c->gated != 1) return GLIDE_ERR_INVALID_ARG;
+  if (c->reserved_ != 0) return GLIDE_ERR_INVALID_ARG;
+  if (c->phi == GLIDE_PHI_PROJ_SOFTMAX2) {
+    if (!c->phi_wq || !c->phi_wk || !aligned16(c->phi_wq) || !aligned16(c->phi_wk)) return GLIDE_ERR_INVALID_ARG;
+    // the learned map runs on the CUDA-core kernels and on the streaming decode kernel
+    if (c->decode_impl == GLIDE_DECODE_MMA) return GLIDE_ERR_UNSUPPORTED;
+    if (c->prefill_impl == GLIDE_PREFILL_MMA_SYNC || c->prefill_impl == GLIDE_PREFILL_TCGEN05) return GLIDE_ERR_UNSUPPORTED;
+  } else if (c->phi_wq || c->phi_wk) {
+    return GLIDE_ERR_INVALID_ARG;
+  }
+  if (c->gated) {   // the gated recurrence runs on the CUDA-core kernels
+    if (c->decode_impl == GLIDE_DECODE_MMA || c->decode_impl == GLIDE_DECODE_STREAM) return GLIDE_ERR_UNSUPPORTED;
+    if (c->prefill_impl == GLIDE_PREFILL_MMA_SYNC || c->prefill_impl == GLIDE_PREFILL_TCGEN05) return GLIDE_ERR_UNSUPPORTED;
+  }
   if (c->merge < GLIDE_MERGE_SHARED || c->merge > GLIDE_MERGE_SUM_ALL) return GLIDE_ERR_INVALID_ARG;
   if (c->merge != GLIDE_MERGE_SHARED &&
       (c->decode_impl == GLIDE_DECODE_MMA || c->prefill_impl == GLIDE_PREFILL_MMA_SYNC))
@@ -88,6 +102,7 @@ int glide::plan_context(const glide_config *cfg, glide_ctx *ctx, std::vector<Wor
   ctx->cfg = *cfg;
   const int L = cfg->n_layers, B = cfg->batch, H = cfg->n_q_heads, Hkv = cfg->n_kv_heads, d = cfg->head_dim;
   ctx->G = H / Hkv;
+  ctx->dp = cfg->phi == GLIDE_PHI_PROJ_SOFTMAX2 ? 2 * d : d;
   ctx->elem = cfg->io_dtype == GLIDE_F32 ? 4 : 2;
   ctx->scale = cfg->softmax_scale > 0.f ? cfg->softmax_scale : 1.0f / std::sqrt(float(d));
   ctx->prefill_chunk = cfg->prefill_chunk ? cfg->prefill_chunk : 256;
@@ -104,6 +119,7 @@ int glide::plan_context(const glide_config *cfg, glide_ctx *ctx, std::vector<Wor
   }
   ctx->cfg.windows = nullptr;
   ctx->cfg.q_to_kv = nullptr;
+  const int dp = ctx->dp;
   ctx->n_host.assign(L, 0);
   ctx->seq_off.assign(size_t(cfg->batch), 0);
   ctx->parked.assign(size_t(cfg->batch), 0);
@@ -113,7 +129,7 @@ int glide::plan_context(const glide_config *cfg, glide_ctx *ctx, std::vector<Wor
   // window slots per split-K item: fixed by the caller, or 128 (512 for very long windows, to bound the
   // number of partials one merge has to read)
   auto chunk_of = [&](int64_t cap) -> int { return cfg->decode_chunk ? cfg->decode_chunk : (cap > 8192 ? 512 : 128); };
-  const int splits = cfg->decode_state_splits ? std::min<int>(cfg->decode_state_splits, d) : (d == 128 ? 4 : 2);
+  const int splits = (cfg->decode_state_splits ? std::min<int>(cfg->decode_state_splits, d) : (d == 128 ? 4 : 2)) * (dp / d);
   const int64_t units_per_layer = int64_t(B) * Hkv;
 
   if (int64_t(L) * units_per_layer > (int64_t(1) << 30)) return GLIDE_ERR_UNSUPPORTED;   // unit indices are 32-bit
@@ -168,10 +184,15 @@ int glide::plan_context(const glide_config *cfg, glide_ctx *ctx, std::vector<Wor
   ctx->off_tmaps = off;
   off = align_up(off + size_t(128) * 5 * L, 256);   // per layer 3 maps of 16-row boxes, then (from 3 L on) 2 of 128-row boxes
   ctx->off_phik = off;
-  off = align_up(off + sizeof(float) * size_t(L) * units_per_layer * ctx->prefill_chunk * d, 256);
+  off = align_up(off + sizeof(float) * size_t(L) * units_per_layer * ctx->prefill_chunk * dp, 256);
   ctx->off_zcum = off;   // running sums of phi(K') over the chunk: only the sum-of-terms merges use them
   if (cfg->merge != GLIDE_MERGE_SHARED)
-    off = align_up(off + sizeof(float) * size_t(L) * units_per_layer * ctx->prefill_chunk * d, 256);
+    off = align_up(off + sizeof(float) * size_t(L) * units_per_layer * ctx->prefill_chunk * dp, 256);
+  ctx->off_phit = off;   // learned feature map: phi(q_h), phi(k_e) of one decode step
+  if (cfg->phi == GLIDE_PHI_PROJ_SOFTMAX2)
+    off = align_up(off + sizeof(float) * size_t(L) * units_per_layer * dp * (ctx->G + 1), 256);
+  ctx->off_gcum = off;   // gated: running sums of log(gate) over the chunk's delayed tokens
+  if (cfg->gated) off = align_up(off + sizeof(float) * size_t(L) * units_per_layer * ctx->prefill_chunk, 256);
   ctx->off_seqoff = off;   // per-sequence position offsets
   off = align_up(off + sizeof(int64_t) * size_t(cfg->batch), 256);
   // the streamed arrays start on a 2 MiB boundary of the workspace whatever the sizes of the small tables before
@@ -180,11 +201,11 @@ int glide::plan_context(const glide_config *cfg, glide_ctx *ctx, std::vector<Wor
   ctx->off_state = off;
   for (int l = 0; l < L; ++l) {
     ctx->layers[l].S = off;
-    off += sizeof(float) * size_t(units_per_layer) * d * d;
+    off += sizeof(float) * size_t(units_per_layer) * dp * d;
   }
   for (int l = 0; l < L; ++l) {
     ctx->layers[l].z = off;
-    off += sizeof(float) * size_t(units_per_layer) * d;
+    off += sizeof(float) * size_t(units_per_layer) * dp;
   }
   ctx->state_bytes = off - ctx->off_state;
   off = align_up(off, 256);
@@ -204,6 +225,11 @@ int glide::plan_context(const glide_config *cfg, glide_ctx *ctx, std::vector<Wor
     ctx->layers[l].ringV = off;
     off += bytes;
   }
+  if (cfg->gated)
+    for (int l = 0; l < L; ++l) {
+      ctx->layers[l].ringG = off;
+      off += align_up(sizeof(float) * size_t(units_per_layer) * size_t(ctx->layers[l].cap), 256);
+    }
   ctx->total = align_up(off, 256);
 
   if (items) {
@@ -231,7 +257,7 @@ int glide::plan_context(const glide_config *cfg, glide_ctx *ctx, std::vector<Wor
           it.layer = l;
           it.kind = kItemState;
           it.part = part++;
-          int r0 = int(int64_t(d) * i / ld.n_state_items), r1 = int(int64_t(d) * (i + 1) / ld.n_state_items);
+          int r0 = int(int64_t(dp) * i / ld.n_state_items), r1 = int(int64_t(dp) * (i + 1) / ld.n_state_items);
           it.begin = r0;
           it.count = r1 - r0;
           items->push_back(it);
@@ -243,7 +269,7 @@ int glide::plan_context(const glide_config *cfg, glide_ctx *ctx, std::vector<Wor
     const size_t elem = ctx->elem;
     auto layer_cost = [&](int l) -> size_t {
       const LayerDev &ld = ctx->layers[l];
-      return size_t(ld.cap) * d * elem * 2 + (ld.evicts ? size_t(d) * d * 4 * 2 : 0);
+      return size_t(ld.cap) * d * elem * 2 + (ld.evicts ? size_t(dp) * d * 4 * 2 : 0);
     };
     std::stable_sort(items->begin(), items->end(), [&](const WorkItem &a, const WorkItem &b) {
       const size_t ca = layer_cost(a.layer), cb = layer_cost(b.layer);
@@ -295,7 +321,7 @@ int glide_create(const glide_config *cfg, void *dev_workspace, size_t workspace_
   int per_sm = 0;
   // kernel choice: fp32 -> CUDA cores; bf16 -> streaming tensor-core kernel when it applies, else per-item one
   ctx->decode_kind = 0;
-  if (ok && cfg->io_dtype == GLIDE_BF16 && cfg->decode_impl != GLIDE_DECODE_FMA) {
+  if (ok && cfg->io_dtype == GLIDE_BF16 && cfg->decode_impl != GLIDE_DECODE_FMA && !cfg->gated) {
     ok = build_ring_tensor_maps(ctx) == GLIDE_OK;
     const bool want_stream = cfg->decode_impl == GLIDE_DECODE_AUTO || cfg->decode_impl == GLIDE_DECODE_STREAM;
     if (ok && want_stream && stream_decode_supported(ctx) && ctx->sm_count * GLIDE_STREAM_CTAS_PER_SM <= kMaxStreamCtas) {
@@ -308,10 +334,11 @@ int glide_create(const glide_config *cfg, void *dev_workspace, size_t workspace_
         delete ctx;
         return GLIDE_ERR_UNSUPPORTED;
       }
-      if (cfg->merge == GLIDE_MERGE_SHARED) {
+      if (cfg->merge == GLIDE_MERGE_SHARED && cfg->phi == GLIDE_PHI_SOFTMAX) {
         ok = mma_decode_setup(ctx) == GLIDE_OK;
         ctx->decode_kind = 1;
-      }   // the per-item tensor-core kernel has the shared normaliser only: other merges use the CUDA-core kernel
+      }   // the per-item tensor-core kernel has the shared normaliser and the parameter-free map only: other merges and
+          // the learned map use the CUDA-core kernel
     }
   }
   if (ok && ctx->decode_kind == 0) {
@@ -384,8 +411,9 @@ int set_seq_off(glide_ctx *ctx, int b, int64_t off, cudaStream_t st) {
 }
 }  // namespace
 
-int glide_decode_step_layers(glide_ctx *ctx, int32_t layer_begin, int32_t layer_count, const void *q, const void *k,
-                             const void *v, void *out, void *stream) {
+namespace {
+int decode_step_layers(glide_ctx *ctx, int32_t layer_begin, int32_t layer_count, const void *q, const void *k,
+                       const void *v, const float *gate, void *out, void *stream) {
   if (!ctx || !q || !k || !v || !out) return GLIDE_ERR_INVALID_ARG;
   Range range("glide_decode_step");
   if (layer_begin < 0 || layer_count < 1 || layer_begin + layer_count > ctx->cfg.n_layers) return GLIDE_ERR_INVALID_ARG;
@@ -393,10 +421,22 @@ int glide_decode_step_layers(glide_ctx *ctx, int32_t layer_begin, int32_t layer_
   for (int l = layer_begin + 1; l < layer_begin + layer_count; ++l)
     if (ctx->n_host[l] != ctx->n_host[layer_begin]) return GLIDE_ERR_STATE;
   if (ctx->n_host[layer_begin] + max_seq_off(ctx) + 1 > ctx->cfg.max_tokens) return GLIDE_ERR_CAPACITY;
-  int rc = launch_decode(ctx, layer_begin, layer_count, q, k, v, out, as_stream(stream));
+  int rc = launch_decode(ctx, layer_begin, layer_count, q, k, v, gate, out, as_stream(stream));
   if (rc) return rc;
   for (int l = layer_begin; l < layer_begin + layer_count; ++l) ctx->n_host[l] += 1;
   return GLIDE_OK;
+}
+}  // namespace
+
+int glide_decode_step_layers(glide_ctx *ctx, int32_t layer_begin, int32_t layer_count, const void *q, const void *k,
+                             const void *v, void *out, void *stream) {
+  return decode_step_layers(ctx, layer_begin, layer_count, q, k, v, nullptr, out, stream);
+}
+
+int glide_decode_step_gated(glide_ctx *ctx, const void *q, const void *k, const void *v, const float *gate, void *out,
+                            void *stream) {
+  if (!ctx || !ctx->cfg.gated || !aligned16(gate)) return GLIDE_ERR_INVALID_ARG;
+  return decode_step_layers(ctx, 0, ctx->cfg.n_layers, q, k, v, gate, out, stream);
 }
 
 int glide_decode_step(glide_ctx *ctx, const void *q, const void *k, const void *v, void *out, void *stream) {
@@ -418,8 +458,9 @@ int glide_decode_step_noalloc(glide_ctx *ctx, const void *q, const void *k, cons
   return GLIDE_OK;
 }
 
-int glide_prefill(glide_ctx *ctx, int32_t layer_begin, int32_t layer_count, int64_t T, const void *q, const void *k,
-                  const void *v, void *out, void *stream) {
+namespace {
+int prefill_layers(glide_ctx *ctx, int32_t layer_begin, int32_t layer_count, int64_t T, const void *q, const void *k,
+                   const void *v, const float *gate, void *out, void *stream) {
   if (!ctx || !k || !v || T < 0) return GLIDE_ERR_INVALID_ARG;
   Range range("glide_prefill");
   if (out && !q) return GLIDE_ERR_INVALID_ARG;
@@ -433,11 +474,23 @@ int glide_prefill(glide_ctx *ctx, int32_t layer_begin, int32_t layer_count, int6
     if (ctx->seq_off[b] != ctx->seq_off[0] || ctx->parked[b]) return GLIDE_ERR_STATE;
   if (ctx->n_host[layer_begin] + ctx->seq_off[0] + T > ctx->cfg.max_tokens) return GLIDE_ERR_CAPACITY;
   if (T == 0) return GLIDE_OK;
-  int rc = launch_prefill(ctx, layer_begin, layer_count, T, q, k, v, out, -1, ctx->n_host[layer_begin] + ctx->seq_off[0],
-                          as_stream(stream));
+  int rc = launch_prefill(ctx, layer_begin, layer_count, T, q, k, v, gate, out, -1,
+                          ctx->n_host[layer_begin] + ctx->seq_off[0], as_stream(stream));
   if (rc) return rc;
   for (int l = layer_begin; l < layer_begin + layer_count; ++l) ctx->n_host[l] += T;
   return GLIDE_OK;
+}
+}  // namespace
+
+int glide_prefill(glide_ctx *ctx, int32_t layer_begin, int32_t layer_count, int64_t T, const void *q, const void *k,
+                  const void *v, void *out, void *stream) {
+  return prefill_layers(ctx, layer_begin, layer_count, T, q, k, v, nullptr, out, stream);
+}
+
+int glide_prefill_gated(glide_ctx *ctx, int32_t layer_begin, int32_t layer_count, int64_t T, const void *q, const void *k,
+                        const void *v, const float *gate, void *out, void *stream) {
+  if (!ctx || !ctx->cfg.gated || !aligned16(gate)) return GLIDE_ERR_INVALID_ARG;
+  return prefill_layers(ctx, layer_begin, layer_count, T, q, k, v, gate, out, stream);
 }
 
 int glide_prefill_seq(glide_ctx *ctx, int32_t b, int64_t T, const void *q, const void *k, const void *v, void *out,
@@ -451,7 +504,7 @@ int glide_prefill_seq(glide_ctx *ctx, int32_t b, int64_t T, const void *q, const
   const int64_t n0 = ctx->n_host[0] + ctx->seq_off[size_t(b)];
   if (n0 + T > ctx->cfg.max_tokens) return GLIDE_ERR_CAPACITY;
   if (T == 0) return GLIDE_OK;
-  int rc = launch_prefill(ctx, 0, ctx->cfg.n_layers, T, q, k, v, out, b, n0, as_stream(stream));
+  int rc = launch_prefill(ctx, 0, ctx->cfg.n_layers, T, q, k, v, nullptr, out, b, n0, as_stream(stream));
   if (rc) return rc;
   return set_seq_off(ctx, b, ctx->seq_off[size_t(b)] + T, as_stream(stream));
 }
@@ -464,8 +517,9 @@ int glide_reset_seq(glide_ctx *ctx, int32_t b, void *stream) {
   const size_t d = size_t(ctx->cfg.head_dim), Hkv = size_t(ctx->cfg.n_kv_heads);
   bool ok = true;
   for (const LayerDev &ld : ctx->layers) {
-    ok = ok && cudaMemsetAsync(ctx->ws + ld.S + size_t(b) * Hkv * d * d * 4, 0, Hkv * d * d * 4, st) == cudaSuccess;
-    ok = ok && cudaMemsetAsync(ctx->ws + ld.z + size_t(b) * Hkv * d * 4, 0, Hkv * d * 4, st) == cudaSuccess;
+    const size_t dp = size_t(ctx->dp);
+    ok = ok && cudaMemsetAsync(ctx->ws + ld.S + size_t(b) * Hkv * dp * d * 4, 0, Hkv * dp * d * 4, st) == cudaSuccess;
+    ok = ok && cudaMemsetAsync(ctx->ws + ld.z + size_t(b) * Hkv * dp * 4, 0, Hkv * dp * 4, st) == cudaSuccess;
   }
   if (!ok) {
     cudaGetLastError();
@@ -529,8 +583,9 @@ int glide_export_state(glide_ctx *ctx, int32_t layer, void *ringK, void *ringV, 
   bool ok = true;
   if (ringK && ring_bytes) ok = ok && cudaMemcpyAsync(ringK, ctx->ws + ld.ringK, ring_bytes, cudaMemcpyDeviceToDevice, st) == cudaSuccess;
   if (ringV && ring_bytes) ok = ok && cudaMemcpyAsync(ringV, ctx->ws + ld.ringV, ring_bytes, cudaMemcpyDeviceToDevice, st) == cudaSuccess;
-  if (S) ok = ok && cudaMemcpyAsync(S, ctx->ws + ld.S, units * d * d * 4, cudaMemcpyDeviceToDevice, st) == cudaSuccess;
-  if (z) ok = ok && cudaMemcpyAsync(z, ctx->ws + ld.z, units * d * 4, cudaMemcpyDeviceToDevice, st) == cudaSuccess;
+  const size_t dp = size_t(ctx->dp);
+  if (S) ok = ok && cudaMemcpyAsync(S, ctx->ws + ld.S, units * dp * d * 4, cudaMemcpyDeviceToDevice, st) == cudaSuccess;
+  if (z) ok = ok && cudaMemcpyAsync(z, ctx->ws + ld.z, units * dp * 4, cudaMemcpyDeviceToDevice, st) == cudaSuccess;
   if (!ok) {
     cudaGetLastError();
     return GLIDE_ERR_CUDA;
@@ -549,8 +604,9 @@ int glide_import_state(glide_ctx *ctx, int32_t layer, int64_t n, const void *rin
   bool ok = true;
   if (ringK && ring_bytes) ok = ok && cudaMemcpyAsync(ctx->ws + ld.ringK, ringK, ring_bytes, cudaMemcpyDeviceToDevice, st) == cudaSuccess;
   if (ringV && ring_bytes) ok = ok && cudaMemcpyAsync(ctx->ws + ld.ringV, ringV, ring_bytes, cudaMemcpyDeviceToDevice, st) == cudaSuccess;
-  if (S) ok = ok && cudaMemcpyAsync(ctx->ws + ld.S, S, units * d * d * 4, cudaMemcpyDeviceToDevice, st) == cudaSuccess;
-  if (z) ok = ok && cudaMemcpyAsync(ctx->ws + ld.z, z, units * d * 4, cudaMemcpyDeviceToDevice, st) == cudaSuccess;
+  const size_t dp = size_t(ctx->dp);
+  if (S) ok = ok && cudaMemcpyAsync(ctx->ws + ld.S, S, units * dp * d * 4, cudaMemcpyDeviceToDevice, st) == cudaSuccess;
+  if (z) ok = ok && cudaMemcpyAsync(ctx->ws + ld.z, z, units * dp * 4, cudaMemcpyDeviceToDevice, st) == cudaSuccess;
   // the counter is a pageable 8-byte source: the runtime stages it before returning
   ok = ok && cudaMemcpyAsync(ctx->ws + ctx->off_ndev + sizeof(int64_t) * layer, &n, sizeof(int64_t),
                              cudaMemcpyHostToDevice, st) == cudaSuccess;
@@ -560,6 +616,30 @@ int glide_import_state(glide_ctx *ctx, int32_t layer, int64_t n, const void *rin
   }
   ctx->n_host[layer] = n;
   return GLIDE_OK;
+}
+
+namespace {
+int copy_gates(glide_ctx *ctx, int32_t layer, float *out, const float *in, void *stream) {
+  if (!ctx || layer < 0 || layer >= ctx->cfg.n_layers || (!out && !in)) return GLIDE_ERR_INVALID_ARG;
+  if (!ctx->cfg.gated) return GLIDE_ERR_INVALID_ARG;
+  const LayerDev &ld = ctx->layers[layer];
+  const size_t bytes = sizeof(float) * size_t(ctx->cfg.batch) * ctx->cfg.n_kv_heads * size_t(ld.cap);
+  if (bytes == 0) return GLIDE_OK;
+  const cudaError_t e = out ? cudaMemcpyAsync(out, ctx->ws + ld.ringG, bytes, cudaMemcpyDeviceToDevice, as_stream(stream))
+                            : cudaMemcpyAsync(ctx->ws + ld.ringG, in, bytes, cudaMemcpyDeviceToDevice, as_stream(stream));
+  if (e != cudaSuccess) {
+    cudaGetLastError();
+    return GLIDE_ERR_CUDA;
+  }
+  return GLIDE_OK;
+}
+}  // namespace
+
+int glide_export_gates(glide_ctx *ctx, int32_t layer, float *dev_gates, void *stream) {
+  return copy_gates(ctx, layer, dev_gates, nullptr, stream);
+}
+int glide_import_gates(glide_ctx *ctx, int32_t layer, const float *dev_gates, void *stream) {
+  return copy_gates(ctx, layer, nullptr, dev_gates, stream);
 }
 
 int glide_reset(glide_ctx *ctx, void *stream) {

@@ -29,6 +29,8 @@ struct LayerDev {
   int32_t evicts;       // 1 if the layer has a state that ever receives tokens: wlin < max_tokens
   int32_t merge;        // glide_merge
   int64_t wlin;         // a token enters the state wlin steps after it arrives: w, or 0 when the state holds all tokens
+  size_t ringG;         // byte offset: gates of the ring's tokens [B][Hkv][cap] fp32 (gated contexts only)
+  size_t pad2_;
 };
 
 // One work item of the decode kernel.
@@ -88,6 +90,15 @@ struct DecodeParams {
   float scale_log2;          // softmax_scale * log2(e)
   int64_t t_host;            // position of the token being decoded as the host tracks it (= device counter)
   int32_t layer_begin, layer_count;   // layers of this launch; q, k, v, out are indexed with the absolute layer
+  // learned feature map: the step's phi(q_h) and phi(k_e), written by the feature kernel in front of the decode kernel,
+  // [unit][D_phi / 16][G + 1][16] fp32 (row G: the key that enters the state); null for the parameter-free map
+  float *phit;
+  const void *wq, *wk;       // [L][H][d][d], [L][Hkv][d][d] in the I/O dtype
+  int32_t dp;                // feature dimension D_phi
+  int32_t gated;
+  const float *gate;         // this step's gates [L][B][Hkv] (indexed with the absolute layer), or null for gates of 1
+  int32_t tensors_absolute;  // q, k, v, out are indexed with the absolute layer (per-item kernels) or from the range's first
+  int32_t pad3_;
 };
 
 #ifndef GLIDE_STREAM_WARPS
@@ -158,6 +169,11 @@ struct PrefillParams {
   int32_t L, B, H, Hkv;      // B: sequences of the call's tensors
   int32_t b0;                // sequence slot of the context that the call's sequence 0 is (0 unless one sequence is prefilled)
   float scale_log2;
+  int32_t phi, dp;           // glide_phi and its feature dimension
+  const void *wq, *wk;       // learned feature map: [L][H][d][d], [L][Hkv][d][d] in the I/O dtype
+  int32_t gated;
+  const float *gate;         // the call's gates [layer_count][B][T][Hkv], or null for gates of 1
+  float *gcum;               // gated: running sums of log(gate) of the chunk's delayed tokens, [units][Cmax]
 };
 
 }  // namespace glide
@@ -189,6 +205,8 @@ struct glide_ctx {
   size_t stream_seg_capacity = 0, stream_rec_capacity = 0;
   size_t off_stream_segs = 0, off_stream_cta = 0;
   int G = 0;
+  int dp = 0;                       // feature dimension of the linear part: d, or 2d for the learned map
+  size_t off_phit = 0, off_gcum = 0;
   int device = 0;
   int sm_count = 0;
   int decode_grid = 0;
@@ -223,13 +241,13 @@ int stream_decode_setup(glide_ctx *ctx);      // builds the static schedule (hos
 int launch_decode_stream(glide_ctx *ctx, const DecodeParams &p, int schedule, cudaStream_t stream);
 int launch_decode_mma(glide_ctx *ctx, const DecodeParams &p, cudaStream_t stream);
 int launch_decode_noalloc(glide_ctx *ctx, const void *q, const void *k, const void *v, void *out, cudaStream_t stream);
-int launch_decode(glide_ctx *ctx, int layer_begin, int layer_count, const void *q, const void *k, const void *v, void *out,
-                  cudaStream_t stream);
+int launch_decode(glide_ctx *ctx, int layer_begin, int layer_count, const void *q, const void *k, const void *v,
+                  const float *gate, void *out, cudaStream_t stream);
 int decode_occupancy(const glide_ctx *ctx, int *blocks_per_sm);
 // seq < 0: the call's tensors hold all B sequences, the layers' counters advance; otherwise they hold sequence slot
 // `seq` alone ([layer_count][1][T]...), which is at position n0, and no counter is touched
 int launch_prefill(glide_ctx *ctx, int layer_begin, int layer_count, int64_t T, const void *q, const void *k,
-                   const void *v, void *out, int seq, int64_t n0, cudaStream_t stream);
+                   const void *v, const float *gate, void *out, int seq, int64_t n0, cudaStream_t stream);
 bool prefill_attn_tc_supported(const glide_ctx *ctx);
 int launch_prefill_attn_tc(glide_ctx *ctx, const PrefillParams &p, cudaStream_t stream);
 bool prefill_attn_mma_supported(const glide_ctx *ctx);

@@ -42,6 +42,12 @@ struct RowSource {
   __device__ __forceinline__ const T *v(int64_t j, int D) const {
     return j >= n0 ? callV + (j - n0) * call_stride : ringV + (j % cap) * D;
   }
+  // gate of token j (gated contexts): from the call's gates, or from the ring of gates; 1 when the call has none
+  const float *ringG, *callG;   // unit base [cap]; (layer, sequence) base [T][Hkv], already offset to KV head g
+  int64_t gate_stride;          // Hkv
+  __device__ __forceinline__ float gate(int64_t j) const {
+    return j >= n0 ? (callG ? callG[(j - n0) * gate_stride] : 1.f) : ringG[j % cap];
+  }
 };
 
 template <typename T, int D>
@@ -56,13 +62,51 @@ __device__ __forceinline__ RowSource<T> make_source(const PrefillParams &p, cons
   s.n0 = p.n0;
   s.cap = ld.cap > 0 ? ld.cap : 1;
   s.call_stride = int64_t(p.Hkv) * D;
+  s.ringG = p.gated ? reinterpret_cast<const float *>(p.ws + ld.ringG) + unit_rows : nullptr;
+  s.callG = p.gate ? p.gate + (size_t(lrel) * p.B + b) * size_t(p.T) * p.Hkv + g : nullptr;
+  s.gate_stride = p.Hkv;
   return s;
+}
+
+// Learned feature map of N rows held by a warp (lane: entries lane*E .. lane*E+E-1 of each row): y = W^T x with the
+// head's d x d matrix W read once for all N rows (row i of W: 32 lanes x E consecutive entries, coalesced), then the
+// two softmax halves.  lo / hi receive softmax(y) and softmax(-y) in the same lane layout.
+template <typename T, int D, int N>
+__device__ __forceinline__ void warp_phi_learned(const T *W, const float (&x)[N][D / 32], float (&lo)[N][D / 32],
+                                                 float (&hi)[N][D / 32]) {
+  constexpr int E = D / 32;
+  const int lane = threadIdx.x & 31;
+#pragma unroll
+  for (int n = 0; n < N; ++n)
+#pragma unroll
+    for (int e = 0; e < E; ++e) lo[n][e] = 0.f;
+#pragma unroll 4
+  for (int il = 0; il < 32; ++il) {
+#pragma unroll
+    for (int ie = 0; ie < E; ++ie) {
+      float w[E];
+      load_elems<T, E>(W + size_t(il * E + ie) * D + lane * E, w);
+#pragma unroll
+      for (int n = 0; n < N; ++n) {
+        const float xi = __shfl_sync(0xffffffffu, x[n][ie], il);
+#pragma unroll
+        for (int e = 0; e < E; ++e) lo[n][e] = fmaf(xi, w[e], lo[n][e]);
+      }
+    }
+  }
+#pragma unroll
+  for (int n = 0; n < N; ++n) {
+#pragma unroll
+    for (int e = 0; e < E; ++e) hi[n][e] = -lo[n][e];
+    warp_phi<E>(lo[n]);
+    warp_phi<E>(hi[n]);
+  }
 }
 
 // 1. phi of the delayed keys of this chunk: one warp per (unit, kTokPerWarp consecutive chunk tokens), the rows'
 // loads issued together (with one row per warp the kernel was bound by the latency of its single load)
 constexpr int kTokPerWarp = 4;
-template <typename T, int D>
+template <typename T, int D, int DP>
 __global__ void __launch_bounds__(kPrefillThreads) prefill_phi_kernel(const PrefillParams p) {
   constexpr int E = D / 32;
   const int lane = threadIdx.x & 31;
@@ -86,22 +130,67 @@ __global__ void __launch_bounds__(kPrefillThreads) prefill_phi_kernel(const Pref
     valid[r] = i0 + r < p.C && j >= 0;
     if (valid[r]) load_elems<T, E>(src.k(j, D) + lane * E, x[r]);
   }
+  if constexpr (DP == D) {
 #pragma unroll
-  for (int r = 0; r < kTokPerWarp; ++r) {
-    if (!valid[r]) continue;   // warp-uniform
-    warp_phi<E>(x[r]);
-    float *dst = p.phik + (size_t(u) * p.Cmax + i0 + r) * D + lane * E;
+    for (int r = 0; r < kTokPerWarp; ++r) {
+      if (!valid[r]) continue;   // warp-uniform
+      warp_phi<E>(x[r]);
+      float *dst = p.phik + (size_t(u) * p.Cmax + i0 + r) * D + lane * E;
 #pragma unroll
-    for (int e = 0; e < E; ++e) dst[e] = x[r][e];
+      for (int e = 0; e < E; ++e) dst[e] = x[r][e];
+    }
+  } else {
+#pragma unroll
+    for (int r = 0; r < kTokPerWarp; ++r)
+      if (!valid[r])
+#pragma unroll
+        for (int e = 0; e < E; ++e) x[r][e] = 0.f;
+    float lo[kTokPerWarp][E], hi[kTokPerWarp][E];
+    const T *W = reinterpret_cast<const T *>(p.wk) + (size_t(p.layer_begin + lrel) * p.Hkv + g) * D * D;
+    warp_phi_learned<T, D, kTokPerWarp>(W, x, lo, hi);
+#pragma unroll
+    for (int r = 0; r < kTokPerWarp; ++r) {
+      if (!valid[r]) continue;
+      float *dst = p.phik + (size_t(u) * p.Cmax + i0 + r) * DP + lane * E;
+#pragma unroll
+      for (int e = 0; e < E; ++e) {
+        dst[e] = lo[r][e];
+        dst[D + e] = hi[r][e];
+      }
+    }
+  }
+}
+
+// 1c. (gated contexts) running sums of log(gate) over the chunk's delayed tokens: gcum[i] = sum over the valid delayed
+// indices ii <= i of log gate(k'_ii).  exp(gcum[i] - gcum[ii]) is then the decay a delayed token ii has suffered when
+// delayed token i has entered the state, exp(gcum[i]) the decay of the state the chunk started from.
+// One thread per unit, sequential over the chunk (C <= 1024).
+template <typename T, int D>
+__global__ void __launch_bounds__(kPrefillThreads) prefill_gcum_kernel(const PrefillParams p) {
+  const int64_t u = int64_t(blockIdx.x) * kPrefillThreads + threadIdx.x;
+  const int64_t units = int64_t(p.layer_count) * p.B * p.Hkv;
+  if (u >= units) return;
+  const int g = int(u % p.Hkv);
+  const int b = int((u / p.Hkv) % p.B);
+  const int lrel = int(u / (int64_t(p.Hkv) * p.B));
+  const LayerDev ld = p.layers[p.layer_begin + lrel];
+  if (!ld.evicts) return;
+  const RowSource<T> src = make_source<T, D>(p, ld, lrel, b, g);
+  float run = 0.f;
+  for (int i = 0; i < p.C; ++i) {
+    const int64_t j = p.n0 + p.c0 + i - ld.wlin;
+    if (j >= 0) run += logf(src.gate(j));
+    p.gcum[size_t(u) * p.Cmax + i] = run;
   }
 }
 
 // 2. outputs: one warp per (unit, query token), G heads at once
-template <typename T, int D, int G>
+template <typename T, int D, int G, int DP>
 __global__ void __launch_bounds__(kPrefillThreads) prefill_attn_kernel(const PrefillParams p) {
   constexpr int E = D / 32;
   constexpr int NW = kPrefillThreads / 32;
-  __shared__ float sm_phiq[NW][G][D];
+  constexpr int NH = DP / D;   // halves of the feature vector: lane holds entries lane*E .. +E-1 of each
+  __shared__ float sm_phiq[NW][G][DP];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int64_t wid = int64_t(blockIdx.x) * NW + warp;
   const int64_t units = int64_t(p.layer_count) * p.B * p.Hkv;
@@ -122,15 +211,27 @@ __global__ void __launch_bounds__(kPrefillThreads) prefill_attn_kernel(const Pre
   for (int h = 0; h < G; ++h) {
     const int head = p.heads_of[g * G + h];
     load_elems<T, E>(qbase + size_t(head) * D + lane * E, qr[h]);
-    float x[E];
+    if constexpr (DP == D) {
+      float x[E];
 #pragma unroll
-    for (int e = 0; e < E; ++e) x[e] = qr[h][e];
-    warp_phi<E>(x);
+      for (int e = 0; e < E; ++e) x[e] = qr[h][e];
+      warp_phi<E>(x);
 #pragma unroll
-    for (int e = 0; e < E; ++e) {
-      sm_phiq[warp][h][lane * E + e] = x[e];
-      qr[h][e] *= p.scale_log2;
+      for (int e = 0; e < E; ++e) sm_phiq[warp][h][lane * E + e] = x[e];
+    } else {
+      float x[1][E], lo[1][E], hi[1][E];
+#pragma unroll
+      for (int e = 0; e < E; ++e) x[0][e] = qr[h][e];
+      warp_phi_learned<T, D, 1>(reinterpret_cast<const T *>(p.wq) + (size_t(p.layer_begin + lrel) * p.H + head) * D * D, x,
+                                lo, hi);
+#pragma unroll
+      for (int e = 0; e < E; ++e) {
+        sm_phiq[warp][h][lane * E + e] = lo[0][e];
+        sm_phiq[warp][h][D + lane * E + e] = hi[0][e];
+      }
     }
+#pragma unroll
+    for (int e = 0; e < E; ++e) qr[h][e] *= p.scale_log2;
   }
   __syncwarp();
 
@@ -168,44 +269,55 @@ __global__ void __launch_bounds__(kPrefillThreads) prefill_attn_kernel(const Pre
   }
   if (ld.evicts && tq >= ld.wlin) {
     const int64_t folded_at_chunk_start = p.n0 + p.c0 - ld.wlin;  // tokens < this are in S,z
+    // gated: the decays come from the running sums of log(gate) over the chunk's delayed tokens
+    const float *gc = p.gated ? p.gcum + size_t(u) * p.Cmax : nullptr;
+    const float g_own = gc ? gc[i] : 0.f;
     if (folded_at_chunk_start > 0) {
-      const float *Sb = reinterpret_cast<const float *>(p.ws + ld.S) + size_t(ub) * D * D;
-      const float *zb = reinterpret_cast<const float *>(p.ws + ld.z) + size_t(ub) * D;
-      for (int r = 0; r < D; ++r) {
+      const float *Sb = reinterpret_cast<const float *>(p.ws + ld.S) + size_t(ub) * DP * D;
+      const float *zb = reinterpret_cast<const float *>(p.ws + ld.z) + size_t(ub) * DP;
+      const float dec0 = gc ? expf(g_own) : 1.f;   // what the state of the chunk's start has decayed to by now
+      for (int r = 0; r < DP; ++r) {
         float s[E];
         load_elems<float, E>(Sb + size_t(r) * D + lane * E, s);
 #pragma unroll
         for (int h = 0; h < G; ++h) {
-          const float f = sm_phiq[warp][h][r];
+          const float f = sm_phiq[warp][h][r] * dec0;
 #pragma unroll
           for (int e = 0; e < E; ++e) lin[h][e] = fmaf(f, s[e], lin[h][e]);
         }
       }
-      float zz[E];
-      load_elems<float, E>(zb + lane * E, zz);
 #pragma unroll
       for (int h = 0; h < G; ++h) {
         float part = 0.f;
 #pragma unroll
-        for (int e = 0; e < E; ++e) part = fmaf(sm_phiq[warp][h][lane * E + e], zz[e], part);
-        bl[h] = warp_sum(part);
+        for (int nh = 0; nh < NH; ++nh) {
+          float zz[E];
+          load_elems<float, E>(zb + nh * D + lane * E, zz);
+#pragma unroll
+          for (int e = 0; e < E; ++e) part = fmaf(sm_phiq[warp][h][nh * D + lane * E + e], zz[e], part);
+        }
+        bl[h] = warp_sum(part) * dec0;
       }
     }
     // delayed tokens of this chunk, up to and including the query's own delayed token
-    const float *pk = p.phik + size_t(u) * p.Cmax * D;
+    const float *pk = p.phik + size_t(u) * p.Cmax * DP;
     int i_lo = 0;
     if (folded_at_chunk_start < 0) i_lo = int(-folded_at_chunk_start);  // delayed index < 0 does not exist
     for (int ii = i_lo; ii <= i; ++ii) {
       const int64_t j = p.n0 + p.c0 + ii - ld.wlin;
-      float fk[E], vx[E];
-      load_elems<float, E>(pk + size_t(ii) * D + lane * E, fk);
+      float fk[NH][E], vx[E];
+#pragma unroll
+      for (int nh = 0; nh < NH; ++nh) load_elems<float, E>(pk + size_t(ii) * DP + nh * D + lane * E, fk[nh]);
       load_elems<T, E>(src.v(j, D) + lane * E, vx);
+      const float dec = gc ? expf(g_own - gc[ii]) : 1.f;
 #pragma unroll
       for (int h = 0; h < G; ++h) {
         float part = 0.f;
 #pragma unroll
-        for (int e = 0; e < E; ++e) part = fmaf(sm_phiq[warp][h][lane * E + e], fk[e], part);
-        const float c = warp_sum(part);
+        for (int nh = 0; nh < NH; ++nh)
+#pragma unroll
+          for (int e = 0; e < E; ++e) part = fmaf(sm_phiq[warp][h][nh * D + lane * E + e], fk[nh][e], part);
+        const float c = warp_sum(part) * dec;
         bl[h] += c;
 #pragma unroll
         for (int e = 0; e < E; ++e) lin[h][e] = fmaf(c, vx[e], lin[h][e]);
@@ -264,7 +376,8 @@ __global__ void __launch_bounds__(kPrefillThreads) prefill_state_kernel(const Pr
   constexpr int kVBytes = kStateTok * D * int(sizeof(T));
   constexpr int kVChunks = D * int(sizeof(T)) / 16;   // 16-byte chunks per V row
   __shared__ __align__(16) unsigned char stage[2][kPhiBytes + kVBytes];
-  const int blocks_per_unit = D / kStateRows;
+  const int dp = p.dp;
+  const int blocks_per_unit = dp / kStateRows;
   const int64_t u = blockIdx.x / blocks_per_unit;
   const int rb = blockIdx.x % blocks_per_unit;
   const int g = int(u % p.Hkv);
@@ -278,7 +391,9 @@ __global__ void __launch_bounds__(kPrefillThreads) prefill_state_kernel(const Pr
   const RowSource<T> src = make_source<T, D>(p, ld, lrel, b, g);
   const int ub = (b + p.b0) * p.Hkv + g;
   const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
-  const float *pk = p.phik + size_t(u) * p.Cmax * D + rb * kStateRows;
+  const float *pk = p.phik + size_t(u) * p.Cmax * dp + rb * kStateRows;
+  const float *gc = p.gated ? p.gcum + size_t(u) * p.Cmax : nullptr;
+  const float g_end = gc ? gc[p.C - 1] : 0.f;
   float acc[8][4 * CG];
 #pragma unroll
   for (int r = 0; r < 8; ++r)
@@ -291,7 +406,7 @@ __global__ void __launch_bounds__(kPrefillThreads) prefill_state_kernel(const Pr
     const uint32_t sphi = smem_u32(stage[buf]), sv = sphi + kPhiBytes;
     for (int e = tid; e < kStateTok * (kStateRows / 4); e += kPrefillThreads) {
       const int i = e / (kStateRows / 4), c4 = e % (kStateRows / 4);
-      cp_async16(sphi + uint32_t(i * kStateRows + c4 * 4) * 4u, pk + size_t(i0 + (i < nt ? i : 0)) * D + c4 * 4, i < nt);
+      cp_async16(sphi + uint32_t(i * kStateRows + c4 * 4) * 4u, pk + size_t(i0 + (i < nt ? i : 0)) * dp + c4 * 4, i < nt);
     }
     for (int e = tid; e < kStateTok * kVChunks; e += kPrefillThreads) {
       const int i = e / kVChunks, c = e % kVChunks;
@@ -316,7 +431,9 @@ __global__ void __launch_bounds__(kPrefillThreads) prefill_state_kernel(const Pr
     for (int i = 0; i < kStateTok; ++i) {
       const float4 fa = *reinterpret_cast<const float4 *>(sphi + i * kStateRows + ty * 4);
       const float4 fb = *reinterpret_cast<const float4 *>(sphi + i * kStateRows + 32 + ty * 4);
-      const float fr[8] = {fa.x, fa.y, fa.z, fa.w, fb.x, fb.y, fb.z, fb.w};
+      // gated: what this token has decayed to by the end of the chunk (tokens past the chunk's end are zero rows)
+      const float dc = (gc && i0 + i < p.C) ? expf(g_end - gc[i0 + i]) : 1.f;
+      const float fr[8] = {fa.x * dc, fa.y * dc, fa.z * dc, fa.w * dc, fb.x * dc, fb.y * dc, fb.z * dc, fb.w * dc};
       float vc[4 * CG];
 #pragma unroll
       for (int cg = 0; cg < CG; ++cg) {
@@ -331,11 +448,13 @@ __global__ void __launch_bounds__(kPrefillThreads) prefill_state_kernel(const Pr
     }
     if (tid < kStateRows) {
 #pragma unroll 8
-      for (int i = 0; i < kStateTok; ++i) zacc += sphi[i * kStateRows + tid];
+      for (int i = 0; i < kStateTok; ++i)
+        zacc = fmaf(sphi[i * kStateRows + tid], (gc && i0 + i < p.C) ? expf(g_end - gc[i0 + i]) : 1.f, zacc);
     }
     __syncthreads();   // the stage is refilled by the next iteration's issue
   }
-  float *Sb = reinterpret_cast<float *>(p.ws + ld.S) + size_t(ub) * D * D + size_t(rb) * kStateRows * D;
+  float *Sb = reinterpret_cast<float *>(p.ws + ld.S) + size_t(ub) * dp * D + size_t(rb) * kStateRows * D;
+  const float dec_all = gc ? expf(g_end) : 1.f;   // the state the chunk started from, after the whole chunk has entered
 #pragma unroll
   for (int r = 0; r < 8; ++r) {
     const int row = (r >> 2) * 32 + ty * 4 + (r & 3);
@@ -343,16 +462,16 @@ __global__ void __launch_bounds__(kPrefillThreads) prefill_state_kernel(const Pr
     for (int cg = 0; cg < CG; ++cg) {
       float4 *dst = reinterpret_cast<float4 *>(Sb + size_t(row) * D + cg * 64 + tx * 4);
       float4 cur = *dst;
-      cur.x += acc[r][cg * 4 + 0];
-      cur.y += acc[r][cg * 4 + 1];
-      cur.z += acc[r][cg * 4 + 2];
-      cur.w += acc[r][cg * 4 + 3];
+      cur.x = fmaf(cur.x, dec_all, acc[r][cg * 4 + 0]);
+      cur.y = fmaf(cur.y, dec_all, acc[r][cg * 4 + 1]);
+      cur.z = fmaf(cur.z, dec_all, acc[r][cg * 4 + 2]);
+      cur.w = fmaf(cur.w, dec_all, acc[r][cg * 4 + 3]);
       *dst = cur;
     }
   }
   if (tid < kStateRows) {
-    float *zb = reinterpret_cast<float *>(p.ws + ld.z) + size_t(ub) * D + rb * kStateRows;
-    zb[tid] += zacc;
+    float *zb = reinterpret_cast<float *>(p.ws + ld.z) + size_t(ub) * dp + rb * kStateRows;
+    zb[tid] = fmaf(zb[tid], dec_all, zacc);
   }
 }
 
@@ -363,20 +482,21 @@ template <int D>
 __global__ void __launch_bounds__(kPrefillThreads) prefill_zcum_kernel(const PrefillParams p) {
   const int64_t idx = int64_t(blockIdx.x) * kPrefillThreads + threadIdx.x;
   const int64_t units = int64_t(p.layer_count) * p.B * p.Hkv;
-  if (idx >= units * D) return;
-  const int r = int(idx % D);
-  const int64_t u = idx / D;
+  const int dp = p.dp;
+  if (idx >= units * dp) return;
+  const int r = int(idx % dp);
+  const int64_t u = idx / dp;
   const int lrel = int(u / (int64_t(p.Hkv) * p.B));
   const LayerDev ld = p.layers[p.layer_begin + lrel];
   if (!ld.evicts) return;
   const int64_t first = p.n0 + p.c0 - ld.wlin;
   const int i_lo = first < 0 ? int(first < -int64_t(p.C) ? p.C : -first) : 0;
-  const float *pk = p.phik + size_t(u) * p.Cmax * D + r;
-  float *zc = p.zcum + size_t(u) * p.Cmax * D + r;
+  const float *pk = p.phik + size_t(u) * p.Cmax * dp + r;
+  float *zc = p.zcum + size_t(u) * p.Cmax * dp + r;
   float run = 0.f;
   for (int i = 0; i < p.C; ++i) {
-    if (i >= i_lo) run += pk[size_t(i) * D];
-    zc[size_t(i) * D] = run;
+    if (i >= i_lo) run += pk[size_t(i) * dp];
+    zc[size_t(i) * dp] = run;
   }
 }
 
@@ -425,13 +545,18 @@ __global__ void __launch_bounds__(kPrefillThreads) prefill_ring_kernel(const Pre
       kd[e] = kx[r][e];
       vd[e] = vx[r][e];
     }
+    if (p.gated && lane == 0) {   // the token's gate waits in the ring with it
+      const size_t slot = (size_t(b + p.b0) * p.Hkv + g) * size_t(ld.cap) + size_t(j % ld.cap);
+      reinterpret_cast<float *>(p.ws + ld.ringG)[slot] =
+          p.gate ? p.gate[((size_t(lrel) * p.B + b) * size_t(p.T) + size_t(p.c0 + i0 + r)) * p.Hkv + g] : 1.f;
+    }
   }
 }
 
 }  // namespace
 
 int launch_prefill(glide_ctx *ctx, int layer_begin, int layer_count, int64_t T, const void *q, const void *k,
-                   const void *v, void *out, int seq, int64_t n0, cudaStream_t stream) {
+                   const void *v, const float *gate, void *out, int seq, int64_t n0, cudaStream_t stream) {
   PrefillParams p{};
   p.ws = ctx->ws;
   p.layers = reinterpret_cast<const LayerDev *>(ctx->ws + ctx->off_layers);
@@ -455,10 +580,19 @@ int launch_prefill(glide_ctx *ctx, int layer_begin, int layer_count, int64_t T, 
   p.H = ctx->cfg.n_q_heads;
   p.Hkv = ctx->cfg.n_kv_heads;
   p.scale_log2 = ctx->scale * kLog2e;
+  p.phi = ctx->cfg.phi;
+  p.dp = ctx->dp;
+  p.wq = ctx->cfg.phi_wq;
+  p.wk = ctx->cfg.phi_wk;
+  p.gated = ctx->cfg.gated;
+  p.gate = gate;
+  p.gcum = reinterpret_cast<float *>(ctx->ws + ctx->off_gcum);
   const int64_t units = int64_t(layer_count) * p.B * p.Hkv;
+  const bool plain = ctx->cfg.phi == GLIDE_PHI_SOFTMAX && !ctx->cfg.gated;   // what the tensor-core kernels compute
   int impl = ctx->cfg.prefill_impl;
   if (impl == GLIDE_PREFILL_AUTO)
-    impl = (prefill_attn_mma_supported(ctx) && ctx->cfg.decode_impl != GLIDE_DECODE_FMA) ? GLIDE_PREFILL_TCGEN05 : GLIDE_PREFILL_FMA;
+    impl = (plain && prefill_attn_mma_supported(ctx) && ctx->cfg.decode_impl != GLIDE_DECODE_FMA) ? GLIDE_PREFILL_TCGEN05
+                                                                                              : GLIDE_PREFILL_FMA;
   // the tcgen05 kernel needs the ring descriptors of the tensor-core decode kernels (absent when decode_impl asks
   // for the CUDA-core kernel); without them the call uses the mma.sync kernel
   const bool use_tc = impl == GLIDE_PREFILL_TCGEN05 && prefill_attn_tc_supported(ctx);
@@ -467,13 +601,13 @@ int launch_prefill(glide_ctx *ctx, int layer_begin, int layer_count, int64_t T, 
                        prefill_attn_mma_supported(ctx) && ctx->cfg.merge == GLIDE_MERGE_SHARED;
   // carry of the chunk scan: tensor cores with an error-free three-way bf16 split of phi(K') (bf16, d = 128), or the
   // CUDA-core kernel (fp32 I/O, d = 64, and whenever the CUDA-core prefill is asked for)
-  const bool state_mma = prefill_state_mma_supported(ctx) && impl != GLIDE_PREFILL_FMA;
+  const bool state_mma = plain && prefill_state_mma_supported(ctx) && impl != GLIDE_PREFILL_FMA;
   bool any_evicts = false;
   for (int l = layer_begin; l < layer_begin + layer_count; ++l) any_evicts = any_evicts || ctx->layers[l].evicts;
 
-  int rc = dispatch_config(ctx->cfg.io_dtype, ctx->cfg.head_dim, ctx->G, [&](auto tt, auto dd, auto gg) -> int {
+  auto run_chunks = [&](auto tt, auto dd, auto gg, auto pp) -> int {
     using TT = typename decltype(tt)::type;
-    constexpr int D = decltype(dd)::value, G = decltype(gg)::value;
+    constexpr int D = decltype(dd)::value, G = decltype(gg)::value, DP = decltype(pp)::value;
     for (int64_t c0 = 0; c0 < T; c0 += p.Cmax) {
       p.c0 = c0;
       p.C = int(std::min<int64_t>(p.Cmax, T - c0));
@@ -481,7 +615,9 @@ int launch_prefill(glide_ctx *ctx, int layer_begin, int layer_count, int64_t T, 
       const unsigned warp_blocks = unsigned((warps * 32 + kPrefillThreads - 1) / kPrefillThreads);
       const int64_t warps4 = units * ((p.C + kTokPerWarp - 1) / kTokPerWarp);
       const unsigned warp4_blocks = unsigned((warps4 * 32 + kPrefillThreads - 1) / kPrefillThreads);
-      if (any_evicts) prefill_phi_kernel<TT, D><<<warp4_blocks, kPrefillThreads, 0, stream>>>(p);
+      if (any_evicts) prefill_phi_kernel<TT, D, DP><<<warp4_blocks, kPrefillThreads, 0, stream>>>(p);
+      if (any_evicts && p.gated)
+        prefill_gcum_kernel<TT, D><<<unsigned((units + kPrefillThreads - 1) / kPrefillThreads), kPrefillThreads, 0, stream>>>(p);
       if (out) {
         if (use_tc) {
           if (any_evicts && p.merge != GLIDE_MERGE_SHARED)
@@ -490,20 +626,25 @@ int launch_prefill(glide_ctx *ctx, int layer_begin, int layer_count, int64_t T, 
         } else if (use_mma) {
           if (launch_prefill_attn_mma(ctx, p, stream) != GLIDE_OK) return GLIDE_ERR_CUDA;
         } else {
-          prefill_attn_kernel<TT, D, G><<<warp_blocks, kPrefillThreads, 0, stream>>>(p);
+          prefill_attn_kernel<TT, D, G, DP><<<warp_blocks, kPrefillThreads, 0, stream>>>(p);
         }
       }
       if (any_evicts) {
         if (state_mma) {
           if (launch_prefill_state_mma(ctx, p, stream) != GLIDE_OK) return GLIDE_ERR_CUDA;
         } else {
-          prefill_state_kernel<TT, D><<<unsigned(units * (D / kStateRows)), kPrefillThreads, 0, stream>>>(p);
+          prefill_state_kernel<TT, D><<<unsigned(units * (DP / kStateRows)), kPrefillThreads, 0, stream>>>(p);
         }
       }
       prefill_ring_kernel<TT, D><<<warp4_blocks, kPrefillThreads, 0, stream>>>(p);
       if (cudaGetLastError() != cudaSuccess) return GLIDE_ERR_CUDA;
     }
     return GLIDE_OK;
+  };
+  int rc = dispatch_config(ctx->cfg.io_dtype, ctx->cfg.head_dim, ctx->G, [&](auto tt, auto dd, auto gg) -> int {
+    constexpr int D = decltype(dd)::value;
+    if (ctx->dp == D) return run_chunks(tt, dd, gg, IntTag<D>{});
+    return run_chunks(tt, dd, gg, IntTag<2 * D>{});
   });
   if (rc) return rc;
   return seq < 0 ? launch_advance(ctx, layer_begin, layer_count, T, stream) : GLIDE_OK;

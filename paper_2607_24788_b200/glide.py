@@ -16,7 +16,7 @@ _PKG = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_PKG, "libglide.so")
 
 GLIDE_F32, GLIDE_BF16 = 0, 1
-GLIDE_PHI_SOFTMAX = 0
+GLIDE_PHI_SOFTMAX, GLIDE_PHI_PROJ_SOFTMAX2 = 0, 1
 GLIDE_MERGE_SHARED, GLIDE_MERGE_SUM_EVICTED, GLIDE_MERGE_SUM_ALL = 0, 1, 2
 GLIDE_DECODE_AUTO, GLIDE_DECODE_MMA, GLIDE_DECODE_FMA, GLIDE_DECODE_STREAM = 0, 1, 2, 3
 GLIDE_PREFILL_AUTO, GLIDE_PREFILL_MMA_SYNC, GLIDE_PREFILL_TCGEN05, GLIDE_PREFILL_FMA = 0, 1, 2, 3
@@ -46,6 +46,7 @@ class glide_config(ctypes.Structure):
         ("max_tokens", ctypes.c_int64), ("softmax_scale", ctypes.c_float), ("prefill_chunk", ctypes.c_int32),
         ("decode_chunk", ctypes.c_int32), ("decode_state_splits", ctypes.c_int32), ("decode_impl", ctypes.c_int32),
         ("prefill_impl", ctypes.c_int32),
+        ("phi_wq", ctypes.c_void_p), ("phi_wk", ctypes.c_void_p), ("gated", ctypes.c_int32), ("reserved_", ctypes.c_int32),
     ]
 
 
@@ -72,6 +73,10 @@ def load_library() -> ctypes.CDLL:
     lib.glide_prefill.argtypes = [vp, i32, i32, i64, vp, vp, vp, vp, vp]
     lib.glide_decode_step.argtypes = [vp, vp, vp, vp, vp, vp]
     lib.glide_decode_step_noalloc.argtypes = [vp, vp, vp, vp, vp, vp]
+    lib.glide_prefill_gated.argtypes = [vp, i32, i32, i64, vp, vp, vp, vp, vp, vp]
+    lib.glide_decode_step_gated.argtypes = [vp, vp, vp, vp, vp, vp, vp]
+    lib.glide_export_gates.argtypes = [vp, i32, vp, vp]
+    lib.glide_import_gates.argtypes = [vp, i32, vp, vp]
     lib.glide_decode_step_layers.argtypes = [vp, i32, i32, vp, vp, vp, vp, vp]
     lib.glide_reset_seq.argtypes = [vp, i32, vp]
     lib.glide_park_seq.argtypes = [vp, i32, vp]
@@ -90,7 +95,8 @@ def load_library() -> ctypes.CDLL:
     lib.glide_strerror.argtypes = [ctypes.c_int]
     lib.glide_strerror.restype = ctypes.c_char_p
     for name in ("glide_workspace_bytes", "glide_create", "glide_prefill", "glide_decode_step", "glide_destroy",
-                 "glide_decode_step_noalloc", "glide_decode_step_layers",
+                 "glide_decode_step_noalloc", "glide_decode_step_layers", "glide_prefill_gated",
+                 "glide_decode_step_gated", "glide_export_gates", "glide_import_gates",
                  "glide_layer_info", "glide_export_state", "glide_import_state", "glide_reset",
                  "glide_device_status", "glide_decode_launch_info"):
         getattr(lib, name).restype = ctypes.c_int
@@ -137,14 +143,24 @@ def _stream(stream: Optional[torch.cuda.Stream]) -> Optional[int]:
 def make_config(windows: Sequence[int], batch: int, n_q_heads: int, n_kv_heads: int, head_dim: int, max_tokens: int,
                 dtype: torch.dtype = torch.bfloat16, q_to_kv: Optional[Sequence[int]] = None,
                 softmax_scale: float = 0.0, prefill_chunk: int = 0, decode_chunk: int = 0,
-                decode_state_splits: int = 0, decode_impl: int = 0, prefill_impl: int = 0, merge: int = 0):
-    """Returns (glide_config, keepalive) -- keepalive holds the host arrays the struct points to."""
+                decode_state_splits: int = 0, decode_impl: int = 0, prefill_impl: int = 0, merge: int = 0,
+                phi: int = GLIDE_PHI_SOFTMAX, phi_wq: Optional[torch.Tensor] = None,
+                phi_wk: Optional[torch.Tensor] = None, gated: bool = False):
+    """Returns (glide_config, keepalive) -- keepalive holds the host arrays the struct points to.
+    phi = GLIDE_PHI_PROJ_SOFTMAX2 takes the projections phi_wq [L][H][d][d], phi_wk [L][Hkv][d][d] (device tensors of
+    the I/O dtype; the library borrows them)."""
     win = (ctypes.c_int64 * len(windows))(*[int(w) for w in windows])
     qmap = (ctypes.c_int32 * len(q_to_kv))(*[int(x) for x in q_to_kv]) if q_to_kv is not None else None
     cfg = glide_config()
     cfg.n_layers, cfg.batch, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim = len(windows), batch, n_q_heads, n_kv_heads, head_dim
     cfg.io_dtype = {torch.float32: GLIDE_F32, torch.bfloat16: GLIDE_BF16}[dtype]
-    cfg.phi, cfg.merge = GLIDE_PHI_SOFTMAX, int(merge)
+    cfg.phi, cfg.merge = int(phi), int(merge)
+    if phi_wq is not None or phi_wk is not None:
+        L = len(windows)
+        assert phi_wq.shape == (L, n_q_heads, head_dim, head_dim) and phi_wk.shape == (L, n_kv_heads, head_dim, head_dim)
+        assert phi_wq.dtype == dtype and phi_wk.dtype == dtype
+    cfg.phi_wq, cfg.phi_wk = _ptr(phi_wq), _ptr(phi_wk)
+    cfg.gated, cfg.reserved_ = int(bool(gated)), 0
     cfg.windows = ctypes.cast(win, ctypes.POINTER(ctypes.c_int64))
     cfg.q_to_kv = ctypes.cast(qmap, ctypes.POINTER(ctypes.c_int32)) if qmap is not None else None
     cfg.max_tokens = int(max_tokens)
@@ -152,7 +168,7 @@ def make_config(windows: Sequence[int], batch: int, n_q_heads: int, n_kv_heads: 
     cfg.prefill_chunk, cfg.decode_chunk, cfg.decode_state_splits = int(prefill_chunk), int(decode_chunk), int(decode_state_splits)
     cfg.decode_impl = int(decode_impl)
     cfg.prefill_impl = int(prefill_impl)
-    return cfg, (win, qmap)
+    return cfg, (win, qmap, phi_wq, phi_wk)
 
 
 def glide_workspace_bytes(cfg: glide_config) -> int:
@@ -172,6 +188,8 @@ class Glide:
         self.L, self.B, self.H, self.Hkv, self.d = len(windows), batch, n_q_heads, n_kv_heads, head_dim
         self.windows = [int(w) for w in windows]
         self.max_tokens = int(max_tokens)
+        self.dp = 2 * head_dim if kw.get("phi", GLIDE_PHI_SOFTMAX) == GLIDE_PHI_PROJ_SOFTMAX2 else head_dim
+        self.gated = bool(kw.get("gated", False))
         self.cfg, self._keep = make_config(windows, batch, n_q_heads, n_kv_heads, head_dim, max_tokens, dtype, **kw)
         self.workspace_bytes = glide_workspace_bytes(self.cfg)
         with torch.cuda.device(self.device):
@@ -205,6 +223,29 @@ class Glide:
         assert q.dtype == k.dtype == v.dtype == out.dtype == self.dtype
         _check(self.lib.glide_decode_step(self._h, _ptr(q), _ptr(k), _ptr(v), _ptr(out), _stream(stream)),
                "glide_decode_step")
+
+    def glide_prefill_gated(self, q: Optional[torch.Tensor], k: torch.Tensor, v: torch.Tensor,
+                            gate: Optional[torch.Tensor], out: Optional[torch.Tensor] = None, layer_begin: int = 0,
+                            layer_count: Optional[int] = None, stream=None) -> None:
+        """glide_prefill of a gated context: gate fp32 [layer_count][B][T][H_kv] in (0, 1], or None for gates of 1."""
+        lc = self.L - layer_begin if layer_count is None else layer_count
+        T = k.shape[2]
+        assert k.shape == (lc, self.B, T, self.Hkv, self.d) and v.shape == k.shape and k.dtype == self.dtype
+        assert gate is None or (gate.shape == (lc, self.B, T, self.Hkv) and gate.dtype == torch.float32)
+        if out is not None:
+            assert q is not None and q.shape == (lc, self.B, T, self.H, self.d) and out.shape == q.shape
+        _check(self.lib.glide_prefill_gated(self._h, layer_begin, lc, T, _ptr(q), _ptr(k), _ptr(v), _ptr(gate), _ptr(out),
+                                            _stream(stream)), "glide_prefill_gated")
+
+    def glide_decode_step_gated(self, q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, gate: Optional[torch.Tensor],
+                                out: torch.Tensor, stream=None) -> None:
+        """glide_decode_step of a gated context: gate fp32 [L][B][H_kv] in (0, 1], or None for gates of 1."""
+        assert q.shape == (self.L, self.B, self.H, self.d) and out.shape == q.shape
+        assert k.shape == (self.L, self.B, self.Hkv, self.d) and v.shape == k.shape
+        assert q.dtype == k.dtype == v.dtype == out.dtype == self.dtype
+        assert gate is None or (gate.shape == (self.L, self.B, self.Hkv) and gate.dtype == torch.float32)
+        _check(self.lib.glide_decode_step_gated(self._h, _ptr(q), _ptr(k), _ptr(v), _ptr(gate), _ptr(out),
+                                                _stream(stream)), "glide_decode_step_gated")
 
     def glide_decode_step_layers(self, q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, out: torch.Tensor,
                                  layer_begin: int, layer_count: int, stream=None) -> None:
@@ -279,8 +320,8 @@ class Glide:
         cap = self.capacity(layer)
         rk = torch.empty((self.B, self.Hkv, cap, self.d), dtype=self.dtype, device=self.device)
         rv = torch.empty_like(rk)
-        S = torch.empty((self.B, self.Hkv, self.d, self.d), dtype=torch.float32, device=self.device)
-        z = torch.empty((self.B, self.Hkv, self.d), dtype=torch.float32, device=self.device)
+        S = torch.empty((self.B, self.Hkv, self.dp, self.d), dtype=torch.float32, device=self.device)
+        z = torch.empty((self.B, self.Hkv, self.dp), dtype=torch.float32, device=self.device)
         _check(self.lib.glide_export_state(self._h, layer, _ptr(rk) if cap else None, _ptr(rv) if cap else None,
                                            _ptr(S), _ptr(z), _stream(None)), "glide_export_state")
         return rk, rv, S, z
@@ -288,6 +329,16 @@ class Glide:
     def glide_import_state(self, layer: int, n: int, ringK=None, ringV=None, S=None, z=None) -> None:
         _check(self.lib.glide_import_state(self._h, layer, int(n), _ptr(ringK), _ptr(ringV), _ptr(S), _ptr(z),
                                            _stream(None)), "glide_import_state")
+
+    def glide_export_gates(self, layer: int) -> torch.Tensor:
+        """[B][H_kv][capacity] fp32: the gates of the ring's tokens (gated contexts)."""
+        gates = torch.empty((self.B, self.Hkv, self.capacity(layer)), dtype=torch.float32, device=self.device)
+        _check(self.lib.glide_export_gates(self._h, layer, _ptr(gates), _stream(None)), "glide_export_gates")
+        return gates
+
+    def glide_import_gates(self, layer: int, gates: torch.Tensor) -> None:
+        assert gates.shape == (self.B, self.Hkv, self.capacity(layer)) and gates.dtype == torch.float32
+        _check(self.lib.glide_import_gates(self._h, layer, _ptr(gates), _stream(None)), "glide_import_gates")
 
     def glide_reset(self) -> None:
         _check(self.lib.glide_reset(self._h, _stream(None)), "glide_reset")

@@ -71,35 +71,68 @@ def check_state(g: "glide.Glide", stack: orc.Stack, what: str = ""):
                 np.testing.assert_array_equal(to_np(rk[b])[:, valid], ork[:, valid], err_msg=f"{what} ringK l{l} b{b}")
                 np.testing.assert_array_equal(to_np(rv[b])[:, valid], orv[:, valid], err_msg=f"{what} ringV l{l} b{b}")
             for name, a, r in (("S", to_np(S[b]), oS), ("z", to_np(z[b]), oz)):
+                assert a.shape == r.shape, (what, name, a.shape, r.shape)
                 nr = np.linalg.norm(r)
                 if nr == 0:
                     assert np.abs(a).max() == 0, f"{what} {name} l{l} b{b} should be zero"
                 else:
                     rel = np.linalg.norm(a - r) / nr
                     assert rel <= STATE_REL_L2, f"{what} {name} l{l} b{b}: rel-L2 {rel:.3e}"
+            if getattr(g, "gated", False) and len(valid):   # the ring's gates are copies of the callers' fp32 values
+                gr = to_np(g.glide_export_gates(l)[b])
+                np.testing.assert_array_equal(gr[:, valid], cell.export_gates()[:, valid], err_msg=f"{what} gates l{l} b{b}")
+
+
+def learned_phi_weights(L: int, H: int, Hkv: int, d: int, dtype: torch.dtype, seed: int, device="cuda"):
+    """The projections of the learned feature map, entries N(0, 1/d) rounded to the I/O dtype: (wq [L][H][d][d],
+    wk [L][Hkv][d][d]) on the device; both sides use these rounded values."""
+    gen = torch.Generator().manual_seed(1000 + seed)
+    wq = (torch.randn((L, H, d, d), generator=gen) / math.sqrt(d)).to(dtype)
+    wk = (torch.randn((L, Hkv, d, d), generator=gen) / math.sqrt(d)).to(dtype)
+    return wq.to(device), wk.to(device)
+
+
+def gates_for(shape, seed: int, lo: float = 0.6, device="cuda") -> torch.Tensor:
+    """fp32 gates in (lo, 1) of the given shape, seeded."""
+    gen = torch.Generator().manual_seed(2000 + seed)
+    return (lo + (1.0 - lo) * torch.rand(shape, generator=gen)).to(torch.float32).to(device)
 
 
 def run_case(windows: Sequence[int], B: int, H: int, Hkv: int, d: int, dtype: torch.dtype, prompt_calls: Sequence[int],
              n_decode: int, amp: float = 1.0, seed: int = 0, q_to_kv: Optional[Sequence[int]] = None,
-             max_tokens: Optional[int] = None, check_prefill_outputs: bool = True, state_checks: bool = True, **cfg_kw):
-    """prefill (one call per entry of prompt_calls) then n_decode steps on both sides; asserts parity."""
+             max_tokens: Optional[int] = None, check_prefill_outputs: bool = True, state_checks: bool = True,
+             phi: int = 0, gated: bool = False, **cfg_kw):
+    """prefill (one call per entry of prompt_calls) then n_decode steps on both sides; asserts parity.
+    phi = 1: the learned feature map with seeded projections; gated: seeded gates with every call."""
     dev = "cuda"
     L = len(windows)
     total = sum(prompt_calls) + n_decode
     max_tokens = max_tokens or max(total, 1)
     scale = f32_scale(d)
     wl = synth.Workload(seed, L, B, H, Hkv, d, dtype, amp)
+    wq = wk = None
+    if phi:
+        wq, wk = learned_phi_weights(L, H, Hkv, d, dtype, seed)
+        cfg_kw = dict(cfg_kw, phi=phi, phi_wq=wq, phi_wk=wk)
+    if gated:
+        cfg_kw = dict(cfg_kw, gated=True)
     g = glide.Glide(windows, B, H, Hkv, d, max_tokens, dtype=dtype, device=dev, q_to_kv=q_to_kv, softmax_scale=scale,
                     **cfg_kw)
     stack = orc.Stack(windows, B, H, Hkv, d, scale, q_to_kv=None if q_to_kv is None else np.asarray(q_to_kv, np.int32),
-                      merge=cfg_kw.get("merge", 0))
+                      merge=cfg_kw.get("merge", 0), phi=phi, wq=None if wq is None else to_np(wq),
+                      wk=None if wk is None else to_np(wk))
     pos = 0
     worst = 0.0
     for T in prompt_calls:
         q, k, v = wl.qkv(range(L), range(B), range(pos, pos + T), device=dev)
         out = torch.full_like(q, float("nan")) if check_prefill_outputs else None
-        g.glide_prefill(q if check_prefill_outputs else None, k, v, out)
-        ref = stack.prefill(to_np(q), to_np(k), to_np(v), outputs=check_prefill_outputs)
+        gate = gates_for((L, B, T, Hkv), seed * 131 + pos) if gated else None
+        if gated:
+            g.glide_prefill_gated(q if check_prefill_outputs else None, k, v, gate, out)
+        else:
+            g.glide_prefill(q if check_prefill_outputs else None, k, v, out)
+        ref = stack.prefill(to_np(q), to_np(k), to_np(v), outputs=check_prefill_outputs,
+                            gate=None if gate is None else to_np(gate))
         if check_prefill_outputs:
             worst = max(worst, check_outputs(out, ref, dtype, f"prefill@{pos}+{T}"))
         pos += T
@@ -108,8 +141,12 @@ def run_case(windows: Sequence[int], B: int, H: int, Hkv: int, d: int, dtype: to
     for s in range(n_decode):
         q, k, v = wl.decode_qkv(pos, device=dev)
         out = torch.full_like(q, float("nan"))
-        g.glide_decode_step(q, k, v, out)
-        ref = stack.decode(to_np(q), to_np(k), to_np(v))
+        gate = gates_for((L, B, Hkv), seed * 131 + pos) if gated else None
+        if gated:
+            g.glide_decode_step_gated(q, k, v, gate, out)
+        else:
+            g.glide_decode_step(q, k, v, out)
+        ref = stack.decode(to_np(q), to_np(k), to_np(v), gate=None if gate is None else to_np(gate))
         worst = max(worst, check_outputs(out, ref, dtype, f"decode step {s} (t={pos})"))
         pos += 1
     if state_checks:

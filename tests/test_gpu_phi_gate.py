@@ -1,0 +1,84 @@
+"""GPU parity of the learned feature map (phi = GLIDE_PHI_PROJ_SOFTMAX2, feature dimension 2d) and of the gated
+recurrence against the CPU oracle, through the C ABI: prefill calls with outputs (several, unaligned), decode steps,
+exported S [2d][d] / z [2d], ring rows, gates and counters."""
+import pytest
+import torch
+
+from paper_2607_24788_b200 import glide
+from tests.parity_util import run_case
+
+pytestmark = pytest.mark.gpu
+BF16, F32 = torch.bfloat16, torch.float32
+
+
+def test_config0_tiny_fp32_with_the_learned_map():
+    """Config 0 (1 layer, 4 = 4 heads, d = 64, w = 64, 512-token prompt, 16 decode steps, N(0,1) inputs) with the
+    d x d projection of N(0, 1/d) weights and 2d features."""
+    run_case([64], 1, 4, 4, 64, F32, [512], 16, amp=1.0, phi=1)
+
+
+@pytest.mark.parametrize("dtype,d,G", [(F32, 64, 1), (F32, 128, 2), (BF16, 64, 4), (BF16, 128, 4), (BF16, 128, 8)])
+def test_learned_map_prefill_then_decode(dtype, d, G):
+    Hkv = 2
+    amp = 1.0 if dtype == F32 else 4 * d ** -0.5
+    run_case([24, 0, 100, 5], 2, Hkv * G, Hkv, d, dtype, [37, 1, 50], 6, amp=amp, seed=3 + G, phi=1,
+             prefill_chunk=32, max_tokens=100)
+
+
+@pytest.mark.parametrize("merge", [glide.GLIDE_MERGE_SUM_EVICTED, glide.GLIDE_MERGE_SUM_ALL])
+def test_learned_map_with_the_sum_of_terms_merges(merge):
+    run_case([16, 0, 40], 2, 8, 2, 128, BF16, [45, 20], 5, amp=4 * 128 ** -0.5, seed=5, phi=1, merge=merge)
+
+
+def test_learned_map_forced_cuda_core_kernels_bf16():
+    run_case([32, 8], 3, 8, 2, 128, BF16, [70], 5, amp=4 * 128 ** -0.5, seed=6, phi=1,
+             decode_impl=glide.GLIDE_DECODE_FMA, prefill_impl=glide.GLIDE_PREFILL_FMA)
+
+
+@pytest.mark.parametrize("dtype,d,phi", [(F32, 64, 0), (BF16, 128, 0), (F32, 64, 1), (BF16, 128, 1)])
+def test_gated_recurrence_prefill_then_decode(dtype, d, phi):
+    amp = 1.0 if dtype == F32 else 4 * d ** -0.5
+    run_case([12, 0, 90, 3], 2, 8, 2, d, dtype, [29, 2, 40], 8, amp=amp, seed=7 + phi, phi=phi, gated=True,
+             prefill_chunk=16, max_tokens=90)
+
+
+def test_gated_context_without_gates_is_the_plain_method():
+    """gamma = 1 everywhere: the calls without gates on a gated context, against the ungated oracle."""
+    import numpy as np
+    from oracle import glide_oracle as orc
+    from paper_2607_24788_b200 import synth
+    from tests.parity_util import check_outputs, check_state, f32_scale, to_np
+    windows, B, H, Hkv, d, T = [10, 0], 2, 4, 2, 64, 33
+    wl = synth.Workload(9, len(windows), B, H, Hkv, d, F32, 1.0)
+    g = glide.Glide(windows, B, H, Hkv, d, T + 4, dtype=F32, softmax_scale=f32_scale(d), gated=True)
+    stack = orc.Stack(windows, B, H, Hkv, d, f32_scale(d))
+    q, k, v = wl.qkv(range(len(windows)), range(B), range(T), device="cuda")
+    out = torch.empty_like(q)
+    g.glide_prefill(q, k, v, out)
+    check_outputs(out, stack.prefill(to_np(q), to_np(k), to_np(v)), F32, "prefill")
+    for s in range(4):
+        q, k, v = wl.decode_qkv(T + s, device="cuda")
+        out = torch.empty_like(q)
+        g.glide_decode_step(q, k, v, out)
+        check_outputs(out, stack.decode(to_np(q), to_np(k), to_np(v)), F32, f"decode {s}")
+    check_state(g, stack, "ungated calls on a gated context")
+
+
+def test_feature_map_and_gate_argument_checks():
+    d = 128
+    wq = torch.zeros((1, 4, d, d), dtype=BF16, device="cuda")
+    wk = torch.zeros((1, 2, d, d), dtype=BF16, device="cuda")
+    for kw, code in ((dict(phi=1), glide.GLIDE_ERR_INVALID_ARG),                                  # no weights
+                     (dict(phi=0, phi_wq=wq, phi_wk=wk), glide.GLIDE_ERR_INVALID_ARG),            # weights without the map
+                     (dict(phi=1, phi_wq=wq, phi_wk=wk, decode_impl=glide.GLIDE_DECODE_MMA), glide.GLIDE_ERR_UNSUPPORTED),
+                     (dict(phi=1, phi_wq=wq, phi_wk=wk, prefill_impl=glide.GLIDE_PREFILL_TCGEN05), glide.GLIDE_ERR_UNSUPPORTED),
+                     (dict(gated=True, decode_impl=glide.GLIDE_DECODE_STREAM), glide.GLIDE_ERR_UNSUPPORTED)):
+        with pytest.raises(glide.GlideError) as e:
+            glide.Glide([16], 1, 4, 2, d, 64, dtype=BF16, **kw)
+        assert e.value.code == code, kw
+    plain = glide.Glide([16], 1, 4, 2, d, 64, dtype=BF16)
+    q = torch.zeros((1, 1, 4, d), dtype=BF16, device="cuda")
+    k = torch.zeros((1, 1, 2, d), dtype=BF16, device="cuda")
+    with pytest.raises(glide.GlideError) as e:   # gated call on a context without gates
+        plain.glide_decode_step_gated(q, k, k, None, torch.empty_like(q))
+    assert e.value.code == glide.GLIDE_ERR_INVALID_ARG
