@@ -46,6 +46,24 @@ NCU_TRAFFIC_BYTES = {"c1_llama8b_b1_32k": 143.1e6}   # profiles/decode_stream_c1
 MIN_TIMED_S = 0.5     # the K-step region is repeated until this much timed work has accumulated
 MAX_REPS = 4000
 KERNEL_KNOBS = {}   # tuning overrides from the command line (decode_chunk, decode_state_splits, decode_impl)
+PHI = {"kind": 0}   # --phi 1: the learned feature map (d x d projections with N(0, 1/d) weights, 2d features)
+_phi_weights = {}
+
+
+def glide_kwargs(shape, device):
+    """Keyword arguments of glide.Glide / make_config for this run: the kernel knobs and, for --phi 1, the feature
+    map's projections (seeded, one set per shape and device, shared by every context built for it)."""
+    kw = dict(KERNEL_KNOBS)
+    if PHI["kind"]:
+        key = (shape.name, str(device))
+        if key not in _phi_weights:
+            gen = torch.Generator().manual_seed(shape.seed + 77)
+            d, dt = shape.head_dim, torch_dtype(shape)
+            wq = (torch.randn((shape.n_layers, shape.n_q_heads, d, d), generator=gen) / math.sqrt(d)).to(dt)
+            wk = (torch.randn((shape.n_layers, shape.n_kv_heads, d, d), generator=gen) / math.sqrt(d)).to(dt)
+            _phi_weights[key] = (wq.to(device), wk.to(device))
+        kw.update(phi=PHI["kind"], phi_wq=_phi_weights[key][0], phi_wk=_phi_weights[key][1])
+    return kw
 
 
 def load_peaks():
@@ -149,7 +167,15 @@ def oracle_decode_rate(shape, steps: int, warmup: int, single_steps: int = 0):
     single_s = {}
     for w, layers in classes.items():
         l = layers[0]
-        stack = orc.Stack([w], 1, shape.n_q_heads, shape.n_kv_heads, shape.head_dim, scale, merge=KERNEL_KNOBS.get("merge", 0))
+        okw = {}
+        if PHI["kind"]:
+            gen = torch.Generator().manual_seed(shape.seed + 77 + l)
+            d = shape.head_dim
+            okw = dict(phi=PHI["kind"],
+                       wq=[(torch.randn((shape.n_q_heads, d, d), generator=gen) / math.sqrt(d)).to(dt).double().numpy()],
+                       wk=[(torch.randn((shape.n_kv_heads, d, d), generator=gen) / math.sqrt(d)).to(dt).double().numpy()])
+        stack = orc.Stack([w], 1, shape.n_q_heads, shape.n_kv_heads, shape.head_dim, scale, merge=KERNEL_KNOBS.get("merge", 0),
+                          **okw)
         # only the tokens that can still matter are absorbed one piece at a time
         piece = 2048
         for pos in range(0, shape.context, piece):
@@ -188,7 +214,8 @@ def workload_config(shape, extra=None):
     """The `config` object of a bench line: what was run, the same keys for both arms."""
     cfg = {"workload": shape.name, "batch": shape.batch, "context": shape.context, "n_layers": shape.n_layers,
            "sum_windows": sum(shape.windows), "q_heads": shape.n_q_heads, "kv_heads": shape.n_kv_heads,
-           "head_dim": shape.head_dim, "multi_gpu": "replicas only", "merge": KERNEL_KNOBS.get("merge", 0)}
+           "head_dim": shape.head_dim, "multi_gpu": "replicas only", "merge": KERNEL_KNOBS.get("merge", 0),
+           "phi": "softmax over the features (d)" if not PHI["kind"] else "learned projection, two softmax halves (2d)"}
     if extra:
         cfg.update(extra)
     return cfg
@@ -222,7 +249,7 @@ def build_states(shape, n_replicas: int, extra_tokens: int, device):
     wl = make_workload(shape)
     max_tokens = shape.context + extra_tokens
     ctxs = [glide.Glide(shape.windows, shape.batch, shape.n_q_heads, shape.n_kv_heads, shape.head_dim, max_tokens,
-                        dtype=dt, device=device, prefill_chunk=shape.prefill_chunk, **KERNEL_KNOBS)
+                        dtype=dt, device=device, prefill_chunk=shape.prefill_chunk, **glide_kwargs(shape, device))
              for _ in range(n_replicas)]
     g0 = ctxs[0]
     # prompt -> state (no outputs needed for a decode benchmark); layers in groups to bound the k/v buffers
@@ -272,8 +299,14 @@ def whole_job_tokens_per_s(world: int, batch: int, steps: int, ms: float) -> flo
 
 
 def roofline_bytes(shape):
-    """(the benchmark spec's bytes, bytes with the step's own q/k/v/out rows and the ring append) of one decode step."""
-    return configs.decode_step_stream_bytes(shape, shape.context), configs.decode_step_bytes(shape, shape.context)
+    """(the benchmark spec's bytes, bytes with the step's own q/k/v/out rows and the ring append) of one decode step.  With
+    the learned feature map the state is twice as large and the step also reads the projections once."""
+    fm = 2 if PHI["kind"] else 1
+    extra = 0
+    if PHI["kind"]:
+        extra = shape.n_layers * (shape.n_q_heads + shape.n_kv_heads) * shape.head_dim ** 2 * shape.elem_bytes
+    return (configs.decode_step_stream_bytes(shape, shape.context, fm),
+            configs.decode_step_bytes(shape, shape.context, fm) + extra)
 
 
 class DecodeBench:
@@ -287,7 +320,7 @@ class DecodeBench:
         free_b, _ = torch.cuda.mem_get_info(device)
         n_rep = max(1, min(16, math.ceil(8 * L2_BYTES / self.bytes_io)))
         # positions a state copy may advance before it is rewound (and room for the prefill measurement at the end)
-        self.slack = max(256, 6 * K + 64) + 3 * prefill_tokens
+        self.slack = max(256, 8 * K + 64) + 3 * prefill_tokens
         cfg_probe = self._workspace_bytes(shape, self.slack)
         n_rep = max(1, min(n_rep, int(0.8 * free_b // max(cfg_probe, 1))))
         self.n_rep = n_rep
@@ -312,7 +345,7 @@ class DecodeBench:
         from paper_2607_24788_b200 import glide
         cfg, keep = glide.make_config(shape.windows, shape.batch, shape.n_q_heads, shape.n_kv_heads, shape.head_dim,
                                       shape.context + slack, dtype=torch_dtype(shape), prefill_chunk=shape.prefill_chunk,
-                                      **KERNEL_KNOBS)
+                                      **glide_kwargs(shape, "cuda"))
         return glide.glide_workspace_bytes(cfg)
 
     def views(self, buf):
@@ -486,7 +519,7 @@ def run_glide(args, shape):
 
     per_layer = None
     if world == 1 and b.bytes_io <= (8 << 30):
-        b.make_room(1)
+        b.make_room(3 * K + 8)   # the per-layer pass steps a clone of copy 0 forward 3 + 3 K times
         per_layer = measure_per_layer_launch(b.ctxs[0], shape, b.views(b.dev_in[0]), b.outs[0], K, device)
 
     t_ms, hot_ms, e2e_t = max_over_ranks([t_ms, hot_ms, e2e_t], dist, device)
@@ -572,7 +605,7 @@ def measure_per_layer_launch(g0, shape, qkv, out, steps, device):
     dt = torch_dtype(shape)
     n = g0.glide_layer_info(0)["n"]
     g = glide.Glide(shape.windows, shape.batch, shape.n_q_heads, shape.n_kv_heads, shape.head_dim, g0.max_tokens,
-                    dtype=dt, device=device, prefill_chunk=shape.prefill_chunk, **KERNEL_KNOBS)
+                    dtype=dt, device=device, prefill_chunk=shape.prefill_chunk, **glide_kwargs(shape, device))
     for l in range(L):
         rk, rv, S, z = g0.glide_export_state(l)
         cap = g.capacity(l)
@@ -661,6 +694,9 @@ def main():
     ap.add_argument("--decode-impl", type=int, default=0,
                     help="0 auto, 1 per-item tensor-core/TMA kernel, 2 CUDA-core kernel, 3 streaming tensor-core/TMA kernel")
     ap.add_argument("--prefill-impl", type=int, default=0, help="0 auto, 1 mma.sync, 2 tcgen05 + TMEM, 3 CUDA cores")
+    ap.add_argument("--phi", type=int, default=0,
+                    help="0 softmax over the head features (the paper's default), 1 the learned map: d x d projections "
+                         "with N(0, 1/d) weights, 2d features")
     ap.add_argument("--merge", type=int, default=0,
                     help="0 shared normaliser (the paper's default), 1 / 2 the appendix' sums of two normalised terms "
                          "(evicted-token / all-token state)")
@@ -668,6 +704,7 @@ def main():
     shape = configs.ALL[args.workload]
     KERNEL_KNOBS.update(decode_chunk=args.decode_chunk, decode_state_splits=args.state_splits,
                         decode_impl=args.decode_impl, prefill_impl=args.prefill_impl, merge=args.merge)
+    PHI["kind"] = args.phi
     if args.impl == "reference":
         run_reference(args, shape)
     else:

@@ -82,23 +82,24 @@ def kv_io_bytes_per_token(windows: Sequence[int], n_kv_heads: int = 8, head_dim:
     return sum(int(w) for w in windows) * 2 * n_kv_heads * head_dim * elem_bytes
 
 
-def decode_step_bytes(shape: GlideShape, n: int) -> int:
+def decode_step_bytes(shape: GlideShape, n: int, feature_mult: int = 1) -> int:
     """Algorithmic bytes one decode step must move when n tokens are already absorbed (all sequences):
     per layer, the window slots read (one of them the token that leaves the window), the recurrent state
-    read and written once the layer evicts, the new K/V row written, and q,k,v in / out."""
+    read and written once the layer evicts, the new K/V row written, and q,k,v in / out.
+    feature_mult: feature dimension of the linear part over head_dim (2 for the learned map)."""
     H, Hkv, d, eb = shape.n_q_heads, shape.n_kv_heads, shape.head_dim, shape.elem_bytes
     total = 0
     for w in shape.windows:
         total += 2 * min(w, n + 1) * Hkv * d * eb
         if n >= w:
-            total += 2 * (Hkv * d * d + Hkv * d) * 4
+            total += 2 * feature_mult * (Hkv * d * d + Hkv * d) * 4
         if w > 0:
             total += 2 * Hkv * d * eb
         total += (2 * H + 2 * Hkv) * d * eb
     return total * shape.batch
 
 
-def decode_step_stream_bytes(shape: GlideShape, n: int) -> int:
+def decode_step_stream_bytes(shape: GlideShape, n: int, feature_mult: int = 1) -> int:
     """The roofline bytes of one decode step as the task states them: per layer and sequence the window's K and V rows,
     2 w H_kv d elem, plus the recurrent state S, z read and written once the layer evicts (all sequences)."""
     Hkv, d, eb = shape.n_kv_heads, shape.head_dim, shape.elem_bytes
@@ -106,7 +107,7 @@ def decode_step_stream_bytes(shape: GlideShape, n: int) -> int:
     for w in shape.windows:
         total += 2 * min(w, n + 1) * Hkv * d * eb
         if n >= w:
-            total += 2 * (Hkv * d * d + Hkv * d) * 4
+            total += 2 * feature_mult * (Hkv * d * d + Hkv * d) * 4
     return total * shape.batch
 
 

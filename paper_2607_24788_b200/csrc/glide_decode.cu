@@ -390,107 +390,96 @@ __global__ void __launch_bounds__(kDecodeThreads) glide_decode_kernel(const Deco
 
 // ---- learned feature map of one decode step ------------------------------------------------------
 // phi_W(x) = [softmax(W^T x); softmax(-W^T x)] of the step's queries and of the key that enters the state, for every
-// unit of the launch, into p.phit [unit][DP / 16][G + 1][16] (row G: the key).  One CTA of D threads per (layer, KV
-// head, row of the group): thread j owns output j; the d x d matrix of the head is read once, coalesced over j, for
-// all sequences of the batch (kPhiSeqs at a time in registers).
-constexpr int kPhiSeqs = 8;
-template <typename T, int D, int G>
-__global__ void __launch_bounds__(D) glide_decode_phi_kernel(const DecodeParams p) {
+// unit of the launch, into p.phit [unit][DP / 16][G + 1][16] (row G: the key).  kPhiSplit warps per (layer, KV head,
+// row of the group), each with its share of the rows of the head's d x d matrix: every lane owns D / 32 outputs
+// (the partial sums of the warps meet in shared memory), the matrix is streamed row by row, coalesced, many rows in
+// flight, for kPhiSeqs sequences of the batch at a time.
+constexpr int kPhiSplit = 2;    // warps per matrix
+constexpr int kPhiHeads = 2;    // matrices per CTA
+template <typename T, int D, int G, int kPhiSeqs>
+__global__ void __launch_bounds__(kPhiSplit * kPhiHeads * 32) glide_decode_phi_kernel(const DecodeParams p) {
   constexpr int DP = 2 * D;
-  __shared__ float sx[kPhiSeqs][D];
-  __shared__ float red[kPhiSeqs][2][D / 32];
-  const int j = threadIdx.x, warp = j >> 5, lane = j & 31;
-  const int row = blockIdx.x % (G + 1);
-  const int g = (blockIdx.x / (G + 1)) % p.Hkv;
-  const int lrel = blockIdx.x / ((G + 1) * p.Hkv);
+  constexpr int E = D / 32;
+  __shared__ float part[kPhiHeads][kPhiSplit][kPhiSeqs][D];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int hslot = warp / kPhiSplit, split = warp % kPhiSplit;
+  const int total = p.layer_count * p.Hkv * (G + 1);
+  int wid = blockIdx.x * kPhiHeads + hslot;
+  const bool active = wid < total;
+  if (!active) wid = total - 1;   // (keeps the warp in the CTA's barriers; it writes nothing)
+  const int row = wid % (G + 1);
+  const int g = (wid / (G + 1)) % p.Hkv;
+  const int lrel = wid / ((G + 1) * p.Hkv);
   const int layer = p.layer_begin + lrel;
   const LayerDev ld = p.layers[layer];
-  if (row == G && !ld.evicts) return;
+  const bool has_work = active && !(row == G && !ld.evicts);
   const int head = row < G ? p.heads_of[g * G + row] : 0;
   const T *W = row < G ? reinterpret_cast<const T *>(p.wq) + (size_t(layer) * p.H + head) * D * D
                        : reinterpret_cast<const T *>(p.wk) + (size_t(layer) * p.Hkv + g) * D * D;
+  // the per-item kernels index q, k, v with the absolute layer (their base pointers are moved back)
+  const int lq = p.tensors_absolute ? layer : lrel;
+  const int64_t n = p.n_dev[layer];
   for (int b0 = 0; b0 < p.B; b0 += kPhiSeqs) {
-    const int nb = min(kPhiSeqs, p.B - b0);
+    float x[kPhiSeqs][E], y[kPhiSeqs][E];
     bool live[kPhiSeqs];
-    __syncthreads();
 #pragma unroll
     for (int bi = 0; bi < kPhiSeqs; ++bi) {
-      live[bi] = false;
-      if (bi >= nb) continue;
       const int b = b0 + bi;
-      const int64_t t = p.n_dev[layer] + (p.seq_off ? p.seq_off[b] : 0);
+      live[bi] = false;
+#pragma unroll
+      for (int e = 0; e < E; ++e) x[bi][e] = y[bi][e] = 0.f;
+      if (b >= p.B || !has_work) continue;
+      const int64_t t = n + (p.seq_off ? p.seq_off[b] : 0);
       if (t < 0) continue;   // parked slot
       const int ub = b * p.Hkv + g;
-      const T *x;
-      // the per-item kernels index q, k, v with the absolute layer (their base pointers are moved back)
-      const int lq = p.tensors_absolute ? layer : lrel;
+      const T *src;
       if (row < G) {
-        x = reinterpret_cast<const T *>(p.q) + ((size_t(lq) * p.B + b) * p.H + head) * D;
+        src = reinterpret_cast<const T *>(p.q) + ((size_t(lq) * p.B + b) * p.H + head) * D;
       } else if (t < ld.wlin) {
         continue;            // nothing enters the state at this step
       } else if (ld.wlin == 0) {
-        x = reinterpret_cast<const T *>(p.k) + (size_t(lq) * p.B * p.Hkv + ub) * D;
+        src = reinterpret_cast<const T *>(p.k) + (size_t(lq) * p.B * p.Hkv + ub) * D;
       } else {
-        x = reinterpret_cast<const T *>(p.ws + ld.ringK) + (size_t(ub) * size_t(ld.cap) + size_t(t % ld.cap)) * D;
+        src = reinterpret_cast<const T *>(p.ws + ld.ringK) + (size_t(ub) * size_t(ld.cap) + size_t(t % ld.cap)) * D;
       }
       live[bi] = true;
-      sx[bi][j] = to_f32(x[j]);
+      load_elems<T, E>(src + lane * E, x[bi]);
+    }
+    if (has_work)
+      warp_project_rows<T, D, kPhiSeqs, (sizeof(T) == 2 ? 8 : 4)>(W, x, y, split * (32 / kPhiSplit),
+                                                                  (split + 1) * (32 / kPhiSplit));
+    __syncthreads();   // the previous batch's partial sums have been read
+    if (split > 0) {
+#pragma unroll
+      for (int bi = 0; bi < kPhiSeqs; ++bi)
+#pragma unroll
+        for (int e = 0; e < E; ++e) part[hslot][split][bi][lane * E + e] = y[bi][e];
     }
     __syncthreads();
-    float y[kPhiSeqs];
+    if (split == 0 && has_work) {
 #pragma unroll
-    for (int bi = 0; bi < kPhiSeqs; ++bi) y[bi] = 0.f;
-#pragma unroll 8
-    for (int i = 0; i < D; ++i) {
-      const float w = to_f32(W[size_t(i) * D + j]);
+      for (int bi = 0; bi < kPhiSeqs; ++bi) {
+        if (!live[bi]) continue;
+        float lo[E], hi[E];
 #pragma unroll
-      for (int bi = 0; bi < kPhiSeqs; ++bi) y[bi] = fmaf(sx[bi][i], w, y[bi]);
-    }
-    // the two softmax halves over the D outputs: maxima of y and -y, then the sums
-    float e0[kPhiSeqs], e1[kPhiSeqs];
+        for (int e = 0; e < E; ++e) {
+          float sum = y[bi][e];
 #pragma unroll
-    for (int bi = 0; bi < kPhiSeqs; ++bi) {
-      const float mx = warp_max(y[bi]), mn = warp_max(-y[bi]);
-      if (lane == 0) {
-        red[bi][0][warp] = mx;
-        red[bi][1][warp] = mn;
+          for (int sp = 1; sp < kPhiSplit; ++sp) sum += part[hslot][sp][bi][lane * E + e];
+          lo[e] = sum;
+          hi[e] = -sum;
+        }
+        warp_phi<E>(lo);
+        warp_phi<E>(hi);
+        const size_t unit = (size_t(lrel) * p.B + (b0 + bi)) * p.Hkv + g;
+        float *ph = p.phit + unit * DP * (G + 1);
+#pragma unroll
+        for (int e = 0; e < E; ++e) {
+          const int j = lane * E + e;
+          ph[(size_t(j >> 4) * (G + 1) + row) * 16 + (j & 15)] = lo[e];
+          ph[(size_t((D + j) >> 4) * (G + 1) + row) * 16 + (j & 15)] = hi[e];
+        }
       }
-    }
-    __syncthreads();
-#pragma unroll
-    for (int bi = 0; bi < kPhiSeqs; ++bi) {
-      float mx = red[bi][0][0], mn = red[bi][1][0];
-#pragma unroll
-      for (int w = 1; w < D / 32; ++w) {
-        mx = fmaxf(mx, red[bi][0][w]);
-        mn = fmaxf(mn, red[bi][1][w]);
-      }
-      e0[bi] = exp2f((y[bi] - mx) * kLog2e);
-      e1[bi] = exp2f((-y[bi] - mn) * kLog2e);
-    }
-    __syncthreads();
-#pragma unroll
-    for (int bi = 0; bi < kPhiSeqs; ++bi) {
-      const float s0 = warp_sum(e0[bi]), s1 = warp_sum(e1[bi]);
-      if (lane == 0) {
-        red[bi][0][warp] = s0;
-        red[bi][1][warp] = s1;
-      }
-    }
-    __syncthreads();
-#pragma unroll
-    for (int bi = 0; bi < kPhiSeqs; ++bi) {
-      if (!live[bi]) continue;
-      float s0 = 0.f, s1 = 0.f;
-#pragma unroll
-      for (int w = 0; w < D / 32; ++w) {
-        s0 += red[bi][0][w];
-        s1 += red[bi][1][w];
-      }
-      const size_t unit = (size_t(lrel) * p.B + (b0 + bi)) * p.Hkv + g;
-      float *ph = p.phit + unit * DP * (G + 1);
-      ph[(size_t(j >> 4) * (G + 1) + row) * 16 + (j & 15)] = e0[bi] / s0;
-      ph[(size_t((D + j) >> 4) * (G + 1) + row) * 16 + (j & 15)] = e1[bi] / s1;
     }
   }
 }
@@ -580,8 +569,13 @@ int launch_decode_phi(glide_ctx *ctx, const DecodeParams &p, cudaStream_t stream
   return dispatch_config(ctx->cfg.io_dtype, ctx->cfg.head_dim, ctx->G, [&](auto tt, auto dd, auto gg) -> int {
     using T = typename decltype(tt)::type;
     constexpr int D = decltype(dd)::value, G = decltype(gg)::value;
-    const unsigned grid = unsigned(p.layer_count) * unsigned(p.Hkv) * unsigned(G + 1);
-    glide_decode_phi_kernel<T, D, G><<<grid, D, 0, stream>>>(p);
+    const unsigned mats = unsigned(p.layer_count) * unsigned(p.Hkv) * unsigned(G + 1);
+    const unsigned grid = (mats + kPhiHeads - 1) / kPhiHeads, block = kPhiSplit * kPhiHeads * 32;
+    // (a single sequence gets its own instantiation: no work for absent sequences)
+    if (p.B == 1)
+      glide_decode_phi_kernel<T, D, G, 1><<<grid, block, 0, stream>>>(p);
+    else
+      glide_decode_phi_kernel<T, D, G, 4><<<grid, block, 0, stream>>>(p);
     if (cudaGetLastError() != cudaSuccess) return GLIDE_ERR_CUDA;
     return GLIDE_OK;
   });

@@ -259,10 +259,15 @@ __device__ __forceinline__ void warp_sum_multi(float (&x)[N]) {
 }
 
 // ---- the kernel -----------------------------------------------------------------------------
-template <int G, int STAGES, bool SUM, bool RAGGED>
+// MODE 0: shared normaliser; 1: the sum of two normalised terms; 2: shared normaliser with the learned feature map
+// (feature dimension 2 kD: 16 state tiles per unit, and every state tile arrives with its 16 entries of phi(q_h) and
+// of phi(k_e), which the feature kernel in front of this launch has written)
+template <int G, int STAGES, int MODE, bool RAGGED>
 __global__ void __launch_bounds__(kThreads, GLIDE_STREAM_CTAS_PER_SM)
 glide_decode_stream_kernel(const DecodeParams p, const StreamParams sp) {
   using bf16 = __nv_bfloat16;
+  constexpr bool SUM = MODE == 1, PHI2 = MODE == 2;
+  constexpr int kPhiTile = (G + 1) * 16;   // floats of feature values per state tile
   using L = Layout<G, SUM>;
   constexpr int KS = kD / 16;
 
@@ -274,7 +279,8 @@ glide_decode_stream_kernel(const DecodeParams p, const StreamParams sp) {
   StreamSegment *sm_segs = reinterpret_cast<StreamSegment *>(sm_z + kWarps * STAGES * 16);   // [max_segs]
   uint64_t *sm_bars = reinterpret_cast<uint64_t *>(sm_segs + sp.max_segs);          // [kWarps][STAGES + 1]
   int *sm_ctr = reinterpret_cast<int *>(sm_bars + kWarps * (STAGES + 1));             // [kStreamMaxGroups]
-  float *sm_pool = reinterpret_cast<float *>(sm_ctr + kStreamMaxGroups);              // [pool slots][kRecFloats]
+  float *sm_phi = reinterpret_cast<float *>(sm_ctr + kStreamMaxGroups);               // PHI2: [kWarps][STAGES][kPhiTile]
+  float *sm_pool = sm_phi + (PHI2 ? kWarps * STAGES * kPhiTile : 0);                  // [pool slots][kRecFloats]
   int64_t *sm_t = reinterpret_cast<int64_t *>(base + sp.t_off);                       // [max_segs], behind the pool
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -298,6 +304,8 @@ glide_decode_stream_kernel(const DecodeParams p, const StreamParams sp) {
   const uint32_t my_hdr = smem_u32(my_hdr_ptr);
   float *my_z_ptr = sm_z + warp * STAGES * 16;
   const uint32_t my_z = smem_u32(my_z_ptr);
+  float *my_phi_ptr = sm_phi + warp * STAGES * kPhiTile;
+  const uint32_t my_phi = smem_u32(my_phi_ptr);
   const uint32_t my_bars = smem_u32(sm_bars + warp * (STAGES + 1));
   const uint32_t hdr_bar = my_bars + STAGES * 8;
   if (tid < kStreamMaxGroups) sm_ctr[tid] = 0;
@@ -390,11 +398,14 @@ glide_decode_stream_kernel(const DecodeParams p, const StreamParams sp) {
                        p.status, (void)0);
         if (icur.k < icur.n_state_eff) {
           const int st = sg.state0 + icur.k;
-          mbar_expect_tx(bar, kStageBytes + 64);
+          mbar_expect_tx(bar, kStageBytes + 64 + (PHI2 ? kPhiTile * 4 : 0));
           const float *Sg = reinterpret_cast<const float *>(p.ws + size_t(sg.S_off256) * 256) + size_t(st) * kTileRows * kD;
           const float *zg = reinterpret_cast<const float *>(p.ws + size_t(sg.z_off256) * 256) + st * kTileRows;
           bulk_load(dst, Sg, kStageBytes, bar);
           bulk_load(my_z + issue_stage * 64, zg, 64, bar);
+          if (PHI2)   // the tile's rows of phi(q_h), h < G, and of phi(k_e): [unit][tile][G + 1][16]
+            bulk_load(my_phi + issue_stage * kPhiTile * 4,
+                      p.phit + (size_t(sg.unit) * (2 * kD / kTileRows) + st) * kPhiTile, kPhiTile * 4, bar);
         } else {
           const int wt = sg.win0 + icur.k - icur.n_state_eff;
           mbar_expect_tx(bar, kStageBytes);
@@ -511,12 +522,13 @@ glide_decode_stream_kernel(const DecodeParams p, const StreamParams sp) {
 
   // ---- state tile: 16 rows of S and z, updated in the stage and stored back by the async proxy ---------
   // (bulk stores are not ordered by this warp's later fences, so a ticket never waits for state traffic)
-  auto consume_state = [&](const StreamSegment &sg, int stile, float4 *st, float *zs, uint32_t st_addr, uint32_t z_addr) {
+  auto consume_state = [&](const StreamSegment &sg, int stile, float4 *st, float *zs, uint32_t st_addr, uint32_t z_addr,
+                           const float *sphi) {
     const int src0 = stile * 4;   // lane that holds phi entries of the tile's first row (4 rows per lane)
 #pragma unroll
     for (int r = 0; r < kTileRows; ++r) {
       float4 s = st[r * (kD / 4) + lane];
-      const float pk = __shfl_sync(0xffffffffu, phi[G][r & 3], src0 + (r >> 2));
+      const float pk = PHI2 ? sphi[G * 16 + r] : __shfl_sync(0xffffffffu, phi[G][r & 3], src0 + (r >> 2));
       s.x = fmaf(pk, ve[0], s.x);
       s.y = fmaf(pk, ve[1], s.y);
       s.z = fmaf(pk, ve[2], s.z);
@@ -524,7 +536,7 @@ glide_decode_stream_kernel(const DecodeParams p, const StreamParams sp) {
       st[r * (kD / 4) + lane] = s;
 #pragma unroll
       for (int h = 0; h < G; ++h) {
-        const float f = __shfl_sync(0xffffffffu, phi[h][r & 3], src0 + (r >> 2));
+        const float f = PHI2 ? sphi[h * 16 + r] : __shfl_sync(0xffffffffu, phi[h][r & 3], src0 + (r >> 2));
         a[h].x = fmaf(f, s.x, a[h].x);
         a[h].y = fmaf(f, s.y, a[h].y);
         a[h].z = fmaf(f, s.z, a[h].z);
@@ -537,10 +549,14 @@ glide_decode_stream_kernel(const DecodeParams p, const StreamParams sp) {
 #pragma unroll
     for (int h = 0; h <= G; ++h) {
       float f = 0.f;
+      if (PHI2) {
+        f = sphi[((h + G) % (G + 1)) * 16 + (lane & 15)];
+      } else {
 #pragma unroll
-      for (int j = 0; j < 4; ++j) {
-        const float v = __shfl_sync(0xffffffffu, phi[(h + G) % (G + 1)][j], zsrc);   // phi(k_e) first, then the heads
-        if ((lane & 3) == j) f = v;
+        for (int j = 0; j < 4; ++j) {
+          const float v = __shfl_sync(0xffffffffu, phi[(h + G) % (G + 1)][j], zsrc);   // phi(k_e) first, then the heads
+          if ((lane & 3) == j) f = v;
+        }
       }
       if (h == 0) {
         if (lane < 16) {
@@ -604,9 +620,11 @@ glide_decode_stream_kernel(const DecodeParams p, const StreamParams sp) {
 #pragma unroll
       for (int h = 0; h < G; ++h) scur[h] = has_win ? scur[h] * p.scale_log2 : -CUDART_INF_F;
       if (n_state_eff > 0) {
-        load_elems<bf16, 4>(h0 + G * kD + lane * 4, phi[G]);
         load_elems<bf16, 4>(h0 + (G + 1) * kD + lane * 4, ve);
-        warp_phi_multi<G + 1>(phi);
+        if (!PHI2) {   // (the learned map's features arrive with the state tiles)
+          load_elems<bf16, 4>(h0 + G * kD + lane * 4, phi[G]);
+          warp_phi_multi<G + 1>(phi);
+        }
       }
     }
     __syncwarp();
@@ -642,7 +660,8 @@ glide_decode_stream_kernel(const DecodeParams p, const StreamParams sp) {
       GLIDE_TRACE_EVENT(k < n_state_eff ? 4 : 3);
       if (k < n_state_eff)
         consume_state(sg, sg.state0 + k, reinterpret_cast<float4 *>(my_stages_ptr + stage * kStageBytes),
-                      my_z_ptr + stage * 16, my_stages + stage * kStageBytes, my_z + stage * 64);
+                      my_z_ptr + stage * 16, my_stages + stage * kStageBytes, my_z + stage * 64,
+                      my_phi_ptr + stage * kPhiTile);
       else
         consume_window(sg.win0 + k - n_state_eff, my_stages + stage * kStageBytes);
       last_stage = stage;
@@ -1025,21 +1044,28 @@ glide_decode_stream_kernel(const DecodeParams p, const StreamParams sp) {
 
 }
 
-template <int G, int STAGES, bool SUM>
+template <int G, int STAGES, int MODE>
 size_t stream_smem_bytes(int max_segs, int pool_slots) {
-  using L = Layout<G, SUM>;
+  using L = Layout<G, MODE == 1>;
   return 1024 + size_t(kWarps) * STAGES * kStageBytes + size_t(kWarps) * L::kHdrBytes + size_t(kWarps) * STAGES * 64 +
          size_t(max_segs) * sizeof(StreamSegment) + size_t(kWarps) * (STAGES + 1) * 8 + size_t(kStreamMaxGroups) * 4 +
-         size_t(pool_slots) * L::kRecFloats * 4 + size_t(max_segs) * 8;
+         (MODE == 2 ? size_t(kWarps) * STAGES * (G + 1) * 64 : 0) + size_t(pool_slots) * L::kRecFloats * 4 +
+         size_t(max_segs) * 8;
 }
 
-// f(group size, stages, sum-of-terms merge)
+// the kernel's MODE for a context
+int stream_mode(const glide_ctx *ctx) {
+  return ctx->cfg.phi == GLIDE_PHI_PROJ_SOFTMAX2 ? 2 : (ctx->cfg.merge != GLIDE_MERGE_SHARED ? 1 : 0);
+}
+
+// f(group size, stages, mode)
 template <typename F>
-int dispatch_stream(int G, bool sum, F &&f) {
-#define GLIDE_STREAM_CASE(GG)                                                        \
-  case GG:                                                                           \
-    return sum ? f(IntTag<GG>{}, IntTag<GLIDE_STREAM_STAGES>{}, IntTag<1>{})         \
-               : f(IntTag<GG>{}, IntTag<GLIDE_STREAM_STAGES>{}, IntTag<0>{});
+int dispatch_stream(int G, int mode, F &&f) {
+#define GLIDE_STREAM_CASE(GG)                                                                   \
+  case GG:                                                                                      \
+    return mode == 2   ? f(IntTag<GG>{}, IntTag<GLIDE_STREAM_STAGES>{}, IntTag<2>{})            \
+           : mode == 1 ? f(IntTag<GG>{}, IntTag<GLIDE_STREAM_STAGES>{}, IntTag<1>{})            \
+                       : f(IntTag<GG>{}, IntTag<GLIDE_STREAM_STAGES>{}, IntTag<0>{});
   switch (G) {
     GLIDE_STREAM_CASE(1)
     GLIDE_STREAM_CASE(2)
@@ -1084,7 +1110,7 @@ void build_stream_schedule(const glide_ctx *ctx, int layer_begin, int layer_coun
   for (int l = layer_begin; l < layer_begin + layer_count; ++l) {
     const LayerDev &ld = ctx->layers[l];
     for (int64_t u = 0; u < units_per_layer; ++u) {
-      Piece pc{l, int(int64_t(l - layer_begin) * units_per_layer + u), n_units++, 0, ld.evicts ? d / kTileRows : 0, 0,
+      Piece pc{l, int(int64_t(l - layer_begin) * units_per_layer + u), n_units++, 0, ld.evicts ? ctx->dp / kTileRows : 0, 0,
                int((ld.cap + kTileRows - 1) / kTileRows)};
       pieces.push_back(pc);
       total_w += pc.weight();
@@ -1210,8 +1236,8 @@ void build_stream_schedule(const glide_ctx *ctx, int layer_begin, int layer_coun
         sg.cap = int32_t(ld.cap);
         sg.w = int32_t(std::min<int64_t>(ld.w, INT32_MAX));
         sg.evicts = ld.evicts ? (ld.wlin == 0 ? 3 : 1) : 0;
-        sg.S_off256 = int32_t((ld.S + size_t(ub) * d * d * 4) / 256);
-        sg.z_off256 = int32_t((ld.z + size_t(ub) * d * 4) / 256);
+        sg.S_off256 = int32_t((ld.S + size_t(ub) * ctx->dp * d * 4) / 256);
+        sg.z_off256 = int32_t((ld.z + size_t(ub) * ctx->dp * 4) / 256);
         sg.ringK_off256 = int32_t(ld.ringK / 256);
         sg.ringV_off256 = int32_t(ld.ringV / 256);
         sg.g = int32_t(ub % Hkv);
@@ -1284,7 +1310,9 @@ void build_stream_schedule(const glide_ctx *ctx, int layer_begin, int layer_coun
 }
 
 int stream_decode_supported(const glide_ctx *ctx) {
-  return ctx->cfg.io_dtype == GLIDE_BF16 && ctx->cfg.head_dim == kD && ctx->cfg.phi == GLIDE_PHI_SOFTMAX && !ctx->cfg.gated;
+  // (the learned feature map with the shared normaliser only; the gated recurrence runs on the CUDA-core kernel)
+  return ctx->cfg.io_dtype == GLIDE_BF16 && ctx->cfg.head_dim == kD && !ctx->cfg.gated &&
+         (ctx->cfg.phi == GLIDE_PHI_SOFTMAX || ctx->cfg.merge == GLIDE_MERGE_SHARED);
 }
 
 // Host-only part of the set-up: every schedule of the context for a device with n_ctas SMs and smem_limit bytes of
@@ -1296,9 +1324,9 @@ int stream_decode_plan(glide_ctx *ctx, int n_ctas, size_t smem_limit) {
     for (int i = 1; i < ctx->G; ++i)
       contiguous = contiguous && ctx->heads_of[size_t(g) * ctx->G + i] == ctx->heads_of[size_t(g) * ctx->G] + i;
   ctx->stream_heads_contiguous = contiguous;
-  return dispatch_stream(ctx->G, ctx->cfg.merge != GLIDE_MERGE_SHARED, [&](auto gg, auto ss, auto mm) -> int {
+  return dispatch_stream(ctx->G, stream_mode(ctx), [&](auto gg, auto ss, auto mm) -> int {
     constexpr int G = decltype(gg)::value, S = decltype(ss)::value;
-    constexpr bool SUM = decltype(mm)::value != 0;
+    constexpr int SUM = decltype(mm)::value;   // the kernel's MODE
     // The record pool for the shared-memory groups takes what the segment table leaves, up to kStreamPoolBytes: with
     // many small units per CTA (large batches) the table is large and hardly any unit is shared between warps.
     const int rec_bytes = ctx->stream_rec_floats * 4;
@@ -1344,9 +1372,9 @@ int stream_decode_setup(glide_ctx *ctx) {
   }
   const int rc = stream_decode_plan(ctx, n_ctas, size_t(dev_max));
   if (rc) return rc;
-  return dispatch_stream(ctx->G, ctx->cfg.merge != GLIDE_MERGE_SHARED, [&](auto gg, auto ss, auto mm) -> int {
+  return dispatch_stream(ctx->G, stream_mode(ctx), [&](auto gg, auto ss, auto mm) -> int {
     constexpr int G = decltype(gg)::value, S = decltype(ss)::value;
-    constexpr bool SUM = decltype(mm)::value != 0;
+    constexpr int SUM = decltype(mm)::value;   // the kernel's MODE
     // the attribute belongs to the kernel, not to the context: ask for the device maximum so that contexts with
     // different schedules (different table sizes) can be alive together
     if (cudaFuncSetAttribute(glide_decode_stream_kernel<G, S, SUM, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -1371,9 +1399,9 @@ int launch_decode_stream(glide_ctx *ctx, const DecodeParams &p, int schedule, cu
   sp.heads_contiguous = ctx->stream_heads_contiguous ? 1 : 0;
   sp.kv4d = ctx->tmaps_kv4d ? 1 : 0;
   sp.t_off = int32_t(ctx->stream_smem - 1024 - size_t(ctx->stream_max_segs) * 8);
-  return dispatch_stream(ctx->G, ctx->cfg.merge != GLIDE_MERGE_SHARED, [&](auto gg, auto ss, auto mm) -> int {
+  return dispatch_stream(ctx->G, stream_mode(ctx), [&](auto gg, auto ss, auto mm) -> int {
     constexpr int G = decltype(gg)::value, S = decltype(ss)::value;
-    constexpr bool SUM = decltype(mm)::value != 0;
+    constexpr int SUM = decltype(mm)::value;   // the kernel's MODE
     cudaLaunchConfig_t cfg{};
     cfg.gridDim = dim3(unsigned(ctx->decode_grid));
     cfg.blockDim = dim3(kThreads);

@@ -101,6 +101,52 @@ __device__ __forceinline__ void warp_phi(float (&x)[E]) {
   for (int i = 0; i < E; ++i) x[i] *= inv;
 }
 
+// Projection of the learned feature map for N vectors held by a warp (lane: entries lane*E .. lane*E+E-1 of each):
+// y += (rows [il0*E, il1*E) of W)^T x, with the head's d x d matrix W read row by row (row i: 32 lanes x E consecutive
+// entries, coalesced).  The rows are fetched UB * E at a time into registers before any of them is used, so that
+// many loads are in flight per lane.  y is in the same lane layout.
+template <typename T, int D, int N, int UB>
+__device__ __forceinline__ void warp_project_rows(const T *W, const float (&x)[N][D / 32], float (&y)[N][D / 32],
+                                                  int il_begin, int il_end) {
+  constexpr int E = D / 32;
+  const int lane = threadIdx.x & 31;
+  for (int il0 = il_begin; il0 < il_end; il0 += UB) {
+    float w[UB * E][E];
+#pragma unroll
+    for (int u = 0; u < UB * E; ++u) load_elems<T, E>(W + size_t(il0 * E + u) * D + lane * E, w[u]);
+#pragma unroll
+    for (int u = 0; u < UB * E; ++u) {
+#pragma unroll
+      for (int n = 0; n < N; ++n) {
+        const float xi = __shfl_sync(0xffffffffu, x[n][u % E], il0 + u / E);
+#pragma unroll
+        for (int e = 0; e < E; ++e) y[n][e] = fmaf(xi, w[u][e], y[n][e]);
+      }
+    }
+  }
+}
+
+// Learned feature map of N vectors held by a warp: y = W^T x, then the two softmax halves; lo / hi receive
+// softmax(y) and softmax(-y) in the lane layout of x.
+template <typename T, int D, int N, int UB = 2>
+__device__ __forceinline__ void warp_phi_learned(const T *W, const float (&x)[N][D / 32], float (&lo)[N][D / 32],
+                                                 float (&hi)[N][D / 32]) {
+  constexpr int E = D / 32;
+  static_assert(32 % UB == 0, "batches of rows");
+#pragma unroll
+  for (int n = 0; n < N; ++n)
+#pragma unroll
+    for (int e = 0; e < E; ++e) lo[n][e] = 0.f;
+  warp_project_rows<T, D, N, UB>(W, x, lo, 0, 32);
+#pragma unroll
+  for (int n = 0; n < N; ++n) {
+#pragma unroll
+    for (int e = 0; e < E; ++e) hi[n][e] = -lo[n][e];
+    warp_phi<E>(lo[n]);
+    warp_phi<E>(hi[n]);
+  }
+}
+
 // One key/value row folded into a per-warp online softmax over G heads (log2 domain).
 template <int E, int G>
 __device__ __forceinline__ void online_row(const float (&qr)[G][E], const float (&kx)[E], const float (&vx)[E],

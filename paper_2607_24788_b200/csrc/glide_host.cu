@@ -675,7 +675,7 @@ int glide_device_status(glide_ctx *ctx, void *stream, int32_t *status_out) {
 
 int glide_decode_launch_info(glide_ctx *ctx, int32_t *n_launches, int32_t *n_work_items, int32_t *grid_size) {
   if (!ctx) return GLIDE_ERR_INVALID_ARG;
-  if (n_launches) *n_launches = 1;
+  if (n_launches) *n_launches = ctx->cfg.phi == GLIDE_PHI_PROJ_SOFTMAX2 ? 2 : 1;   // the feature kernel, then the step
   if (n_work_items) *n_work_items = ctx->decode_kind == 2 ? int32_t(ctx->stream_scheds[0].n_segs) : ctx->n_items;
   if (grid_size) *grid_size = ctx->decode_grid;
   return GLIDE_OK;

@@ -68,41 +68,6 @@ __device__ __forceinline__ RowSource<T> make_source(const PrefillParams &p, cons
   return s;
 }
 
-// Learned feature map of N rows held by a warp (lane: entries lane*E .. lane*E+E-1 of each row): y = W^T x with the
-// head's d x d matrix W read once for all N rows (row i of W: 32 lanes x E consecutive entries, coalesced), then the
-// two softmax halves.  lo / hi receive softmax(y) and softmax(-y) in the same lane layout.
-template <typename T, int D, int N>
-__device__ __forceinline__ void warp_phi_learned(const T *W, const float (&x)[N][D / 32], float (&lo)[N][D / 32],
-                                                 float (&hi)[N][D / 32]) {
-  constexpr int E = D / 32;
-  const int lane = threadIdx.x & 31;
-#pragma unroll
-  for (int n = 0; n < N; ++n)
-#pragma unroll
-    for (int e = 0; e < E; ++e) lo[n][e] = 0.f;
-#pragma unroll 4
-  for (int il = 0; il < 32; ++il) {
-#pragma unroll
-    for (int ie = 0; ie < E; ++ie) {
-      float w[E];
-      load_elems<T, E>(W + size_t(il * E + ie) * D + lane * E, w);
-#pragma unroll
-      for (int n = 0; n < N; ++n) {
-        const float xi = __shfl_sync(0xffffffffu, x[n][ie], il);
-#pragma unroll
-        for (int e = 0; e < E; ++e) lo[n][e] = fmaf(xi, w[e], lo[n][e]);
-      }
-    }
-  }
-#pragma unroll
-  for (int n = 0; n < N; ++n) {
-#pragma unroll
-    for (int e = 0; e < E; ++e) hi[n][e] = -lo[n][e];
-    warp_phi<E>(lo[n]);
-    warp_phi<E>(hi[n]);
-  }
-}
-
 // 1. phi of the delayed keys of this chunk: one warp per (unit, kTokPerWarp consecutive chunk tokens), the rows'
 // loads issued together (with one row per warp the kernel was bound by the latency of its single load)
 constexpr int kTokPerWarp = 4;

@@ -82,3 +82,50 @@ def test_feature_map_and_gate_argument_checks():
     with pytest.raises(glide.GlideError) as e:   # gated call on a context without gates
         plain.glide_decode_step_gated(q, k, k, None, torch.empty_like(q))
     assert e.value.code == glide.GLIDE_ERR_INVALID_ARG
+
+
+@pytest.mark.parametrize("G,B", [(4, 1), (1, 3), (8, 2)])
+def test_learned_map_on_the_streaming_kernel_units_cut_across_ctas(G, B):
+    """Windows long enough for units to be cut across warps and CTAs (global records, tickets, merges) with 16 state
+    tiles per unit; layers without a ring and layers that never evict; decode steps that cross a ring wrap."""
+    Hkv = 2
+    run_case([1500, 64, 0, 5000, 300], B, Hkv * G, Hkv, 128, BF16, [1490, 7], 12, amp=4 * 128 ** -0.5, seed=11 + G,
+             phi=1, check_prefill_outputs=False, decode_impl=glide.GLIDE_DECODE_STREAM)
+
+
+def test_learned_map_streaming_layer_by_layer_and_ragged_slots():
+    """glide_decode_step_layers (one schedule per layer) and slots of different lengths with the learned map."""
+    import numpy as np
+    from oracle import glide_oracle as orc
+    from paper_2607_24788_b200 import synth
+    from tests.parity_util import check_outputs, f32_scale, learned_phi_weights, to_np
+    windows, B, H, Hkv, d = [40, 0, 200], 2, 8, 2, 128
+    L = len(windows)
+    wq, wk = learned_phi_weights(L, H, Hkv, d, BF16, 5)
+    wl = synth.Workload(13, L, B, H, Hkv, d, BF16, 4 * d ** -0.5)
+    g = glide.Glide(windows, B, H, Hkv, d, 400, dtype=BF16, softmax_scale=f32_scale(d), phi=1, phi_wq=wq, phi_wk=wk)
+    cells = [[orc.Cell(H, Hkv, d, w, f32_scale(d), phi=1, wq=to_np(wq[l]), wk=to_np(wk[l])) for _ in range(B)]
+             for l, w in enumerate(windows)]
+    lens = [90, 33]
+    for b in range(B):   # slots prefilled one by one to different lengths
+        q, k, v = wl.qkv(range(L), [b], range(lens[b]), device="cuda")
+        g.glide_reset_seq(b)
+        g.glide_prefill_seq(b, None, k[:, 0], v[:, 0], None)
+        for l in range(L):
+            cells[l][b].prefill(None, to_np(k[l, 0]), to_np(v[l, 0]), outputs=False)
+    for s in range(6):
+        qs, ks, vs = [], [], []
+        for b in range(B):
+            q, k, v = wl.qkv(range(L), [b], [lens[b] + s], device="cuda")
+            qs.append(q[:, 0, 0]); ks.append(k[:, 0, 0]); vs.append(v[:, 0, 0])
+        q, k, v = (torch.stack(x, 1).contiguous() for x in (qs, ks, vs))     # [L][B][heads][d]
+        out = torch.full_like(q, float("nan"))
+        if s % 2 == 0:
+            g.glide_decode_step(q, k, v, out)
+        else:
+            for l in range(L):
+                g.glide_decode_step_layers(q[l:l + 1], k[l:l + 1], v[l:l + 1], out[l:l + 1], l, 1)
+        ref = np.stack([[cells[l][b].decode(to_np(q[l, b]), to_np(k[l, b]), to_np(v[l, b])) for b in range(B)]
+                        for l in range(L)])
+        check_outputs(out, ref, BF16, f"step {s}")
+    assert g.glide_device_status() == 0
