@@ -681,6 +681,9 @@ def main():
     ap.add_argument("--reps", type=int, default=15,
                     help="least number of repetitions of the K-step timed region (median reported; repeated further "
                          "until half a second of timed work has accumulated)")
+    ap.add_argument("--min-time", type=float, default=MIN_TIMED_S,
+                    help="seconds of timed work a figure accumulates at least (0: just --reps repetitions, for "
+                         "profiler captures)")
     ap.add_argument("--side-workloads", default="all",
                     help="'all', 'none' or a comma-separated list: the other configurations and controls timed after "
                          "the headline workload (one GPU only)")
@@ -705,6 +708,7 @@ def main():
     KERNEL_KNOBS.update(decode_chunk=args.decode_chunk, decode_state_splits=args.state_splits,
                         decode_impl=args.decode_impl, prefill_impl=args.prefill_impl, merge=args.merge)
     PHI["kind"] = args.phi
+    globals()["MIN_TIMED_S"] = args.min_time
     if args.impl == "reference":
         run_reference(args, shape)
     else:
