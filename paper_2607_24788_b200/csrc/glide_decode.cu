@@ -521,6 +521,8 @@ DecodeParams make_decode_params(const glide_ctx *ctx, int layer_begin, int layer
   p.gated = ctx->cfg.gated;
   p.gate = nullptr;
   p.tensors_absolute = ctx->decode_kind != 2;
+  if (++ctx->launch_seq == 0) ++ctx->launch_seq;
+  p.launch_tag = ctx->launch_seq;
   p.q = q;
   p.k = k;
   p.v = v;

@@ -16,9 +16,13 @@
 // The linear readout is folded into the softmax partial as a term with logit 0 (exact: the shared
 // normaliser's reference m* is max(window max, 0)), so a unit needs ONE (m, l, acc) record per warp.
 // A unit that lies inside one warp's range is finished by that warp alone (current token's own term,
-// normalise, write, ring append) without touching global scratch.  Only units cut by a range boundary
-// go through one global record per warp and a ticket; the warp holding the last ticket merges them.
-// No warp waits for another warp; the only waits are on the warp's own mbarriers, and are bounded.
+// normalise, write, ring append) without touching global scratch.  Units shared by warps of one CTA are
+// reduced in shared memory by the last of them to arrive.  Only units cut by a CTA boundary go through global
+// scratch: one record per CTA, every value stored beside the launch's tag in one 8-byte word, so that neither
+// a fence nor a counter is needed; the warp that holds the unit's last piece merges the records at the end of
+// its range, polling the words it is about to use until they carry the tag.  That poll is the only place where
+// a warp waits for another one (all CTAs of a launch are resident: one per SM); like the waits on the warp's
+// own mbarriers it is bounded, and a wait that runs out sets the context's status word.
 #include <cuda.h>
 
 #include <algorithm>
@@ -47,6 +51,9 @@ constexpr int kHdrSlots = 3;
 #define GLIDE_W_STATE 15
 #define GLIDE_W_WIN 10
 #define GLIDE_W_UNIT 27
+#endif
+#ifndef GLIDE_W_GROUP
+#define GLIDE_W_GROUP 0   // extra weight of a segment whose unit is shared with other warps of the CTA
 #endif
 #ifndef GLIDE_STREAM_FILL
 #define GLIDE_STREAM_FILL 100
@@ -160,6 +167,37 @@ __device__ __forceinline__ float4 lds_f32x4(uint32_t addr) {
 __device__ __forceinline__ void prefetch_tensormap(const void *tmap) {
   asm volatile("prefetch.tensormap [%0];" ::"l"(tmap) : "memory");
 }
+// ---- records of units cut across CTAs: every 4-byte value travels with the launch's tag in one 8-byte store ------
+// A 64-bit store is a single access, so a reader that sees the tag sees the value: no fence orders the record
+// before a ticket, and the reader needs no ticket either -- it polls the pairs it is about to use.
+__device__ __forceinline__ unsigned long long ll_pack(float v, uint32_t tag) {
+  return (static_cast<unsigned long long>(tag) << 32) | __float_as_uint(v);
+}
+__device__ __forceinline__ void ll_store2(unsigned long long *dst, float a, float b, uint32_t tag) {   // dst 16-byte aligned
+  asm volatile("st.relaxed.gpu.global.v2.u64 [%0], {%1, %2};" ::"l"(dst), "l"(ll_pack(a, tag)), "l"(ll_pack(b, tag)) : "memory");
+}
+__device__ __forceinline__ void ll_store1(unsigned long long *dst, float a, uint32_t tag) {
+  asm volatile("st.relaxed.gpu.global.u64 [%0], %1;" ::"l"(dst), "l"(ll_pack(a, tag)) : "memory");
+}
+__device__ __forceinline__ bool ll_load2(const unsigned long long *src, uint32_t tag, float &a, float &b) {
+  unsigned long long x, y;
+  asm volatile("ld.relaxed.gpu.global.v2.u64 {%0, %1}, [%2];" : "=l"(x), "=l"(y) : "l"(src) : "memory");
+  a = __uint_as_float(uint32_t(x));
+  b = __uint_as_float(uint32_t(y));
+  return uint32_t(x >> 32) == tag && uint32_t(y >> 32) == tag;
+}
+__device__ __forceinline__ bool ll_load1(const unsigned long long *src, uint32_t tag, float &a) {
+  unsigned long long x;
+  asm volatile("ld.relaxed.gpu.global.u64 %0, [%1];" : "=l"(x) : "l"(src) : "memory");
+  a = __uint_as_float(uint32_t(x));
+  return uint32_t(x >> 32) == tag;
+}
+__device__ __forceinline__ bool ll_load4(const unsigned long long *src, uint32_t tag, float4 &v) {   // four consecutive pairs
+  const bool a = ll_load2(src, tag, v.x, v.y);
+  const bool b = ll_load2(src + 2, tag, v.z, v.w);
+  return a && b;
+}
+
 // ---- schedule walking ------------------------------------------------------------------------
 __device__ __forceinline__ float ex2_approx(float x) {   // 2^x, 2 ulp, 2^-inf = 0
   float y;
@@ -521,7 +559,7 @@ glide_decode_stream_kernel(const DecodeParams p, const StreamParams sp) {
   };
 
   // ---- state tile: 16 rows of S and z, updated in the stage and stored back by the async proxy ---------
-  // (bulk stores are not ordered by this warp's later fences, so a ticket never waits for state traffic)
+  // (nothing later in the warp waits for these bulk stores except the wait for all of them before it exits)
   auto consume_state = [&](const StreamSegment &sg, int stile, float4 *st, float *zs, uint32_t st_addr, uint32_t z_addr,
                            const float *sphi) {
     const int src0 = stile * 4;   // lane that holds phi entries of the tile's first row (4 rows per lane)
@@ -631,7 +669,7 @@ glide_decode_stream_kernel(const DecodeParams p, const StreamParams sp) {
     if (s + 1 < seg_hi) issue_header(s + 1);
     // A parked slot (negative position; only batches with slot offsets have them) goes through the header hand-over
     // like every segment and then leaves: it has no tiles, and nothing of it is reduced or written.  All segments
-    // of a unit share the position, so its group counters and tickets stay untouched as well.
+    // of a unit share the position, so its group counters and records stay untouched as well.
     if (RAGGED && t < 0) continue;
     if (has_win) {
       const int64_t lim = t < int64_t(sg.cap) ? t : int64_t(sg.cap);
@@ -815,21 +853,27 @@ glide_decode_stream_kernel(const DecodeParams p, const StreamParams sp) {
       GLIDE_TRACE_EVENT(22);
     }
     if (sg.part >= 0) {
-      // the unit is cut by a CTA boundary: this record goes to global scratch; its ticket is taken
-      // at the end of the range, so that the streaming loop never stalls on a fence or an atomic
-      float *grec = p.partials + (size_t(sg.rec0) + sg.part) * p.rec_floats;
+      // the unit is cut by a CTA boundary: this CTA's record goes to global scratch, every value paired with the
+      // launch's tag.  The CTA that holds the unit's last piece merges the records at the end of this warp's range.
+      unsigned long long *grec = reinterpret_cast<unsigned long long *>(p.partials) + (size_t(sg.rec0) + sg.part) * p.rec_floats;
 #pragma unroll
       for (int h = 0; h < G; ++h) {
-        *reinterpret_cast<float4 *>(grec + h * kD + lane * 4) = acc[h];
-        if (SUM) *reinterpret_cast<float4 *>(grec + L::kRecW + h * kD + lane * 4) = a[h];
+        ll_store2(grec + h * kD + lane * 4, acc[h].x, acc[h].y, p.launch_tag);
+        ll_store2(grec + h * kD + lane * 4 + 2, acc[h].z, acc[h].w, p.launch_tag);
+        if (SUM) {
+          ll_store2(grec + L::kRecW + h * kD + lane * 4, a[h].x, a[h].y, p.launch_tag);
+          ll_store2(grec + L::kRecW + h * kD + lane * 4 + 2, a[h].z, a[h].w, p.launch_tag);
+        }
         if (lane == 0) {
-          grec[G * kD + h] = mh[h];
-          grec[G * kD + G + h] = lh[h];
-          if (SUM) grec[L::kRecW + G * kD + h] = bp[h];
+          ll_store1(grec + G * kD + h, mh[h], p.launch_tag);
+          ll_store1(grec + G * kD + G + h, lh[h], p.launch_tag);
+          if (SUM) ll_store1(grec + L::kRecW + G * kD + h, bp[h], p.launch_tag);
         }
       }
-      if (n_pending == 0) pend0 = s; else pend1 = s;
-      ++n_pending;
+      if (sg.part == sg.n_parts - 1) {
+        if (n_pending == 0) pend0 = s; else pend1 = s;
+        ++n_pending;
+      }
     } else {
       // the whole unit is in this range: current token's own term, shared normaliser, output row, ring append
       float vx[4];
@@ -866,27 +910,17 @@ glide_decode_stream_kernel(const DecodeParams p, const StreamParams sp) {
   }
   GLIDE_TRACE_EVENT(14);
 
-  // ---- tickets of the units this range shares with its neighbours; the last ticket of a unit merges -----
+  // ---- units whose last piece this range holds: merge the CTAs' records as they become visible -------------------
   if (n_pending > 0 && !failed) {
-    __threadfence();
-    __syncwarp();
-    int last = 0;
-    if (lane < n_pending) {
-      const StreamSegment &sg = sm_segs[lane == 0 ? pend0 : pend1];
-      last = atomicAdd(&p.tickets[sg.unit], 1) == sg.n_parts - 1;
-    }
-    const unsigned last_mask = __ballot_sync(0xffffffffu, last != 0);
     GLIDE_TRACE_EVENT(12);
-    for (int pi = 0; pi < n_pending; ++pi) {
-      if (!((last_mask >> pi) & 1u)) continue;
-      __threadfence();
+    for (int pi = 0; pi < n_pending && !failed; ++pi) {
       const StreamSegment &sg = sm_segs[pi == 0 ? pend0 : pend1];
       const bool has_win = sg.cap > 0;
       // reload the unit's query rows and current token (this warp may have moved on to another unit since);
       // every load of the merge's first batch is issued before anything is reduced
       const bf16 *qall = reinterpret_cast<const bf16 *>(p.q);
-      const float *r0 = p.partials + size_t(sg.rec0) * p.rec_floats;
-      constexpr int RPB = 32 / G;   // records per batch
+      const unsigned long long *r0 = reinterpret_cast<const unsigned long long *>(p.partials) + size_t(sg.rec0) * p.rec_floats;
+      constexpr int RPB = 16 / G;   // records per batch (every value arrives as an 8-byte pair: two registers)
       const uint2 ktb = *reinterpret_cast<const uint2 *>(reinterpret_cast<const bf16 *>(p.k) + size_t(sg.unit) * kD + lane * 4);
       const uint2 vtb = *reinterpret_cast<const uint2 *>(reinterpret_cast<const bf16 *>(p.v) + size_t(sg.unit) * kD + lane * 4);
       int orow[G];
@@ -896,18 +930,46 @@ glide_decode_stream_kernel(const DecodeParams p, const StreamParams sp) {
         orow[h] = sg.qrow0 + (sp.heads_contiguous ? h : p.heads_of[sg.g * G + h]);
         qbits[h] = *reinterpret_cast<const uint2 *>(qall + size_t(orow[h]) * kD + lane * 4);
       }
-      float me0, le0;
+      float me0 = -CUDART_INF_F, le0 = 0.f;
       float4 vv0[RPB][G];
-      {
-        const int ri = lane / G, rh = lane % G;
-        const bool valid = ri < sg.n_parts;
-        me0 = valid ? __ldcg(r0 + size_t(ri) * p.rec_floats + G * kD + rh) : -CUDART_INF_F;
-        le0 = valid ? __ldcg(r0 + size_t(ri) * p.rec_floats + G * kD + G + rh) : 0.f;
+      // one batch of records: polled until every pair this lane uses carries the launch's tag (bounded)
+      auto load_batch = [&](int i0, float &me, float &le) -> bool {
+        const int ri = i0 + lane / G, rh = lane % G;
+        const int nb = sg.n_parts - i0 < RPB ? sg.n_parts - i0 : RPB;
+        const bool mine = lane < RPB * G && ri < sg.n_parts;
+        // every load is issued before any tag is looked at (records past the unit's last one re-read the batch's first)
+        const unsigned long long *ml = r0 + size_t(mine ? ri : i0) * p.rec_floats + G * kD + rh;
+        for (uint32_t spins = 0;; ++spins) {
+          unsigned long long raw[RPB][G][4], rm, rl;
+          asm volatile("ld.relaxed.gpu.global.u64 %0, [%1];" : "=l"(rm) : "l"(ml));
+          asm volatile("ld.relaxed.gpu.global.u64 %0, [%1];" : "=l"(rl) : "l"(ml + G));
 #pragma unroll
-        for (int u = 0; u < RPB; ++u)
+          for (int u = 0; u < RPB; ++u)
 #pragma unroll
-          for (int h = 0; h < G; ++h)
-            if (u < sg.n_parts) vv0[u][h] = __ldcg(reinterpret_cast<const float4 *>(r0 + size_t(u) * p.rec_floats + h * kD + lane * 4));
+            for (int h = 0; h < G; ++h) {
+              const unsigned long long *src = r0 + size_t(u < nb ? i0 + u : i0) * p.rec_floats + h * kD + lane * 4;
+              asm volatile("ld.relaxed.gpu.global.v2.u64 {%0, %1}, [%2];" : "=l"(raw[u][h][0]), "=l"(raw[u][h][1]) : "l"(src));
+              asm volatile("ld.relaxed.gpu.global.v2.u64 {%0, %1}, [%2];" : "=l"(raw[u][h][2]), "=l"(raw[u][h][3]) : "l"(src + 2));
+            }
+          uint32_t diff = (uint32_t(rm >> 32) ^ p.launch_tag) | (uint32_t(rl >> 32) ^ p.launch_tag);
+#pragma unroll
+          for (int u = 0; u < RPB; ++u)
+#pragma unroll
+            for (int h = 0; h < G; ++h) {
+#pragma unroll
+              for (int c = 0; c < 4; ++c) diff |= uint32_t(raw[u][h][c] >> 32) ^ p.launch_tag;
+              vv0[u][h] = make_float4(__uint_as_float(uint32_t(raw[u][h][0])), __uint_as_float(uint32_t(raw[u][h][1])),
+                                      __uint_as_float(uint32_t(raw[u][h][2])), __uint_as_float(uint32_t(raw[u][h][3])));
+            }
+          me = mine ? __uint_as_float(uint32_t(rm)) : -CUDART_INF_F;
+          le = mine ? __uint_as_float(uint32_t(rl)) : 0.f;
+          if (__all_sync(0xffffffffu, diff == 0)) return true;
+          if (spins > (kWaitLimit >> 6)) return false;
+        }
+      };
+      if (!load_batch(0, me0, le0)) {
+        failed = true;
+        break;
       }
       float sc[G];
       {
@@ -940,16 +1002,9 @@ glide_decode_stream_kernel(const DecodeParams p, const StreamParams sp) {
         const int rh = lane % G;
         const int nb = sg.n_parts - i0 < RPB ? sg.n_parts - i0 : RPB;
         float me = me0, le = le0;
-        if (i0 > 0) {   // further batches (units cut into more than RPB records)
-          const int ri = i0 + lane / G;
-          const bool valid = ri < sg.n_parts;
-          me = valid ? __ldcg(r0 + size_t(ri) * p.rec_floats + G * kD + rh) : -CUDART_INF_F;
-          le = valid ? __ldcg(r0 + size_t(ri) * p.rec_floats + G * kD + G + rh) : 0.f;
-#pragma unroll
-          for (int u = 0; u < RPB; ++u)
-#pragma unroll
-            for (int h = 0; h < G; ++h)
-              if (u < nb) vv0[u][h] = __ldcg(reinterpret_cast<const float4 *>(r0 + size_t(i0 + u) * p.rec_floats + h * kD + lane * 4));
+        if (i0 > 0 && !load_batch(i0, me, le)) {   // further batches (units cut into more than RPB records)
+          failed = true;
+          break;
         }
         float Mn[G];
 #pragma unroll
@@ -992,7 +1047,6 @@ glide_decode_stream_kernel(const DecodeParams p, const StreamParams sp) {
       vx[1] = __uint_as_float(vtb.x & 0xffff0000u);
       vx[2] = __uint_as_float(vtb.y << 16);
       vx[3] = __uint_as_float(vtb.y & 0xffff0000u);
-#pragma unroll
       float4 al[G];
       float bl[G];
       if (SUM) {   // linear parts of all records: plain sums
@@ -1001,15 +1055,23 @@ glide_decode_stream_kernel(const DecodeParams p, const StreamParams sp) {
           al[h] = make_float4(0.f, 0.f, 0.f, 0.f);
           bl[h] = 0.f;
         }
-        for (int i = 0; i < sg.n_parts; ++i) {
+        for (int i = 0; i < sg.n_parts && !failed; ++i) {
 #pragma unroll
           for (int h = 0; h < G; ++h) {
-            const float4 av = __ldcg(reinterpret_cast<const float4 *>(r0 + size_t(i) * p.rec_floats + L::kRecW + h * kD + lane * 4));
+            float4 av;
+            float bv;
+            uint32_t spins = 0;   // (the window half of the record carried the tag already: these follow at once)
+            while (!__all_sync(0xffffffffu, ll_load4(r0 + size_t(i) * p.rec_floats + L::kRecW + h * kD + lane * 4, p.launch_tag, av) &&
+                                                ll_load1(r0 + size_t(i) * p.rec_floats + L::kRecW + G * kD + h, p.launch_tag, bv)))
+              if (++spins > (kWaitLimit >> 6)) {
+                failed = true;
+                break;
+              }
             al[h].x += av.x;
             al[h].y += av.y;
             al[h].z += av.z;
             al[h].w += av.w;
-            bl[h] += __ldcg(r0 + size_t(i) * p.rec_floats + L::kRecW + G * kD + h);
+            bl[h] += bv;
           }
         }
       }
@@ -1034,7 +1096,6 @@ glide_decode_stream_kernel(const DecodeParams p, const StreamParams sp) {
         reinterpret_cast<uint2 *>(reinterpret_cast<bf16 *>(p.ws + size_t(sg.ringK_off256) * 256) + row)[lane] = ktb;
         reinterpret_cast<uint2 *>(reinterpret_cast<bf16 *>(p.ws + size_t(sg.ringV_off256) * 256) + row)[lane] = vtb;
       }
-      if (lane == 0) p.tickets[sg.unit] = 0;
       GLIDE_TRACE_EVENT(13);
     }
   }
@@ -1083,9 +1144,10 @@ int dispatch_stream(int G, int mode, F &&f) {
 //   1. Units (layer x sequence x KV head) are packed whole into CTAs, heaviest first onto the least loaded CTA;
 //      a unit heavier than a CTA's share is first cut into equal pieces.  So almost every unit lives inside one
 //      CTA and is reduced in shared memory; only the oversized ones need global records and a merge.
-//   2. Inside a CTA the list of pieces is cut into 8 contiguous, equally heavy ranges, one per warp.
+//   2. Inside a CTA the list of pieces is cut into 8 contiguous ranges, one per warp, whose heaviest is as light as
+//      a cut at tile boundaries allows (bisection on the limit of a greedy split).
 // Schedule for the layers [layer_begin, layer_begin + layer_count).  Units and query rows are numbered relative to
-// the first layer of the range (that is how a launch for the range addresses q, k, v, out and the tickets); the
+// the first layer of the range (that is how a launch for the range addresses q, k, v and out); the
 // layer index itself stays absolute (descriptors, layer table).
 void build_stream_schedule(const glide_ctx *ctx, int layer_begin, int layer_count, int n_ranges, int pool_slots,
                            std::vector<StreamSegment> *segs, std::vector<int32_t> *range_seg_begin, int *max_segs_per_cta,
@@ -1135,15 +1197,21 @@ void build_stream_schedule(const glide_ctx *ctx, int layer_begin, int layer_coun
   //     cut at cumulative targets, so that what one CTA leaves unused goes to the next one instead of piling up
   //     on the last; only these units need global records and a merge
   size_t oi = 0;
+  int n_heavy_ctas = 0;
+  int64_t heavy_slack = 0;
   {
     int64_t heavy_w = 0;
     size_t n_heavy = 0;
     while (n_heavy < order.size() && pieces[order[n_heavy]].weight() > cta_share) heavy_w += pieces[order[n_heavy++]].weight();
-    // these CTAs end with a ticket + merge chain of a few microseconds: they get less than a full share
+    // these CTAs end with the merge of their units' records: they may be given less than a full share
     const int64_t heavy_share = std::max<int64_t>(1, cta_share * GLIDE_STREAM_FILL / 100);
     const int n_h = int(std::max<int64_t>(1, std::min<int64_t>(n_used, (heavy_w + heavy_share / 2) / heavy_share)));
     // every CTA boundary inside a unit opens one more piece with its own fixed cost
     const int64_t target = (heavy_w + int64_t(n_h) * kSegWeight) / n_h + 1;
+    if (n_heavy > 0) {
+      n_heavy_ctas = n_h;
+      heavy_slack = cta_share - heavy_share;
+    }
     int cta = 0;
     int64_t cum = 0;   // weight laid out so far over all heavy CTAs
     for (; oi < n_heavy; ++oi) {
@@ -1179,7 +1247,8 @@ void build_stream_schedule(const glide_ctx *ctx, int layer_begin, int layer_coun
   }
   // CTAs beyond n_used stay empty
   for (size_t c = size_t(n_used); c < cta_load.size(); ++c) cta_load[c] = INT64_MAX / 2;
-  // (b) every other unit goes whole onto the least loaded CTA
+  // (b) every other unit goes whole onto the least loaded CTA (the share the heavy CTAs leave unused is not on offer)
+  for (int c = 0; c < n_heavy_ctas; ++c) cta_load[size_t(c)] += heavy_slack;
   for (; oi < order.size(); ++oi) {
     size_t best = 0;
     for (size_t c = 1; c < cta_load.size(); ++c)
@@ -1188,49 +1257,92 @@ void build_stream_schedule(const glide_ctx *ctx, int layer_begin, int layer_coun
     cta_load[best] += pieces[order[oi]].weight();
   }
   for (size_t c = size_t(n_used); c < cta_load.size(); ++c) cta_load[c] = 0;
+  for (int c = 0; c < n_heavy_ctas; ++c) cta_load[size_t(c)] -= heavy_slack;
 
   segs->clear();
   range_seg_begin->assign(size_t(n_ranges) + 1, 0);
   std::vector<std::vector<size_t>> unit_segs;
   unit_segs.resize(size_t(n_units));
   std::vector<int> seg_range;
-  for (int cta = 0; cta < n_ctas; ++cta) {
-    const std::vector<size_t> &list = cta_pieces[size_t(cta)];
-    // the CTA's pieces cut into kWarps contiguous ranges; every range boundary inside a piece adds a segment
-    const int64_t cta_total = cta_load[size_t(cta)] + int64_t(kWarps) * kSegWeight;
+  // Runs of tiles of one piece: what a segment covers.
+  struct Run {
+    size_t piece;
+    int st0, nst, w0, nw;
+  };
+  // The CTA's pieces cut into kWarps contiguous ranges whose heaviest is as light as possible: for a limit on a warp's
+  // weight every warp takes, in order, whole pieces while they fit and then as many tiles of the next piece as fit
+  // (a piece shared by several warps costs every one of them a record and a place in the reduction); the smallest
+  // limit that places all tiles is found by bisection.
+  constexpr int64_t kGroupWeight = GLIDE_W_GROUP;
+  auto split_cta = [&](const std::vector<size_t> &list, int64_t limit, std::vector<std::vector<Run>> *out) -> bool {
     size_t pi = 0;
     int st_done = 0, w_done = 0;
-    int64_t cum = 0;
+    if (out) out->assign(size_t(kWarps), {});
+    for (int wi = 0; wi < kWarps && pi < list.size(); ++wi) {
+      int64_t cum = 0;
+      bool empty = true;
+      while (pi < list.size()) {
+        const Piece &pc = pieces[list[pi]];
+        const int rem_st = pc.nst - st_done, rem_w = pc.nw - w_done;
+        const bool begun = st_done > 0 || w_done > 0;
+        const int64_t whole = kSegWeight + (begun ? kGroupWeight : 0) + kStateWeight * rem_st + kWinWeight * rem_w;
+        Run r{list[pi], pc.st0 + st_done, rem_st, pc.w0 + w_done, rem_w};
+        bool full = false;
+        if (cum + whole > limit && wi + 1 < kWarps) {
+          int64_t room = limit - cum - kSegWeight - kGroupWeight;
+          r.nst = int(std::max<int64_t>(0, std::min<int64_t>(rem_st, room / kStateWeight)));
+          room -= kStateWeight * int64_t(r.nst);
+          r.nw = r.nst == rem_st ? int(std::max<int64_t>(0, std::min<int64_t>(rem_w, room / kWinWeight))) : 0;
+          if (r.nst + r.nw < (empty ? 1 : 2)) {   // a tile more does not fit (and one alone is not worth a segment)
+            if (empty) return false;
+            break;
+          }
+          full = true;
+        } else if (cum + whole > limit) {
+          return false;   // the last warp would have to take more than the limit
+        }
+        empty = false;
+        cum += kSegWeight + ((begun || full) ? kGroupWeight : 0) + kStateWeight * r.nst + kWinWeight * r.nw;
+        if (out) (*out)[size_t(wi)].push_back(r);
+        st_done += r.nst;
+        w_done += r.nw;
+        if (st_done == pc.nst && w_done == pc.nw) {
+          ++pi;
+          st_done = w_done = 0;
+        }
+        if (full) break;
+      }
+    }
+    return pi == list.size();
+  };
+  for (int cta = 0; cta < n_ctas; ++cta) {
+    const std::vector<size_t> &list = cta_pieces[size_t(cta)];
+    std::vector<std::vector<Run>> runs;
+    runs.resize(size_t(kWarps));
+    if (!list.empty()) {
+      int64_t hi = 0;
+      for (size_t i : list) hi += pieces[i].weight() + kGroupWeight;
+      int64_t lo = hi / kWarps;   // lo - 1 is not enough, hi always is (one warp takes everything)
+      while (lo < hi) {
+        const int64_t mid = lo + (hi - lo) / 2;
+        if (split_cta(list, mid, nullptr)) hi = mid; else lo = mid + 1;
+      }
+      split_cta(list, hi, &runs);
+    }
     for (int wi = 0; wi < kWarps; ++wi) {
       const int c = cta * kWarps + wi;
       (*range_seg_begin)[size_t(c)] = int32_t(segs->size());
-      // an equal share of what is left, so that a range that stops short does not load up the last warp
-      const int64_t target = (wi + 1 == kWarps) ? INT64_MAX : cum + (std::max<int64_t>(cta_total - cum, 0) + (kWarps - wi) - 1) / (kWarps - wi);
-      bool first = true;
-      while (pi < list.size() && cum < target) {
-        const Piece &pc = pieces[list[pi]];
+      for (const Run &r : runs[size_t(wi)]) {
+        const Piece &pc = pieces[r.piece];
         const LayerDev &ld = ctx->layers[pc.layer];
-        const int64_t rem = kStateWeight * (pc.nst - st_done) + kWinWeight * (pc.nw - w_done);
-        int64_t room = target == INT64_MAX ? INT64_MAX / 4 : target - cum - kSegWeight;
         StreamSegment sg{};
-        if (rem <= room + cta_total / (kWarps * 8)) {   // finishing the piece here overshoots by little: keep it whole
-          sg.n_state = pc.nst - st_done;
-          sg.n_win = pc.nw - w_done;
-        } else {
-          if (!first && room < 2 * kWinWeight) break;   // not worth opening a segment for a tile or two
-          room = std::max<int64_t>(room, 1);
-          sg.n_state = int(std::min<int64_t>(pc.nst - st_done, (room + kStateWeight - 1) / kStateWeight));
-          room -= kStateWeight * int64_t(sg.n_state);
-          sg.n_win = (st_done + sg.n_state == pc.nst)
-                         ? int(std::min<int64_t>(pc.nw - w_done, (std::max<int64_t>(room, 0) + kWinWeight - 1) / kWinWeight))
-                         : 0;
-        }
-        first = false;
+        sg.n_state = r.nst;
+        sg.n_win = r.nw;
         sg.unit = pc.unit;
         sg.layer = pc.layer;
         sg.range = wi;
-        sg.state0 = pc.st0 + st_done;
-        sg.win0 = pc.w0 + w_done;
+        sg.state0 = r.st0;
+        sg.win0 = r.w0;
         const int64_t ub = pc.unit - int64_t(pc.layer - layer_begin) * units_per_layer;
         sg.row_base = int32_t(ub * ld.cap);
         sg.cap = int32_t(ld.cap);
@@ -1246,16 +1358,9 @@ void build_stream_schedule(const glide_ctx *ctx, int layer_begin, int layer_coun
           const int64_t row = (int64_t(pc.layer - layer_begin) * B + b) * ctx->cfg.n_q_heads;
           sg.qrow0 = int32_t(row + (contiguous_heads ? ctx->heads_of[size_t(sg.g) * ctx->G] : 0));
         }
-        st_done += sg.n_state;
-        w_done += sg.n_win;
-        cum += kSegWeight + kStateWeight * int64_t(sg.n_state) + kWinWeight * int64_t(sg.n_win);
         unit_segs[size_t(pc.uidx)].push_back(segs->size());
         seg_range.push_back(c);
         segs->push_back(sg);
-        if (st_done == pc.nst && w_done == pc.nw) {
-          ++pi;
-          st_done = w_done = 0;
-        }
       }
     }
   }

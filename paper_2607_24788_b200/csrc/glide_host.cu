@@ -175,7 +175,8 @@ int glide::plan_context(const glide_config *cfg, glide_ctx *ctx, std::vector<Wor
   // the all-layer schedule plus one schedule per layer (glide_decode_step_layers)
   ctx->stream_rec_capacity = size_t(L) * units_per_layer + size_t(kMaxStreamCtas) * kStreamWarps;
   ctx->stream_seg_capacity = 2 * size_t(L) * units_per_layer + size_t(L + 1) * kMaxStreamCtas * kStreamWarps;
-  part_floats = std::max(part_floats, ctx->stream_rec_capacity * size_t(ctx->stream_rec_floats));
+  // (the streaming kernel stores every value of a cross-CTA record beside the launch's tag: 8 bytes per value)
+  part_floats = std::max(part_floats, 2 * ctx->stream_rec_capacity * size_t(ctx->stream_rec_floats));
   off = align_up(off + sizeof(float) * part_floats, 256);
   ctx->off_stream_segs = off;
   off = align_up(off + sizeof(StreamSegment) * ctx->stream_seg_capacity, 256);
@@ -354,8 +355,9 @@ int glide_create(const glide_config *cfg, void *dev_workspace, size_t workspace_
                            sizeof(StreamSegment) * ctx->stream_segs.size(), cudaMemcpyHostToDevice, st) == cudaSuccess &&
            true;
     }
-    // control words, counters, tickets, S and z start at zero
+    // control words, counters, tickets, S and z start at zero; so do the records (no launch has the tag 0)
     ok = ok && cudaMemsetAsync(ctx->ws, 0, ctx->off_layers, st) == cudaSuccess &&
+         cudaMemsetAsync(ctx->ws + ctx->off_partials, 0, ctx->off_stream_segs - ctx->off_partials, st) == cudaSuccess &&
          cudaMemsetAsync(ctx->ws + ctx->off_seqoff, 0, sizeof(int64_t) * size_t(ctx->cfg.batch), st) == cudaSuccess &&
          cudaMemsetAsync(ctx->ws + ctx->off_tickets, 0, ctx->off_partials - ctx->off_tickets, st) == cudaSuccess &&
          cudaMemsetAsync(ctx->ws + ctx->off_state, 0, ctx->state_bytes, st) == cudaSuccess;

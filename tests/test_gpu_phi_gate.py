@@ -86,7 +86,7 @@ def test_feature_map_and_gate_argument_checks():
 
 @pytest.mark.parametrize("G,B", [(4, 1), (1, 3), (8, 2)])
 def test_learned_map_on_the_streaming_kernel_units_cut_across_ctas(G, B):
-    """Windows long enough for units to be cut across warps and CTAs (global records, tickets, merges) with 16 state
+    """Windows long enough for units to be cut across warps and CTAs (global records and their merges) with 16 state
     tiles per unit; layers without a ring and layers that never evict; decode steps that cross a ring wrap."""
     Hkv = 2
     run_case([1500, 64, 0, 5000, 300], B, Hkv * G, Hkv, 128, BF16, [1490, 7], 12, amp=4 * 128 ** -0.5, seed=11 + G,

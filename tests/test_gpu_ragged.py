@@ -245,7 +245,7 @@ def test_ragged_random_schedules(seed):
 
 def test_ragged_llama_shape_long_sequences_sampled_layers():
     """Config-1 shapes (32 layers, H = 32, H_kv = 8, d = 128) with four sequences of very different lengths: heavy
-    units are cut across CTAs and merged through tickets while every sequence sits at its own position.  The oracle
+    units are cut across CTAs and merged through global records while every sequence sits at its own position.  The oracle
     follows one layer of every window size."""
     from paper_2607_24788_b200 import configs as C
     windows = list(C.C1.windows)

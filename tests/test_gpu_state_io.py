@@ -117,8 +117,8 @@ def _run_sequence(windows, B, H, Hkv, d, dtype, prompt, steps, seed, **kw):
     dict(merge=glide.GLIDE_MERGE_SUM_EVICTED),
 ])
 def test_same_steps_on_two_contexts_give_the_same_bits(kw):
-    """Config 1's window schedule at batch 1 (units heavier than a CTA's share, cut across CTAs and merged by the
-    last ticket; units shared by the warps of a CTA; units inside one warp) with a prompt that fills the windows."""
+    """Config 1's window schedule at batch 1 (units heavier than a CTA's share, cut across CTAs and merged from
+    their global records; units shared by the warps of a CTA; units inside one warp) with a prompt that fills the windows."""
     windows = [4096] * 2 + [1024] * 3 + [256] * 5 + [64] * 4
     args = (windows, 1, 32, 8, 128, BF16, 4200, 6, 31)
     a = _run_sequence(*args, **kw)
