@@ -192,6 +192,12 @@ __device__ __forceinline__ bool ll_load1(const unsigned long long *src, uint32_t
   a = __uint_as_float(uint32_t(x));
   return uint32_t(x >> 32) == tag;
 }
+// 8-byte load that stays where it is written (ahead of the polling loop it is meant to overlap with)
+__device__ __forceinline__ uint2 ld_u2_pinned(const void *src) {
+  uint2 v;
+  asm volatile("ld.global.v2.u32 {%0, %1}, [%2];" : "=r"(v.x), "=r"(v.y) : "l"(src));
+  return v;
+}
 __device__ __forceinline__ bool ll_load4(const unsigned long long *src, uint32_t tag, float4 &v) {   // four consecutive pairs
   const bool a = ll_load2(src, tag, v.x, v.y);
   const bool b = ll_load2(src + 2, tag, v.z, v.w);
@@ -232,6 +238,11 @@ __device__ __forceinline__ int seg_valid_win(const StreamSegment &s, int64_t t) 
 }
 
 // A position in the warp's range: segment, tile within the segment, and the segment's tile counts.
+// ring slot of position t (t >= 0): 32-bit arithmetic while the position allows it (a 64-bit remainder is a call)
+__device__ __forceinline__ int slot_of(int64_t t, int cap) {
+  return t <= int64_t(0x7fffffff) ? int(uint32_t(t) % uint32_t(cap)) : int(t % int64_t(cap));
+}
+
 struct Cursor {
   int seg;
   int k;          // next tile of the segment: [0, n_state_eff) state tiles, then window tiles
@@ -408,7 +419,7 @@ glide_decode_stream_kernel(const DecodeParams p, const StreamParams sp) {
           bulk_load(my_hdr + G * 256, kt, 256, hdr_bar);
           bulk_load(my_hdr + G * 256 + 256, vt, 256, hdr_bar);
         } else {
-          const size_t row = (size_t(sg.row_base) + size_t(t % int64_t(sg.cap))) * kD;
+          const size_t row = (size_t(sg.row_base) + size_t(slot_of(t, sg.cap))) * kD;
           bulk_load(my_hdr + G * 256, reinterpret_cast<const bf16 *>(p.ws + size_t(sg.ringK_off256) * 256) + row, 256, hdr_bar);
           bulk_load(my_hdr + G * 256 + 256, reinterpret_cast<const bf16 *>(p.ws + size_t(sg.ringV_off256) * 256) + row, 256, hdr_bar);
         }
@@ -674,7 +685,7 @@ glide_decode_stream_kernel(const DecodeParams p, const StreamParams sp) {
     if (has_win) {
       const int64_t lim = t < int64_t(sg.cap) ? t : int64_t(sg.cap);
       win_end = int(lim);
-      win_cur = int(t % int64_t(sg.cap));
+      win_cur = slot_of(t, sg.cap);
     }
 #pragma unroll
     for (int mt = 0; mt < KS; ++mt) o[mt][0] = o[mt][1] = o[mt][2] = o[mt][3] = 0.f;
@@ -921,14 +932,14 @@ glide_decode_stream_kernel(const DecodeParams p, const StreamParams sp) {
       const bf16 *qall = reinterpret_cast<const bf16 *>(p.q);
       const unsigned long long *r0 = reinterpret_cast<const unsigned long long *>(p.partials) + size_t(sg.rec0) * p.rec_floats;
       constexpr int RPB = 16 / G;   // records per batch (every value arrives as an 8-byte pair: two registers)
-      const uint2 ktb = *reinterpret_cast<const uint2 *>(reinterpret_cast<const bf16 *>(p.k) + size_t(sg.unit) * kD + lane * 4);
-      const uint2 vtb = *reinterpret_cast<const uint2 *>(reinterpret_cast<const bf16 *>(p.v) + size_t(sg.unit) * kD + lane * 4);
+      const uint2 ktb = ld_u2_pinned(reinterpret_cast<const bf16 *>(p.k) + size_t(sg.unit) * kD + lane * 4);
+      const uint2 vtb = ld_u2_pinned(reinterpret_cast<const bf16 *>(p.v) + size_t(sg.unit) * kD + lane * 4);
       int orow[G];
       uint2 qbits[G];
 #pragma unroll
       for (int h = 0; h < G; ++h) {
         orow[h] = sg.qrow0 + (sp.heads_contiguous ? h : p.heads_of[sg.g * G + h]);
-        qbits[h] = *reinterpret_cast<const uint2 *>(qall + size_t(orow[h]) * kD + lane * 4);
+        qbits[h] = ld_u2_pinned(qall + size_t(orow[h]) * kD + lane * 4);
       }
       float me0 = -CUDART_INF_F, le0 = 0.f;
       float4 vv0[RPB][G];
@@ -971,6 +982,7 @@ glide_decode_stream_kernel(const DecodeParams p, const StreamParams sp) {
         failed = true;
         break;
       }
+      GLIDE_TRACE_EVENT(15);
       float sc[G];
       {
         float kx[4];
@@ -989,6 +1001,7 @@ glide_decode_stream_kernel(const DecodeParams p, const StreamParams sp) {
 #pragma unroll
         for (int h = 0; h < G; ++h) sc[h] = has_win ? sc[h] * p.scale_log2 : -CUDART_INF_F;
       }
+      GLIDE_TRACE_EVENT(16);
       // merge the records: maxima and sums first (one (record, head) pair per lane), then the vectors
       float Mg[G], lg[G];
       float4 acc[G];
@@ -1042,6 +1055,7 @@ glide_decode_stream_kernel(const DecodeParams p, const StreamParams sp) {
               acc[h].w = fmaf(vv0[u][h].w, f, acc[h].w);
             }
       }
+      GLIDE_TRACE_EVENT(17);
       float vx[4];
       vx[0] = __uint_as_float(vtb.x << 16);
       vx[1] = __uint_as_float(vtb.x & 0xffff0000u);
@@ -1092,7 +1106,7 @@ glide_decode_stream_kernel(const DecodeParams p, const StreamParams sp) {
         *reinterpret_cast<uint2 *>(reinterpret_cast<bf16 *>(p.out) + size_t(orow[h]) * kD + lane * 4) = packed;
       }
       if (has_win) {
-        const size_t row = (size_t(sg.row_base) + size_t(pos_of(pi == 0 ? pend0 : pend1) % int64_t(sg.cap))) * kD;
+        const size_t row = (size_t(sg.row_base) + size_t(slot_of(pos_of(pi == 0 ? pend0 : pend1), sg.cap))) * kD;
         reinterpret_cast<uint2 *>(reinterpret_cast<bf16 *>(p.ws + size_t(sg.ringK_off256) * 256) + row)[lane] = ktb;
         reinterpret_cast<uint2 *>(reinterpret_cast<bf16 *>(p.ws + size_t(sg.ringV_off256) * 256) + row)[lane] = vtb;
       }
