@@ -183,7 +183,8 @@ int glide::plan_context(const glide_config *cfg, glide_ctx *ctx, std::vector<Wor
   ctx->off_stream_cta = off;
   off = align_up(off + sizeof(int32_t) * (size_t(kMaxStreamCtas) * kStreamWarps + 1), 256);
   ctx->off_tmaps = off;
-  off = align_up(off + size_t(128) * 5 * L, 256);   // per layer 3 maps of 16-row boxes, then (from 3 L on) 2 of 128-row boxes
+  // per layer 3 maps of 16-row boxes, then (from 3 L on) 2 of 128-row boxes, then the two bf16 scratch arrays of prefill
+  off = align_up(off + size_t(128) * (5 * L + 2), 256);
   ctx->off_phik = off;
   off = align_up(off + sizeof(float) * size_t(L) * units_per_layer * ctx->prefill_chunk * dp, 256);
   ctx->off_zcum = off;   // running sums of phi(K') over the chunk: only the sum-of-terms merges use them
@@ -194,6 +195,14 @@ int glide::plan_context(const glide_config *cfg, glide_ctx *ctx, std::vector<Wor
     off = align_up(off + sizeof(float) * size_t(L) * units_per_layer * dp * (ctx->G + 1), 256);
   ctx->off_gcum = off;   // gated: running sums of log(gate) over the chunk's delayed tokens
   if (cfg->gated) off = align_up(off + sizeof(float) * size_t(L) * units_per_layer * ctx->prefill_chunk, 256);
+  // tcgen05 prefill kernel (bf16, head_dim 128, plain feature map): bf16 copies of the chunk's phi(K') rows and of S,
+  // which its CTAs fetch by TMA instead of converting the fp32 arrays themselves
+  if (cfg->io_dtype == GLIDE_BF16 && d == 128 && cfg->phi == GLIDE_PHI_SOFTMAX && !cfg->gated) {
+    ctx->off_phik16 = off;
+    off = align_up(off + 2 * size_t(L) * units_per_layer * ctx->prefill_chunk * d, 256);
+    ctx->off_s16 = off;
+    off = align_up(off + 2 * size_t(L) * units_per_layer * d * d, 256);
+  }
   ctx->off_seqoff = off;   // per-sequence position offsets
   off = align_up(off + sizeof(int64_t) * size_t(cfg->batch), 256);
   // the streamed arrays start on a 2 MiB boundary of the workspace whatever the sizes of the small tables before

@@ -103,6 +103,11 @@ __global__ void __launch_bounds__(kPrefillThreads) prefill_phi_kernel(const Pref
       float *dst = p.phik + (size_t(u) * p.Cmax + i0 + r) * D + lane * E;
 #pragma unroll
       for (int e = 0; e < E; ++e) dst[e] = x[r][e];
+      if (p.phik16) {   // the same row rounded to bf16 for the tensor-core attention kernel
+        __nv_bfloat16 *d16 = reinterpret_cast<__nv_bfloat16 *>(p.phik16) + (size_t(u) * p.Cmax + i0 + r) * D + lane * E;
+#pragma unroll
+        for (int e = 0; e < E; ++e) d16[e] = __float2bfloat16_rn(x[r][e]);
+      }
     }
   } else {
 #pragma unroll
@@ -518,6 +523,27 @@ __global__ void __launch_bounds__(kPrefillThreads) prefill_ring_kernel(const Pre
   }
 }
 
+// bf16 copy of the state of every unit of the call as it is before the chunk's state update: what the tcgen05 attention
+// kernel multiplies phi(Q) with (one 16-byte store per thread)
+__global__ void __launch_bounds__(kPrefillThreads) prefill_s16_kernel(const PrefillParams p) {
+  constexpr int D = 128;
+  const int64_t id = int64_t(blockIdx.x) * kPrefillThreads + threadIdx.x;   // 8 consecutive entries of one unit's S
+  const int64_t per_unit = D * D / 8;
+  const int64_t u = id / per_unit;
+  if (u >= int64_t(p.layer_count) * p.B * p.Hkv) return;
+  const int g = int(u % p.Hkv);
+  const int b = int((u / p.Hkv) % p.B);
+  const int lrel = int(u / (int64_t(p.Hkv) * p.B));
+  const LayerDev ld = p.layers[p.layer_begin + lrel];
+  if (!ld.evicts) return;
+  const size_t e0 = size_t(id % per_unit) * 8;
+  const float *src = reinterpret_cast<const float *>(p.ws + ld.S) + (size_t(b + p.b0) * p.Hkv + g) * D * D + e0;
+  const float4 f0 = *reinterpret_cast<const float4 *>(src), f1 = *reinterpret_cast<const float4 *>(src + 4);
+  __nv_bfloat162 o[4] = {__floats2bfloat162_rn(f0.x, f0.y), __floats2bfloat162_rn(f0.z, f0.w),
+                         __floats2bfloat162_rn(f1.x, f1.y), __floats2bfloat162_rn(f1.z, f1.w)};
+  *reinterpret_cast<uint4 *>(reinterpret_cast<__nv_bfloat16 *>(p.s16) + size_t(u) * D * D + e0) = *reinterpret_cast<const uint4 *>(o);
+}
+
 }  // namespace
 
 int launch_prefill(glide_ctx *ctx, int layer_begin, int layer_count, int64_t T, const void *q, const void *k,
@@ -561,6 +587,8 @@ int launch_prefill(glide_ctx *ctx, int layer_begin, int layer_count, int64_t T, 
   // the tcgen05 kernel needs the ring descriptors of the tensor-core decode kernels (absent when decode_impl asks
   // for the CUDA-core kernel); without them the call uses the mma.sync kernel
   const bool use_tc = impl == GLIDE_PREFILL_TCGEN05 && prefill_attn_tc_supported(ctx);
+  p.phik16 = use_tc && out ? ctx->ws + ctx->off_phik16 : nullptr;
+  p.s16 = use_tc && out ? ctx->ws + ctx->off_s16 : nullptr;
   // (the mma.sync kernel has the shared normaliser only: the other merges fall through to the CUDA-core kernel)
   const bool use_mma = (impl == GLIDE_PREFILL_MMA_SYNC || (impl == GLIDE_PREFILL_TCGEN05 && !use_tc)) &&
                        prefill_attn_mma_supported(ctx) && ctx->cfg.merge == GLIDE_MERGE_SHARED;
@@ -585,6 +613,8 @@ int launch_prefill(glide_ctx *ctx, int layer_begin, int layer_count, int64_t T, 
         prefill_gcum_kernel<TT, D><<<unsigned((units + kPrefillThreads - 1) / kPrefillThreads), kPrefillThreads, 0, stream>>>(p);
       if (out) {
         if (use_tc) {
+          if (any_evicts)
+            prefill_s16_kernel<<<unsigned((units * (128 * 128 / 8) + kPrefillThreads - 1) / kPrefillThreads), kPrefillThreads, 0, stream>>>(p);
           if (any_evicts && p.merge != GLIDE_MERGE_SHARED)
             prefill_zcum_kernel<D><<<unsigned((units * D + kPrefillThreads - 1) / kPrefillThreads), kPrefillThreads, 0, stream>>>(p);
           if (launch_prefill_attn_tc(ctx, p, stream) != GLIDE_OK) return GLIDE_ERR_CUDA;

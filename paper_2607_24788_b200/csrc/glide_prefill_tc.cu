@@ -206,6 +206,21 @@ __device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&r)[16
       : "memory");
 }
 
+#ifdef GLIDE_PF_CLOCKS
+// debug builds only: clock cycles per phase of thread 0 of every CTA, summed over the CTAs ([8] phases, [8] = CTAs)
+__device__ unsigned long long g_pf_clk[16];
+#define PF_CLK(i)                                                   \
+  do {                                                              \
+    if (threadIdx.x == 0) {                                         \
+      const long long now_ = clock64();                             \
+      atomicAdd(&g_pf_clk[i], (unsigned long long)(now_ - pf_t_));  \
+      pf_t_ = now_;                                                 \
+    }                                                               \
+  } while (0)
+#else
+#define PF_CLK(i) do { } while (0)
+#endif
+
 struct Smem {
   unsigned char q[2][kTileBytes];        // Q_A, Q_B; later phi(Q) 2^-m*
   unsigned char kv[kStages][kTileBytes]; // K and V tiles in turn; linear part: bf16 state, phi(K') tile, V' tile
@@ -217,7 +232,9 @@ struct Smem {
   uint64_t bar_p[2];                     // P_X of the current tile is in TMEM (128 arrivals)
   uint64_t bar_done;                     // every window MMA has completed
   uint64_t bar_lin;                      // linear part: the MMAs issued so far have completed
-  uint64_t bar_state;                    // S (fp32) and z of the unit have landed
+  uint64_t bar_state;                    // the bf16 copy of S and z of the unit have landed
+  uint64_t bar_pk[2];                    // the phi(K') tile of an intra-chunk step has landed (even / odd steps)
+  uint64_t bar_vp[2];                    // the V' tile of the first / second intra-chunk step has landed (2 arrivals)
   uint32_t tmem_base;
   int failed;
 };
@@ -258,6 +275,10 @@ prefill_attn_tc_kernel(const PrefillParams p, const CUtensorMap *ring_maps, cons
   const size_t unit_rows = (size_t(b + p.b0) * p.Hkv + g) * size_t(ld.cap);   // b + b0: the sequence's slot in the context
   const size_t seq = (size_t(lrel) * p.B + b) * size_t(p.T);
   volatile int *failed = &sm.failed;
+#ifdef GLIDE_PF_CLOCKS
+  long long pf_t_ = clock64();
+  if (threadIdx.x == 0) atomicAdd(&g_pf_clk[8], 1ull);
+#endif
 
   // a time-out recorded by an earlier CTA ends the launch quickly
   if (*reinterpret_cast<volatile int32_t *>(&p.ctl->status) == kDevWaitTimeout) return;
@@ -281,6 +302,10 @@ prefill_attn_tc_kernel(const PrefillParams p, const CUtensorMap *ring_maps, cons
     mbar_init(smem_u32(&sm.bar_done), 1);
     mbar_init(smem_u32(&sm.bar_lin), 1);
     mbar_init(smem_u32(&sm.bar_state), 1);
+    mbar_init(smem_u32(&sm.bar_pk[0]), 1);
+    mbar_init(smem_u32(&sm.bar_pk[1]), 1);
+    mbar_init(smem_u32(&sm.bar_vp[0]), 2);
+    mbar_init(smem_u32(&sm.bar_vp[1]), 2);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     sm.failed = 0;
   }
@@ -301,22 +326,61 @@ prefill_attn_tc_kernel(const PrefillParams p, const CUtensorMap *ring_maps, cons
       for (int i = tid; i < n16; i += kThreads) dst[i] = make_uint4(0u, 0u, 0u, 0u);
     }
   }
+  // Q_X: 128 rows x 16 chunks by the 128 threads of each row tile, asked for before the set-up's barrier so that the copy
+  // runs while the other warps finish setting up (it needs nothing of that; nothing else writes these tiles).
+  {
+    const int Xq = (tid >> 7) & 1, rq = tid & 127;
+    const int ntokXq = Xq ? ntokB : ntokA;
+    if (tid < kSoftmaxThreads && ntokXq > 0) {
+      const bf16 *qbase = reinterpret_cast<const bf16 *>(p.q) + (seq + size_t(p.c0 + tok0 + Xq * TOKT)) * p.H * kD;
+      const uint32_t sQx = smem_u32(sm.q[Xq]);
+#pragma unroll 4
+      for (int i = 0; i < kRows * 16 / kRows; ++i) {
+        const int id = rq + kRows * i;
+        const int r = id >> 4, c = id & 15;
+        const int tk = r / G, h2 = r - tk * G;
+        const bool valid = tk < ntokXq;
+        cp_async16(sQx + sw128(r, c), qbase + (size_t(valid ? tk : 0) * p.H + p.heads_of[g * G + h2]) * kD + c * 8, valid);
+      }
+      cp_async_commit();
+    }
+  }
   fence_async_smem();
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = sm.tmem_base;
+  PF_CLK(0);
   const uint32_t sQ[2] = {smem_u32(sm.q[0]), smem_u32(sm.q[1])};
   const uint32_t sKV0 = smem_u32(sm.kv[0]);
   auto kv_addr = [&](int slot) { return sKV0 + uint32_t(slot) * kTileBytes; };
+  // Linear part: what it needs is known now, so that the loader can fetch it behind the last key tiles.
+  const bool linear = ld.evicts && tq_last >= wl;
+  const int64_t folded = p.n0 + p.c0 - wl;   // tokens below this index are in S, z at the start of the chunk
+  const bool need_state = linear && folded > 0;
+  // intra-chunk steps: delayed tokens of this chunk up to the CTA's last token, 128 at a time
+  const int i_lo = folded < 0 ? int(-folded < int64_t(p.C) ? -folded : int64_t(p.C)) : 0;
+  const int i_hi = tok0 + ntok - 1;
+  const int it0 = i_lo & ~(kKT - 1);
+  const int n_itiles = (linear && it0 <= i_hi) ? (i_hi - it0) / kKT + 1 : 0;
   // Roles of the five buffers after the window loop, by the order in which the loop stops using them (load number
-  // 2 n_tiles - 5 + k; a negative number is a buffer the loop never used): the two that come free first receive the
-  // unit's fp32 state (64 KiB, bulk-copied while the last key tiles are still being processed), the others hold the
-  // bf16 state tile, the phi(K') tile and the V' tile of the linear part.
+  // 2 n_tiles - 5 + k; a negative number is a buffer the loop never used): the first to come free receives the bf16
+  // copy of the unit's state, the next two the phi(K') tiles of the first two intra-chunk steps (all three by TMA
+  // while the last key tiles are still being processed), the last two the V' tiles of those steps.  Later steps
+  // take the buffers of the step before the previous one.
   auto late_seq = [&](int k) { return 2 * n_tiles - kStages + k; };
   auto late_slot = [&](int k) { const int sq = late_seq(k); return sq >= 0 ? sq % kStages : sq + kStages; };
-  const int slotS0 = late_slot(0), slotS1 = late_slot(1), slotSb = late_slot(2), slotPk = late_slot(3), slotV = late_slot(4);
-  const bool need_state = ld.evicts && tq_last >= wl && p.n0 + p.c0 - wl > 0;
+  const int slotSb = late_slot(0);
+  const int slotPk[2] = {late_slot(1), late_slot(2)}, slotVp[2] = {late_slot(3), late_slot(4)};
+  const CUtensorMap *map_pk = ring_maps + 5 * p.L, *map_s16 = map_pk + 1;
+  auto load_pk = [&](int t) {   // one thread: the phi(K') rows of intra-chunk step t
+    const uint32_t bar = smem_u32(&sm.bar_pk[t & 1]);
+    const uint32_t dst = kv_addr(slotPk[t & 1]);
+    const int y = int(u * p.Cmax) + it0 + t * kKT;
+    mbar_expect_tx(bar, kTileBytes);
+    tma_load_2d(dst, map_pk, 0, y, bar);
+    tma_load_2d(dst + kBoxBytes, map_pk, 64, y, bar);
+  };
 
   // ---- softmax threads: per-row state that lives across the window and the linear part ----------------------
   const int X = (tid >> 7) & 1;                   // row tile of this thread (softmax warps only)
@@ -377,18 +441,7 @@ prefill_attn_tc_kernel(const PrefillParams p, const CUtensorMap *ring_maps, cons
   // =========================== window part: warp-specialised ===========================
   if (tid < kSoftmaxThreads) {
     if (activeX) {
-      // Q_X: 128 rows x 16 chunks by the 128 threads of the row tile
-      const bf16 *qbase = reinterpret_cast<const bf16 *>(p.q) + (seq + size_t(p.c0 + tok0 + X * TOKT)) * p.H * kD;
-#pragma unroll 4
-      for (int i = 0; i < kRows * 16 / kRows; ++i) {
-        const int id = row + kRows * i;
-        const int r = id >> 4, c = id & 15;
-        const int tk = r / G, h2 = r - tk * G;
-        const bool valid = tk < ntokX;
-        cp_async16(sQ[X] + sw128(r, c), qbase + (size_t(valid ? tk : 0) * p.H + p.heads_of[g * G + h2]) * kD + c * 8, valid);
-      }
-      cp_async_commit();
-      cp_async_wait_all();
+      cp_async_wait_all();   // Q_X (asked for before the set-up's barrier) has landed
       fence_async_smem();
       mbar_arrive(smem_u32(&sm.bar_q[X]));
 
@@ -484,124 +537,140 @@ prefill_attn_tc_kernel(const PrefillParams p, const CUtensorMap *ring_maps, cons
     // arithmetic of the groups runs in parallel.  A group that straddles the call boundary or a ring wrap is copied
     // row by row by the whole warp (at most a few per tile).  Each buffer's barrier takes two arrivals: the
     // expect-tx one before the TMA boxes are issued and a plain one after the row copies.
-    if (n_tiles > 0) {
-      const CUtensorMap *ringK = ring_maps + 3 * layer, *ringV = ringK + 1;
-      const CUtensorMap *ringK128 = ring_maps + 3 * p.L + 2 * layer, *ringV128 = ringK128 + 1;
-      const bf16 *ringKp = reinterpret_cast<const bf16 *>(p.ws + ld.ringK) + unit_rows * kD;
-      const bf16 *ringVp = reinterpret_cast<const bf16 *>(p.ws + ld.ringV) + unit_rows * kD;
-      const bf16 *callKp = reinterpret_cast<const bf16 *>(p.k) + (seq * p.Hkv + g) * kD;
-      const bf16 *callVp = reinterpret_cast<const bf16 *>(p.v) + (seq * p.Hkv + g) * kD;
-      const int64_t call_stride = int64_t(p.Hkv) * kD;
-      const int gi = lane;
-      bool ok = true;
-      for (int sq = 0; sq < 2 * n_tiles; ++sq) {
-        const int t = sq >> 1, slot = sq % kStages;
-        const bool is_v = sq & 1;
-        if (sq >= kStages) ok = mbar_wait(smem_u32(&sm.bar_free[slot]), uint32_t(sq / kStages - 1) & 1u, failed);
-        if (!__all_sync(0xffffffffu, ok)) break;
-        const int64_t j0 = j_lo + int64_t(t) * kKT;
-        const int64_t left = tq_last - j0;                       // >= 0: the tile holds at least one valid token
-        const int ngroups = left >= kKT - 1 ? kKT / kGroup : int(left / kGroup) + 1;
-        const uint32_t bar = smem_u32(&sm.bar_full[slot]);
-        // A full tile that lies in one source without a wrap takes two boxes of 128 rows (the layout in shared memory
-        // is that of eight 16-row boxes).  Tiles that reach past the CTA's last token keep the 16-row path, which
-        // never loads a later token's row.
-        {
-          const uint32_t slot_row0 = (j0 >> 32) == 0 ? uint32_t(j0) % cap : uint32_t(uint64_t(j0) % cap);
-          const bool all_call = j0 >= p.n0;
-          const bool all_ring = j0 + kKT <= p.n0 && slot_row0 + kKT <= cap;
-          // (left >= kKT - 1: every row of the tile is a token up to the CTA's last one; eight groups alone would also
-          // admit a last group that is only partly valid)
-          if (left >= kKT - 1 && (all_call || all_ring)) {
-            if (lane == 0) {
-              mbar_expect_tx(bar, kTileBytes);
-              const uint32_t dst = kv_addr(slot);
-              if (all_call) {
-                const CUtensorMap *m = is_v ? &cm.v128 : &cm.k128;
-                tma_load_4d(dst, m, 0, g, int(j0 - p.n0), lrel * p.B + b, bar);
-                tma_load_4d(dst + kBoxBytes, m, 64, g, int(j0 - p.n0), lrel * p.B + b, bar);
-              } else {
-                const CUtensorMap *m = is_v ? ringV128 : ringK128;
-                const int y = int(unit_rows + slot_row0);
-                tma_load_2d(dst, m, 0, y, bar);
-                tma_load_2d(dst + kBoxBytes, m, 64, y, bar);
-              }
-              mbar_arrive(bar);   // the barrier's second arrival (after the row copies on the other path)
+    const CUtensorMap *ringK = ring_maps + 3 * layer, *ringV = ringK + 1;
+    const CUtensorMap *ringK128 = ring_maps + 3 * p.L + 2 * layer, *ringV128 = ringK128 + 1;
+    const bf16 *ringKp = reinterpret_cast<const bf16 *>(p.ws + ld.ringK) + unit_rows * kD;
+    const bf16 *ringVp = reinterpret_cast<const bf16 *>(p.ws + ld.ringV) + unit_rows * kD;
+    const bf16 *callKp = reinterpret_cast<const bf16 *>(p.k) + (seq * p.Hkv + g) * kD;
+    const bf16 *callVp = reinterpret_cast<const bf16 *>(p.v) + (seq * p.Hkv + g) * kD;
+    const int64_t call_stride = int64_t(p.Hkv) * kD;
+    const int gi = lane;
+    // Rows of tokens j0 .. j0 + 127 (K or V) into buffer `slot` (the whole warp); rows of tokens below 0 are zero;
+    // 16-row groups that lie wholly above j_max are zero too (zero_rest) or not written at all.  j0 need
+    // not be a multiple of the box size: a ring row or a token of the call is a TMA coordinate like any other.
+    auto load_tile = [&](int64_t j0, bool is_v, int slot, uint32_t bar, int64_t j_max, bool zero_rest) {
+      const int64_t left = j_max - j0;                         // >= 0: the tile holds at least one valid token
+      const int ngroups = left >= kKT - 1 ? kKT / kGroup : int(left / kGroup) + 1;
+      // A full tile that lies in one source without a wrap takes two boxes of 128 rows (the layout in shared memory
+      // is that of eight 16-row boxes).  Tiles that reach past the last token keep the 16-row path, which never
+      // loads a later token's row.
+      if (j0 >= 0) {
+        const uint32_t slot_row0 = (j0 >> 32) == 0 ? uint32_t(j0) % cap : uint32_t(uint64_t(j0) % cap);
+        const bool all_call = j0 >= p.n0;
+        const bool all_ring = j0 + kKT <= p.n0 && slot_row0 + kKT <= cap;
+        // (left >= kKT - 1: every row of the tile is a token up to the last one; eight groups alone would also
+        // admit a last group that is only partly valid)
+        if (left >= kKT - 1 && (all_call || all_ring)) {
+          if (lane == 0) {
+            mbar_expect_tx(bar, kTileBytes);
+            const uint32_t dst = kv_addr(slot);
+            if (all_call) {
+              const CUtensorMap *m = is_v ? &cm.v128 : &cm.k128;
+              tma_load_4d(dst, m, 0, g, int(j0 - p.n0), lrel * p.B + b, bar);
+              tma_load_4d(dst + kBoxBytes, m, 64, g, int(j0 - p.n0), lrel * p.B + b, bar);
+            } else {
+              const CUtensorMap *m = is_v ? ringV128 : ringK128;
+              const int y = int(unit_rows + slot_row0);
+              tma_load_2d(dst, m, 0, y, bar);
+              tma_load_2d(dst + kBoxBytes, m, 64, y, bar);
             }
-            continue;
+            mbar_arrive(bar);   // the barrier's second arrival (after the row copies on the other path)
           }
+          return;
         }
-        // this lane's group: where it comes from and whether one box covers it
-        const int64_t j = j0 + gi * kGroup;
-        const bool mine = gi < ngroups;
-        const bool from_call = j >= p.n0;
-        const uint32_t slot_row = (j >> 32) == 0 ? uint32_t(j) % cap : uint32_t(uint64_t(j) % cap);
-        const bool boxed = mine && (from_call || (j + kGroup <= p.n0 && slot_row + kGroup <= cap));
-        const unsigned boxed_mask = __ballot_sync(0xffffffffu, boxed);
-        const unsigned manual_mask = __ballot_sync(0xffffffffu, mine && !boxed);
-        if (lane == 0) mbar_expect_tx(bar, uint32_t(__popc(boxed_mask)) * 2u * kGroupBytes);
-        __syncwarp();
-        if (boxed) {
-          const uint32_t dst = kv_addr(slot) + uint32_t(gi) * kGroupBytes;
-          if (from_call) {
-            const CUtensorMap *m = is_v ? &cm.v : &cm.k;
-            tma_load_4d(dst, m, 0, g, int(j - p.n0), lrel * p.B + b, bar);
-            tma_load_4d(dst + kBoxBytes, m, 64, g, int(j - p.n0), lrel * p.B + b, bar);
-          } else {
-            const CUtensorMap *m = is_v ? ringV : ringK;
-            const int y = int(unit_rows + slot_row);
-            tma_load_2d(dst, m, 0, y, bar);
-            tma_load_2d(dst + kBoxBytes, m, 64, y, bar);
-          }
+      }
+      // this lane's group: where it comes from and whether one box covers it
+      const int64_t j = j0 + gi * kGroup;
+      const bool mine = gi < kKT / kGroup && (zero_rest || gi < ngroups);
+      const bool from_call = j >= p.n0;
+      const uint32_t slot_row = j < 0 ? 0u : ((j >> 32) == 0 ? uint32_t(j) % cap : uint32_t(uint64_t(j) % cap));
+      const bool boxed = mine && gi < ngroups && j >= 0 && (from_call || (j + kGroup <= p.n0 && slot_row + kGroup <= cap));
+      const unsigned boxed_mask = __ballot_sync(0xffffffffu, boxed);
+      const unsigned manual_mask = __ballot_sync(0xffffffffu, mine && !boxed);
+      if (lane == 0) mbar_expect_tx(bar, uint32_t(__popc(boxed_mask)) * 2u * kGroupBytes);
+      __syncwarp();
+      if (boxed) {
+        const uint32_t dst = kv_addr(slot) + uint32_t(gi) * kGroupBytes;
+        if (from_call) {
+          const CUtensorMap *m = is_v ? &cm.v : &cm.k;
+          tma_load_4d(dst, m, 0, g, int(j - p.n0), lrel * p.B + b, bar);
+          tma_load_4d(dst + kBoxBytes, m, 64, g, int(j - p.n0), lrel * p.B + b, bar);
+        } else {
+          const CUtensorMap *m = is_v ? ringV : ringK;
+          const int y = int(unit_rows + slot_row);
+          tma_load_2d(dst, m, 0, y, bar);
+          tma_load_2d(dst + kBoxBytes, m, 64, y, bar);
         }
-        for (unsigned mm = manual_mask; mm; mm &= mm - 1) {
-          const int gm = __ffs(int(mm)) - 1;
-          unsigned char *tile = sm.kv[slot];
+      }
+      for (unsigned mm = manual_mask; mm; mm &= mm - 1) {
+        const int gm = __ffs(int(mm)) - 1;
+        unsigned char *tile = sm.kv[slot];
 #pragma unroll
-          for (int i = 0; i < kGroup * 16 / 32; ++i) {
-            const int id = lane + 32 * i;
-            const int r = id >> 4, c = id & 15;
-            const int64_t jj = j0 + gm * kGroup + r;
-            uint4 val = make_uint4(0u, 0u, 0u, 0u);
-            if (jj <= tq_last) {
-              const bf16 *src = jj >= p.n0 ? (is_v ? callVp : callKp) + size_t(jj - p.n0) * call_stride
-                                           : (is_v ? ringVp : ringKp) + size_t(uint64_t(jj) % cap) * kD;
-              val = *reinterpret_cast<const uint4 *>(src + c * 8);
-            }
-            *reinterpret_cast<uint4 *>(tile + sw128(gm * kGroup + r, c)) = val;
+        for (int i = 0; i < kGroup * 16 / 32; ++i) {
+          const int id = lane + 32 * i;
+          const int r = id >> 4, c = id & 15;
+          const int64_t jj = j0 + gm * kGroup + r;
+          uint4 val = make_uint4(0u, 0u, 0u, 0u);
+          if (jj >= 0 && jj <= j_max) {
+            const bf16 *src = jj >= p.n0 ? (is_v ? callVp : callKp) + size_t(jj - p.n0) * call_stride
+                                         : (is_v ? ringVp : ringKp) + size_t(uint64_t(jj) % cap) * kD;
+            val = *reinterpret_cast<const uint4 *>(src + c * 8);
           }
+          *reinterpret_cast<uint4 *>(tile + sw128(gm * kGroup + r, c)) = val;
         }
-        fence_async_smem();   // the row copies are read by the tensor core (async proxy)
-        __syncwarp();
-        if (lane == 0) mbar_arrive(bar);
+      }
+      fence_async_smem();   // the row copies are read by the tensor core (async proxy)
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar);
+    };
+    bool ok = true;
+    for (int sq = 0; sq < 2 * n_tiles; ++sq) {
+      const int t = sq >> 1, slot = sq % kStages;
+      if (sq >= kStages) ok = mbar_wait(smem_u32(&sm.bar_free[slot]), uint32_t(sq / kStages - 1) & 1u, failed);
+      if (!__all_sync(0xffffffffu, ok)) break;
+      load_tile(j_lo + int64_t(t) * kKT, sq & 1, slot, smem_u32(&sm.bar_full[slot]), tq_last, false);
+    }
+    if (lane == 0 && linear && !*failed) {
+      // the linear part's operands into the buffers the window loop leaves first: the bf16 state (with z), then the
+      // phi(K') tiles of the first two intra-chunk steps
+      const int n_late = 1 + (n_itiles < 2 ? n_itiles : 2);
+      for (int k = 0; k < n_late; ++k) {
+        const int sq = late_seq(k);
+        if (sq >= 0 && !mbar_wait(smem_u32(&sm.bar_free[sq % kStages]), uint32_t(sq / kStages) & 1u, failed)) break;
+        if (k == 0) {
+          if (!need_state) continue;
+          const int ub = (b + p.b0) * p.Hkv + g;
+          const uint32_t bar = smem_u32(&sm.bar_state);
+          mbar_expect_tx(bar, kTileBytes + uint32_t(kD * sizeof(float)));
+          tma_load_2d(kv_addr(slotSb), map_s16, 0, int(u * kD), bar);
+          tma_load_2d(kv_addr(slotSb) + kBoxBytes, map_s16, 64, int(u * kD), bar);
+          bulk_load(smem_u32(sm.z), p.ws + ld.z + size_t(ub) * kD * sizeof(float), uint32_t(kD * sizeof(float)), bar);
+        } else {
+          load_pk(k - 1);
+        }
       }
     }
-    if (lane == 0 && need_state && !*failed) {
-      // S (fp32) and z as they are at the start of the chunk, into the two buffers the window loop leaves first
-      bool ok = true;
-      for (int k = 0; k < 2 && ok; ++k) {
-        const int sq = late_seq(k);
-        if (sq >= 0) ok = mbar_wait(smem_u32(&sm.bar_free[sq % kStages]), uint32_t(sq / kStages) & 1u, failed);
-      }
-      if (ok) {
-        const int ub = (b + p.b0) * p.Hkv + g;
-        const unsigned char *Sg = p.ws + ld.S + size_t(ub) * kD * kD * sizeof(float);
-        const uint32_t bar = smem_u32(&sm.bar_state);
-        mbar_expect_tx(bar, uint32_t(kD * kD * sizeof(float) + kD * sizeof(float)));
-        for (int i = 0; i < 4; ++i)
-          bulk_load(kv_addr(i < 2 ? slotS0 : slotS1) + uint32_t(i & 1) * 16384u, Sg + size_t(i) * 16384, 16384u, bar);
-        bulk_load(smem_u32(sm.z), p.ws + ld.z + size_t(ub) * kD * sizeof(float), uint32_t(kD * sizeof(float)), bar);
-      }
+    __syncwarp();
+    // the V rows of the delayed tokens of the first two intra-chunk steps, behind the window loop's last tiles (the
+    // rows of tokens that do not exist yet, below 0, are zero: their weights are, and 0 x anything must stay 0)
+    for (int t = 0; t < n_itiles && t < 2 && __all_sync(0xffffffffu, ok && !*failed); ++t) {
+      const int sq = late_seq(3 + t);
+      if (sq >= 0) ok = mbar_wait(smem_u32(&sm.bar_free[sq % kStages]), uint32_t(sq / kStages) & 1u, failed);
+      if (!__all_sync(0xffffffffu, ok)) break;
+      load_tile(folded + it0 + int64_t(t) * kKT, true, slotVp[t], smem_u32(&sm.bar_vp[t]), tq_last, true);
     }
   }
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
 
+  PF_CLK(1);
   // =========================== linear part: the whole CTA in step ===========================
   // (no early exits from here on: every thread passes the same __syncthreads; after a time-out the waits return
   // at once and the results are discarded)
-  const bool linear = ld.evicts && tq_last >= wl;
+  // Operands: phi(Q) 2^-M from the softmax threads; the bf16 state and the phi(K') tiles by TMA (issued by the loader
+  // behind the window loop, see above); the delayed tokens' V rows row by row (they come from the ring or from the
+  // call, with a wrap or the call boundary anywhere) by the loader as well, with the key tiles' own routine.
   bool o_init = n_tiles > 0;   // O_X holds a valid accumulation (uniform over the CTA)
   uint32_t lin_phase = 0;
   const int mma_tid = kMmaWarp * 32;
@@ -611,7 +680,26 @@ prefill_attn_tc_kernel(const PrefillParams p, const CUtensorMap *ring_maps, cons
     tc_fence_after();
   };
   if (linear) {
-    const int64_t folded = p.n0 + p.c0 - wl;   // tokens below this index are in S, z at the start of the chunk
+    const bf16 *ringV = reinterpret_cast<const bf16 *>(p.ws + ld.ringV) + unit_rows * kD;
+    const bf16 *callV = reinterpret_cast<const bf16 *>(p.v) + (seq * p.Hkv + g) * kD;
+    const int64_t call_stride = int64_t(p.Hkv) * kD;
+    auto load_vp = [&](int t) {   // softmax threads, steps after the second: V rows of the delayed tokens (MN-major), zero where none
+      const int i0 = it0 + t * kKT;
+      const uint32_t dst = kv_addr(slotVp[t & 1]);
+#pragma unroll 4
+      for (int i = 0; i < kKT * 16 / kSoftmaxThreads; ++i) {
+        const int id = tid + kSoftmaxThreads * i;
+        const int r = id >> 4, c = id & 15;
+        const int ii = i0 + r;
+        const bool valid = ii >= i_lo && ii <= i_hi;
+        const int64_t jj = valid ? folded + ii : 0;
+        const bool from_call = jj >= p.n0;
+        const uint32_t slot_row = (jj >> 32) == 0 ? uint32_t(jj) % cap : uint32_t(uint64_t(jj) % cap);
+        const bf16 *src = from_call ? callV + size_t(jj - p.n0) * call_stride : ringV + size_t(slot_row) * kD;
+        cp_async16(dst + sw128(r, c), src + c * 8, valid);
+      }
+      cp_async_commit();
+    };
     uint32_t phq[kD / 2];                      // phi(q) 2^-m* of this row, packed bf16
     if (activeX) {
       // Any common reference M >= m_ref gives the same quotient O / l.  M = max(m_ref, 0) would rescale O for every
@@ -680,82 +768,39 @@ prefill_attn_tc_kernel(const PrefillParams p, const CUtensorMap *ring_maps, cons
       for (int c = 0; c < 16; ++c)
         *reinterpret_cast<uint4 *>(sm.q[X] + sw128(row, c)) = make_uint4(phq[c * 4], phq[c * 4 + 1], phq[c * 4 + 2], phq[c * 4 + 3]);
     }
-    if (folded > 0 && tid < kSoftmaxThreads) {
-      // bf16 copy of the state as the MN-major B tile of the inter-chunk product
-      mbar_wait(smem_u32(&sm.bar_state), 0u, failed);
-#pragma unroll 4
-      for (int i = 0; i < kD * 16 / kSoftmaxThreads; ++i) {
-        const int id = tid + kSoftmaxThreads * i;
-        const int r = id >> 4, c = id & 15;
-        const float *Sg = reinterpret_cast<const float *>(sm.kv[r < 64 ? slotS0 : slotS1]) + size_t(r & 63) * kD;
-        const float4 f0 = *reinterpret_cast<const float4 *>(Sg + c * 8);
-        const float4 f1 = *reinterpret_cast<const float4 *>(Sg + c * 8 + 4);
-        *reinterpret_cast<uint4 *>(sm.kv[slotSb] + sw128(r, c)) =
-            make_uint4(pack_bf16x2(f0.x, f0.y), pack_bf16x2(f0.z, f0.w), pack_bf16x2(f1.x, f1.y), pack_bf16x2(f1.z, f1.w));
-      }
-    }
+    PF_CLK(10);
     fence_async_smem();
     tc_fence_before();
     __syncthreads();
-    if (folded > 0) {
-      if (tid == mma_tid) {
-        tc_fence_after();
+    PF_CLK(2);
+    // inter-chunk product into O and the first intra-chunk C in one batch
+    if (tid == mma_tid) {
+      tc_fence_after();
+      if (need_state) {
+        mbar_wait(smem_u32(&sm.bar_state), 0u, failed);
         issue_mma(tmem + 256, sQ[0], kv_addr(slotSb), true, o_init);
         if (hasB) issue_mma(tmem + 384, sQ[1], kv_addr(slotSb), true, o_init);
-        mma_commit(smem_u32(&sm.bar_lin));
       }
-      if (activeX) {
-        float dot = 0.f;
-#pragma unroll
-        for (int i = 0; i < kD / 2; ++i)
-          dot += __uint_as_float(phq[i] << 16) * sm.z[2 * i] + __uint_as_float(phq[i] & 0xffff0000u) * sm.z[2 * i + 1];
-        if (!sum_terms) l_sum += dot;
+      if (n_itiles > 0) {
+        mbar_wait(smem_u32(&sm.bar_pk[0]), 0u, failed);
+        issue_mma(tmem, sQ[0], kv_addr(slotPk[0]), false, false);   // C_X = (phi(Q_X) 2^-m*) phi(K')^T
+        if (hasB) issue_mma(tmem + 128, sQ[1], kv_addr(slotPk[0]), false, false);
       }
-      wait_lin();
-      o_init = true;
+      if (need_state || n_itiles > 0) mma_commit(smem_u32(&sm.bar_lin));
     }
-    // intra-chunk: delayed tokens of this chunk up to the CTA's last token, 128 at a time
-    const int i_lo = folded < 0 ? int(-folded < int64_t(p.C) ? -folded : int64_t(p.C)) : 0;
-    const int i_hi = tok0 + ntok - 1;
-    const float *pkp = p.phik + size_t(u) * p.Cmax * kD;
-    const bf16 *ringV = reinterpret_cast<const bf16 *>(p.ws + ld.ringV) + unit_rows * kD;
-    const bf16 *callV = reinterpret_cast<const bf16 *>(p.v) + (seq * p.Hkv + g) * kD;
-    const int64_t call_stride = int64_t(p.Hkv) * kD;
-    for (int i0 = i_lo & ~(kKT - 1); i0 <= i_hi; i0 += kKT) {
-      if (tid < kSoftmaxThreads) {
-        // phi(K') tile (fp32 scratch -> bf16, K-major) and the delayed tokens' V rows (MN-major)
-#pragma unroll 4
-        for (int i = 0; i < kKT * 16 / kSoftmaxThreads; ++i) {
-          const int id = tid + kSoftmaxThreads * i;
-          const int r = id >> 4, c = id & 15;
-          const int ii = i0 + r;
-          const bool valid = ii >= i_lo && ii <= i_hi;
-          uint4 pkd = make_uint4(0u, 0u, 0u, 0u);
-          if (valid) {
-            const float4 f0 = *reinterpret_cast<const float4 *>(pkp + size_t(ii) * kD + c * 8);
-            const float4 f1 = *reinterpret_cast<const float4 *>(pkp + size_t(ii) * kD + c * 8 + 4);
-            pkd = make_uint4(pack_bf16x2(f0.x, f0.y), pack_bf16x2(f0.z, f0.w), pack_bf16x2(f1.x, f1.y), pack_bf16x2(f1.z, f1.w));
-          }
-          *reinterpret_cast<uint4 *>(sm.kv[slotPk] + sw128(r, c)) = pkd;
-          const int64_t jj = valid ? p.n0 + p.c0 - wl + ii : 0;
-          const bool from_call = jj >= p.n0;
-          const uint32_t slot_row = (jj >> 32) == 0 ? uint32_t(jj) % cap : uint32_t(uint64_t(jj) % cap);
-          const bf16 *src = from_call ? callV + size_t(jj - p.n0) * call_stride : ringV + size_t(slot_row) * kD;
-          cp_async16(kv_addr(slotV) + sw128(r, c), src + c * 8, valid);
-        }
-        cp_async_commit();
-        cp_async_wait_all();
-      }
-      fence_async_smem();
-      tc_fence_before();
-      __syncthreads();
-      if (tid == mma_tid) {
-        tc_fence_after();
-        issue_mma(tmem, sQ[0], kv_addr(slotPk), false, false);   // C_X = (phi(Q_X) 2^-m*) phi(K')^T
-        if (hasB) issue_mma(tmem + 128, sQ[1], kv_addr(slotPk), false, false);
-        mma_commit(smem_u32(&sm.bar_lin));
-      }
-      wait_lin();
+    if (need_state && activeX) {
+      mbar_wait(smem_u32(&sm.bar_state), 0u, failed);   // z has landed
+      float dot = 0.f;
+#pragma unroll
+      for (int i = 0; i < kD / 2; ++i)
+        dot += __uint_as_float(phq[i] << 16) * sm.z[2 * i] + __uint_as_float(phq[i] & 0xffff0000u) * sm.z[2 * i + 1];
+      if (!sum_terms) l_sum += dot;
+    }
+    if (need_state || n_itiles > 0) wait_lin();
+    if (need_state) o_init = true;
+    PF_CLK(3);
+    for (int t = 0; t < n_itiles; ++t) {
+      const int i0 = it0 + t * kKT;
       if (activeX) {
         // C row -> bf16, masked to delayed tokens j' <= i of this row (the values already carry 2^-m*)
         float sum0 = 0.f, sum1 = 0.f;
@@ -792,16 +837,30 @@ prefill_attn_tc_kernel(const PrefillParams p, const CUtensorMap *ring_maps, cons
         tmem_wait_st();
         if (!sum_terms) l_sum += sum0 + sum1;
       }
+      PF_CLK(4);
+      if (t >= 2 && tid < kSoftmaxThreads) cp_async_wait_all();   // (steps after the second: rows copied by these threads)
+      fence_async_smem();
       tc_fence_before();
       __syncthreads();
       if (tid == mma_tid) {
+        if (t < 2) mbar_wait(smem_u32(&sm.bar_vp[t]), 0u, failed);   // the loader's V' tile
         tc_fence_after();
-        issue_mma_ts(tmem + 256, tmem, kv_addr(slotV), o_init);
-        if (hasB) issue_mma_ts(tmem + 384, tmem + 128, kv_addr(slotV), o_init);
+        issue_mma_ts(tmem + 256, tmem, kv_addr(slotVp[t & 1]), o_init);
+        if (hasB) issue_mma_ts(tmem + 384, tmem + 128, kv_addr(slotVp[t & 1]), o_init);
+        if (t + 1 < n_itiles) {   // the next step's C follows in the same batch (the tensor pipe keeps the order)
+          mbar_wait(smem_u32(&sm.bar_pk[(t + 1) & 1]), uint32_t((t + 1) >> 1) & 1u, failed);
+          issue_mma(tmem, sQ[0], kv_addr(slotPk[(t + 1) & 1]), false, false);
+          if (hasB) issue_mma(tmem + 128, sQ[1], kv_addr(slotPk[(t + 1) & 1]), false, false);
+        }
         mma_commit(smem_u32(&sm.bar_lin));
       }
       wait_lin();
+      PF_CLK(5);
       o_init = true;
+      if (t + 2 < n_itiles) {   // this step's buffers are free again: the operands of the step after the next
+        if (tid == mma_tid) load_pk(t + 2);
+        if (tid < kSoftmaxThreads) load_vp(t + 2);
+      }
     }
   }
 
@@ -815,10 +874,13 @@ prefill_attn_tc_kernel(const PrefillParams p, const CUtensorMap *ring_maps, cons
     const float inv = store ? 1.0f / l_sum : 0.f;
     bf16 *op = reinterpret_cast<bf16 *>(p.out) +
                ((seq + size_t(p.c0 + (store ? tl : tok0))) * p.H + p.heads_of[g * G + hh]) * kD;
-#pragma unroll 1
+    uint32_t ra[32], rb[32];
+    tmem_ld32_nowait(tO, ra);
+#pragma unroll
     for (int c0 = 0; c0 < kD; c0 += 32) {
-      uint32_t r[32];
-      tmem_ld32(tO + c0, r);
+      uint32_t (&r)[32] = ((c0 >> 5) & 1) ? rb : ra;
+      tmem_wait_ld();
+      if (c0 + 32 < kD) tmem_ld32_nowait(tO + c0 + 32, ((c0 >> 5) & 1) ? ra : rb);   // the next columns are on their way
 #pragma unroll
       for (int q4 = 0; q4 < 4; ++q4) {
         uint32_t pk[4];
@@ -831,6 +893,7 @@ prefill_attn_tc_kernel(const PrefillParams p, const CUtensorMap *ring_maps, cons
   }
   tc_fence_before();
   __syncthreads();
+  PF_CLK(6);
   if (warp == 0) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 512;" ::"r"(tmem) : "memory");
 }
 
@@ -838,8 +901,19 @@ prefill_attn_tc_kernel(const PrefillParams p, const CUtensorMap *ring_maps, cons
 
 
 // The kernel needs the ring descriptors made for the tensor-core decode kernels.
+#ifdef GLIDE_PF_CLOCKS
+extern "C" int glide_debug_pf_clocks(unsigned long long *host16, int reset) {
+  if (cudaMemcpyFromSymbol(host16, g_pf_clk, sizeof(g_pf_clk)) != cudaSuccess) return 6;
+  if (reset) {
+    unsigned long long z[16] = {};
+    if (cudaMemcpyToSymbol(g_pf_clk, z, sizeof(z)) != cudaSuccess) return 6;
+  }
+  return 0;
+}
+#endif
+
 bool prefill_attn_tc_supported(const glide_ctx *ctx) {
-  return ctx->cfg.io_dtype == GLIDE_BF16 && ctx->cfg.head_dim == kD && ctx->decode_kind >= 1;
+  return ctx->cfg.io_dtype == GLIDE_BF16 && ctx->cfg.head_dim == kD && ctx->decode_kind >= 1 && ctx->off_phik16 != 0;
 }
 
 namespace {
