@@ -237,6 +237,39 @@ def test_decode_step_layers(dtype, d, impl, merge):
     assert g.glide_device_status() == 0
 
 
+@pytest.mark.parametrize("merge,G", [(0, 4), (0, 8), (1, 4), (0, 1)])
+def test_units_cut_into_many_records(merge, G):
+    """One long-window layer at batch 1: its few units are spread over all CTAs (about 18 records per unit with
+    w = 4096 on 148 SMs), so the merging warp reads them in several batches, each polled until it carries the
+    launch's tag; run as one-layer launches and as a whole-stack launch, for several steps (the tags move on)."""
+    import numpy as np
+    from paper_2607_24788_b200 import glide, synth
+    from oracle import glide_oracle as orc
+    from tests.parity_util import f32_scale, to_np, check_outputs, check_state
+    windows, B, Hkv, d, T = [4096, 64], 1, 2, 128, 4200
+    H = Hkv * G
+    wl = synth.Workload(41 + G, len(windows), B, H, Hkv, d, BF16, d ** -0.5 * 4)
+    g = glide.Glide(windows, B, H, Hkv, d, T + 16, dtype=BF16, softmax_scale=f32_scale(d), merge=merge)
+    sched = glide.glide_stream_schedule(g.cfg)   # columns 10, 11: record index of the segment, records of its unit
+    assert sched[:, 11].max() > 16, "the whole-stack schedule should cut the long-window units into many records"
+    stack = orc.Stack(windows, B, H, Hkv, d, f32_scale(d), merge=merge)
+    q, k, v = wl.qkv(range(2), range(B), range(T), device="cuda")
+    g.glide_prefill(None, k, v, None)
+    stack.prefill(None, to_np(k), to_np(v), outputs=False)
+    for t in range(T, T + 6):
+        q, k, v = wl.decode_qkv(t, "cuda")
+        out = torch.full_like(q, float("nan"))
+        ref = stack.decode(to_np(q), to_np(k), to_np(v))
+        if t % 2 == 0:
+            for l in range(2):
+                g.glide_decode_step_layers(q[l:l + 1], k[l:l + 1], v[l:l + 1], out[l:l + 1], l, 1)
+        else:
+            g.glide_decode_step(q, k, v, out)
+        check_outputs(out, ref, BF16, f"step {t}")
+    check_state(g, stack, "after steps with many records per unit")
+    assert g.glide_device_status() == 0
+
+
 def test_bf16_prefill_tcgen05_after_decode_steps():
     # a prompt, a few decode steps, then another prompt (a second turn): the second call starts at a position that
     # is not a multiple of 16 and its first key tiles mix ring rows, wrapped ring rows and the call's rows
