@@ -521,7 +521,10 @@ DecodeParams make_decode_params(const glide_ctx *ctx, int layer_begin, int layer
   p.gated = ctx->cfg.gated;
   p.gate = nullptr;
   p.tensors_absolute = ctx->decode_kind != 2;
-  if (++ctx->launch_seq == 0) ++ctx->launch_seq;
+  if (++ctx->launch_seq == 0) {   // tag 0 is what a never-written record holds
+    ctx->launch_seq = 1;
+    ctx->launch_wrapped = true;
+  }
   p.launch_tag = ctx->launch_seq;
   p.q = q;
   p.k = k;

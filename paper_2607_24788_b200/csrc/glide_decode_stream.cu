@@ -52,6 +52,9 @@ constexpr int kHdrSlots = 3;
 #define GLIDE_W_WIN 10
 #define GLIDE_W_UNIT 27
 #endif
+#ifndef GLIDE_STREAM_MAX_PARTS
+#define GLIDE_STREAM_MAX_PARTS 8
+#endif
 #ifndef GLIDE_W_GROUP
 #define GLIDE_W_GROUP 0   // extra weight of a segment whose unit is shared with other warps of the CTA
 #endif
@@ -1219,7 +1222,11 @@ void build_stream_schedule(const glide_ctx *ctx, int layer_begin, int layer_coun
     while (n_heavy < order.size() && pieces[order[n_heavy]].weight() > cta_share) heavy_w += pieces[order[n_heavy++]].weight();
     // these CTAs end with the merge of their units' records: they may be given less than a full share
     const int64_t heavy_share = std::max<int64_t>(1, cta_share * GLIDE_STREAM_FILL / 100);
-    const int n_h = int(std::max<int64_t>(1, std::min<int64_t>(n_used, (heavy_w + heavy_share / 2) / heavy_share)));
+    int n_h = int(std::max<int64_t>(1, std::min<int64_t>(n_used, (heavy_w + heavy_share / 2) / heavy_share)));
+    // Where spreading leaves a CTA only a few dozen tiles (a one-layer launch of a long window at a small batch), a
+    // unit is cut into at most about GLIDE_STREAM_MAX_PARTS records: the merging warp reads them a few at a time, each
+    // batch a round trip to L2, and that costs more than the shorter streams save.  Large problems keep every SM.
+    if (heavy_w / n_h < 40 * kWinWeight) n_h = int(std::max<int64_t>(1, std::min<int64_t>(n_h, int64_t(GLIDE_STREAM_MAX_PARTS) * int64_t(n_heavy))));
     // every CTA boundary inside a unit opens one more piece with its own fixed cost
     const int64_t target = (heavy_w + int64_t(n_h) * kSegWeight) / n_h + 1;
     if (n_heavy > 0) {
@@ -1510,6 +1517,15 @@ int stream_decode_setup(glide_ctx *ctx) {
 int launch_decode_stream(glide_ctx *ctx, const DecodeParams &p, int schedule, cudaStream_t stream) {
   if (schedule < 0 || size_t(schedule) >= ctx->stream_scheds.size()) return GLIDE_ERR_INVALID_ARG;
   const glide_ctx::StreamSchedule &sc = ctx->stream_scheds[size_t(schedule)];
+  if (p.launch_tag == 1 && ctx->launch_wrapped) {
+    // the launch counter has gone round: a record slot that no schedule has written for 2^32 launches could carry this
+    // launch's tag already, so the records start from zero again (stream-ordered behind the preceding launch)
+    if (cudaMemsetAsync(ctx->ws + ctx->off_partials, 0, ctx->off_stream_segs - ctx->off_partials, stream) != cudaSuccess) {
+      cudaGetLastError();
+      return GLIDE_ERR_CUDA;
+    }
+    ctx->launch_wrapped = false;
+  }
   StreamParams sp{};
   sp.segs = reinterpret_cast<const StreamSegment *>(ctx->ws + ctx->off_stream_segs) + sc.seg_base;
   for (int c = 0; c <= ctx->decode_grid; ++c) sp.cta_seg_begin[c] = sc.range_begin[size_t(c) * kWarps];

@@ -216,6 +216,7 @@ struct glide_ctx {
   int n_items = 0;
   int rec_floats = 0;
   mutable uint32_t launch_seq = 0;  // launches so far: the tag of the next launch's cross-CTA records
+  mutable bool launch_wrapped = false;   // the counter has passed 2^32: the records are cleared before the next launch
   int stream_rec_floats = 0;        // record size of the streaming kernel (twice as large for the sum-of-terms merges)
   int prefill_chunk = 0;
   float scale = 0.f;

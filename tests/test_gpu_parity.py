@@ -239,9 +239,10 @@ def test_decode_step_layers(dtype, d, impl, merge):
 
 @pytest.mark.parametrize("merge,G", [(0, 4), (0, 8), (1, 4), (0, 1)])
 def test_units_cut_into_many_records(merge, G):
-    """One long-window layer at batch 1: its few units are spread over all CTAs (about 18 records per unit with
-    w = 4096 on 148 SMs), so the merging warp reads them in several batches, each polled until it carries the
-    launch's tag; run as one-layer launches and as a whole-stack launch, for several steps (the tags move on)."""
+    """One long-window layer at batch 1: its few units are spread over many CTAs (eight or nine records per unit), so
+    the merging warp reads them in several batches of 16 / G records (one batch for G = 1), each polled until it
+    carries the launch's tag; run as one-layer launches and as a whole-stack launch, for several steps (the tags
+    move on)."""
     import numpy as np
     from paper_2607_24788_b200 import glide, synth
     from oracle import glide_oracle as orc
@@ -251,7 +252,7 @@ def test_units_cut_into_many_records(merge, G):
     wl = synth.Workload(41 + G, len(windows), B, H, Hkv, d, BF16, d ** -0.5 * 4)
     g = glide.Glide(windows, B, H, Hkv, d, T + 16, dtype=BF16, softmax_scale=f32_scale(d), merge=merge)
     sched = glide.glide_stream_schedule(g.cfg)   # columns 10, 11: record index of the segment, records of its unit
-    assert sched[:, 11].max() > 16, "the whole-stack schedule should cut the long-window units into many records"
+    assert sched[:, 11].max() >= 6, "the whole-stack schedule should cut the long-window units into many records"
     stack = orc.Stack(windows, B, H, Hkv, d, f32_scale(d), merge=merge)
     q, k, v = wl.qkv(range(2), range(B), range(T), device="cuda")
     g.glide_prefill(None, k, v, None)
