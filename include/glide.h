@@ -121,7 +121,8 @@ typedef struct {
                               waits in the ring with its key and value, and the state decays by the gate of the token
                               that enters it: S <- gamma S + phi(k) v^T, z <- gamma z + phi(k).  Gates are passed to
                               glide_prefill_gated / glide_decode_step_gated; the calls without gates use gamma = 1.
-                              Runs on the CUDA-core kernels (decode_impl AUTO or FMA, prefill_impl AUTO or FMA). */
+                              Decode: the streaming kernel (bf16, head_dim 128) or the CUDA-core kernel (decode_impl
+                              AUTO, STREAM or FMA); prefill: the CUDA-core kernels (prefill_impl AUTO or FMA). */
   int32_t reserved_;       /* must be 0 */
 } glide_config;
 

@@ -594,10 +594,11 @@ int launch_decode(glide_ctx *ctx, int layer_begin, int layer_count, const void *
     const size_t qrow = size_t(ctx->cfg.head_dim) * ctx->elem * size_t(ctx->cfg.batch) * ctx->cfg.n_q_heads;
     const size_t krow = size_t(ctx->cfg.head_dim) * ctx->elem * size_t(ctx->cfg.batch) * ctx->cfg.n_kv_heads;
     for (int i = 0; i < layer_count; ++i) {
-      const DecodeParams pl = make_decode_params(ctx, layer_begin + i, 1, static_cast<const unsigned char *>(q) + qrow * i,
-                                                 static_cast<const unsigned char *>(k) + krow * i,
-                                                 static_cast<const unsigned char *>(v) + krow * i,
-                                                 static_cast<unsigned char *>(out) + qrow * i);
+      DecodeParams pl = make_decode_params(ctx, layer_begin + i, 1, static_cast<const unsigned char *>(q) + qrow * i,
+                                           static_cast<const unsigned char *>(k) + krow * i,
+                                           static_cast<const unsigned char *>(v) + krow * i,
+                                           static_cast<unsigned char *>(out) + qrow * i);
+      pl.gate = gate ? gate + size_t(i) * ctx->cfg.batch * ctx->cfg.n_kv_heads : nullptr;
       int rc = launch_decode_phi(ctx, pl, stream);
       if (rc) return rc;
       rc = launch_decode_stream(ctx, pl, 1 + layer_begin + i, stream);

@@ -487,6 +487,7 @@ glide_decode_stream_kernel(const DecodeParams p, const StreamParams sp) {
   float m0, m1, l0, l1;
   float phi[G + 1][4];     // phi(q_h) for the G heads, then phi(k_e); lane holds entries 4*lane .. 4*lane+3
   float ve[4];
+  float gamma = 1.f;       // gated recurrence: gate of the token that enters the state at this step
   float4 a[G];
   float bp[G];
   float scur[G];           // the current token's own logit per head (log2 domain)
@@ -581,10 +582,10 @@ glide_decode_stream_kernel(const DecodeParams p, const StreamParams sp) {
     for (int r = 0; r < kTileRows; ++r) {
       float4 s = st[r * (kD / 4) + lane];
       const float pk = PHI2 ? sphi[G * 16 + r] : __shfl_sync(0xffffffffu, phi[G][r & 3], src0 + (r >> 2));
-      s.x = fmaf(pk, ve[0], s.x);
-      s.y = fmaf(pk, ve[1], s.y);
-      s.z = fmaf(pk, ve[2], s.z);
-      s.w = fmaf(pk, ve[3], s.w);
+      s.x = fmaf(pk, ve[0], gamma * s.x);   // (gamma = 1 without gates: the product is exact)
+      s.y = fmaf(pk, ve[1], gamma * s.y);
+      s.z = fmaf(pk, ve[2], gamma * s.z);
+      s.w = fmaf(pk, ve[3], gamma * s.w);
       st[r * (kD / 4) + lane] = s;
 #pragma unroll
       for (int h = 0; h < G; ++h) {
@@ -612,7 +613,7 @@ glide_decode_stream_kernel(const DecodeParams p, const StreamParams sp) {
       }
       if (h == 0) {
         if (lane < 16) {
-          zn = zs[lane] + f;
+          zn = fmaf(gamma, zs[lane], f);
           zs[lane] = zn;
         }
       } else if (lane < 16) {
@@ -642,6 +643,16 @@ glide_decode_stream_kernel(const DecodeParams p, const StreamParams sp) {
 
     // -- header: q fragments, current token, feature maps -> registers; then prefetch the next header --
     GLIDE_TRACE_EVENT(6);
+    gamma = 1.f;
+    if (p.gated && n_state_eff > 0) {
+      // the gate of the token that enters the state: the current token's (no ring, or a state that holds every
+      // token), else the one waiting in the ring of gates beside the token that leaves the window
+      if (sg.evicts & 2) {
+        if (p.gate) gamma = p.gate[sg.unit];
+      } else {
+        gamma = reinterpret_cast<const float *>(p.ws + p.layers[sg.layer].ringG)[size_t(sg.row_base) + size_t(slot_of(t, sg.cap))];
+      }
+    }
     if (!mbar_wait(hdr_bar, (phases >> STAGES) & 1u)) failed = true;
     phases ^= 1u << STAGES;
     if (__any_sync(0xffffffffu, failed)) {
@@ -919,6 +930,9 @@ glide_decode_stream_kernel(const DecodeParams p, const StreamParams sp) {
         const size_t row = (size_t(sg.row_base) + size_t(win_cur)) * kD;
         reinterpret_cast<uint2 *>(reinterpret_cast<bf16 *>(p.ws + size_t(sg.ringK_off256) * 256) + row)[lane] = kt_bits;
         reinterpret_cast<uint2 *>(reinterpret_cast<bf16 *>(p.ws + size_t(sg.ringV_off256) * 256) + row)[lane] = vt_bits;
+        if (p.gated && lane == 0)   // the token's gate waits in the ring with it
+          reinterpret_cast<float *>(p.ws + p.layers[sg.layer].ringG)[size_t(sg.row_base) + size_t(win_cur)] =
+              p.gate ? p.gate[sg.unit] : 1.f;
       }
     }
   }
@@ -1112,6 +1126,8 @@ glide_decode_stream_kernel(const DecodeParams p, const StreamParams sp) {
         const size_t row = (size_t(sg.row_base) + size_t(slot_of(pos_of(pi == 0 ? pend0 : pend1), sg.cap))) * kD;
         reinterpret_cast<uint2 *>(reinterpret_cast<bf16 *>(p.ws + size_t(sg.ringK_off256) * 256) + row)[lane] = ktb;
         reinterpret_cast<uint2 *>(reinterpret_cast<bf16 *>(p.ws + size_t(sg.ringV_off256) * 256) + row)[lane] = vtb;
+        if (p.gated && lane == 0)
+          reinterpret_cast<float *>(p.ws + p.layers[sg.layer].ringG)[row / kD] = p.gate ? p.gate[sg.unit] : 1.f;
       }
       GLIDE_TRACE_EVENT(13);
     }
@@ -1436,8 +1452,8 @@ void build_stream_schedule(const glide_ctx *ctx, int layer_begin, int layer_coun
 }
 
 int stream_decode_supported(const glide_ctx *ctx) {
-  // (the learned feature map with the shared normaliser only; the gated recurrence runs on the CUDA-core kernel)
-  return ctx->cfg.io_dtype == GLIDE_BF16 && ctx->cfg.head_dim == kD && !ctx->cfg.gated &&
+  // (the learned feature map with the shared normaliser only)
+  return ctx->cfg.io_dtype == GLIDE_BF16 && ctx->cfg.head_dim == kD &&
          (ctx->cfg.phi == GLIDE_PHI_SOFTMAX || ctx->cfg.merge == GLIDE_MERGE_SHARED);
 }
 

@@ -67,8 +67,8 @@ int validate_config(const glide_config *c) {
   } else if (c->phi_wq || c->phi_wk) {
     return GLIDE_ERR_INVALID_ARG;
   }
-  if (c->gated) {   // the gated recurrence runs on the CUDA-core kernels
-    if (c->decode_impl == GLIDE_DECODE_MMA || c->decode_impl == GLIDE_DECODE_STREAM) return GLIDE_ERR_UNSUPPORTED;
+  if (c->gated) {   // the gated recurrence runs on the CUDA-core kernels and on the streaming decode kernel
+    if (c->decode_impl == GLIDE_DECODE_MMA) return GLIDE_ERR_UNSUPPORTED;
     if (c->prefill_impl == GLIDE_PREFILL_MMA_SYNC || c->prefill_impl == GLIDE_PREFILL_TCGEN05) return GLIDE_ERR_UNSUPPORTED;
   }
   if (c->merge < GLIDE_MERGE_SHARED || c->merge > GLIDE_MERGE_SUM_ALL) return GLIDE_ERR_INVALID_ARG;
@@ -331,7 +331,7 @@ int glide_create(const glide_config *cfg, void *dev_workspace, size_t workspace_
   int per_sm = 0;
   // kernel choice: fp32 -> CUDA cores; bf16 -> streaming tensor-core kernel when it applies, else per-item one
   ctx->decode_kind = 0;
-  if (ok && cfg->io_dtype == GLIDE_BF16 && cfg->decode_impl != GLIDE_DECODE_FMA && !cfg->gated) {
+  if (ok && cfg->io_dtype == GLIDE_BF16 && cfg->decode_impl != GLIDE_DECODE_FMA) {
     ok = build_ring_tensor_maps(ctx) == GLIDE_OK;
     const bool want_stream = cfg->decode_impl == GLIDE_DECODE_AUTO || cfg->decode_impl == GLIDE_DECODE_STREAM;
     if (ok && want_stream && stream_decode_supported(ctx) && ctx->sm_count * GLIDE_STREAM_CTAS_PER_SM <= kMaxStreamCtas) {
@@ -344,11 +344,11 @@ int glide_create(const glide_config *cfg, void *dev_workspace, size_t workspace_
         delete ctx;
         return GLIDE_ERR_UNSUPPORTED;
       }
-      if (cfg->merge == GLIDE_MERGE_SHARED && cfg->phi == GLIDE_PHI_SOFTMAX) {
+      if (cfg->merge == GLIDE_MERGE_SHARED && cfg->phi == GLIDE_PHI_SOFTMAX && !cfg->gated) {
         ok = mma_decode_setup(ctx) == GLIDE_OK;
         ctx->decode_kind = 1;
-      }   // the per-item tensor-core kernel has the shared normaliser and the parameter-free map only: other merges and
-          // the learned map use the CUDA-core kernel
+      }   // the per-item tensor-core kernel has the shared normaliser and the parameter-free map only: other merges,
+          // the learned map and gates use the CUDA-core kernel
     }
   }
   if (ok && ctx->decode_kind == 0) {

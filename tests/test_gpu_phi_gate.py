@@ -72,7 +72,8 @@ def test_feature_map_and_gate_argument_checks():
                      (dict(phi=0, phi_wq=wq, phi_wk=wk), glide.GLIDE_ERR_INVALID_ARG),            # weights without the map
                      (dict(phi=1, phi_wq=wq, phi_wk=wk, decode_impl=glide.GLIDE_DECODE_MMA), glide.GLIDE_ERR_UNSUPPORTED),
                      (dict(phi=1, phi_wq=wq, phi_wk=wk, prefill_impl=glide.GLIDE_PREFILL_TCGEN05), glide.GLIDE_ERR_UNSUPPORTED),
-                     (dict(gated=True, decode_impl=glide.GLIDE_DECODE_STREAM), glide.GLIDE_ERR_UNSUPPORTED)):
+                     (dict(gated=True, decode_impl=glide.GLIDE_DECODE_MMA), glide.GLIDE_ERR_UNSUPPORTED),
+                     (dict(gated=True, prefill_impl=glide.GLIDE_PREFILL_TCGEN05), glide.GLIDE_ERR_UNSUPPORTED)):
         with pytest.raises(glide.GlideError) as e:
             glide.Glide([16], 1, 4, 2, d, 64, dtype=BF16, **kw)
         assert e.value.code == code, kw
@@ -91,6 +92,42 @@ def test_learned_map_on_the_streaming_kernel_units_cut_across_ctas(G, B):
     Hkv = 2
     run_case([1500, 64, 0, 5000, 300], B, Hkv * G, Hkv, 128, BF16, [1490, 7], 12, amp=4 * 128 ** -0.5, seed=11 + G,
              phi=1, check_prefill_outputs=False, decode_impl=glide.GLIDE_DECODE_STREAM)
+
+
+@pytest.mark.parametrize("phi,G,B", [(0, 4, 1), (0, 8, 2), (1, 4, 1), (0, 1, 3)])
+def test_gated_recurrence_on_the_streaming_kernel(phi, G, B):
+    """Gates on the bf16 streaming decode kernel: units inside one warp, shared by the warps of a CTA and cut across
+    CTAs; a layer without a ring (the current token's gate decays the state), one that never evicts, and decode
+    steps that cross a ring wrap (the gate of the leaving token comes from the ring of gates written by earlier
+    steps and by the prefill)."""
+    Hkv = 2
+    run_case([1500, 64, 0, 5000, 300], B, Hkv * G, Hkv, 128, BF16, [1490, 7], 12, amp=4 * 128 ** -0.5, seed=17 + G,
+             phi=phi, gated=True, check_prefill_outputs=False, decode_impl=glide.GLIDE_DECODE_STREAM)
+
+
+def test_gated_streaming_kernel_without_gates_is_bit_identical_to_the_plain_one():
+    """A gated context driven without gates multiplies by gamma = 1: the same bits as a context without gates."""
+    from paper_2607_24788_b200 import synth
+    from tests.parity_util import f32_scale
+    windows, B, H, Hkv, d, T = [300, 0, 64], 1, 8, 2, 128, 400
+    wl = synth.Workload(19, len(windows), B, H, Hkv, d, BF16, 4 * d ** -0.5)
+    outs = []
+    for gated in (False, True):
+        g = glide.Glide(windows, B, H, Hkv, d, T + 8, dtype=BF16, softmax_scale=f32_scale(d), gated=gated,
+                        decode_impl=glide.GLIDE_DECODE_STREAM, prefill_impl=glide.GLIDE_PREFILL_FMA)
+        q, k, v = wl.qkv(range(len(windows)), range(B), range(T), device="cuda")
+        g.glide_prefill(None, k, v, None)
+        got = []
+        for s in range(6):
+            q, k, v = wl.decode_qkv(T + s, device="cuda")
+            out = torch.empty_like(q)
+            g.glide_decode_step(q, k, v, out)
+            got.append(out)
+        got.extend(g.glide_export_state(0)[2:])
+        assert g.glide_device_status() == 0
+        outs.append(got)
+    for x, y in zip(*outs):
+        assert torch.equal(x.view(torch.uint8), y.view(torch.uint8))
 
 
 def test_learned_map_streaming_layer_by_layer_and_ragged_slots():
