@@ -18,11 +18,12 @@
 // A unit that lies inside one warp's range is finished by that warp alone (current token's own term,
 // normalise, write, ring append) without touching global scratch.  Units shared by warps of one CTA are
 // reduced in shared memory by the last of them to arrive.  Only units cut by a CTA boundary go through global
-// scratch: one record per CTA, every value stored beside the launch's tag in one 8-byte word, so that neither
-// a fence nor a counter is needed; the warp that holds the unit's last piece merges the records at the end of
-// its range, polling the words it is about to use until they carry the tag.  That poll is the only place where
-// a warp waits for another one (all CTAs of a launch are resident: one per SM); like the waits on the warp's
-// own mbarriers it is bounded, and a wait that runs out sets the context's status word.
+// scratch: one record per CTA, every value stored beside the launch's tag in one 8-byte word, and a ticket per
+// unit taken with a relaxed atomic (no fence between the record and the ticket: the tags say when a value has
+// arrived).  The warp that draws a unit's last ticket merges the records at the end of its range, polling the
+// words it is about to use until they carry the tag: every one of them has been stored by then, so the poll
+// never waits for a CTA that is not running.  Like the waits on the warp's own mbarriers it is bounded, and a
+// wait that runs out sets the context's status word.
 #include <cuda.h>
 
 #include <algorithm>
@@ -172,7 +173,7 @@ __device__ __forceinline__ void prefetch_tensormap(const void *tmap) {
 }
 // ---- records of units cut across CTAs: every 4-byte value travels with the launch's tag in one 8-byte store ------
 // A 64-bit store is a single access, so a reader that sees the tag sees the value: no fence orders the record
-// before a ticket, and the reader needs no ticket either -- it polls the pairs it is about to use.
+// before the unit's ticket: whoever draws the last ticket polls the pairs it is about to use.
 __device__ __forceinline__ unsigned long long ll_pack(float v, uint32_t tag) {
   return (static_cast<unsigned long long>(tag) << 32) | __float_as_uint(v);
 }
@@ -496,6 +497,7 @@ glide_decode_stream_kernel(const DecodeParams p, const StreamParams sp) {
   uint32_t phases = 0;     // parity expected by the next wait on each stage; bit STAGES: header barrier
   int stage = 0;
   int n_pending = 0, pend0 = 0, pend1 = 0;   // segments of this range whose unit is shared with a neighbour (at most two)
+  unsigned tick0 = 0, tick1 = 0;             // their tickets (lane 0)
 
   // ---- window tile ------------------------------------------------------------------------------
   auto consume_window = [&](int wtile, uint32_t stage_addr) {
@@ -632,6 +634,11 @@ glide_decode_stream_kernel(const DecodeParams p, const StreamParams sp) {
     }
   };
 
+  // the record of the segment that has just finished (after the loop: of the range's last segment, which the merge
+  // below takes from here instead of reading it back from global memory)
+  float mh[G], lh[G];
+  float4 acc[G];
+  int own_seg = -1;   // segment whose global record these registers still hold
   // ---- main loop over this warp's segments ------------------------------------------------------------
   for (int s = seg_lo; s < seg_hi && !failed; ++s) {
     const StreamSegment &sg = sm_segs[s];
@@ -734,8 +741,6 @@ glide_decode_stream_kernel(const DecodeParams p, const StreamParams sp) {
     }
     if (failed) break;
     // -- finish: record (m, l, acc) in a common layout: lane holds features 4*lane..4*lane+3 of every head --
-    float mh[G], lh[G];
-    float4 acc[G];
     if (n_total > n_state_eff) {   // window tiles were processed: move the accumulator fragments through the freed stage
       float *scr = reinterpret_cast<float *>(my_stages_ptr + last_stage * kStageBytes);
       const float lq0 = quad_col_sum(l0), lq1 = quad_col_sum(l1);
@@ -879,7 +884,7 @@ glide_decode_stream_kernel(const DecodeParams p, const StreamParams sp) {
     }
     if (sg.part >= 0) {
       // the unit is cut by a CTA boundary: this CTA's record goes to global scratch, every value paired with the
-      // launch's tag.  The CTA that holds the unit's last piece merges the records at the end of this warp's range.
+      // launch's tag; the unit's last ticket merges the records (at the end of that warp's range).
       unsigned long long *grec = reinterpret_cast<unsigned long long *>(p.partials) + (size_t(sg.rec0) + sg.part) * p.rec_floats;
 #pragma unroll
       for (int h = 0; h < G; ++h) {
@@ -895,10 +900,20 @@ glide_decode_stream_kernel(const DecodeParams p, const StreamParams sp) {
           if (SUM) ll_store1(grec + L::kRecW + G * kD + h, bp[h], p.launch_tag);
         }
       }
-      if (sg.part == sg.n_parts - 1) {
-        if (n_pending == 0) pend0 = s; else pend1 = s;
-        ++n_pending;
+      // the unit's ticket, taken without a fence: the result is looked at only at the end of this warp's range, so
+      // the round trip runs beside the tiles of the range's remaining segments
+      unsigned tick = 0;
+      if (lane == 0)
+        asm volatile("atom.relaxed.gpu.global.add.u32 %0, [%1], 1;" : "=r"(tick) : "l"(p.tickets + sg.unit) : "memory");
+      if (n_pending == 0) {
+        pend0 = s;
+        tick0 = tick;
+      } else {
+        pend1 = s;
+        tick1 = tick;
       }
+      ++n_pending;
+      own_seg = s;
     } else {
       // the whole unit is in this range: current token's own term, shared normaliser, output row, ring append
       float vx[4];
@@ -938,11 +953,18 @@ glide_decode_stream_kernel(const DecodeParams p, const StreamParams sp) {
   }
   GLIDE_TRACE_EVENT(14);
 
-  // ---- units whose last piece this range holds: merge the CTAs' records as they become visible -------------------
+  // ---- units this range shares with other CTAs: whoever holds a unit's last ticket merges its records ---------------
+  // (every record of the unit has been stored by then, though perhaps not arrived: the merge polls the tags.  It
+  // never waits for a CTA that has not run yet, so launches that share the GPU cannot block each other.)
   if (n_pending > 0 && !failed) {
     GLIDE_TRACE_EVENT(12);
     for (int pi = 0; pi < n_pending && !failed; ++pi) {
       const StreamSegment &sg = sm_segs[pi == 0 ? pend0 : pend1];
+      const int pseg = pi == 0 ? pend0 : pend1;
+      // this warp's own record of the unit is still in registers when the unit's segment was the last of the range: it
+      // is taken from there (same values, same place in the order of the merge) instead of being awaited from memory
+      // (groups of 8 heads: the record is 40 registers wide and keeping it would spill; it is read back like the others)
+      const int own = (G <= 4 && pseg == own_seg && pseg == seg_hi - 1) ? sg.part : -1;
       const bool has_win = sg.cap > 0;
       // reload the unit's query rows and current token (this warp may have moved on to another unit since);
       // every load of the merge's first batch is issued before anything is reduced
@@ -961,7 +983,7 @@ glide_decode_stream_kernel(const DecodeParams p, const StreamParams sp) {
       float me0 = -CUDART_INF_F, le0 = 0.f;
       float4 vv0[RPB][G];
       // one batch of records: polled until every pair this lane uses carries the launch's tag (bounded)
-      auto load_batch = [&](int i0, float &me, float &le) -> bool {
+      auto load_batch = [&](int i0, float &me, float &le, uint32_t max_spins) -> bool {
         const int ri = i0 + lane / G, rh = lane % G;
         const int nb = sg.n_parts - i0 < RPB ? sg.n_parts - i0 : RPB;
         const bool mine = lane < RPB * G && ri < sg.n_parts;
@@ -979,23 +1001,40 @@ glide_decode_stream_kernel(const DecodeParams p, const StreamParams sp) {
               asm volatile("ld.relaxed.gpu.global.v2.u64 {%0, %1}, [%2];" : "=l"(raw[u][h][0]), "=l"(raw[u][h][1]) : "l"(src));
               asm volatile("ld.relaxed.gpu.global.v2.u64 {%0, %1}, [%2];" : "=l"(raw[u][h][2]), "=l"(raw[u][h][3]) : "l"(src + 2));
             }
-          uint32_t diff = (uint32_t(rm >> 32) ^ p.launch_tag) | (uint32_t(rl >> 32) ^ p.launch_tag);
+          uint32_t diff = (!mine || ri != own) ? (uint32_t(rm >> 32) ^ p.launch_tag) | (uint32_t(rl >> 32) ^ p.launch_tag) : 0u;
 #pragma unroll
           for (int u = 0; u < RPB; ++u)
 #pragma unroll
             for (int h = 0; h < G; ++h) {
+              const bool is_own = i0 + u == own;
 #pragma unroll
-              for (int c = 0; c < 4; ++c) diff |= uint32_t(raw[u][h][c] >> 32) ^ p.launch_tag;
-              vv0[u][h] = make_float4(__uint_as_float(uint32_t(raw[u][h][0])), __uint_as_float(uint32_t(raw[u][h][1])),
-                                      __uint_as_float(uint32_t(raw[u][h][2])), __uint_as_float(uint32_t(raw[u][h][3])));
+              for (int c = 0; c < 4; ++c)
+                if (!is_own) diff |= uint32_t(raw[u][h][c] >> 32) ^ p.launch_tag;
+              vv0[u][h] = is_own ? acc[h]
+                                 : make_float4(__uint_as_float(uint32_t(raw[u][h][0])), __uint_as_float(uint32_t(raw[u][h][1])),
+                                               __uint_as_float(uint32_t(raw[u][h][2])), __uint_as_float(uint32_t(raw[u][h][3])));
             }
           me = mine ? __uint_as_float(uint32_t(rm)) : -CUDART_INF_F;
           le = mine ? __uint_as_float(uint32_t(rl)) : 0.f;
+          if (mine && ri == own) {
+#pragma unroll
+            for (int h = 0; h < G; ++h)
+              if (rh == h) {
+                me = mh[h];
+                le = lh[h];
+              }
+          }
           if (__all_sync(0xffffffffu, diff == 0)) return true;
-          if (spins > (kWaitLimit >> 6)) return false;
+          if (spins >= max_spins) return false;
         }
       };
-      if (!load_batch(0, me0, le0)) {
+      // The first batch is read once before the ticket is looked at, so that for the warp that turns out to hold the
+      // last ticket the ticket's round trip and these loads run side by side (the other parts stored their records
+      // before they took their tickets; this warp's own record is not awaited).  The others have read a few KiB of
+      // L2 for nothing, at the idle end of their range.
+      const bool early = load_batch(0, me0, le0, 0u);
+      if (__shfl_sync(0xffffffffu, pi == 0 ? tick0 : tick1, 0) != unsigned(sg.n_parts - 1)) continue;
+      if (!early && !load_batch(0, me0, le0, kWaitLimit >> 6)) {
         failed = true;
         break;
       }
@@ -1021,18 +1060,18 @@ glide_decode_stream_kernel(const DecodeParams p, const StreamParams sp) {
       GLIDE_TRACE_EVENT(16);
       // merge the records: maxima and sums first (one (record, head) pair per lane), then the vectors
       float Mg[G], lg[G];
-      float4 acc[G];
+      float4 macc[G];
 #pragma unroll
       for (int h = 0; h < G; ++h) {
         Mg[h] = -CUDART_INF_F;
         lg[h] = 0.f;
-        acc[h] = make_float4(0.f, 0.f, 0.f, 0.f);
+        macc[h] = make_float4(0.f, 0.f, 0.f, 0.f);
       }
       for (int i0 = 0; i0 < sg.n_parts; i0 += RPB) {
         const int rh = lane % G;
         const int nb = sg.n_parts - i0 < RPB ? sg.n_parts - i0 : RPB;
         float me = me0, le = le0;
-        if (i0 > 0 && !load_batch(i0, me, le)) {   // further batches (units cut into more than RPB records)
+        if (i0 > 0 && !load_batch(i0, me, le, kWaitLimit >> 6)) {   // further batches (units cut into more than RPB records)
           failed = true;
           break;
         }
@@ -1049,10 +1088,10 @@ glide_decode_stream_kernel(const DecodeParams p, const StreamParams sp) {
           Mn[h] = fmaxf(Mn[h], Mg[h]);
           const float resc = exp2_or_zero(Mg[h], Mn[h]);
           lg[h] *= resc;
-          acc[h].x *= resc;
-          acc[h].y *= resc;
-          acc[h].z *= resc;
-          acc[h].w *= resc;
+          macc[h].x *= resc;
+          macc[h].y *= resc;
+          macc[h].z *= resc;
+          macc[h].w *= resc;
           Mg[h] = Mn[h];
           if (rh == h) fe = exp2_or_zero(me, Mn[h]);
           lpart[h] = rh == h ? le * fe : 0.f;
@@ -1066,10 +1105,10 @@ glide_decode_stream_kernel(const DecodeParams p, const StreamParams sp) {
           for (int h = 0; h < G; ++h)
             if (u < nb) {
               const float f = __shfl_sync(0xffffffffu, fe, u * G + h);
-              acc[h].x = fmaf(vv0[u][h].x, f, acc[h].x);
-              acc[h].y = fmaf(vv0[u][h].y, f, acc[h].y);
-              acc[h].z = fmaf(vv0[u][h].z, f, acc[h].z);
-              acc[h].w = fmaf(vv0[u][h].w, f, acc[h].w);
+              macc[h].x = fmaf(vv0[u][h].x, f, macc[h].x);
+              macc[h].y = fmaf(vv0[u][h].y, f, macc[h].y);
+              macc[h].z = fmaf(vv0[u][h].z, f, macc[h].z);
+              macc[h].w = fmaf(vv0[u][h].w, f, macc[h].w);
             }
       }
       GLIDE_TRACE_EVENT(17);
@@ -1089,10 +1128,10 @@ glide_decode_stream_kernel(const DecodeParams p, const StreamParams sp) {
         for (int i = 0; i < sg.n_parts && !failed; ++i) {
 #pragma unroll
           for (int h = 0; h < G; ++h) {
-            float4 av;
-            float bv;
+            float4 av = a[h];
+            float bv = bp[h];
             uint32_t spins = 0;   // (the window half of the record carried the tag already: these follow at once)
-            while (!__all_sync(0xffffffffu, ll_load4(r0 + size_t(i) * p.rec_floats + L::kRecW + h * kD + lane * 4, p.launch_tag, av) &&
+            while (i != own && !__all_sync(0xffffffffu, ll_load4(r0 + size_t(i) * p.rec_floats + L::kRecW + h * kD + lane * 4, p.launch_tag, av) &&
                                                 ll_load1(r0 + size_t(i) * p.rec_floats + L::kRecW + G * kD + h, p.launch_tag, bv)))
               if (++spins > (kWaitLimit >> 6)) {
                 failed = true;
@@ -1113,10 +1152,10 @@ glide_decode_stream_kernel(const DecodeParams p, const StreamParams sp) {
         const float den = fmaf(lg[h], fr, fc);
         const float inv = (!SUM || den > 0.f) ? 1.0f / den : 0.f;
         const float il = (SUM && bl[h] > 0.f) ? 1.0f / bl[h] : 0.f;
-        const __nv_bfloat162 lo = __floats2bfloat162_rn(fmaf(fmaf(acc[h].x, fr, fc * vx[0]), inv, SUM ? al[h].x * il : 0.f),
-                                                        fmaf(fmaf(acc[h].y, fr, fc * vx[1]), inv, SUM ? al[h].y * il : 0.f));
-        const __nv_bfloat162 hi = __floats2bfloat162_rn(fmaf(fmaf(acc[h].z, fr, fc * vx[2]), inv, SUM ? al[h].z * il : 0.f),
-                                                        fmaf(fmaf(acc[h].w, fr, fc * vx[3]), inv, SUM ? al[h].w * il : 0.f));
+        const __nv_bfloat162 lo = __floats2bfloat162_rn(fmaf(fmaf(macc[h].x, fr, fc * vx[0]), inv, SUM ? al[h].x * il : 0.f),
+                                                        fmaf(fmaf(macc[h].y, fr, fc * vx[1]), inv, SUM ? al[h].y * il : 0.f));
+        const __nv_bfloat162 hi = __floats2bfloat162_rn(fmaf(fmaf(macc[h].z, fr, fc * vx[2]), inv, SUM ? al[h].z * il : 0.f),
+                                                        fmaf(fmaf(macc[h].w, fr, fc * vx[3]), inv, SUM ? al[h].w * il : 0.f));
         uint2 packed;
         packed.x = *reinterpret_cast<const uint32_t *>(&lo);
         packed.y = *reinterpret_cast<const uint32_t *>(&hi);
@@ -1129,6 +1168,7 @@ glide_decode_stream_kernel(const DecodeParams p, const StreamParams sp) {
         if (p.gated && lane == 0)
           reinterpret_cast<float *>(p.ws + p.layers[sg.layer].ringG)[row / kD] = p.gate ? p.gate[sg.unit] : 1.f;
       }
+      if (lane == 0) p.tickets[sg.unit] = 0;   // for the next launch
       GLIDE_TRACE_EVENT(13);
     }
   }

@@ -78,7 +78,7 @@ struct DecodeParams {
   const int32_t *heads_of;   // [Hkv][G] query heads of each KV head
   Control *ctl;              // work and completion counters (the allocation-free step keeps them in the static buffer)
   int32_t *status;           // the context's status word, in its workspace for every entry point (glide_device_status)
-  int32_t *tickets;          // [units] (per-item kernels; the streaming kernel tags its records instead)
+  int32_t *tickets;          // [units]: arrivals at a unit's global records; the last one merges and clears it
   float *partials;
   int64_t *n_dev;            // [L]
   const int64_t *seq_off;    // [B] position of sequence b minus the layer's counter; null when every offset is zero
@@ -123,7 +123,7 @@ struct StreamSegment {
   int32_t n_state, state0;   // state tiles [state0, state0 + n_state): 16 rows of S each
   int32_t n_win, win0;       // window tiles [win0, win0 + n_win): 16 ring slots each
   int32_t part;              // this group's record among the unit's global records, -1 if the whole unit is in this group
-  int32_t n_parts;           // records of the unit; the warp with part n_parts - 1 merges them
+  int32_t n_parts;           // records of the unit (ticket target)
   int32_t rec0;              // index of the unit's first record in the split-K scratch
   int32_t row_base;          // row of the unit's slot 0 in the layer's [rows][d] ring tensor
   int32_t cap;               // ring slots
