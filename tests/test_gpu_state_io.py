@@ -133,3 +133,40 @@ def test_same_steps_twice_fp32_and_batched():
     b = _run_sequence([64, 200, 0], 4, 8, 4, 64, F32, 300, 5, 37)
     for i, (x, y) in enumerate(zip(a, b)):
         assert torch.equal(x.view(torch.uint8), y.view(torch.uint8)), f"tensor {i} differs between two runs"
+
+
+def test_two_contexts_stepping_on_two_streams_at_once():
+    """Two contexts of config 1's window schedule decode on two streams with nothing ordering one stream against the
+    other, so launches of the streaming kernel may share the SMs.  Each context must produce the bits it produces
+    alone, and no bounded wait may have run out (a merge must never wait for a CTA that is not running)."""
+    windows = [4096] * 2 + [1024] * 3 + [256] * 5 + [64] * 4
+    B, H, Hkv, d, prompt, steps = 1, 32, 8, 128, 4200, 40
+    L = len(windows)
+
+    def build(seed):
+        wl = synth.Workload(seed, L, B, H, Hkv, d, BF16, 4 * d ** -0.5)
+        g = glide.Glide(windows, B, H, Hkv, d, prompt + steps, dtype=BF16, softmax_scale=f32_scale(d))
+        _, k, v = wl.qkv(range(L), range(B), range(prompt), device="cuda")
+        g.glide_prefill(None, k, v, None)
+        inputs = [wl.decode_qkv(prompt + s, device="cuda") for s in range(steps)]
+        return g, inputs
+
+    def run(pairs, streams):
+        outs = [[torch.empty_like(inp[0][0]) for _ in range(steps)] for _, inp in pairs]
+        torch.cuda.synchronize()
+        for s in range(steps):
+            for i, (g, inp) in enumerate(pairs):
+                q, k, v = inp[s]
+                g.glide_decode_step(q, k, v, outs[i][s], stream=streams[i])
+        torch.cuda.synchronize()
+        for g, _ in pairs:
+            assert g.glide_device_status() == 0
+        return outs
+
+    one = torch.cuda.current_stream()
+    alone = run([build(51), build(52)], [one, one])
+    s1, s2 = torch.cuda.Stream(), torch.cuda.Stream()
+    together = run([build(51), build(52)], [s1, s2])
+    for a, b in zip(alone, together):
+        for x, y in zip(a, b):
+            assert torch.equal(x.view(torch.uint8), y.view(torch.uint8))
