@@ -42,7 +42,7 @@ from paper_2607_24788_b200 import configs, synth  # noqa: E402
 L2_BYTES = 126e6
 # dram__bytes_read.sum + dram__bytes_write.sum per decode launch from the committed ncu capture
 # (profiles/), keyed by workload name; None until a capture exists for that workload.
-NCU_TRAFFIC_BYTES = {"c1_llama8b_b1_32k": 141.2e6}   # profiles/decode_stream_c1.md
+NCU_TRAFFIC_BYTES = {"c1_llama8b_b1_32k": 142.1e6}   # profiles/decode_stream_c1.md
 MIN_TIMED_S = 0.5     # the K-step region is repeated until this much timed work has accumulated
 MAX_REPS = 4000
 KERNEL_KNOBS = {}   # tuning overrides from the command line (decode_chunk, decode_state_splits, decode_impl)
