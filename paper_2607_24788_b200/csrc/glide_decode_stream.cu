@@ -1001,7 +1001,7 @@ glide_decode_stream_kernel(const DecodeParams p, const StreamParams sp) {
               asm volatile("ld.relaxed.gpu.global.v2.u64 {%0, %1}, [%2];" : "=l"(raw[u][h][0]), "=l"(raw[u][h][1]) : "l"(src));
               asm volatile("ld.relaxed.gpu.global.v2.u64 {%0, %1}, [%2];" : "=l"(raw[u][h][2]), "=l"(raw[u][h][3]) : "l"(src + 2));
             }
-          uint32_t diff = (!mine || ri != own) ? (uint32_t(rm >> 32) ^ p.launch_tag) | (uint32_t(rl >> 32) ^ p.launch_tag) : 0u;
+          uint32_t diff = (mine && ri != own) ? (uint32_t(rm >> 32) ^ p.launch_tag) | (uint32_t(rl >> 32) ^ p.launch_tag) : 0u;
 #pragma unroll
           for (int u = 0; u < RPB; ++u)
 #pragma unroll
@@ -1009,7 +1009,7 @@ glide_decode_stream_kernel(const DecodeParams p, const StreamParams sp) {
               const bool is_own = i0 + u == own;
 #pragma unroll
               for (int c = 0; c < 4; ++c)
-                if (!is_own) diff |= uint32_t(raw[u][h][c] >> 32) ^ p.launch_tag;
+                if (!is_own && u < nb) diff |= uint32_t(raw[u][h][c] >> 32) ^ p.launch_tag;   // (slots past the last record are not used)
               vv0[u][h] = is_own ? acc[h]
                                  : make_float4(__uint_as_float(uint32_t(raw[u][h][0])), __uint_as_float(uint32_t(raw[u][h][1])),
                                                __uint_as_float(uint32_t(raw[u][h][2])), __uint_as_float(uint32_t(raw[u][h][3])));
