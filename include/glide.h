@@ -69,7 +69,8 @@ typedef enum { GLIDE_F32 = 0, GLIDE_BF16 = 1 } glide_dtype;
  *   phi_W(x) = [ softmax(y) ; softmax(-y) ],   feature dimension 2 * head_dim,
  * a matrix per layer and query head for the queries (phi_wq) and per layer and KV head for the keys (phi_wk).
  * S is then [2d][d] and z [2d] per KV head.  It runs on the CUDA-core kernels and, for bf16 I/O with head_dim 128,
- * the decode step on the streaming kernel (decode_impl AUTO, FMA or STREAM; prefill_impl AUTO or FMA). */
+ * the decode step on the streaming kernel and, under the shared normaliser, prefill outputs on the tcgen05 kernel
+ * (decode_impl AUTO, FMA or STREAM; prefill_impl AUTO, FMA or, with GLIDE_MERGE_SHARED, TCGEN05). */
 typedef enum { GLIDE_PHI_SOFTMAX = 0, GLIDE_PHI_PROJ_SOFTMAX2 = 1 } glide_phi;
 
 /* How the window part and the linear part are merged (Sec. III-B "(+)"; appendix

@@ -680,7 +680,7 @@ int build_ring_tensor_maps(glide_ctx *ctx) {
   }
   EncodeFn encode = reinterpret_cast<EncodeFn>(fn);
   const int L = ctx->cfg.n_layers, D = ctx->cfg.head_dim;
-  ctx->tmaps_host.assign((size_t(L) * 5 + 2) * sizeof(CUtensorMap), 0);
+  ctx->tmaps_host.assign((size_t(L) * 5 + 3) * sizeof(CUtensorMap), 0);
   ctx->tmaps_kv4d = D == 128;
   CUtensorMap *maps = reinterpret_cast<CUtensorMap *>(ctx->tmaps_host.data());
   for (int l = 0; l < L; ++l) {
@@ -721,17 +721,21 @@ int build_ring_tensor_maps(glide_ctx *ctx) {
     }
   }
   if (D == 128 && ctx->off_phik16 != 0) {
-    // prefill scratch as [rows][128] bf16 with boxes of a whole 128-row tile: phi(K') rows of the chunk, [unit][chunk]
-    // rows, and the bf16 copy of S, [unit][128] rows
+    // prefill scratch as [rows][128] bf16 with boxes of a whole 128-row tile: phi(K') rows of the chunk ([unit][chunk]
+    // rows), the bf16 copy of S ([unit][128] rows) and, for the learned map, phi(Q) ([unit][chunk][G] rows); with the
+    // learned map every array holds its two 128-column halves one after the other
     const cuuint64_t units = cuuint64_t(L) * ctx->cfg.batch * ctx->cfg.n_kv_heads;
+    const cuuint64_t halves = cuuint64_t(ctx->dp / D);
     const cuuint64_t strides[1] = {cuuint64_t(D) * 2};
     const cuuint32_t box128[2] = {64, 128};
     const cuuint32_t estr[2] = {1, 1};
-    for (int i = 0; i < 2; ++i) {
-      const cuuint64_t dims[2] = {cuuint64_t(D), units * cuuint64_t(i == 0 ? ctx->prefill_chunk : D)};
-      CUresult r = encode(&maps[5 * L + i], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, ctx->ws + (i == 0 ? ctx->off_phik16 : ctx->off_s16),
-                          dims, strides, box128, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
-                          CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    for (int i = 0; i < (ctx->off_phiq16 ? 3 : 2); ++i) {
+      const cuuint64_t rows = halves * units * (i == 0 ? cuuint64_t(ctx->prefill_chunk) : i == 1 ? cuuint64_t(D) : cuuint64_t(ctx->prefill_chunk) * ctx->G);
+      const cuuint64_t dims[2] = {cuuint64_t(D), rows};
+      const size_t base = i == 0 ? ctx->off_phik16 : i == 1 ? ctx->off_s16 : ctx->off_phiq16;
+      CUresult r = encode(&maps[5 * L + i], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, ctx->ws + base, dims, strides, box128, estr,
+                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
       if (r != CUDA_SUCCESS) return GLIDE_ERR_CUDA;
     }
   }

@@ -61,9 +61,11 @@ int validate_config(const glide_config *c) {
   if (c->reserved_ != 0) return GLIDE_ERR_INVALID_ARG;
   if (c->phi == GLIDE_PHI_PROJ_SOFTMAX2) {
     if (!c->phi_wq || !c->phi_wk || !aligned16(c->phi_wq) || !aligned16(c->phi_wk)) return GLIDE_ERR_INVALID_ARG;
-    // the learned map runs on the CUDA-core kernels and on the streaming decode kernel
+    // the learned map runs on the CUDA-core kernels, on the streaming decode kernel and (shared normaliser) on the
+    // tcgen05 prefill kernel
     if (c->decode_impl == GLIDE_DECODE_MMA) return GLIDE_ERR_UNSUPPORTED;
-    if (c->prefill_impl == GLIDE_PREFILL_MMA_SYNC || c->prefill_impl == GLIDE_PREFILL_TCGEN05) return GLIDE_ERR_UNSUPPORTED;
+    if (c->prefill_impl == GLIDE_PREFILL_MMA_SYNC) return GLIDE_ERR_UNSUPPORTED;
+    if (c->prefill_impl == GLIDE_PREFILL_TCGEN05 && c->merge != GLIDE_MERGE_SHARED) return GLIDE_ERR_UNSUPPORTED;
   } else if (c->phi_wq || c->phi_wk) {
     return GLIDE_ERR_INVALID_ARG;
   }
@@ -183,8 +185,8 @@ int glide::plan_context(const glide_config *cfg, glide_ctx *ctx, std::vector<Wor
   ctx->off_stream_cta = off;
   off = align_up(off + sizeof(int32_t) * (size_t(kMaxStreamCtas) * kStreamWarps + 1), 256);
   ctx->off_tmaps = off;
-  // per layer 3 maps of 16-row boxes, then (from 3 L on) 2 of 128-row boxes, then the two bf16 scratch arrays of prefill
-  off = align_up(off + size_t(128) * (5 * L + 2), 256);
+  // per layer 3 maps of 16-row boxes, then (from 3 L on) 2 of 128-row boxes, then the three bf16 scratch arrays of prefill
+  off = align_up(off + size_t(128) * (5 * L + 3), 256);
   ctx->off_phik = off;
   off = align_up(off + sizeof(float) * size_t(L) * units_per_layer * ctx->prefill_chunk * dp, 256);
   ctx->off_zcum = off;   // running sums of phi(K') over the chunk: only the sum-of-terms merges use them
@@ -197,11 +199,17 @@ int glide::plan_context(const glide_config *cfg, glide_ctx *ctx, std::vector<Wor
   if (cfg->gated) off = align_up(off + sizeof(float) * size_t(L) * units_per_layer * ctx->prefill_chunk, 256);
   // tcgen05 prefill kernel (bf16, head_dim 128, plain feature map): bf16 copies of the chunk's phi(K') rows and of S,
   // which its CTAs fetch by TMA instead of converting the fp32 arrays themselves
-  if (cfg->io_dtype == GLIDE_BF16 && d == 128 && cfg->phi == GLIDE_PHI_SOFTMAX && !cfg->gated) {
+  if (cfg->io_dtype == GLIDE_BF16 && d == 128 && !cfg->gated &&
+      (cfg->phi == GLIDE_PHI_SOFTMAX || cfg->merge == GLIDE_MERGE_SHARED)) {
+    const size_t halves = size_t(dp / d);   // the learned map's two softmax halves are kept apart (one 128-column tensor each)
     ctx->off_phik16 = off;
-    off = align_up(off + 2 * size_t(L) * units_per_layer * ctx->prefill_chunk * d, 256);
+    off = align_up(off + 2 * halves * size_t(L) * units_per_layer * ctx->prefill_chunk * d, 256);
     ctx->off_s16 = off;
-    off = align_up(off + 2 * size_t(L) * units_per_layer * d * d, 256);
+    off = align_up(off + 2 * halves * size_t(L) * units_per_layer * d * d, 256);
+    if (halves == 2) {
+      ctx->off_phiq16 = off;
+      off = align_up(off + 2 * halves * size_t(L) * units_per_layer * ctx->prefill_chunk * ctx->G * d, 256);
+    }
   }
   ctx->off_seqoff = off;   // per-sequence position offsets
   off = align_up(off + sizeof(int64_t) * size_t(cfg->batch), 256);

@@ -156,8 +156,13 @@ struct PrefillParams {
   const int32_t *heads_of;
   Control *ctl;
   float *phik;               // chunk scratch: [layer_count][B][Hkv][C][d] fp32, phi of the delayed keys
-  void *phik16;              // tcgen05 kernel: the same rows as bf16 (read by TMA); nullptr when that kernel is not in use
-  void *s16;                 // tcgen05 kernel: bf16 copy of every unit's S as it is at the start of the chunk, [unit][d][d]
+  void *phik16;              // tcgen05 kernel: the same rows as bf16 (read by TMA), [dp / d halves][units_cap * Cmax][d];
+                             // nullptr when that kernel is not in use
+  void *s16;                 // tcgen05 kernel: bf16 copy of every unit's S as it is at the start of the chunk,
+                             // [dp / d halves][units_cap][d][d]
+  void *phiq16;              // tcgen05 kernel, learned map: phi(q) of the chunk's query rows as bf16,
+                             // [2 halves][units_cap * Cmax * G][d], row = (unit * Cmax + token) * G + head of the group
+  int64_t units_cap;         // L * B * H_kv of the context: what separates the halves in the three arrays above
   float *zcum;               // sum-of-terms merges on the tcgen05 kernel: running sums of phik over the chunk, same shape
   int32_t merge;             // glide_merge
   const void *q, *k, *v;     // the call's inputs
@@ -209,7 +214,7 @@ struct glide_ctx {
   int G = 0;
   int dp = 0;                       // feature dimension of the linear part: d, or 2d for the learned map
   size_t off_phit = 0, off_gcum = 0;
-  size_t off_phik16 = 0, off_s16 = 0;   // bf16 scratch of the tcgen05 prefill kernel (0: not laid out)
+  size_t off_phik16 = 0, off_s16 = 0, off_phiq16 = 0;   // bf16 scratch of the tcgen05 prefill kernel (0: not laid out)
   int device = 0;
   int sm_count = 0;
   int decode_grid = 0;

@@ -127,6 +127,15 @@ __global__ void __launch_bounds__(kPrefillThreads) prefill_phi_kernel(const Pref
         dst[e] = lo[r][e];
         dst[D + e] = hi[r][e];
       }
+      if (p.phik16) {   // the two halves rounded to bf16, each in its own array, for the tensor-core attention kernel
+        __nv_bfloat16 *d16 = reinterpret_cast<__nv_bfloat16 *>(p.phik16) + (size_t(u) * p.Cmax + i0 + r) * D + lane * E;
+        const size_t half = size_t(p.units_cap) * p.Cmax * D;
+#pragma unroll
+        for (int e = 0; e < E; ++e) {
+          d16[e] = __float2bfloat16_rn(lo[r][e]);
+          d16[half + e] = __float2bfloat16_rn(hi[r][e]);
+        }
+      }
     }
   }
 }
@@ -524,11 +533,12 @@ __global__ void __launch_bounds__(kPrefillThreads) prefill_ring_kernel(const Pre
 }
 
 // bf16 copy of the state of every unit of the call as it is before the chunk's state update: what the tcgen05 attention
-// kernel multiplies phi(Q) with (one 16-byte store per thread)
+// kernel multiplies phi(Q) with (one 16-byte store per thread).  With the learned map S has 2 d rows: rows d .. 2d - 1
+// go to the second half of the array.
 __global__ void __launch_bounds__(kPrefillThreads) prefill_s16_kernel(const PrefillParams p) {
   constexpr int D = 128;
   const int64_t id = int64_t(blockIdx.x) * kPrefillThreads + threadIdx.x;   // 8 consecutive entries of one unit's S
-  const int64_t per_unit = D * D / 8;
+  const int64_t per_unit = int64_t(p.dp) * D / 8;
   const int64_t u = id / per_unit;
   if (u >= int64_t(p.layer_count) * p.B * p.Hkv) return;
   const int g = int(u % p.Hkv);
@@ -536,12 +546,62 @@ __global__ void __launch_bounds__(kPrefillThreads) prefill_s16_kernel(const Pref
   const int lrel = int(u / (int64_t(p.Hkv) * p.B));
   const LayerDev ld = p.layers[p.layer_begin + lrel];
   if (!ld.evicts) return;
-  const size_t e0 = size_t(id % per_unit) * 8;
-  const float *src = reinterpret_cast<const float *>(p.ws + ld.S) + (size_t(b + p.b0) * p.Hkv + g) * D * D + e0;
+  const size_t e0 = size_t(id % per_unit) * 8;   // entry of S [dp][d]
+  const float *src = reinterpret_cast<const float *>(p.ws + ld.S) + (size_t(b + p.b0) * p.Hkv + g) * size_t(p.dp) * D + e0;
   const float4 f0 = *reinterpret_cast<const float4 *>(src), f1 = *reinterpret_cast<const float4 *>(src + 4);
   __nv_bfloat162 o[4] = {__floats2bfloat162_rn(f0.x, f0.y), __floats2bfloat162_rn(f0.z, f0.w),
                          __floats2bfloat162_rn(f1.x, f1.y), __floats2bfloat162_rn(f1.z, f1.w)};
-  *reinterpret_cast<uint4 *>(reinterpret_cast<__nv_bfloat16 *>(p.s16) + size_t(u) * D * D + e0) = *reinterpret_cast<const uint4 *>(o);
+  const size_t half = e0 / (size_t(D) * D);
+  *reinterpret_cast<uint4 *>(reinterpret_cast<__nv_bfloat16 *>(p.s16) + half * size_t(p.units_cap) * D * D + size_t(u) * D * D +
+                             (e0 - half * D * D)) = *reinterpret_cast<const uint4 *>(o);
+}
+
+// Learned feature map, tcgen05 attention kernel: phi(q) of every query row of the chunk as bf16, the two softmax halves
+// in two arrays of rows (unit, token, head of the group).  A warp takes kTokPerWarp tokens of one query head (they
+// share the head's projection).
+template <int G>
+__global__ void __launch_bounds__(kPrefillThreads) prefill_phiq16_kernel(const PrefillParams p) {
+  using T = __nv_bfloat16;
+  constexpr int D = 128, E = D / 32;
+  const int lane = threadIdx.x & 31;
+  const int64_t wid = (int64_t(blockIdx.x) * kPrefillThreads + threadIdx.x) >> 5;
+  const int64_t units = int64_t(p.layer_count) * p.B * p.Hkv;
+  const int groups = (p.C + kTokPerWarp - 1) / kTokPerWarp;
+  if (wid >= units * G * groups) return;
+  const int i0 = int(wid % groups) * kTokPerWarp;
+  const int hh = int((wid / groups) % G);
+  const int64_t u = wid / (int64_t(groups) * G);
+  const int g = int(u % p.Hkv);
+  const int b = int((u / p.Hkv) % p.B);
+  const int lrel = int(u / (int64_t(p.Hkv) * p.B));
+  const LayerDev ld = p.layers[p.layer_begin + lrel];
+  if (!ld.evicts) return;
+  const int head = p.heads_of[g * G + hh];
+  const T *qrow = reinterpret_cast<const T *>(p.q) + ((size_t(lrel) * p.B + b) * size_t(p.T) + size_t(p.c0)) * p.H * D + size_t(head) * D;
+  float x[kTokPerWarp][E];
+#pragma unroll
+  for (int r = 0; r < kTokPerWarp; ++r) {
+    if (i0 + r < p.C) {
+      load_elems<T, E>(qrow + size_t(i0 + r) * p.H * D + lane * E, x[r]);
+    } else {
+#pragma unroll
+      for (int e = 0; e < E; ++e) x[r][e] = 0.f;
+    }
+  }
+  float lo[kTokPerWarp][E], hi[kTokPerWarp][E];
+  const T *W = reinterpret_cast<const T *>(p.wq) + (size_t(p.layer_begin + lrel) * p.H + head) * D * D;
+  warp_phi_learned<T, D, kTokPerWarp>(W, x, lo, hi);
+  const size_t half = size_t(p.units_cap) * p.Cmax * G * D;
+#pragma unroll
+  for (int r = 0; r < kTokPerWarp; ++r) {
+    if (i0 + r >= p.C) continue;
+    T *dst = reinterpret_cast<T *>(p.phiq16) + ((size_t(u) * p.Cmax + i0 + r) * G + hh) * D + lane * E;
+#pragma unroll
+    for (int e = 0; e < E; ++e) {
+      dst[e] = __float2bfloat16_rn(lo[r][e]);
+      dst[half + e] = __float2bfloat16_rn(hi[r][e]);
+    }
+  }
 }
 
 }  // namespace
@@ -581,16 +641,20 @@ int launch_prefill(glide_ctx *ctx, int layer_begin, int layer_count, int64_t T, 
   const int64_t units = int64_t(layer_count) * p.B * p.Hkv;
   const bool plain = ctx->cfg.phi == GLIDE_PHI_SOFTMAX && !ctx->cfg.gated;   // what the tensor-core kernels compute
   int impl = ctx->cfg.prefill_impl;
+  // the tcgen05 kernel also takes the learned map under the shared normaliser (its two halves as two linear parts)
+  const bool tc_kind = !ctx->cfg.gated && (ctx->cfg.phi == GLIDE_PHI_SOFTMAX || ctx->cfg.merge == GLIDE_MERGE_SHARED);
   if (impl == GLIDE_PREFILL_AUTO)
-    impl = (plain && prefill_attn_mma_supported(ctx) && ctx->cfg.decode_impl != GLIDE_DECODE_FMA) ? GLIDE_PREFILL_TCGEN05
-                                                                                              : GLIDE_PREFILL_FMA;
+    impl = (tc_kind && prefill_attn_mma_supported(ctx) && ctx->cfg.decode_impl != GLIDE_DECODE_FMA) ? GLIDE_PREFILL_TCGEN05
+                                                                                                : GLIDE_PREFILL_FMA;
   // the tcgen05 kernel needs the ring descriptors of the tensor-core decode kernels (absent when decode_impl asks
   // for the CUDA-core kernel); without them the call uses the mma.sync kernel
-  const bool use_tc = impl == GLIDE_PREFILL_TCGEN05 && prefill_attn_tc_supported(ctx);
+  const bool use_tc = impl == GLIDE_PREFILL_TCGEN05 && tc_kind && prefill_attn_tc_supported(ctx);
   p.phik16 = use_tc && out ? ctx->ws + ctx->off_phik16 : nullptr;
   p.s16 = use_tc && out ? ctx->ws + ctx->off_s16 : nullptr;
+  p.phiq16 = use_tc && out && ctx->off_phiq16 ? ctx->ws + ctx->off_phiq16 : nullptr;
+  p.units_cap = int64_t(ctx->cfg.n_layers) * ctx->cfg.batch * ctx->cfg.n_kv_heads;
   // (the mma.sync kernel has the shared normaliser only: the other merges fall through to the CUDA-core kernel)
-  const bool use_mma = (impl == GLIDE_PREFILL_MMA_SYNC || (impl == GLIDE_PREFILL_TCGEN05 && !use_tc)) &&
+  const bool use_mma = plain && (impl == GLIDE_PREFILL_MMA_SYNC || (impl == GLIDE_PREFILL_TCGEN05 && !use_tc)) &&
                        prefill_attn_mma_supported(ctx) && ctx->cfg.merge == GLIDE_MERGE_SHARED;
   // carry of the chunk scan: tensor cores with an error-free three-way bf16 split of phi(K') (bf16, d = 128), or the
   // CUDA-core kernel (fp32 I/O, d = 64, and whenever the CUDA-core prefill is asked for)
@@ -614,7 +678,11 @@ int launch_prefill(glide_ctx *ctx, int layer_begin, int layer_count, int64_t T, 
       if (out) {
         if (use_tc) {
           if (any_evicts)
-            prefill_s16_kernel<<<unsigned((units * (128 * 128 / 8) + kPrefillThreads - 1) / kPrefillThreads), kPrefillThreads, 0, stream>>>(p);
+            prefill_s16_kernel<<<unsigned((units * (int64_t(p.dp) * 128 / 8) + kPrefillThreads - 1) / kPrefillThreads), kPrefillThreads, 0, stream>>>(p);
+          if (any_evicts && p.phiq16) {
+            const int64_t wq = units * G * ((p.C + kTokPerWarp - 1) / kTokPerWarp);
+            prefill_phiq16_kernel<G><<<unsigned((wq * 32 + kPrefillThreads - 1) / kPrefillThreads), kPrefillThreads, 0, stream>>>(p);
+          }
           if (any_evicts && p.merge != GLIDE_MERGE_SHARED)
             prefill_zcum_kernel<D><<<unsigned((units * D + kPrefillThreads - 1) / kPrefillThreads), kPrefillThreads, 0, stream>>>(p);
           if (launch_prefill_attn_tc(ctx, p, stream) != GLIDE_OK) return GLIDE_ERR_CUDA;

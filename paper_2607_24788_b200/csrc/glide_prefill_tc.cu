@@ -224,7 +224,7 @@ __device__ unsigned long long g_pf_clk[16];
 struct Smem {
   unsigned char q[2][kTileBytes];        // Q_A, Q_B; later phi(Q) 2^-m*
   unsigned char kv[kStages][kTileBytes]; // K and V tiles in turn; linear part: bf16 state, phi(K') tile, V' tile
-  float z[kD];
+  float z[2 * kD];                       // z of the unit (both halves with the learned map)
   uint64_t bar_full[kStages];            // TMA bytes of the buffer have landed
   uint64_t bar_free[kStages];            // the MMAs that read the buffer have completed
   uint64_t bar_q[2];                     // Q_X staged (128 arrivals)
@@ -246,7 +246,7 @@ struct CallMaps {
   CUtensorMap k128, v128;   // boxes of a whole 128-key tile
 };
 
-template <int G, bool SUM>
+template <int G, bool SUM, bool PHI2>
 __global__ void __launch_bounds__(kThreads, 1)   // 10 warps = 3 on one scheduler: 168 registers per thread at most
 prefill_attn_tc_kernel(const PrefillParams p, const CUtensorMap *ring_maps, const __grid_constant__ CallMaps cm) {
   using bf16 = __nv_bfloat16;
@@ -630,7 +630,7 @@ prefill_attn_tc_kernel(const PrefillParams p, const CUtensorMap *ring_maps, cons
       if (!__all_sync(0xffffffffu, ok)) break;
       load_tile(j_lo + int64_t(t) * kKT, sq & 1, slot, smem_u32(&sm.bar_full[slot]), tq_last, false);
     }
-    if (lane == 0 && linear && !*failed) {
+    if (!PHI2 && lane == 0 && linear && !*failed) {
       // the linear part's operands into the buffers the window loop leaves first: the bf16 state (with z), then the
       // phi(K') tiles of the first two intra-chunk steps
       const int n_late = 1 + (n_itiles < 2 ? n_itiles : 2);
@@ -653,7 +653,7 @@ prefill_attn_tc_kernel(const PrefillParams p, const CUtensorMap *ring_maps, cons
     __syncwarp();
     // the V rows of the delayed tokens of the first two intra-chunk steps, behind the window loop's last tiles (the
     // rows of tokens that do not exist yet, below 0, are zero: their weights are, and 0 x anything must stay 0)
-    for (int t = 0; t < n_itiles && t < 2 && __all_sync(0xffffffffu, ok && !*failed); ++t) {
+    for (int t = 0; !PHI2 && t < n_itiles && t < 2 && __all_sync(0xffffffffu, ok && !*failed); ++t) {
       const int sq = late_seq(3 + t);
       if (sq >= 0) ok = mbar_wait(smem_u32(&sm.bar_free[sq % kStages]), uint32_t(sq / kStages) & 1u, failed);
       if (!__all_sync(0xffffffffu, ok)) break;
@@ -679,7 +679,48 @@ prefill_attn_tc_kernel(const PrefillParams p, const CUtensorMap *ring_maps, cons
     ++lin_phase;
     tc_fence_after();
   };
-  if (linear) {
+  // C row of this thread -> bf16 over the same TMEM columns, masked to the delayed tokens j' <= i of the row (the
+  // values already carry 2^-m*); the row's weight sum goes to l
+  auto convert_c = [&](int i0) {
+    if (activeX) {
+      // C row -> bf16, masked to delayed tokens j' <= i of this row (the values already carry 2^-m*)
+      float sum0 = 0.f, sum1 = 0.f;
+      const int lo = i_lo - i0, hi = tl - i0;
+      // a tile that lies wholly before the row tile's first token (and after the first delayed token) needs no mask
+      const bool whole = i0 + kKT - 1 <= tok0 + X * TOKT && i0 >= i_lo;
+      uint32_t ra[32], rb[32];
+      tmem_ld32_nowait(tS, ra);
+#pragma unroll
+      for (int c0 = 0; c0 < kKT; c0 += 32) {
+        uint32_t (&r)[32] = ((c0 >> 5) & 1) ? rb : ra;
+        uint32_t pk[16];
+        tmem_wait_ld();
+        if (c0 + 32 < kKT) tmem_ld32_nowait(tS + c0 + 32, ((c0 >> 5) & 1) ? ra : rb);
+        if (whole) {
+#pragma unroll
+          for (int e = 0; e < 16; ++e) pk[e] = pack_bf16x2(__uint_as_float(r[e * 2]), __uint_as_float(r[e * 2 + 1]));
+        } else {
+#pragma unroll
+          for (int e = 0; e < 16; ++e) {
+            const int i = c0 + e * 2;
+            const float a0 = (i >= lo && i <= hi) ? __uint_as_float(r[e * 2]) : 0.f;
+            const float a1 = (i + 1 >= lo && i + 1 <= hi) ? __uint_as_float(r[e * 2 + 1]) : 0.f;
+            pk[e] = pack_bf16x2(a0, a1);
+          }
+        }
+#pragma unroll
+        for (int e = 0; e < 16; ++e) {
+          sum0 += __uint_as_float(pk[e] << 16);
+          sum1 += __uint_as_float(pk[e] & 0xffff0000u);
+        }
+        tmem_st16(tS + (c0 >> 1), pk);
+      }
+      tmem_wait_st();
+      if (!sum_terms) l_sum += sum0 + sum1;
+    }
+    PF_CLK(4);
+  };
+  if (linear && !PHI2) {
     const bf16 *ringV = reinterpret_cast<const bf16 *>(p.ws + ld.ringV) + unit_rows * kD;
     const bf16 *callV = reinterpret_cast<const bf16 *>(p.v) + (seq * p.Hkv + g) * kD;
     const int64_t call_stride = int64_t(p.Hkv) * kD;
@@ -801,43 +842,7 @@ prefill_attn_tc_kernel(const PrefillParams p, const CUtensorMap *ring_maps, cons
     PF_CLK(3);
     for (int t = 0; t < n_itiles; ++t) {
       const int i0 = it0 + t * kKT;
-      if (activeX) {
-        // C row -> bf16, masked to delayed tokens j' <= i of this row (the values already carry 2^-m*)
-        float sum0 = 0.f, sum1 = 0.f;
-        const int lo = i_lo - i0, hi = tl - i0;
-        // a tile that lies wholly before the row tile's first token (and after the first delayed token) needs no mask
-        const bool whole = i0 + kKT - 1 <= tok0 + X * TOKT && i0 >= i_lo;
-        uint32_t ra[32], rb[32];
-        tmem_ld32_nowait(tS, ra);
-#pragma unroll
-        for (int c0 = 0; c0 < kKT; c0 += 32) {
-          uint32_t (&r)[32] = ((c0 >> 5) & 1) ? rb : ra;
-          uint32_t pk[16];
-          tmem_wait_ld();
-          if (c0 + 32 < kKT) tmem_ld32_nowait(tS + c0 + 32, ((c0 >> 5) & 1) ? ra : rb);
-          if (whole) {
-#pragma unroll
-            for (int e = 0; e < 16; ++e) pk[e] = pack_bf16x2(__uint_as_float(r[e * 2]), __uint_as_float(r[e * 2 + 1]));
-          } else {
-#pragma unroll
-            for (int e = 0; e < 16; ++e) {
-              const int i = c0 + e * 2;
-              const float a0 = (i >= lo && i <= hi) ? __uint_as_float(r[e * 2]) : 0.f;
-              const float a1 = (i + 1 >= lo && i + 1 <= hi) ? __uint_as_float(r[e * 2 + 1]) : 0.f;
-              pk[e] = pack_bf16x2(a0, a1);
-            }
-          }
-#pragma unroll
-          for (int e = 0; e < 16; ++e) {
-            sum0 += __uint_as_float(pk[e] << 16);
-            sum1 += __uint_as_float(pk[e] & 0xffff0000u);
-          }
-          tmem_st16(tS + (c0 >> 1), pk);
-        }
-        tmem_wait_st();
-        if (!sum_terms) l_sum += sum0 + sum1;
-      }
-      PF_CLK(4);
+      convert_c(i0);
       if (t >= 2 && tid < kSoftmaxThreads) cp_async_wait_all();   // (steps after the second: rows copied by these threads)
       fence_async_smem();
       tc_fence_before();
@@ -864,6 +869,136 @@ prefill_attn_tc_kernel(const PrefillParams p, const CUtensorMap *ring_maps, cons
     }
   }
 
+  // Learned feature map (shared normaliser): phi(q) = [softmax(W^T q); softmax(-W^T q)] has 2 d entries, and
+  // phi(q)^T S, phi(q)^T z and phi(Q) phi(K')^T are sums over its two halves; every half is a linear part of the
+  // kind above with its own 128-column tensors.  phi(Q) comes from a kernel in front of this one (the projections
+  // differ per head, and a row tile mixes the heads of the group), as bf16 rows that this thread only scales by
+  // 2^-M.  Everything arrives by TMA after the window loop (the Q tiles and all five K/V buffers are free then):
+  // phi+ of the two row tiles in the Q tiles, phi- in buffers 0 and 1, the state halves and then the phi(K') halves of
+  // each intra-chunk step in buffers 2 and 3, the step's V' rows in buffer 4.
+  if (linear && PHI2) {
+    const bf16 *ringV = reinterpret_cast<const bf16 *>(p.ws + ld.ringV) + unit_rows * kD;
+    const bf16 *callV = reinterpret_cast<const bf16 *>(p.v) + (seq * p.Hkv + g) * kD;
+    const int64_t call_stride = int64_t(p.Hkv) * kD;
+    auto load_vp = [&](int t) {   // softmax threads: V rows of the delayed tokens of step t (MN-major), zero where none
+      const int i0 = it0 + t * kKT;
+      const uint32_t dst = kv_addr(4);
+#pragma unroll 4
+      for (int i = 0; i < kKT * 16 / kSoftmaxThreads; ++i) {
+        const int id = tid + kSoftmaxThreads * i;
+        const int r = id >> 4, c = id & 15;
+        const int ii = i0 + r;
+        const bool valid = ii >= i_lo && ii <= i_hi;
+        const int64_t jj = valid ? folded + ii : 0;
+        const bool from_call = jj >= p.n0;
+        const uint32_t slot_row = (jj >> 32) == 0 ? uint32_t(jj) % cap : uint32_t(uint64_t(jj) % cap);
+        const bf16 *src = from_call ? callV + size_t(jj - p.n0) * call_stride : ringV + size_t(slot_row) * kD;
+        cp_async16(dst + sw128(r, c), src + c * 8, valid);
+      }
+      cp_async_commit();
+    };
+    const CUtensorMap *map_pq = map_pk + 2;
+    const int rows_q = int(p.units_cap) * p.Cmax * G, rows_s = int(p.units_cap) * kD, rows_k = int(p.units_cap) * p.Cmax;
+    auto tma_tile = [&](uint32_t dst, const CUtensorMap *m, int y, uint32_t bar) {
+      tma_load_2d(dst, m, 0, y, bar);
+      tma_load_2d(dst + kBoxBytes, m, 64, y, bar);
+    };
+    if (tid == mma_tid) {
+      const uint32_t bar = smem_u32(&sm.bar_state);
+      mbar_expect_tx(bar, (hasB ? 4u : 2u) * kTileBytes + (need_state ? 2u * kTileBytes + uint32_t(2 * kD * sizeof(float)) : 0u));
+      for (int hf = 0; hf < 2; ++hf)
+        for (int x = 0; x < 2; ++x) {
+          if (x == 1 && !hasB) break;
+          tma_tile(hf == 0 ? sQ[x] : kv_addr(x), map_pq, hf * rows_q + (int(u) * p.Cmax + tok0 + x * TOKT) * G, bar);
+        }
+      if (need_state) {
+        const int ub = (b + p.b0) * p.Hkv + g;
+        tma_tile(kv_addr(2), map_s16, int(u) * kD, bar);
+        tma_tile(kv_addr(3), map_s16, rows_s + int(u) * kD, bar);
+        bulk_load(smem_u32(sm.z), p.ws + ld.z + size_t(ub) * 2 * kD * sizeof(float), uint32_t(2 * kD * sizeof(float)), bar);
+      }
+    }
+    if (tid < kSoftmaxThreads && n_itiles > 0) load_vp(0);
+    float dot = 0.f;
+    if (activeX) {
+      const bool has_lin = tok_abs >= wl;
+      const float M = has_lin ? fmaxf(m_ref, -64.f) : m_ref;   // (the reference of the shared normaliser, as above)
+      const float fw = m_ref == -CUDART_INF_F ? 0.f : ex2(m_ref - M);
+      const float fl = has_lin ? ex2(-M) : 0.f;
+      if (o_init && __any_sync(0xffffffffu, fw != 1.f)) scale_o(fw);
+      l_sum *= fw;
+      mbar_wait(smem_u32(&sm.bar_state), 0u, failed);
+      // this thread's row of phi+ and of phi-: times 2^-M, back as bf16; the dot with z uses the rounded values
+#pragma unroll 1
+      for (int hf = 0; hf < 2; ++hf) {
+        unsigned char *tile = hf == 0 ? sm.q[X] : sm.kv[X];
+#pragma unroll
+        for (int c = 0; c < 16; ++c) {
+          uint4 v4 = *reinterpret_cast<const uint4 *>(tile + sw128(row, c));
+          uint32_t w4[4] = {v4.x, v4.y, v4.z, v4.w};
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            w4[e] = pack_bf16x2(__uint_as_float(w4[e] << 16) * fl, __uint_as_float(w4[e] & 0xffff0000u) * fl);
+            if (need_state)
+              dot += __uint_as_float(w4[e] << 16) * sm.z[hf * kD + c * 8 + e * 2] +
+                     __uint_as_float(w4[e] & 0xffff0000u) * sm.z[hf * kD + c * 8 + e * 2 + 1];
+          }
+          *reinterpret_cast<uint4 *>(tile + sw128(row, c)) = make_uint4(w4[0], w4[1], w4[2], w4[3]);
+        }
+      }
+    }
+    fence_async_smem();
+    tc_fence_before();
+    __syncthreads();
+    if (need_state) {
+      if (tid == mma_tid) {
+        tc_fence_after();
+        mbar_wait(smem_u32(&sm.bar_state), 0u, failed);
+        for (int x = 0; x < 2; ++x) {
+          if (x == 1 && !hasB) break;
+          issue_mma(tmem + 256 + x * 128, sQ[x], kv_addr(2), true, o_init);
+          issue_mma(tmem + 256 + x * 128, kv_addr(x), kv_addr(3), true, true);
+        }
+        mma_commit(smem_u32(&sm.bar_lin));
+      }
+      if (activeX) l_sum += dot;
+      wait_lin();
+      o_init = true;
+    }
+    for (int t = 0; t < n_itiles; ++t) {
+      const int i0 = it0 + t * kKT;
+      if (tid == mma_tid) {
+        // buffers 2 and 3 are free: the products that read them have completed
+        const uint32_t bar = smem_u32(&sm.bar_pk[0]);
+        mbar_expect_tx(bar, 2u * kTileBytes);
+        tma_tile(kv_addr(2), map_pk, int(u) * p.Cmax + i0, bar);
+        tma_tile(kv_addr(3), map_pk, rows_k + int(u) * p.Cmax + i0, bar);
+        mbar_wait(bar, uint32_t(t) & 1u, failed);
+        tc_fence_after();
+        for (int x = 0; x < 2; ++x) {
+          if (x == 1 && !hasB) break;
+          issue_mma(tmem + x * 128, sQ[x], kv_addr(2), false, false);      // C_X = phi+(Q_X) phi+(K')^T ...
+          issue_mma(tmem + x * 128, kv_addr(x), kv_addr(3), false, true);  // ... + phi-(Q_X) phi-(K')^T
+        }
+        mma_commit(smem_u32(&sm.bar_lin));
+      }
+      wait_lin();
+      convert_c(i0);
+      if (tid < kSoftmaxThreads) cp_async_wait_all();   // the step's V' rows
+      fence_async_smem();
+      tc_fence_before();
+      __syncthreads();
+      if (tid == mma_tid) {
+        tc_fence_after();
+        issue_mma_ts(tmem + 256, tmem, kv_addr(4), o_init);
+        if (hasB) issue_mma_ts(tmem + 384, tmem + 128, kv_addr(4), o_init);
+        mma_commit(smem_u32(&sm.bar_lin));
+      }
+      wait_lin();
+      o_init = true;
+      if (t + 1 < n_itiles && tid < kSoftmaxThreads) load_vp(t + 1);
+    }
+  }
   // ---- shared normaliser and store: one contiguous 256-byte row per thread ------------------------------------
   __syncthreads();
   const bool bad = sm.failed != 0;
@@ -969,7 +1104,8 @@ int launch_prefill_attn_tc(glide_ctx *ctx, const PrefillParams &p, cudaStream_t 
       kern<<<unsigned(blocks), kThreads, smem, stream>>>(p, ring_maps, cm);
       return cudaGetLastError() == cudaSuccess ? GLIDE_OK : GLIDE_ERR_CUDA;
     };
-    return p.merge == GLIDE_MERGE_SHARED ? run(prefill_attn_tc_kernel<G, false>) : run(prefill_attn_tc_kernel<G, true>);
+    if (p.phiq16) return run(prefill_attn_tc_kernel<G, false, true>);   // learned map (shared normaliser only)
+    return p.merge == GLIDE_MERGE_SHARED ? run(prefill_attn_tc_kernel<G, false, false>) : run(prefill_attn_tc_kernel<G, true, false>);
   };
   switch (ctx->G) {
     case 1: return launch(IntTag<1>{});

@@ -71,7 +71,9 @@ def test_feature_map_and_gate_argument_checks():
     for kw, code in ((dict(phi=1), glide.GLIDE_ERR_INVALID_ARG),                                  # no weights
                      (dict(phi=0, phi_wq=wq, phi_wk=wk), glide.GLIDE_ERR_INVALID_ARG),            # weights without the map
                      (dict(phi=1, phi_wq=wq, phi_wk=wk, decode_impl=glide.GLIDE_DECODE_MMA), glide.GLIDE_ERR_UNSUPPORTED),
-                     (dict(phi=1, phi_wq=wq, phi_wk=wk, prefill_impl=glide.GLIDE_PREFILL_TCGEN05), glide.GLIDE_ERR_UNSUPPORTED),
+                     (dict(phi=1, phi_wq=wq, phi_wk=wk, prefill_impl=glide.GLIDE_PREFILL_MMA_SYNC), glide.GLIDE_ERR_UNSUPPORTED),
+                     (dict(phi=1, phi_wq=wq, phi_wk=wk, prefill_impl=glide.GLIDE_PREFILL_TCGEN05,
+                           merge=glide.GLIDE_MERGE_SUM_EVICTED), glide.GLIDE_ERR_UNSUPPORTED),
                      (dict(gated=True, decode_impl=glide.GLIDE_DECODE_MMA), glide.GLIDE_ERR_UNSUPPORTED),
                      (dict(gated=True, prefill_impl=glide.GLIDE_PREFILL_TCGEN05), glide.GLIDE_ERR_UNSUPPORTED)):
         with pytest.raises(glide.GlideError) as e:
@@ -92,6 +94,41 @@ def test_learned_map_on_the_streaming_kernel_units_cut_across_ctas(G, B):
     Hkv = 2
     run_case([1500, 64, 0, 5000, 300], B, Hkv * G, Hkv, 128, BF16, [1490, 7], 12, amp=4 * 128 ** -0.5, seed=11 + G,
              phi=1, check_prefill_outputs=False, decode_impl=glide.GLIDE_DECODE_STREAM)
+
+
+@pytest.mark.parametrize("G,chunk,calls", [(4, 0, [144, 130, 61]), (1, 64, [144, 130, 61]), (2, 128, [144, 130, 61]),
+                                           (8, 256, [144, 61]), (1, 512, [300, 40])])
+def test_learned_map_prefill_on_tcgen05(G, chunk, calls):
+    """The learned map's two halves as two linear parts of the tcgen05 prefill kernel: calls that are not multiples of
+    anything, several chunks per call, layers without a ring, with short and long windows and one that never evicts;
+    outputs at every position, the state after every call, decode steps on top."""
+    run_case([0, 16, 100, 128, 304, 1 << 20], 2, 2 * G, 2, 128, BF16, calls, 4, amp=128 ** -0.5 * 4,
+             seed=23 + G, phi=1, prefill_chunk=chunk, prefill_impl=glide.GLIDE_PREFILL_TCGEN05)
+
+
+def test_learned_map_prefill_tcgen05_equals_the_cuda_core_kernel_closely():
+    """Same inputs through the tensor-core and the CUDA-core prefill: both within tolerance of the oracle, and the
+    states they leave (made by the same carry kernel) bit-identical."""
+    from paper_2607_24788_b200 import synth
+    from tests.parity_util import f32_scale, learned_phi_weights
+    windows, B, H, Hkv, d, T = [64, 0, 300], 1, 8, 2, 128, 700
+    L = len(windows)
+    wq, wk = learned_phi_weights(L, H, Hkv, d, BF16, 3)
+    wl = synth.Workload(29, L, B, H, Hkv, d, BF16, 4 * d ** -0.5)
+    q, k, v = wl.qkv(range(L), range(B), range(T), device="cuda")
+    res = []
+    for impl in (glide.GLIDE_PREFILL_TCGEN05, glide.GLIDE_PREFILL_FMA):
+        g = glide.Glide(windows, B, H, Hkv, d, T, dtype=BF16, softmax_scale=f32_scale(d), phi=1, phi_wq=wq, phi_wk=wk,
+                        prefill_impl=impl)
+        out = torch.empty_like(q)
+        g.glide_prefill(q, k, v, out)
+        res.append((out, [g.glide_export_state(l)[2] for l in range(L)]))
+        assert g.glide_device_status() == 0
+    a, b = res
+    err = (a[0].float() - b[0].float()).abs().max().item()
+    assert err <= 2e-2, err
+    for x, y in zip(a[1], b[1]):
+        assert torch.equal(x, y)
 
 
 @pytest.mark.parametrize("phi,G,B", [(0, 4, 1), (0, 8, 2), (1, 4, 1), (0, 1, 3)])
