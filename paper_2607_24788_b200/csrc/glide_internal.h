@@ -243,6 +243,7 @@ int plan_context(const glide_config *cfg, glide_ctx *ctx, std::vector<WorkItem> 
 
 DecodeParams make_decode_params(const glide_ctx *ctx, int layer_begin, int layer_count, const void *q, const void *k,
                                 const void *v, void *out);
+int launch_prefill_project(glide_ctx *ctx, const PrefillParams &p, bool keys, cudaStream_t stream);   // learned map on the tensor cores
 int build_ring_tensor_maps(glide_ctx *ctx);   // TMA descriptors of every layer's K and V ring (host copy)
 int mma_decode_setup(glide_ctx *ctx);         // sizes the grid of the per-item tensor-core kernel
 int stream_decode_supported(const glide_ctx *ctx);

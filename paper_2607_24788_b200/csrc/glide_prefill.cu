@@ -12,6 +12,7 @@
 // The delayed rows and the window rows older than the call come from the ring, which step 4 of
 // the same chunk overwrites only after steps 1-3 have read it.
 #include <algorithm>
+#include <type_traits>
 
 #include "glide_device.cuh"
 
@@ -556,54 +557,6 @@ __global__ void __launch_bounds__(kPrefillThreads) prefill_s16_kernel(const Pref
                              (e0 - half * D * D)) = *reinterpret_cast<const uint4 *>(o);
 }
 
-// Learned feature map, tcgen05 attention kernel: phi(q) of every query row of the chunk as bf16, the two softmax halves
-// in two arrays of rows (unit, token, head of the group).  A warp takes kTokPerWarp tokens of one query head (they
-// share the head's projection).
-template <int G>
-__global__ void __launch_bounds__(kPrefillThreads) prefill_phiq16_kernel(const PrefillParams p) {
-  using T = __nv_bfloat16;
-  constexpr int D = 128, E = D / 32;
-  const int lane = threadIdx.x & 31;
-  const int64_t wid = (int64_t(blockIdx.x) * kPrefillThreads + threadIdx.x) >> 5;
-  const int64_t units = int64_t(p.layer_count) * p.B * p.Hkv;
-  const int groups = (p.C + kTokPerWarp - 1) / kTokPerWarp;
-  if (wid >= units * G * groups) return;
-  const int i0 = int(wid % groups) * kTokPerWarp;
-  const int hh = int((wid / groups) % G);
-  const int64_t u = wid / (int64_t(groups) * G);
-  const int g = int(u % p.Hkv);
-  const int b = int((u / p.Hkv) % p.B);
-  const int lrel = int(u / (int64_t(p.Hkv) * p.B));
-  const LayerDev ld = p.layers[p.layer_begin + lrel];
-  if (!ld.evicts) return;
-  const int head = p.heads_of[g * G + hh];
-  const T *qrow = reinterpret_cast<const T *>(p.q) + ((size_t(lrel) * p.B + b) * size_t(p.T) + size_t(p.c0)) * p.H * D + size_t(head) * D;
-  float x[kTokPerWarp][E];
-#pragma unroll
-  for (int r = 0; r < kTokPerWarp; ++r) {
-    if (i0 + r < p.C) {
-      load_elems<T, E>(qrow + size_t(i0 + r) * p.H * D + lane * E, x[r]);
-    } else {
-#pragma unroll
-      for (int e = 0; e < E; ++e) x[r][e] = 0.f;
-    }
-  }
-  float lo[kTokPerWarp][E], hi[kTokPerWarp][E];
-  const T *W = reinterpret_cast<const T *>(p.wq) + (size_t(p.layer_begin + lrel) * p.H + head) * D * D;
-  warp_phi_learned<T, D, kTokPerWarp>(W, x, lo, hi);
-  const size_t half = size_t(p.units_cap) * p.Cmax * G * D;
-#pragma unroll
-  for (int r = 0; r < kTokPerWarp; ++r) {
-    if (i0 + r >= p.C) continue;
-    T *dst = reinterpret_cast<T *>(p.phiq16) + ((size_t(u) * p.Cmax + i0 + r) * G + hh) * D + lane * E;
-#pragma unroll
-    for (int e = 0; e < E; ++e) {
-      dst[e] = __float2bfloat16_rn(lo[r][e]);
-      dst[half + e] = __float2bfloat16_rn(hi[r][e]);
-    }
-  }
-}
-
 }  // namespace
 
 int launch_prefill(glide_ctx *ctx, int layer_begin, int layer_count, int64_t T, const void *q, const void *k,
@@ -672,17 +625,21 @@ int launch_prefill(glide_ctx *ctx, int layer_begin, int layer_count, int64_t T, 
       const unsigned warp_blocks = unsigned((warps * 32 + kPrefillThreads - 1) / kPrefillThreads);
       const int64_t warps4 = units * ((p.C + kTokPerWarp - 1) / kTokPerWarp);
       const unsigned warp4_blocks = unsigned((warps4 * 32 + kPrefillThreads - 1) / kPrefillThreads);
-      if (any_evicts) prefill_phi_kernel<TT, D, DP><<<warp4_blocks, kPrefillThreads, 0, stream>>>(p);
+      // the learned map's projections of the delayed keys go to the tensor cores for bf16 / d = 128 unless the
+      // CUDA-core prefill was asked for
+      constexpr bool kCanProject = DP == 2 * D && D == 128 && std::is_same<TT, __nv_bfloat16>::value;
+      if (any_evicts && kCanProject && impl != GLIDE_PREFILL_FMA) {
+        if (launch_prefill_project(ctx, p, true, stream) != GLIDE_OK) return GLIDE_ERR_CUDA;
+      } else if (any_evicts) {
+        prefill_phi_kernel<TT, D, DP><<<warp4_blocks, kPrefillThreads, 0, stream>>>(p);
+      }
       if (any_evicts && p.gated)
         prefill_gcum_kernel<TT, D><<<unsigned((units + kPrefillThreads - 1) / kPrefillThreads), kPrefillThreads, 0, stream>>>(p);
       if (out) {
         if (use_tc) {
           if (any_evicts)
             prefill_s16_kernel<<<unsigned((units * (int64_t(p.dp) * 128 / 8) + kPrefillThreads - 1) / kPrefillThreads), kPrefillThreads, 0, stream>>>(p);
-          if (any_evicts && p.phiq16) {
-            const int64_t wq = units * G * ((p.C + kTokPerWarp - 1) / kTokPerWarp);
-            prefill_phiq16_kernel<G><<<unsigned((wq * 32 + kPrefillThreads - 1) / kPrefillThreads), kPrefillThreads, 0, stream>>>(p);
-          }
+          if (any_evicts && p.phiq16 && launch_prefill_project(ctx, p, false, stream) != GLIDE_OK) return GLIDE_ERR_CUDA;
           if (any_evicts && p.merge != GLIDE_MERGE_SHARED)
             prefill_zcum_kernel<D><<<unsigned((units * D + kPrefillThreads - 1) / kPrefillThreads), kPrefillThreads, 0, stream>>>(p);
           if (launch_prefill_attn_tc(ctx, p, stream) != GLIDE_OK) return GLIDE_ERR_CUDA;

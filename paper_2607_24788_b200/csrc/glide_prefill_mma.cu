@@ -480,6 +480,156 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_attn_mma_kernel(const Pre
 
 }  // namespace
 
+namespace {
+// Learned feature map of the chunk's query rows for the tcgen05 attention kernel: Y = X W on the tensor cores (X: 128
+// tokens of one query head, bf16; W: the head's d x d projection; fp32 accumulation), then phi = [softmax(Y);
+// softmax(-Y)] per row, written as bf16 into the two half arrays, row (unit, token, head of the group).
+// One CTA of 8 warps per (layer, sequence, query head, 128 tokens); a warp owns 16 rows, whose 128 outputs sit in its
+// accumulator fragments (a row's entries across the four lanes of a quad).
+constexpr int kProjRows = 128;
+struct ProjSmem {
+  unsigned char x[kProjRows * kRowBytes];   // swizzled [token][128] bf16
+  unsigned char w[kD * kRowBytes];          // swizzled [i][j] bf16
+};
+// KEYS: the same for the chunk's delayed keys k'_i = k_(i - w) of one unit (ring rows for tokens older than the call, the
+// call's rows otherwise; the KV head's projection): fp32 rows [unit][chunk][2d] for the carry and the bf16 halves.
+template <int G, bool KEYS>
+__global__ void __launch_bounds__(kThreads) prefill_project_mma_kernel(const PrefillParams p) {
+  using bf16 = __nv_bfloat16;
+  extern __shared__ __align__(128) unsigned char proj_raw[];
+  ProjSmem &sm = *reinterpret_cast<ProjSmem *>(proj_raw);
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int blocks_per_head = (p.C + kProjRows - 1) / kProjRows;
+  const int i0 = int(blockIdx.x % blocks_per_head) * kProjRows;
+  const int64_t uh = blockIdx.x / blocks_per_head;   // (unit, head of the group); KEYS: the unit
+  const int hh = KEYS ? 0 : int(uh % G);
+  const int64_t u = KEYS ? uh : uh / G;
+  const int g = int(u % p.Hkv);
+  const int b = int((u / p.Hkv) % p.B);
+  const int lrel = int(u / (int64_t(p.Hkv) * p.B));
+  const LayerDev ld = p.layers[p.layer_begin + lrel];
+  if (!ld.evicts) return;
+  const int head = p.heads_of[g * G + hh];
+  const int ntok = min(kProjRows, p.C - i0);
+  const size_t seq = (size_t(lrel) * p.B + b) * size_t(p.T);
+  const bf16 *qrow = reinterpret_cast<const bf16 *>(p.q) + (seq + size_t(p.c0 + i0)) * p.H * kD + size_t(head) * kD;
+  const bf16 *callK = reinterpret_cast<const bf16 *>(p.k) + (seq * p.Hkv + g) * kD;
+  const uint64_t cap = ld.cap > 0 ? uint64_t(ld.cap) : 1u;
+  const bf16 *ringK = reinterpret_cast<const bf16 *>(p.ws + ld.ringK) + (size_t(b + p.b0) * p.Hkv + g) * size_t(ld.cap) * kD;
+  const int64_t j0 = p.n0 + p.c0 + i0 - ld.wlin;   // the delayed token of the tile's first row
+  const bf16 *W = KEYS ? reinterpret_cast<const bf16 *>(p.wk) + (size_t(p.layer_begin + lrel) * p.Hkv + g) * kD * kD
+                       : reinterpret_cast<const bf16 *>(p.wq) + (size_t(p.layer_begin + lrel) * p.H + head) * kD * kD;
+  const uint32_t sX = smem_u32(sm.x), sW = smem_u32(sm.w);
+  for (int id = tid; id < kProjRows * 16; id += kThreads) {
+    const int r = id >> 4, c = id & 15;
+    if (KEYS) {
+      const int64_t j = j0 + r;
+      const bool valid = r < ntok && j >= 0;
+      const bf16 *src = !valid ? callK : (j >= p.n0 ? callK + size_t(j - p.n0) * p.Hkv * kD : ringK + size_t(uint64_t(j) % cap) * kD);
+      cp_async16(sX + swz(r, c), src + c * 8, valid);
+    } else {
+      cp_async16(sX + swz(r, c), qrow + size_t(r < ntok ? r : 0) * p.H * kD + c * 8, r < ntok);
+    }
+  }
+  for (int id = tid; id < kD * 16; id += kThreads) {
+    const int r = id >> 4, c = id & 15;
+    cp_async16(sW + swz(r, c), W + size_t(r) * kD + c * 8, true);
+  }
+  cp_async_commit();
+  cp_async_wait<0>();
+  __syncthreads();
+
+  const int r0 = warp * 16;
+  float y[kD / 8][4];
+#pragma unroll
+  for (int nt = 0; nt < kD / 8; ++nt) y[nt][0] = y[nt][1] = y[nt][2] = y[nt][3] = 0.f;
+#pragma unroll
+  for (int ks = 0; ks < kD / 16; ++ks) {
+    uint32_t af[4];
+    ldsm_x4(af, sX + swz(r0 + (lane & 7) + ((lane >> 3) & 1) * 8, 2 * ks + (lane >> 4)));
+    const int krow = ks * 16 + (lane & 7) + ((lane >> 3) & 1) * 8;
+#pragma unroll
+    for (int dp = 0; dp < kD / 16; ++dp) {
+      uint32_t bfr[4];
+      ldsm_x4_trans(bfr, sW + swz(krow, 2 * dp + (lane >> 4)));
+      mma16816(y[2 * dp], af, bfr[0], bfr[1]);
+      mma16816(y[2 * dp + 1], af, bfr[2], bfr[3]);
+    }
+  }
+  // rows r0 + lane / 4 (entries [.][0], [.][1]) and that + 8 (entries [.][2], [.][3]); columns nt * 8 + (lane & 3) * 2 + {0, 1}
+  constexpr float kLog2e = 1.4426950408889634f;
+#pragma unroll
+  for (int rr = 0; rr < 2; ++rr) {
+    float mx = -CUDART_INF_F, mn = CUDART_INF_F;
+#pragma unroll
+    for (int nt = 0; nt < kD / 8; ++nt) {
+      mx = fmaxf(mx, fmaxf(y[nt][2 * rr], y[nt][2 * rr + 1]));
+      mn = fminf(mn, fminf(y[nt][2 * rr], y[nt][2 * rr + 1]));
+    }
+    mx = quad_max(mx);
+    mn = -quad_max(-mn);
+    float sp = 0.f, sn = 0.f;
+    float ep[kD / 8][2], en[kD / 8][2];
+#pragma unroll
+    for (int nt = 0; nt < kD / 8; ++nt)
+#pragma unroll
+      for (int e = 0; e < 2; ++e) {
+        ep[nt][e] = ex2((y[nt][2 * rr + e] - mx) * kLog2e);
+        en[nt][e] = ex2((mn - y[nt][2 * rr + e]) * kLog2e);
+        sp += ep[nt][e];
+        sn += en[nt][e];
+      }
+    const float ip = 1.0f / quad_sum(sp), in = 1.0f / quad_sum(sn);
+    const int tok = r0 + (lane >> 2) + rr * 8;
+    if (tok >= ntok || (KEYS && j0 + tok < 0)) continue;
+    const int col = (lane & 3) * 2;
+    if (KEYS) {
+      float *d32 = p.phik + (size_t(u) * p.Cmax + i0 + tok) * (2 * kD) + col;
+#pragma unroll
+      for (int nt = 0; nt < kD / 8; ++nt) {
+        *reinterpret_cast<float2 *>(d32 + nt * 8) = make_float2(ep[nt][0] * ip, ep[nt][1] * ip);
+        *reinterpret_cast<float2 *>(d32 + kD + nt * 8) = make_float2(en[nt][0] * in, en[nt][1] * in);
+      }
+    }
+    bf16 *dst = KEYS ? reinterpret_cast<bf16 *>(p.phik16) + (size_t(u) * p.Cmax + i0 + tok) * kD + col
+                     : reinterpret_cast<bf16 *>(p.phiq16) + ((size_t(u) * p.Cmax + i0 + tok) * G + hh) * kD + col;
+    const size_t half = KEYS ? size_t(p.units_cap) * p.Cmax * kD : size_t(p.units_cap) * p.Cmax * G * kD;
+    if (dst != nullptr && (!KEYS || p.phik16)) {
+#pragma unroll
+      for (int nt = 0; nt < kD / 8; ++nt) {
+        *reinterpret_cast<__nv_bfloat162 *>(dst + nt * 8) = __floats2bfloat162_rn(ep[nt][0] * ip, ep[nt][1] * ip);
+        *reinterpret_cast<__nv_bfloat162 *>(dst + half + nt * 8) = __floats2bfloat162_rn(en[nt][0] * in, en[nt][1] * in);
+      }
+    }
+  }
+}
+}  // namespace
+
+// phi_W of the chunk's query rows (keys = false) or of its delayed keys (keys = true) on the tensor cores (see the kernel)
+int launch_prefill_project(glide_ctx *ctx, const PrefillParams &p, bool keys, cudaStream_t stream) {
+  const int64_t units = int64_t(p.layer_count) * p.B * p.Hkv;
+  auto launch = [&](auto gg) -> int {
+    constexpr int G = decltype(gg)::value;
+    auto run = [&](auto kern, int64_t blocks) -> int {
+      if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, int(sizeof(ProjSmem))) != cudaSuccess) {
+        cudaGetLastError();
+        return GLIDE_ERR_CUDA;
+      }
+      kern<<<unsigned(blocks), kThreads, sizeof(ProjSmem), stream>>>(p);
+      return cudaGetLastError() == cudaSuccess ? GLIDE_OK : GLIDE_ERR_CUDA;
+    };
+    const int64_t tiles = (p.C + kProjRows - 1) / kProjRows;
+    return keys ? run(prefill_project_mma_kernel<G, true>, units * tiles) : run(prefill_project_mma_kernel<G, false>, units * G * tiles);
+  };
+  switch (ctx->G) {
+    case 1: return launch(IntTag<1>{});
+    case 2: return launch(IntTag<2>{});
+    case 4: return launch(IntTag<4>{});
+    case 8: return launch(IntTag<8>{});
+    default: return GLIDE_ERR_UNSUPPORTED;
+  }
+}
+
 bool prefill_attn_mma_supported(const glide_ctx *ctx) {
   return ctx->cfg.io_dtype == GLIDE_BF16 && ctx->cfg.head_dim == kD;
 }

@@ -107,8 +107,9 @@ def test_learned_map_prefill_on_tcgen05(G, chunk, calls):
 
 
 def test_learned_map_prefill_tcgen05_equals_the_cuda_core_kernel_closely():
-    """Same inputs through the tensor-core and the CUDA-core prefill: both within tolerance of the oracle, and the
-    states they leave (made by the same carry kernel) bit-identical."""
+    """Same inputs through the tensor-core and the CUDA-core prefill: outputs within the bf16 tolerance of each other,
+    and the states they leave (same carry kernel; the keys' features from the tensor cores on one route, from the
+    CUDA cores on the other) within the state tolerance."""
     from paper_2607_24788_b200 import synth
     from tests.parity_util import f32_scale, learned_phi_weights
     windows, B, H, Hkv, d, T = [64, 0, 300], 1, 8, 2, 128, 700
@@ -128,7 +129,8 @@ def test_learned_map_prefill_tcgen05_equals_the_cuda_core_kernel_closely():
     err = (a[0].float() - b[0].float()).abs().max().item()
     assert err <= 2e-2, err
     for x, y in zip(a[1], b[1]):
-        assert torch.equal(x, y)
+        rel = ((x.double() - y.double()).norm() / y.double().norm().clamp_min(1e-30)).item()
+        assert rel <= 1e-5, rel
 
 
 @pytest.mark.parametrize("phi,G,B", [(0, 4, 1), (0, 8, 2), (1, 4, 1), (0, 1, 3)])
