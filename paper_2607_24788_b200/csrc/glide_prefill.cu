@@ -611,7 +611,7 @@ int launch_prefill(glide_ctx *ctx, int layer_begin, int layer_count, int64_t T, 
                        prefill_attn_mma_supported(ctx) && ctx->cfg.merge == GLIDE_MERGE_SHARED;
   // carry of the chunk scan: tensor cores with an error-free three-way bf16 split of phi(K') (bf16, d = 128), or the
   // CUDA-core kernel (fp32 I/O, d = 64, and whenever the CUDA-core prefill is asked for)
-  const bool state_mma = plain && prefill_state_mma_supported(ctx) && impl != GLIDE_PREFILL_FMA;
+  const bool state_mma = !ctx->cfg.gated && prefill_state_mma_supported(ctx) && impl != GLIDE_PREFILL_FMA;   // (either feature map)
   bool any_evicts = false;
   for (int l = layer_begin; l < layer_begin + layer_count; ++l) any_evicts = any_evicts || ctx->layers[l].evicts;
 

@@ -58,7 +58,7 @@ __device__ __forceinline__ void split3(float x0, float x1, uint32_t &hi, uint32_
 __global__ void __launch_bounds__(kThreads) prefill_state_mma_kernel(const PrefillParams p) {
   using bf16 = __nv_bfloat16;
   __shared__ __align__(16) unsigned char stage[2][kPhiBytes + kVBytes];
-  constexpr int blocks_per_unit = kD / kRowsPerCta;
+  const int blocks_per_unit = p.dp / kRowsPerCta;   // rows of S: d, or 2 d with the learned feature map
   const int64_t u = blockIdx.x / blocks_per_unit;
   const int rb = blockIdx.x % blocks_per_unit;
   const int g = int(u % p.Hkv);
@@ -77,7 +77,7 @@ __global__ void __launch_bounds__(kThreads) prefill_state_mma_kernel(const Prefi
   const bf16 *ringV = reinterpret_cast<const bf16 *>(p.ws + ld.ringV) + size_t(ub) * size_t(ld.cap) * kD;
   const bf16 *callV = reinterpret_cast<const bf16 *>(p.v) + ((size_t(lrel) * p.B + b) * size_t(p.T) * p.Hkv + g) * kD;
   const int64_t call_stride = int64_t(p.Hkv) * kD;
-  const float *pk = p.phik + size_t(u) * p.Cmax * kD + rb * kRowsPerCta;
+  const float *pk = p.phik + size_t(u) * p.Cmax * p.dp + rb * kRowsPerCta;
 
   float acc[kD / 8][4];
 #pragma unroll
@@ -90,7 +90,7 @@ __global__ void __launch_bounds__(kThreads) prefill_state_mma_kernel(const Prefi
     const uint32_t sphi = smem_addr(stage[buf]), sv = sphi + kPhiBytes;
     for (int e = tid; e < kTok * (kRowsPerCta / 4); e += kThreads) {
       const int i = e / (kRowsPerCta / 4), c4 = e % (kRowsPerCta / 4);
-      cp16(sphi + uint32_t(i * kPhiStride + c4 * 4) * 4u, pk + size_t(i0 + (i < nt ? i : 0)) * kD + c4 * 4, i < nt);
+      cp16(sphi + uint32_t(i * kPhiStride + c4 * 4) * 4u, pk + size_t(i0 + (i < nt ? i : 0)) * p.dp + c4 * 4, i < nt);
     }
     for (int e = tid; e < kTok * 16; e += kThreads) {
       const int i = e >> 4, c = e & 15;
@@ -143,7 +143,7 @@ __global__ void __launch_bounds__(kThreads) prefill_state_mma_kernel(const Prefi
     __syncthreads();   // the stage is refilled by the next iteration's issue
   }
   // accumulator fragment: c0, c1 -> (row gid, cols 2 tig + {0,1}); c2, c3 -> row gid + 8
-  float *Sb = reinterpret_cast<float *>(p.ws + ld.S) + size_t(ub) * kD * kD + size_t(rb * kRowsPerCta + warp * 16) * kD;
+  float *Sb = reinterpret_cast<float *>(p.ws + ld.S) + size_t(ub) * p.dp * kD + size_t(rb * kRowsPerCta + warp * 16) * kD;
 #pragma unroll
   for (int n = 0; n < kD / 8; ++n) {
     float2 *d0 = reinterpret_cast<float2 *>(Sb + size_t(gid) * kD + n * 8 + 2 * tig);
@@ -157,7 +157,7 @@ __global__ void __launch_bounds__(kThreads) prefill_state_mma_kernel(const Prefi
     *d1 = c1;
   }
   if (tid < kRowsPerCta) {
-    float *zb = reinterpret_cast<float *>(p.ws + ld.z) + size_t(ub) * kD + rb * kRowsPerCta;
+    float *zb = reinterpret_cast<float *>(p.ws + ld.z) + size_t(ub) * p.dp + rb * kRowsPerCta;
     zb[tid] += zacc;
   }
 }
@@ -171,7 +171,7 @@ bool prefill_state_mma_supported(const glide_ctx *ctx) {
 int launch_prefill_state_mma(glide_ctx *ctx, const PrefillParams &p, cudaStream_t stream) {
   (void)ctx;
   const int64_t units = int64_t(p.layer_count) * p.B * p.Hkv;
-  prefill_state_mma_kernel<<<unsigned(units * (kD / kRowsPerCta)), kThreads, 0, stream>>>(p);
+  prefill_state_mma_kernel<<<unsigned(units * (p.dp / kRowsPerCta)), kThreads, 0, stream>>>(p);
   return cudaGetLastError() == cudaSuccess ? GLIDE_OK : GLIDE_ERR_CUDA;
 }
 
