@@ -312,14 +312,14 @@ __device__ __forceinline__ void warp_sum_multi(float (&x)[N]) {
 }
 
 // ---- the kernel -----------------------------------------------------------------------------
-// MODE 0: shared normaliser; 1: the sum of two normalised terms; 2: shared normaliser with the learned feature map
+// MODE bit 0: the sum of two normalised terms instead of the shared normaliser; bit 1: the learned feature map
 // (feature dimension 2 kD: 16 state tiles per unit, and every state tile arrives with its 16 entries of phi(q_h) and
 // of phi(k_e), which the feature kernel in front of this launch has written)
 template <int G, int STAGES, int MODE, bool RAGGED>
 __global__ void __launch_bounds__(kThreads, GLIDE_STREAM_CTAS_PER_SM)
 glide_decode_stream_kernel(const DecodeParams p, const StreamParams sp) {
   using bf16 = __nv_bfloat16;
-  constexpr bool SUM = MODE == 1, PHI2 = MODE == 2;
+  constexpr bool SUM = (MODE & 1) != 0, PHI2 = (MODE & 2) != 0;
   constexpr int kPhiTile = (G + 1) * 16;   // floats of feature values per state tile
   using L = Layout<G, SUM>;
   constexpr int KS = kD / 16;
@@ -1180,16 +1180,16 @@ glide_decode_stream_kernel(const DecodeParams p, const StreamParams sp) {
 
 template <int G, int STAGES, int MODE>
 size_t stream_smem_bytes(int max_segs, int pool_slots) {
-  using L = Layout<G, MODE == 1>;
+  using L = Layout<G, (MODE & 1) != 0>;
   return 1024 + size_t(kWarps) * STAGES * kStageBytes + size_t(kWarps) * L::kHdrBytes + size_t(kWarps) * STAGES * 64 +
          size_t(max_segs) * sizeof(StreamSegment) + size_t(kWarps) * (STAGES + 1) * 8 + size_t(kStreamMaxGroups) * 4 +
-         (MODE == 2 ? size_t(kWarps) * STAGES * (G + 1) * 64 : 0) + size_t(pool_slots) * L::kRecFloats * 4 +
+         ((MODE & 2) ? size_t(kWarps) * STAGES * (G + 1) * 64 : 0) + size_t(pool_slots) * L::kRecFloats * 4 +
          size_t(max_segs) * 8;
 }
 
 // the kernel's MODE for a context
 int stream_mode(const glide_ctx *ctx) {
-  return ctx->cfg.phi == GLIDE_PHI_PROJ_SOFTMAX2 ? 2 : (ctx->cfg.merge != GLIDE_MERGE_SHARED ? 1 : 0);
+  return (ctx->cfg.phi == GLIDE_PHI_PROJ_SOFTMAX2 ? 2 : 0) | (ctx->cfg.merge != GLIDE_MERGE_SHARED ? 1 : 0);
 }
 
 // f(group size, stages, mode)
@@ -1197,7 +1197,8 @@ template <typename F>
 int dispatch_stream(int G, int mode, F &&f) {
 #define GLIDE_STREAM_CASE(GG)                                                                   \
   case GG:                                                                                      \
-    return mode == 2   ? f(IntTag<GG>{}, IntTag<GLIDE_STREAM_STAGES>{}, IntTag<2>{})            \
+    return mode == 3   ? f(IntTag<GG>{}, IntTag<GLIDE_STREAM_STAGES>{}, IntTag<3>{})            \
+           : mode == 2 ? f(IntTag<GG>{}, IntTag<GLIDE_STREAM_STAGES>{}, IntTag<2>{})            \
            : mode == 1 ? f(IntTag<GG>{}, IntTag<GLIDE_STREAM_STAGES>{}, IntTag<1>{})            \
                        : f(IntTag<GG>{}, IntTag<GLIDE_STREAM_STAGES>{}, IntTag<0>{});
   switch (G) {
@@ -1492,9 +1493,7 @@ void build_stream_schedule(const glide_ctx *ctx, int layer_begin, int layer_coun
 }
 
 int stream_decode_supported(const glide_ctx *ctx) {
-  // (the learned feature map with the shared normaliser only)
-  return ctx->cfg.io_dtype == GLIDE_BF16 && ctx->cfg.head_dim == kD &&
-         (ctx->cfg.phi == GLIDE_PHI_SOFTMAX || ctx->cfg.merge == GLIDE_MERGE_SHARED);
+  return ctx->cfg.io_dtype == GLIDE_BF16 && ctx->cfg.head_dim == kD;
 }
 
 // Host-only part of the set-up: every schedule of the context for a device with n_ctas SMs and smem_limit bytes of

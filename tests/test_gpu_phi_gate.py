@@ -87,6 +87,16 @@ def test_feature_map_and_gate_argument_checks():
     assert e.value.code == glide.GLIDE_ERR_INVALID_ARG
 
 
+@pytest.mark.parametrize("merge,G", [(glide.GLIDE_MERGE_SUM_EVICTED, 4), (glide.GLIDE_MERGE_SUM_ALL, 4),
+                                     (glide.GLIDE_MERGE_SUM_EVICTED, 8), (glide.GLIDE_MERGE_SUM_ALL, 1)])
+def test_learned_map_with_sum_of_terms_merges_on_the_streaming_kernel(merge, G):
+    """Both options at once on the streaming decode kernel (records twice as wide, 16 state tiles per unit), with
+    units inside one warp, shared by the warps of a CTA and cut across CTAs."""
+    Hkv = 2
+    run_case([1500, 64, 0, 5000, 300], 1, Hkv * G, Hkv, 128, BF16, [1490, 7], 10, amp=4 * 128 ** -0.5, seed=31 + G,
+             phi=1, merge=merge, check_prefill_outputs=False, decode_impl=glide.GLIDE_DECODE_STREAM)
+
+
 @pytest.mark.parametrize("G,B", [(4, 1), (1, 3), (8, 2)])
 def test_learned_map_on_the_streaming_kernel_units_cut_across_ctas(G, B):
     """Windows long enough for units to be cut across warps and CTAs (global records and their merges) with 16 state
