@@ -33,7 +33,8 @@
  *     advances its own bookkeeping per call.  A launch that is recorded once and replayed
  *     (a CUDA graph) would run again at the recorded position: issue every prefill and
  *     decode step through these calls.
- *   - Not thread-safe per context; different contexts are independent.
+ *   - Not thread-safe per context; different contexts are independent, also on the GPU: their launches may run on
+ *     different streams at the same time (no kernel of the library waits for a thread block that is not running).
  */
 #ifndef GLIDE_H_
 #define GLIDE_H_
