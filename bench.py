@@ -543,7 +543,7 @@ def run_glide(args, shape):
                           f"programmatic dependent launch; median of {n_reps} repetitions (>= {MIN_TIMED_S} s of timed "
                           f"work); the isolated-step latency is per_step_attention_latency_us"}),
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                         "traffic": NCU_TRAFFIC_BYTES.get(shape.name), "peak_kind": f"of {peak_kind}",
+                         "traffic": None if PHI["kind"] else NCU_TRAFFIC_BYTES.get(shape.name), "peak_kind": f"of {peak_kind}",
                          "kernel": decode_kernel_name(shape), "algorithmic_bytes_per_launch": b.bytes_stream,
                          "bytes_formula": "sum over layers and sequences of 2 w H_kv d 2B (window) + S,z read and written",
                          "algorithmic_bytes_incl_io": b.bytes_io,
