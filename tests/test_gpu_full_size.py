@@ -22,8 +22,16 @@ def _unit_inputs(wl, l, b, g, tokens, G):
             v[0, 0, :, g:g + 1].double().numpy())
 
 
-def _check(shape, units, extra_prefill=40, n_decode=3):
+def _check(shape, units, extra_prefill=40, n_decode=3, phi=0):
     dev = torch.device("cuda", 0)
+    bench.PHI["kind"] = phi   # (build_states creates the contexts with bench.glide_kwargs: the seeded projections)
+    try:
+        _check_body(shape, units, extra_prefill, n_decode, phi, dev)
+    finally:
+        bench.PHI["kind"] = 0
+
+
+def _check_body(shape, units, extra_prefill, n_decode, phi, dev):
     dt = bench.torch_dtype(shape)
     G = shape.n_q_heads // shape.n_kv_heads
     d, ctx_len = shape.head_dim, shape.context
@@ -32,7 +40,11 @@ def _check(shape, units, extra_prefill=40, n_decode=3):
     scale = f32_scale(d)
     cells = {}
     for (l, b, kv) in units:
-        cell = orc.Cell(G, 1, d, shape.windows[l], scale)
+        okw = {}
+        if phi:
+            kw = bench.glide_kwargs(shape, dev)
+            okw = dict(phi=phi, wq=to_np(kw["phi_wq"][l, kv * G:(kv + 1) * G]), wk=to_np(kw["phi_wk"][l, kv:kv + 1]))
+        cell = orc.Cell(G, 1, d, shape.windows[l], scale, **okw)
         piece = 16384
         for pos in range(0, ctx_len, piece):
             _, k, v = _unit_inputs(wl, l, b, kv, range(pos, min(pos + piece, ctx_len)), G)
@@ -94,6 +106,13 @@ def test_config1_shape_with_unit_scale_values():
     from dataclasses import replace
     shape = replace(C.C1, name="c1_unit_scale_values", value_scales=(4.0 / C.C1.head_dim ** 0.5, 1.0), seed=3)
     _check(shape, [(1, 0, 4), (7, 0, 0), (15, 0, 3), (28, 0, 6)])
+
+
+def test_config1_full_size_with_the_learned_feature_map():
+    """Config 1 with phi = GLIDE_PHI_PROJ_SOFTMAX2: state built by the tensor-core projection and carry kernels over the
+    32K prompt, a prefill call with outputs on the tcgen05 kernel's two-halves linear part, decode steps on the
+    streaming kernel with 16 state tiles per unit."""
+    _check(C.C1, [(0, 0, 0), (5, 0, 2), (12, 0, 1), (24, 0, 0), (31, 0, 7)], phi=1)
 
 
 def test_config4_mistral_b8_8k_full_size():
