@@ -197,3 +197,30 @@ def test_stream_schedule_refuses_what_the_kernel_does_not_run(glide):
     with pytest.raises(glide.GlideError) as e:
         glide.glide_stream_schedule(cfg)
     assert e.value.code == glide.GLIDE_ERR_UNSUPPORTED
+
+
+def test_stream_schedule_balances_the_warps_of_a_cta(glide):
+    """Config 1: inside every CTA the heaviest warp (in the schedule's own weights: 15 per state tile, 10 per window
+    tile, 27 per segment) is at most one window tile and one segment above the CTA's mean warp, and no unit is cut into
+    more records than the whole-stack problem needs (a unit of a 4096-token window is about 2.2 CTA shares)."""
+    import numpy as np
+    windows = [4096] * 4 + [1024] * 8 + [256] * 12 + [64] * 8
+    cfg, keep = glide.make_config(windows, 1, 32, 8, 128, 32768 + 64, dtype=torch.bfloat16)
+    rows = glide.glide_stream_schedule(cfg)
+    w = rows[:, 4] * 15 + rows[:, 6] * 10 + 27
+    warp = rows[:, 0] * 8 + rows[:, 1]
+    per_warp = np.bincount(warp, weights=w, minlength=148 * 8).reshape(148, 8)
+    assert (per_warp.max(axis=1) <= per_warp.sum(axis=1) / 8 + 10 + 27 + 15).all()
+    assert rows[:, 11].max() <= 5
+    assert per_warp.sum(axis=1).max() <= 1.1 * per_warp.sum(axis=1).mean()
+
+
+def test_stream_schedule_limits_the_records_of_a_small_problem(glide):
+    """One long-window layer at batch 1 leaves a CTA only a few dozen tiles: its units are then cut into at most about
+    eight records each (the merge reads them a few at a time); a problem with hundreds of tiles per CTA keeps all SMs."""
+    cfg, keep = glide.make_config([4096], 1, 32, 8, 128, 8192, dtype=torch.bfloat16)
+    rows = glide.glide_stream_schedule(cfg)
+    assert rows[:, 11].max() <= 10 and len(set(rows[:, 0].tolist())) <= 8 * 8 + 8
+    cfg, keep = glide.make_config([131072], 1, 32, 8, 128, 131072 + 64, dtype=torch.bfloat16)
+    rows = glide.glide_stream_schedule(cfg)
+    assert len(set(rows[:, 0].tolist())) == 148
